@@ -1,0 +1,279 @@
+"""Pins for oracle/tabed.py (CPU only): the round's structure against what the paper fixes."""
+import numpy as np
+import pytest
+
+from oracle import definitions as D
+from oracle import exact32 as X
+from oracle.drafter import OracleDrafter
+from oracle.tabed import TabedOracle
+from paper_2601_20357_b200 import workloads as W
+
+F = np.float32
+
+
+def lat(rng, shape):
+    return W.lattice_uniforms(rng, shape)
+
+
+def mk(m=3, B=2, gamma=3, h=2, policy=W.POLICY_SOFTMAX_INV_ERR, V=64, **kw):
+    return TabedOracle(n_inputs=m, n_requests=B, gamma=gamma, window_h=h, policy=policy, vocab=V, **kw)
+
+
+def rand_logits(rng, gamma, B, m, V, scale=1.0):
+    return (rng.standard_normal((gamma, B, m, V)) * scale).astype(F)
+
+
+def test_initial_weights_are_static_equal():
+    o = mk(m=4)
+    assert np.all(o.w == F(0.25))
+
+
+def test_single_input_round_equals_plain_speculative_decoding():
+    """m = 1: TABED reduces to single drafting.  Compare with a separately written SD round."""
+    rng = np.random.default_rng(0)
+    V, G = 50, 4
+    for trial in range(30):
+        o = mk(m=1, B=1, gamma=G, h=2, V=V)
+        lg = rand_logits(rng, G, 1, 1, V, 1.5)
+        tl = (rng.standard_normal((1, G + 1, V)) * 1.5).astype(F)
+        ud, ua, ur = lat(rng, (1, G)), lat(rng, (1, G)), lat(rng, (1,))
+        toks, q = o.draft_round_logits(lg, ud)
+        a, z = o.verify(tl, ua, ur)
+        w, am = o.update_weights()
+        # plain SD, Sec. 3 items 1-3
+        qs = [X.softmax_exact(lg[i, 0, 0]) for i in range(G)]
+        ps = [X.softmax_exact(tl[0, i]) for i in range(G + 1)]
+        ys = [X.draw(X.masses(qs[i]), ud[0, i]) for i in range(G)]
+        acc = 0
+        while acc < G and X.accept(ps[acc][ys[acc]], qs[acc][ys[acc]], ua[0, acc]):
+            acc += 1
+        if acc < G:
+            mr = X.residual_masses(ps[acc], qs[acc])
+            zz = X.draw(mr if mr.sum() > 0 else X.masses(ps[acc]), ur[0])
+        else:
+            zz = X.draw(X.masses(ps[G]), ur[0])
+        assert list(toks[0]) == ys and int(a[0]) == acc and int(z[0]) == zz
+        assert np.array_equal(q[0], np.stack(qs))
+        assert w.shape == (1, 1) and w[0, 0] == 1.0 and am[0] == 0
+
+
+def test_q_equals_p_accepts_every_token():
+    rng = np.random.default_rng(1)
+    G, V = 5, 200
+    for trial in range(20):
+        o = mk(m=1, B=2, gamma=G, V=V)
+        lg = rand_logits(rng, G, 2, 1, V, 2.0)
+        toks, _ = o.draft_round_logits(lg, lat(rng, (2, G)))
+        tl = np.concatenate([lg[:, :, 0, :].transpose(1, 0, 2), lg[-1:, :, 0, :].transpose(1, 0, 2)], axis=1)
+        a, z = o.verify(tl, lat(rng, (2, G)), lat(rng, (2,)))
+        assert np.all(a == G)
+
+
+def test_zero_target_probability_rejects_and_later_tokens_are_discarded():
+    rng = np.random.default_rng(2)
+    G, V = 4, 30
+    o = mk(m=2, B=1, gamma=G, V=V, policy=W.POLICY_GRID_MT)
+    lg = rand_logits(rng, G, 1, 2, V)
+    toks, q = o.draft_round_logits(lg, lat(rng, (1, G)))
+    tl = np.einsum("gbnv->bgv", lg)[:, :, :] / 2
+    tl = np.concatenate([tl, tl[:, -1:]], axis=1).astype(F)
+    tl[0, 1, toks[0, 1]] = -200.0                     # target gives the 2nd drafted token probability 0
+    tl[0, 0] = lg[0, 0].mean(0) + 50.0 * np.eye(V, dtype=F)[toks[0, 0]]   # and makes the 1st certain
+    a, z = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+    assert a[0] == 1 and z[0] != toks[0, 1]
+    # the replacement is drawn from the residual: it must have p > q there
+    assert o.p[0, 1, z[0]] > o.q[0, 1, z[0]]
+
+
+def test_greedy_mode():
+    rng = np.random.default_rng(3)
+    G, V = 3, 40
+    o = mk(m=2, B=1, gamma=G, V=V, policy=W.POLICY_STATIC, sample_mode=W.MODE_GREEDY)
+    lg = rand_logits(rng, G, 1, 2, V)
+    toks, q = o.draft_round_logits(lg, lat(rng, (1, G)))
+    assert list(toks[0]) == [int(np.argmax(q[0, i])) for i in range(G)]
+    tl = (rng.standard_normal((1, G + 1, V))).astype(F)
+    tl[0, 0, toks[0, 0]] = 30.0
+    a, z = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+    exp_a = 0
+    while exp_a < G and int(np.argmax(tl[0, exp_a])) == toks[0, exp_a]:
+        exp_a += 1
+    assert a[0] == exp_a >= 1 and z[0] == int(np.argmax(tl[0, a[0]]))
+
+
+def test_weights_sum_to_one_and_track_the_better_drafter():
+    """Sec. 4.1: methods with higher weights are closer to the target."""
+    rng = np.random.default_rng(4)
+    G, V, m = 3, 300, 3
+    o = mk(m=m, B=1, gamma=G, h=4, V=V)
+    for rnd in range(6):
+        lg = rand_logits(rng, G, 1, m, V, 1.0)
+        o.draft_round_logits(lg, lat(rng, (1, G)))
+        tl = np.concatenate([lg[:, :, 1, :], lg[-1:, :, 1, :]], axis=0).transpose(1, 0, 2)   # target = drafter 1
+        tl = (tl + 0.05 * rng.standard_normal(tl.shape)).astype(F)
+        o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+        w, am = o.update_weights()
+        assert np.all(w >= 0) and abs(float(w.astype(np.float64).sum()) - 1) < 1e-6
+        assert am[0] == 1 and w[0, 1] > w[0, 0] and w[0, 1] > w[0, 2]
+
+
+def test_grid_policy_matches_definition_and_endpoints():
+    rng = np.random.default_rng(5)
+    G, V = 3, 120
+    o = mk(m=2, B=1, gamma=G, h=0, V=V, policy=W.POLICY_GRID_MT)
+    ps, qks = [], []
+    for rnd in range(4):
+        lg = rand_logits(rng, G, 1, 2, V, 1.0)
+        o.draft_round_logits(lg, lat(rng, (1, G)))
+        mix = 0.7 * lg[:, :, 0, :] + 0.3 * lg[:, :, 1, :]
+        tl = np.concatenate([mix, mix[-1:]], axis=0).transpose(1, 0, 2)
+        tl = (tl + 0.3 * rng.standard_normal(tl.shape)).astype(F)
+        a, z = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+        for i in range(min(int(a[0]), G - 1) + 1):
+            ps.append(o.p[0, i].copy()); qks.append(o.qk[0, i].copy())
+        w, am = o.update_weights()
+        j_def, w_def, G_def = D.policy_grid(ps, qks)
+        np.testing.assert_allclose(o.window_error(0), G_def, atol=2e-5)
+        assert int(o.j_star[0]) == j_def
+        np.testing.assert_allclose(w[0], w_def, atol=1e-7)
+        e0 = sum(D.kl_divergence(p, qk[0]) for p, qk in zip(ps, qks))
+        e1 = sum(D.kl_divergence(p, qk[1]) for p, qk in zip(ps, qks))
+        we = o.window_error(0)
+        assert abs(we[0] - e0) < 2e-5 and abs(we[10] - e1) < 2e-5 and we.min() <= min(we[0], we[10])
+
+
+def test_window_h1_depends_only_on_last_verified_position():
+    """App. B: h = 1 uses only the ground truth of the previous decoding step."""
+    rng = np.random.default_rng(6)
+    G, V, m = 3, 80, 3
+    outs = []
+    last_lg = rand_logits(rng, G, 1, m, V)
+    last_tl = (rng.standard_normal((1, G + 1, V))).astype(F)
+    ud, ua, ur = lat(rng, (1, G)), lat(rng, (1, G)), lat(rng, (1,))
+    for history in range(2):
+        o = mk(m=m, B=1, gamma=G, h=1, V=V, policy=W.POLICY_STATIC)   # static: drafts do not depend on w
+        o.policy = W.POLICY_SOFTMAX_INV_ERR
+        o.n_dev = m
+        for _ in range(history * 3):
+            o.w[:] = X.policy_static(m)
+            o.draft_round_logits(rand_logits(rng, G, 1, m, V), lat(rng, (1, G)))
+            o.verify((rng.standard_normal((1, G + 1, V))).astype(F), lat(rng, (1, G)), lat(rng, (1,)))
+            o.update_weights()
+        o.w[:] = X.policy_static(m)
+        o.draft_round_logits(last_lg, ud)
+        a, _ = o.verify(last_tl, ua, ur)
+        w, _ = o.update_weights()
+        i_last = min(int(a[0]), G - 1)
+        e = [X.fixed_to_float(X.kl_fixed(o.p[0, i_last], o.qk[0, i_last, k])) for k in range(m)]
+        assert np.array_equal(w[0], X.policy_softmax_inv_err(np.array(e, F)))
+        outs.append(w.copy())
+    assert np.array_equal(outs[0], outs[1])
+
+
+def test_window_sum_equals_sum_of_last_h_positions_and_all_mode():
+    rng = np.random.default_rng(7)
+    G, V, m, h = 2, 60, 2, 3
+    o = mk(m=m, B=1, gamma=G, h=h, V=V)
+    o_all = mk(m=m, B=1, gamma=G, h=0, V=V)
+    hist = []
+    for rnd in range(5):
+        lg = rand_logits(rng, G, 1, m, V)
+        tl = (rng.standard_normal((1, G + 1, V))).astype(F)
+        ud, ua, ur = lat(rng, (1, G)), lat(rng, (1, G)), lat(rng, (1,))
+        for oo in (o, o_all):
+            oo.w[:] = X.policy_static(m)
+            oo.draft_round_logits(lg, ud)
+            a, _ = oo.verify(tl, ua, ur)
+        for i in range(min(int(a[0]), G - 1) + 1):
+            hist.append([D.kl_divergence(o.p[0, i], o.qk[0, i, k]) for k in range(m)])
+        o.update_weights(); o_all.update_weights()
+        np.testing.assert_allclose(o.window_error(0), np.sum(hist[-h:], axis=0), atol=1e-5)
+        np.testing.assert_allclose(o_all.window_error(0), np.sum(hist, axis=0), atol=1e-5)
+
+
+def test_positions_after_first_rejection_and_bonus_are_not_in_window():
+    rng = np.random.default_rng(8)
+    G, V, m = 4, 50, 2
+    for want_a in (0, 2, G):
+        o = mk(m=m, B=1, gamma=G, h=0, V=V)
+        lg = rand_logits(rng, G, 1, m, V)
+        toks, q = o.draft_round_logits(lg, lat(rng, (1, G)))
+        tl = np.zeros((1, G + 1, V), F)
+        for i in range(G):
+            tl[0, i] = 40.0 * np.eye(V, dtype=F)[toks[0, i]] if i < want_a else -60.0 * np.eye(V, dtype=F)[toks[0, i]]
+        a, z = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+        assert a[0] == want_a
+        o.update_weights()
+        assert o.count[0] == min(want_a, G - 1) + 1
+
+
+def test_drafter_bookkeeping_lengths_and_pending():
+    cfg = W.DrafterCfg(1, 32, 2, 2, 64, 40, "fp32")
+    wl = W.Workload(name="t", config_id=77, drafter=cfg, n_inputs=2, n_requests=1, gamma=3, window_h=2,
+                    rounds=1, policy=W.POLICY_STATIC)
+    dr = OracleDrafter(cfg, W.make_weights(wl))
+    rng = np.random.default_rng(9)
+    o = TabedOracle(n_inputs=2, n_requests=1, gamma=3, window_h=2, policy=W.POLICY_STATIC, vocab=40,
+                    drafter=dr, kv_capacity=64)
+    o.prefill(0, [W.Segment("tokens", np.arange(5, dtype=np.int32))])
+    o.prefill(1, [W.Segment("embeds", rng.standard_normal((2, 32)).astype(F))])
+    o.set_pending([7])
+    assert list(o.kv_lengths()) == [5, 2]
+    # round 1: force full acceptance -> two pending tokens, lengths advance by 1 + gamma - 1
+    toks, q = o.draft_round(lat(rng, (1, 3)))
+    assert list(o.kv_lengths()) == [5 + 3, 2 + 3]
+    tl = np.stack([40.0 * np.eye(40, dtype=F)[t] for t in list(toks[0]) + [11]])[None]
+    a, z = o.verify(tl, lat(rng, (1, 3)), lat(rng, (1,)))
+    assert a[0] == 3 and z[0] == 11
+    o.update_weights()
+    assert list(o.kv_lengths()) == [8, 5] and o.pending[0] == [int(toks[0, 2]), 11]
+    # round 2: reject at once -> catch-up consumed both pending tokens, drafts rolled back
+    toks2, _ = o.draft_round(lat(rng, (1, 3)))
+    assert list(o.kv_lengths()) == [8 + 2 + 2, 5 + 2 + 2]
+    tl = np.stack([-60.0 * np.eye(40, dtype=F)[t] for t in list(toks2[0]) + [0]])[None]
+    a, z = o.verify(tl, lat(rng, (1, 3)), lat(rng, (1,)))
+    assert a[0] == 0
+    o.update_weights()
+    assert list(o.kv_lengths()) == [10, 7] and o.pending[0] == [int(z[0])]
+    # the drafter saw the same continuation on both rows: logits of the two rows differ only by prefix
+    assert not np.array_equal(o.logits[0, 0, 0], o.logits[0, 0, 1])
+
+
+def test_identical_prefixes_make_ensemble_independent_of_weights():
+    cfg = W.DrafterCfg(1, 32, 2, 2, 64, 40, "fp32")
+    wl = W.Workload(name="t", config_id=78, drafter=cfg, n_inputs=2, n_requests=1, gamma=2, window_h=2,
+                    rounds=1, policy=W.POLICY_STATIC)
+    dr = OracleDrafter(cfg, W.make_weights(wl))
+    rng = np.random.default_rng(10)
+    ud = lat(rng, (1, 2))
+    res = []
+    for w in ([0.5, 0.5], [0.9, 0.1]):
+        o = TabedOracle(n_inputs=2, n_requests=1, gamma=2, window_h=2, policy=W.POLICY_STATIC, vocab=40,
+                        drafter=dr, kv_capacity=32)
+        for r in range(2):
+            o.prefill(r, [W.Segment("tokens", np.arange(6, dtype=np.int32))])
+        o.set_pending([3])
+        o.w[0] = np.asarray(w, F)
+        toks, q = o.draft_round(ud)
+        res.append((toks.copy(), q.copy()))
+    assert np.array_equal(res[0][0], res[1][0])
+    assert np.max(np.abs(res[0][1] - res[1][1])) < 1e-8
+
+
+def test_tiny_workload_free_run_smoke():
+    wl = W.TINY
+    dr = OracleDrafter(wl.drafter, W.make_weights(wl))
+    o = TabedOracle(n_inputs=2, n_requests=1, gamma=wl.gamma, window_h=wl.window_h, policy=wl.policy,
+                    vocab=wl.drafter.vocab, drafter=dr, kv_capacity=wl.kv_capacity)
+    for r, segs in enumerate(W.make_prefixes(wl)):
+        o.prefill(r, segs)
+    o.set_pending(W.initial_pending(wl))
+    acc = []
+    for rnd in range(4):
+        ud, ua, ur = W.round_uniforms(wl, rnd)
+        o.draft_round(ud)
+        a, z = o.verify(W.target_logits(wl, rnd, o.logits), ua, ur)
+        w, am = o.update_weights()
+        acc.append(int(a[0]))
+        assert abs(float(w.sum()) - 1) < 1e-6 and 0 <= a[0] <= wl.gamma and 0 <= z[0] < wl.drafter.vocab
+    assert o.count[0] == sum(min(a, wl.gamma - 1) + 1 for a in acc)
