@@ -1,0 +1,227 @@
+/*
+ * tabed.h - C boundary of the B200 TABED speculative-decoding library.
+ *
+ * One speculative-decoding round of Test-time Adaptive Batched Ensemble Drafting:
+ *   Algorithm 1 (batched shared-weight drafting of m inputs for gamma steps, weighted-average
+ *   ensemble and Sample at every step), the verification of Sec. 3 item 3 (accept with
+ *   probability min(1, p/q), resample the first rejected token from norm(max(0, p - q))), and
+ *   the test-time weight adaptation of Sec. 4.1 / App. B (deviation of each drafter from the
+ *   target over a window of h verified positions -> next block's ensemble weights).
+ *
+ * Conventions
+ *   - Every function returns TABED_OK (0) or a negative TABED_ERR_* code; nothing throws, aborts
+ *     or prints.  tabed_strerror() names a code.
+ *   - Unless a parameter says "host", array arguments are DEVICE pointers on config.device.
+ *     Work is enqueued on config.stream and the call returns without synchronising the host;
+ *     results are valid once the caller has synchronised that stream.  The *_host entry points
+ *     take HOST pointers, copy in, run, copy out and synchronise.
+ *   - The caller owns weights, inputs and outputs (weights must outlive the handle).  The library
+ *     owns KV caches, the window ring, the per-round q / q^(k) / p buffers and all scratch, all
+ *     allocated in tabed_init and released in tabed_destroy; no call in between allocates.
+ *   - Layouts are row-major with the last index fastest.  B = n_requests, m = n_inputs,
+ *     R = B*m rows (row = request*m + input), V = vocab, G = gamma.
+ *   - Uniforms are caller-supplied floats on the lattice u = (k + 1/2) * 2^-23, 0 <= k < 2^23.
+ *   - Per round the order is fixed: draft (tabed_draft_round or tabed_draft_round_logits) ->
+ *     tabed_verify -> tabed_update_weights; anything else returns TABED_ERR_BAD_STATE.
+ *   - Integer outputs (tokens, accept counts, weight argmax) are functions of the fp32 logits
+ *     evaluated with order-independent arithmetic: every floating-point step is one correctly
+ *     rounded binary32 operation and every vocabulary-wide sum is a sum of integers
+ *     (masses trunc(q_v * 2^40)), so they do not depend on grid shape or scheduling.
+ */
+#ifndef TABED_H
+#define TABED_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TABED_OK                0
+#define TABED_ERR_INVALID_ARG  -1
+#define TABED_ERR_NULL_PTR     -2
+#define TABED_ERR_BAD_STATE    -3
+#define TABED_ERR_KV_OVERFLOW  -4
+#define TABED_ERR_CUDA         -5
+#define TABED_ERR_TIMEOUT      -6
+#define TABED_ERR_UNSUPPORTED  -7
+
+#define TABED_DTYPE_FP32 0      /* fp32 weights and KV cache, no intermediate rounding          */
+#define TABED_DTYPE_BF16 1      /* bf16 weights and KV cache, fp32 accumulation, matmul inputs
+                                   rounded to bf16 (nearest even)                               */
+
+#define TABED_POLICY_STATIC          0   /* w_k = 1/m (the paper's Static baseline)              */
+#define TABED_POLICY_GRID_MT         1   /* m = 2: w^j = [1-j/10, j/10], j = 0..10, argmin error  */
+#define TABED_POLICY_SOFTMAX_INV_ERR 2   /* w = softmax(1/e^(1..m); tau)                          */
+
+#define TABED_DIST_KL   0       /* D = KL(p || q)        */
+#define TABED_DIST_TVD  1       /* D = 1/2 sum |p - q|   */
+
+#define TABED_MODE_SAMPLE 0     /* tokens drawn from q with the supplied uniforms */
+#define TABED_MODE_GREEDY 1     /* argmax decoding, lowest id on ties             */
+
+#define TABED_MAX_INPUTS 8
+
+/* tabed_debug_view selectors (device buffers owned by the handle) */
+#define TABED_VIEW_QK          0   /* float  [B][G][m][V]  per-drafter distributions of the round     */
+#define TABED_VIEW_Q           1   /* float  [B][G][V]     ensembled distributions of the round        */
+#define TABED_VIEW_P           2   /* float  [B][G+1][V]   target distributions (after tabed_verify)   */
+#define TABED_VIEW_LOGITS      3   /* float  [G][B][m][V]  drafter logits of the round's own forward   */
+#define TABED_VIEW_KV_LEN      4   /* int32  [R]           committed cache length of every row         */
+#define TABED_VIEW_WEIGHTS     5   /* float  [B][m]        current ensemble weights w*                 */
+#define TABED_VIEW_WINDOW_SUM  6   /* int64  [B][n_dev]    windowed deviation, fixed point 2^-40 (KL)
+                                                           or 2^-41 (TVD); n_dev = 11 (grid) or m     */
+#define TABED_VIEW_PENDING     7   /* int32  [B][3]        {count, token0, token1}                     */
+#define TABED_VIEW_GRID_J      8   /* int32  [B]           j* of the grid policy (-1 before any update)*/
+#define TABED_VIEW_ERROR_FLAG  9   /* int32  [1]           non-zero if a device-side check failed      */
+
+typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, d_ffn, vocab;
+  int32_t dtype;              /* TABED_DTYPE_* */
+  float   rms_eps;            /* e.g. 1e-5 */
+  float   rope_theta;         /* e.g. 10000 */
+  int32_t n_inputs;           /* m: drafting inputs per request, 1..TABED_MAX_INPUTS */
+  int32_t n_requests;         /* B >= 1 */
+  int32_t gamma;              /* block length, 1..16 */
+  int32_t window_h;           /* h; 0 = ALL (unbounded running sum) ; <= 64 */
+  int32_t policy;             /* TABED_POLICY_* */
+  int32_t distance;           /* TABED_DIST_* */
+  int32_t sample_mode;        /* TABED_MODE_* */
+  float   tau;                /* temperature of TABED_POLICY_SOFTMAX_INV_ERR, > 0 */
+  int32_t kv_capacity;        /* tokens per row */
+  int32_t device;             /* CUDA device ordinal */
+  void*   stream;             /* cudaStream_t, caller-owned; NULL = legacy default stream */
+} tabed_config;
+
+/* Device pointers to the drafter M_q, element type per config.dtype (float or bf16), every matrix
+ * [out][in] row-major; per-layer arrays are HOST arrays of n_layers device pointers.
+ * wq [d][d], wk/wv [Hkv*hd][d], wo [d][d], w_gate/w_up [F][d], w_down [d][F], norms [d],
+ * embed [V][d], lm_head [V][d] (untied), final_norm [d].  A NULL drafter (weights == NULL in
+ * tabed_init) gives a handle on which only the logits-driven calls are available. */
+typedef struct {
+  const void *embed, *lm_head, *final_norm;
+  const void *const *wq, *const *wk, *const *wv, *const *wo;
+  const void *const *w_gate, *const *w_up, *const *w_down;
+  const void *const *norm1, *const *norm2;
+} tabed_weights;
+
+/* Create a handle: validates the configuration, allocates every library-owned buffer, sets the
+ * ensemble weights to 1/m (no history yet) and leaves every row cache empty.
+ * Errors: NULL_PTR, INVALID_ARG (sizes out of range, head_dim not in {32,64,128}, d_model or
+ * d_ffn not a multiple of 8, grid policy with m != 2), UNSUPPORTED, CUDA (allocation failed). */
+int tabed_init(const tabed_config* cfg, const tabed_weights* weights, tabed_handle** out);
+
+/* Release everything tabed_init allocated.  NULL is accepted. */
+void tabed_destroy(tabed_handle* h);
+
+const char* tabed_strerror(int code);
+
+/* Load a synthetic cache into one row: k, v are [L][Hkv][len][hd] in the drafter's dtype;
+ * sets the row's committed length to len.  Errors: INVALID_ARG (row / len out of range). */
+int tabed_load_prefix_kv(tabed_handle* h, int32_t row, const void* k, const void* v, int32_t len);
+
+/* Consume a prompt prefix into one row's cache by running the drafter over it position by
+ * position (Algorithm 1's prefix x^(k)).  tokens: int32 [len]; embeds: float [len][d] (projected
+ * image tokens enter as embeddings).  Appends at the row's committed length.
+ * Errors: INVALID_ARG, KV_OVERFLOW, BAD_STATE (handle without drafter). */
+int tabed_prefill_tokens(tabed_handle* h, int32_t row, const int32_t* tokens, int32_t len);
+int tabed_prefill_embeds(tabed_handle* h, int32_t row, const float* embeds, int32_t len);
+
+/* Set the verified-but-not-yet-consumed token(s) of every request: tok int32 [B][2],
+ * cnt int32 [B] with values 1 or 2.  Normally only needed once, before the first round. */
+int tabed_set_pending(tabed_handle* h, const int32_t* tok, const int32_t* cnt);
+
+/* One batched shared-weight decoder step outside a round (Algorithm 1 step 5 alone): feeds
+ * tok[b] to all m rows of request b at each row's own position, appends K,V, advances the
+ * committed lengths by one, and writes logits float [B][m][V] unless out_logits is NULL (then
+ * the LM head is skipped).  Errors: KV_OVERFLOW, BAD_STATE (mid-round or no drafter). */
+int tabed_decode_step(tabed_handle* h, const int32_t* tok, float* out_logits);
+
+/* Algorithm 1 steps 6-7 on caller-supplied logits float [B][m][V]: q^(k) = softmax(logits^(k)),
+ * q = sum_k w_k q^(k), y = Sample(q; u) (or argmax in greedy mode).  w float [B][m] may be NULL
+ * (use the handle's current w*).  u float [B].  Outputs: y int32 [B]; q float [B][V] and
+ * qk float [B][m][V] may each be NULL.  Stateless with respect to the round. */
+int tabed_ensemble_step(tabed_handle* h, const float* logits, const float* w, const float* u,
+                        int32_t* y, float* q, float* qk);
+
+/* Algorithm 1: gamma batched drafting steps with the handle's w*, feeding the pending token(s)
+ * first (two pending tokens are consumed in the same weight pass).  u_draft float [B][G].
+ * Outputs: out_tokens int32 [B][G]; out_q float [B][G][V] may be NULL (the library keeps its own
+ * copy either way).  The rows' caches receive the pending and the first G-1 drafted tokens; the
+ * committed lengths do not move until tabed_update_weights.
+ * Errors: BAD_STATE, KV_OVERFLOW (conservative host-side bound), NULL_PTR. */
+int tabed_draft_round(tabed_handle* h, const float* u_draft, int32_t* out_tokens, float* out_q);
+
+/* The same round on caller-supplied drafter logits float [G][B][m][V] (for callers that run M_q
+ * themselves): no forward pass, caches untouched. */
+int tabed_draft_round_logits(tabed_handle* h, const float* drafter_logits, const float* u_draft,
+                             int32_t* out_tokens, float* out_q);
+
+/* Sec. 3 item 3 on the round just drafted.  target_logits float [B][G+1][V] (position G is the
+ * bonus position), u_accept float [B][G], u_resid float [B].  p_i = softmax(target_logits_i);
+ * token i is accepted iff p_i(y_i) >= q_i(y_i) or u_i * q_i(y_i) < p_i(y_i), stopping at the first
+ * rejection; n_accept = a.  next_token: a < G -> drawn from norm(max(0, p_a - q_a)) (from p_a if
+ * that residual has no mass); a == G -> drawn from p_G.  Greedy mode: accept iff
+ * argmax p_i == y_i, next_token = argmax p_a.  Outputs int32 [B] each. */
+int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_accept,
+                 const float* u_resid, int32_t* out_n_accept, int32_t* out_next_token);
+
+/* Sec. 4.1 / App. B on the round just verified: for every verified position i <= min(a, G-1)
+ * computes the deviation D(p_i, q_i^(k)) of each drafter (or of each of the 11 grid candidates),
+ * pushes it into the request's window of the last h positions, evaluates the policy on the
+ * window sums to get the next block's w* (Algorithm 1 steps 2-3), then commits the caches:
+ * length += pending + (a < G ? a : G-1), pending <- {next_token} or {y_{G-1}, next_token}.
+ * Outputs: out_w float [B][m], out_w_argmax int32 [B] (lowest index on ties); either may be NULL. */
+int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax);
+
+/* Host-buffer round: tabed_draft_round -> tabed_verify -> tabed_update_weights with HOST pointers
+ * (pageable or pinned) for every argument, same shapes as above.  Copies the inputs to the
+ * device, runs the round, copies the results back and synchronises the stream before returning.
+ * out_w and out_w_argmax may be NULL. */
+int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accept,
+                     const float* u_resid, const float* target_logits, int32_t* out_tokens,
+                     int32_t* out_n_accept, int32_t* out_next_token, float* out_w,
+                     int32_t* out_w_argmax);
+
+/* Pointer and size of a library-owned device buffer (TABED_VIEW_*).  Read-only for the caller. */
+int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* bytes);
+
+/* Replay aid: while set (non-NULL), tabed_draft_round still runs its own forward pass (caches and
+ * TABED_VIEW_LOGITS are written as usual) but steps 6-7 of Algorithm 1 read these logits
+ * float [G][B][m][V] instead, so that a recorded trajectory can be followed exactly while the
+ * forward pass is compared against it.  The buffer must stay valid until cleared with NULL. */
+int tabed_debug_override_logits(tabed_handle* h, const float* drafter_logits);
+
+/* Small host-side snapshot of the adaptive state (weights, window ring, pending tokens, committed
+ * lengths); cache contents stay on the device.  Call with host == NULL to get the size in *bytes.
+ * Both calls synchronise the stream. */
+int tabed_state_export(tabed_handle* h, void* host, size_t* bytes);
+int tabed_state_import(tabed_handle* h, const void* host, size_t bytes);
+
+/* Device timing of one kernel class: between tabed_profile_begin and tabed_profile_end the library
+ * records a CUDA event pair on config.stream around every launch (group) of that class;
+ * tabed_profile_end synchronises the stream and returns the summed elapsed milliseconds and the
+ * number of timed intervals.  TABED_PROF_ATTENTION, _ENSEMBLE, _VERIFY and _UPDATE time their group
+ * of kernels as one interval; the others time a single kernel per interval. */
+#define TABED_PROF_QKV        0
+#define TABED_PROF_ATTENTION  1
+#define TABED_PROF_OPROJ      2
+#define TABED_PROF_GATEUP     3
+#define TABED_PROF_DOWN       4
+#define TABED_PROF_LM_HEAD    5
+#define TABED_PROF_ENSEMBLE   6
+#define TABED_PROF_VERIFY     7
+#define TABED_PROF_UPDATE     8
+int tabed_profile_begin(tabed_handle* h, int32_t kernel_class);
+int tabed_profile_end(tabed_handle* h, double* total_ms, int64_t* n_intervals);
+
+/* Number of kernels the library has launched on this handle since tabed_init (host counter). */
+int64_t tabed_launch_count(const tabed_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TABED_H */

@@ -1,0 +1,737 @@
+// C boundary of the TABED round: handle, state, launch sequences.  See include/tabed.h for the
+// contract of every entry point; the kernels live in forward_kernels.cuh / decide_kernels.cuh.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <type_traits>
+#include <vector>
+
+#include "../../include/tabed.h"
+#include "exact_math.cuh"
+#include "forward_kernels.cuh"
+#include "decide_kernels.cuh"
+
+using namespace tabed;
+
+namespace {
+
+enum Phase { PH_IDLE = 0, PH_DRAFTED = 1, PH_VERIFIED = 2 };
+
+struct DeviceGuard {
+  int prev = -1; bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+struct tabed_handle {
+  tabed_config cfg;
+  bool has_drafter = false;
+  cudaStream_t stream = nullptr;
+  int R = 0, B = 0, m = 0, G = 0, V = 0, d = 0, F = 0, H = 0, Hkv = 0, hd = 0, L = 0, cap = 0;
+  int n_dev = 0, n_chunks = 0, ns = 1, max_splits = 0, qkv_w = 0;
+  size_t esz = 4;
+  // drafter (caller-owned device memory)
+  const void *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  std::vector<const void*> wq, wk, wv, wo, w_gate, w_up, w_down, norm1, norm2;
+  // library-owned device memory
+  std::vector<void*> allocs;
+  void *kc = nullptr, *vc = nullptr;
+  float *rope_cos = nullptr, *rope_sin = nullptr;
+  int *kv_len = nullptr, *pending = nullptr;
+  float *w = nullptr;
+  long long *dev = nullptr, *ring = nullptr, *running = nullptr, *pushed = nullptr;
+  int *ring_head = nullptr, *ring_count = nullptr, *grid_j = nullptr;
+  SlotDesc* slots = nullptr; int* last_slot = nullptr;
+  float *x = nullptr, *qkv = nullptr, *attn_out = nullptr, *mid = nullptr, *part_o = nullptr, *part_ml = nullptr;
+  float *logits_own = nullptr, *qk = nullptr, *q = nullptr, *p = nullptr, *scratch_q = nullptr;
+  int *tokens = nullptr, *n_accept = nullptr, *next_token = nullptr, *w_argmax = nullptr;
+  uint32_t* rowmax = nullptr; unsigned long long* rowsum = nullptr;
+  unsigned long long* chunk_mass = nullptr; ChunkBest* chunk_best = nullptr;
+  int* err = nullptr;
+  // staging for the host-buffer entry point
+  float *st_u_draft = nullptr, *st_u_accept = nullptr, *st_u_resid = nullptr, *st_target = nullptr;
+  int* st_tokens = nullptr;
+  // host-side state
+  int phase = PH_IDLE;
+  bool round_has_forward = false;
+  const float* logits_override = nullptr;   // tabed_debug_override_logits
+  std::vector<int> len_ub;          // upper bound of every row's committed length
+  int64_t launches = 0;
+  // per-kernel-class timing (tabed_profile_begin / tabed_profile_end)
+  int prof_class = -1;
+  std::vector<cudaEvent_t> prof_events;     // start/stop pairs
+  size_t prof_used = 0;
+};
+
+namespace {
+
+// Records a start/stop event pair on the handle's stream around the launches of one kernel class.
+struct ProfScope {
+  tabed_handle* h; bool on;
+  ProfScope(tabed_handle* hh, int cls) : h(hh), on(hh->prof_class == cls) { if (on) rec(); }
+  ~ProfScope() { if (on) rec(); }
+  void rec() {
+    if (h->prof_used == h->prof_events.size()) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+      h->prof_events.push_back(e);
+    }
+    cudaEventRecord(h->prof_events[h->prof_used++], h->stream);
+  }
+};
+
+#define TABED_LAUNCH(h, kern, grid, block, smem, ...)                 \
+  do {                                                                \
+    kern<<<(grid), (block), (smem), (h)->stream>>>(__VA_ARGS__);      \
+    (h)->launches++;                                                  \
+  } while (0)
+
+template <typename T>
+int dev_alloc(tabed_handle* h, T** out, size_t count, bool zero = true) {
+  void* ptr = nullptr;
+  const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+  if (cudaMalloc(&ptr, bytes) != cudaSuccess) { cudaGetLastError(); return TABED_ERR_CUDA; }
+  h->allocs.push_back(ptr);
+  if (zero && cudaMemsetAsync(ptr, 0, bytes, h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+  *out = reinterpret_cast<T*>(ptr);
+  return TABED_OK;
+}
+
+int pick_ns(int n) {            // accumulator columns per weight pass
+  const int opts[] = {1, 2, 3, 4, 6, 8};
+  for (int o : opts) if (o >= std::min(n, 8)) return o;
+  return 8;
+}
+
+// ---- projection dispatch ---------------------------------------------------------------------
+template <typename T, int NS, int RPW, int EPI>
+void launch_gemv_inst(tabed_handle* h, const GemvArgs& a, int n_chunks) {
+  constexpr bool ROUND_IN = !std::is_same<T, float>::value;
+  auto kern = k_gemv<T, NS, RPW, EPI, ROUND_IN>;
+  const size_t smem = (size_t)NS * a.K * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    attr_set = true;
+  }
+  const int n_out = (EPI == EPI_SWIGLU) ? a.rows0 : (a.rows0 + a.rows1 + a.rows2);
+  const int n_groups = (n_out + RPW - 1) / RPW;
+  const int ctas = std::max(1, std::min((n_groups + kGemvWarps - 1) / kGemvWarps, 148 * 8));
+  TABED_LAUNCH(h, kern, dim3(ctas, n_chunks), kGemvThreads, smem, a);
+}
+
+template <typename T, int NS, int EPI>
+void launch_gemv_rpw(tabed_handle* h, const GemvArgs& a, int n_chunks) {
+  const int n_out = (EPI == EPI_SWIGLU) ? a.rows0 : (a.rows0 + a.rows1 + a.rows2);
+  const int per_row = (EPI == EPI_SWIGLU) ? 2 : 1;
+  const int warps_full = 148 * kGemvWarps * 2;
+  if constexpr (NS <= 4 && EPI != EPI_SWIGLU) {
+    if (n_out >= warps_full * 4) { launch_gemv_inst<T, NS, 4, EPI>(h, a, n_chunks); return; }
+  }
+  if constexpr (NS <= 4 || EPI != EPI_SWIGLU) {
+    if (n_out >= warps_full * 2) { launch_gemv_inst<T, NS, 2, EPI>(h, a, n_chunks); return; }
+  }
+  (void)per_row;
+  launch_gemv_inst<T, NS, 1, EPI>(h, a, n_chunks);
+}
+
+template <typename T, int EPI>
+void launch_gemv_ns(tabed_handle* h, const GemvArgs& a, int ns) {
+  const int n_chunks = (a.n_slots + ns - 1) / ns;
+  switch (ns) {
+    case 1: launch_gemv_rpw<T, 1, EPI>(h, a, n_chunks); break;
+    case 2: launch_gemv_rpw<T, 2, EPI>(h, a, n_chunks); break;
+    case 3: launch_gemv_rpw<T, 3, EPI>(h, a, n_chunks); break;
+    case 4: launch_gemv_rpw<T, 4, EPI>(h, a, n_chunks); break;
+    case 6: launch_gemv_rpw<T, 6, EPI>(h, a, n_chunks); break;
+    default: launch_gemv_rpw<T, 8, EPI>(h, a, n_chunks); break;
+  }
+}
+
+void launch_gemv(tabed_handle* h, const GemvArgs& a, int epi, int ns) {
+  const bool f32 = h->cfg.dtype == TABED_DTYPE_FP32;
+  if (epi == EPI_STORE) { if (f32) launch_gemv_ns<float, EPI_STORE>(h, a, ns); else launch_gemv_ns<__nv_bfloat16, EPI_STORE>(h, a, ns); }
+  else if (epi == EPI_RESID) { if (f32) launch_gemv_ns<float, EPI_RESID>(h, a, ns); else launch_gemv_ns<__nv_bfloat16, EPI_RESID>(h, a, ns); }
+  else { if (f32) launch_gemv_ns<float, EPI_SWIGLU>(h, a, ns); else launch_gemv_ns<__nv_bfloat16, EPI_SWIGLU>(h, a, ns); }
+}
+
+template <typename T, int HD>
+void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
+  const int split_len = (max_pos > 2048) ? 256 : 128;
+  const int splits = std::max(1, (max_pos + split_len - 1) / split_len);
+  const float scale = 1.0f / sqrtf((float)h->hd);
+  auto part = k_attn_partial<T, HD>;
+  auto merge = k_attn_merge<HD>;
+  TABED_LAUNCH(h, part, dim3(splits, h->Hkv, n_slots), kAttnThreads, 0, h->qkv, h->slots, h->H, h->Hkv,
+               reinterpret_cast<const T*>(h->kc), reinterpret_cast<const T*>(h->vc), layer, h->L, h->cap, split_len,
+               h->part_o, h->part_ml, h->max_splits, scale);
+  TABED_LAUNCH(h, merge, dim3(h->H, n_slots), HD, 0, h->slots, h->H, split_len, h->part_o, h->part_ml,
+               h->max_splits, h->attn_out);
+}
+
+template <typename T>
+void launch_attention_t(tabed_handle* h, int layer, int n_slots, int max_pos) {
+  switch (h->hd) {
+    case 32: launch_attention_hd<T, 32>(h, layer, n_slots, max_pos); break;
+    case 64: launch_attention_hd<T, 64>(h, layer, n_slots, max_pos); break;
+    default: launch_attention_hd<T, 128>(h, layer, n_slots, max_pos); break;
+  }
+}
+
+// One shared-weight decoder step over `n_slots` slots.  max_pos: host upper bound of (position+1).
+void run_step(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* logits_out) {
+  const bool f32 = h->cfg.dtype == TABED_DTYPE_FP32;
+  sa.R = h->R; sa.m = h->m; sa.d = h->d; sa.G = h->G;
+  sa.kv_len = h->kv_len; sa.pending = h->pending;
+  sa.slots = h->slots; sa.last_slot = h->last_slot; sa.x = h->x; sa.err = h->err; sa.kv_capacity = h->cap;
+  if (f32) TABED_LAUNCH(h, k_begin_step<float>, n_slots, 128, 0, sa, reinterpret_cast<const float*>(h->embed));
+  else TABED_LAUNCH(h, k_begin_step<__nv_bfloat16>, n_slots, 128, 0, sa, reinterpret_cast<const __nv_bfloat16*>(h->embed));
+  const int ns = (sa.mode == STEP_PREFILL) ? 1 : h->ns;
+  const int kvd = h->Hkv * h->hd;
+  for (int l = 0; l < h->L; ++l) {
+    GemvArgs a{};
+    a.W0 = h->wq[l]; a.W1 = h->wk[l]; a.W2 = h->wv[l]; a.rows0 = h->d; a.rows1 = kvd; a.rows2 = kvd;
+    a.K = h->d; a.in = h->x; a.in_stride = h->d; a.gain = h->norm1[l]; a.eps = h->cfg.rms_eps;
+    a.out = h->qkv; a.out_stride = h->qkv_w; a.slots = h->slots; a.n_slots = n_slots;
+    { ProfScope ps(h, TABED_PROF_QKV); launch_gemv(h, a, EPI_STORE, ns); }
+    ProfScope* pa = new ProfScope(h, TABED_PROF_ATTENTION);
+    if (f32) {
+      TABED_LAUNCH(h, k_rope_append<float>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos,
+                   h->rope_sin, reinterpret_cast<float*>(h->kc), reinterpret_cast<float*>(h->vc), l, h->L, h->cap);
+      launch_attention_t<float>(h, l, n_slots, max_pos);
+    } else {
+      TABED_LAUNCH(h, k_rope_append<__nv_bfloat16>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd,
+                   h->rope_cos, h->rope_sin, reinterpret_cast<__nv_bfloat16*>(h->kc),
+                   reinterpret_cast<__nv_bfloat16*>(h->vc), l, h->L, h->cap);
+      launch_attention_t<__nv_bfloat16>(h, l, n_slots, max_pos);
+    }
+    delete pa;
+    GemvArgs o{};
+    o.W0 = h->wo[l]; o.rows0 = h->d; o.K = h->H * h->hd; o.in = h->attn_out; o.in_stride = h->H * h->hd;
+    o.out = h->x; o.out_stride = h->d; o.slots = h->slots; o.n_slots = n_slots;
+    { ProfScope ps(h, TABED_PROF_OPROJ); launch_gemv(h, o, EPI_RESID, ns); }
+    GemvArgs gu{};
+    gu.W0 = h->w_gate[l]; gu.W1 = h->w_up[l]; gu.rows0 = h->F; gu.rows1 = h->F; gu.K = h->d;
+    gu.in = h->x; gu.in_stride = h->d; gu.gain = h->norm2[l]; gu.eps = h->cfg.rms_eps;
+    gu.out = h->mid; gu.out_stride = h->F; gu.slots = h->slots; gu.n_slots = n_slots;
+    { ProfScope ps(h, TABED_PROF_GATEUP); launch_gemv(h, gu, EPI_SWIGLU, ns); }
+    GemvArgs dn{};
+    dn.W0 = h->w_down[l]; dn.rows0 = h->d; dn.K = h->F; dn.in = h->mid; dn.in_stride = h->F;
+    dn.out = h->x; dn.out_stride = h->d; dn.slots = h->slots; dn.n_slots = n_slots;
+    { ProfScope ps(h, TABED_PROF_DOWN); launch_gemv(h, dn, EPI_RESID, ns); }
+  }
+  if (logits_out) {
+    GemvArgs hd{};
+    hd.W0 = h->lm_head; hd.rows0 = h->V; hd.K = h->d; hd.in = h->x; hd.in_stride = h->d;
+    hd.src_slot = h->last_slot; hd.gain = h->final_norm; hd.eps = h->cfg.rms_eps;
+    hd.out = logits_out; hd.out_stride = h->V; hd.slots = nullptr; hd.n_slots = h->R;
+    ProfScope ps(h, TABED_PROF_LM_HEAD);
+    launch_gemv(h, hd, EPI_STORE, h->ns);
+  }
+}
+
+// Algorithm 1 steps 6-7 for all requests on logits [B][m][V].
+void run_ensemble(tabed_handle* h, const float* logits, const float* w, const float* u, int u_stride,
+                  int* y0, int y0_stride, int* y1, int y1_stride, float* qk_out, long long qk_stride,
+                  float* q_out, long long q_stride) {
+  const int greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
+  ProfScope ps(h, TABED_PROF_ENSEMBLE);
+  cudaMemsetAsync(h->rowmax, 0, sizeof(uint32_t) * h->R, h->stream);
+  cudaMemsetAsync(h->rowsum, 0, sizeof(unsigned long long) * h->R, h->stream);
+  const dim3 grid_rows(h->n_chunks, h->R), grid_req(h->n_chunks, h->B);
+  TABED_LAUNCH(h, k_rowmax, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax);
+  TABED_LAUNCH(h, k_expsum, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
+  TABED_LAUNCH(h, k_mix, grid_req, kDecThreads, 0, logits, h->V, h->m, w, h->rowmax, h->rowsum, qk_out, qk_stride,
+               q_out, q_stride, h->chunk_mass, h->chunk_best, h->n_chunks, greedy);
+  SelectArgs s{};
+  s.V = h->V; s.n_chunks = h->n_chunks; s.G = h->G; s.greedy = greedy;
+  s.q = q_out; s.q_req_stride = q_stride; s.u = u; s.u_stride = u_stride;
+  s.chunk_mass = h->chunk_mass; s.chunk_best = h->chunk_best;
+  s.out0 = y0; s.out0_stride = y0_stride; s.out1 = y1; s.out1_stride = y1_stride; s.err = h->err;
+  TABED_LAUNCH(h, k_select<0>, h->B, kDecThreads, 0, s);
+}
+
+int check_cuda() { return cudaGetLastError() == cudaSuccess ? TABED_OK : TABED_ERR_CUDA; }
+
+int max_len_ub(const tabed_handle* h) {
+  int mx = 0;
+  for (int v : h->len_ub) mx = std::max(mx, v);
+  return mx;
+}
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+const char* tabed_strerror(int code) {
+  switch (code) {
+    case TABED_OK: return "ok";
+    case TABED_ERR_INVALID_ARG: return "invalid argument";
+    case TABED_ERR_NULL_PTR: return "null pointer";
+    case TABED_ERR_BAD_STATE: return "call out of order for the handle's state";
+    case TABED_ERR_KV_OVERFLOW: return "row cache capacity would be exceeded";
+    case TABED_ERR_CUDA: return "CUDA runtime error";
+    case TABED_ERR_TIMEOUT: return "device-side wait ran out";
+    case TABED_ERR_UNSUPPORTED: return "unsupported configuration";
+    default: return "unknown error code";
+  }
+}
+
+int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle** out) {
+  if (!cfg || !out) return TABED_ERR_NULL_PTR;
+  *out = nullptr;
+  const tabed_config& c = *cfg;
+  if (c.vocab < 2 || c.n_inputs < 1 || c.n_inputs > TABED_MAX_INPUTS || c.n_requests < 1 || c.gamma < 1 ||
+      c.gamma > 16 || c.window_h < 0 || c.window_h > 64 || c.policy < 0 || c.policy > 2 || c.distance < 0 ||
+      c.distance > 1 || c.sample_mode < 0 || c.sample_mode > 1 || !(c.tau > 0.0f) || c.device < 0)
+    return TABED_ERR_INVALID_ARG;
+  if (c.policy == TABED_POLICY_GRID_MT && c.n_inputs != 2) return TABED_ERR_INVALID_ARG;
+  if ((long long)c.n_requests * c.n_inputs > 4096) return TABED_ERR_UNSUPPORTED;
+  if (wts) {
+    if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 8 || c.kv_capacity < 1 ||
+        c.dtype < 0 || c.dtype > 1 || !(c.rms_eps > 0.0f) || !(c.rope_theta > 0.0f))
+      return TABED_ERR_INVALID_ARG;
+    if (c.d_model % c.n_heads || c.n_heads % c.n_kv_heads || c.d_model % 8 || c.d_ffn % 8) return TABED_ERR_INVALID_ARG;
+    const int hd = c.d_model / c.n_heads;
+    if (hd != 32 && hd != 64 && hd != 128) return TABED_ERR_INVALID_ARG;
+    if (!wts->embed || !wts->lm_head || !wts->final_norm || !wts->wq || !wts->wk || !wts->wv || !wts->wo ||
+        !wts->w_gate || !wts->w_up || !wts->w_down || !wts->norm1 || !wts->norm2)
+      return TABED_ERR_NULL_PTR;
+    for (int l = 0; l < c.n_layers; ++l)
+      if (!wts->wq[l] || !wts->wk[l] || !wts->wv[l] || !wts->wo[l] || !wts->w_gate[l] || !wts->w_up[l] ||
+          !wts->w_down[l] || !wts->norm1[l] || !wts->norm2[l])
+        return TABED_ERR_NULL_PTR;
+  }
+  int n_devices = 0;
+  if (cudaGetDeviceCount(&n_devices) != cudaSuccess || c.device >= n_devices) { cudaGetLastError(); return TABED_ERR_CUDA; }
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return TABED_ERR_CUDA;
+
+  tabed_handle* h = new (std::nothrow) tabed_handle();
+  if (!h) return TABED_ERR_CUDA;
+  h->cfg = c; h->stream = reinterpret_cast<cudaStream_t>(c.stream);
+  h->B = c.n_requests; h->m = c.n_inputs; h->R = h->B * h->m; h->G = c.gamma; h->V = c.vocab;
+  h->n_dev = (c.policy == TABED_POLICY_GRID_MT) ? kGridCand : h->m;
+  h->n_chunks = (h->V + kChunk - 1) / kChunk;
+  h->ns = pick_ns(h->R);
+  h->has_drafter = wts != nullptr;
+  int rc = TABED_OK;
+  auto A = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count); };
+  const size_t B = h->B, m = h->m, R = h->R, G = h->G, V = h->V;
+  A(&h->w, B * m); A(&h->pending, B * 3);
+  A(&h->dev, B * G * kMaxDev); A(&h->ring, B * std::max(1, c.window_h) * kMaxDev); A(&h->running, B * kMaxDev);
+  A(&h->pushed, B); A(&h->ring_head, B); A(&h->ring_count, B); A(&h->grid_j, B);
+  A(&h->qk, B * G * m * V); A(&h->q, B * G * V); A(&h->p, B * (G + 1) * V); A(&h->scratch_q, B * V);
+  A(&h->tokens, B * G); A(&h->n_accept, B); A(&h->next_token, B); A(&h->w_argmax, B);
+  const size_t max_rows = std::max(R, B * (G + 1));
+  A(&h->rowmax, max_rows); A(&h->rowsum, max_rows);
+  A(&h->chunk_mass, B * h->n_chunks); A(&h->chunk_best, B * (G + 1) * h->n_chunks);
+  A(&h->err, 1);
+  A(&h->st_u_draft, B * G); A(&h->st_u_accept, B * G); A(&h->st_u_resid, B); A(&h->st_target, B * (G + 1) * V); A(&h->st_tokens, B * G);
+  if (h->has_drafter) {
+    h->L = c.n_layers; h->d = c.d_model; h->F = c.d_ffn; h->H = c.n_heads; h->Hkv = c.n_kv_heads;
+    h->hd = c.d_model / c.n_heads; h->cap = c.kv_capacity; h->esz = c.dtype == TABED_DTYPE_FP32 ? 4 : 2;
+    h->qkv_w = (h->H + 2 * h->Hkv) * h->hd;
+    while (h->ns > 1 && (size_t)h->ns * std::max(h->d, h->F) * sizeof(float) > 200u * 1024u) {
+      const int opts[] = {1, 2, 3, 4, 6, 8};
+      int lower = 1;
+      for (int o : opts) if (o < h->ns) lower = o;
+      h->ns = lower;
+    }
+    h->max_splits = (h->cap + 127) / 128;
+    h->embed = wts->embed; h->lm_head = wts->lm_head; h->final_norm = wts->final_norm;
+    for (int l = 0; l < h->L; ++l) {
+      h->wq.push_back(wts->wq[l]); h->wk.push_back(wts->wk[l]); h->wv.push_back(wts->wv[l]); h->wo.push_back(wts->wo[l]);
+      h->w_gate.push_back(wts->w_gate[l]); h->w_up.push_back(wts->w_up[l]); h->w_down.push_back(wts->w_down[l]);
+      h->norm1.push_back(wts->norm1[l]); h->norm2.push_back(wts->norm2[l]);
+    }
+    const size_t kv_elems = R * h->L * h->Hkv * (size_t)h->cap * h->hd;
+    unsigned char *kcb = nullptr, *vcb = nullptr;
+    A(&kcb, kv_elems * h->esz); A(&vcb, kv_elems * h->esz);
+    h->kc = kcb; h->vc = vcb;
+    A(&h->kv_len, R); A(&h->slots, 2 * R); A(&h->last_slot, R);
+    A(&h->x, 2 * R * h->d); A(&h->qkv, 2 * R * h->qkv_w); A(&h->attn_out, 2 * R * h->H * h->hd); A(&h->mid, 2 * R * h->F);
+    A(&h->part_o, 2 * R * h->H * (size_t)h->max_splits * h->hd); A(&h->part_ml, 2 * R * h->H * (size_t)h->max_splits * 2);
+    A(&h->logits_own, G * R * V);
+    A(&h->rope_cos, (size_t)h->cap * (h->hd / 2)); A(&h->rope_sin, (size_t)h->cap * (h->hd / 2));
+    if (rc == TABED_OK) {
+      const int half = h->hd / 2;
+      std::vector<float> hc((size_t)h->cap * half), hs((size_t)h->cap * half);
+      for (int i = 0; i < half; ++i) {
+        const double inv = pow((double)c.rope_theta, -2.0 * i / h->hd);
+        for (int pos = 0; pos < h->cap; ++pos) {
+          const double ang = pos * inv;
+          hc[(size_t)pos * half + i] = (float)cos(ang);
+          hs[(size_t)pos * half + i] = (float)sin(ang);
+        }
+      }
+      if (cudaMemcpyAsync(h->rope_cos, hc.data(), hc.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+          cudaMemcpyAsync(h->rope_sin, hs.data(), hs.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+          cudaStreamSynchronize(h->stream) != cudaSuccess)
+        rc = TABED_ERR_CUDA;
+    }
+    h->len_ub.assign(R, 0);
+  }
+  if (rc == TABED_OK) {
+    // equal weights before any history; one pending slot per request; grid j* undefined
+    std::vector<float> w0(B * m, 1.0f / (float)m);
+    std::vector<int> pend(B * 3, 0), gj(B, -1);
+    for (size_t b = 0; b < B; ++b) pend[b * 3] = 1;
+    if (cudaMemcpyAsync(h->w, w0.data(), w0.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(h->pending, pend.data(), pend.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(h->grid_j, gj.data(), gj.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->stream) != cudaSuccess)
+      rc = TABED_ERR_CUDA;
+  }
+  if (rc != TABED_OK) { tabed_destroy(h); cudaGetLastError(); return rc; }
+  *out = h;
+  return TABED_OK;
+}
+
+void tabed_destroy(tabed_handle* h) {
+  if (!h) return;
+  DeviceGuard guard(h->cfg.device);
+  cudaStreamSynchronize(h->stream);
+  for (void* ptr : h->allocs) cudaFree(ptr);
+  for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+  cudaGetLastError();
+  delete h;
+}
+
+int64_t tabed_launch_count(const tabed_handle* h) { return h ? h->launches : 0; }
+
+int tabed_load_prefix_kv(tabed_handle* h, int32_t row, const void* k, const void* v, int32_t len) {
+  if (!h || !k || !v) return TABED_ERR_NULL_PTR;
+  if (!h->has_drafter || h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  if (row < 0 || row >= h->R || len < 1 || len > h->cap) return TABED_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  const size_t row_elems = (size_t)h->L * h->Hkv * h->cap * h->hd;
+  const size_t width = (size_t)len * h->hd * h->esz, dpitch = (size_t)h->cap * h->hd * h->esz;
+  unsigned char* kd = reinterpret_cast<unsigned char*>(h->kc) + row * row_elems * h->esz;
+  unsigned char* vd = reinterpret_cast<unsigned char*>(h->vc) + row * row_elems * h->esz;
+  if (cudaMemcpy2DAsync(kd, dpitch, k, width, width, (size_t)h->L * h->Hkv, cudaMemcpyDeviceToDevice, h->stream) != cudaSuccess ||
+      cudaMemcpy2DAsync(vd, dpitch, v, width, width, (size_t)h->L * h->Hkv, cudaMemcpyDeviceToDevice, h->stream) != cudaSuccess ||
+      cudaMemcpyAsync(h->kv_len + row, &len, sizeof(int), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)   // &len is a stack address
+    return TABED_ERR_CUDA;
+  h->len_ub[row] = len;
+  return TABED_OK;
+}
+
+static int prefill_common(tabed_handle* h, int32_t row, const int32_t* tokens, const float* embeds, int32_t len) {
+  if (!h || (!tokens && !embeds)) return TABED_ERR_NULL_PTR;
+  if (!h->has_drafter || h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  if (row < 0 || row >= h->R || len < 1) return TABED_ERR_INVALID_ARG;
+  if (h->len_ub[row] + len > h->cap) return TABED_ERR_KV_OVERFLOW;
+  DeviceGuard guard(h->cfg.device);
+  for (int t = 0; t < len; ++t) {
+    StepArgs sa{};
+    sa.mode = STEP_PREFILL; sa.prefill_row = row; sa.prefill_off = t;
+    sa.prefill_tokens = tokens; sa.prefill_embeds = embeds;
+    run_step(h, sa, 1, h->len_ub[row] + t + 1, nullptr);
+  }
+  TABED_LAUNCH(h, k_advance_len, (h->R + 127) / 128, 128, 0, h->kv_len, h->R, row, len);
+  h->len_ub[row] += len;
+  return check_cuda();
+}
+
+int tabed_prefill_tokens(tabed_handle* h, int32_t row, const int32_t* tokens, int32_t len) {
+  return prefill_common(h, row, tokens, nullptr, len);
+}
+int tabed_prefill_embeds(tabed_handle* h, int32_t row, const float* embeds, int32_t len) {
+  return prefill_common(h, row, nullptr, embeds, len);
+}
+
+int tabed_set_pending(tabed_handle* h, const int32_t* tok, const int32_t* cnt) {
+  if (!h || !tok || !cnt) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  DeviceGuard guard(h->cfg.device);
+  std::vector<int> ht(h->B * 2), hc(h->B), pend(h->B * 3);
+  if (cudaMemcpyAsync(ht.data(), tok, ht.size() * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaMemcpyAsync(hc.data(), cnt, hc.size() * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  for (int b = 0; b < h->B; ++b) {
+    if (hc[b] < 1 || hc[b] > 2) return TABED_ERR_INVALID_ARG;
+    for (int j = 0; j < hc[b]; ++j) if (ht[b * 2 + j] < 0 || ht[b * 2 + j] >= h->V) return TABED_ERR_INVALID_ARG;
+    pend[b * 3] = hc[b]; pend[b * 3 + 1] = ht[b * 2]; pend[b * 3 + 2] = hc[b] == 2 ? ht[b * 2 + 1] : 0;
+  }
+  if (cudaMemcpyAsync(h->pending, pend.data(), pend.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  return TABED_OK;
+}
+
+int tabed_decode_step(tabed_handle* h, const int32_t* tok, float* out_logits) {
+  if (!h || !tok) return TABED_ERR_NULL_PTR;
+  if (!h->has_drafter || h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  if (max_len_ub(h) + 1 > h->cap) return TABED_ERR_KV_OVERFLOW;
+  DeviceGuard guard(h->cfg.device);
+  StepArgs sa{};
+  sa.mode = STEP_FREE; sa.tokens = tok;
+  run_step(h, sa, h->R, max_len_ub(h) + 1, out_logits);
+  TABED_LAUNCH(h, k_advance_len, (h->R + 127) / 128, 128, 0, h->kv_len, h->R, -1, 1);
+  for (int& v : h->len_ub) v += 1;
+  return check_cuda();
+}
+
+int tabed_ensemble_step(tabed_handle* h, const float* logits, const float* w, const float* u, int32_t* y,
+                        float* q, float* qk) {
+  if (!h || !logits || !u || !y) return TABED_ERR_NULL_PTR;
+  DeviceGuard guard(h->cfg.device);
+  run_ensemble(h, logits, w ? w : h->w, u, 1, y, 1, nullptr, 0, qk, (long long)h->m * h->V,
+               q ? q : h->scratch_q, (long long)h->V);
+  return check_cuda();
+}
+
+static int draft_common(tabed_handle* h, const float* ext_logits, const float* u_draft, int32_t* out_tokens,
+                        float* out_q) {
+  if (!h || !u_draft || !out_tokens) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  const bool fwd = ext_logits == nullptr;
+  if (fwd && !h->has_drafter) return TABED_ERR_BAD_STATE;
+  if (fwd && max_len_ub(h) + 2 + h->G - 1 > h->cap) return TABED_ERR_KV_OVERFLOW;
+  DeviceGuard guard(h->cfg.device);
+  const long long RV = (long long)h->R * h->V, GV = (long long)h->G * h->V;
+  for (int i = 0; i < h->G; ++i) {
+    const float* lg;
+    if (fwd) {
+      StepArgs sa{};
+      sa.mode = (i == 0) ? STEP_ROUND_FIRST : STEP_ROUND_NEXT; sa.step = i; sa.tokens = h->tokens;
+      float* own = h->logits_own + i * RV;
+      run_step(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
+      lg = h->logits_override ? h->logits_override + i * RV : own;
+    } else {
+      lg = ext_logits + i * RV;
+    }
+    run_ensemble(h, lg, h->w, u_draft + i, h->G, h->tokens + i, h->G, out_tokens + i, h->G,
+                 h->qk + (long long)i * h->m * h->V, GV * h->m, h->q + (long long)i * h->V, GV);
+  }
+  if (out_q && cudaMemcpyAsync(out_q, h->q, sizeof(float) * h->B * GV, cudaMemcpyDeviceToDevice, h->stream) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  h->phase = PH_DRAFTED;
+  h->round_has_forward = fwd;
+  return check_cuda();
+}
+
+int tabed_draft_round(tabed_handle* h, const float* u_draft, int32_t* out_tokens, float* out_q) {
+  return draft_common(h, nullptr, u_draft, out_tokens, out_q);
+}
+
+int tabed_draft_round_logits(tabed_handle* h, const float* drafter_logits, const float* u_draft,
+                             int32_t* out_tokens, float* out_q) {
+  if (!drafter_logits) return TABED_ERR_NULL_PTR;
+  return draft_common(h, drafter_logits, u_draft, out_tokens, out_q);
+}
+
+int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_accept, const float* u_resid,
+                 int32_t* out_n_accept, int32_t* out_next_token) {
+  if (!h || !target_logits || !u_accept || !u_resid || !out_n_accept || !out_next_token) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_DRAFTED) return TABED_ERR_BAD_STATE;
+  DeviceGuard guard(h->cfg.device);
+  const int greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
+  const int rows = h->B * (h->G + 1);
+  const long long GV = (long long)h->G * h->V;
+  ProfScope ps(h, TABED_PROF_VERIFY);
+  cudaMemsetAsync(h->rowmax, 0, sizeof(uint32_t) * rows, h->stream);
+  cudaMemsetAsync(h->rowsum, 0, sizeof(unsigned long long) * rows, h->stream);
+  const dim3 grid_rows(h->n_chunks, rows), grid_req(h->n_chunks, h->B);
+  TABED_LAUNCH(h, k_rowmax, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax);
+  TABED_LAUNCH(h, k_expsum, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
+  TABED_LAUNCH(h, k_normalize, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum, h->p);
+  if (greedy) TABED_LAUNCH(h, k_row_best, grid_rows, kDecThreads, 0, h->p, h->V, h->n_chunks, h->chunk_best);
+  TABED_LAUNCH(h, k_accept, (h->B + 127) / 128, 128, 0, h->B, h->G, h->V, h->p, h->q, GV, h->tokens, u_accept,
+               h->chunk_best, h->n_chunks, greedy, h->n_accept, out_n_accept);
+  if (!greedy)
+    TABED_LAUNCH(h, k_resid_chunks, grid_req, kDecThreads, 0, h->V, h->G, h->p, h->q, GV, h->n_accept, h->chunk_mass, h->n_chunks);
+  SelectArgs s{};
+  s.V = h->V; s.n_chunks = h->n_chunks; s.G = h->G; s.greedy = greedy;
+  s.q = h->q; s.q_req_stride = GV; s.p = h->p; s.n_accept = h->n_accept; s.u = u_resid; s.u_stride = 1;
+  s.chunk_mass = h->chunk_mass; s.chunk_best = h->chunk_best;
+  s.out0 = h->next_token; s.out0_stride = 1; s.out1 = out_next_token; s.out1_stride = 1; s.err = h->err;
+  TABED_LAUNCH(h, k_select<1>, h->B, kDecThreads, 0, s);
+  h->phase = PH_VERIFIED;
+  return check_cuda();
+}
+
+int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_VERIFIED) return TABED_ERR_BAD_STATE;
+  DeviceGuard guard(h->cfg.device);
+  const int tvd = h->cfg.distance == TABED_DIST_TVD;
+  ProfScope* ps = new ProfScope(h, TABED_PROF_UPDATE);
+  TABED_LAUNCH(h, k_deviation, dim3(h->n_chunks, h->G, h->B), kDecThreads, 0, h->V, h->G, h->m, h->n_dev,
+                 h->cfg.policy == TABED_POLICY_GRID_MT ? 1 : 0, tvd, h->p, h->qk, h->n_accept, h->dev);
+  PolicyArgs a{};
+  a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
+  a.tau = h->cfg.tau; a.n_accept = h->n_accept; a.next_token = h->next_token; a.tokens = h->tokens;
+  a.dev = h->dev; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
+  a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
+  a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
+  a.pending = h->pending; a.out_w = out_w; a.out_argmax = out_w_argmax;
+  TABED_LAUNCH(h, k_policy, (h->B + 127) / 128, 128, 0, a);
+  delete ps;
+  if (h->has_drafter && h->round_has_forward) for (int& v : h->len_ub) v = std::min(v + h->G + 1, h->cap);
+  h->phase = PH_IDLE;
+  return check_cuda();
+}
+
+int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accept, const float* u_resid,
+                     const float* target_logits, int32_t* out_tokens, int32_t* out_n_accept,
+                     int32_t* out_next_token, float* out_w, int32_t* out_w_argmax) {
+  if (!h || !u_draft || !u_accept || !u_resid || !target_logits || !out_tokens || !out_n_accept || !out_next_token)
+    return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE || !h->has_drafter) return TABED_ERR_BAD_STATE;
+  DeviceGuard guard(h->cfg.device);
+  const size_t BG = (size_t)h->B * h->G;
+  cudaStream_t st = h->stream;
+  if (cudaMemcpyAsync(h->st_u_draft, u_draft, BG * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(h->st_u_accept, u_accept, BG * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(h->st_u_resid, u_resid, (size_t)h->B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(h->st_target, target_logits, (size_t)h->B * (h->G + 1) * h->V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  // outputs land in library buffers first (tokens / n_accept / next_token / w / w_argmax)
+  int rc = tabed_draft_round(h, h->st_u_draft, h->st_tokens, nullptr);
+  if (rc != TABED_OK) return rc;
+  rc = tabed_verify(h, h->st_target, h->st_u_accept, h->st_u_resid, h->n_accept, h->next_token);
+  if (rc != TABED_OK) return rc;
+  rc = tabed_update_weights(h, nullptr, h->w_argmax);
+  if (rc != TABED_OK) return rc;
+  if (cudaMemcpyAsync(out_tokens, h->tokens, BG * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(out_n_accept, h->n_accept, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(out_next_token, h->next_token, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      (out_w && cudaMemcpyAsync(out_w, h->w, (size_t)h->B * h->m * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) ||
+      (out_w_argmax && cudaMemcpyAsync(out_w_argmax, h->w_argmax, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  return TABED_OK;
+}
+
+int tabed_profile_begin(tabed_handle* h, int32_t kernel_class) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (kernel_class < 0 || kernel_class > TABED_PROF_UPDATE) return TABED_ERR_INVALID_ARG;
+  h->prof_class = kernel_class;
+  h->prof_used = 0;
+  return TABED_OK;
+}
+
+int tabed_profile_end(tabed_handle* h, double* total_ms, int64_t* n_intervals) {
+  if (!h || !total_ms || !n_intervals) return TABED_ERR_NULL_PTR;
+  DeviceGuard guard(h->cfg.device);
+  h->prof_class = -1;
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+  double tot = 0.0;
+  const size_t pairs = h->prof_used / 2;
+  for (size_t i = 0; i < pairs; ++i) {
+    float ms = 0.0f;
+    if (cudaEventElapsedTime(&ms, h->prof_events[2 * i], h->prof_events[2 * i + 1]) != cudaSuccess) return TABED_ERR_CUDA;
+    tot += ms;
+  }
+  *total_ms = tot; *n_intervals = (int64_t)pairs;
+  h->prof_used = 0;
+  return TABED_OK;
+}
+
+int tabed_debug_override_logits(tabed_handle* h, const float* drafter_logits) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  h->logits_override = drafter_logits;
+  return TABED_OK;
+}
+
+int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* bytes) {
+  if (!h || !dev_ptr || !bytes) return TABED_ERR_NULL_PTR;
+  const size_t B = h->B, m = h->m, G = h->G, V = h->V, R = h->R;
+  switch (what) {
+    case TABED_VIEW_QK: *dev_ptr = h->qk; *bytes = B * G * m * V * 4; break;
+    case TABED_VIEW_Q: *dev_ptr = h->q; *bytes = B * G * V * 4; break;
+    case TABED_VIEW_P: *dev_ptr = h->p; *bytes = B * (G + 1) * V * 4; break;
+    case TABED_VIEW_LOGITS: if (!h->has_drafter) return TABED_ERR_BAD_STATE; *dev_ptr = h->logits_own; *bytes = G * R * V * 4; break;
+    case TABED_VIEW_KV_LEN: if (!h->has_drafter) return TABED_ERR_BAD_STATE; *dev_ptr = h->kv_len; *bytes = R * 4; break;
+    case TABED_VIEW_WEIGHTS: *dev_ptr = h->w; *bytes = B * m * 4; break;
+    case TABED_VIEW_WINDOW_SUM: *dev_ptr = h->running; *bytes = B * kMaxDev * 8; break;
+    case TABED_VIEW_PENDING: *dev_ptr = h->pending; *bytes = B * 3 * 4; break;
+    case TABED_VIEW_GRID_J: *dev_ptr = h->grid_j; *bytes = B * 4; break;
+    case TABED_VIEW_ERROR_FLAG: *dev_ptr = h->err; *bytes = 4; break;
+    default: return TABED_ERR_INVALID_ARG;
+  }
+  return TABED_OK;
+}
+
+// snapshot layout: header {magic, B, m, h, has_kv, R} then the arrays in a fixed order
+struct Snap { void* ptr; size_t bytes; };
+static std::vector<Snap> snap_parts(tabed_handle* h) {
+  const size_t B = h->B, hh = std::max(1, h->cfg.window_h);
+  std::vector<Snap> v = {
+      {h->w, B * h->m * 4}, {h->pending, B * 3 * 4}, {h->ring, B * hh * kMaxDev * 8}, {h->running, B * kMaxDev * 8},
+      {h->pushed, B * 8}, {h->ring_head, B * 4}, {h->ring_count, B * 4}, {h->grid_j, B * 4}};
+  if (h->has_drafter) v.push_back({h->kv_len, (size_t)h->R * 4});
+  return v;
+}
+
+int tabed_state_export(tabed_handle* h, void* host, size_t* bytes) {
+  if (!h || !bytes) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  const auto parts = snap_parts(h);
+  size_t total = 6 * sizeof(int32_t);
+  for (const auto& s : parts) total += s.bytes;
+  if (!host) { *bytes = total; return TABED_OK; }
+  if (*bytes < total) return TABED_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  int32_t hdr[6] = {0x7ABED, h->B, h->m, h->cfg.window_h, h->has_drafter ? 1 : 0, h->R};
+  unsigned char* o = reinterpret_cast<unsigned char*>(host);
+  memcpy(o, hdr, sizeof(hdr)); o += sizeof(hdr);
+  for (const auto& s : parts) {
+    if (cudaMemcpyAsync(o, s.ptr, s.bytes, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+    o += s.bytes;
+  }
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+  if (h->has_drafter) {
+    const int32_t* lens = reinterpret_cast<const int32_t*>(o - (size_t)h->R * 4);
+    for (int r = 0; r < h->R; ++r) h->len_ub[r] = lens[r];      // tighten the host-side bound
+  }
+  *bytes = total;
+  return TABED_OK;
+}
+
+int tabed_state_import(tabed_handle* h, const void* host, size_t bytes) {
+  if (!h || !host) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  const auto parts = snap_parts(h);
+  size_t total = 6 * sizeof(int32_t);
+  for (const auto& s : parts) total += s.bytes;
+  if (bytes != total) return TABED_ERR_INVALID_ARG;
+  const unsigned char* in = reinterpret_cast<const unsigned char*>(host);
+  int32_t hdr[6];
+  memcpy(hdr, in, sizeof(hdr)); in += sizeof(hdr);
+  if (hdr[0] != 0x7ABED || hdr[1] != h->B || hdr[2] != h->m || hdr[3] != h->cfg.window_h ||
+      hdr[4] != (h->has_drafter ? 1 : 0) || hdr[5] != h->R)
+    return TABED_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  for (const auto& s : parts) {
+    if (cudaMemcpyAsync(s.ptr, in, s.bytes, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+    in += s.bytes;
+  }
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+  if (h->has_drafter) {
+    const int32_t* lens = reinterpret_cast<const int32_t*>(in - (size_t)h->R * 4);
+    for (int r = 0; r < h->R; ++r) {
+      if (lens[r] < 0 || lens[r] > h->cap) return TABED_ERR_INVALID_ARG;
+      h->len_ub[r] = lens[r];
+    }
+  }
+  return TABED_OK;
+}
+
+}  // extern "C"

@@ -152,3 +152,31 @@ def test_workload_bf16_grid_helpers_against_torch():
     t = torch.tensor(x).to(torch.bfloat16)
     assert np.array_equal(g, t.to(torch.float32).numpy())
     assert np.array_equal(W.f32_to_bf16_bits(g), t.view(torch.int16).numpy().view(np.uint16))
+
+
+def test_bf16_rounding_flip_noise_sets_the_logit_tolerance():
+    """Two evaluations that differ by 1e-7 relative before each bf16 rounding (what fp32 against fp64
+    accumulation amounts to) disagree on some roundings; this measures how far the logits move and
+    checks it stays inside the bound the GPU parity tests use for a bf16 drafter."""
+    cfg = W.DrafterCfg(2, 256, 4, 2, 640, 3000, "bf16")
+    wl = W.Workload(name="flip", config_id=41, drafter=cfg, n_inputs=1, n_requests=1, gamma=2, window_h=2,
+                    rounds=1, policy=W.POLICY_STATIC)
+    weights = W.make_weights(wl)
+
+    class Perturbed(OracleDrafter):
+        def rb(self, x):
+            return round_bf16(x * (1 + 1e-7 * self.noise.standard_normal(x.shape)))
+
+    a, b = OracleDrafter(cfg, weights), Perturbed(cfg, weights)
+    b.noise = np.random.default_rng(0)
+    tokens = np.random.default_rng(1).integers(0, cfg.vocab, size=150)
+    ca, cb = a.new_cache(160), b.new_cache(160)
+    a.forward(ca, a.embed_tokens(tokens[:-1]), want_logits=False)
+    b.forward(cb, b.embed_tokens(tokens[:-1]), want_logits=False)
+    la = a.forward(ca, a.embed_tokens(tokens[-1:]))
+    lb = b.forward(cb, b.embed_tokens(tokens[-1:]))
+    err = np.abs(la - lb)
+    assert 1e-5 < err.mean() < 1e-2 and err.max() < 6e-2
+    # and the probabilities stay inside the 1e-5 bar
+    from oracle import definitions as D
+    assert np.max(np.abs(D.softmax(la) - D.softmax(lb))) < 1e-5
