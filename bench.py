@@ -1,0 +1,430 @@
+#!/usr/bin/env python
+"""Benchmark of one TABED speculative-decoding round on B200.
+
+A step is one round of the whole hot path on one batch of synthetic input:
+tabed_draft_round (gamma batched shared-weight drafter steps with ensemble + draw at each) ->
+tabed_verify -> tabed_update_weights.  The stand-in for the target model (it only has to produce
+target logits) is outside the path: its logits are prepared by an untimed rehearsal of exactly the
+rounds that are then timed (the library is deterministic, so the replay sees the same rounds).
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU checker instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_20357_b200 import workloads as W  # noqa: E402
+
+METRIC = "sd_rounds_per_sec"
+UNIT = "rounds/s"
+PAPER_CONTEXT = ("paper (A100 80GB, fp16): expected walltime speedup 1.74x over autoregressive decoding, "
+                 "~5% block-efficiency gain over single drafting; no rounds/s published")
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        os.unlink(self.path)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU checker as baseline / reference arm
+# --------------------------------------------------------------------------------------------------
+def oracle_setup(wl):
+    from oracle.drafter import OracleDrafter
+    from oracle.tabed import TabedOracle
+    weights = W.make_weights(wl)
+    orc = TabedOracle(n_inputs=wl.n_inputs, n_requests=wl.n_requests, gamma=wl.gamma, window_h=wl.window_h,
+                      policy=wl.policy, vocab=wl.drafter.vocab, distance=wl.distance, sample_mode=wl.sample_mode,
+                      tau=wl.tau, drafter=OracleDrafter(wl.drafter, weights), kv_capacity=wl.kv_capacity)
+    if wl.synthetic_kv_len is not None:
+        lens = W.synthetic_kv_lengths(wl)
+        for row in range(wl.n_rows):
+            k, v = W.make_synthetic_kv(wl, row, int(lens[row]))
+            orc.load_kv(row, k, v)
+    else:
+        for b in range(wl.n_requests):
+            for k, segs in enumerate(W.make_prefixes(wl, b)):
+                orc.prefill(b * wl.n_inputs + k, segs)
+    orc.set_pending(W.initial_pending(wl))
+    return orc
+
+
+def oracle_round(orc, wl, rnd):
+    ud, ua, ur = W.round_uniforms(wl, rnd)
+    orc.draft_round(ud)
+    a, _ = orc.verify(W.target_logits(wl, rnd, orc.logits), ua, ur)
+    orc.update_weights()
+    return int(a.sum())
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(wl, rounds, warmup=0):
+    orc = oracle_setup(wl)
+    for r in range(warmup):
+        oracle_round(orc, wl, r)
+    t0 = time.perf_counter()
+    for r in range(warmup, warmup + rounds):
+        oracle_round(orc, wl, r)
+    dt = time.perf_counter() - t0
+    return wl.n_requests * rounds / dt, dt
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    value, dt = time_oracle(wl, args.steps, args.warmup)
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1000.0 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "n_inputs": wl.n_inputs, "n_requests": wl.n_requests, "gamma": wl.gamma,
+                   "window_h": wl.window_h, "vocab": wl.drafter.vocab},
+        "drafted_tokens_per_sec": value * wl.gamma,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{args.steps} rounds of {wl.name} after {args.warmup} warm-up rounds, every round whole"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# CUDA arm
+# --------------------------------------------------------------------------------------------------
+def gpu_setup(wl, device):
+    import torch
+    from paper_2601_20357_b200 import binding as TB
+    weights = TB.weights_to_device(wl.drafter, W.make_weights(wl), device)
+    g = TB.Tabed(n_inputs=wl.n_inputs, n_requests=wl.n_requests, gamma=wl.gamma, window_h=wl.window_h,
+                 policy=wl.policy, vocab=wl.drafter.vocab, distance=wl.distance, sample_mode=wl.sample_mode,
+                 tau=wl.tau, drafter=wl.drafter, weights=weights, kv_capacity=wl.kv_capacity, device=device.index)
+    tdt = torch.float32 if wl.drafter.dtype == "fp32" else torch.bfloat16
+    dev = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(device) if dt is None
+                              else torch.from_numpy(np.ascontiguousarray(a)).to(device).to(dt))
+    if wl.synthetic_kv_len is not None:
+        lens = W.synthetic_kv_lengths(wl)
+        for row in range(wl.n_rows):
+            k, v = W.make_synthetic_kv(wl, row, int(lens[row]))
+            g.load_prefix_kv(row, dev(k, tdt), dev(v, tdt))
+    else:
+        for b in range(wl.n_requests):
+            for k, segs in enumerate(W.make_prefixes(wl, b)):
+                for seg in segs:
+                    if seg.kind == "tokens":
+                        g.prefill_tokens(b * wl.n_inputs + k, dev(seg.data))
+                    else:
+                        g.prefill_embeds(b * wl.n_inputs + k, dev(seg.data))
+    tok = np.zeros((wl.n_requests, 2), np.int32)
+    tok[:, 0] = W.initial_pending(wl)
+    g.set_pending(dev(tok), dev(np.ones(wl.n_requests, np.int32)))
+    torch.cuda.synchronize(device)
+    return g
+
+
+def class_bytes(wl, kv_tokens_total, mean_accept):
+    """Algorithmic bytes one timed interval of each kernel class has to move."""
+    c = wl.drafter
+    e = 4 if c.dtype == "fp32" else 2
+    R, B, m, G, V, d, F = wl.n_rows, wl.n_requests, wl.n_inputs, wl.gamma, c.vocab, c.d_model, c.d_ffn
+    kvd = c.n_kv_heads * c.head_dim
+    valid = min(mean_accept, G - 1) + 1
+    return {
+        "qkv": (d * d + 2 * kvd * d) * e + R * d * 4 + R * (d + 2 * kvd) * 4,
+        "attention": kv_tokens_total * 2 * kvd * e + R * (d + 2 * kvd) * 4 + R * d * 4,
+        "oproj": d * d * e + 2 * R * d * 4,
+        "gateup": 2 * F * d * e + R * d * 4 + R * F * 4,
+        "down": d * F * e + R * F * 4 + 2 * R * d * 4,
+        "lm_head": V * d * e + R * d * 4 + R * V * 4,
+        "ensemble": R * V * 4 + B * V * 4 + R * V * 4,
+        "verify": (G + 1) * B * V * 4 * 2 + G * B * V * 4,
+        "update": valid * (m + 1) * B * V * 4,
+    }
+
+
+def run_ours(args, wl):
+    import torch
+    from paper_2601_20357_b200 import binding as TB
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+    K, Wm = args.steps, args.warmup
+    total = K + Wm
+    B, G, m, V = wl.n_requests, wl.gamma, wl.n_inputs, wl.drafter.vocab
+    if wl.kv_capacity and wl.synthetic_kv_len is None:
+        need = max(sum(l for _, l in pre) for pre in wl.prefixes) + (total + args.e2e_steps + 24) * (G + 1) + 8
+        if need > wl.kv_capacity:
+            wl = wl.replace(kv_capacity=need)
+    g = gpu_setup(wl, device)
+    snap = g.state_export()
+    alpha = torch.from_numpy(W.request_alpha(wl)).to(device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(W.MASTER_SEED + rank)
+
+    # uniforms for every round, resident on the device
+    u = [tuple(torch.from_numpy(x).to(device) for x in W.round_uniforms(wl, r)) for r in range(total)]
+    toks = torch.empty((B, G), dtype=torch.int32, device=device)
+    a = torch.empty(B, dtype=torch.int32, device=device)
+    z = torch.empty_like(a)
+    am = torch.empty_like(a)
+    w = torch.empty((B, m), dtype=torch.float32, device=device)
+
+    def synth_target(rnd):
+        lg = g.debug_view(TB.VIEW_LOGITS)                               # [G][B][m][V]
+        mix = torch.einsum("gbnv,bn->bgv", lg, alpha)
+        tl = torch.empty((B, G + 1, V), dtype=torch.float32, device=device)
+        tl[:, :G] = mix
+        tl[:, G] = mix[:, G - 1]
+        tl += wl.sigma(rnd) * torch.randn(tl.shape, generator=gen, device=device)
+        return tl
+
+    # ---- rehearsal: produce the target logits of every round (untimed) ----
+    targets, accepted = [], 0
+    for r in range(total):
+        g.draft_round(u[r][0], toks)
+        tl = synth_target(r)
+        g.verify(tl, u[r][1], u[r][2], a, z)
+        g.update_weights(w, am)
+        targets.append(tl)
+        accepted += int(a.sum())
+    torch.cuda.synchronize(device)
+    mean_accept = accepted / (total * B)
+    kv_mean = float(g.debug_view(TB.VIEW_KV_LEN).float().sum())       # tokens cached at the end of the rehearsal
+    g.state_import(snap)
+    kv_start = float(g.debug_view(TB.VIEW_KV_LEN).float().sum())
+    kv_tokens_total = 0.5 * (kv_start + kv_mean) + wl.n_rows * (1 + G / 2)
+
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+
+    def one_round(r):
+        g.draft_round(u[r][0], toks)
+        g.verify(targets[r], u[r][1], u[r][2], a, z)
+        g.update_weights(w, am)
+
+    for r in range(Wm):
+        flush.zero_()
+        one_round(r)
+    torch.cuda.synchronize(device)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = g.launch_count()
+    g.profile_begin(TB.PROF_LM_HEAD)
+    wall0 = time.perf_counter()
+    for i in range(K):
+        flush.zero_()                       # the target model's pass between rounds evicts L2 in deployment
+        ev[i][0].record()
+        one_round(Wm + i)
+        ev[i][1].record()
+    head_ms, head_n = g.profile_end()       # synchronises the stream
+    torch.cuda.synchronize(device)
+    wall = time.perf_counter() - wall0
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    clocks = sampler.stop()
+    launches = g.launch_count() - launches0
+    per_round = np.array([s.elapsed_time(e) for s, e in ev])
+    dev_ms = float(per_round.sum())
+    if dist is not None:
+        tt = torch.tensor([dev_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dev_ms = float(tt.item())
+    value = world * B * K / (dev_ms / 1000.0)
+
+    peak, peak_kind = read_peaks()
+    cb = class_bytes(wl, kv_tokens_total, mean_accept)
+    head_dur = head_ms / max(head_n, 1)
+    head_gbs = cb["lm_head"] / (head_dur * 1e-3) / 1e9
+
+    # ---- per-class breakdown (separate untimed-for-the-headline passes over the same rounds) ----
+    kernels = {}
+    if rank == 0 and not args.no_breakdown:
+        names = ["qkv", "attention", "oproj", "gateup", "down", "lm_head", "ensemble", "verify", "update"]
+        nb = min(K, 12)
+        for cls, nm in enumerate(names):
+            g.state_import(snap)
+            for r in range(Wm):
+                one_round(r)
+            g.profile_begin(cls)
+            for i in range(nb):
+                flush.zero_()
+                one_round(Wm + i)
+            ms, n = g.profile_end()
+            dur = ms / max(n, 1)
+            kernels[nm] = {"intervals_per_round": n / nb, "avg_us": 1000.0 * dur, "bytes": int(cb[nm]),
+                           "gbs": cb[nm] / (dur * 1e-3) / 1e9 if dur > 0 else None,
+                           "frac_of_peak": cb[nm] / (dur * 1e-3) / 1e9 / peak if dur > 0 else None,
+                           "share_of_round": ms / nb / float(per_round.mean())}
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e = None
+    if rank == 0 and args.e2e_steps > 0:
+        ne = min(args.e2e_steps, K)
+        g.state_import(snap)
+        for r in range(Wm):
+            one_round(r)
+        torch.cuda.synchronize(device)
+        pin = lambda x: x.cpu().pin_memory()
+        hu = [(pin(u[Wm + i][0]), pin(u[Wm + i][1]), pin(u[Wm + i][2]), pin(targets[Wm + i])) for i in range(ne)]
+        h_toks = torch.empty((B, G), dtype=torch.int32).pin_memory()
+        h_a = torch.empty(B, dtype=torch.int32).pin_memory()
+        h_z = torch.empty(B, dtype=torch.int32).pin_memory()
+        h_am = torch.empty(B, dtype=torch.int32).pin_memory()
+        h_w = torch.empty((B, m), dtype=torch.float32).pin_memory()
+        t0 = time.perf_counter()
+        for i in range(ne):
+            g.round_host(hu[i][0], hu[i][1], hu[i][2], hu[i][3], h_toks, h_a, h_z, h_w, h_am)
+        dt = time.perf_counter() - t0
+        h2d = sum(x.numel() * x.element_size() for x in hu[0])
+        d2h = sum(x.numel() * x.element_size() for x in (h_toks, h_a, h_z, h_am, h_w))
+        e2e = {"value": B * ne / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+               "steps": ne, "note": "tabed_round_host, pinned host buffers, L2 not flushed between rounds"}
+
+    if rank != 0:
+        return
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        n_cpu = args.cpu_rounds
+        v, dt = time_oracle(wl, n_cpu, 0)
+        cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"first {n_cpu} rounds of {wl.name} (whole rounds, prefill untimed), {dt:.1f} s"}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 accumulate over bf16 weights/KV" if wl.drafter.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "n_inputs": m, "n_requests": B, "rows": wl.n_rows, "gamma": G,
+                   "window_h": wl.window_h, "vocab": V, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model,
+                   "l2": "256 MB written between rounds (stands for the target model's pass); rounds timed one by one "
+                         "with CUDA events", "parallelism": f"replicas x{world}"},
+        "drafted_tokens_per_sec": value * G,
+        "block_efficiency": mean_accept + 1.0,
+        "wall_ms_per_step_incl_flush": 1000.0 * wall / K,
+        "roofline": {"kernel": "k_gemv (LM head)", "bound": "hbm", "achieved": head_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": head_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                     "avg_us": 1000.0 * head_dur, "launches_timed": head_n, "bytes_per_launch": int(cb["lm_head"])},
+        "round_roofline": {"bytes_per_round": int(G * (sum(cb[k] for k in ("qkv", "attention", "oproj", "gateup", "down"))
+                                                     * wl.drafter.n_layers + cb["lm_head"] + cb["ensemble"])
+                                                 + cb["verify"] + cb["update"]),
+                           "note": "algorithmic bytes of one round / measured round time / peak"},
+        "kernels": kernels,
+        "cpu_baseline": cpu,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "context": PAPER_CONTEXT,
+    }
+    rr = line["round_roofline"]
+    rr["achieved_gbs"] = rr["bytes_per_round"] / (dev_ms / K * 1e-3) / 1e9
+    rr["frac"] = rr["achieved_gbs"] / peak
+    print(json.dumps(line), flush=True)
+    g.destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llava_small", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=50)
+    ap.add_argument("--cpu-rounds", type=int, default=60)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-breakdown", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    wl = W.WORKLOADS[args.config]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
