@@ -189,6 +189,36 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
 /* Pointer and size of a library-owned device buffer (TABED_VIEW_*).  Read-only for the caller. */
 int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* bytes);
 
+/* Allocation-free variant of tabed_ensemble_step (the paper has no counterpart: this is a
+ * deployment convenience, not a step of the method).
+ *
+ * For callers that must not allocate device memory at the point of use: a serving process that has
+ * already handed the whole GPU to its own memory pool, a plug-in running under a fixed memory
+ * budget, or a latency-critical path where cudaMalloc (which may synchronise the device and may
+ * fail late) is not acceptable.  Such callers cannot create a handle, because tabed_init allocates.
+ * This entry point needs no handle and calls no cudaMalloc / cudaFree or any allocating routine:
+ * its scratch (row maxima and sums, per-chunk masses) is a fixed 144 KB array compiled into the
+ * library's device image, held by every GPU that loads the library until the process exits.
+ *
+ * Computes exactly what tabed_ensemble_step computes: q^(k) = softmax(logits^(k)),
+ * q = sum_k w_k q^(k), y = Sample(q; u) (argmax when sample_mode is TABED_MODE_GREEDY).
+ * Device pointers on `device`: logits float [B][m][V], w float [B][m] (required), u float [B];
+ * outputs y int32 [B], q float [B][V] (required: the draw re-reads it), qk float [B][m][V] or NULL.
+ * Work is enqueued on `stream` (cudaStream_t, NULL = legacy default stream); no host synchronisation.
+ *
+ * Limits: B*m <= TABED_STATIC_MAX_ROWS and B*ceil(V/2048) <= TABED_STATIC_MAX_CHUNKS; larger
+ * problems return TABED_ERR_UNSUPPORTED (use a handle).  m <= TABED_MAX_INPUTS.
+ * The first call on each device looks up the scratch array's device address (a host-side set-up
+ * step); make that first call before any stream capture begins.
+ * All calls on one device share the one scratch array, which keeps the last call's contents (the
+ * call clears what has to start at zero): two calls whose kernels overlap on the GPU, e.g. on
+ * different streams, race.  Serialise them on one stream or with events. */
+#define TABED_STATIC_MAX_ROWS   1024
+#define TABED_STATIC_MAX_CHUNKS 8192
+int tabed_ensemble_step_static(const float* logits, const float* w, const float* u, int32_t n_requests,
+                               int32_t n_inputs, int32_t vocab, int32_t sample_mode, int32_t device,
+                               void* stream, int32_t* y, float* q, float* qk);
+
 /* Replay aid: while set (non-NULL), tabed_draft_round still runs its own forward pass (caches and
  * TABED_VIEW_LOGITS are written as usual) but steps 6-7 of Algorithm 1 read these logits
  * float [G][B][m][V] instead, so that a recorded trajectory can be followed exactly while the

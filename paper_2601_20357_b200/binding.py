@@ -31,7 +31,7 @@ EXPORTS = [
     "tabed_prefill_embeds", "tabed_set_pending", "tabed_decode_step", "tabed_ensemble_step",
     "tabed_draft_round", "tabed_draft_round_logits", "tabed_verify", "tabed_update_weights",
     "tabed_round_host", "tabed_debug_view", "tabed_debug_override_logits", "tabed_state_export", "tabed_state_import",
-    "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end",
+    "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end", "tabed_ensemble_step_static",
 ]
 
 
@@ -96,6 +96,7 @@ def lib() -> C.CDLL:
         L.tabed_state_import.argtypes = [vp, vp, sz]
         L.tabed_profile_begin.argtypes = [vp, i32]
         L.tabed_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        L.tabed_ensemble_step_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.tabed_launch_count.argtypes = [vp]
         L.tabed_launch_count.restype = C.c_int64
         for name in EXPORTS:
@@ -306,3 +307,22 @@ def weights_to_device(drafter, weights_np: Dict[str, object], device: torch.devi
     for k, v in weights_np.items():
         out[k] = [conv(a) for a in v] if isinstance(v, list) else conv(v)
     return out
+
+
+def ensemble_step_static(logits: torch.Tensor, w: torch.Tensor, u: torch.Tensor, y: torch.Tensor, q: torch.Tensor,
+                         qk: Optional[torch.Tensor] = None, sample_mode: int = MODE_SAMPLE,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+    """tabed_ensemble_step_static: the ensemble step without a handle and without any allocation.
+
+    For callers that cannot allocate device memory where they draft (all memory already owned by a
+    serving pool, fixed budgets, paths that must not hit cudaMalloc): scratch is a fixed array inside
+    the library.  logits [B][m][V], w [B][m], u [B] -> y [B], q [B][V], optional qk [B][m][V].
+    Calls on one device share that scratch, so they must not overlap on the GPU."""
+    B, m, V = logits.shape
+    d = logits.device
+    _check(lib().tabed_ensemble_step_static(
+        _ptr(logits, torch.float32, B * m * V, "logits", d), _ptr(w, torch.float32, B * m, "w", d),
+        _ptr(u, torch.float32, B, "u", d), B, m, V, sample_mode, d.index if d.index is not None else 0,
+        stream.cuda_stream if stream is not None else None,
+        _ptr(y, torch.int32, B, "y", d), _ptr(q, torch.float32, B * V, "q", d),
+        _ptr(qk, torch.float32, B * m * V, "qk", d)), "tabed_ensemble_step_static")

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <type_traits>
 #include <vector>
@@ -732,6 +733,80 @@ int tabed_state_import(tabed_handle* h, const void* host, size_t bytes) {
     }
   }
   return TABED_OK;
+}
+
+// -------------------------------------------------------------------------------------------------
+// Allocation-free ensemble step.
+//
+// Scratch of the softmax / mix / draw kernels (row maxima, row sums, per-chunk masses and bests,
+// an error word) lives in this file-scope device array instead of a buffer from tabed_init.  Every
+// GPU that loads the library holds these 144 KB until the process exits.  In host code the name
+// below is only a stand-in: its device address is fetched per device with cudaGetSymbolAddress.
+// -------------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticRowMaxOff = 0;                                                        // uint32 [MAX_ROWS]
+constexpr size_t kStaticRowSumOff = kStaticRowMaxOff + 4 * (size_t)TABED_STATIC_MAX_ROWS;     // uint64 [MAX_ROWS]
+constexpr size_t kStaticMassOff = kStaticRowSumOff + 8 * (size_t)TABED_STATIC_MAX_ROWS;       // uint64 [MAX_CHUNKS]
+constexpr size_t kStaticBestOff = kStaticMassOff + 8 * (size_t)TABED_STATIC_MAX_CHUNKS;       // ChunkBest [MAX_CHUNKS]
+constexpr size_t kStaticErrOff = kStaticBestOff + 8 * (size_t)TABED_STATIC_MAX_CHUNKS;        // int32
+constexpr size_t kStaticBytes = kStaticErrOff + 256;
+static_assert(sizeof(ChunkBest) == 8, "scratch layout assumes 8-byte ChunkBest");
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_tabed_static_scratch[kStaticBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {nullptr};
+}  // namespace
+
+int tabed_ensemble_step_static(const float* logits, const float* w, const float* u, int32_t n_requests,
+                               int32_t n_inputs, int32_t vocab, int32_t sample_mode, int32_t device, void* stream,
+                               int32_t* y, float* q, float* qk) {
+  if (!logits || !w || !u || !y || !q) return TABED_ERR_NULL_PTR;
+  if (n_requests < 1 || n_inputs < 1 || n_inputs > TABED_MAX_INPUTS || vocab < 2 || sample_mode < 0 || sample_mode > 1 ||
+      device < 0 || device >= kMaxDevices)
+    return TABED_ERR_INVALID_ARG;
+  const long long rows = (long long)n_requests * n_inputs;
+  const int n_chunks = (vocab + kChunk - 1) / kChunk;
+  if (rows > TABED_STATIC_MAX_ROWS || (long long)n_requests * n_chunks > TABED_STATIC_MAX_CHUNKS)
+    return TABED_ERR_UNSUPPORTED;                       // beyond the fixed scratch: use a handle instead
+  DeviceGuard guard(device);
+  if (!guard.ok) return TABED_ERR_CUDA;
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {                        // once per device, with that device current
+      void* sym = nullptr;
+      if (cudaGetSymbolAddress(&sym, g_tabed_static_scratch) != cudaSuccess || !sym) { cudaGetLastError(); return TABED_ERR_CUDA; }
+      g_static_ptr[device] = reinterpret_cast<unsigned char*>(sym);
+    }
+    base = g_static_ptr[device];
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint32_t* rowmax = reinterpret_cast<uint32_t*>(base + kStaticRowMaxOff);
+  unsigned long long* rowsum = reinterpret_cast<unsigned long long*>(base + kStaticRowSumOff);
+  unsigned long long* cmass = reinterpret_cast<unsigned long long*>(base + kStaticMassOff);
+  ChunkBest* cbest = reinterpret_cast<ChunkBest*>(base + kStaticBestOff);
+  int* err = reinterpret_cast<int*>(base + kStaticErrOff);
+  // the array keeps the previous call's contents: the running maxima and sums must start at zero
+  if (cudaMemsetAsync(rowmax, 0, sizeof(uint32_t) * rows, st) != cudaSuccess ||
+      cudaMemsetAsync(rowsum, 0, sizeof(unsigned long long) * rows, st) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  const int R = (int)rows, B = n_requests, V = vocab, greedy = sample_mode == TABED_MODE_GREEDY;
+  const dim3 grid_rows(n_chunks, R), grid_req(n_chunks, B);
+  k_rowmax<<<grid_rows, kDecThreads, 0, st>>>(logits, V, (long long)V, rowmax);
+  k_expsum<<<grid_rows, kDecThreads, 0, st>>>(logits, V, (long long)V, rowmax, rowsum);
+  k_mix<<<grid_req, kDecThreads, 0, st>>>(logits, V, n_inputs, w, rowmax, rowsum, qk, (long long)n_inputs * V, q,
+                                          (long long)V, cmass, cbest, n_chunks, greedy);
+  SelectArgs s{};
+  s.V = V; s.n_chunks = n_chunks; s.G = 1; s.greedy = greedy;
+  s.q = q; s.q_req_stride = V; s.u = u; s.u_stride = 1;
+  s.chunk_mass = cmass; s.chunk_best = cbest;
+  s.out0 = y; s.out0_stride = 1; s.out1 = nullptr; s.out1_stride = 0; s.err = err;
+  k_select<0><<<B, kDecThreads, 0, st>>>(s);
+  return check_cuda();
 }
 
 }  // extern "C"
