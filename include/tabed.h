@@ -75,6 +75,17 @@ extern "C" {
 #define TABED_VIEW_PENDING     7   /* int32  [B][3]        {count, token0, token1}                     */
 #define TABED_VIEW_GRID_J      8   /* int32  [B]           j* of the grid policy (-1 before any update)*/
 #define TABED_VIEW_ERROR_FLAG  9   /* int32  [1]           non-zero if a device-side check failed      */
+#define TABED_VIEW_TRACE      10   /* uint64 [G][5L+8]     nanosecond timer after each grid barrier of the
+                                                           persistent drafting kernel (tabed_debug_trace)  */
+
+/* How tabed_draft_round runs Algorithm 1 (tabed_select_path).  Results obey the same contract on
+ * both paths: identical integer decisions for identical logits; logits agree within the forward
+ * pass's floating-point tolerance (summation order differs). */
+#define TABED_PATH_AUTO        0   /* persistent kernel when the drafter qualifies, else per-operation  */
+#define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
+#define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, 2*B*m <= 8
+                                      slots, d_model <= 2048 and a multiple of 16, d_ffn a multiple of 16,
+                                      (H/Hkv)*head_dim <= 512                                            */
 
 typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
 
@@ -186,6 +197,19 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
                      int32_t* out_n_accept, int32_t* out_next_token, float* out_w,
                      int32_t* out_w_argmax);
 
+/* Choose the drafting path (TABED_PATH_*).  Errors: UNSUPPORTED (TABED_PATH_PERSISTENT on a drafter
+ * that does not qualify), BAD_STATE (mid-round), INVALID_ARG.  tabed_current_path returns the path
+ * the next tabed_draft_round will take: TABED_PATH_PER_OP or TABED_PATH_PERSISTENT (positive), or a
+ * negative error code. */
+int tabed_select_path(tabed_handle* h, int32_t path);
+int tabed_current_path(const tabed_handle* h);
+
+/* Switch the phase timeline of the persistent kernel on or off: when on, CTA 0 stores the GPU's
+ * nanosecond timer after every grid barrier into TABED_VIEW_TRACE (row = drafting step).  Barrier
+ * order within a step: per layer QKV, attention, O, gate/up, down; then LM head, [2 more when
+ * tabed_debug_override_logits is set], exp-sum, mix.  Errors: UNSUPPORTED (no persistent path). */
+int tabed_debug_trace(tabed_handle* h, int32_t on);
+
 /* Pointer and size of a library-owned device buffer (TABED_VIEW_*).  Read-only for the caller. */
 int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* bytes);
 
@@ -235,7 +259,8 @@ int tabed_state_import(tabed_handle* h, const void* host, size_t bytes);
  * records a CUDA event pair on config.stream around every launch (group) of that class;
  * tabed_profile_end synchronises the stream and returns the summed elapsed milliseconds and the
  * number of timed intervals.  TABED_PROF_ATTENTION, _ENSEMBLE, _VERIFY and _UPDATE time their group
- * of kernels as one interval; the others time a single kernel per interval. */
+ * of kernels as one interval; the others time a single kernel per interval.  Classes 0-6 only occur
+ * on the per-operation path, TABED_PROF_DRAFT_ROUND only on the persistent path. */
 #define TABED_PROF_QKV        0
 #define TABED_PROF_ATTENTION  1
 #define TABED_PROF_OPROJ      2
@@ -245,6 +270,7 @@ int tabed_state_import(tabed_handle* h, const void* host, size_t bytes);
 #define TABED_PROF_ENSEMBLE   6
 #define TABED_PROF_VERIFY     7
 #define TABED_PROF_UPDATE     8
+#define TABED_PROF_DRAFT_ROUND 9  /* the persistent kernel: one interval per tabed_draft_round */
 int tabed_profile_begin(tabed_handle* h, int32_t kernel_class);
 int tabed_profile_end(tabed_handle* h, double* total_ms, int64_t* n_intervals);
 

@@ -21,10 +21,11 @@ POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR = 0, 1, 2
 DIST_KL, DIST_TVD = 0, 1
 MODE_SAMPLE, MODE_GREEDY = 0, 1
 (VIEW_QK, VIEW_Q, VIEW_P, VIEW_LOGITS, VIEW_KV_LEN, VIEW_WEIGHTS, VIEW_WINDOW_SUM, VIEW_PENDING,
- VIEW_GRID_J, VIEW_ERROR_FLAG) = range(10)
+ VIEW_GRID_J, VIEW_ERROR_FLAG, VIEW_TRACE) = range(11)
+PATH_AUTO, PATH_PER_OP, PATH_PERSISTENT = 0, 1, 2
 MAX_DEV = 11
 (PROF_QKV, PROF_ATTENTION, PROF_OPROJ, PROF_GATEUP, PROF_DOWN, PROF_LM_HEAD, PROF_ENSEMBLE, PROF_VERIFY,
- PROF_UPDATE) = range(9)
+ PROF_UPDATE, PROF_DRAFT_ROUND) = range(10)
 
 EXPORTS = [
     "tabed_init", "tabed_destroy", "tabed_strerror", "tabed_load_prefix_kv", "tabed_prefill_tokens",
@@ -32,6 +33,7 @@ EXPORTS = [
     "tabed_draft_round", "tabed_draft_round_logits", "tabed_verify", "tabed_update_weights",
     "tabed_round_host", "tabed_debug_view", "tabed_debug_override_logits", "tabed_state_export", "tabed_state_import",
     "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end", "tabed_ensemble_step_static",
+    "tabed_select_path", "tabed_current_path", "tabed_debug_trace",
 ]
 
 
@@ -97,6 +99,9 @@ def lib() -> C.CDLL:
         L.tabed_profile_begin.argtypes = [vp, i32]
         L.tabed_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.tabed_ensemble_step_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.tabed_select_path.argtypes = [vp, i32]
+        L.tabed_current_path.argtypes = [vp]
+        L.tabed_debug_trace.argtypes = [vp, i32]
         L.tabed_launch_count.argtypes = [vp]
         L.tabed_launch_count.restype = C.c_int64
         for name in EXPORTS:
@@ -267,7 +272,8 @@ class Tabed:
             VIEW_QK: ((B, G, m, V), "<f4"), VIEW_Q: ((B, G, V), "<f4"), VIEW_P: ((B, G + 1, V), "<f4"),
             VIEW_LOGITS: ((G, B, m, V), "<f4"), VIEW_KV_LEN: ((R,), "<i4"), VIEW_WEIGHTS: ((B, m), "<f4"),
             VIEW_WINDOW_SUM: ((B, MAX_DEV), "<i8"), VIEW_PENDING: ((B, 3), "<i4"), VIEW_GRID_J: ((B,), "<i4"),
-            VIEW_ERROR_FLAG: ((1,), "<i4")}[what]
+            VIEW_ERROR_FLAG: ((1,), "<i4"),
+            VIEW_TRACE: ((G, 5 * (self.drafter.n_layers if self.drafter is not None else 0) + 8), "<u8")}[what]
         return torch.as_tensor(_DeviceView(ptr.value, shape, ts), device=self.device)
 
     def debug_override_logits(self, drafter_logits: Optional[torch.Tensor]) -> None:
@@ -294,6 +300,18 @@ class Tabed:
         ms, n = C.c_double(), C.c_int64()
         _check(lib().tabed_profile_end(self._h, C.byref(ms), C.byref(n)), "tabed_profile_end")
         return ms.value, n.value
+
+    def select_path(self, path: int) -> None:
+        _check(lib().tabed_select_path(self._h, path), "tabed_select_path")
+
+    def current_path(self) -> int:
+        rc = lib().tabed_current_path(self._h)
+        if rc < 0:
+            raise TabedError(rc, "tabed_current_path")
+        return rc
+
+    def debug_trace(self, on: bool) -> None:
+        _check(lib().tabed_debug_trace(self._h, 1 if on else 0), "tabed_debug_trace")
 
     def launch_count(self) -> int:
         return int(lib().tabed_launch_count(self._h))

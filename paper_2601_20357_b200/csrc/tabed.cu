@@ -16,6 +16,7 @@
 #include "exact_math.cuh"
 #include "forward_kernels.cuh"
 #include "decide_kernels.cuh"
+#include "round_kernel.cuh"
 
 using namespace tabed;
 
@@ -68,6 +69,17 @@ struct tabed_handle {
   const float* logits_override = nullptr;   // tabed_debug_override_logits
   std::vector<int> len_ub;          // upper bound of every row's committed length
   int64_t launches = 0;
+  // persistent drafting-round kernel (bf16 drafters with at most kPSlots slots per step)
+  bool persist_ok = false;
+  int path_sel = 0;                 // 0 auto, 1 per-operation kernels, 2 persistent kernel
+  RoundArgs ra{};                   // everything that does not change between rounds
+  int n_cta = 0; size_t persist_smem = 0;
+  unsigned launches_persist = 0;
+  LayerW* layer_tab = nullptr;
+  float *xa = nullptr, *x1 = nullptr, *pq = nullptr, *po = nullptr, *pd = nullptr;
+  int* tickets = nullptr; unsigned* bar = nullptr;
+  uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
+  unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false;
   // per-kernel-class timing (tabed_profile_begin / tabed_profile_end)
   int prof_class = -1;
   std::vector<cudaEvent_t> prof_events;     // start/stop pairs
@@ -262,6 +274,111 @@ void run_ensemble(tabed_handle* h, const float* logits, const float* w, const fl
   TABED_LAUNCH(h, k_select<0>, h->B, kDecThreads, 0, s);
 }
 
+// ---- persistent drafting-round kernel: geometry and set-up -----------------------------------------
+// Split a [16*n_tiles][K] weight matrix into units of 16 rows x kchunk columns so that the busiest
+// CTA has as little to do as possible: cost = units per CTA x (columns per unit + fixed overhead).
+PhaseGeom pick_geom(int n_tiles, int K, int n_cta, int kcap, bool whole_rows) {
+  PhaseGeom best{n_tiles, 0, 0, 0};
+  long best_cost = -1;
+  const int nkb = K / 16;
+  for (int ks = 1; ks <= 16; ++ks) {
+    if (nkb % ks) continue;
+    const int kchunk = K / ks;
+    if (kchunk > kcap) continue;
+    if (whole_rows && ks != 1) break;
+    const long units = (long)n_tiles * ks;
+    const long cost = ((units + n_cta - 1) / n_cta) * (kchunk + 128);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = PhaseGeom{n_tiles, ks, kchunk, (int)units}; }
+  }
+  return best;
+}
+
+// Decides whether the handle's drafter can run on the persistent kernel and allocates its buffers.
+int setup_persistent(tabed_handle* h) {
+  const tabed_config& c = h->cfg;
+  h->persist_ok = false;
+  if (c.dtype != TABED_DTYPE_BF16) return TABED_OK;
+  const int grp = h->H / h->Hkv;
+  if (2 * h->R > kPSlots || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
+      grp > kMaxGroup || grp * h->hd > 512 || h->L > 1024)
+    return TABED_OK;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return TABED_ERR_CUDA;
+  if (!prop.cooperativeLaunch) return TABED_OK;
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, k_draft_round) != cudaSuccess) return TABED_ERR_CUDA;
+  const int n_cta = prop.multiProcessorCount;
+  RoundArgs& A = h->ra;
+  const int kcap = std::max(h->d, 1024);
+  A.geom[KIND_QKV] = pick_geom(h->qkv_w / 16, h->d, n_cta, kcap, false);
+  A.geom[KIND_O] = pick_geom(h->d / 16, h->H * h->hd, n_cta, kcap, false);
+  A.geom[KIND_GU] = pick_geom(h->F / 8, h->d, n_cta, kcap, true);
+  A.geom[KIND_DN] = pick_geom(h->d / 16, h->F, n_cta, kcap, false);
+  A.geom[KIND_LM] = pick_geom((h->V + 15) / 16, h->d, n_cta, kcap, true);
+  int kmax = 0;
+  for (int k = 0; k < 5; ++k) { if (A.geom[k].KS == 0) return TABED_OK; kmax = std::max(kmax, A.geom[k].kchunk); }
+  A.slot_bytes = 16 * (kmax * 2 + 16);
+  A.act_bytes = ((kPSlots * (kmax + 8) * 2) + 127) / 128 * 128;
+  const size_t u_bytes = std::max<size_t>((size_t)A.act_bytes + 2 * kPW * 128 * sizeof(float), (size_t)kPW * 512 * sizeof(float));
+  const size_t avail = (size_t)prop.sharedMemPerBlockOptin - fa.sharedSizeBytes - 1024;
+  if (avail < u_bytes + 2 * (size_t)A.slot_bytes) return TABED_OK;
+  A.n_ring = (int)std::min<size_t>(kPRing, (avail - u_bytes) / A.slot_bytes);
+  h->persist_smem = (size_t)A.n_ring * A.slot_bytes + u_bytes;
+  if (cudaFuncSetAttribute(k_draft_round, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_draft_round, kPT, h->persist_smem) != cudaSuccess) return TABED_ERR_CUDA;
+  if (per_sm < 1) return TABED_OK;
+  h->n_cta = n_cta;
+
+  int rc = TABED_OK;
+  auto A2 = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count); };
+  const size_t d = h->d;
+  A2(&h->layer_tab, (size_t)h->L); A2(&h->xa, kPSlots * d); A2(&h->x1, kPSlots * d);
+  A2(&h->pq, (size_t)A.geom[KIND_QKV].KS * kPSlots * h->qkv_w); A2(&h->po, (size_t)A.geom[KIND_O].KS * kPSlots * d);
+  A2(&h->pd, (size_t)A.geom[KIND_DN].KS * kPSlots * d);
+  A2(&h->tickets, (size_t)kPSlots * h->Hkv); A2(&h->bar, 2);
+  A2(&h->rowmax_g, (size_t)h->G * h->R); A2(&h->rowsum_g, (size_t)h->G * h->R);
+  h->trace_stride = 5 * h->L + 8;
+  A2(&h->trace, (size_t)h->G * h->trace_stride);
+  if (rc != TABED_OK) return rc;
+  std::vector<LayerW> tab(h->L);
+  using bf = __nv_bfloat16;
+  for (int l = 0; l < h->L; ++l)
+    tab[l] = LayerW{(const bf*)h->wq[l], (const bf*)h->wk[l], (const bf*)h->wv[l], (const bf*)h->wo[l], (const bf*)h->w_gate[l],
+                    (const bf*)h->w_up[l], (const bf*)h->w_down[l], (const bf*)h->norm1[l], (const bf*)h->norm2[l]};
+  if (cudaMemcpyAsync(h->layer_tab, tab.data(), tab.size() * sizeof(LayerW), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  A.layers = h->layer_tab; A.embed = (const bf*)h->embed; A.lm_head = (const bf*)h->lm_head; A.final_norm = (const bf*)h->final_norm;
+  A.rope_cos = h->rope_cos; A.rope_sin = h->rope_sin;
+  A.L = h->L; A.d = h->d; A.F = h->F; A.H = h->H; A.Hkv = h->Hkv; A.hd = h->hd; A.V = h->V; A.cap = h->cap; A.qkv_w = h->qkv_w;
+  A.eps = c.rms_eps; A.attn_scale = 1.0f / sqrtf((float)h->hd);
+  A.R = h->R; A.B = h->B; A.m = h->m; A.G = h->G; A.greedy = c.sample_mode == TABED_MODE_GREEDY;
+  A.kv_len = h->kv_len; A.pending = h->pending; A.kc = (bf*)h->kc; A.vc = (bf*)h->vc;
+  A.xa = h->xa; A.x1 = h->x1; A.pq = h->pq; A.po = h->po; A.pd = h->pd; A.mid = h->mid; A.attn_out = h->attn_out;
+  A.part_o = h->part_o; A.part_ml = h->part_ml; A.max_splits = h->max_splits; A.tickets = h->tickets;
+  A.logits_own = h->logits_own; A.w = h->w; A.qk = h->qk; A.q = h->q;
+  A.rowmax = h->rowmax_g; A.rowsum = h->rowsum_g; A.chunk_mass = h->chunk_mass; A.chunk_best = h->chunk_best;
+  A.n_chunks = h->n_chunks; A.tokens = h->tokens; A.bar = h->bar; A.err = h->err; A.trace_stride = h->trace_stride;
+  h->persist_ok = true;
+  return TABED_OK;
+}
+
+int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_tokens, int max_pos) {
+  RoundArgs A = h->ra;
+  A.u = u_draft; A.out_tokens = out_tokens; A.logits_override = h->logits_override;
+  A.split_len = (max_pos > 2048) ? 256 : 128;
+  A.bar_sel = (int)(h->launches_persist & 1u);
+  A.trace = h->trace_on ? h->trace : nullptr;
+  void* args[] = {&A};
+  if (cudaLaunchCooperativeKernel((const void*)k_draft_round, dim3(h->n_cta), dim3(kPT), args, h->persist_smem, h->stream) != cudaSuccess)
+    return TABED_ERR_CUDA;
+  h->launches_persist++;
+  h->launches++;
+  return TABED_OK;
+}
+
 int check_cuda() { return cudaGetLastError() == cudaSuccess ? TABED_OK : TABED_ERR_CUDA; }
 
 int max_len_ub(const tabed_handle* h) {
@@ -383,6 +500,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
         rc = TABED_ERR_CUDA;
     }
     h->len_ub.assign(R, 0);
+    if (rc == TABED_OK) rc = setup_persistent(h);
   }
   if (rc == TABED_OK) {
     // equal weights before any history; one pending slot per request; grid j* undefined
@@ -505,6 +623,19 @@ static int draft_common(tabed_handle* h, const float* ext_logits, const float* u
   if (fwd && max_len_ub(h) + 2 + h->G - 1 > h->cap) return TABED_ERR_KV_OVERFLOW;
   DeviceGuard guard(h->cfg.device);
   const long long RV = (long long)h->R * h->V, GV = (long long)h->G * h->V;
+  if (fwd && h->persist_ok && h->path_sel != 1) {
+    // the whole round (gamma decoder steps, each with its ensemble + draw) in one cooperative launch
+    {
+      ProfScope ps(h, TABED_PROF_DRAFT_ROUND);
+      const int rc = launch_persistent_round(h, u_draft, out_tokens, max_len_ub(h) + 2 + h->G - 1);
+      if (rc != TABED_OK) { cudaGetLastError(); return rc; }
+    }
+    if (out_q && cudaMemcpyAsync(out_q, h->q, sizeof(float) * h->B * GV, cudaMemcpyDeviceToDevice, h->stream) != cudaSuccess)
+      return TABED_ERR_CUDA;
+    h->phase = PH_DRAFTED;
+    h->round_has_forward = true;
+    return check_cuda();
+  }
   for (int i = 0; i < h->G; ++i) {
     const float* lg;
     if (fwd) {
@@ -621,7 +752,7 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
 
 int tabed_profile_begin(tabed_handle* h, int32_t kernel_class) {
   if (!h) return TABED_ERR_NULL_PTR;
-  if (kernel_class < 0 || kernel_class > TABED_PROF_UPDATE) return TABED_ERR_INVALID_ARG;
+  if (kernel_class < 0 || kernel_class > TABED_PROF_DRAFT_ROUND) return TABED_ERR_INVALID_ARG;
   h->prof_class = kernel_class;
   h->prof_used = 0;
   return TABED_OK;
@@ -651,6 +782,27 @@ int tabed_debug_override_logits(tabed_handle* h, const float* drafter_logits) {
   return TABED_OK;
 }
 
+int tabed_select_path(tabed_handle* h, int32_t path) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (path < TABED_PATH_AUTO || path > TABED_PATH_PERSISTENT) return TABED_ERR_INVALID_ARG;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  if (path == TABED_PATH_PERSISTENT && !h->persist_ok) return TABED_ERR_UNSUPPORTED;
+  h->path_sel = path;
+  return TABED_OK;
+}
+
+int tabed_current_path(const tabed_handle* h) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  return (h->persist_ok && h->path_sel != TABED_PATH_PER_OP) ? TABED_PATH_PERSISTENT : TABED_PATH_PER_OP;
+}
+
+int tabed_debug_trace(tabed_handle* h, int32_t on) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (!h->persist_ok) return TABED_ERR_UNSUPPORTED;
+  h->trace_on = on != 0;
+  return TABED_OK;
+}
+
 int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* bytes) {
   if (!h || !dev_ptr || !bytes) return TABED_ERR_NULL_PTR;
   const size_t B = h->B, m = h->m, G = h->G, V = h->V, R = h->R;
@@ -665,6 +817,9 @@ int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* byte
     case TABED_VIEW_PENDING: *dev_ptr = h->pending; *bytes = B * 3 * 4; break;
     case TABED_VIEW_GRID_J: *dev_ptr = h->grid_j; *bytes = B * 4; break;
     case TABED_VIEW_ERROR_FLAG: *dev_ptr = h->err; *bytes = 4; break;
+    case TABED_VIEW_TRACE:
+      if (!h->persist_ok) return TABED_ERR_BAD_STATE;
+      *dev_ptr = h->trace; *bytes = (size_t)h->G * h->trace_stride * 8; break;
     default: return TABED_ERR_INVALID_ARG;
   }
   return TABED_OK;
