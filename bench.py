@@ -200,7 +200,7 @@ def class_bytes(wl, kv_tokens_total, mean_accept):
     R, B, m, G, V, d, F = wl.n_rows, wl.n_requests, wl.n_inputs, wl.gamma, c.vocab, c.d_model, c.d_ffn
     kvd = c.n_kv_heads * c.head_dim
     valid = min(mean_accept, G - 1) + 1
-    return {
+    cb = {
         "qkv": (d * d + 2 * kvd * d) * e + R * d * 4 + R * (d + 2 * kvd) * 4,
         "attention": kv_tokens_total * 2 * kvd * e + R * (d + 2 * kvd) * 4 + R * d * 4,
         "oproj": d * d * e + 2 * R * d * 4,
@@ -211,6 +211,10 @@ def class_bytes(wl, kv_tokens_total, mean_accept):
         "verify": (G + 1) * B * V * 4 * 2 + G * B * V * 4,
         "update": valid * (m + 1) * B * V * 4,
     }
+    # the persistent kernel runs the whole drafting round: gamma x (all layers + LM head + ensemble)
+    cb["draft_round"] = G * (c.n_layers * (cb["qkv"] + cb["attention"] + cb["oproj"] + cb["gateup"] + cb["down"])
+                             + cb["lm_head"] + cb["ensemble"])
+    return cb
 
 
 def run_ours(args, wl):
@@ -234,6 +238,8 @@ def run_ours(args, wl):
         if need > wl.kv_capacity:
             wl = wl.replace(kv_capacity=need)
     g = gpu_setup(wl, device)
+    if args.path == "per-op":
+        g.select_path(TB.PATH_PER_OP)
     snap = g.state_export()
     alpha = torch.from_numpy(W.request_alpha(wl)).to(device)
     gen = torch.Generator(device=device)
@@ -290,7 +296,10 @@ def run_ours(args, wl):
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = g.launch_count()
-    g.profile_begin(TB.PROF_LM_HEAD)
+    persistent = g.current_path() == TB.PATH_PERSISTENT
+    top_cls, top_name, top_kernel = ((TB.PROF_DRAFT_ROUND, "draft_round", "k_draft_round (persistent: gamma decoder steps + ensemble)")
+                                     if persistent else (TB.PROF_LM_HEAD, "lm_head", "k_gemv (LM head)"))
+    g.profile_begin(top_cls)
     wall0 = time.perf_counter()
     for i in range(K):
         flush.zero_()                       # the target model's pass between rounds evicts L2 in deployment
@@ -316,14 +325,16 @@ def run_ours(args, wl):
     peak, peak_kind = read_peaks()
     cb = class_bytes(wl, kv_tokens_total, mean_accept)
     head_dur = head_ms / max(head_n, 1)
-    head_gbs = cb["lm_head"] / (head_dur * 1e-3) / 1e9
+    head_gbs = cb[top_name] / (head_dur * 1e-3) / 1e9
 
     # ---- per-class breakdown (separate untimed-for-the-headline passes over the same rounds) ----
     kernels = {}
     if rank == 0 and not args.no_breakdown:
-        names = ["qkv", "attention", "oproj", "gateup", "down", "lm_head", "ensemble", "verify", "update"]
+        names = ["qkv", "attention", "oproj", "gateup", "down", "lm_head", "ensemble", "verify", "update", "draft_round"]
         nb = min(K, 12)
         for cls, nm in enumerate(names):
+            if (nm == "draft_round") != persistent and nm not in ("verify", "update"):
+                continue
             g.state_import(snap)
             for r in range(Wm):
                 one_round(r)
@@ -362,6 +373,34 @@ def run_ours(args, wl):
         e2e = {"value": B * ne / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "steps": ne, "note": "tabed_round_host, pinned host buffers, L2 not flushed between rounds"}
 
+    if rank == 0 and args.trace and persistent:
+        g.state_import(snap)
+        for r in range(Wm):
+            one_round(r)
+        g.debug_trace(True)
+        flush.zero_()
+        g.draft_round(u[Wm][0], toks)
+        torch.cuda.synchronize(device)
+        g.debug_trace(False)
+        tr = g.debug_view(TB.VIEW_TRACE).cpu().numpy().astype(np.int64)
+        g.verify(targets[Wm], u[Wm][1], u[Wm][2], a, z)
+        g.update_weights(w, am)
+        L = wl.drafter.n_layers
+        nb_step = 7 * L + 3
+        names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "res1", "gateup", "down", "res2")] + ["lm_head", "expsum", "mix"]
+        mhz = float(clocks.get("sm_mhz") or 1965.0)
+        with open(args.trace, "w") as f:
+            f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA 0): us from the previous grid barrier to this one,\n"
+                    f"# then CTA 0's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue, epilogue/other, barrier\n")
+            prev = None
+            for st in range(G):
+                for j in range(nb_step):
+                    tcur = int(tr[st, j, 0])
+                    secs = " ".join(f"{int(c) / mhz:7.2f}" for c in tr[st, j, 1:7])
+                    f.write(f"step {st} {names_b[j]:>12s} {((tcur - prev) / 1000.0 if prev is not None else 0.0):8.2f}   {secs}\n")
+                    prev = tcur
+            f.write(f"# first barrier to last barrier: {(int(tr[G - 1, nb_step - 1, 0]) - int(tr[0, 0, 0])) / 1000.0:.1f} us\n")
+
     if rank != 0:
         return
     cpu = None
@@ -378,16 +417,15 @@ def run_ours(args, wl):
         "config": {"workload": wl.name, "n_inputs": m, "n_requests": B, "rows": wl.n_rows, "gamma": G,
                    "window_h": wl.window_h, "vocab": V, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model,
                    "l2": "256 MB written between rounds (stands for the target model's pass); rounds timed one by one "
-                         "with CUDA events", "parallelism": f"replicas x{world}"},
+                         "with CUDA events", "parallelism": f"replicas x{world}",
+                   "path": "persistent" if persistent else "per-operation"},
         "drafted_tokens_per_sec": value * G,
         "block_efficiency": mean_accept + 1.0,
         "wall_ms_per_step_incl_flush": 1000.0 * wall / K,
-        "roofline": {"kernel": "k_gemv (LM head)", "bound": "hbm", "achieved": head_gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": top_kernel, "bound": "hbm", "achieved": head_gbs, "peak": peak, "unit": "GB/s",
                      "frac": head_gbs / peak, "peak_kind": peak_kind, "traffic": None,
-                     "avg_us": 1000.0 * head_dur, "launches_timed": head_n, "bytes_per_launch": int(cb["lm_head"])},
-        "round_roofline": {"bytes_per_round": int(G * (sum(cb[k] for k in ("qkv", "attention", "oproj", "gateup", "down"))
-                                                     * wl.drafter.n_layers + cb["lm_head"] + cb["ensemble"])
-                                                 + cb["verify"] + cb["update"]),
+                     "avg_us": 1000.0 * head_dur, "launches_timed": head_n, "bytes_per_launch": int(cb[top_name])},
+        "round_roofline": {"bytes_per_round": int(cb["draft_round"] + cb["verify"] + cb["update"]),
                            "note": "algorithmic bytes of one round / measured round time / peak"},
         "kernels": kernels,
         "cpu_baseline": cpu,
@@ -416,6 +454,8 @@ def main():
     ap.add_argument("--cpu-rounds", type=int, default=60)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
+    ap.add_argument("--trace", default=None, help="write the persistent kernel's phase timeline of one round to this file")
+    ap.add_argument("--path", default="auto", choices=["auto", "per-op"], help="drafting path (per-op forces one kernel per operation)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -75,8 +75,8 @@ extern "C" {
 #define TABED_VIEW_PENDING     7   /* int32  [B][3]        {count, token0, token1}                     */
 #define TABED_VIEW_GRID_J      8   /* int32  [B]           j* of the grid policy (-1 before any update)*/
 #define TABED_VIEW_ERROR_FLAG  9   /* int32  [1]           non-zero if a device-side check failed      */
-#define TABED_VIEW_TRACE      10   /* uint64 [G][5L+8]     nanosecond timer after each grid barrier of the
-                                                           persistent drafting kernel (tabed_debug_trace)  */
+#define TABED_VIEW_TRACE      10   /* uint64 [G][7L+8][8]  phase timeline of the persistent drafting kernel
+                                                           (tabed_debug_trace): one record per grid barrier */
 
 /* How tabed_draft_round runs Algorithm 1 (tabed_select_path).  Results obey the same contract on
  * both paths: identical integer decisions for identical logits; logits agree within the forward
@@ -85,7 +85,7 @@ extern "C" {
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
 #define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, 2*B*m <= 8
                                       slots, d_model <= 2048 and a multiple of 16, d_ffn a multiple of 16,
-                                      (H/Hkv)*head_dim <= 512                                            */
+                                      (H/Hkv)*head_dim <= 512, <= 64 layers, kv_capacity <= 32768        */
 
 typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
 
@@ -204,10 +204,15 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
 int tabed_select_path(tabed_handle* h, int32_t path);
 int tabed_current_path(const tabed_handle* h);
 
-/* Switch the phase timeline of the persistent kernel on or off: when on, CTA 0 stores the GPU's
- * nanosecond timer after every grid barrier into TABED_VIEW_TRACE (row = drafting step).  Barrier
- * order within a step: per layer QKV, attention, O, gate/up, down; then LM head, [2 more when
- * tabed_debug_override_logits is set], exp-sum, mix.  Errors: UNSUPPORTED (no persistent path). */
+/* Switch the phase timeline of the persistent kernel on or off: when on, CTA 0 stores one record of
+ * 8 words per grid barrier into TABED_VIEW_TRACE (first index = drafting step): [0] the GPU's
+ * nanosecond timer after the barrier; [1..6] SM clock cycles that CTA 0 spent since the previous
+ * barrier resolving and staging activations, waiting for weight tiles, in the tensor-core products,
+ * issuing weight copies, in epilogues (or, for the phases without weights, in all of the phase), and
+ * in the barrier itself; [7] unused.  Barrier order within a step: per layer QKV, attention, O,
+ * resolve, gate/up, down, resolve; then LM head, [2 more when tabed_debug_override_logits is set],
+ * exp-sum, mix.
+ * Errors: UNSUPPORTED (no persistent path). */
 int tabed_debug_trace(tabed_handle* h, int32_t on);
 
 /* Pointer and size of a library-owned device buffer (TABED_VIEW_*).  Read-only for the caller. */

@@ -11,6 +11,14 @@
 //     HBM stays busy across the grid barriers;
 //   * a phase is: grid barrier -> stage the (tiny) activations from L2 -> tensor-core products
 //     of the 16-row weight tiles already sitting in shared memory -> results back to L2;
+//   * the critical path is the chain of phases, so every phase is built to cost one L2 round trip
+//     plus the barrier: split-K partial sums are reduced once, slice by slice, in a short
+//     "resolve" phase of their own (not 148 times by every consumer), a CTA issues all loads of an
+//     attention item (K, V, q) before it uses any;
+//   * the weights are read from a private copy laid out for this kernel at set-up: every unit (16
+//     rows x kchunk columns, rows already padded to the bank-conflict-free shared-memory pitch) is
+//     one contiguous block, so a unit is ONE bulk copy (16 per-row copies cost ~1 us of issue time
+//     per unit on the critical path);
 //   * projections use mma.sync m16n8k16 (bf16 x bf16 -> fp32): 16 weight rows x up to 8 slots.
 //     The contraction is HBM-bound (<= 8 flop per weight byte), the tensor pipe is used only to
 //     keep the ALUs off the critical path;
@@ -36,6 +44,9 @@ constexpr int kPRing = 16;               // upper bound of ring slots
 constexpr int kPPer = kChunk / kPT;      // vocabulary elements per thread and chunk (4)
 constexpr int kPMaxD = 2048;             // d_model bound (4 residual elements per thread and slot)
 constexpr int kPXE = kPMaxD / kPT;
+constexpr int kTraceRec = 8;             // words per record of the phase timeline
+constexpr int kPMaxL = 64;               // layers (their pointer table lives in shared memory)
+constexpr int kResW = 16;                // upper bound of a CTA's slice of d_model in a resolve phase
 
 enum { KIND_QKV = 0, KIND_O = 1, KIND_GU = 2, KIND_DN = 3, KIND_LM = 4 };
 enum { PERR_BARRIER = 8, PERR_COPY = 16, PERR_KV = 4 };
@@ -54,6 +65,9 @@ struct RoundArgs {
   int L, d, F, H, Hkv, hd, V, cap, qkv_w;
   float eps, attn_scale;
   PhaseGeom geom[5];
+  const unsigned char* packed;          // weights re-laid out unit by unit (k_pack_units)
+  unsigned long long pack_off[5];       // byte offset of a kind's units inside a layer block (LM: absolute)
+  unsigned long long pack_layer_stride;
   int slot_bytes, n_ring, act_bytes, split_len;
   // round
   int R, B, m, G, greedy;
@@ -62,6 +76,7 @@ struct RoundArgs {
   __nv_bfloat16 *kc, *vc;               // [R][L][Hkv][cap][hd]
   // activations exchanged through L2
   float *xa, *x1;                       // [8][d] residual before / after the attention block
+  float* ssq;                           // [n_cta][8] per-CTA partial sums of squares of the last resolve
   float *pq, *po, *pd;                  // split-K partial sums [KS][8][width]
   float *mid, *attn_out;                // [8][F], [8][H*hd]
   float *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2]
@@ -83,7 +98,7 @@ struct RoundArgs {
   unsigned* bar;                        // [2] grid barrier counters, used alternately by launches
   int bar_sel;
   int* err;
-  unsigned long long* trace;            // optional [G][trace_stride] globaltimer after each barrier
+  unsigned long long* trace;            // optional [G][trace_stride][kTraceRec] phase timeline
   int trace_stride;
 };
 
@@ -144,13 +159,16 @@ struct PSlot { int row, pos, active, tok; };
 
 struct PShared {
   uint64_t full[kPRing];
+  LayerW layers[kPMaxL];
   float sc[kMaxGroup][kAttnSplitMax];
   float q[kMaxGroup][128];
   float kf[2][128], vf[2][128];
   float red[kPW][kPSlots];
   unsigned long long red64[kPW];
+  unsigned long long cm[kPT];
   float bestv[kPW]; int besti[kPW];
   float scale[kPSlots];
+  float mix_mx[kMaxInputs], mix_sn[kMaxInputs], mix_w[kMaxInputs];
   float m_[kMaxGroup], l_[kMaxGroup];
   PSlot slot[kPSlots];
   int lm_src[kPSlots];
@@ -182,35 +200,46 @@ __device__ __forceinline__ bool next_unit(const RoundArgs& A, int cta, int NC, U
   return false;
 }
 
-// Issue the bulk copies of one unit into a ring slot (called by all lanes of warp 0).
-__device__ __forceinline__ void issue_unit(const RoundArgs& A, const UnitRef& ur, unsigned char* slot_base,
-                                           uint64_t* bar, int lane) {
-  const PhaseGeom g = A.geom[ur.kind];
-  const int ks = ur.u / g.n_tiles, tile = ur.u - ks * g.n_tiles;
-  const unsigned row_bytes = (unsigned)g.kchunk * 2u;
-  if (lane == 0) mbar_expect_tx(bar, row_bytes * 16u);
-  __syncwarp();
-  if (lane < 16) {
-    const LayerW* lw = A.layers + ur.layer;
-    const __nv_bfloat16* base;
-    int row, K;
-    if (ur.kind == KIND_QKV) {
-      K = A.d; row = tile * 16 + lane;
-      const int kvd = A.Hkv * A.hd;
-      if (row < A.d) base = lw->wq;
-      else if (row < A.d + kvd) { base = lw->wk; row -= A.d; }
-      else { base = lw->wv; row -= A.d + kvd; }
-    } else if (ur.kind == KIND_O) {
-      K = A.H * A.hd; row = tile * 16 + lane; base = lw->wo;
-    } else if (ur.kind == KIND_GU) {            // rows 0-7: gate rows, rows 8-15: the matching up rows
-      K = A.d; row = tile * 8 + (lane & 7); base = (lane < 8) ? lw->wg : lw->wu;
-    } else if (ur.kind == KIND_DN) {
-      K = A.F; row = tile * 16 + lane; base = lw->wd;
-    } else {
-      K = A.d; row = min(tile * 16 + lane, A.V - 1); base = A.lm_head;
+// Issue the bulk copy of one unit into a ring slot (one thread).
+__device__ __forceinline__ void issue_unit(const RoundArgs& A, const UnitRef& ur, unsigned char* slot_base, uint64_t* bar) {
+  const unsigned bytes = 16u * ((unsigned)A.geom[ur.kind].kchunk * 2u + 16u);
+  const unsigned char* src = A.packed + A.pack_off[ur.kind] + (size_t)ur.u * bytes +
+                             (ur.kind == KIND_LM ? 0ull : (unsigned long long)ur.layer * A.pack_layer_stride);
+  mbar_expect_tx(bar, bytes);
+  bulk_g2s(slot_base, src, bytes, bar);
+}
+
+// Re-lay one weight matrix (or the QKV / gate-up group) of one layer into units.  grid (n_units), block 256.
+// Row r of unit (ks, tile): QKV rows are the concatenation wq | wk | wv; gate/up units hold 8 gate
+// rows then the 8 matching up rows; LM-head rows beyond V are zero.
+struct PackArgs {
+  const __nv_bfloat16 *w0, *w1, *w2;    // source matrices [rows_i][K]
+  int rows0, rows1, rows2, K, kind;
+  PhaseGeom g;
+  unsigned char* dst;                   // first unit of this (layer, kind)
+};
+__global__ void k_pack_units(const PackArgs P) {
+  const int u = blockIdx.x;
+  const int ks = u / P.g.n_tiles, tile = u - ks * P.g.n_tiles;
+  const int pitch = P.g.kchunk * 2 + 16;
+  unsigned char* unit = P.dst + (size_t)u * 16 * pitch;
+  const int vec_per_row = pitch / 16;                      // 16-byte vectors per padded row
+  for (int idx = threadIdx.x; idx < 16 * vec_per_row; idx += blockDim.x) {
+    const int r = idx / vec_per_row, c16 = idx - r * vec_per_row;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (c16 * 8 < P.g.kchunk) {
+      const __nv_bfloat16* base = nullptr;
+      int row;
+      if (P.kind == KIND_GU) { row = tile * 8 + (r & 7); base = (r < 8) ? P.w0 : P.w1; if (row >= P.rows0) base = nullptr; }
+      else {
+        row = tile * 16 + r;
+        if (row < P.rows0) base = P.w0;
+        else if (row < P.rows0 + P.rows1) { base = P.w1; row -= P.rows0; }
+        else if (row < P.rows0 + P.rows1 + P.rows2) { base = P.w2; row -= P.rows0 + P.rows1; }
+      }
+      if (base) v = *reinterpret_cast<const uint4*>(base + (size_t)row * P.K + (size_t)ks * P.g.kchunk + c16 * 8);
     }
-    const __nv_bfloat16* src = base + (size_t)row * K + (size_t)ks * g.kchunk;
-    bulk_g2s(slot_base + (size_t)lane * (row_bytes + 16u), src, row_bytes, bar);
+    *reinterpret_cast<uint4*>(unit + (size_t)r * pitch + (size_t)c16 * 16) = v;
   }
 }
 
@@ -226,10 +255,12 @@ __device__ __forceinline__ bool wait_full(PShared& S, int slot, unsigned parity,
   return true;
 }
 
-// Grid-wide barrier on a monotonically increasing counter.  Returns false if the CTA is dead.
+// Grid-wide barrier on a counter that only grows during a launch.  (One flag per CTA polled by all
+// CTAs in parallel was measured 3-4x slower: 148 x 148 concurrent polls saturate the L2 slice.)
+// Returns false if the wait ran out.
 __device__ __forceinline__ bool grid_barrier(PShared& S, unsigned* bar, unsigned target, int* err) {
   __syncthreads();
-  if (threadIdx.x == 0 && !S.dead) {
+  if (threadIdx.x == 0) {
     __threadfence();
     atomicAdd(bar, 1u);
     unsigned spins = 0;
@@ -277,6 +308,7 @@ __device__ __forceinline__ void store4(float* __restrict__ row, int v0, int V, b
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
+template <bool TRACE>
 __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
   __shared__ PShared S;
@@ -287,9 +319,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(U);               // [8][apitch]
   float* cpart = reinterpret_cast<float*>(U + A.act_bytes);               // [2][kPW][128]
   float* s_o = reinterpret_cast<float*>(U);                               // attention: [kPW][grp*hd]
-  unsigned* bar = A.bar + A.bar_sel;
+  float* rbuf = reinterpret_cast<float*>(U);                              // resolve: [terms][8][kResW]
   const int kvd = A.Hkv * A.hd, HD = A.H * A.hd, grp = A.H / A.Hkv, half = A.hd >> 1;
   const int R = A.R, B = A.B, m = A.m, G = A.G, V = A.V, d = A.d;
+  const int d4 = d >> 2;                                // float4 groups of the residual; thread t owns group t
+  const int lo = (int)((long long)cta * d / NC), hi = (int)((long long)(cta + 1) * d / NC);   // resolve slice
 
   // ---- set-up -----------------------------------------------------------------------------------
   if (tid == 0) {
@@ -298,6 +332,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     S.dead = 0;
   }
+  for (int i = tid; i < A.L * (int)(sizeof(LayerW) / sizeof(void*)); i += kPT)
+    reinterpret_cast<const void**>(S.layers)[i] = reinterpret_cast<const void* const*>(A.layers)[i];
   if (cta == 0) {
     for (int i = tid; i < G * R; i += kPT) { A.rowmax[i] = 0u; A.rowsum[i] = 0ull; }
     for (int i = tid; i < kPSlots * A.Hkv; i += kPT) A.tickets[i] = 0;
@@ -307,25 +343,46 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 
   UnitCursor pc{0, 0, 0, 0};
   unsigned prod_i = 0, cons_i = 0;
-  if (warp == 0) {
+  if (tid == 0) {
     for (int k = 0; k < A.n_ring; ++k) {
       UnitRef ur;
       if (!next_unit(A, cta, NC, pc, ur)) break;
-      issue_unit(A, ur, ring + (size_t)k * A.slot_bytes, &S.full[k], lane);
+      issue_unit(A, ur, ring + (size_t)k * A.slot_bytes, &S.full[k]);
       ++prod_i;
     }
   }
+  unsigned* bar = A.bar + A.bar_sel;
   unsigned bar_target = 0;
   bool alive = true;
 
+  // phase timeline (CTA 0, thread 0): per grid barrier one record of kTraceRec words:
+  // [0] nanosecond timer after the barrier, [1..6] clock cycles spent since the previous barrier in
+  // resolve+stage, waiting for weight tiles, mma+partials, issuing copies, epilogue/other, the barrier
+  const bool tr_on = TRACE && A.trace != nullptr && cta == 0 && tid == 0;
+  long long t_sec[6] = {0, 0, 0, 0, 0, 0};
+  long long t_mark = 0;
+#define TSEC(k)                                       \
+  do {                                                \
+    if (TRACE && tr_on) {                             \
+      const long long t_now = clock64();              \
+      t_sec[k] += t_now - t_mark;                     \
+      t_mark = t_now;                                 \
+    }                                                 \
+  } while (0)
 #define GRID_SYNC()                                                        \
   do {                                                                     \
+    TSEC(4);                                                               \
     bar_target += (unsigned)NC;                                            \
     alive = grid_barrier(S, bar, bar_target, A.err);                       \
-    if (A.trace && cta == 0 && tid == 0 && trace_n < A.trace_stride)       \
-      A.trace[(size_t)step * A.trace_stride + trace_n++] = global_timer(); \
+    TSEC(5);                                                               \
+    if (TRACE && tr_on && trace_n < A.trace_stride) {                      \
+      unsigned long long* rec = A.trace + ((size_t)step * A.trace_stride + trace_n++) * kTraceRec; \
+      rec[0] = global_timer();                                             \
+      for (int k = 0; k < 6; ++k) { rec[1 + k] = (unsigned long long)t_sec[k]; t_sec[k] = 0; }     \
+    }                                                                      \
     if (!alive) goto drain;                                                \
   } while (0)
+  if (tr_on) t_mark = clock64();
 
   for (int step = 0; step < G; ++step) {
     int trace_n = 0;
@@ -363,58 +420,21 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
     for (int phase = 0; phase <= 4 * A.L; ++phase) {
       const int kind = (phase == 4 * A.L) ? KIND_LM : (phase & 3);
       const int layer = phase >> 2;
-      const LayerW* lw = A.layers + (kind == KIND_LM ? 0 : layer);
+      const LayerW& lw = S.layers[kind == KIND_LM ? 0 : layer];
       const PhaseGeom g = A.geom[kind];
       const int apitch = g.kchunk + 8;                       // bf16 elements
       const int n_in = (kind == KIND_LM) ? R : ns;           // activation rows of the phase
+      const bool norm_kind = kind == KIND_QKV || kind == KIND_GU || kind == KIND_LM;
 
-      // ---- resolve the phase input (residual + split-K partials), RMSNorm statistics -------------
-      float xv[kPSlots][kPXE];
-      if (kind == KIND_QKV || kind == KIND_GU || kind == KIND_LM) {
-        const int KSp = (kind == KIND_GU) ? A.geom[KIND_O].KS : A.geom[KIND_DN].KS;
-        const float* part = (kind == KIND_GU) ? A.po : A.pd;
-        const float* basebuf = (kind == KIND_GU) ? A.xa : A.x1;
-        float* outbuf = (kind == KIND_QKV) ? A.xa : (kind == KIND_GU ? A.x1 : nullptr);
-        const int lo = (int)((long long)cta * d / NC), hi = (int)((long long)(cta + 1) * d / NC);
-        float ss[kPSlots];
-#pragma unroll
-        for (int s = 0; s < kPSlots; ++s) {
-          ss[s] = 0.0f;
-          if (s >= n_in) continue;
-          const int src = (kind == KIND_LM) ? S.lm_src[s] : s;
-          const bool act_s = (kind == KIND_LM) ? true : (S.slot[s].active != 0);
-#pragma unroll
-          for (int i = 0; i < kPXE; ++i) {
-            const int e = tid + i * kPT;
-            float v = 0.0f;
-            if (e < d && act_s) {
-              if (kind == KIND_QKV && layer == 0) {
-                v = __bfloat162float(A.embed[(size_t)S.slot[s].tok * d + e]);
-              } else {
-                v = __ldcg(basebuf + (size_t)src * d + e);
-                for (int ks = 0; ks < KSp; ++ks) v += __ldcg(part + ((size_t)ks * kPSlots + src) * d + e);
-              }
-              if (outbuf && e >= lo && e < hi) outbuf[(size_t)s * d + e] = v;
-            }
-            xv[s][i] = v;
-            ss[s] = fmaf(v, v, ss[s]);
-          }
+      if (kind == KIND_QKV && layer == 0) {
+        // the residual entering layer 0 is the embedding itself: publish this CTA's slice of it
+        const int wsl = hi - lo;
+        if (tid < ns * wsl) {
+          const int s = tid / wsl, e = lo + (tid - s * wsl);
+          if (S.slot[s].active) A.xa[(size_t)s * d + e] = __bfloat162float(A.embed[(size_t)S.slot[s].tok * d + e]);
         }
-#pragma unroll
-        for (int s = 0; s < kPSlots; ++s) ss[s] = warp_sum_f32(ss[s]);
-        if (lane == 0) {
-#pragma unroll
-          for (int s = 0; s < kPSlots; ++s) S.red[warp][s] = ss[s];
-        }
-        __syncthreads();
-        if (tid < kPSlots) {
-          float tot = 0.0f;
-#pragma unroll
-          for (int w2 = 0; w2 < kPW; ++w2) tot += S.red[w2][tid];
-          S.scale[tid] = 1.0f / sqrtf(tot / (float)d + A.eps);
-        }
-        __syncthreads();
       }
+      TSEC(0);
 
       // ---- units of this CTA ------------------------------------------------------------------------
       int first = cta - off;
@@ -426,17 +446,64 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         if (ks != cur_ks) {
           // stage the activation chunk [n_in][kchunk] as bf16 (matmul inputs are rounded to bf16)
           const int k0 = ks * g.kchunk;
-          if (kind == KIND_QKV || kind == KIND_GU || kind == KIND_LM) {
-            const __nv_bfloat16* gain = (kind == KIND_QKV) ? lw->n1 : (kind == KIND_GU ? lw->n2 : A.final_norm);
+          if (norm_kind) {
+            // resolved residual (one L2 trip), RMSNorm statistics, normalised chunk -> bf16
+            const bool from_embed = kind == KIND_QKV && layer == 0;
+            const float* xbuf = (kind == KIND_GU) ? A.x1 : A.xa;
+            float4 xv[kPSlots];
+            float ss[kPSlots];
+            const __nv_bfloat16* gain = (kind == KIND_QKV) ? lw.n1 : (kind == KIND_GU ? lw.n2 : A.final_norm);
+            uint2 g2 = make_uint2(0u, 0u);
+            if (tid < d4) g2 = __ldg(reinterpret_cast<const uint2*>(gain) + tid);
 #pragma unroll
             for (int s = 0; s < kPSlots; ++s) {
-              if (s >= n_in) continue;
-              const float sc = S.scale[s];
+              xv[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+              ss[s] = 0.0f;
+              if (s >= n_in || tid >= d4) continue;
+              if (from_embed) {
+                if (S.slot[s].active) {
+                  const uint2 e2 = __ldg(reinterpret_cast<const uint2*>(A.embed + (size_t)S.slot[s].tok * d) + tid);
+                  xv[s] = make_float4(__uint_as_float(e2.x << 16), __uint_as_float(e2.x & 0xFFFF0000u),
+                                      __uint_as_float(e2.y << 16), __uint_as_float(e2.y & 0xFFFF0000u));
+                  ss[s] = fmaf(xv[s].x, xv[s].x, fmaf(xv[s].y, xv[s].y, fmaf(xv[s].z, xv[s].z, xv[s].w * xv[s].w)));
+                }
+              } else {
+                const int src = (kind == KIND_LM) ? S.lm_src[s] : s;
+                if (kind == KIND_LM || S.slot[s].active) xv[s] = __ldcg(reinterpret_cast<const float4*>(xbuf + (size_t)src * d) + tid);
+              }
+            }
+            if (!from_embed && tid < NC) {
+              // partial sums of squares left by the resolve phase, one set per CTA
+              const float4 p0 = __ldcg(reinterpret_cast<const float4*>(A.ssq + (size_t)tid * kPSlots));
+              const float4 p1 = __ldcg(reinterpret_cast<const float4*>(A.ssq + (size_t)tid * kPSlots) + 1);
+              ss[0] = p0.x; ss[1] = p0.y; ss[2] = p0.z; ss[3] = p0.w; ss[4] = p1.x; ss[5] = p1.y; ss[6] = p1.z; ss[7] = p1.w;
+            }
 #pragma unroll
-              for (int i = 0; i < kPXE; ++i) {
-                const int e = tid + i * kPT;
-                if (e >= k0 && e < k0 + g.kchunk && e < d)
-                  act[s * apitch + (e - k0)] = __float2bfloat16_rn(xv[s][i] * sc * __bfloat162float(gain[e]));
+            for (int s = 0; s < kPSlots; ++s) ss[s] = warp_sum_f32(ss[s]);
+            if (lane == 0) {
+#pragma unroll
+              for (int s = 0; s < kPSlots; ++s) S.red[warp][s] = ss[s];
+            }
+            __syncthreads();
+            if (tid < kPSlots) {
+              float tot = 0.0f;
+#pragma unroll
+              for (int w2 = 0; w2 < kPW; ++w2) tot += S.red[w2][tid];
+              S.scale[tid] = 1.0f / sqrtf(tot / (float)d + A.eps);
+            }
+            __syncthreads();
+            const int e0 = tid * 4;
+            if (tid < d4 && e0 >= k0 && e0 < k0 + g.kchunk) {
+              const float g0 = __uint_as_float(g2.x << 16), g1 = __uint_as_float(g2.x & 0xFFFF0000u);
+              const float g2f = __uint_as_float(g2.y << 16), g3 = __uint_as_float(g2.y & 0xFFFF0000u);
+#pragma unroll
+              for (int s = 0; s < kPSlots; ++s) {
+                if (s >= n_in) continue;
+                const float sc = S.scale[(kind == KIND_LM) ? S.lm_src[s] : s];
+                uint2 pk;
+                pk.x = pack_bf16(xv[s].x * sc * g0, xv[s].y * sc * g1);
+                pk.y = pack_bf16(xv[s].z * sc * g2f, xv[s].w * sc * g3);
+                *reinterpret_cast<uint2*>(act + s * apitch + (e0 - k0)) = pk;
               }
             }
           } else {
@@ -453,11 +520,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           cur_ks = ks;
           __syncthreads();
+          TSEC(0);
         }
         const int slot = (int)(cons_i % (unsigned)A.n_ring);
         const unsigned parity = (cons_i / (unsigned)A.n_ring) & 1u;
         const bool landed = wait_full(S, slot, parity, A.err);
         if (__syncthreads_or(!landed)) { alive = false; goto drain; }
+        TSEC(1);
         const unsigned char* tile_s = ring + (size_t)slot * A.slot_bytes;
         const uint32_t tpitch = (uint32_t)g.kchunk * 2u + 16u;
         float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -480,17 +549,19 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           *reinterpret_cast<float2*>(w0 + (gq + 8) * 8 + tq * 2) = make_float2(c[2], c[3]);
         }
         __syncthreads();                        // slot fully read, partial tiles complete
-        if (warp == 0) {                        // refill the slot that was just released
+        TSEC(2);
+        ++cons_i;
+        if (tid == 0) {                         // refill the slot that was just released ...
           UnitRef ur;
           if (next_unit(A, cta, NC, pc, ur)) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue_unit(A, ur, ring + (size_t)slot * A.slot_bytes, &S.full[slot], lane);
+            issue_unit(A, ur, ring + (size_t)slot * A.slot_bytes, &S.full[slot]);
             ++prod_i;
           }
+          TSEC(3);
         }
-        ++cons_i;
-        if (tid < 128) {                        // sum the warps' partial tiles, epilogue
-          const int r = tid & 15, n = tid >> 4;
+        if (warp >= 1 && warp <= 4) {           // ... while warps 1-4 sum the partial tiles and store
+          const int et = tid - 32;
+          const int r = et & 15, n = et >> 4;
           float v = 0.0f;
 #pragma unroll
           for (int w2 = 0; w2 < kPW; ++w2) v += cp[w2 * 128 + r * 8 + n];
@@ -514,14 +585,58 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         }
       }
       off = (off + g.n_units) % NC;
-      if (kind == KIND_LM && tid < 128 && (tid & 15) == 0 && (tid >> 4) < R && lm_max > -INFINITY)
-        atomicMax(A.rowmax + step * R + (tid >> 4), ord_encode(lm_max));
+      if (kind == KIND_LM && warp >= 1 && warp <= 4 && ((tid - 32) & 15) == 0 && ((tid - 32) >> 4) < R && lm_max > -INFINITY)
+        atomicMax(A.rowmax + step * R + ((tid - 32) >> 4), ord_encode(lm_max));
       GRID_SYNC();
+
+      // ---- resolve: residual + split-K partials of the phase just finished, this CTA's slice --------
+      if (kind == KIND_O || kind == KIND_DN) {
+        const float* basebuf = (kind == KIND_O) ? A.xa : A.x1;
+        float* outbuf = (kind == KIND_O) ? A.x1 : A.xa;
+        const float* part = (kind == KIND_O) ? A.po : A.pd;
+        const int wsl = hi - lo, terms = g.KS + 1;
+        // thread -> (term t = tid/128 + 4*it, slot s, element j): all loads of a thread are independent
+        constexpr int kIt = (17 + 3) / 4;
+        const int rs = (tid >> 4) & (kPSlots - 1), rj = tid & (kResW - 1), rt0 = tid >> 7;
+        const bool r_on = rs < ns && rj < wsl && S.slot[rs].active;
+        float val[kIt];
+#pragma unroll
+        for (int it = 0; it < kIt; ++it) {
+          const int t = rt0 + it * 4;
+          val[it] = 0.0f;
+          if (r_on && t < terms)
+            val[it] = (t == 0) ? __ldcg(basebuf + (size_t)rs * d + lo + rj)
+                               : __ldcg(part + ((size_t)(t - 1) * kPSlots + rs) * d + lo + rj);
+        }
+#pragma unroll
+        for (int it = 0; it < kIt; ++it) {
+          const int t = rt0 + it * 4;
+          if (t < terms) rbuf[(t * kPSlots + rs) * kResW + rj] = val[it];
+        }
+        __syncthreads();
+        if (tid < kPSlots * kResW) {
+          const int s = tid / kResW, j = tid - s * kResW;
+          float sq = 0.0f;
+          if (s < ns && j < wsl && S.slot[s].active) {
+            float v = 0.0f;
+            for (int t = 0; t < terms; ++t) v += rbuf[(t * kPSlots + s) * kResW + j];
+            outbuf[(size_t)s * d + lo + j] = v;
+            sq = v * v;
+          }
+#pragma unroll
+          for (int o = kResW / 2; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          if (j == 0) A.ssq[(size_t)cta * kPSlots + s] = sq;
+        }
+        GRID_SYNC();
+      }
 
       // ---- attention over the rows' caches (after the QKV phase) -----------------------------------
       if (kind == KIND_QKV) {
         const int KSq = A.geom[KIND_QKV].KS;
         const int split_len = A.split_len;
+        const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
+        const int PPW = 32 / LPR, PPB = kPW * PPW;     // positions per warp / per CTA pass
+        const int sub = lane % LPR, pgrp = lane / LPR;
         int total_items = 0;
         for (int s = 0; s < ns; ++s)
           if (S.slot[s].active) total_items += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
@@ -539,75 +654,82 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           const int p_lo = split * split_len, p_hi = min(p_lo + split_len, n_pos), cnt = p_hi - p_lo;
           const int second = s >= R;
           const int n_fresh = second ? 2 : 1;          // positions whose K,V are produced in this very phase
-          // stage q (all heads of the group), fresh k and v: split-K sums, RoPE, bf16 rounding
-          for (int idx = tid; idx < grp * half; idx += kPT) {
-            const int t = idx / half, i = idx - t * half;
-            const int col = (gk * grp + t) * A.hd + i;
-            float x1 = 0.0f, x2 = 0.0f;
-            for (int ks = 0; ks < KSq; ++ks) {
-              const float* pr = A.pq + ((size_t)ks * kPSlots + s) * A.qkv_w + col;
-              x1 += __ldcg(pr); x2 += __ldcg(pr + half);
-            }
-            const float cs = A.rope_cos[(size_t)pos * half + i], sn = A.rope_sin[(size_t)pos * half + i];
-            S.q[t][i] = round_bf16(x1 * cs - x2 * sn);
-            S.q[t][i + half] = round_bf16(x2 * cs + x1 * sn);
+          const int fresh_lo = pos - (n_fresh - 1);    // absolute positions >= fresh_lo are fresh
+          const size_t cache_off = ((((size_t)si.row * A.L + layer) * A.Hkv + gk) * A.cap) * A.hd;
+          const __nv_bfloat16* kbase = A.kc + cache_off;
+          const __nv_bfloat16* vbase = A.vc + cache_off;
+          // all cache loads of the item go out first: one memory round trip for K, V and q together
+          uint4 kreg[4], vreg[4];
+#pragma unroll
+          for (int ps = 0; ps < 4; ++ps) {
+            const int p = ps * PPB + warp * PPW + pgrp;
+            kreg[ps] = make_uint4(0u, 0u, 0u, 0u);
+            if (p < cnt && p_lo + p < fresh_lo)
+              kreg[ps] = __ldcg(reinterpret_cast<const uint4*>(kbase + (size_t)(p_lo + p) * A.hd + sub * 8));
           }
-          for (int idx = tid; idx < n_fresh * half; idx += kPT) {
-            const int j = idx / half, i = idx - j * half;
-            const int sj = s - j * R, pj = pos - j;
-            const int col = d + gk * A.hd + i;
-            float x1 = 0.0f, x2 = 0.0f;
-            for (int ks = 0; ks < KSq; ++ks) {
-              const float* pr = A.pq + ((size_t)ks * kPSlots + sj) * A.qkv_w + col;
-              x1 += __ldcg(pr); x2 += __ldcg(pr + half);
-            }
-            const float cs = A.rope_cos[(size_t)pj * half + i], sn = A.rope_sin[(size_t)pj * half + i];
-            S.kf[j][i] = round_bf16(x1 * cs - x2 * sn);
-            S.kf[j][i + half] = round_bf16(x2 * cs + x1 * sn);
+#pragma unroll
+          for (int ps = 0; ps < 4; ++ps) {
+            const int p = ps * PPB + warp * PPW + pgrp;
+            vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
+            if (p < cnt && p_lo + p < fresh_lo)
+              vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(vbase + (size_t)(p_lo + p) * A.hd + sub * 8));
           }
-          for (int idx = tid; idx < n_fresh * A.hd; idx += kPT) {
-            const int j = idx / A.hd, i = idx - j * A.hd;
-            const int sj = s - j * R;
-            float x = 0.0f;
-            for (int ks = 0; ks < KSq; ++ks) x += __ldcg(A.pq + ((size_t)ks * kPSlots + sj) * A.qkv_w + d + kvd + gk * A.hd + i);
-            S.vf[j][i] = round_bf16(x);
+          // stage q (all heads of the group), fresh k and v: split-K sums, RoPE, bf16 rounding.
+          // One index space so that every element is fetched by a different thread in one round trip.
+          {
+            const int n_q = grp * half, n_k = n_fresh * half, n_v = n_fresh * A.hd;
+            for (int idx = tid; idx < n_q + n_k + n_v; idx += kPT) {
+              int sj, col, pj, i;
+              float* dst;
+              bool pair = true;
+              if (idx < n_q) {
+                const int t = idx / half; i = idx - t * half;
+                sj = s; pj = pos; col = (gk * grp + t) * A.hd + i; dst = &S.q[t][i];
+              } else if (idx < n_q + n_k) {
+                const int j = (idx - n_q) / half; i = (idx - n_q) - j * half;
+                sj = s - j * R; pj = pos - j; col = d + gk * A.hd + i; dst = &S.kf[j][i];
+              } else {
+                const int j = (idx - n_q - n_k) / A.hd; i = (idx - n_q - n_k) - j * A.hd;
+                sj = s - j * R; pj = pos; col = d + kvd + gk * A.hd + i; dst = &S.vf[j][i]; pair = false;
+              }
+              float cs = 1.0f, sn = 0.0f;
+              if (pair) { cs = A.rope_cos[(size_t)pj * half + i]; sn = A.rope_sin[(size_t)pj * half + i]; }
+              float x1 = 0.0f, x2 = 0.0f;
+#pragma unroll 1
+              for (int ks = 0; ks < KSq; ++ks) {
+                const float* pr = A.pq + ((size_t)ks * kPSlots + sj) * A.qkv_w + col;
+                x1 += __ldcg(pr);
+                if (pair) x2 += __ldcg(pr + half);
+              }
+              dst[0] = round_bf16(x1 * cs - x2 * sn);
+              if (pair) dst[half] = round_bf16(x2 * cs + x1 * sn);
+            }
           }
           __syncthreads();
-          const size_t cache_off = ((((size_t)si.row * A.L + layer) * A.Hkv + gk) * A.cap) * A.hd;
+          TSEC(0);
           if (split == nsplit - 1 && tid < A.hd) {       // this item owns the append of its own position
             A.kc[cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.kf[0][tid]);
             A.vc[cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
           }
-          const __nv_bfloat16* kbase = A.kc + cache_off;
-          const __nv_bfloat16* vbase = A.vc + cache_off;
-          const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
-          const int PPW = 32 / LPR;
-          const int sub = lane % LPR, pgrp = lane / LPR;
-          // ---- scores ----
-          for (int t0 = 0; t0 < grp; t0 += 4) {          // query heads in groups of 4 (register budget)
-            float qf[4][8];
+          // ---- scores of the cached positions, one query head at a time (K stays in registers) ----
+#pragma unroll 1
+          for (int t = 0; t < grp; ++t) {
+            float qf[8];
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
+            for (int e = 0; e < 8; ++e) qf[e] = S.q[t][sub * 8 + e];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) qf[t][e] = (t0 + t < grp) ? S.q[t0 + t][sub * 8 + e] : 0.0f;
-            for (int pb = warp * PPW; pb < cnt; pb += kPW * PPW) {
-              const int p = pb + pgrp;
-              const bool valid = p < cnt;
-              uint4 kv = make_uint4(0u, 0u, 0u, 0u);
-              if (valid) kv = __ldcg(reinterpret_cast<const uint4*>(kbase + (size_t)(p_lo + p) * A.hd + sub * 8));
+            for (int ps = 0; ps < 4; ++ps) {
+              if (ps * PPB >= cnt) break;                 // uniform over the CTA
+              const int p = ps * PPB + warp * PPW + pgrp;
               float kf8[8];
-              Elem<__nv_bfloat16>::unpack(kv, kf8);
+              Elem<__nv_bfloat16>::unpack(kreg[ps], kf8);
+              float dd = 0.0f;
 #pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                float dd = 0.0f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) dd = fmaf(kf8[e], qf[t][e], dd);
-                for (int o = LPR >> 1; o > 0; o >>= 1) dd += __shfl_xor_sync(0xffffffffu, dd, o);
-                if (valid && sub == 0 && t0 + t < grp) S.sc[t0 + t][p] = dd * A.attn_scale;
-              }
+              for (int e = 0; e < 8; ++e) dd = fmaf(kf8[e], qf[e], dd);
+              for (int o = LPR >> 1; o > 0; o >>= 1) dd += __shfl_xor_sync(0xffffffffu, dd, o);
+              if (sub == 0 && p < cnt && p_lo + p < fresh_lo) S.sc[t][p] = dd * A.attn_scale;
             }
           }
-          __syncthreads();
           // scores of the fresh positions come from the staged k, not from the cache
           for (int combo = warp; combo < grp * n_fresh; combo += kPW) {
             const int t = combo / n_fresh, j = combo - t * n_fresh;
@@ -620,52 +742,58 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             }
           }
           __syncthreads();
-          for (int t = warp; t < grp; t += kPW) {
+          {
+            // softmax statistics: 16/grp warps share a head
+            const int wph = (grp >= kPW) ? 1 : kPW / grp;
+            const int t = warp / wph, wi = warp - t * wph;
             float mx = -INFINITY;
-            for (int p = lane; p < cnt; p += 32) mx = fmaxf(mx, S.sc[t][p]);
+            if (t < grp) for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) mx = fmaxf(mx, S.sc[t][p]);
             mx = warp_max_f32(mx);
+            if (lane == 0) S.red[warp][0] = mx;
+            __syncthreads();
             float sum = 0.0f;
-            for (int p = lane; p < cnt; p += 32) { const float e = expf(S.sc[t][p] - mx); S.sc[t][p] = e; sum += e; }
+            if (t < grp) {
+              mx = S.red[t * wph][0];
+              for (int w2 = 1; w2 < wph; ++w2) mx = fmaxf(mx, S.red[t * wph + w2][0]);
+              for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) { const float e = expf(S.sc[t][p] - mx); S.sc[t][p] = e; sum += e; }
+            }
             sum = warp_sum_f32(sum);
-            if (lane == 0) { S.m_[t] = mx; S.l_[t] = sum; }
+            if (lane == 0) S.red[warp][1] = sum;
+            __syncthreads();
+            if (t < grp && wi == 0 && lane == 0) {
+              float tot = 0.0f;
+              for (int w2 = 0; w2 < wph; ++w2) tot += S.red[t * wph + w2][1];
+              S.m_[t] = mx; S.l_[t] = tot;
+            }
           }
-          __syncthreads();
-          // ---- P V over the cached positions ----
-          const int fresh_lo = pos - (n_fresh - 1);      // absolute positions >= fresh_lo are fresh
-          for (int t0 = 0; t0 < grp; t0 += 4) {
-            float oacc[4][8];
+          TSEC(1);
+          // ---- P V over the cached positions, one head at a time (V stays in registers) ----
+#pragma unroll 1
+          for (int t = 0; t < grp; ++t) {
+            float oacc[8];
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
+            for (int e = 0; e < 8; ++e) oacc[e] = 0.0f;
 #pragma unroll
-              for (int e = 0; e < 8; ++e) oacc[t][e] = 0.0f;
-            for (int p = warp * PPW + pgrp; p < cnt; p += kPW * PPW) {
-              if (p_lo + p >= fresh_lo) continue;
-              const uint4 vv = __ldcg(reinterpret_cast<const uint4*>(vbase + (size_t)(p_lo + p) * A.hd + sub * 8));
-              float vf8[8];
-              Elem<__nv_bfloat16>::unpack(vv, vf8);
+            for (int ps = 0; ps < 4; ++ps) {
+              if (ps * PPB >= cnt) break;
+              const int p = ps * PPB + warp * PPW + pgrp;
+              if (p < cnt && p_lo + p < fresh_lo) {
+                float vf8[8];
+                Elem<__nv_bfloat16>::unpack(vreg[ps], vf8);
+                const float pw = S.sc[t][p];
 #pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                if (t0 + t >= grp) break;
-                const float pw = S.sc[t0 + t][p];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) oacc[t][e] = fmaf(pw, vf8[e], oacc[t][e]);
+                for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf8[e], oacc[e]);
               }
             }
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                float v = oacc[t][e];
-                for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                oacc[t][e] = v;
-              }
+            for (int e = 0; e < 8; ++e) {
+              float v = oacc[e];
+              for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+              oacc[e] = v;
+            }
             if (pgrp == 0) {
 #pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                if (t0 + t >= grp) break;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) s_o[((size_t)warp * grp + t0 + t) * A.hd + sub * 8 + e] = oacc[t][e];
-              }
+              for (int e = 0; e < 8; ++e) s_o[((size_t)warp * grp + t) * A.hd + sub * 8 + e] = oacc[e];
             }
           }
           __syncthreads();
@@ -688,6 +816,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               if (dd == 0) { A.part_ml[pi * 2] = S.m_[t]; A.part_ml[pi * 2 + 1] = S.l_[t]; }
             }
           }
+          TSEC(2);
           if (!single) {
             // the CTA that finishes the last split of a (slot, kv head) merges them in split order
             __threadfence();
@@ -696,24 +825,36 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             __syncthreads();
             if (S.flag) {
               __threadfence();
+              for (int t = warp; t < grp; t += kPW) {      // rescaling factors of the splits, one warp per head
+                const size_t base = ((size_t)s * A.H + gk * grp + t) * A.max_splits;
+                float M = -INFINITY;
+                for (int j = lane; j < nsplit; j += 32) M = fmaxf(M, __ldcg(A.part_ml + (base + j) * 2));
+                M = warp_max_f32(M);
+                float den = 0.0f;
+                for (int j = lane; j < nsplit; j += 32) {
+                  const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + j) * 2));
+                  const float f = expf(ml.x - M);
+                  S.sc[t][j] = f;
+                  den = fmaf(f, ml.y, den);
+                }
+                den = warp_sum_f32(den);
+                if (lane == 0) S.l_[t] = den;
+              }
+              __syncthreads();
               for (int idx = tid; idx < grp * A.hd; idx += kPT) {
                 const int t = idx / A.hd, dd = idx - t * A.hd;
                 const int head = gk * grp + t;
                 const size_t base = ((size_t)s * A.H + head) * A.max_splits;
-                float M = -INFINITY;
-                for (int j = 0; j < nsplit; ++j) M = fmaxf(M, __ldcg(A.part_ml + (base + j) * 2));
-                float num = 0.0f, den = 0.0f;
-                for (int j = 0; j < nsplit; ++j) {
-                  const float f = expf(__ldcg(A.part_ml + (base + j) * 2) - M);
-                  num = fmaf(f, __ldcg(A.part_o + (base + j) * A.hd + dd), num);
-                  den = fmaf(f, __ldcg(A.part_ml + (base + j) * 2 + 1), den);
-                }
-                A.attn_out[(size_t)s * HD + head * A.hd + dd] = num / den;
+                float num = 0.0f;
+#pragma unroll 8
+                for (int j = 0; j < nsplit; ++j) num = fmaf(S.sc[t][j], __ldcg(A.part_o + (base + j) * A.hd + dd), num);
+                A.attn_out[(size_t)s * HD + head * A.hd + dd] = num / S.l_[t];
               }
               if (tid == 0) A.tickets[s * A.Hkv + gk] = 0;
             }
           }
           __syncthreads();
+          TSEC(3);
         }
         GRID_SYNC();
       }
@@ -742,9 +883,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       for (int item = cta; item < R * n_chunks; item += NC) {
         const int row = item / n_chunks, ch = item - row * n_chunks;
         const int v0 = ch * kChunk + tid * kPPer;
-        const float mx = ord_decode(__ldcg(rowmax + row));
         float a[kPPer];
         load4_cg(lg + (size_t)row * V, v0, V, vec, -INFINITY, a);
+        const float mx = ord_decode(__ldcg(rowmax + row));
         unsigned long long sm = 0;
 #pragma unroll
         for (int j = 0; j < kPPer; ++j) if (v0 + j < V) sm += mass_of(xexp(__fsub_rn(a[j], mx)));
@@ -757,17 +898,27 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         const int v0 = ch * kChunk + tid * kPPer;
         float acc[kPPer];
         float* qk_b = A.qk + ((size_t)b * G + step) * m * V;
+        __syncthreads();
+        if (tid < m) {
+          const int row = b * m + tid;
+          S.mix_mx[tid] = ord_decode(__ldcg(rowmax + row));
+          S.mix_sn[tid] = norm_of(__ldcg(rowsum + row));
+          S.mix_w[tid] = A.w[row];
+        }
+        float nxt[kPPer];
+        load4_cg(lg + (size_t)(b * m) * V, v0, V, vec, -INFINITY, nxt);
+        __syncthreads();
+#pragma unroll 1
         for (int k = 0; k < m; ++k) {
-          const int row = b * m + k;
-          const float mx = ord_decode(__ldcg(rowmax + row));
-          const float Sn = norm_of(__ldcg(rowsum + row));
-          const float wk = A.w[row];
           float a[kPPer];
-          load4_cg(lg + (size_t)row * V, v0, V, vec, -INFINITY, a);
+#pragma unroll
+          for (int j = 0; j < kPPer; ++j) a[j] = nxt[j];
+          if (k + 1 < m) load4_cg(lg + (size_t)(b * m + k + 1) * V, v0, V, vec, -INFINITY, nxt);
+          const float mxk = S.mix_mx[k], snk = S.mix_sn[k], wkk = S.mix_w[k];
 #pragma unroll
           for (int j = 0; j < kPPer; ++j) {
-            a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx)), Sn);
-            const float t = __fmul_rn(wk, a[j]);
+            a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mxk)), snk);
+            const float t = __fmul_rn(wkk, a[j]);
             acc[j] = (k == 0) ? t : __fadd_rn(acc[j], t);
           }
           store4(qk_b + (size_t)k * V, v0, V, (V & 3) == 0, a);
@@ -828,16 +979,26 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           continue;
         }
         const unsigned long long* cm = A.chunk_mass + (size_t)b * n_chunks;
+        // chunk masses in parallel into shared memory, then one thread walks them
+        unsigned long long T = 0;
+        for (int c0 = 0; c0 < n_chunks; c0 += kPT) {
+          const unsigned long long mine = (c0 + tid < n_chunks) ? __ldcg(cm + c0 + tid) : 0ull;
+          T += block_sum_u64_p(mine, S);
+        }
+        if (n_chunks <= kPT && tid < n_chunks) S.cm[tid] = __ldcg(cm + tid);
+        __syncthreads();
         if (tid == 0) {
-          unsigned long long T = 0;
-          for (int c2 = 0; c2 < n_chunks; ++c2) T += __ldcg(cm + c2);
           S.result = 0x7fffffff;
           if (T == 0ull) { atomicOr(A.err, 1); S.chunk = -1; }
           else {
             const unsigned long long thr = draw_threshold(A.u[b * G + step], T);
             int c2 = 0;
             unsigned long long pre = 0;
-            for (; c2 < n_chunks - 1; ++c2) { const unsigned long long nx = pre + __ldcg(cm + c2); if (nx > thr) break; pre = nx; }
+            for (; c2 < n_chunks - 1; ++c2) {
+              const unsigned long long nx = pre + (n_chunks <= kPT ? S.cm[c2] : __ldcg(cm + c2));
+              if (nx > thr) break;
+              pre = nx;
+            }
             S.chunk = c2; S.thr = thr - pre;
           }
         }
@@ -887,6 +1048,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
     }
   }  // steps
 #undef GRID_SYNC
+#undef TSEC
   return;
 
 drain:

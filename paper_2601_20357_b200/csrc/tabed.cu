@@ -77,7 +77,8 @@ struct tabed_handle {
   unsigned launches_persist = 0;
   LayerW* layer_tab = nullptr;
   float *xa = nullptr, *x1 = nullptr, *pq = nullptr, *po = nullptr, *pd = nullptr;
-  int* tickets = nullptr; unsigned* bar = nullptr;
+  int* tickets = nullptr; unsigned* bar = nullptr; float* ssq = nullptr;
+  unsigned char* packed = nullptr;
   uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
   unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false;
   // per-kernel-class timing (tabed_profile_begin / tabed_profile_end)
@@ -300,14 +301,15 @@ int setup_persistent(tabed_handle* h) {
   if (c.dtype != TABED_DTYPE_BF16) return TABED_OK;
   const int grp = h->H / h->Hkv;
   if (2 * h->R > kPSlots || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
-      grp > kMaxGroup || grp * h->hd > 512 || h->L > 1024)
+      grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || h->max_splits > kAttnSplitMax)
     return TABED_OK;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return TABED_ERR_CUDA;
   if (!prop.cooperativeLaunch) return TABED_OK;
   cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, k_draft_round) != cudaSuccess) return TABED_ERR_CUDA;
+  if (cudaFuncGetAttributes(&fa, k_draft_round<true>) != cudaSuccess) return TABED_ERR_CUDA;
   const int n_cta = prop.multiProcessorCount;
+  if (n_cta > kPT || (h->d + n_cta - 1) / n_cta + 1 > kResW) return TABED_OK;
   RoundArgs& A = h->ra;
   const int kcap = std::max(h->d, 1024);
   A.geom[KIND_QKV] = pick_geom(h->qkv_w / 16, h->d, n_cta, kcap, false);
@@ -324,10 +326,11 @@ int setup_persistent(tabed_handle* h) {
   if (avail < u_bytes + 2 * (size_t)A.slot_bytes) return TABED_OK;
   A.n_ring = (int)std::min<size_t>(kPRing, (avail - u_bytes) / A.slot_bytes);
   h->persist_smem = (size_t)A.n_ring * A.slot_bytes + u_bytes;
-  if (cudaFuncSetAttribute(k_draft_round, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_draft_round<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess ||
+      cudaFuncSetAttribute(k_draft_round<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess)
     return TABED_ERR_CUDA;
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_draft_round, kPT, h->persist_smem) != cudaSuccess) return TABED_ERR_CUDA;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_draft_round<true>, kPT, h->persist_smem) != cudaSuccess) return TABED_ERR_CUDA;
   if (per_sm < 1) return TABED_OK;
   h->n_cta = n_cta;
 
@@ -337,19 +340,52 @@ int setup_persistent(tabed_handle* h) {
   A2(&h->layer_tab, (size_t)h->L); A2(&h->xa, kPSlots * d); A2(&h->x1, kPSlots * d);
   A2(&h->pq, (size_t)A.geom[KIND_QKV].KS * kPSlots * h->qkv_w); A2(&h->po, (size_t)A.geom[KIND_O].KS * kPSlots * d);
   A2(&h->pd, (size_t)A.geom[KIND_DN].KS * kPSlots * d);
-  A2(&h->tickets, (size_t)kPSlots * h->Hkv); A2(&h->bar, 2);
+  A2(&h->tickets, (size_t)kPSlots * h->Hkv); A2(&h->bar, 2); A2(&h->ssq, (size_t)n_cta * kPSlots);
+  // private copy of the weights, unit by unit (one contiguous block per bulk copy)
+  size_t unit_bytes[5], kind_bytes[5];
+  for (int k = 0; k < 5; ++k) {
+    unit_bytes[k] = 16 * ((size_t)A.geom[k].kchunk * 2 + 16);
+    kind_bytes[k] = unit_bytes[k] * A.geom[k].n_units;
+  }
+  A.pack_off[KIND_QKV] = 0;
+  A.pack_off[KIND_O] = A.pack_off[KIND_QKV] + kind_bytes[KIND_QKV];
+  A.pack_off[KIND_GU] = A.pack_off[KIND_O] + kind_bytes[KIND_O];
+  A.pack_off[KIND_DN] = A.pack_off[KIND_GU] + kind_bytes[KIND_GU];
+  A.pack_layer_stride = A.pack_off[KIND_DN] + kind_bytes[KIND_DN];
+  A.pack_off[KIND_LM] = A.pack_layer_stride * h->L;
+  if (rc == TABED_OK) {
+    void* ptr = nullptr;
+    if (cudaMalloc(&ptr, A.pack_off[KIND_LM] + kind_bytes[KIND_LM]) != cudaSuccess) { cudaGetLastError(); return TABED_OK; }   // no room: per-operation path
+    h->allocs.push_back(ptr);
+    h->packed = reinterpret_cast<unsigned char*>(ptr);
+  }
   A2(&h->rowmax_g, (size_t)h->G * h->R); A2(&h->rowsum_g, (size_t)h->G * h->R);
-  h->trace_stride = 5 * h->L + 8;
-  A2(&h->trace, (size_t)h->G * h->trace_stride);
+  h->trace_stride = 7 * h->L + 8;
+  A2(&h->trace, (size_t)h->G * h->trace_stride * kTraceRec);
   if (rc != TABED_OK) return rc;
   std::vector<LayerW> tab(h->L);
   using bf = __nv_bfloat16;
   for (int l = 0; l < h->L; ++l)
     tab[l] = LayerW{(const bf*)h->wq[l], (const bf*)h->wk[l], (const bf*)h->wv[l], (const bf*)h->wo[l], (const bf*)h->w_gate[l],
                     (const bf*)h->w_up[l], (const bf*)h->w_down[l], (const bf*)h->norm1[l], (const bf*)h->norm2[l]};
-  if (cudaMemcpyAsync(h->layer_tab, tab.data(), tab.size() * sizeof(LayerW), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
-      cudaStreamSynchronize(h->stream) != cudaSuccess)
+  if (cudaMemcpyAsync(h->layer_tab, tab.data(), tab.size() * sizeof(LayerW), cudaMemcpyHostToDevice, h->stream) != cudaSuccess)
     return TABED_ERR_CUDA;
+  const int kvd = h->Hkv * h->hd;
+  for (int l = 0; l <= h->L; ++l) {
+    for (int k = 0; k < 5; ++k) {
+      if ((l == h->L) != (k == KIND_LM)) continue;
+      PackArgs P{};
+      P.kind = k; P.g = A.geom[k];
+      P.dst = h->packed + A.pack_off[k] + (k == KIND_LM ? 0 : (size_t)l * A.pack_layer_stride);
+      if (k == KIND_QKV) { P.w0 = tab[l].wq; P.w1 = tab[l].wk; P.w2 = tab[l].wv; P.rows0 = h->d; P.rows1 = kvd; P.rows2 = kvd; P.K = h->d; }
+      else if (k == KIND_O) { P.w0 = tab[l].wo; P.rows0 = h->d; P.K = h->H * h->hd; }
+      else if (k == KIND_GU) { P.w0 = tab[l].wg; P.w1 = tab[l].wu; P.rows0 = h->F; P.rows1 = h->F; P.K = h->d; }
+      else if (k == KIND_DN) { P.w0 = tab[l].wd; P.rows0 = h->d; P.K = h->F; }
+      else { P.w0 = (const bf*)h->lm_head; P.rows0 = h->V; P.K = h->d; }
+      k_pack_units<<<A.geom[k].n_units, 256, 0, h->stream>>>(P);
+    }
+  }
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
   A.layers = h->layer_tab; A.embed = (const bf*)h->embed; A.lm_head = (const bf*)h->lm_head; A.final_norm = (const bf*)h->final_norm;
   A.rope_cos = h->rope_cos; A.rope_sin = h->rope_sin;
   A.L = h->L; A.d = h->d; A.F = h->F; A.H = h->H; A.Hkv = h->Hkv; A.hd = h->hd; A.V = h->V; A.cap = h->cap; A.qkv_w = h->qkv_w;
@@ -360,7 +396,8 @@ int setup_persistent(tabed_handle* h) {
   A.part_o = h->part_o; A.part_ml = h->part_ml; A.max_splits = h->max_splits; A.tickets = h->tickets;
   A.logits_own = h->logits_own; A.w = h->w; A.qk = h->qk; A.q = h->q;
   A.rowmax = h->rowmax_g; A.rowsum = h->rowsum_g; A.chunk_mass = h->chunk_mass; A.chunk_best = h->chunk_best;
-  A.n_chunks = h->n_chunks; A.tokens = h->tokens; A.bar = h->bar; A.err = h->err; A.trace_stride = h->trace_stride;
+  A.n_chunks = h->n_chunks; A.tokens = h->tokens; A.bar = h->bar; A.ssq = h->ssq; A.err = h->err; A.packed = h->packed;
+  A.trace_stride = h->trace_stride;
   h->persist_ok = true;
   return TABED_OK;
 }
@@ -368,11 +405,13 @@ int setup_persistent(tabed_handle* h) {
 int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_tokens, int max_pos) {
   RoundArgs A = h->ra;
   A.u = u_draft; A.out_tokens = out_tokens; A.logits_override = h->logits_override;
-  A.split_len = (max_pos > 2048) ? 256 : 128;
+  (void)max_pos;
+  A.split_len = (h->hd <= 64) ? 256 : 128;          // positions per attention item: 4 register passes of the CTA
   A.bar_sel = (int)(h->launches_persist & 1u);
   A.trace = h->trace_on ? h->trace : nullptr;
   void* args[] = {&A};
-  if (cudaLaunchCooperativeKernel((const void*)k_draft_round, dim3(h->n_cta), dim3(kPT), args, h->persist_smem, h->stream) != cudaSuccess)
+  const void* kern = h->trace_on ? (const void*)k_draft_round<true> : (const void*)k_draft_round<false>;
+  if (cudaLaunchCooperativeKernel(kern, dim3(h->n_cta), dim3(kPT), args, h->persist_smem, h->stream) != cudaSuccess)
     return TABED_ERR_CUDA;
   h->launches_persist++;
   h->launches++;
@@ -819,7 +858,7 @@ int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* byte
     case TABED_VIEW_ERROR_FLAG: *dev_ptr = h->err; *bytes = 4; break;
     case TABED_VIEW_TRACE:
       if (!h->persist_ok) return TABED_ERR_BAD_STATE;
-      *dev_ptr = h->trace; *bytes = (size_t)h->G * h->trace_stride * 8; break;
+      *dev_ptr = h->trace; *bytes = (size_t)h->G * h->trace_stride * kTraceRec * 8; break;
     default: return TABED_ERR_INVALID_ARG;
   }
   return TABED_OK;
