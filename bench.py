@@ -386,8 +386,8 @@ def run_ours(args, wl):
         g.verify(targets[Wm], u[Wm][1], u[Wm][2], a, z)
         g.update_weights(w, am)
         L = wl.drafter.n_layers
-        nb_step = 7 * L + 3
-        names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "res1", "gateup", "down", "res2")] + ["lm_head", "expsum", "mix"]
+        nb_step = 5 * L + 3
+        names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "gateup", "down")] + ["lm_head", "expsum", "mix"]
         mhz = float(clocks.get("sm_mhz") or 1965.0)
         with open(args.trace, "w") as f:
             f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA 0): us from the previous grid barrier to this one,\n"

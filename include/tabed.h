@@ -75,7 +75,7 @@ extern "C" {
 #define TABED_VIEW_PENDING     7   /* int32  [B][3]        {count, token0, token1}                     */
 #define TABED_VIEW_GRID_J      8   /* int32  [B]           j* of the grid policy (-1 before any update)*/
 #define TABED_VIEW_ERROR_FLAG  9   /* int32  [1]           non-zero if a device-side check failed      */
-#define TABED_VIEW_TRACE      10   /* uint64 [G][7L+8][8]  phase timeline of the persistent drafting kernel
+#define TABED_VIEW_TRACE      10   /* uint64 [G][5L+8][8]  phase timeline of the persistent drafting kernel
                                                            (tabed_debug_trace): one record per grid barrier */
 
 /* How tabed_draft_round runs Algorithm 1 (tabed_select_path).  Results obey the same contract on
@@ -210,7 +210,7 @@ int tabed_current_path(const tabed_handle* h);
  * barrier resolving and staging activations, waiting for weight tiles, in the tensor-core products,
  * issuing weight copies, in epilogues (or, for the phases without weights, in all of the phase), and
  * in the barrier itself; [7] unused.  Barrier order within a step: per layer QKV, attention, O,
- * resolve, gate/up, down, resolve; then LM head, [2 more when tabed_debug_override_logits is set],
+ * gate/up, down; then LM head, [2 more when tabed_debug_override_logits is set],
  * exp-sum, mix.
  * Errors: UNSUPPORTED (no persistent path). */
 int tabed_debug_trace(tabed_handle* h, int32_t on);

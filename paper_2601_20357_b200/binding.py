@@ -273,7 +273,7 @@ class Tabed:
             VIEW_LOGITS: ((G, B, m, V), "<f4"), VIEW_KV_LEN: ((R,), "<i4"), VIEW_WEIGHTS: ((B, m), "<f4"),
             VIEW_WINDOW_SUM: ((B, MAX_DEV), "<i8"), VIEW_PENDING: ((B, 3), "<i4"), VIEW_GRID_J: ((B,), "<i4"),
             VIEW_ERROR_FLAG: ((1,), "<i4"),
-            VIEW_TRACE: ((G, 7 * (self.drafter.n_layers if self.drafter is not None else 0) + 8, 8), "<u8")}[what]
+            VIEW_TRACE: ((G, 5 * (self.drafter.n_layers if self.drafter is not None else 0) + 8, 8), "<u8")}[what]
         return torch.as_tensor(_DeviceView(ptr.value, shape, ts), device=self.device)
 
     def debug_override_logits(self, drafter_logits: Optional[torch.Tensor]) -> None:

@@ -3,26 +3,28 @@
 // cooperative launch with one CTA per SM.
 //
 // Why one kernel: with m <= 4 drafting inputs a decoder step moves ~125-630 MB of weights through
-// ~25-65 strictly dependent phases; as separate launches every phase pays a launch plus a cold
+// dozens of strictly dependent phases; as separate launches every phase pays a launch plus a cold
 // DRAM round trip.  Here
-//   * the weights never stop streaming: every CTA owns a fixed, round-robin share of the weight
-//     tiles of every phase, and one warp keeps a ring of shared-memory slots filled with bulk
-//     asynchronous copies (cp.async.bulk + mbarrier) several phases ahead of the arithmetic, so
-//     HBM stays busy across the grid barriers;
-//   * a phase is: grid barrier -> stage the (tiny) activations from L2 -> tensor-core products
-//     of the 16-row weight tiles already sitting in shared memory -> results back to L2;
-//   * the critical path is the chain of phases, so every phase is built to cost one L2 round trip
-//     plus the barrier: split-K partial sums are reduced once, slice by slice, in a short
-//     "resolve" phase of their own (not 148 times by every consumer), a CTA issues all loads of an
-//     attention item (K, V, q) before it uses any;
+//   * the weights never stop streaming: every CTA owns a fixed share of the weight tiles of every
+//     phase (its unit list is built once, in shared memory), and a ring of shared-memory slots is
+//     kept full by bulk asynchronous copies (cp.async.bulk + mbarrier) several phases ahead of the
+//     arithmetic, so HBM stays busy across the grid barriers;
 //   * the weights are read from a private copy laid out for this kernel at set-up: every unit (16
-//     rows x kchunk columns, rows already padded to the bank-conflict-free shared-memory pitch) is
-//     one contiguous block, so a unit is ONE bulk copy (16 per-row copies cost ~1 us of issue time
-//     per unit on the critical path);
-//   * projections use mma.sync m16n8k16 (bf16 x bf16 -> fp32): 16 weight rows x up to 8 slots.
-//     The contraction is HBM-bound (<= 8 flop per weight byte), the tensor pipe is used only to
-//     keep the ALUs off the critical path;
-//   * all cross-CTA data is read with ld.global.cg (L2) because L1 is not coherent across SMs.
+//     output rows x kchunk input columns, rows padded to a bank-conflict-free shared-memory pitch)
+//     is one contiguous block, hence ONE bulk copy;
+//   * a phase is: grid barrier -> stage the (tiny) activations from L2 -> tensor-core products of
+//     the weight tiles already sitting in shared memory -> results back to L2.  The chain of phases
+//     is the critical path, so it is kept short: 5 barriers per layer (QKV, attention, O, gate/up,
+//     down).  A 16-row tile always takes its whole input dimension on ONE CTA (long rows as
+//     sub-units whose products accumulate in registers), so no projection leaves split-K partial
+//     sums behind and the residual adds and RMSNorm statistics ride in the epilogues;
+//   * four warp groups work on four units at a time (mma.sync m16n8k16, bf16 x bf16 -> fp32:
+//     16 weight rows x up to 8 slots).  The contraction is HBM-bound (<= 8 flop per weight byte);
+//     the tensor pipe only keeps the ALUs off the critical path;
+//   * an attention item issues all its loads (K, V, q) before it uses any;
+//   * all cross-CTA data is read with ld.global.cg (L2) because L1 is not coherent across SMs;
+//   * loops are deliberately not unrolled except the few hot ones: every phase runs its code once,
+//     so unrolling buys nothing and only inflates the instruction footprint.
 //
 // Waits are bounded: a grid barrier or a copy that does not complete within the spin limit sets an
 // error bit, the CTA drains its copies in flight and returns.
@@ -39,28 +41,30 @@ namespace tabed {
 
 constexpr int kPT = 512;                 // threads per CTA
 constexpr int kPW = kPT / 32;            // warps per CTA
+constexpr int kWG = 4;                   // warp groups (each works on its own unit)
+constexpr int kGW = kPW / kWG;           // warps per group
 constexpr int kPSlots = 8;               // slots (row, position) per step: one mma n-tile
 constexpr int kPRing = 16;               // upper bound of ring slots
 constexpr int kPPer = kChunk / kPT;      // vocabulary elements per thread and chunk (4)
-constexpr int kPMaxD = 2048;             // d_model bound (4 residual elements per thread and slot)
-constexpr int kPXE = kPMaxD / kPT;
+constexpr int kPMaxD = 2048;             // d_model bound
 constexpr int kTraceRec = 8;             // words per record of the phase timeline
 constexpr int kPMaxL = 64;               // layers (their pointer table lives in shared memory)
-constexpr int kResW = 16;                // upper bound of a CTA's slice of d_model in a resolve phase
+constexpr int kMaxUnits = 3072;          // units of one CTA in one decoder step
+constexpr int kMaxPhase = 4 * kPMaxL + 1;
 
 enum { KIND_QKV = 0, KIND_O = 1, KIND_GU = 2, KIND_DN = 3, KIND_LM = 4 };
 enum { PERR_BARRIER = 8, PERR_COPY = 16, PERR_KV = 4 };
 
 struct LayerW { const __nv_bfloat16 *wq, *wk, *wv, *wo, *wg, *wu, *wd, *n1, *n2; };
 
-// A phase's weight matrix is cut into units: 16 output rows x kchunk input columns.
-// unit u -> k-split ks = u / n_tiles, tile = u % n_tiles.
-struct PhaseGeom { int n_tiles, KS, kchunk, n_units; };
+// A phase's weight matrix is cut into tiles of 16 output rows; a tile is nsub units of kchunk input
+// columns each (nsub in {1, 2} or a multiple of 4).  unit u -> tile = u / nsub, sub = u % nsub.
+struct PhaseGeom { int n_tiles, nsub, kchunk, n_units; };
 
 struct RoundArgs {
   // drafter
   const LayerW* layers;
-  const __nv_bfloat16 *embed, *lm_head, *final_norm;
+  const __nv_bfloat16 *embed, *final_norm;
   const float *rope_cos, *rope_sin;
   int L, d, F, H, Hkv, hd, V, cap, qkv_w;
   float eps, attn_scale;
@@ -68,17 +72,16 @@ struct RoundArgs {
   const unsigned char* packed;          // weights re-laid out unit by unit (k_pack_units)
   unsigned long long pack_off[5];       // byte offset of a kind's units inside a layer block (LM: absolute)
   unsigned long long pack_layer_stride;
-  int slot_bytes, n_ring, act_bytes, split_len;
+  int slot_bytes, n_ring, act_bytes, act_slots, split_len;
   // round
   int R, B, m, G, greedy;
   const int* kv_len;                    // [R] committed lengths (constant during the round)
   const int* pending;                   // [B][3]
   __nv_bfloat16 *kc, *vc;               // [R][L][Hkv][cap][hd]
   // activations exchanged through L2
-  float *xa, *x1;                       // [8][d] residual before / after the attention block
-  float* ssq;                           // [n_cta][8] per-CTA partial sums of squares of the last resolve
-  float *pq, *po, *pd;                  // split-K partial sums [KS][8][width]
-  float *mid, *attn_out;                // [8][F], [8][H*hd]
+  float *xa, *x1;                       // [8][d] residual entering a layer / after its attention block
+  float* ssq;                           // [d/16][8] sums of squares of the last residual, per 16-row tile
+  float *qkv, *mid, *attn_out;          // [8][qkv_w], [8][F], [8][H*hd]
   float *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2]
   int max_splits;
   int* tickets;                         // [8][Hkv]
@@ -152,6 +155,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+__device__ __forceinline__ float4 bf16x4_to_float4(uint2 v) {
+  return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                     __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+}
+
 // ------------------------------------------------------------------------------------------------
 // per-CTA state
 // ------------------------------------------------------------------------------------------------
@@ -160,6 +168,8 @@ struct PSlot { int row, pos, active, tok; };
 struct PShared {
   uint64_t full[kPRing];
   LayerW layers[kPMaxL];
+  uint32_t ulist[kMaxUnits];            // this CTA's units of one decoder step, in consumption order
+  uint16_t pstart[kMaxPhase + 1];       // first entry of every phase in ulist
   float sc[kMaxGroup][kAttnSplitMax];
   float q[kMaxGroup][128];
   float kf[2][128], vf[2][128];
@@ -168,49 +178,32 @@ struct PShared {
   unsigned long long cm[kPT];
   float bestv[kPW]; int besti[kPW];
   float scale[kPSlots];
+  uint32_t lmmax[kPSlots];
   float mix_mx[kMaxInputs], mix_sn[kMaxInputs], mix_w[kMaxInputs];
   float m_[kMaxGroup], l_[kMaxGroup];
   PSlot slot[kPSlots];
   int lm_src[kPSlots];
   int tok[kPSlots];
   int dead, flag, result, chunk;
-  unsigned long long thr, total;
+  unsigned long long thr;
 };
 
-// Walks the CTA's units in consumption order: for each step, for each layer QKV, O, GU, DN, then
-// the LM head.  Units of a phase are dealt round-robin over the CTAs, continuing where the
-// previous phase stopped, so every CTA streams the same number of bytes (+-1 unit).
-struct UnitCursor { int step, p, j, off; };
-struct UnitRef { int kind, layer, u; };
+__device__ __forceinline__ uint32_t unit_pack(int kind, int layer, int u) { return (uint32_t)kind | ((uint32_t)layer << 3) | ((uint32_t)u << 10); }
 
-__device__ __forceinline__ bool next_unit(const RoundArgs& A, int cta, int NC, UnitCursor& c, UnitRef& out) {
-  const int n_phase = 4 * A.L + 1;
-  while (c.step < A.G) {
-    while (c.p < n_phase) {
-      const int kind = (c.p == n_phase - 1) ? KIND_LM : (c.p & 3);
-      const int n = A.geom[kind].n_units;
-      int first = cta - c.off;
-      if (first < 0) first += NC;
-      const int u = first + c.j * NC;
-      if (u < n) { out.kind = kind; out.layer = c.p >> 2; out.u = u; c.j++; return true; }
-      c.off = (c.off + n) % NC; c.p++; c.j = 0;
-    }
-    c.step++; c.p = 0; c.j = 0; c.off = 0;
-  }
-  return false;
-}
-
-// Issue the bulk copy of one unit into a ring slot (one thread).
-__device__ __forceinline__ void issue_unit(const RoundArgs& A, const UnitRef& ur, unsigned char* slot_base, uint64_t* bar) {
-  const unsigned bytes = 16u * ((unsigned)A.geom[ur.kind].kchunk * 2u + 16u);
-  const unsigned char* src = A.packed + A.pack_off[ur.kind] + (size_t)ur.u * bytes +
-                             (ur.kind == KIND_LM ? 0ull : (unsigned long long)ur.layer * A.pack_layer_stride);
-  mbar_expect_tx(bar, bytes);
-  bulk_g2s(slot_base, src, bytes, bar);
+// Issue the bulk copy of unit number k (counted over the whole round) into its ring slot (one thread).
+__device__ __forceinline__ void issue_unit(const RoundArgs& A, PShared& S, unsigned char* ring, unsigned k, unsigned per_step) {
+  const uint32_t e = S.ulist[k % per_step];
+  const int kind = e & 7, layer = (e >> 3) & 127, u = e >> 10;
+  const unsigned bytes = 16u * ((unsigned)A.geom[kind].kchunk * 2u + 16u);
+  const unsigned char* src = A.packed + A.pack_off[kind] + (size_t)u * bytes +
+                             (kind == KIND_LM ? 0ull : (unsigned long long)layer * A.pack_layer_stride);
+  const int slot = (int)(k % (unsigned)A.n_ring);
+  mbar_expect_tx(&S.full[slot], bytes);
+  bulk_g2s(ring + (size_t)slot * A.slot_bytes, src, bytes, &S.full[slot]);
 }
 
 // Re-lay one weight matrix (or the QKV / gate-up group) of one layer into units.  grid (n_units), block 256.
-// Row r of unit (ks, tile): QKV rows are the concatenation wq | wk | wv; gate/up units hold 8 gate
+// Row r of unit (tile, sub): QKV rows are the concatenation wq | wk | wv; gate/up units hold 8 gate
 // rows then the 8 matching up rows; LM-head rows beyond V are zero.
 struct PackArgs {
   const __nv_bfloat16 *w0, *w1, *w2;    // source matrices [rows_i][K]
@@ -220,7 +213,7 @@ struct PackArgs {
 };
 __global__ void k_pack_units(const PackArgs P) {
   const int u = blockIdx.x;
-  const int ks = u / P.g.n_tiles, tile = u - ks * P.g.n_tiles;
+  const int tile = u / P.g.nsub, sub = u - tile * P.g.nsub;
   const int pitch = P.g.kchunk * 2 + 16;
   unsigned char* unit = P.dst + (size_t)u * 16 * pitch;
   const int vec_per_row = pitch / 16;                      // 16-byte vectors per padded row
@@ -237,7 +230,7 @@ __global__ void k_pack_units(const PackArgs P) {
         else if (row < P.rows0 + P.rows1) { base = P.w1; row -= P.rows0; }
         else if (row < P.rows0 + P.rows1 + P.rows2) { base = P.w2; row -= P.rows0 + P.rows1; }
       }
-      if (base) v = *reinterpret_cast<const uint4*>(base + (size_t)row * P.K + (size_t)ks * P.g.kchunk + c16 * 8);
+      if (base) v = *reinterpret_cast<const uint4*>(base + (size_t)row * P.K + (size_t)sub * P.g.kchunk + c16 * 8);
     }
     *reinterpret_cast<uint4*>(unit + (size_t)r * pitch + (size_t)c16 * 16) = v;
   }
@@ -245,11 +238,11 @@ __global__ void k_pack_units(const PackArgs P) {
 
 constexpr unsigned kSpinLimit = 1u << 21;
 
-// Bounded wait for a ring slot.  Returns false (and marks the CTA dead) on timeout.
+// Bounded wait for a ring slot.  Returns false on timeout.
 __device__ __forceinline__ bool wait_full(PShared& S, int slot, unsigned parity, int* err) {
   unsigned spins = 0;
   while (!mbar_try_wait(&S.full[slot], parity)) {
-    if (++spins > kSpinLimit) { atomicOr(err, PERR_COPY); S.dead = 1; return false; }
+    if (++spins > kSpinLimit) { atomicOr(err, PERR_COPY); return false; }
     if (spins > 4096) __nanosleep(64);
   }
   return true;
@@ -258,7 +251,7 @@ __device__ __forceinline__ bool wait_full(PShared& S, int slot, unsigned parity,
 // Grid-wide barrier on a counter that only grows during a launch.  (One flag per CTA polled by all
 // CTAs in parallel was measured 3-4x slower: 148 x 148 concurrent polls saturate the L2 slice.)
 // Returns false if the wait ran out.
-__device__ __forceinline__ bool grid_barrier(PShared& S, unsigned* bar, unsigned target, int* err) {
+__device__ __noinline__ bool grid_barrier(PShared& S, unsigned* bar, unsigned target, int* err) {
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -268,7 +261,6 @@ __device__ __forceinline__ bool grid_barrier(PShared& S, unsigned* bar, unsigned
       if (++spins > kSpinLimit) { atomicOr(err, PERR_BARRIER); S.dead = 1; break; }
       if (spins > 4096) __nanosleep(64);
     }
-    __threadfence();
   }
   __syncthreads();
   return S.dead == 0;
@@ -313,51 +305,90 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   extern __shared__ __align__(128) unsigned char dyn_smem[];
   __shared__ PShared S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wgrp = warp / kGW, wl = warp % kGW;          // warp group and warp within the group
   const int cta = blockIdx.x, NC = gridDim.x;
   unsigned char* ring = dyn_smem;
   unsigned char* U = dyn_smem + (size_t)A.n_ring * A.slot_bytes;
-  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(U);               // [8][apitch]
+  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(U);               // [areas][act_slots][apitch]
   float* cpart = reinterpret_cast<float*>(U + A.act_bytes);               // [2][kPW][128]
   float* s_o = reinterpret_cast<float*>(U);                               // attention: [kPW][grp*hd]
-  float* rbuf = reinterpret_cast<float*>(U);                              // resolve: [terms][8][kResW]
   const int kvd = A.Hkv * A.hd, HD = A.H * A.hd, grp = A.H / A.Hkv, half = A.hd >> 1;
   const int R = A.R, B = A.B, m = A.m, G = A.G, V = A.V, d = A.d;
-  const int d4 = d >> 2;                                // float4 groups of the residual; thread t owns group t
-  const int lo = (int)((long long)cta * d / NC), hi = (int)((long long)(cta + 1) * d / NC);   // resolve slice
+  const int d4 = d >> 2, n_phase = 4 * A.L + 1;
 
   // ---- set-up -----------------------------------------------------------------------------------
   if (tid == 0) {
+#pragma unroll 1
     for (int s = 0; s < A.n_ring; ++s) mbar_init(&S.full[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     S.dead = 0;
   }
+#pragma unroll 1
   for (int i = tid; i < A.L * (int)(sizeof(LayerW) / sizeof(void*)); i += kPT)
     reinterpret_cast<const void**>(S.layers)[i] = reinterpret_cast<const void* const*>(A.layers)[i];
   if (cta == 0) {
+#pragma unroll 1
     for (int i = tid; i < G * R; i += kPT) { A.rowmax[i] = 0u; A.rowsum[i] = 0ull; }
+#pragma unroll 1
     for (int i = tid; i < kPSlots * A.Hkv; i += kPT) A.tickets[i] = 0;
     if (tid == 0) A.bar[A.bar_sel ^ 1] = 0u;          // the next launch's counter
   }
-  __syncthreads();
-
-  UnitCursor pc{0, 0, 0, 0};
-  unsigned prod_i = 0, cons_i = 0;
-  if (tid == 0) {
-    for (int k = 0; k < A.n_ring; ++k) {
-      UnitRef ur;
-      if (!next_unit(A, cta, NC, pc, ur)) break;
-      issue_unit(A, ur, ring + (size_t)k * A.slot_bytes, &S.full[k]);
-      ++prod_i;
+  // unit list of one decoder step: tiles of phase p are dealt round-robin over the CTAs, starting
+  // where phase p-1 stopped, so that every CTA streams about the same number of bytes
+#pragma unroll 1
+  for (int p = tid; p <= n_phase; p += kPT) {
+    int cnt = 0;
+    if (p < n_phase) {
+      const int kind = (p == n_phase - 1) ? KIND_LM : (p & 3);
+      int off = 0;                                     // tiles dealt before this phase, modulo NC
+#pragma unroll 1
+      for (int q2 = 0; q2 < p; ++q2) off = (off + A.geom[(q2 & 3)].n_tiles) % NC;
+      int first = cta - off;
+      if (first < 0) first += NC;
+      const int nt = A.geom[kind].n_tiles;
+      cnt = (first < nt) ? ((nt - 1 - first) / NC + 1) * A.geom[kind].nsub : 0;
     }
+    S.pstart[p] = (uint16_t)cnt;                       // counts first, offsets after the scan below
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+#pragma unroll 1
+    for (int p = 0; p <= n_phase; ++p) { const int c2 = S.pstart[p]; S.pstart[p] = (uint16_t)run; run += c2; }
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int p = tid; p < n_phase; p += kPT) {
+    const int kind = (p == n_phase - 1) ? KIND_LM : (p & 3);
+    int off = 0;
+#pragma unroll 1
+    for (int q2 = 0; q2 < p; ++q2) off = (off + A.geom[(q2 & 3)].n_tiles) % NC;
+    int first = cta - off;
+    if (first < 0) first += NC;
+    int n = S.pstart[p];
+    const int nsub = A.geom[kind].nsub;
+#pragma unroll 1
+    for (int t = first; t < A.geom[kind].n_tiles; t += NC)
+#pragma unroll 1
+      for (int sb = 0; sb < nsub; ++sb) S.ulist[n++] = unit_pack(kind, p >> 2, t * nsub + sb);
+  }
+  __syncthreads();
+  const unsigned per_step = S.pstart[n_phase];
+  const unsigned total_units = per_step * (unsigned)G;
+  if (tid == 0) {
+#pragma unroll 1
+    for (unsigned k = 0; k < (unsigned)A.n_ring && k < total_units; ++k) issue_unit(A, S, ring, k, per_step);
   }
   unsigned* bar = A.bar + A.bar_sel;
   unsigned bar_target = 0;
   bool alive = true;
+  unsigned cons_done = 0;                                // units consumed so far (for the drain)
 
   // phase timeline (CTA 0, thread 0): per grid barrier one record of kTraceRec words:
   // [0] nanosecond timer after the barrier, [1..6] clock cycles spent since the previous barrier in
-  // resolve+stage, waiting for weight tiles, mma+partials, issuing copies, epilogue/other, the barrier
+  // staging activations, waiting for weight tiles, mma+partials, issuing copies + epilogue (for
+  // attention: its four sections in slots 1-4), everything else, and in the barrier itself
   const bool tr_on = TRACE && A.trace != nullptr && cta == 0 && tid == 0;
   long long t_sec[6] = {0, 0, 0, 0, 0, 0};
   long long t_mark = 0;
@@ -384,11 +415,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   } while (0)
   if (tr_on) t_mark = clock64();
 
+#pragma unroll 1
   for (int step = 0; step < G; ++step) {
     int trace_n = 0;
     // ---- slot table of the step ------------------------------------------------------------------
     int ns = R;
     if (step == 0) {
+#pragma unroll 1
       for (int b = 0; b < B; ++b) if (A.pending[b * 3] == 2) ns = 2 * R;
     }
     if (tid < kPSlots) {
@@ -409,239 +442,247 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         if (sl.active && sl.pos >= A.cap) { sl.active = 0; atomicOr(A.err, PERR_KV); }
       }
       S.slot[tid] = sl;
+      S.lmmax[tid] = 0u;
       if (tid < R) {
         const int b = tid / m;
         S.lm_src[tid] = (step == 0 && A.pending[b * 3] == 2) ? R + tid : tid;
       }
     }
     __syncthreads();
-    int off = 0;                                    // round-robin offset of the current phase
 
-    for (int phase = 0; phase <= 4 * A.L; ++phase) {
-      const int kind = (phase == 4 * A.L) ? KIND_LM : (phase & 3);
+#pragma unroll 1
+    for (int phase = 0; phase < n_phase; ++phase) {
+      const int kind = (phase == n_phase - 1) ? KIND_LM : (phase & 3);
       const int layer = phase >> 2;
       const LayerW& lw = S.layers[kind == KIND_LM ? 0 : layer];
       const PhaseGeom g = A.geom[kind];
       const int apitch = g.kchunk + 8;                       // bf16 elements
+      const int area_elems = A.act_slots * apitch;           // one staging area: [act_slots][apitch]
       const int n_in = (kind == KIND_LM) ? R : ns;           // activation rows of the phase
       const bool norm_kind = kind == KIND_QKV || kind == KIND_GU || kind == KIND_LM;
+      const unsigned ka = (unsigned)step * per_step + S.pstart[phase], kb = (unsigned)step * per_step + S.pstart[phase + 1];
 
       if (kind == KIND_QKV && layer == 0) {
         // the residual entering layer 0 is the embedding itself: publish this CTA's slice of it
-        const int wsl = hi - lo;
+        const int lo = (int)((long long)cta * d / NC), hi = (int)((long long)(cta + 1) * d / NC), wsl = hi - lo;
         if (tid < ns * wsl) {
           const int s = tid / wsl, e = lo + (tid - s * wsl);
           if (S.slot[s].active) A.xa[(size_t)s * d + e] = __bfloat162float(A.embed[(size_t)S.slot[s].tok * d + e]);
         }
       }
-      TSEC(0);
-
-      // ---- units of this CTA ------------------------------------------------------------------------
-      int first = cta - off;
-      if (first < 0) first += NC;
-      int cur_ks = -1;
-      float lm_max = -INFINITY;
-      for (int u = first; u < g.n_units; u += NC) {
-        const int ks = u / g.n_tiles, tile = u - ks * g.n_tiles;
-        if (ks != cur_ks) {
-          // stage the activation chunk [n_in][kchunk] as bf16 (matmul inputs are rounded to bf16)
-          const int k0 = ks * g.kchunk;
-          if (norm_kind) {
-            // resolved residual (one L2 trip), RMSNorm statistics, normalised chunk -> bf16
-            const bool from_embed = kind == KIND_QKV && layer == 0;
-            const float* xbuf = (kind == KIND_GU) ? A.x1 : A.xa;
-            float4 xv[kPSlots];
-            float ss[kPSlots];
-            const __nv_bfloat16* gain = (kind == KIND_QKV) ? lw.n1 : (kind == KIND_GU ? lw.n2 : A.final_norm);
-            uint2 g2 = make_uint2(0u, 0u);
-            if (tid < d4) g2 = __ldg(reinterpret_cast<const uint2*>(gain) + tid);
+      if (norm_kind && ka < kb) {
+        // ---- stage RMSNorm(x) * gain as bf16, whole rows (these phases have kchunk == d) -----------
+        const bool from_embed = kind == KIND_QKV && layer == 0;
+        const float* xbuf = (kind == KIND_GU) ? A.x1 : A.xa;
+        const __nv_bfloat16* gain = (kind == KIND_QKV) ? lw.n1 : (kind == KIND_GU ? lw.n2 : A.final_norm);
+        const int total = n_in * d4;
+#pragma unroll 1
+        for (int it0 = 0; it0 < total; it0 += 2 * kPT) {
+          float4 xv[2];
+          uint2 gv[2];
+          int ss[2];
 #pragma unroll
-            for (int s = 0; s < kPSlots; ++s) {
-              xv[s] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-              ss[s] = 0.0f;
-              if (s >= n_in || tid >= d4) continue;
-              if (from_embed) {
-                if (S.slot[s].active) {
-                  const uint2 e2 = __ldg(reinterpret_cast<const uint2*>(A.embed + (size_t)S.slot[s].tok * d) + tid);
-                  xv[s] = make_float4(__uint_as_float(e2.x << 16), __uint_as_float(e2.x & 0xFFFF0000u),
-                                      __uint_as_float(e2.y << 16), __uint_as_float(e2.y & 0xFFFF0000u));
-                  ss[s] = fmaf(xv[s].x, xv[s].x, fmaf(xv[s].y, xv[s].y, fmaf(xv[s].z, xv[s].z, xv[s].w * xv[s].w)));
-                }
-              } else {
-                const int src = (kind == KIND_LM) ? S.lm_src[s] : s;
-                if (kind == KIND_LM || S.slot[s].active) xv[s] = __ldcg(reinterpret_cast<const float4*>(xbuf + (size_t)src * d) + tid);
+          for (int j = 0; j < 2; ++j) {
+            const int item = it0 + j * kPT + tid;
+            xv[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            gv[j] = make_uint2(0u, 0u);
+            ss[j] = -1;
+            if (item < total) {
+              const int s = item / d4, e4 = item - s * d4;
+              const int src = (kind == KIND_LM) ? S.lm_src[s] : s;
+              ss[j] = s * 65536 + e4;
+              gv[j] = __ldg(reinterpret_cast<const uint2*>(gain) + e4);
+              if (kind == KIND_LM || S.slot[s].active) {
+                if (from_embed) xv[j] = bf16x4_to_float4(__ldg(reinterpret_cast<const uint2*>(A.embed + (size_t)S.slot[s].tok * d) + e4));
+                else xv[j] = __ldcg(reinterpret_cast<const float4*>(xbuf + (size_t)src * d) + e4);
               }
-            }
-            if (!from_embed && tid < NC) {
-              // partial sums of squares left by the resolve phase, one set per CTA
-              const float4 p0 = __ldcg(reinterpret_cast<const float4*>(A.ssq + (size_t)tid * kPSlots));
-              const float4 p1 = __ldcg(reinterpret_cast<const float4*>(A.ssq + (size_t)tid * kPSlots) + 1);
-              ss[0] = p0.x; ss[1] = p0.y; ss[2] = p0.z; ss[3] = p0.w; ss[4] = p1.x; ss[5] = p1.y; ss[6] = p1.z; ss[7] = p1.w;
-            }
-#pragma unroll
-            for (int s = 0; s < kPSlots; ++s) ss[s] = warp_sum_f32(ss[s]);
-            if (lane == 0) {
-#pragma unroll
-              for (int s = 0; s < kPSlots; ++s) S.red[warp][s] = ss[s];
-            }
-            __syncthreads();
-            if (tid < kPSlots) {
-              float tot = 0.0f;
-#pragma unroll
-              for (int w2 = 0; w2 < kPW; ++w2) tot += S.red[w2][tid];
-              S.scale[tid] = 1.0f / sqrtf(tot / (float)d + A.eps);
-            }
-            __syncthreads();
-            const int e0 = tid * 4;
-            if (tid < d4 && e0 >= k0 && e0 < k0 + g.kchunk) {
-              const float g0 = __uint_as_float(g2.x << 16), g1 = __uint_as_float(g2.x & 0xFFFF0000u);
-              const float g2f = __uint_as_float(g2.y << 16), g3 = __uint_as_float(g2.y & 0xFFFF0000u);
-#pragma unroll
-              for (int s = 0; s < kPSlots; ++s) {
-                if (s >= n_in) continue;
-                const float sc = S.scale[(kind == KIND_LM) ? S.lm_src[s] : s];
-                uint2 pk;
-                pk.x = pack_bf16(xv[s].x * sc * g0, xv[s].y * sc * g1);
-                pk.y = pack_bf16(xv[s].z * sc * g2f, xv[s].w * sc * g3);
-                *reinterpret_cast<uint2*>(act + s * apitch + (e0 - k0)) = pk;
-              }
-            }
-          } else {
-            const float* src = (kind == KIND_O) ? A.attn_out : A.mid;
-            const int stride = (kind == KIND_O) ? HD : A.F;
-            const int nvec = g.kchunk >> 2;
-            for (int idx = tid; idx < n_in * nvec; idx += kPT) {
-              const int s = idx / nvec, j = (idx - s * nvec) << 2;
-              const float4 v = __ldcg(reinterpret_cast<const float4*>(src + (size_t)s * stride + k0 + j));
-              uint2 pk;
-              pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
-              *reinterpret_cast<uint2*>(act + s * apitch + j) = pk;
             }
           }
-          cur_ks = ks;
+          if (it0 == 0) {
+            // statistics: warp w owns slot w
+            if (warp < kPSlots) {
+              float sq = 0.0f;
+              if (from_embed) {
+                if (warp < ns && S.slot[warp].active) {
+                  const uint2* er = reinterpret_cast<const uint2*>(A.embed + (size_t)S.slot[warp].tok * d);
+#pragma unroll 1
+                  for (int e4 = lane; e4 < d4; e4 += 32) {
+                    const float4 v = bf16x4_to_float4(__ldg(er + e4));
+                    sq = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, sq))));
+                  }
+                }
+              } else {
+#pragma unroll 1
+                for (int t = lane; t < (d >> 4); t += 32) sq += __ldcg(A.ssq + (size_t)t * kPSlots + warp);
+              }
+              sq = warp_sum_f32(sq);
+              if (lane == 0) S.scale[warp] = 1.0f / sqrtf(sq / (float)d + A.eps);
+            }
+            __syncthreads();
+          }
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (ss[j] < 0) continue;
+            const int s = ss[j] >> 16, e4 = ss[j] & 65535;
+            const float sc = S.scale[(kind == KIND_LM) ? S.lm_src[s] : s];
+            const float4 gf = bf16x4_to_float4(gv[j]);
+            uint2 pk;
+            pk.x = pack_bf16(xv[j].x * sc * gf.x, xv[j].y * sc * gf.y);
+            pk.y = pack_bf16(xv[j].z * sc * gf.z, xv[j].w * sc * gf.w);
+            *reinterpret_cast<uint2*>(act + s * apitch + e4 * 4) = pk;
+          }
+        }
+        __syncthreads();
+      } else if (kind == KIND_O && ka < kb) {
+        // ---- stage the attention output, whole rows ------------------------------------------------
+        const int nvec = g.kchunk >> 2;
+#pragma unroll 1
+        for (int idx = tid; idx < n_in * nvec; idx += kPT) {
+          const int s = idx / nvec, j = (idx - s * nvec) << 2;
+          const float4 v = __ldcg(reinterpret_cast<const float4*>(A.attn_out + (size_t)s * HD + j));
+          uint2 pk;
+          pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
+          *reinterpret_cast<uint2*>(act + s * apitch + j) = pk;
+        }
+        __syncthreads();
+      }
+      TSEC(0);
+
+      // ---- units of this CTA: rounds of kWG units, one per warp group --------------------------------
+      float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      float lm_max = -INFINITY;
+      const int nsub_eff = g.nsub < kWG ? g.nsub : kWG;       // groups that share one tile in a round
+#pragma unroll 1
+      for (unsigned k0 = ka; k0 < kb; k0 += kWG) {
+        const unsigned k = k0 + (unsigned)wgrp;
+        const bool has = k < kb;
+        int u = 0, sub = 0;
+        if (has) { u = (int)(S.ulist[k - (unsigned)step * per_step] >> 10); sub = u % g.nsub; }
+        if (kind == KIND_DN) {
+          // stage this round's chunks of the gated product: area of group w <- columns of its sub-unit
+          const int nvec = g.kchunk >> 2;
+#pragma unroll 1
+          for (int idx = tid; idx < kWG * n_in * nvec; idx += kPT) {
+            const int w2 = idx / (n_in * nvec), r2 = idx - w2 * (n_in * nvec);
+            const int s = r2 / nvec, j = (r2 - s * nvec) << 2;
+            const unsigned kq = k0 + (unsigned)w2;
+            if (kq < kb) {
+              const int sq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10) % g.nsub;
+              const float4 v = __ldcg(reinterpret_cast<const float4*>(A.mid + (size_t)s * A.F + (size_t)sq * g.kchunk + j));
+              uint2 pk;
+              pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
+              *reinterpret_cast<uint2*>(act + w2 * area_elems + s * apitch + j) = pk;
+            }
+          }
           __syncthreads();
           TSEC(0);
         }
-        const int slot = (int)(cons_i % (unsigned)A.n_ring);
-        const unsigned parity = (cons_i / (unsigned)A.n_ring) & 1u;
-        const bool landed = wait_full(S, slot, parity, A.err);
+        bool landed = true;
+        if (has) {
+          const int slot = (int)(k % (unsigned)A.n_ring);
+          landed = wait_full(S, slot, (k / (unsigned)A.n_ring) & 1u, A.err);
+        }
         if (__syncthreads_or(!landed)) { alive = false; goto drain; }
         TSEC(1);
-        const unsigned char* tile_s = ring + (size_t)slot * A.slot_bytes;
-        const uint32_t tpitch = (uint32_t)g.kchunk * 2u + 16u;
-        float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        {
+        if (has) {
+          if (sub < kWG) { c[0] = 0.0f; c[1] = 0.0f; c[2] = 0.0f; c[3] = 0.0f; }     // first round of a tile
+          const unsigned char* tile_s = ring + (size_t)(k % (unsigned)A.n_ring) * A.slot_bytes;
+          const uint32_t tpitch = (uint32_t)g.kchunk * 2u + 16u;
+          const __nv_bfloat16* act_g = act + ((kind == KIND_DN) ? wgrp * area_elems : 0);
           const uint32_t a_base = smem_u32(tile_s) + (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * tpitch + (uint32_t)(lane >> 4) * 16u;
-          const uint32_t b_base = smem_u32(act) + (uint32_t)(lane & 7) * (uint32_t)apitch * 2u + (uint32_t)((lane >> 3) & 1) * 16u;
+          const uint32_t b_base = smem_u32(act_g) + (uint32_t)(lane & 7) * (uint32_t)apitch * 2u + (uint32_t)((lane >> 3) & 1) * 16u;
           const int nkb = g.kchunk >> 4;
-          for (int kb = warp; kb < nkb; kb += kPW) {
+#pragma unroll 2
+          for (int kblk = wl; kblk < nkb; kblk += kGW) {
             uint32_t a[4], bfr[2];
-            ldsm_x4(a, a_base + (uint32_t)kb * 32u);
-            ldsm_x2(bfr, b_base + (uint32_t)kb * 32u);
+            ldsm_x4(a, a_base + (uint32_t)kblk * 32u);
+            ldsm_x2(bfr, b_base + (uint32_t)kblk * 32u);
             mma_bf16(c, a, bfr);
           }
         }
-        float* cp = cpart + (size_t)(cons_i & 1u) * (kPW * 128);
+        float* cp = cpart + (size_t)((k0 / kWG) & 1u) * (kPW * 128);
         {
           const int gq = lane >> 2, tq = lane & 3;
           float* w0 = cp + warp * 128;
           *reinterpret_cast<float2*>(w0 + gq * 8 + tq * 2) = make_float2(c[0], c[1]);
           *reinterpret_cast<float2*>(w0 + (gq + 8) * 8 + tq * 2) = make_float2(c[2], c[3]);
         }
-        __syncthreads();                        // slot fully read, partial tiles complete
+        __syncthreads();                        // slots fully read, partial tiles complete
         TSEC(2);
-        ++cons_i;
-        if (tid == 0) {                         // refill the slot that was just released ...
-          UnitRef ur;
-          if (next_unit(A, cta, NC, pc, ur)) {
-            issue_unit(A, ur, ring + (size_t)slot * A.slot_bytes, &S.full[slot]);
-            ++prod_i;
-          }
-          TSEC(3);
+        if (has && wl == 0 && lane == 0) {      // refill the slot this group has just released
+          const unsigned kn = k + (unsigned)A.n_ring;
+          if (kn < total_units) issue_unit(A, S, ring, kn, per_step);
         }
-        if (warp >= 1 && warp <= 4) {           // ... while warps 1-4 sum the partial tiles and store
-          const int et = tid - 32;
-          const int r = et & 15, n = et >> 4;
+        cons_done = (kb < k0 + kWG) ? kb : k0 + kWG;
+        // epilogue: thread (group q, row r, slot n); the first group of a tile's set sums the set's warps
+        {
+          const int q = tid >> 7, e = tid & 127, r = e & 15, n = e >> 4;
+          const unsigned kq = k0 + (unsigned)q;
+          int uq = 0, sq = 0;
+          const bool on = kq < kb;
+          if (on) { uq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10); sq = uq % g.nsub; }
+          const bool lead = on && (q % nsub_eff) == 0 && (sq + nsub_eff == g.nsub);   // tile complete in this round
+          const int tile = uq / g.nsub;
+          const bool slot_on = n < n_in && (kind == KIND_LM || S.slot[n].active);
+          const int o = tile * 16 + r;
+          float base = 0.0f;
+          if (lead && slot_on && (kind == KIND_O || kind == KIND_DN))
+            base = __ldcg((kind == KIND_O ? A.xa : A.x1) + (size_t)n * d + o);
           float v = 0.0f;
-#pragma unroll
-          for (int w2 = 0; w2 < kPW; ++w2) v += cp[w2 * 128 + r * 8 + n];
+          if (lead) {
+            const int w_hi = (q + nsub_eff) * kGW;
+#pragma unroll 1
+            for (int w2 = q * kGW; w2 < w_hi; ++w2) v += cp[w2 * 128 + r * 8 + n];
+          }
           if (kind == KIND_GU) {
             const float up = __shfl_down_sync(0xffffffffu, v, 8);
-            if (r < 8 && n < n_in && S.slot[n].active)
-              A.mid[(size_t)n * A.F + tile * 8 + r] = v / (1.0f + expf(-v)) * up;
+            if (lead && r < 8 && slot_on) A.mid[(size_t)n * A.F + tile * 8 + r] = v / (1.0f + expf(-v)) * up;
           } else if (kind == KIND_LM) {
-            const int vi = tile * 16 + r;
-            float mx = (vi < V && n < n_in) ? v : -INFINITY;
+            if (lead && slot_on && o < V) {
+              A.logits_own[((size_t)step * R + n) * V + o] = v;
+              lm_max = fmaxf(lm_max, v);
+            }
+          } else if (kind == KIND_QKV) {
+            if (lead && slot_on) A.qkv[(size_t)n * A.qkv_w + o] = v;
+          } else {
+            // residual add + this tile's share of the next RMSNorm's sum of squares
+            const float xn = base + v;
+            float sq2 = (lead && slot_on) ? xn * xn : 0.0f;
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            lm_max = fmaxf(lm_max, mx);
-            if (vi < V && n < n_in) A.logits_own[((size_t)step * R + n) * V + vi] = v;
-          } else if (n < n_in && S.slot[n].active) {
-            const int o = tile * 16 + r;
-            if (kind == KIND_QKV) A.pq[((size_t)ks * kPSlots + n) * A.qkv_w + o] = v;
-            else if (kind == KIND_O) A.po[((size_t)ks * kPSlots + n) * d + o] = v;
-            else A.pd[((size_t)ks * kPSlots + n) * d + o] = v;
+            for (int o2 = 8; o2 > 0; o2 >>= 1) sq2 += __shfl_xor_sync(0xffffffffu, sq2, o2);
+            if (lead && slot_on) {
+              (kind == KIND_O ? A.x1 : A.xa)[(size_t)n * d + o] = xn;
+              if (r == 0) A.ssq[(size_t)tile * kPSlots + n] = sq2;
+            }
           }
         }
+        TSEC(3);
       }
-      off = (off + g.n_units) % NC;
-      if (kind == KIND_LM && warp >= 1 && warp <= 4 && ((tid - 32) & 15) == 0 && ((tid - 32) >> 4) < R && lm_max > -INFINITY)
-        atomicMax(A.rowmax + step * R + ((tid - 32) >> 4), ord_encode(lm_max));
-      GRID_SYNC();
-
-      // ---- resolve: residual + split-K partials of the phase just finished, this CTA's slice --------
-      if (kind == KIND_O || kind == KIND_DN) {
-        const float* basebuf = (kind == KIND_O) ? A.xa : A.x1;
-        float* outbuf = (kind == KIND_O) ? A.x1 : A.xa;
-        const float* part = (kind == KIND_O) ? A.po : A.pd;
-        const int wsl = hi - lo, terms = g.KS + 1;
-        // thread -> (term t = tid/128 + 4*it, slot s, element j): all loads of a thread are independent
-        constexpr int kIt = (17 + 3) / 4;
-        const int rs = (tid >> 4) & (kPSlots - 1), rj = tid & (kResW - 1), rt0 = tid >> 7;
-        const bool r_on = rs < ns && rj < wsl && S.slot[rs].active;
-        float val[kIt];
+      if (kind == KIND_LM) {
+        // running maxima of the logits: 16 lanes of a slot, then the CTA, then one atomic per row
 #pragma unroll
-        for (int it = 0; it < kIt; ++it) {
-          const int t = rt0 + it * 4;
-          val[it] = 0.0f;
-          if (r_on && t < terms)
-            val[it] = (t == 0) ? __ldcg(basebuf + (size_t)rs * d + lo + rj)
-                               : __ldcg(part + ((size_t)(t - 1) * kPSlots + rs) * d + lo + rj);
-        }
-#pragma unroll
-        for (int it = 0; it < kIt; ++it) {
-          const int t = rt0 + it * 4;
-          if (t < terms) rbuf[(t * kPSlots + rs) * kResW + rj] = val[it];
-        }
+        for (int o2 = 8; o2 > 0; o2 >>= 1) lm_max = fmaxf(lm_max, __shfl_xor_sync(0xffffffffu, lm_max, o2));
+        const int n = (tid & 127) >> 4;
+        if ((tid & 15) == 0 && n < R && lm_max > -INFINITY) atomicMax(&S.lmmax[n], ord_encode(lm_max));
         __syncthreads();
-        if (tid < kPSlots * kResW) {
-          const int s = tid / kResW, j = tid - s * kResW;
-          float sq = 0.0f;
-          if (s < ns && j < wsl && S.slot[s].active) {
-            float v = 0.0f;
-            for (int t = 0; t < terms; ++t) v += rbuf[(t * kPSlots + s) * kResW + j];
-            outbuf[(size_t)s * d + lo + j] = v;
-            sq = v * v;
-          }
-#pragma unroll
-          for (int o = kResW / 2; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-          if (j == 0) A.ssq[(size_t)cta * kPSlots + s] = sq;
-        }
-        GRID_SYNC();
+        if (tid < R && S.lmmax[tid] != 0u) atomicMax(A.rowmax + step * R + tid, S.lmmax[tid]);
       }
+      GRID_SYNC();
 
       // ---- attention over the rows' caches (after the QKV phase) -----------------------------------
       if (kind == KIND_QKV) {
-        const int KSq = A.geom[KIND_QKV].KS;
         const int split_len = A.split_len;
         const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
         const int PPW = 32 / LPR, PPB = kPW * PPW;     // positions per warp / per CTA pass
         const int sub = lane % LPR, pgrp = lane / LPR;
         int total_items = 0;
+#pragma unroll 1
         for (int s = 0; s < ns; ++s)
           if (S.slot[s].active) total_items += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
+#pragma unroll 1
         for (int item = cta; item < total_items; item += NC) {
           int s = 0, rem = item, nsplit = 0;
+#pragma unroll 1
           for (; s < ns; ++s) {
             nsplit = S.slot[s].active ? (S.slot[s].pos + split_len) / split_len : 0;
             if (rem < A.Hkv * nsplit) break;
@@ -674,10 +715,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             if (p < cnt && p_lo + p < fresh_lo)
               vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(vbase + (size_t)(p_lo + p) * A.hd + sub * 8));
           }
-          // stage q (all heads of the group), fresh k and v: split-K sums, RoPE, bf16 rounding.
+          // stage q (all heads of the group), fresh k and v: RoPE, bf16 rounding.
           // One index space so that every element is fetched by a different thread in one round trip.
           {
             const int n_q = grp * half, n_k = n_fresh * half, n_v = n_fresh * A.hd;
+#pragma unroll 1
             for (int idx = tid; idx < n_q + n_k + n_v; idx += kPT) {
               int sj, col, pj, i;
               float* dst;
@@ -692,15 +734,10 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
                 const int j = (idx - n_q - n_k) / A.hd; i = (idx - n_q - n_k) - j * A.hd;
                 sj = s - j * R; pj = pos; col = d + kvd + gk * A.hd + i; dst = &S.vf[j][i]; pair = false;
               }
-              float cs = 1.0f, sn = 0.0f;
-              if (pair) { cs = A.rope_cos[(size_t)pj * half + i]; sn = A.rope_sin[(size_t)pj * half + i]; }
-              float x1 = 0.0f, x2 = 0.0f;
-#pragma unroll 1
-              for (int ks = 0; ks < KSq; ++ks) {
-                const float* pr = A.pq + ((size_t)ks * kPSlots + sj) * A.qkv_w + col;
-                x1 += __ldcg(pr);
-                if (pair) x2 += __ldcg(pr + half);
-              }
+              const float* pr = A.qkv + (size_t)sj * A.qkv_w + col;
+              float cs = 1.0f, sn = 0.0f, x2 = 0.0f;
+              if (pair) { cs = A.rope_cos[(size_t)pj * half + i]; sn = A.rope_sin[(size_t)pj * half + i]; x2 = __ldcg(pr + half); }
+              const float x1 = __ldcg(pr);
               dst[0] = round_bf16(x1 * cs - x2 * sn);
               if (pair) dst[half] = round_bf16(x2 * cs + x1 * sn);
             }
@@ -726,16 +763,19 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               float dd = 0.0f;
 #pragma unroll
               for (int e = 0; e < 8; ++e) dd = fmaf(kf8[e], qf[e], dd);
+#pragma unroll 1
               for (int o = LPR >> 1; o > 0; o >>= 1) dd += __shfl_xor_sync(0xffffffffu, dd, o);
               if (sub == 0 && p < cnt && p_lo + p < fresh_lo) S.sc[t][p] = dd * A.attn_scale;
             }
           }
           // scores of the fresh positions come from the staged k, not from the cache
+#pragma unroll 1
           for (int combo = warp; combo < grp * n_fresh; combo += kPW) {
             const int t = combo / n_fresh, j = combo - t * n_fresh;
             const int pj = pos - j;
             if (pj >= p_lo && pj < p_hi) {
               float dd = 0.0f;
+#pragma unroll 1
               for (int i = lane; i < A.hd; i += 32) dd = fmaf(S.kf[j][i], S.q[t][i], dd);
               dd = warp_sum_f32(dd);
               if (lane == 0) S.sc[t][pj - p_lo] = dd * A.attn_scale;
@@ -754,7 +794,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             float sum = 0.0f;
             if (t < grp) {
               mx = S.red[t * wph][0];
+#pragma unroll 1
               for (int w2 = 1; w2 < wph; ++w2) mx = fmaxf(mx, S.red[t * wph + w2][0]);
+#pragma unroll 1
               for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) { const float e = expf(S.sc[t][p] - mx); S.sc[t][p] = e; sum += e; }
             }
             sum = warp_sum_f32(sum);
@@ -762,6 +804,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             __syncthreads();
             if (t < grp && wi == 0 && lane == 0) {
               float tot = 0.0f;
+#pragma unroll 1
               for (int w2 = 0; w2 < wph; ++w2) tot += S.red[t * wph + w2][1];
               S.m_[t] = mx; S.l_[t] = tot;
             }
@@ -788,6 +831,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               float v = oacc[e];
+#pragma unroll 1
               for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
               oacc[e] = v;
             }
@@ -798,11 +842,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           __syncthreads();
           const bool single = nsplit == 1;
+#pragma unroll 1
           for (int idx = tid; idx < grp * A.hd; idx += kPT) {
             const int t = idx / A.hd, dd = idx - t * A.hd;
             float v = 0.0f;
 #pragma unroll
             for (int w2 = 0; w2 < kPW; ++w2) v += s_o[((size_t)w2 * grp + t) * A.hd + dd];
+#pragma unroll 1
             for (int j = 0; j < n_fresh; ++j) {
               const int pj = pos - j;
               if (pj >= p_lo && pj < p_hi) v = fmaf(S.sc[t][pj - p_lo], S.vf[j][dd], v);
@@ -825,12 +871,15 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             __syncthreads();
             if (S.flag) {
               __threadfence();
+#pragma unroll 1
               for (int t = warp; t < grp; t += kPW) {      // rescaling factors of the splits, one warp per head
                 const size_t base = ((size_t)s * A.H + gk * grp + t) * A.max_splits;
                 float M = -INFINITY;
+#pragma unroll 1
                 for (int j = lane; j < nsplit; j += 32) M = fmaxf(M, __ldcg(A.part_ml + (base + j) * 2));
                 M = warp_max_f32(M);
                 float den = 0.0f;
+#pragma unroll 1
                 for (int j = lane; j < nsplit; j += 32) {
                   const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + j) * 2));
                   const float f = expf(ml.x - M);
@@ -841,6 +890,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
                 if (lane == 0) S.l_[t] = den;
               }
               __syncthreads();
+#pragma unroll 1
               for (int idx = tid; idx < grp * A.hd; idx += kPT) {
                 const int t = idx / A.hd, dd = idx - t * A.hd;
                 const int head = gk * grp + t;
@@ -870,6 +920,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       if (A.logits_override) {                        // the maxima gathered by the LM head belong to other logits
         if (cta == 0 && tid < R) rowmax[tid] = 0u;
         GRID_SYNC();
+#pragma unroll 1
         for (int item = cta; item < R * n_chunks; item += NC) {
           const int row = item / n_chunks, ch = item - row * n_chunks;
           float a[kPPer];
@@ -880,6 +931,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         }
         GRID_SYNC();
       }
+#pragma unroll 1
       for (int item = cta; item < R * n_chunks; item += NC) {
         const int row = item / n_chunks, ch = item - row * n_chunks;
         const int v0 = ch * kChunk + tid * kPPer;
@@ -893,6 +945,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         if (tid == 0 && sm) atomicAdd(rowsum + row, sm);
       }
       GRID_SYNC();
+#pragma unroll 1
       for (int item = cta; item < B * n_chunks; item += NC) {
         const int b = item / n_chunks, ch = item - b * n_chunks;
         const int v0 = ch * kChunk + tid * kPPer;
@@ -944,6 +997,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           if (lane == 0) { S.bestv[warp] = bv; S.besti[warp] = bi; }
           __syncthreads();
           if (tid == 0) {
+#pragma unroll 1
             for (int i = 1; i < kPW; ++i)
               if (S.bestv[i] > bv || (S.bestv[i] == bv && S.besti[i] < bi)) { bv = S.bestv[i]; bi = S.besti[i]; }
             A.chunk_best[(size_t)b * n_chunks + ch] = ChunkBest{bv, bi};
@@ -952,9 +1006,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       }
       GRID_SYNC();
       // every CTA locates the drawn token itself (the next step's embedding gather needs it)
+#pragma unroll 1
       for (int b = 0; b < B; ++b) {
         if (A.greedy) {
           float bv = -1.0f; int bi = 0x7fffffff;
+#pragma unroll 1
           for (int c2 = tid; c2 < n_chunks; c2 += kPT) {
             ChunkBest cb;
             *reinterpret_cast<unsigned long long*>(&cb) =
@@ -971,6 +1027,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           if (lane == 0) { S.bestv[warp] = bv; S.besti[warp] = bi; }
           __syncthreads();
           if (tid == 0) {
+#pragma unroll 1
             for (int i = 1; i < kPW; ++i)
               if (S.bestv[i] > bv || (S.bestv[i] == bv && S.besti[i] < bi)) { bv = S.bestv[i]; bi = S.besti[i]; }
             S.tok[b] = bi;
@@ -981,6 +1038,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         const unsigned long long* cm = A.chunk_mass + (size_t)b * n_chunks;
         // chunk masses in parallel into shared memory, then one thread walks them
         unsigned long long T = 0;
+#pragma unroll 1
         for (int c0 = 0; c0 < n_chunks; c0 += kPT) {
           const unsigned long long mine = (c0 + tid < n_chunks) ? __ldcg(cm + c0 + tid) : 0ull;
           T += block_sum_u64_p(mine, S);
@@ -994,6 +1052,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             const unsigned long long thr = draw_threshold(A.u[b * G + step], T);
             int c2 = 0;
             unsigned long long pre = 0;
+#pragma unroll 1
             for (; c2 < n_chunks - 1; ++c2) {
               const unsigned long long nx = pre + (n_chunks <= kPT ? S.cm[c2] : __ldcg(cm + c2));
               if (nx > thr) break;
@@ -1022,6 +1081,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           if (lane == 31) S.red64[warp] = incl;
           __syncthreads();
           unsigned long long wpre = 0;
+#pragma unroll 1
           for (int i = 0; i < warp; ++i) wpre += S.red64[i];
           unsigned long long run = wpre + incl - tsum;
           if (run <= thr) {
@@ -1052,9 +1112,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   return;
 
 drain:
-  // a wait ran out: let the copies already issued land before the shared memory is released
+  // a wait ran out: let the copies already issued land before the shared memory is released.
+  // Units below cons_done have been consumed; every consumed unit k had unit k + n_ring issued.
   if (tid == 0) {
-    for (unsigned k = cons_i; k < prod_i; ++k) {
+    unsigned hi = cons_done + (unsigned)A.n_ring;
+    if (hi > total_units) hi = total_units;
+#pragma unroll 1
+    for (unsigned k = cons_done; k < hi; ++k) {
       const int slot = (int)(k % (unsigned)A.n_ring);
       const unsigned parity = (k / (unsigned)A.n_ring) & 1u;
       unsigned spins = 0;

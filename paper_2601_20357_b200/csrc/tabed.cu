@@ -76,7 +76,7 @@ struct tabed_handle {
   int n_cta = 0; size_t persist_smem = 0;
   unsigned launches_persist = 0;
   LayerW* layer_tab = nullptr;
-  float *xa = nullptr, *x1 = nullptr, *pq = nullptr, *po = nullptr, *pd = nullptr;
+  float *xa = nullptr, *x1 = nullptr;
   int* tickets = nullptr; unsigned* bar = nullptr; float* ssq = nullptr;
   unsigned char* packed = nullptr;
   uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
@@ -276,22 +276,15 @@ void run_ensemble(tabed_handle* h, const float* logits, const float* w, const fl
 }
 
 // ---- persistent drafting-round kernel: geometry and set-up -----------------------------------------
-// Split a [16*n_tiles][K] weight matrix into units of 16 rows x kchunk columns so that the busiest
-// CTA has as little to do as possible: cost = units per CTA x (columns per unit + fixed overhead).
-PhaseGeom pick_geom(int n_tiles, int K, int n_cta, int kcap, bool whole_rows) {
-  PhaseGeom best{n_tiles, 0, 0, 0};
-  long best_cost = -1;
+// Cut a [16*n_tiles][K] weight matrix into tiles of 16 rows; a tile whose rows are longer than kcap
+// becomes nsub sub-units (1, 2 or a multiple of 4, so that they line up with the 4 warp groups).
+PhaseGeom pick_geom(int n_tiles, int K, int kcap) {
   const int nkb = K / 16;
-  for (int ks = 1; ks <= 16; ++ks) {
-    if (nkb % ks) continue;
-    const int kchunk = K / ks;
-    if (kchunk > kcap) continue;
-    if (whole_rows && ks != 1) break;
-    const long units = (long)n_tiles * ks;
-    const long cost = ((units + n_cta - 1) / n_cta) * (kchunk + 128);
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = PhaseGeom{n_tiles, ks, kchunk, (int)units}; }
+  for (int nsub = 1; nsub <= 64; nsub = (nsub < 4) ? nsub * 2 : nsub + 4) {
+    if (nkb % nsub || K / nsub > kcap) continue;
+    return PhaseGeom{n_tiles, nsub, K / nsub, n_tiles * nsub};
   }
-  return best;
+  return PhaseGeom{n_tiles, 0, 0, 0};
 }
 
 // Decides whether the handle's drafter can run on the persistent kernel and allocates its buffers.
@@ -309,21 +302,30 @@ int setup_persistent(tabed_handle* h) {
   cudaFuncAttributes fa;
   if (cudaFuncGetAttributes(&fa, k_draft_round<true>) != cudaSuccess) return TABED_ERR_CUDA;
   const int n_cta = prop.multiProcessorCount;
-  if (n_cta > kPT || (h->d + n_cta - 1) / n_cta + 1 > kResW) return TABED_OK;
+  if (n_cta > kPT) return TABED_OK;
   RoundArgs& A = h->ra;
-  const int kcap = std::max(h->d, 1024);
-  A.geom[KIND_QKV] = pick_geom(h->qkv_w / 16, h->d, n_cta, kcap, false);
-  A.geom[KIND_O] = pick_geom(h->d / 16, h->H * h->hd, n_cta, kcap, false);
-  A.geom[KIND_GU] = pick_geom(h->F / 8, h->d, n_cta, kcap, true);
-  A.geom[KIND_DN] = pick_geom(h->d / 16, h->F, n_cta, kcap, false);
-  A.geom[KIND_LM] = pick_geom((h->V + 15) / 16, h->d, n_cta, kcap, true);
+  // QKV, O, gate/up and LM head rows are d_model long and stay whole; only the down projection is cut
+  A.geom[KIND_QKV] = pick_geom(h->qkv_w / 16, h->d, h->d);
+  A.geom[KIND_O] = pick_geom(h->d / 16, h->H * h->hd, h->d);
+  A.geom[KIND_GU] = pick_geom(h->F / 8, h->d, h->d);
+  A.geom[KIND_DN] = pick_geom(h->d / 16, h->F, std::max(h->d, 512));
+  A.geom[KIND_LM] = pick_geom((h->V + 15) / 16, h->d, h->d);
   int kmax = 0;
-  for (int k = 0; k < 5; ++k) { if (A.geom[k].KS == 0) return TABED_OK; kmax = std::max(kmax, A.geom[k].kchunk); }
+  long per_step = 0;                                  // upper bound of one CTA's units per decoder step
+  for (int k = 0; k < 5; ++k) {
+    if (A.geom[k].nsub == 0) return TABED_OK;
+    kmax = std::max(kmax, A.geom[k].kchunk);
+    per_step += (long)((A.geom[k].n_tiles + n_cta - 1) / n_cta) * A.geom[k].nsub * (k == KIND_LM ? 1 : h->L);
+  }
+  if (per_step > kMaxUnits) return TABED_OK;
   A.slot_bytes = 16 * (kmax * 2 + 16);
-  A.act_bytes = ((kPSlots * (kmax + 8) * 2) + 127) / 128 * 128;
+  A.act_slots = std::min(kPSlots, 2 * h->R);
+  const int dn_areas = std::min(A.geom[KIND_DN].nsub, kWG);
+  const size_t act_raw = std::max((size_t)A.act_slots * (h->d + 8) * 2, (size_t)dn_areas * A.act_slots * (A.geom[KIND_DN].kchunk + 8) * 2);
+  A.act_bytes = (int)((act_raw + 127) / 128 * 128);
   const size_t u_bytes = std::max<size_t>((size_t)A.act_bytes + 2 * kPW * 128 * sizeof(float), (size_t)kPW * 512 * sizeof(float));
   const size_t avail = (size_t)prop.sharedMemPerBlockOptin - fa.sharedSizeBytes - 1024;
-  if (avail < u_bytes + 2 * (size_t)A.slot_bytes) return TABED_OK;
+  if (avail < u_bytes + (size_t)kWG * A.slot_bytes) return TABED_OK;      // a round needs kWG units in flight
   A.n_ring = (int)std::min<size_t>(kPRing, (avail - u_bytes) / A.slot_bytes);
   h->persist_smem = (size_t)A.n_ring * A.slot_bytes + u_bytes;
   if (cudaFuncSetAttribute(k_draft_round<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess ||
@@ -338,9 +340,7 @@ int setup_persistent(tabed_handle* h) {
   auto A2 = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count); };
   const size_t d = h->d;
   A2(&h->layer_tab, (size_t)h->L); A2(&h->xa, kPSlots * d); A2(&h->x1, kPSlots * d);
-  A2(&h->pq, (size_t)A.geom[KIND_QKV].KS * kPSlots * h->qkv_w); A2(&h->po, (size_t)A.geom[KIND_O].KS * kPSlots * d);
-  A2(&h->pd, (size_t)A.geom[KIND_DN].KS * kPSlots * d);
-  A2(&h->tickets, (size_t)kPSlots * h->Hkv); A2(&h->bar, 2); A2(&h->ssq, (size_t)n_cta * kPSlots);
+  A2(&h->tickets, (size_t)kPSlots * h->Hkv); A2(&h->bar, 2); A2(&h->ssq, (size_t)(h->d / 16) * kPSlots);
   // private copy of the weights, unit by unit (one contiguous block per bulk copy)
   size_t unit_bytes[5], kind_bytes[5];
   for (int k = 0; k < 5; ++k) {
@@ -360,7 +360,7 @@ int setup_persistent(tabed_handle* h) {
     h->packed = reinterpret_cast<unsigned char*>(ptr);
   }
   A2(&h->rowmax_g, (size_t)h->G * h->R); A2(&h->rowsum_g, (size_t)h->G * h->R);
-  h->trace_stride = 7 * h->L + 8;
+  h->trace_stride = 5 * h->L + 8;
   A2(&h->trace, (size_t)h->G * h->trace_stride * kTraceRec);
   if (rc != TABED_OK) return rc;
   std::vector<LayerW> tab(h->L);
@@ -386,13 +386,13 @@ int setup_persistent(tabed_handle* h) {
     }
   }
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
-  A.layers = h->layer_tab; A.embed = (const bf*)h->embed; A.lm_head = (const bf*)h->lm_head; A.final_norm = (const bf*)h->final_norm;
+  A.layers = h->layer_tab; A.embed = (const bf*)h->embed; A.final_norm = (const bf*)h->final_norm;
   A.rope_cos = h->rope_cos; A.rope_sin = h->rope_sin;
   A.L = h->L; A.d = h->d; A.F = h->F; A.H = h->H; A.Hkv = h->Hkv; A.hd = h->hd; A.V = h->V; A.cap = h->cap; A.qkv_w = h->qkv_w;
   A.eps = c.rms_eps; A.attn_scale = 1.0f / sqrtf((float)h->hd);
   A.R = h->R; A.B = h->B; A.m = h->m; A.G = h->G; A.greedy = c.sample_mode == TABED_MODE_GREEDY;
   A.kv_len = h->kv_len; A.pending = h->pending; A.kc = (bf*)h->kc; A.vc = (bf*)h->vc;
-  A.xa = h->xa; A.x1 = h->x1; A.pq = h->pq; A.po = h->po; A.pd = h->pd; A.mid = h->mid; A.attn_out = h->attn_out;
+  A.xa = h->xa; A.x1 = h->x1; A.qkv = h->qkv; A.mid = h->mid; A.attn_out = h->attn_out;
   A.part_o = h->part_o; A.part_ml = h->part_ml; A.max_splits = h->max_splits; A.tickets = h->tickets;
   A.logits_own = h->logits_own; A.w = h->w; A.qk = h->qk; A.q = h->q;
   A.rowmax = h->rowmax_g; A.rowsum = h->rowsum_g; A.chunk_mass = h->chunk_mass; A.chunk_best = h->chunk_best;
