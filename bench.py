@@ -33,6 +33,12 @@ PAPER_CONTEXT = ("paper (A100 80GB, fp16): expected walltime speedup 1.74x over 
                  "~5% block-efficiency gain over single drafting; no rounds/s published")
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ ; keyed by (workload, kernel class).  Entries are removed when the kernel changes.
+NCU_TRAFFIC = {("llava_small", "draft_round"): {"bytes": 690.0e6, "algorithmic_bytes_of_that_launch": 698.3e6,
+                                                "source": "profiles/k_draft_round_llava_small_ncu_full.md"}}
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -45,7 +51,8 @@ def read_peaks():
 # clocks
 # --------------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """nvidia-smi in a loop (every 20 ms); only samples stamped inside [mark_begin, mark_end] are used."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -53,39 +60,55 @@ class ClockSampler:
         self.path = tempfile.mktemp(suffix=".csv")
         self.proc = None
         self.gpu_index = gpu_index
+        self.t0 = self.t1 = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            time.sleep(0.5)                      # let the first samples arrive before the timed region opens
         except OSError:
             self.proc = None
 
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
     def stop(self):
+        import datetime
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, all_sm = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                f_sm, f_mx = float(parts[1]), float(parts[2])
             except ValueError:
                 continue
+            all_sm.append(f_sm)
+            if self.t0 is not None and not (self.t0 - 0.02 <= ts <= self.t1 + 0.02):
+                continue
+            sm.append(f_sm); mx.append(f_mx)
             for nm, val in zip(names, parts[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         os.unlink(self.path)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": float(np.median(sm)) if sm else (float(np.median(all_sm)) if all_sm else None),
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "samples_total": len(all_sm),
+                "reasons": sorted(reasons)}
 
 
 # --------------------------------------------------------------------------------------------------
@@ -286,6 +309,8 @@ def run_ours(args, wl):
         g.verify(targets[r], u[r][1], u[r][2], a, z)
         g.update_weights(w, am)
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for r in range(Wm):
         flush.zero_()
         one_round(r)
@@ -293,13 +318,12 @@ def run_ours(args, wl):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(device)
-    sampler = ClockSampler(local)
-    sampler.start()
     launches0 = g.launch_count()
     persistent = g.current_path() == TB.PATH_PERSISTENT
     top_cls, top_name, top_kernel = ((TB.PROF_DRAFT_ROUND, "draft_round", "k_draft_round (persistent: gamma decoder steps + ensemble)")
                                      if persistent else (TB.PROF_LM_HEAD, "lm_head", "k_gemv (LM head)"))
     g.profile_begin(top_cls)
+    sampler.mark_begin()
     wall0 = time.perf_counter()
     for i in range(K):
         flush.zero_()                       # the target model's pass between rounds evicts L2 in deployment
@@ -309,6 +333,7 @@ def run_ours(args, wl):
     head_ms, head_n = g.profile_end()       # synchronises the stream
     torch.cuda.synchronize(device)
     wall = time.perf_counter() - wall0
+    sampler.mark_end()
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(device)
@@ -391,7 +416,8 @@ def run_ours(args, wl):
         mhz = float(clocks.get("sm_mhz") or 1965.0)
         with open(args.trace, "w") as f:
             f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA 0): us from the previous grid barrier to this one,\n"
-                    f"# then CTA 0's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue, epilogue/other, barrier\n")
+                    f"# then CTA 0's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
+                    f"# (attention phases: load+stage q/k/v, scores+softmax, PV+write, split merge, -, barrier)\n")
             prev = None
             for st in range(G):
                 for j in range(nb_step):
@@ -423,7 +449,9 @@ def run_ours(args, wl):
         "block_efficiency": mean_accept + 1.0,
         "wall_ms_per_step_incl_flush": 1000.0 * wall / K,
         "roofline": {"kernel": top_kernel, "bound": "hbm", "achieved": head_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": head_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                     "frac": head_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": (NCU_TRAFFIC.get((wl.name, top_name)) or {}).get("bytes"),
+                     "traffic_note": NCU_TRAFFIC.get((wl.name, top_name)),
                      "avg_us": 1000.0 * head_dur, "launches_timed": head_n, "bytes_per_launch": int(cb[top_name])},
         "round_roofline": {"bytes_per_round": int(cb["draft_round"] + cb["verify"] + cb["update"]),
                            "note": "algorithmic bytes of one round / measured round time / peak"},
@@ -446,7 +474,7 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="llava_small", choices=sorted(W.WORKLOADS))
