@@ -248,6 +248,16 @@ int tabed_ensemble_step_static(const float* logits, const float* w, const float*
                                int32_t n_inputs, int32_t vocab, int32_t sample_mode, int32_t device,
                                void* stream, int32_t* y, float* q, float* qk);
 
+/* Stand-alone run of the tensor-core projection used for many shared-weight rows (Sec. 4.1 "batched
+ * inference": all rows share the parameters, so a projection is one weights x rows contraction):
+ * out[s][o] = sum_k w[o][k] * bf16(act[s][k]), fp32 accumulation.  w bf16 [rows][K], act float [n][K],
+ * out float [n][rows], all device pointers on `device`; K a multiple of 8, n <= 128; ks = number of
+ * splits of the input dimension (partial sums are added in split order).  Allocates and frees its
+ * own temporaries and synchronises the stream: a test and tuning aid, not part of the round.
+ * Errors: INVALID_ARG, CUDA, TIMEOUT (a bounded device-side wait ran out). */
+int tabed_debug_gemm_tc(const void* w, const float* act, int32_t rows, int32_t K, int32_t n, int32_t ks,
+                        float* out, int32_t device, void* stream);
+
 /* Replay aid: while set (non-NULL), tabed_draft_round still runs its own forward pass (caches and
  * TABED_VIEW_LOGITS are written as usual) but steps 6-7 of Algorithm 1 read these logits
  * float [G][B][m][V] instead, so that a recorded trajectory can be followed exactly while the

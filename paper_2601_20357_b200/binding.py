@@ -33,7 +33,7 @@ EXPORTS = [
     "tabed_draft_round", "tabed_draft_round_logits", "tabed_verify", "tabed_update_weights",
     "tabed_round_host", "tabed_debug_view", "tabed_debug_override_logits", "tabed_state_export", "tabed_state_import",
     "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end", "tabed_ensemble_step_static",
-    "tabed_select_path", "tabed_current_path", "tabed_debug_trace",
+    "tabed_select_path", "tabed_current_path", "tabed_debug_trace", "tabed_debug_gemm_tc",
 ]
 
 
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
         L.tabed_select_path.argtypes = [vp, i32]
         L.tabed_current_path.argtypes = [vp]
         L.tabed_debug_trace.argtypes = [vp, i32]
+        L.tabed_debug_gemm_tc.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, vp]
         L.tabed_launch_count.argtypes = [vp]
         L.tabed_launch_count.restype = C.c_int64
         for name in EXPORTS:
@@ -324,6 +325,16 @@ def weights_to_device(drafter, weights_np: Dict[str, object], device: torch.devi
     out: Dict[str, object] = {}
     for k, v in weights_np.items():
         out[k] = [conv(a) for a in v] if isinstance(v, list) else conv(v)
+    return out
+
+
+def debug_gemm_tc(w: torch.Tensor, act: torch.Tensor, ks: int = 1) -> torch.Tensor:
+    """tabed_debug_gemm_tc: out[s][o] = sum_k w[o][k] * bf16(act[s][k]) on the tcgen05 path.  w bf16 [rows][K], act float [n][K]."""
+    rows, K = w.shape
+    n = act.shape[0]
+    out = torch.empty((n, rows), dtype=torch.float32, device=w.device)
+    _check(lib().tabed_debug_gemm_tc(_ptr(w, torch.bfloat16, rows * K, "w", w.device), _ptr(act, torch.float32, n * K, "act", w.device),
+                                     rows, K, n, ks, out.data_ptr(), w.device.index or 0, None), "tabed_debug_gemm_tc")
     return out
 
 

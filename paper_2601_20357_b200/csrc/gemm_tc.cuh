@@ -1,0 +1,239 @@
+// Weight-shared projections for MANY rows (batched serving: 32 requests x 3 inputs = 96 shared-weight
+// rows, 192 slots when every request feeds two pending tokens): out[slot][o] = sum_k W[o][k] act[slot][k]
+// on the 5th-generation tensor cores.  With ~100 rows per weight byte this is a real dense
+// contraction (the SIMT path re-reads the weights once per 8 rows), so it runs as tcgen05.mma with
+// the accumulator in tensor memory:
+//
+//   D[128 weight rows][N slots] += A[128][16] * B[N][16]^T     (kind::f16, bf16 inputs, fp32 accumulate)
+//
+// * A work unit is (tile of 128 weight rows, range of input columns); split-K over the input
+//   dimension gives >= one unit per SM even for the 768-row projections.  Units write fp32 partial
+//   sums [k-split][slot][row]; the consumer of the projection adds them in k-split order (deterministic).
+// * Operands reach shared memory by bulk asynchronous copies (cp.async.bulk + mbarrier), three stages of
+//   128 input columns.  Both operands are stored in global memory already in the tensor core's canonical
+//   K-major, no-swizzle layout (8 rows x 16 bytes core matrices), so a stage is two contiguous copies and
+//   needs no tensor map: the weights are re-laid once at set-up (k_pack_tc), the activations by the kernel
+//   that normalises and rounds them (k_prep_act).
+// * One thread issues the copies and the MMAs; tcgen05.commit releases a stage / signals the epilogue;
+//   four warps read the accumulator with tcgen05.ld (warp w owns TMEM lanes 32w..32w+31) and store
+//   coalesced rows.  Every wait is bounded; on a timeout the CTA sets an error bit, drains and frees TMEM.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "round_kernel.cuh"   // PTX wrappers: mbarrier, bulk copy
+
+namespace tabed {
+
+constexpr int kTcM = 128;          // weight rows per tile (MMA M)
+constexpr int kTcKC = 128;         // input columns per pipeline stage
+constexpr int kTcStages = 3;
+constexpr int kTcThreads = 128;
+constexpr int kTcMaxN = 256;       // slots per launch (MMA N), a multiple of 16
+
+// Canonical K-major no-swizzle operand block of `rows` rows x kTcKC columns (bf16):
+// element (r, k) at ((k/8) * (rows/8) + r/8) * 128 + (r%8) * 16 + (k%8) * 2 bytes.
+__host__ __device__ inline size_t tc_block_bytes(int rows) { return (size_t)rows * kTcKC * 2; }
+
+struct TcGemmArgs {
+  const unsigned char* a_packed;   // [m_tiles][k_chunks] blocks of 128 rows
+  const unsigned char* b_packed;   // [k_chunks] blocks of n_pad rows
+  float* partial;                  // [ks][n_slots][rows_total]
+  int rows_total;                  // output rows of the projection (multiple of 128 after padding in a_packed)
+  int rows_valid;                  // rows actually stored
+  int n_pad, n_slots;              // MMA N (multiple of 16) / slots stored
+  int k_chunks;                    // chunks of 128 columns over the whole input dimension
+  int ks;                          // k-splits; unit (m_tile, split) covers chunks [split*cps, min((split+1)*cps, k_chunks))
+  int cps;                         // chunks per split
+  int* err;
+};
+
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  // shared-memory matrix descriptor: start address, leading (K) and stride (row group) byte offsets in
+  // 16-byte units, descriptor version 1 (bits 46-47), no swizzle (bits 61-63 = 0)
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, unsigned parity, int* err) {
+  unsigned spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if (++spins > (1u << 20)) { atomicOr(err, PERR_COPY); return false; }
+    if (spins > 2048) __nanosleep(64);
+  }
+  return true;
+}
+
+// grid (m_tiles * ks), block 128, dynamic shared memory kTcStages * (A block + B block) + 1 KB
+__global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
+  extern __shared__ __align__(1024) unsigned char tc_smem[];
+  __shared__ uint64_t s_full[kTcStages], s_empty[kTcStages], s_done;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_bad;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m_tile = blockIdx.x / G.ks, split = blockIdx.x - m_tile * G.ks;
+  const int c_lo = split * G.cps, c_hi = min(c_lo + G.cps, G.k_chunks), n_ch = c_hi - c_lo;
+  const size_t a_bytes = tc_block_bytes(kTcM), b_bytes = tc_block_bytes(G.n_pad);
+  const uint32_t tmem_cols = G.n_pad <= 32 ? 32u : (G.n_pad <= 64 ? 64u : (G.n_pad <= 128 ? 128u : 256u));
+
+  if (tid == 0) {
+    for (int s = 0; s < kTcStages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
+    mbar_init(&s_done, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_bad = 0;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+
+  if (tid == 0 && n_ch > 0) {
+    // instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N and M
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G.n_pad >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
+    const unsigned char* a_src = G.a_packed + ((size_t)m_tile * G.k_chunks + c_lo) * a_bytes;
+    const unsigned char* b_src = G.b_packed + (size_t)c_lo * b_bytes;
+    bool ok = true;
+    const int pre = n_ch < kTcStages ? n_ch : kTcStages;
+    for (int c = 0; c < pre; ++c) {
+      unsigned char* st = tc_smem + (size_t)c * (a_bytes + b_bytes);
+      mbar_expect_tx(&s_full[c], (unsigned)(a_bytes + b_bytes));
+      bulk_g2s(st, a_src + (size_t)c * a_bytes, (unsigned)a_bytes, &s_full[c]);
+      bulk_g2s(st + a_bytes, b_src + (size_t)c * b_bytes, (unsigned)b_bytes, &s_full[c]);
+    }
+    int issued = pre;
+    for (int c = 0; c < n_ch && ok; ++c) {
+      const int s = c % kTcStages;
+      ok = tc_wait(&s_full[s], (unsigned)(c / kTcStages) & 1u, G.err);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t a_s = smem_u32(tc_smem + (size_t)s * (a_bytes + b_bytes));
+      const uint32_t b_s = a_s + (uint32_t)a_bytes;
+      const uint32_t a_lbo = (kTcM / 8) * 128, b_lbo = (uint32_t)(G.n_pad / 8) * 128;
+#pragma unroll 1
+      for (int j = 0; j < kTcKC / 16; ++j) {
+        const uint64_t da = tc_smem_desc(a_s + (uint32_t)j * 2u * a_lbo, a_lbo, 128u);
+        const uint64_t db = tc_smem_desc(b_s + (uint32_t)j * 2u * b_lbo, b_lbo, 128u);
+        const uint32_t acc = (c > 0 || j > 0) ? 1u : 0u;
+        asm volatile(
+            "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+            " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+            ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+      }
+      // the stage may be refilled once these MMAs have read it
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_empty[s])) : "memory");
+      if (issued < n_ch) {
+        ok = tc_wait(&s_empty[s], (unsigned)(c / kTcStages) & 1u, G.err);
+        if (!ok) break;
+        unsigned char* st = tc_smem + (size_t)s * (a_bytes + b_bytes);
+        mbar_expect_tx(&s_full[s], (unsigned)(a_bytes + b_bytes));
+        bulk_g2s(st, a_src + (size_t)issued * a_bytes, (unsigned)a_bytes, &s_full[s]);
+        bulk_g2s(st + a_bytes, b_src + (size_t)issued * b_bytes, (unsigned)b_bytes, &s_full[s]);
+        ++issued;
+      }
+    }
+    if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_done)) : "memory");
+    else {
+      s_bad = 1;
+      // let the copies in flight land before the shared memory is released
+      for (int s = 0; s < kTcStages; ++s) {
+        unsigned spins = 0;
+        while (!mbar_try_wait(&s_full[s], 0) && !mbar_try_wait(&s_full[s], 1) && ++spins < (1u << 16)) __nanosleep(64);
+      }
+    }
+  }
+  __syncwarp();
+  bool done_ok = true;
+  if (n_ch > 0) {
+    // everybody waits for the accumulator (or for the issuing thread to give up)
+    unsigned spins = 0;
+    while (!mbar_try_wait(&s_done, 0)) {
+      if (*(volatile int*)&s_bad) { done_ok = false; break; }
+      if (++spins > (1u << 21)) { atomicOr(G.err, PERR_COPY); done_ok = false; break; }
+      if (spins > 2048) __nanosleep(64);
+    }
+  }
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (done_ok) {
+    const int row = m_tile * kTcM + warp * 32 + lane;
+    float* out = G.partial + (size_t)split * G.n_slots * G.rows_total + row;
+#pragma unroll 1
+    for (int c0 = 0; c0 < G.n_pad; c0 += 16) {
+      uint32_t v[16];
+      if (n_ch > 0) {
+        const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                       "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                     : "r"(taddr));
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = 0u;
+      }
+      if (row < G.rows_valid) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (c0 + j < G.n_slots) out[(size_t)(c0 + j) * G.rows_total] = __uint_as_float(v[j]);
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+}
+
+// ---- operand packing ------------------------------------------------------------------------------
+// Weights [rows][K] (one or two matrices concatenated: rows0 of w0 then rows1 of w1) -> blocks
+// [m_tile][k_chunk] in the canonical layout; rows beyond rows0+rows1 and columns beyond K are zero.
+// grid (k_chunks, m_tiles), block 256.
+__global__ void k_pack_tc(const __nv_bfloat16* __restrict__ w0, int rows0, const __nv_bfloat16* __restrict__ w1, int rows1,
+                          const __nv_bfloat16* __restrict__ w2, int rows2, int K, int k_chunks, unsigned char* __restrict__ dst) {
+  const int kc = blockIdx.x, mt = blockIdx.y;
+  unsigned char* blk = dst + ((size_t)mt * k_chunks + kc) * tc_block_bytes(kTcM);
+  for (int idx = threadIdx.x; idx < kTcM * (kTcKC / 8); idx += blockDim.x) {
+    const int r = idx % kTcM, k8 = idx / kTcM;
+    int row = mt * kTcM + r;
+    const int k = kc * kTcKC + k8 * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    const __nv_bfloat16* base = nullptr;
+    if (row < rows0) base = w0;
+    else if (row < rows0 + rows1) { base = w1; row -= rows0; }
+    else if (row < rows0 + rows1 + rows2) { base = w2; row -= rows0 + rows1; }
+    if (base && k < K) v = *reinterpret_cast<const uint4*>(base + (size_t)row * K + k);
+    *reinterpret_cast<uint4*>(blk + ((size_t)k8 * (kTcM / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
+  }
+}
+
+// Activations fp32 [n][K] (row stride `stride`) -> bf16 blocks [k_chunk] of n_pad rows in the canonical
+// layout; optional per-row scale (RMSNorm) and bf16 gain.  Rows >= n and columns >= K are zero.
+// grid (k_chunks), block 256.
+__global__ void k_prep_act(const float* __restrict__ x, int stride, int n, int n_pad, int K, const float* __restrict__ row_scale,
+                           const __nv_bfloat16* __restrict__ gain, unsigned char* __restrict__ dst) {
+  const int kc = blockIdx.x;
+  unsigned char* blk = dst + (size_t)kc * tc_block_bytes(n_pad);
+  for (int idx = threadIdx.x; idx < n_pad * (kTcKC / 8); idx += blockDim.x) {
+    const int r = idx % n_pad, k8 = idx / n_pad;
+    const int k = kc * kTcKC + k8 * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r < n && k < K) {
+      const float4 a = *reinterpret_cast<const float4*>(x + (size_t)r * stride + k);
+      const float4 b = *reinterpret_cast<const float4*>(x + (size_t)r * stride + k + 4);
+      float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      if (row_scale) {
+        const float sc = row_scale[r];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) f[j] = f[j] * sc * __bfloat162float(gain[k + j]);
+      }
+      v.x = pack_bf16(f[0], f[1]); v.y = pack_bf16(f[2], f[3]); v.z = pack_bf16(f[4], f[5]); v.w = pack_bf16(f[6], f[7]);
+    }
+    *reinterpret_cast<uint4*>(blk + ((size_t)k8 * (n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
+  }
+}
+
+}  // namespace tabed

@@ -17,6 +17,7 @@
 #include "forward_kernels.cuh"
 #include "decide_kernels.cuh"
 #include "round_kernel.cuh"
+#include "gemm_tc.cuh"
 
 using namespace tabed;
 
@@ -927,6 +928,58 @@ int tabed_state_import(tabed_handle* h, const void* host, size_t bytes) {
     }
   }
   return TABED_OK;
+}
+
+// -------------------------------------------------------------------------------------------------
+// Stand-alone run of the tensor-core projection (packing + k_gemm_tc + split-K sum) on caller data.
+// -------------------------------------------------------------------------------------------------
+namespace {
+__global__ void k_sum_partials(const float* __restrict__ part, int ks, size_t elems, float* __restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= elems) return;
+  float v = 0.0f;
+  for (int k = 0; k < ks; ++k) v += part[(size_t)k * elems + i];
+  out[i] = v;
+}
+}  // namespace
+
+int tabed_debug_gemm_tc(const void* w, const float* act, int32_t rows, int32_t K, int32_t n, int32_t ks, float* out,
+                        int32_t device, void* stream) {
+  if (!w || !act || !out) return TABED_ERR_NULL_PTR;
+  if (rows < 1 || K < 8 || (K % 8) || n < 1 || n > kTcMaxN || ks < 1 || device < 0) return TABED_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return TABED_ERR_CUDA;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int m_tiles = (rows + kTcM - 1) / kTcM, k_chunks = (K + kTcKC - 1) / kTcKC, n_pad = (n + 15) / 16 * 16;
+  if (ks > k_chunks) ks = k_chunks;
+  const int cps = (k_chunks + ks - 1) / ks;
+  unsigned char *a_p = nullptr, *b_p = nullptr; float* part = nullptr; int* err = nullptr;
+  int rc = TABED_OK;
+  const size_t smem = (size_t)kTcStages * (tc_block_bytes(kTcM) + tc_block_bytes(n_pad)) + 1024;
+  if (cudaMalloc(&a_p, (size_t)m_tiles * k_chunks * tc_block_bytes(kTcM)) != cudaSuccess ||
+      cudaMalloc(&b_p, (size_t)k_chunks * tc_block_bytes(n_pad)) != cudaSuccess ||
+      cudaMalloc(&part, (size_t)ks * n * rows * sizeof(float)) != cudaSuccess || cudaMalloc(&err, sizeof(int)) != cudaSuccess ||
+      cudaMemsetAsync(err, 0, sizeof(int), st) != cudaSuccess ||
+      cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    rc = TABED_ERR_CUDA;
+  if (rc == TABED_OK) {
+    k_pack_tc<<<dim3(k_chunks, m_tiles), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(w), rows, nullptr, 0, nullptr, 0, K, k_chunks, a_p);
+    k_prep_act<<<k_chunks, 256, 0, st>>>(act, K, n, n_pad, K, nullptr, nullptr, b_p);
+    TcGemmArgs G{};
+    G.a_packed = a_p; G.b_packed = b_p; G.partial = part; G.rows_total = rows; G.rows_valid = rows; G.n_pad = n_pad; G.n_slots = n;
+    G.k_chunks = k_chunks; G.ks = ks; G.cps = cps; G.err = err;
+    k_gemm_tc<<<m_tiles * ks, kTcThreads, smem, st>>>(G);
+    const size_t elems = (size_t)n * rows;
+    k_sum_partials<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(part, ks, elems, out);
+    int herr = 0;
+    if (cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess ||
+        cudaGetLastError() != cudaSuccess)
+      rc = TABED_ERR_CUDA;
+    else if (herr) rc = TABED_ERR_TIMEOUT;
+  }
+  cudaFree(a_p); cudaFree(b_p); cudaFree(part); cudaFree(err);
+  cudaGetLastError();
+  return rc;
 }
 
 // -------------------------------------------------------------------------------------------------
