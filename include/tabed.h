@@ -81,11 +81,14 @@ extern "C" {
 /* How tabed_draft_round runs Algorithm 1 (tabed_select_path).  Results obey the same contract on
  * both paths: identical integer decisions for identical logits; logits agree within the forward
  * pass's floating-point tolerance (summation order differs). */
-#define TABED_PATH_AUTO        0   /* persistent kernel when the drafter qualifies, else per-operation  */
+#define TABED_PATH_AUTO        0   /* persistent kernel if the drafter qualifies, else tensor-core
+                                      projections if it qualifies, else per-operation                   */
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
 #define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, 2*B*m <= 8
                                       slots, d_model <= 2048 and a multiple of 16, d_ffn a multiple of 16,
                                       (H/Hkv)*head_dim <= 512, <= 64 layers, kv_capacity <= 32768        */
+#define TABED_PATH_TENSOR_CORE 3   /* one kernel per operation with the projections as tcgen05 contractions
+                                      over all rows: bf16 drafter, B*m >= 16 rows, not persistent-eligible */
 
 typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
 
@@ -198,9 +201,9 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
                      int32_t* out_w_argmax);
 
 /* Choose the drafting path (TABED_PATH_*).  Errors: UNSUPPORTED (TABED_PATH_PERSISTENT on a drafter
- * that does not qualify), BAD_STATE (mid-round), INVALID_ARG.  tabed_current_path returns the path
- * the next tabed_draft_round will take: TABED_PATH_PER_OP or TABED_PATH_PERSISTENT (positive), or a
- * negative error code. */
+ * that does not qualify; likewise TABED_PATH_TENSOR_CORE), BAD_STATE (mid-round), INVALID_ARG.
+ * tabed_current_path returns the path the next tabed_draft_round will take: TABED_PATH_PER_OP,
+ * TABED_PATH_PERSISTENT or TABED_PATH_TENSOR_CORE (positive), or a negative error code. */
 int tabed_select_path(tabed_handle* h, int32_t path);
 int tabed_current_path(const tabed_handle* h);
 

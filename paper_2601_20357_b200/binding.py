@@ -22,7 +22,7 @@ DIST_KL, DIST_TVD = 0, 1
 MODE_SAMPLE, MODE_GREEDY = 0, 1
 (VIEW_QK, VIEW_Q, VIEW_P, VIEW_LOGITS, VIEW_KV_LEN, VIEW_WEIGHTS, VIEW_WINDOW_SUM, VIEW_PENDING,
  VIEW_GRID_J, VIEW_ERROR_FLAG, VIEW_TRACE) = range(11)
-PATH_AUTO, PATH_PER_OP, PATH_PERSISTENT = 0, 1, 2
+PATH_AUTO, PATH_PER_OP, PATH_PERSISTENT, PATH_TENSOR_CORE = 0, 1, 2, 3
 MAX_DEV = 11
 (PROF_QKV, PROF_ATTENTION, PROF_OPROJ, PROF_GATEUP, PROF_DOWN, PROF_LM_HEAD, PROF_ENSEMBLE, PROF_VERIFY,
  PROF_UPDATE, PROF_DRAFT_ROUND) = range(10)

@@ -30,7 +30,7 @@ constexpr int kTcM = 128;          // weight rows per tile (MMA M)
 constexpr int kTcKC = 128;         // input columns per pipeline stage
 constexpr int kTcStages = 3;
 constexpr int kTcThreads = 128;
-constexpr int kTcMaxN = 256;       // slots per launch (MMA N), a multiple of 16
+constexpr int kTcMaxN = 128;       // slots per launch (MMA N is their count rounded up to 16)
 
 // Canonical K-major no-swizzle operand block of `rows` rows x kTcKC columns (bf16):
 // element (r, k) at ((k/8) * (rows/8) + r/8) * 128 + (r%8) * 16 + (k%8) * 2 bytes.
@@ -39,7 +39,9 @@ __host__ __device__ inline size_t tc_block_bytes(int rows) { return (size_t)rows
 struct TcGemmArgs {
   const unsigned char* a_packed;   // [m_tiles][k_chunks] blocks of 128 rows
   const unsigned char* b_packed;   // [k_chunks] blocks of n_pad rows
-  float* partial;                  // [ks][n_slots][rows_total]
+  float* partial;                  // [ks] slabs of `slab` floats; slab layout [slot][rows_total], first slot of this launch at +0
+  size_t slab;                     // floats between k-split slabs
+  const SlotDesc* slots;           // optional: the launch returns at once when none of its slots is active
   int rows_total;                  // output rows of the projection (multiple of 128 after padding in a_packed)
   int rows_valid;                  // rows actually stored
   int n_pad, n_slots;              // MMA N (multiple of 16) / slots stored
@@ -72,6 +74,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (G.slots) {
+    int any = 0;
+    for (int s = tid; s < G.n_slots; s += kTcThreads) any |= G.slots[s].active;
+    if (!__syncthreads_or(any)) return;
+  }
   const int m_tile = blockIdx.x / G.ks, split = blockIdx.x - m_tile * G.ks;
   const int c_lo = split * G.cps, c_hi = min(c_lo + G.cps, G.k_chunks), n_ch = c_hi - c_lo;
   const size_t a_bytes = tc_block_bytes(kTcM), b_bytes = tc_block_bytes(G.n_pad);
@@ -161,7 +168,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   if (done_ok) {
     const int row = m_tile * kTcM + warp * 32 + lane;
-    float* out = G.partial + (size_t)split * G.n_slots * G.rows_total + row;
+    float* out = G.partial + (size_t)split * G.slab + row;
 #pragma unroll 1
     for (int c0 = 0; c0 < G.n_pad; c0 += 16) {
       uint32_t v[16];
@@ -234,6 +241,116 @@ __global__ void k_prep_act(const float* __restrict__ x, int stride, int n, int n
     }
     *reinterpret_cast<uint4*>(blk + ((size_t)k8 * (n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
   }
+}
+
+// ---- activation preparation for the tensor-core projections ------------------------------------------
+// One CTA per slot of the group: x <- base + sum of the previous projection's k-split partials (written
+// back when `write_back`), optional RMSNorm (gain != null), bf16 rounding, canonical operand layout.
+// src_slot (optional) maps the group's row to the slot whose residual it reads (LM head: last slot of a row).
+struct PrepRowArgs {
+  float* x; int d;                       // residual stream [slot][d]
+  const float* partial; int ks; size_t slab;     // [ks] slabs [slot][d] or null
+  const int* src_slot;                   // or null
+  const SlotDesc* slots;                 // activity of the slots (null: all active)
+  const __nv_bfloat16* gain; float eps;  // RMSNorm gain or null
+  int slot0, n, n_pad, write_back;
+  unsigned char* dst;                    // [k_chunks] blocks of n_pad rows
+};
+__global__ void __launch_bounds__(256) k_prep_row(const PrepRowArgs P) {
+  const int r = blockIdx.x, tid = threadIdx.x;
+  const int s = P.src_slot ? P.src_slot[P.slot0 + r] : P.slot0 + r;
+  if (P.slots && !P.slots[s].active) return;
+  __shared__ float red[8];
+  __shared__ float s_scale;
+  float* xr = P.x + (size_t)s * P.d;
+  float ss = 0.0f;
+  // pass 1: resolve, write back, sum of squares.  Thread owns groups of 8 consecutive elements.
+  for (int k = tid * 8; k < P.d; k += 256 * 8) {
+    float f[8];
+    const float4 a = *reinterpret_cast<const float4*>(xr + k), b = *reinterpret_cast<const float4*>(xr + k + 4);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    for (int q = 0; q < P.ks; ++q) {
+      const float* pp = P.partial + (size_t)q * P.slab + (size_t)s * P.d + k;
+      const float4 c = *reinterpret_cast<const float4*>(pp), e = *reinterpret_cast<const float4*>(pp + 4);
+      f[0] += c.x; f[1] += c.y; f[2] += c.z; f[3] += c.w; f[4] += e.x; f[5] += e.y; f[6] += e.z; f[7] += e.w;
+    }
+    if (P.write_back && P.ks > 0) {
+      *reinterpret_cast<float4*>(xr + k) = make_float4(f[0], f[1], f[2], f[3]);
+      *reinterpret_cast<float4*>(xr + k + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) ss = fmaf(f[j], f[j], ss);
+  }
+  ss = warp_sum_f32(ss);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  if (tid == 0) {
+    float tot = 0.0f;
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    s_scale = P.gain ? 1.0f / sqrtf(tot / (float)P.d + P.eps) : 1.0f;
+  }
+  __syncthreads();
+  const float sc = s_scale;
+  // pass 2: (re-read; the values are in L1/L2) scale, round, store 16-byte pieces of the canonical layout
+  for (int k = tid * 8; k < P.d; k += 256 * 8) {
+    float f[8];
+    const float4 a = *reinterpret_cast<const float4*>(xr + k), b = *reinterpret_cast<const float4*>(xr + k + 4);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    if (!(P.write_back && P.ks > 0)) {
+      for (int q = 0; q < P.ks; ++q) {
+        const float* pp = P.partial + (size_t)q * P.slab + (size_t)s * P.d + k;
+        const float4 c = *reinterpret_cast<const float4*>(pp), e = *reinterpret_cast<const float4*>(pp + 4);
+        f[0] += c.x; f[1] += c.y; f[2] += c.z; f[3] += c.w; f[4] += e.x; f[5] += e.y; f[6] += e.z; f[7] += e.w;
+      }
+    }
+    if (P.gain) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) f[j] = f[j] * sc * __bfloat162float(P.gain[k + j]);
+    }
+    uint4 v;
+    v.x = pack_bf16(f[0], f[1]); v.y = pack_bf16(f[2], f[3]); v.z = pack_bf16(f[4], f[5]); v.w = pack_bf16(f[6], f[7]);
+    const int kc = k / kTcKC, k8 = (k % kTcKC) >> 3;
+    *reinterpret_cast<uint4*>(P.dst + (size_t)kc * tc_block_bytes(P.n_pad) + ((size_t)k8 * (P.n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
+  }
+}
+
+// Gated product for the down projection from the gate|up projection's partials:
+// mid[s][f] = SiLU(sum_q pg[q][s][f]) * (sum_q pg[q][s][F + f]), rounded to bf16, canonical layout.
+// grid (k_chunks of F, slots of the group), block 16 (one thread per 8 columns of the chunk).
+__global__ void k_swiglu_prep(const float* __restrict__ partial, int ks, size_t slab, int F, const SlotDesc* __restrict__ slots,
+                              int slot0, int n_pad, unsigned char* __restrict__ dst) {
+  const int kc = blockIdx.x, r = blockIdx.y, k8 = threadIdx.x;
+  const int s = slot0 + r;
+  if (slots && !slots[s].active) return;
+  const int f0 = kc * kTcKC + k8 * 8;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (f0 < F) {
+    float g[8] = {0, 0, 0, 0, 0, 0, 0, 0}, u[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int q = 0; q < ks; ++q) {
+      const float* pg = partial + (size_t)q * slab + (size_t)s * (2 * F) + f0;
+      const float4 a = *reinterpret_cast<const float4*>(pg), b = *reinterpret_cast<const float4*>(pg + 4);
+      const float4 c = *reinterpret_cast<const float4*>(pg + F), e = *reinterpret_cast<const float4*>(pg + F + 4);
+      g[0] += a.x; g[1] += a.y; g[2] += a.z; g[3] += a.w; g[4] += b.x; g[5] += b.y; g[6] += b.z; g[7] += b.w;
+      u[0] += c.x; u[1] += c.y; u[2] += c.z; u[3] += c.w; u[4] += e.x; u[5] += e.y; u[6] += e.z; u[7] += e.w;
+    }
+    float m[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) m[j] = g[j] / (1.0f + expf(-g[j])) * u[j];
+    v.x = pack_bf16(m[0], m[1]); v.y = pack_bf16(m[2], m[3]); v.z = pack_bf16(m[4], m[5]); v.w = pack_bf16(m[6], m[7]);
+  }
+  *reinterpret_cast<uint4*>(dst + (size_t)kc * tc_block_bytes(n_pad) + ((size_t)k8 * (n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
+}
+
+// out[i] = sum over the k-split slabs (fixed order); grid over elems.
+__global__ void k_sum_slabs(const float* __restrict__ part, int ks, size_t slab, size_t elems, float* __restrict__ out) {
+  const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= elems) return;
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k = 0; k < ks; ++k) {
+    const float4 a = *reinterpret_cast<const float4*>(part + (size_t)k * slab + i);
+    v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+  }
+  *reinterpret_cast<float4*>(out + i) = v;
 }
 
 }  // namespace tabed

@@ -82,6 +82,15 @@ struct tabed_handle {
   unsigned char* packed = nullptr;
   uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
   unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false;
+  // tensor-core projections for many rows (bf16 drafter, more than 8 slots per step)
+  bool tc_ok = false;
+  struct TcKind { int rows, K, m_tiles, k_chunks, ks, cps; size_t bytes; };
+  TcKind tck[5]{};                  // KIND_QKV, KIND_O, KIND_GU (gate|up rows), KIND_DN, KIND_LM
+  unsigned char* tc_w = nullptr;    // [L][QKV | O | GU | DN] then LM, operand blocks of k_pack_tc
+  size_t tc_layer_stride = 0, tc_off[5]{};
+  unsigned char* tc_act = nullptr;  // activation operand blocks of the group being projected
+  float *tc_pq = nullptr, *tc_po = nullptr, *tc_pgu = nullptr, *tc_pd = nullptr;   // k-split partials [ks][2R][rows]
+  size_t tc_smem = 0;
   // per-kernel-class timing (tabed_profile_begin / tabed_profile_end)
   int prof_class = -1;
   std::vector<cudaEvent_t> prof_events;     // start/stop pairs
@@ -419,6 +428,149 @@ int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_
   return TABED_OK;
 }
 
+// ---- tensor-core path for many rows -----------------------------------------------------------------
+int setup_tc(tabed_handle* h) {
+  const tabed_config& c = h->cfg;
+  h->tc_ok = false;
+  if (c.dtype != TABED_DTYPE_BF16 || h->persist_ok || h->R < 16 || h->d % 8 || h->F % 8 || (h->H * h->hd) % 8) return TABED_OK;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return TABED_ERR_CUDA;
+  if (prop.major < 10) return TABED_OK;
+  const int n_sm = prop.multiProcessorCount, kvd = h->Hkv * h->hd;
+  const int rows[5] = {h->qkv_w, h->d, 2 * h->F, h->d, h->V};
+  const int Ks[5] = {h->d, h->H * h->hd, h->d, h->F, h->d};
+  for (int k = 0; k < 5; ++k) {
+    tabed_handle::TcKind& t = h->tck[k];
+    t.rows = rows[k]; t.K = Ks[k];
+    t.m_tiles = (t.rows + kTcM - 1) / kTcM; t.k_chunks = (t.K + kTcKC - 1) / kTcKC;
+    int ks = std::max(1, std::min(t.k_chunks, (n_sm + t.m_tiles - 1) / t.m_tiles));
+    if (k == KIND_LM) ks = 1;                       // logits are stored directly
+    t.cps = (t.k_chunks + ks - 1) / ks;
+    t.ks = (t.k_chunks + t.cps - 1) / t.cps;
+    t.bytes = (size_t)t.m_tiles * t.k_chunks * tc_block_bytes(kTcM);
+  }
+  h->tc_off[KIND_QKV] = 0;
+  h->tc_off[KIND_O] = h->tck[KIND_QKV].bytes;
+  h->tc_off[KIND_GU] = h->tc_off[KIND_O] + h->tck[KIND_O].bytes;
+  h->tc_off[KIND_DN] = h->tc_off[KIND_GU] + h->tck[KIND_GU].bytes;
+  h->tc_layer_stride = h->tc_off[KIND_DN] + h->tck[KIND_DN].bytes;
+  h->tc_off[KIND_LM] = h->tc_layer_stride * h->L;
+  const int n_pad_max = (std::min(h->R, kTcMaxN) + 15) / 16 * 16;
+  h->tc_smem = (size_t)kTcStages * (tc_block_bytes(kTcM) + tc_block_bytes(n_pad_max)) + 1024;
+  if (h->tc_smem > (size_t)prop.sharedMemPerBlockOptin) return TABED_OK;
+  if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->tc_smem) != cudaSuccess) return TABED_ERR_CUDA;
+  int rc = TABED_OK;
+  auto A2 = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count, false); };
+  const size_t S2 = 2 * (size_t)h->R;
+  int kc_max = 0;
+  for (int k = 0; k < 5; ++k) kc_max = std::max(kc_max, h->tck[k].k_chunks);
+  A2(&h->tc_w, h->tc_off[KIND_LM] + h->tck[KIND_LM].bytes);
+  A2(&h->tc_act, (size_t)kc_max * tc_block_bytes(n_pad_max));
+  A2(&h->tc_pq, (size_t)h->tck[KIND_QKV].ks * S2 * h->qkv_w); A2(&h->tc_po, (size_t)h->tck[KIND_O].ks * S2 * h->d);
+  A2(&h->tc_pgu, (size_t)h->tck[KIND_GU].ks * S2 * 2 * h->F); A2(&h->tc_pd, (size_t)h->tck[KIND_DN].ks * S2 * h->d);
+  if (rc != TABED_OK) return rc;
+  using bf = __nv_bfloat16;
+  for (int l = 0; l <= h->L; ++l) {
+    for (int k = 0; k < 5; ++k) {
+      if ((l == h->L) != (k == KIND_LM)) continue;
+      const tabed_handle::TcKind& t = h->tck[k];
+      unsigned char* dst = h->tc_w + h->tc_off[k] + (k == KIND_LM ? 0 : (size_t)l * h->tc_layer_stride);
+      const dim3 grid(t.k_chunks, t.m_tiles);
+      if (k == KIND_QKV) k_pack_tc<<<grid, 256, 0, h->stream>>>((const bf*)h->wq[l], h->d, (const bf*)h->wk[l], kvd, (const bf*)h->wv[l], kvd, t.K, t.k_chunks, dst);
+      else if (k == KIND_O) k_pack_tc<<<grid, 256, 0, h->stream>>>((const bf*)h->wo[l], h->d, nullptr, 0, nullptr, 0, t.K, t.k_chunks, dst);
+      else if (k == KIND_GU) k_pack_tc<<<grid, 256, 0, h->stream>>>((const bf*)h->w_gate[l], h->F, (const bf*)h->w_up[l], h->F, nullptr, 0, t.K, t.k_chunks, dst);
+      else if (k == KIND_DN) k_pack_tc<<<grid, 256, 0, h->stream>>>((const bf*)h->w_down[l], h->d, nullptr, 0, nullptr, 0, t.K, t.k_chunks, dst);
+      else k_pack_tc<<<grid, 256, 0, h->stream>>>((const bf*)h->lm_head, h->V, nullptr, 0, nullptr, 0, t.K, t.k_chunks, dst);
+    }
+  }
+  if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+  h->tc_ok = true;
+  return TABED_OK;
+}
+
+// one tensor-core projection of a slot group whose operand blocks are already in h->tc_act
+void launch_gemm_tc(tabed_handle* h, int kind, int layer, int n, float* partial, size_t slab, const SlotDesc* slots, int rows_valid) {
+  const tabed_handle::TcKind& t = h->tck[kind];
+  TcGemmArgs G{};
+  G.a_packed = h->tc_w + h->tc_off[kind] + (kind == KIND_LM ? 0 : (size_t)layer * h->tc_layer_stride);
+  G.b_packed = h->tc_act; G.partial = partial; G.slab = slab; G.slots = slots;
+  G.rows_total = t.rows; G.rows_valid = rows_valid; G.n_pad = (n + 15) / 16 * 16; G.n_slots = n;
+  G.k_chunks = t.k_chunks; G.ks = t.ks; G.cps = t.cps; G.err = h->err;
+  TABED_LAUNCH(h, k_gemm_tc, t.m_tiles * t.ks, kTcThreads, h->tc_smem, G);
+}
+
+// One shared-weight decoder step over `n_slots` slots with the projections on the tensor cores.
+void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* logits_out) {
+  using bf = __nv_bfloat16;
+  sa.R = h->R; sa.m = h->m; sa.d = h->d; sa.G = h->G;
+  sa.kv_len = h->kv_len; sa.pending = h->pending;
+  sa.slots = h->slots; sa.last_slot = h->last_slot; sa.x = h->x; sa.err = h->err; sa.kv_capacity = h->cap;
+  TABED_LAUNCH(h, k_begin_step<bf>, n_slots, 128, 0, sa, reinterpret_cast<const bf*>(h->embed));
+  const size_t S2 = 2 * (size_t)h->R;
+  const int d = h->d, HD = h->H * h->hd, F = h->F;
+  struct Grp { int s0, n; };
+  std::vector<Grp> groups;                       // groups never straddle the two halves of a first step
+  for (int half = 0; half * h->R < n_slots; ++half)
+    for (int g0 = 0; g0 < h->R; g0 += kTcMaxN) groups.push_back({half * h->R + g0, std::min(kTcMaxN, h->R - g0)});
+  auto prep_row = [&](const Grp& g, const float* partial, int ks, size_t slab, int write_back, const void* gain, const int* src, const SlotDesc* slots) {
+    PrepRowArgs P{};
+    P.x = h->x; P.d = d; P.partial = partial; P.ks = partial ? ks : 0; P.slab = slab; P.src_slot = src; P.slots = slots;
+    P.gain = reinterpret_cast<const bf*>(gain); P.eps = h->cfg.rms_eps; P.slot0 = g.s0; P.n = g.n; P.n_pad = (g.n + 15) / 16 * 16;
+    P.write_back = write_back; P.dst = h->tc_act;
+    TABED_LAUNCH(h, k_prep_row, g.n, 256, 0, P);
+  };
+  for (int l = 0; l < h->L; ++l) {
+    {
+      ProfScope ps(h, TABED_PROF_QKV);
+      for (const Grp& g : groups) {
+        prep_row(g, l == 0 ? nullptr : h->tc_pd, h->tck[KIND_DN].ks, S2 * d, 1, h->norm1[l], nullptr, h->slots);
+        launch_gemm_tc(h, KIND_QKV, l, g.n, h->tc_pq + (size_t)g.s0 * h->qkv_w, S2 * h->qkv_w, h->slots + g.s0, h->qkv_w);
+      }
+      const size_t elems = (size_t)n_slots * h->qkv_w;
+      TABED_LAUNCH(h, k_sum_slabs, (unsigned)((elems / 4 + 255) / 256), 256, 0, h->tc_pq, h->tck[KIND_QKV].ks, S2 * h->qkv_w, elems, h->qkv);
+    }
+    {
+      ProfScope ps(h, TABED_PROF_ATTENTION);
+      TABED_LAUNCH(h, k_rope_append<bf>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos, h->rope_sin,
+                   reinterpret_cast<bf*>(h->kc), reinterpret_cast<bf*>(h->vc), l, h->L, h->cap);
+      launch_attention_t<bf>(h, l, n_slots, max_pos);
+    }
+    {
+      ProfScope ps(h, TABED_PROF_OPROJ);
+      for (const Grp& g : groups) {
+        const int n_pad = (g.n + 15) / 16 * 16;
+        TABED_LAUNCH(h, k_prep_act, h->tck[KIND_O].k_chunks, 256, 0, h->attn_out + (size_t)g.s0 * HD, HD, g.n, n_pad, HD,
+                     (const float*)nullptr, (const bf*)nullptr, h->tc_act);
+        launch_gemm_tc(h, KIND_O, l, g.n, h->tc_po + (size_t)g.s0 * d, S2 * d, h->slots + g.s0, d);
+      }
+    }
+    {
+      ProfScope ps(h, TABED_PROF_GATEUP);
+      for (const Grp& g : groups) {
+        prep_row(g, h->tc_po, h->tck[KIND_O].ks, S2 * d, 1, h->norm2[l], nullptr, h->slots);
+        launch_gemm_tc(h, KIND_GU, l, g.n, h->tc_pgu + (size_t)g.s0 * 2 * F, S2 * 2 * F, h->slots + g.s0, 2 * F);
+      }
+    }
+    {
+      ProfScope ps(h, TABED_PROF_DOWN);
+      for (const Grp& g : groups) {
+        const int n_pad = (g.n + 15) / 16 * 16;
+        TABED_LAUNCH(h, k_swiglu_prep, dim3(h->tck[KIND_DN].k_chunks, g.n), kTcKC / 8, 0, h->tc_pgu, h->tck[KIND_GU].ks, S2 * 2 * F, F,
+                     h->slots, g.s0, n_pad, h->tc_act);
+        launch_gemm_tc(h, KIND_DN, l, g.n, h->tc_pd + (size_t)g.s0 * d, S2 * d, h->slots + g.s0, d);
+      }
+    }
+  }
+  if (logits_out) {
+    ProfScope ps(h, TABED_PROF_LM_HEAD);
+    for (int r0 = 0; r0 < h->R; r0 += kTcMaxN) {
+      const Grp g{r0, std::min(kTcMaxN, h->R - r0)};
+      prep_row(g, h->tc_pd, h->tck[KIND_DN].ks, S2 * d, 0, h->final_norm, h->last_slot, nullptr);
+      launch_gemm_tc(h, KIND_LM, 0, g.n, logits_out + (size_t)r0 * h->V, 0, nullptr, h->V);
+    }
+  }
+}
+
 int check_cuda() { return cudaGetLastError() == cudaSuccess ? TABED_OK : TABED_ERR_CUDA; }
 
 int max_len_ub(const tabed_handle* h) {
@@ -541,6 +693,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
     }
     h->len_ub.assign(R, 0);
     if (rc == TABED_OK) rc = setup_persistent(h);
+    if (rc == TABED_OK) rc = setup_tc(h);
   }
   if (rc == TABED_OK) {
     // equal weights before any history; one pending slot per request; grid j* undefined
@@ -639,7 +792,8 @@ int tabed_decode_step(tabed_handle* h, const int32_t* tok, float* out_logits) {
   DeviceGuard guard(h->cfg.device);
   StepArgs sa{};
   sa.mode = STEP_FREE; sa.tokens = tok;
-  run_step(h, sa, h->R, max_len_ub(h) + 1, out_logits);
+  if (h->tc_ok && h->path_sel != TABED_PATH_PER_OP) run_step_tc(h, sa, h->R, max_len_ub(h) + 1, out_logits);
+  else run_step(h, sa, h->R, max_len_ub(h) + 1, out_logits);
   TABED_LAUNCH(h, k_advance_len, (h->R + 127) / 128, 128, 0, h->kv_len, h->R, -1, 1);
   for (int& v : h->len_ub) v += 1;
   return check_cuda();
@@ -682,7 +836,8 @@ static int draft_common(tabed_handle* h, const float* ext_logits, const float* u
       StepArgs sa{};
       sa.mode = (i == 0) ? STEP_ROUND_FIRST : STEP_ROUND_NEXT; sa.step = i; sa.tokens = h->tokens;
       float* own = h->logits_own + i * RV;
-      run_step(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
+      if (h->tc_ok && h->path_sel != TABED_PATH_PER_OP) run_step_tc(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
+      else run_step(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
       lg = h->logits_override ? h->logits_override + i * RV : own;
     } else {
       lg = ext_logits + i * RV;
@@ -824,16 +979,18 @@ int tabed_debug_override_logits(tabed_handle* h, const float* drafter_logits) {
 
 int tabed_select_path(tabed_handle* h, int32_t path) {
   if (!h) return TABED_ERR_NULL_PTR;
-  if (path < TABED_PATH_AUTO || path > TABED_PATH_PERSISTENT) return TABED_ERR_INVALID_ARG;
+  if (path < TABED_PATH_AUTO || path > TABED_PATH_TENSOR_CORE) return TABED_ERR_INVALID_ARG;
   if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
   if (path == TABED_PATH_PERSISTENT && !h->persist_ok) return TABED_ERR_UNSUPPORTED;
+  if (path == TABED_PATH_TENSOR_CORE && !h->tc_ok) return TABED_ERR_UNSUPPORTED;
   h->path_sel = path;
   return TABED_OK;
 }
 
 int tabed_current_path(const tabed_handle* h) {
   if (!h) return TABED_ERR_NULL_PTR;
-  return (h->persist_ok && h->path_sel != TABED_PATH_PER_OP) ? TABED_PATH_PERSISTENT : TABED_PATH_PER_OP;
+  if (h->path_sel == TABED_PATH_PER_OP) return TABED_PATH_PER_OP;
+  return h->persist_ok ? TABED_PATH_PERSISTENT : (h->tc_ok ? TABED_PATH_TENSOR_CORE : TABED_PATH_PER_OP);
 }
 
 int tabed_debug_trace(tabed_handle* h, int32_t on) {
@@ -966,7 +1123,7 @@ int tabed_debug_gemm_tc(const void* w, const float* act, int32_t rows, int32_t K
     k_pack_tc<<<dim3(k_chunks, m_tiles), 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(w), rows, nullptr, 0, nullptr, 0, K, k_chunks, a_p);
     k_prep_act<<<k_chunks, 256, 0, st>>>(act, K, n, n_pad, K, nullptr, nullptr, b_p);
     TcGemmArgs G{};
-    G.a_packed = a_p; G.b_packed = b_p; G.partial = part; G.rows_total = rows; G.rows_valid = rows; G.n_pad = n_pad; G.n_slots = n;
+    G.a_packed = a_p; G.b_packed = b_p; G.partial = part; G.slab = (size_t)n * rows; G.rows_total = rows; G.rows_valid = rows; G.n_pad = n_pad; G.n_slots = n;
     G.k_chunks = k_chunks; G.ks = ks; G.cps = cps; G.err = err;
     k_gemm_tc<<<m_tiles * ks, kTcThreads, smem, st>>>(G);
     const size_t elems = (size_t)n * rows;

@@ -1,0 +1,77 @@
+"""GPU parity tests of the drafting path whose projections run as tcgen05 contractions over all rows
+(TABED_PATH_TENSOR_CORE: bf16 drafter, 16 or more shared-weight rows), through the C boundary.
+
+Same bars as tests/test_gpu_parity.py (lock step with the checker: integer results and q, q^(k), p
+bit-exact on the checker's logits; the kernel's own logits within the bf16 bound, probabilities
+within 1e-5).  The shapes are chosen for what is special here: input dimensions that are not a
+multiple of the 128-column pipeline stage, an output dimension that is not a multiple of the
+128-row tile (ragged LM-head tile), row counts that are not a multiple of 16, requests with one and
+with two pending tokens in the same step (the second half of the slots is projected in a pass of its
+own that is skipped when nobody needs it)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_20357_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    import gpu_harness as H
+    from paper_2601_20357_b200 import binding as TB
+
+
+def wl_rows(*, B, m, d=256, heads=4, kv_heads=2, ffn=640, vocab=3000, gamma=3, sigma=0.3, cid=81, alpha=None):
+    cfg = W.DrafterCfg(2, d, heads, kv_heads, ffn, vocab, "bf16")
+    prefixes = ((("embeds", 11), ("tokens", 7)), (("tokens", 5),), (("tokens", 40),))[:m]
+    if alpha is None:
+        alpha = tuple([0.5, 0.3, 0.2][:m]) if m == 3 else tuple([1.0 / m] * m)
+    return W.Workload(name=f"tensor{cid}", config_id=cid, drafter=cfg, n_inputs=m, n_requests=B, gamma=gamma, window_h=4,
+                      rounds=4, policy=W.POLICY_SOFTMAX_INV_ERR if m != 2 else W.POLICY_GRID_MT, prefixes=prefixes,
+                      kv_capacity=128, alpha=alpha, sigma_schedule=((0, sigma),))
+
+
+def test_tensor_path_is_selected_for_many_rows():
+    pair = H.build_pair(wl_rows(B=6, m=3))
+    assert pair.gpu.current_path() == TB.PATH_TENSOR_CORE
+    pair.gpu.select_path(TB.PATH_PER_OP)
+    assert pair.gpu.current_path() == TB.PATH_PER_OP
+    pair.gpu.destroy()
+
+
+def test_lockstep_18_rows_ragged_dimensions():
+    """R = 18 rows (MMA N = 32), d = 256, F = 640 (5 stages), V = 3000 (last LM-head tile has 56 rows)."""
+    wl = wl_rows(B=6, m=3)
+    pair = H.build_pair(wl)
+    for rnd in range(3):
+        H.lockstep_round(pair, rnd, override=True)
+    pair.gpu.destroy()
+
+
+def test_lockstep_mixed_pending_counts_40_rows():
+    """20 requests x 2 inputs; small sigma so that some requests accept whole blocks (two pending tokens)
+    while others do not: the pass over the second half of the slots runs with most slots inactive."""
+    wl = wl_rows(B=20, m=2, sigma=0.05, alpha=(0.9, 0.1), cid=82, gamma=2)
+    pair = H.build_pair(wl)
+    full = 0
+    for rnd in range(4):
+        H.lockstep_round(pair, rnd, override=True)
+        full += int((pair.orc.n_accept == wl.gamma).sum())
+    assert 0 < full < 4 * wl.n_requests
+    pair.gpu.destroy()
+
+
+def test_tensor_path_agrees_with_per_operation_path():
+    wl = wl_rows(B=8, m=3, cid=83)
+    a, b = H.build_pair(wl), H.build_pair(wl)
+    b.gpu.select_path(TB.PATH_PER_OP)
+    ud, _, _ = W.round_uniforms(wl, 0)
+    toks = torch.empty((wl.n_requests, wl.gamma), dtype=torch.int32, device=H.DEV)
+    a.gpu.draft_round(H.t(ud), toks)
+    b.gpu.draft_round(H.t(ud), toks.clone())
+    torch.cuda.synchronize()
+    la = a.gpu.debug_view(TB.VIEW_LOGITS)[0].cpu().numpy()
+    lb = b.gpu.debug_view(TB.VIEW_LOGITS)[0].cpu().numpy()
+    assert np.max(np.abs(la - lb)) <= H.LOGIT_TOL["bf16"]
+    H.check_error_flag(a.gpu)
+    a.gpu.destroy(); b.gpu.destroy()
