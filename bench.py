@@ -444,7 +444,8 @@ def run_ours(args, wl):
                    "window_h": wl.window_h, "vocab": V, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model,
                    "l2": "256 MB written between rounds (stands for the target model's pass); rounds timed one by one "
                          "with CUDA events", "parallelism": f"replicas x{world}",
-                   "path": "persistent" if persistent else "per-operation"},
+                   "path": {TB.PATH_PERSISTENT: "persistent", TB.PATH_TENSOR_CORE: "tensor-core projections",
+                            TB.PATH_PER_OP: "per-operation"}[g.current_path()]},
         "drafted_tokens_per_sec": value * G,
         "block_efficiency": mean_accept + 1.0,
         "wall_ms_per_step_incl_flush": 1000.0 * wall / K,

@@ -441,6 +441,136 @@ k_attn_partial(const float* __restrict__ qkv, const SlotDesc* __restrict__ slots
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// K-b, bf16 caches, bandwidth-oriented variant: grid (splits, Hkv, slots), block 256.  A CTA handles
+// kAttnBwPasses * (8 warps * 32/LPR) positions (128 for head_dim 64) and issues ALL its K and V loads
+// (8 x 16 bytes per thread) before it touches any of them, so that one memory round trip covers the
+// item and ~4 resident CTAs keep >100 KB per SM in flight.  Output as k_attn_partial.
+// ------------------------------------------------------------------------------------------------
+constexpr int kAttnBwThreads = 256;
+constexpr int kAttnBwPasses = 4;
+__host__ __device__ inline int attn_bw_split_len(int hd) { return kAttnBwPasses * (kAttnBwThreads / 32) * (32 / (hd / 8)); }
+
+template <int HD>
+__global__ void __launch_bounds__(kAttnBwThreads)
+k_attn_split_bf16(const float* __restrict__ qkv, const SlotDesc* __restrict__ slots, int H, int Hkv,
+                  const __nv_bfloat16* __restrict__ kc, const __nv_bfloat16* __restrict__ vc, int layer, int L, int cap,
+                  float* __restrict__ part_o, float* __restrict__ part_ml, int max_splits, float scale) {
+  constexpr int LPR = HD / 8, PPW = 32 / LPR, NW = kAttnBwThreads / 32, PPB = NW * PPW, SPLIT = kAttnBwPasses * PPB;
+  const int s = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
+  const SlotDesc sd = slots[s];
+  if (!sd.active) return;
+  const int n_pos = sd.pos + 1, p_lo = split * SPLIT;
+  if (p_lo >= n_pos) return;
+  const int cnt = min(SPLIT, n_pos - p_lo);
+  const int grp = H / Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, sub = lane % LPR, pgrp = lane / LPR;
+  extern __shared__ float bw_smem[];
+  float* sc = bw_smem;                          // [grp][SPLIT]
+  float* sq = sc + grp * SPLIT;                 // [grp][HD]
+  float* so = sq + grp * HD;                    // [NW][grp][HD]
+  __shared__ float red[NW][2];
+  __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
+  const size_t base = ((((size_t)sd.row * L + layer) * Hkv + g) * cap) * HD;
+  uint4 kreg[kAttnBwPasses], vreg[kAttnBwPasses];
+#pragma unroll
+  for (int ps = 0; ps < kAttnBwPasses; ++ps) {
+    const int p = ps * PPB + warp * PPW + pgrp;
+    kreg[ps] = make_uint4(0u, 0u, 0u, 0u); vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
+    if (p < cnt) {
+      kreg[ps] = __ldg(reinterpret_cast<const uint4*>(kc + base + (size_t)(p_lo + p) * HD + sub * 8));
+      vreg[ps] = __ldg(reinterpret_cast<const uint4*>(vc + base + (size_t)(p_lo + p) * HD + sub * 8));
+    }
+  }
+  const float* qrow = qkv + (size_t)s * (H + 2 * Hkv) * HD + (size_t)g * grp * HD;
+  for (int i = tid; i < grp * HD; i += kAttnBwThreads) sq[i] = qrow[i];
+  __syncthreads();
+#pragma unroll 1
+  for (int t = 0; t < grp; ++t) {
+    float qf[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) qf[e] = sq[t * HD + sub * 8 + e];
+#pragma unroll
+    for (int ps = 0; ps < kAttnBwPasses; ++ps) {
+      if (ps * PPB >= cnt) break;
+      const int p = ps * PPB + warp * PPW + pgrp;
+      float kf[8];
+      Elem<__nv_bfloat16>::unpack(kreg[ps], kf);
+      float d = 0.0f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) d = fmaf(kf[e], qf[e], d);
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      if (sub == 0 && p < cnt) sc[t * SPLIT + p] = d * scale;
+    }
+  }
+  __syncthreads();
+  {
+    const int wph = (grp >= NW) ? 1 : NW / grp;      // warps sharing a head
+    const int t = warp / wph, wi = warp - t * wph;
+    float mx = -INFINITY;
+    if (t < grp) for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) mx = fmaxf(mx, sc[t * SPLIT + p]);
+    mx = warp_max_f32(mx);
+    if (lane == 0) red[warp][0] = mx;
+    __syncthreads();
+    float sum = 0.0f;
+    if (t < grp) {
+      mx = red[t * wph][0];
+      for (int w = 1; w < wph; ++w) mx = fmaxf(mx, red[t * wph + w][0]);
+      for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) { const float e = expf(sc[t * SPLIT + p] - mx); sc[t * SPLIT + p] = e; sum += e; }
+    }
+    sum = warp_sum_f32(sum);
+    if (lane == 0) red[warp][1] = sum;
+    __syncthreads();
+    if (t < grp && wi == 0 && lane == 0) {
+      float tot = 0.0f;
+      for (int w = 0; w < wph; ++w) tot += red[t * wph + w][1];
+      s_m[t] = mx; s_l[t] = tot;
+    }
+    // heads beyond the warps' reach (grp > NW cannot happen: grp <= kMaxGroup = NW)
+  }
+#pragma unroll 1
+  for (int t = 0; t < grp; ++t) {
+    float oacc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) oacc[e] = 0.0f;
+#pragma unroll
+    for (int ps = 0; ps < kAttnBwPasses; ++ps) {
+      if (ps * PPB >= cnt) break;
+      const int p = ps * PPB + warp * PPW + pgrp;
+      if (p < cnt) {
+        float vf[8];
+        Elem<__nv_bfloat16>::unpack(vreg[ps], vf);
+        const float pw = sc[t * SPLIT + p];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf[e], oacc[e]);
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      float v = oacc[e];
+#pragma unroll
+      for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      oacc[e] = v;
+    }
+    if (pgrp == 0) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) so[((size_t)warp * grp + t) * HD + sub * 8 + e] = oacc[e];
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < grp * HD; idx += kAttnBwThreads) {
+    const int t = idx / HD, dd = idx - t * HD;
+    float v = 0.0f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) v += so[((size_t)w * grp + t) * HD + dd];
+    const int head = g * grp + t;
+    const long long pi = ((long long)s * H + head) * max_splits + split;
+    part_o[pi * HD + dd] = v;
+    if (dd == 0) { part_ml[pi * 2] = s_m[t]; part_ml[pi * 2 + 1] = s_l[t]; }
+  }
+}
+
 // merge the splits in fixed order; grid (H, slots), block HD
 template <int HD>
 __global__ void k_attn_merge(const SlotDesc* __restrict__ slots, int H, int split_len,

@@ -191,6 +191,24 @@ void launch_gemv(tabed_handle* h, const GemvArgs& a, int epi, int ns) {
 
 template <typename T, int HD>
 void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    // bandwidth-oriented kernel: all K, V loads of a split in flight at once
+    const int split_len = attn_bw_split_len(HD);
+    const int splits = std::max(1, (max_pos + split_len - 1) / split_len);
+    const int grp = h->H / h->Hkv;
+    const size_t smem = ((size_t)grp * split_len + (size_t)grp * HD + (size_t)(kAttnBwThreads / 32) * grp * HD) * sizeof(float);
+    auto part = k_attn_split_bf16<HD>;
+    static bool attr_set = false;
+    if (!attr_set) { cudaFuncSetAttribute(part, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr_set = true; }
+    if (smem <= 96 * 1024) {
+      TABED_LAUNCH(h, part, dim3(splits, h->Hkv, n_slots), kAttnBwThreads, smem, h->qkv, h->slots, h->H, h->Hkv,
+                   reinterpret_cast<const __nv_bfloat16*>(h->kc), reinterpret_cast<const __nv_bfloat16*>(h->vc), layer, h->L, h->cap,
+                   h->part_o, h->part_ml, h->max_splits, 1.0f / sqrtf((float)h->hd));
+      auto merge = k_attn_merge<HD>;
+      TABED_LAUNCH(h, merge, dim3(h->H, n_slots), HD, 0, h->slots, h->H, split_len, h->part_o, h->part_ml, h->max_splits, h->attn_out);
+      return;
+    }
+  }
   const int split_len = (max_pos > 2048) ? 256 : 128;
   const int splits = std::max(1, (max_pos + split_len - 1) / split_len);
   const float scale = 1.0f / sqrtf((float)h->hd);
@@ -304,7 +322,7 @@ int setup_persistent(tabed_handle* h) {
   if (c.dtype != TABED_DTYPE_BF16) return TABED_OK;
   const int grp = h->H / h->Hkv;
   if (2 * h->R > kPSlots || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
-      grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || h->max_splits > kAttnSplitMax)
+      grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || (h->cap + 127) / 128 > kAttnSplitMax)
     return TABED_OK;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return TABED_ERR_CUDA;
@@ -659,7 +677,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
       for (int o : opts) if (o < h->ns) lower = o;
       h->ns = lower;
     }
-    h->max_splits = (h->cap + 127) / 128;
+    h->max_splits = (h->cap + 63) / 64;           // the shortest attention split any kernel uses is 64 positions
     h->embed = wts->embed; h->lm_head = wts->lm_head; h->final_norm = wts->final_norm;
     for (int l = 0; l < h->L; ++l) {
       h->wq.push_back(wts->wq[l]); h->wk.push_back(wts->wk[l]); h->wv.push_back(wts->wv[l]); h->wo.push_back(wts->wo[l]);
