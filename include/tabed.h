@@ -254,7 +254,7 @@ int tabed_ensemble_step_static(const float* logits, const float* w, const float*
 /* Stand-alone run of the tensor-core projection used for many shared-weight rows (Sec. 4.1 "batched
  * inference": all rows share the parameters, so a projection is one weights x rows contraction):
  * out[s][o] = sum_k w[o][k] * bf16(act[s][k]), fp32 accumulation.  w bf16 [rows][K], act float [n][K],
- * out float [n][rows], all device pointers on `device`; K a multiple of 8, n <= 128; ks = number of
+ * out float [n][rows], all device pointers on `device`; K a multiple of 8, n <= 256; ks = number of
  * splits of the input dimension (partial sums are added in split order).  Allocates and frees its
  * own temporaries and synchronises the stream: a test and tuning aid, not part of the round.
  * Errors: INVALID_ARG, CUDA, TIMEOUT (a bounded device-side wait ran out). */

@@ -452,7 +452,7 @@ constexpr int kAttnBwPasses = 4;
 __host__ __device__ inline int attn_bw_split_len(int hd) { return kAttnBwPasses * (kAttnBwThreads / 32) * (32 / (hd / 8)); }
 
 template <int HD>
-__global__ void __launch_bounds__(kAttnBwThreads)
+__global__ void __launch_bounds__(kAttnBwThreads, 3)
 k_attn_split_bf16(const float* __restrict__ qkv, const SlotDesc* __restrict__ slots, int H, int Hkv,
                   const __nv_bfloat16* __restrict__ kc, const __nv_bfloat16* __restrict__ vc, int layer, int L, int cap,
                   float* __restrict__ part_o, float* __restrict__ part_ml, int max_splits, float scale) {
@@ -466,11 +466,9 @@ k_attn_split_bf16(const float* __restrict__ qkv, const SlotDesc* __restrict__ sl
   const int grp = H / Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, sub = lane % LPR, pgrp = lane / LPR;
   extern __shared__ float bw_smem[];
-  float* sc = bw_smem;                          // [grp][SPLIT]
-  float* sq = sc + grp * SPLIT;                 // [grp][HD]
-  float* so = sq + grp * HD;                    // [NW][grp][HD]
-  __shared__ float red[NW][2];
-  __shared__ float s_m[kMaxGroup], s_l[kMaxGroup];
+  float* so = bw_smem;                          // [NW][grp][HD] un-normalised outputs of the warps
+  float* sm = so + (size_t)NW * grp * HD;       // [NW][grp] running maxima
+  float* sl = sm + NW * grp;                    // [NW][grp] sums
   const size_t base = ((((size_t)sd.row * L + layer) * Hkv + g) * cap) * HD;
   uint4 kreg[kAttnBwPasses], vreg[kAttnBwPasses];
 #pragma unroll
@@ -483,16 +481,16 @@ k_attn_split_bf16(const float* __restrict__ qkv, const SlotDesc* __restrict__ sl
     }
   }
   const float* qrow = qkv + (size_t)s * (H + 2 * Hkv) * HD + (size_t)g * grp * HD;
-  for (int i = tid; i < grp * HD; i += kAttnBwThreads) sq[i] = qrow[i];
-  __syncthreads();
+  // every warp runs its own softmax over its positions (no block-wide exchange until the end)
 #pragma unroll 1
   for (int t = 0; t < grp; ++t) {
-    float qf[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) qf[e] = sq[t * HD + sub * 8 + e];
+    const float4 q0 = *reinterpret_cast<const float4*>(qrow + t * HD + sub * 8);
+    const float4 q1 = *reinterpret_cast<const float4*>(qrow + t * HD + sub * 8 + 4);
+    const float qf[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+    float sc[kAttnBwPasses];
+    float mx = -INFINITY;
 #pragma unroll
     for (int ps = 0; ps < kAttnBwPasses; ++ps) {
-      if (ps * PPB >= cnt) break;
       const int p = ps * PPB + warp * PPW + pgrp;
       float kf[8];
       Elem<__nv_bfloat16>::unpack(kreg[ps], kf);
@@ -501,73 +499,54 @@ k_attn_split_bf16(const float* __restrict__ qkv, const SlotDesc* __restrict__ sl
       for (int e = 0; e < 8; ++e) d = fmaf(kf[e], qf[e], d);
 #pragma unroll
       for (int o = LPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-      if (sub == 0 && p < cnt) sc[t * SPLIT + p] = d * scale;
+      sc[ps] = (p < cnt) ? d * scale : -INFINITY;
+      mx = fmaxf(mx, sc[ps]);
     }
-  }
-  __syncthreads();
-  {
-    const int wph = (grp >= NW) ? 1 : NW / grp;      // warps sharing a head
-    const int t = warp / wph, wi = warp - t * wph;
-    float mx = -INFINITY;
-    if (t < grp) for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) mx = fmaxf(mx, sc[t * SPLIT + p]);
-    mx = warp_max_f32(mx);
-    if (lane == 0) red[warp][0] = mx;
-    __syncthreads();
-    float sum = 0.0f;
-    if (t < grp) {
-      mx = red[t * wph][0];
-      for (int w = 1; w < wph; ++w) mx = fmaxf(mx, red[t * wph + w][0]);
-      for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) { const float e = expf(sc[t * SPLIT + p] - mx); sc[t * SPLIT + p] = e; sum += e; }
-    }
-    sum = warp_sum_f32(sum);
-    if (lane == 0) red[warp][1] = sum;
-    __syncthreads();
-    if (t < grp && wi == 0 && lane == 0) {
-      float tot = 0.0f;
-      for (int w = 0; w < wph; ++w) tot += red[t * wph + w][1];
-      s_m[t] = mx; s_l[t] = tot;
-    }
-    // heads beyond the warps' reach (grp > NW cannot happen: grp <= kMaxGroup = NW)
-  }
-#pragma unroll 1
-  for (int t = 0; t < grp; ++t) {
-    float oacc[8];
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float oacc[8], sum = 0.0f;
 #pragma unroll
     for (int e = 0; e < 8; ++e) oacc[e] = 0.0f;
 #pragma unroll
     for (int ps = 0; ps < kAttnBwPasses; ++ps) {
-      if (ps * PPB >= cnt) break;
-      const int p = ps * PPB + warp * PPW + pgrp;
-      if (p < cnt) {
-        float vf[8];
-        Elem<__nv_bfloat16>::unpack(vreg[ps], vf);
-        const float pw = sc[t * SPLIT + p];
+      const float pw = (sc[ps] > -INFINITY) ? expf(sc[ps] - mx) : 0.0f;
+      sum += pw;
+      float vf[8];
+      Elem<__nv_bfloat16>::unpack(vreg[ps], vf);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf[e], oacc[e]);
-      }
+      for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf[e], oacc[e]);
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      float v = oacc[e];
+    for (int o = LPR; o < 32; o <<= 1) {
+      sum += __shfl_xor_sync(0xffffffffu, sum, o);
 #pragma unroll
-      for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      oacc[e] = v;
+      for (int e = 0; e < 8; ++e) oacc[e] += __shfl_xor_sync(0xffffffffu, oacc[e], o);
     }
     if (pgrp == 0) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) so[((size_t)warp * grp + t) * HD + sub * 8 + e] = oacc[e];
+      if (sub == 0) { sm[warp * grp + t] = mx; sl[warp * grp + t] = sum; }
     }
   }
   __syncthreads();
+  // merge the warps in warp order
   for (int idx = tid; idx < grp * HD; idx += kAttnBwThreads) {
     const int t = idx / HD, dd = idx - t * HD;
-    float v = 0.0f;
+    float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) v += so[((size_t)w * grp + t) * HD + dd];
+    for (int w = 0; w < NW; ++w) M = fmaxf(M, sm[w * grp + t]);
+    float v = 0.0f, l = 0.0f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float mw = sm[w * grp + t];
+      const float f = (mw > -INFINITY) ? expf(mw - M) : 0.0f;
+      v = fmaf(f, so[((size_t)w * grp + t) * HD + dd], v);
+      l = fmaf(f, sl[w * grp + t], l);
+    }
     const int head = g * grp + t;
     const long long pi = ((long long)s * H + head) * max_splits + split;
     part_o[pi * HD + dd] = v;
-    if (dd == 0) { part_ml[pi * 2] = s_m[t]; part_ml[pi * 2 + 1] = s_l[t]; }
+    if (dd == 0) { part_ml[pi * 2] = M; part_ml[pi * 2 + 1] = l; }
   }
 }
 

@@ -28,9 +28,10 @@ namespace tabed {
 
 constexpr int kTcM = 128;          // weight rows per tile (MMA M)
 constexpr int kTcKC = 128;         // input columns per pipeline stage
-constexpr int kTcStages = 3;
+constexpr int kTcStages = 3;        // pipeline stages (2 when more than 128 slots share the shared memory)
 constexpr int kTcThreads = 128;
-constexpr int kTcMaxN = 128;       // slots per launch (MMA N is their count rounded up to 16)
+constexpr int kTcMaxN = 256;       // slots per launch (MMA N is their count rounded up to 16)
+__host__ __device__ inline int tc_stages(int n_pad) { return n_pad > 128 ? 2 : kTcStages; }
 
 // Canonical K-major no-swizzle operand block of `rows` rows x kTcKC columns (bf16):
 // element (r, k) at ((k/8) * (rows/8) + r/8) * 128 + (r%8) * 16 + (k%8) * 2 bytes.
@@ -82,6 +83,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   const int m_tile = blockIdx.x / G.ks, split = blockIdx.x - m_tile * G.ks;
   const int c_lo = split * G.cps, c_hi = min(c_lo + G.cps, G.k_chunks), n_ch = c_hi - c_lo;
   const size_t a_bytes = tc_block_bytes(kTcM), b_bytes = tc_block_bytes(G.n_pad);
+  const int n_stages = tc_stages(G.n_pad);
   const uint32_t tmem_cols = G.n_pad <= 32 ? 32u : (G.n_pad <= 64 ? 64u : (G.n_pad <= 128 ? 128u : 256u));
 
   if (tid == 0) {
@@ -106,7 +108,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
     const unsigned char* a_src = G.a_packed + ((size_t)m_tile * G.k_chunks + c_lo) * a_bytes;
     const unsigned char* b_src = G.b_packed + (size_t)c_lo * b_bytes;
     bool ok = true;
-    const int pre = n_ch < kTcStages ? n_ch : kTcStages;
+    const int pre = n_ch < n_stages ? n_ch : n_stages;
     for (int c = 0; c < pre; ++c) {
       unsigned char* st = tc_smem + (size_t)c * (a_bytes + b_bytes);
       mbar_expect_tx(&s_full[c], (unsigned)(a_bytes + b_bytes));
@@ -115,8 +117,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
     }
     int issued = pre;
     for (int c = 0; c < n_ch && ok; ++c) {
-      const int s = c % kTcStages;
-      ok = tc_wait(&s_full[s], (unsigned)(c / kTcStages) & 1u, G.err);
+      const int s = c % n_stages;
+      ok = tc_wait(&s_full[s], (unsigned)(c / n_stages) & 1u, G.err);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t a_s = smem_u32(tc_smem + (size_t)s * (a_bytes + b_bytes));
@@ -135,7 +137,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
       // the stage may be refilled once these MMAs have read it
       asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_empty[s])) : "memory");
       if (issued < n_ch) {
-        ok = tc_wait(&s_empty[s], (unsigned)(c / kTcStages) & 1u, G.err);
+        ok = tc_wait(&s_empty[s], (unsigned)(c / n_stages) & 1u, G.err);
         if (!ok) break;
         unsigned char* st = tc_smem + (size_t)s * (a_bytes + b_bytes);
         mbar_expect_tx(&s_full[s], (unsigned)(a_bytes + b_bytes));
@@ -148,7 +150,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
     else {
       s_bad = 1;
       // let the copies in flight land before the shared memory is released
-      for (int s = 0; s < kTcStages; ++s) {
+      for (int s = 0; s < n_stages; ++s) {
         unsigned spins = 0;
         while (!mbar_try_wait(&s_full[s], 0) && !mbar_try_wait(&s_full[s], 1) && ++spins < (1u << 16)) __nanosleep(64);
       }

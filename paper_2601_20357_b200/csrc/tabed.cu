@@ -196,7 +196,7 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
     const int split_len = attn_bw_split_len(HD);
     const int splits = std::max(1, (max_pos + split_len - 1) / split_len);
     const int grp = h->H / h->Hkv;
-    const size_t smem = ((size_t)grp * split_len + (size_t)grp * HD + (size_t)(kAttnBwThreads / 32) * grp * HD) * sizeof(float);
+    const size_t smem = ((size_t)(kAttnBwThreads / 32) * grp * (HD + 2)) * sizeof(float);
     auto part = k_attn_split_bf16<HD>;
     static bool attr_set = false;
     if (!attr_set) { cudaFuncSetAttribute(part, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr_set = true; }
@@ -473,8 +473,10 @@ int setup_tc(tabed_handle* h) {
   h->tc_off[KIND_DN] = h->tc_off[KIND_GU] + h->tck[KIND_GU].bytes;
   h->tc_layer_stride = h->tc_off[KIND_DN] + h->tck[KIND_DN].bytes;
   h->tc_off[KIND_LM] = h->tc_layer_stride * h->L;
-  const int n_pad_max = (std::min(h->R, kTcMaxN) + 15) / 16 * 16;
-  h->tc_smem = (size_t)kTcStages * (tc_block_bytes(kTcM) + tc_block_bytes(n_pad_max)) + 1024;
+  const int n_pad_max = (std::min(2 * h->R, kTcMaxN) + 15) / 16 * 16;
+  h->tc_smem = 0;
+  for (int np = 16; np <= n_pad_max; np += 16)
+    h->tc_smem = std::max(h->tc_smem, (size_t)tc_stages(np) * (tc_block_bytes(kTcM) + tc_block_bytes(np)) + 1024);
   if (h->tc_smem > (size_t)prop.sharedMemPerBlockOptin) return TABED_OK;
   if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->tc_smem) != cudaSuccess) return TABED_ERR_CUDA;
   int rc = TABED_OK;
@@ -514,7 +516,8 @@ void launch_gemm_tc(tabed_handle* h, int kind, int layer, int n, float* partial,
   G.b_packed = h->tc_act; G.partial = partial; G.slab = slab; G.slots = slots;
   G.rows_total = t.rows; G.rows_valid = rows_valid; G.n_pad = (n + 15) / 16 * 16; G.n_slots = n;
   G.k_chunks = t.k_chunks; G.ks = t.ks; G.cps = t.cps; G.err = h->err;
-  TABED_LAUNCH(h, k_gemm_tc, t.m_tiles * t.ks, kTcThreads, h->tc_smem, G);
+  const size_t smem = (size_t)tc_stages(G.n_pad) * (tc_block_bytes(kTcM) + tc_block_bytes(G.n_pad)) + 1024;
+  TABED_LAUNCH(h, k_gemm_tc, t.m_tiles * t.ks, kTcThreads, smem, G);
 }
 
 // One shared-weight decoder step over `n_slots` slots with the projections on the tensor cores.
@@ -527,9 +530,8 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
   const size_t S2 = 2 * (size_t)h->R;
   const int d = h->d, HD = h->H * h->hd, F = h->F;
   struct Grp { int s0, n; };
-  std::vector<Grp> groups;                       // groups never straddle the two halves of a first step
-  for (int half = 0; half * h->R < n_slots; ++half)
-    for (int g0 = 0; g0 < h->R; g0 += kTcMaxN) groups.push_back({half * h->R + g0, std::min(kTcMaxN, h->R - g0)});
+  std::vector<Grp> groups;                       // up to 256 slots share one pass over the weights
+  for (int g0 = 0; g0 < n_slots; g0 += kTcMaxN) groups.push_back({g0, std::min(kTcMaxN, n_slots - g0)});
   auto prep_row = [&](const Grp& g, const float* partial, int ks, size_t slab, int write_back, const void* gain, const int* src, const SlotDesc* slots) {
     PrepRowArgs P{};
     P.x = h->x; P.d = d; P.partial = partial; P.ks = partial ? ks : 0; P.slab = slab; P.src_slot = src; P.slots = slots;
@@ -1130,7 +1132,7 @@ int tabed_debug_gemm_tc(const void* w, const float* act, int32_t rows, int32_t K
   const int cps = (k_chunks + ks - 1) / ks;
   unsigned char *a_p = nullptr, *b_p = nullptr; float* part = nullptr; int* err = nullptr;
   int rc = TABED_OK;
-  const size_t smem = (size_t)kTcStages * (tc_block_bytes(kTcM) + tc_block_bytes(n_pad)) + 1024;
+  const size_t smem = (size_t)tc_stages(n_pad) * (tc_block_bytes(kTcM) + tc_block_bytes(n_pad)) + 1024;
   if (cudaMalloc(&a_p, (size_t)m_tiles * k_chunks * tc_block_bytes(kTcM)) != cudaSuccess ||
       cudaMalloc(&b_p, (size_t)k_chunks * tc_block_bytes(n_pad)) != cudaSuccess ||
       cudaMalloc(&part, (size_t)ks * n * rows * sizeof(float)) != cudaSuccess || cudaMalloc(&err, sizeof(int)) != cudaSuccess ||

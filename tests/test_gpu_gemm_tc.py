@@ -18,7 +18,7 @@ def _case(rows, K, n, seed):
 
 
 @pytest.mark.parametrize("rows,K,n,ks", [(128, 128, 16, 1), (256, 256, 96, 1), (768, 768, 96, 3), (2304, 768, 96, 6),
-                                         (384, 200, 5, 1), (768, 3072, 128, 24), (1000, 768, 33, 2)])
+                                         (384, 200, 5, 1), (768, 3072, 128, 24), (1000, 768, 33, 2), (768, 768, 192, 6), (256, 384, 256, 1)])
 def test_gemm_tc_matches_float64_product(rows, K, n, ks):
     from paper_2601_20357_b200 import binding as TB
     dev = torch.device("cuda", 0)
@@ -38,6 +38,6 @@ def test_gemm_tc_rejects_bad_sizes():
     w, a = _case(128, 132, 4, 7)
     with pytest.raises(TB.TabedError):
         TB.debug_gemm_tc(w.to(dev), a.to(dev), 1)          # K not a multiple of 8
-    w, a = _case(128, 128, 200, 7)
+    w, a = _case(128, 128, 300, 7)
     with pytest.raises(TB.TabedError):
-        TB.debug_gemm_tc(w.to(dev), a.to(dev), 1)          # more than 128 slots per launch
+        TB.debug_gemm_tc(w.to(dev), a.to(dev), 1)          # more than 256 slots per launch
