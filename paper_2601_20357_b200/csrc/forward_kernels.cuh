@@ -476,8 +476,8 @@ k_attn_split_bf16(const float* __restrict__ qkv, const SlotDesc* __restrict__ sl
     const int p = ps * PPB + warp * PPW + pgrp;
     kreg[ps] = make_uint4(0u, 0u, 0u, 0u); vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
     if (p < cnt) {
-      kreg[ps] = __ldg(reinterpret_cast<const uint4*>(kc + base + (size_t)(p_lo + p) * HD + sub * 8));
-      vreg[ps] = __ldg(reinterpret_cast<const uint4*>(vc + base + (size_t)(p_lo + p) * HD + sub * 8));
+      kreg[ps] = __ldcs(reinterpret_cast<const uint4*>(kc + base + (size_t)(p_lo + p) * HD + sub * 8));
+      vreg[ps] = __ldcs(reinterpret_cast<const uint4*>(vc + base + (size_t)(p_lo + p) * HD + sub * 8));
     }
   }
   const float* qrow = qkv + (size_t)s * (H + 2 * Hkv) * HD + (size_t)g * grp * HD;

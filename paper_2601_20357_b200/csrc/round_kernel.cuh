@@ -174,6 +174,7 @@ struct PShared {
   float q[kMaxGroup][128];
   float kf[2][128], vf[2][128];
   float red[kPW][kPSlots];
+  float red2[kPW][kPSlots];
   unsigned long long red64[kPW];
   unsigned long long cm[kPT];
   float bestv[kPW]; int besti[kPW];
@@ -670,6 +671,12 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       GRID_SYNC();
 
       // ---- attention over the rows' caches (after the QKV phase) -----------------------------------
+      // Work item = (slot, KV head, split of split_len positions).  A warp keeps its 4 x PPW positions of K
+      // and V in registers, runs its own softmax over them and leaves (max, sum, un-normalised output) in
+      // shared memory; one block-wide exchange merges the 16 warps and the positions produced in this
+      // very phase (they come from the QKV output, not from the cache).  The next item's K and V loads are
+      // issued as soon as the current item's registers are free, so they fly during the merge and the
+      // next item's staging.
       if (kind == KIND_QKV) {
         const int split_len = A.split_len;
         const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
@@ -679,8 +686,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll 1
         for (int s = 0; s < ns; ++s)
           if (S.slot[s].active) total_items += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
-#pragma unroll 1
-        for (int item = cta; item < total_items; item += NC) {
+        struct Item { int s, gk, split, nsplit, pos, p_lo, cnt, fresh_lo; size_t cache_off; };
+        auto decode = [&](int item, Item& it) -> bool {
+          if (item >= total_items) return false;
           int s = 0, rem = item, nsplit = 0;
 #pragma unroll 1
           for (; s < ns; ++s) {
@@ -688,35 +696,39 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             if (rem < A.Hkv * nsplit) break;
             rem -= A.Hkv * nsplit;
           }
-          if (s >= ns) break;
-          const int gk = rem / nsplit, split = rem - gk * nsplit;
-          const PSlot si = S.slot[s];
-          const int pos = si.pos, n_pos = pos + 1;
-          const int p_lo = split * split_len, p_hi = min(p_lo + split_len, n_pos), cnt = p_hi - p_lo;
-          const int second = s >= R;
-          const int n_fresh = second ? 2 : 1;          // positions whose K,V are produced in this very phase
-          const int fresh_lo = pos - (n_fresh - 1);    // absolute positions >= fresh_lo are fresh
-          const size_t cache_off = ((((size_t)si.row * A.L + layer) * A.Hkv + gk) * A.cap) * A.hd;
-          const __nv_bfloat16* kbase = A.kc + cache_off;
-          const __nv_bfloat16* vbase = A.vc + cache_off;
-          // all cache loads of the item go out first: one memory round trip for K, V and q together
-          uint4 kreg[4], vreg[4];
+          if (s >= ns) return false;
+          it.s = s; it.nsplit = nsplit; it.gk = rem / nsplit; it.split = rem - it.gk * nsplit;
+          it.pos = S.slot[s].pos;
+          it.p_lo = it.split * split_len;
+          it.cnt = min(split_len, it.pos + 1 - it.p_lo);
+          it.fresh_lo = it.pos - (s >= R ? 1 : 0);       // absolute positions >= fresh_lo are produced in this phase
+          it.cache_off = ((((size_t)S.slot[s].row * A.L + layer) * A.Hkv + it.gk) * A.cap) * A.hd;
+          return true;
+        };
+        uint4 kreg[4], vreg[4];
+        Item cur, nxt;
+        bool have = decode(cta, cur);
+        if (have) {
 #pragma unroll
           for (int ps = 0; ps < 4; ++ps) {
             const int p = ps * PPB + warp * PPW + pgrp;
             kreg[ps] = make_uint4(0u, 0u, 0u, 0u);
-            if (p < cnt && p_lo + p < fresh_lo)
-              kreg[ps] = __ldcg(reinterpret_cast<const uint4*>(kbase + (size_t)(p_lo + p) * A.hd + sub * 8));
-          }
-#pragma unroll
-          for (int ps = 0; ps < 4; ++ps) {
-            const int p = ps * PPB + warp * PPW + pgrp;
             vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
-            if (p < cnt && p_lo + p < fresh_lo)
-              vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(vbase + (size_t)(p_lo + p) * A.hd + sub * 8));
+            if (p < cur.cnt && cur.p_lo + p < cur.fresh_lo) {
+              kreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.kc + cur.cache_off + (size_t)(cur.p_lo + p) * A.hd + sub * 8));
+              vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.vc + cur.cache_off + (size_t)(cur.p_lo + p) * A.hd + sub * 8));
+            }
           }
-          // stage q (all heads of the group), fresh k and v: RoPE, bf16 rounding.
-          // One index space so that every element is fetched by a different thread in one round trip.
+        }
+        int item = cta;
+#pragma unroll 1
+        while (have) {
+          const bool have_next = decode(item + NC, nxt);
+          const int s = cur.s, gk = cur.gk, split = cur.split, nsplit = cur.nsplit, pos = cur.pos;
+          const int p_lo = cur.p_lo, cnt = cur.cnt, p_hi = p_lo + cnt, fresh_lo = cur.fresh_lo;
+          const int n_fresh = pos - fresh_lo + 1;
+          // stage q (all heads of the group), fresh k and v: RoPE, bf16 rounding.  One index space so
+          // that every element is fetched by a different thread in one round trip.
           {
             const int n_q = grp * half, n_k = n_fresh * half, n_v = n_fresh * A.hd;
 #pragma unroll 1
@@ -745,18 +757,30 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           __syncthreads();
           TSEC(0);
           if (split == nsplit - 1 && tid < A.hd) {       // this item owns the append of its own position
-            A.kc[cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.kf[0][tid]);
-            A.vc[cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
+            A.kc[cur.cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.kf[0][tid]);
+            A.vc[cur.cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
           }
-          // ---- scores of the cached positions, one query head at a time (K stays in registers) ----
+          // scores of the fresh positions (this split's range only) from the staged k
+#pragma unroll 1
+          for (int combo = warp; combo < grp * n_fresh; combo += kPW) {
+            const int t = combo / n_fresh, j = combo - t * n_fresh;
+            float dd = 0.0f;
+#pragma unroll 1
+            for (int i = lane; i < A.hd; i += 32) dd = fmaf(S.kf[j][i], S.q[t][i], dd);
+            dd = warp_sum_f32(dd);
+            const int pj = pos - j;
+            if (lane == 0) S.sc[t][j] = (pj >= p_lo && pj < p_hi) ? dd * A.attn_scale : -INFINITY;
+          }
+          // ---- per warp: scores, softmax and P V over its cached positions, one query head at a time ----
 #pragma unroll 1
           for (int t = 0; t < grp; ++t) {
             float qf[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) qf[e] = S.q[t][sub * 8 + e];
+            float scv[4];
+            float mx = -INFINITY;
 #pragma unroll
             for (int ps = 0; ps < 4; ++ps) {
-              if (ps * PPB >= cnt) break;                 // uniform over the CTA
               const int p = ps * PPB + warp * PPW + pgrp;
               float kf8[8];
               Elem<__nv_bfloat16>::unpack(kreg[ps], kf8);
@@ -765,101 +789,83 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               for (int e = 0; e < 8; ++e) dd = fmaf(kf8[e], qf[e], dd);
 #pragma unroll 1
               for (int o = LPR >> 1; o > 0; o >>= 1) dd += __shfl_xor_sync(0xffffffffu, dd, o);
-              if (sub == 0 && p < cnt && p_lo + p < fresh_lo) S.sc[t][p] = dd * A.attn_scale;
+              scv[ps] = (p < cnt && p_lo + p < fresh_lo) ? dd * A.attn_scale : -INFINITY;
+              mx = fmaxf(mx, scv[ps]);
             }
-          }
-          // scores of the fresh positions come from the staged k, not from the cache
-#pragma unroll 1
-          for (int combo = warp; combo < grp * n_fresh; combo += kPW) {
-            const int t = combo / n_fresh, j = combo - t * n_fresh;
-            const int pj = pos - j;
-            if (pj >= p_lo && pj < p_hi) {
-              float dd = 0.0f;
-#pragma unroll 1
-              for (int i = lane; i < A.hd; i += 32) dd = fmaf(S.kf[j][i], S.q[t][i], dd);
-              dd = warp_sum_f32(dd);
-              if (lane == 0) S.sc[t][pj - p_lo] = dd * A.attn_scale;
+            if (t == grp - 1 && have_next) {             // K registers are free: the next item's K goes out now
+#pragma unroll
+              for (int ps = 0; ps < 4; ++ps) {
+                const int p = ps * PPB + warp * PPW + pgrp;
+                kreg[ps] = make_uint4(0u, 0u, 0u, 0u);
+                if (p < nxt.cnt && nxt.p_lo + p < nxt.fresh_lo)
+                  kreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.kc + nxt.cache_off + (size_t)(nxt.p_lo + p) * A.hd + sub * 8));
+              }
             }
-          }
-          __syncthreads();
-          {
-            // softmax statistics: 16/grp warps share a head
-            const int wph = (grp >= kPW) ? 1 : kPW / grp;
-            const int t = warp / wph, wi = warp - t * wph;
-            float mx = -INFINITY;
-            if (t < grp) for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) mx = fmaxf(mx, S.sc[t][p]);
-            mx = warp_max_f32(mx);
-            if (lane == 0) S.red[warp][0] = mx;
-            __syncthreads();
-            float sum = 0.0f;
-            if (t < grp) {
-              mx = S.red[t * wph][0];
 #pragma unroll 1
-              for (int w2 = 1; w2 < wph; ++w2) mx = fmaxf(mx, S.red[t * wph + w2][0]);
-#pragma unroll 1
-              for (int p = wi * 32 + lane; p < cnt; p += 32 * wph) { const float e = expf(S.sc[t][p] - mx); S.sc[t][p] = e; sum += e; }
-            }
-            sum = warp_sum_f32(sum);
-            if (lane == 0) S.red[warp][1] = sum;
-            __syncthreads();
-            if (t < grp && wi == 0 && lane == 0) {
-              float tot = 0.0f;
-#pragma unroll 1
-              for (int w2 = 0; w2 < wph; ++w2) tot += S.red[t * wph + w2][1];
-              S.m_[t] = mx; S.l_[t] = tot;
-            }
-          }
-          TSEC(1);
-          // ---- P V over the cached positions, one head at a time (V stays in registers) ----
-#pragma unroll 1
-          for (int t = 0; t < grp; ++t) {
-            float oacc[8];
+            for (int o = LPR; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float oacc[8], sum = 0.0f;
 #pragma unroll
             for (int e = 0; e < 8; ++e) oacc[e] = 0.0f;
 #pragma unroll
             for (int ps = 0; ps < 4; ++ps) {
-              if (ps * PPB >= cnt) break;
-              const int p = ps * PPB + warp * PPW + pgrp;
-              if (p < cnt && p_lo + p < fresh_lo) {
-                float vf8[8];
-                Elem<__nv_bfloat16>::unpack(vreg[ps], vf8);
-                const float pw = S.sc[t][p];
+              const float pw = (scv[ps] > -INFINITY) ? expf(scv[ps] - mx) : 0.0f;
+              sum += pw;
+              float vf8[8];
+              Elem<__nv_bfloat16>::unpack(vreg[ps], vf8);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf8[e], oacc[e]);
+              for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf8[e], oacc[e]);
+            }
+            if (t == grp - 1 && have_next) {             // ... and its V
+#pragma unroll
+              for (int ps = 0; ps < 4; ++ps) {
+                const int p = ps * PPB + warp * PPW + pgrp;
+                vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
+                if (p < nxt.cnt && nxt.p_lo + p < nxt.fresh_lo)
+                  vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.vc + nxt.cache_off + (size_t)(nxt.p_lo + p) * A.hd + sub * 8));
               }
             }
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              float v = oacc[e];
 #pragma unroll 1
-              for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-              oacc[e] = v;
+            for (int o = LPR; o < 32; o <<= 1) {
+              sum += __shfl_xor_sync(0xffffffffu, sum, o);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) oacc[e] += __shfl_xor_sync(0xffffffffu, oacc[e], o);
             }
             if (pgrp == 0) {
 #pragma unroll
               for (int e = 0; e < 8; ++e) s_o[((size_t)warp * grp + t) * A.hd + sub * 8 + e] = oacc[e];
+              if (sub == 0) { S.red[warp][t] = mx; S.red2[warp][t] = sum; }
             }
           }
           __syncthreads();
+          TSEC(1);
+          // ---- merge the warps (in warp order) and the fresh positions ----
           const bool single = nsplit == 1;
 #pragma unroll 1
           for (int idx = tid; idx < grp * A.hd; idx += kPT) {
             const int t = idx / A.hd, dd = idx - t * A.hd;
-            float v = 0.0f;
+            float M = -INFINITY;
 #pragma unroll
-            for (int w2 = 0; w2 < kPW; ++w2) v += s_o[((size_t)w2 * grp + t) * A.hd + dd];
-#pragma unroll 1
+            for (int w2 = 0; w2 < kPW; ++w2) M = fmaxf(M, S.red[w2][t]);
+            for (int j = 0; j < n_fresh; ++j) M = fmaxf(M, S.sc[t][j]);
+            float v = 0.0f, l = 0.0f;
+#pragma unroll
+            for (int w2 = 0; w2 < kPW; ++w2) {
+              const float mw = S.red[w2][t];
+              const float f = (mw > -INFINITY) ? expf(mw - M) : 0.0f;
+              v = fmaf(f, s_o[((size_t)w2 * grp + t) * A.hd + dd], v);
+              l = fmaf(f, S.red2[w2][t], l);
+            }
             for (int j = 0; j < n_fresh; ++j) {
-              const int pj = pos - j;
-              if (pj >= p_lo && pj < p_hi) v = fmaf(S.sc[t][pj - p_lo], S.vf[j][dd], v);
+              const float sf = S.sc[t][j];
+              if (sf > -INFINITY) { const float f = expf(sf - M); v = fmaf(f, S.vf[j][dd], v); l += f; }
             }
             const int head = gk * grp + t;
             if (single) {
-              A.attn_out[(size_t)s * HD + head * A.hd + dd] = v / S.l_[t];
+              A.attn_out[(size_t)s * HD + head * A.hd + dd] = v / l;
             } else {
               const size_t pi = ((size_t)s * A.H + head) * A.max_splits + split;
               A.part_o[pi * A.hd + dd] = v;
-              if (dd == 0) { A.part_ml[pi * 2] = S.m_[t]; A.part_ml[pi * 2 + 1] = S.l_[t]; }
+              if (dd == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
             }
           }
           TSEC(2);
@@ -896,7 +902,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
                 const int head = gk * grp + t;
                 const size_t base = ((size_t)s * A.H + head) * A.max_splits;
                 float num = 0.0f;
-#pragma unroll 8
+#pragma unroll 4
                 for (int j = 0; j < nsplit; ++j) num = fmaf(S.sc[t][j], __ldcg(A.part_o + (base + j) * A.hd + dd), num);
                 A.attn_out[(size_t)s * HD + head * A.hd + dd] = num / S.l_[t];
               }
@@ -905,6 +911,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           __syncthreads();
           TSEC(3);
+          cur = nxt; have = have_next; item += NC;
         }
         GRID_SYNC();
       }

@@ -679,7 +679,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
       for (int o : opts) if (o < h->ns) lower = o;
       h->ns = lower;
     }
-    h->max_splits = (h->cap + 63) / 64;           // the shortest attention split any kernel uses is 64 positions
+    { const int shortest = std::min(64, attn_bw_split_len(h->hd)); h->max_splits = (h->cap + shortest - 1) / shortest; }   // shortest attention split of any kernel
     h->embed = wts->embed; h->lm_head = wts->lm_head; h->final_norm = wts->final_norm;
     for (int l = 0; l < h->L; ++l) {
       h->wq.push_back(wts->wq[l]); h->wk.push_back(wts->wk[l]); h->wv.push_back(wts->wv[l]); h->wo.push_back(wts->wo[l]);
