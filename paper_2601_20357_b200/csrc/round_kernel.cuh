@@ -184,6 +184,7 @@ struct PShared {
   float m_[kMaxGroup], l_[kMaxGroup];
   PSlot slot[kPSlots];
   int lm_src[kPSlots];
+  int segfirst[kPT];
   int tok[kPSlots];
   int dead, flag, result, chunk;
   unsigned long long thr;
@@ -671,65 +672,75 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       GRID_SYNC();
 
       // ---- attention over the rows' caches (after the QKV phase) -----------------------------------
-      // Work item = (slot, KV head, split of split_len positions).  A warp keeps its 4 x PPW positions of K
-      // and V in registers, runs its own softmax over them and leaves (max, sum, un-normalised output) in
-      // shared memory; one block-wide exchange merges the 16 warps and the positions produced in this
-      // very phase (they come from the QKV output, not from the cache).  The next item's K and V loads are
-      // issued as soon as the current item's registers are free, so they fly during the merge and the
-      // next item's staging.
+      // The caches of all (slot, KV head) pairs are cut into chunks of split_len positions; the chunks, in
+      // (slot, head, position) order, are dealt to the CTAs in contiguous ranges, so a CTA walks along one
+      // cache for several chunks.  A warp keeps its positions of K and V in registers, runs its own
+      // softmax and ACCUMULATES (max, sum, un-normalised output) per head in shared memory across the
+      // chunks of a segment (= the part of one pair's cache this CTA owns): no block-wide exchange per
+      // chunk, the next chunk's K and V are requested as soon as the registers are free.  At the end of
+      // a segment the 16 warps are merged (plus the positions produced in this very phase, which come
+      // from the QKV output, not from the cache); pairs that span several CTAs are combined by the CTA
+      // that finishes last (ticket), in segment order.
       if (kind == KIND_QKV) {
-        const int split_len = A.split_len;
         const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
         const int PPW = 32 / LPR, PPB = kPW * PPW;     // positions per warp / per CTA pass
         const int sub = lane % LPR, pgrp = lane / LPR;
-        int total_items = 0;
+        // chunks of split_len positions (4 register passes of the CTA); short caches give fewer chunks than
+        // CTAs - shorter chunks were measured slower there (more segments to merge, the phase is latency-bound)
+        const int split_len = A.split_len;
+        int T = 0;
 #pragma unroll 1
         for (int s = 0; s < ns; ++s)
-          if (S.slot[s].active) total_items += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
-        struct Item { int s, gk, split, nsplit, pos, p_lo, cnt, fresh_lo; size_t cache_off; };
-        auto decode = [&](int item, Item& it) -> bool {
-          if (item >= total_items) return false;
-          int s = 0, rem = item, nsplit = 0;
+          if (S.slot[s].active) T += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
+        // (T <= 8 slots x 64 heads x 256 chunks, so c * T stays far below 2^31)
+        const int g_lo = cta * T / NC, g_hi = (cta + 1) * T / NC;
+        // walker over (slot, head, split) in global chunk order
+        struct Walk { int s, gk, split, nsplit, g0; };          // g0 = global index of the pair's first chunk
+        auto seek = [&](int g, Walk& w) {
+          int s = 0, rem = g, acc = 0, nsplit = 0;
 #pragma unroll 1
           for (; s < ns; ++s) {
             nsplit = S.slot[s].active ? (S.slot[s].pos + split_len) / split_len : 0;
             if (rem < A.Hkv * nsplit) break;
-            rem -= A.Hkv * nsplit;
+            rem -= A.Hkv * nsplit; acc += A.Hkv * nsplit;
           }
-          if (s >= ns) return false;
-          it.s = s; it.nsplit = nsplit; it.gk = rem / nsplit; it.split = rem - it.gk * nsplit;
-          it.pos = S.slot[s].pos;
-          it.p_lo = it.split * split_len;
-          it.cnt = min(split_len, it.pos + 1 - it.p_lo);
-          it.fresh_lo = it.pos - (s >= R ? 1 : 0);       // absolute positions >= fresh_lo are produced in this phase
-          it.cache_off = ((((size_t)S.slot[s].row * A.L + layer) * A.Hkv + it.gk) * A.cap) * A.hd;
-          return true;
+          w.s = s; w.nsplit = nsplit; w.gk = nsplit ? rem / nsplit : 0; w.split = nsplit ? rem - w.gk * nsplit : 0;
+          w.g0 = acc + w.gk * nsplit;
         };
-        uint4 kreg[4], vreg[4];
-        Item cur, nxt;
-        bool have = decode(cta, cur);
-        if (have) {
+        auto issue_loads = [&](const Walk& w, uint4 (&kr)[4], uint4 (&vr)[4], bool want_k, bool want_v) {
+          const int pos = S.slot[w.s].pos;
+          const int p_lo = w.split * split_len, cnt = min(split_len, pos + 1 - p_lo);
+          const int fresh_lo = pos - (w.s >= R ? 1 : 0);
+          const size_t off = ((((size_t)S.slot[w.s].row * A.L + layer) * A.Hkv + w.gk) * A.cap) * A.hd;
 #pragma unroll
           for (int ps = 0; ps < 4; ++ps) {
             const int p = ps * PPB + warp * PPW + pgrp;
-            kreg[ps] = make_uint4(0u, 0u, 0u, 0u);
-            vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
-            if (p < cur.cnt && cur.p_lo + p < cur.fresh_lo) {
-              kreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.kc + cur.cache_off + (size_t)(cur.p_lo + p) * A.hd + sub * 8));
-              vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.vc + cur.cache_off + (size_t)(cur.p_lo + p) * A.hd + sub * 8));
-            }
+            const bool ok = p < cnt && p_lo + p < fresh_lo;
+            if (want_k) kr[ps] = ok ? __ldcg(reinterpret_cast<const uint4*>(A.kc + off + (size_t)(p_lo + p) * A.hd + sub * 8)) : make_uint4(0u, 0u, 0u, 0u);
+            if (want_v) vr[ps] = ok ? __ldcg(reinterpret_cast<const uint4*>(A.vc + off + (size_t)(p_lo + p) * A.hd + sub * 8)) : make_uint4(0u, 0u, 0u, 0u);
           }
-        }
-        int item = cta;
+        };
+        uint4 kreg[4], vreg[4];
+        Walk cur{0, 0, 0, 0, 0}, nxt{0, 0, 0, 0, 0};
+        if (g_lo < g_hi) { seek(g_lo, cur); issue_loads(cur, kreg, vreg, true, true); }
+        int seg_first_split = 0;
 #pragma unroll 1
-        while (have) {
-          const bool have_next = decode(item + NC, nxt);
-          const int s = cur.s, gk = cur.gk, split = cur.split, nsplit = cur.nsplit, pos = cur.pos;
-          const int p_lo = cur.p_lo, cnt = cur.cnt, p_hi = p_lo + cnt, fresh_lo = cur.fresh_lo;
-          const int n_fresh = pos - fresh_lo + 1;
-          // stage q (all heads of the group), fresh k and v: RoPE, bf16 rounding.  One index space so
-          // that every element is fetched by a different thread in one round trip.
-          {
+        for (int g = g_lo; g < g_hi; ++g) {
+          const bool have_next = g + 1 < g_hi;
+          if (have_next) {
+            nxt = cur; nxt.split++;
+            if (nxt.split == nxt.nsplit) seek(g + 1, nxt);
+          }
+          const int s = cur.s, gk = cur.gk, split = cur.split, nsplit = cur.nsplit;
+          const int pos = S.slot[s].pos;
+          const int p_lo = split * split_len, cnt = min(split_len, pos + 1 - p_lo);
+          const int fresh_lo = pos - (s >= R ? 1 : 0), n_fresh = pos - fresh_lo + 1;
+          const bool seg_start = (g == g_lo) || split == 0;
+          const bool seg_end = !have_next || split == nsplit - 1;
+          if (seg_start) {
+            seg_first_split = split;
+            // stage q (all heads of the group), fresh k and v: RoPE, bf16 rounding.  One index space so
+            // that every element is fetched by a different thread in one round trip.
             const int n_q = grp * half, n_k = n_fresh * half, n_v = n_fresh * A.hd;
 #pragma unroll 1
             for (int idx = tid; idx < n_q + n_k + n_v; idx += kPT) {
@@ -753,25 +764,15 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               dst[0] = round_bf16(x1 * cs - x2 * sn);
               if (pair) dst[half] = round_bf16(x2 * cs + x1 * sn);
             }
+            __syncthreads();
+            TSEC(0);
+            if (split + (g_hi - 1 - g) >= nsplit - 1 && tid < A.hd) {   // this segment reaches the pair's last split: it appends the new position
+              const size_t off = ((((size_t)S.slot[s].row * A.L + layer) * A.Hkv + gk) * A.cap) * A.hd;
+              A.kc[off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.kf[0][tid]);
+              A.vc[off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
+            }
           }
-          __syncthreads();
-          TSEC(0);
-          if (split == nsplit - 1 && tid < A.hd) {       // this item owns the append of its own position
-            A.kc[cur.cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.kf[0][tid]);
-            A.vc[cur.cache_off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
-          }
-          // scores of the fresh positions (this split's range only) from the staged k
-#pragma unroll 1
-          for (int combo = warp; combo < grp * n_fresh; combo += kPW) {
-            const int t = combo / n_fresh, j = combo - t * n_fresh;
-            float dd = 0.0f;
-#pragma unroll 1
-            for (int i = lane; i < A.hd; i += 32) dd = fmaf(S.kf[j][i], S.q[t][i], dd);
-            dd = warp_sum_f32(dd);
-            const int pj = pos - j;
-            if (lane == 0) S.sc[t][j] = (pj >= p_lo && pj < p_hi) ? dd * A.attn_scale : -INFINITY;
-          }
-          // ---- per warp: scores, softmax and P V over its cached positions, one query head at a time ----
+          // ---- per warp: scores, softmax, P V over its cached positions of this chunk, head by head ----
 #pragma unroll 1
           for (int t = 0; t < grp; ++t) {
             float qf[8];
@@ -792,15 +793,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               scv[ps] = (p < cnt && p_lo + p < fresh_lo) ? dd * A.attn_scale : -INFINITY;
               mx = fmaxf(mx, scv[ps]);
             }
-            if (t == grp - 1 && have_next) {             // K registers are free: the next item's K goes out now
-#pragma unroll
-              for (int ps = 0; ps < 4; ++ps) {
-                const int p = ps * PPB + warp * PPW + pgrp;
-                kreg[ps] = make_uint4(0u, 0u, 0u, 0u);
-                if (p < nxt.cnt && nxt.p_lo + p < nxt.fresh_lo)
-                  kreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.kc + nxt.cache_off + (size_t)(nxt.p_lo + p) * A.hd + sub * 8));
-              }
-            }
+            if (t == grp - 1 && have_next) issue_loads(nxt, kreg, vreg, true, false);   // K registers are free
 #pragma unroll 1
             for (int o = LPR; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             float oacc[8], sum = 0.0f;
@@ -815,15 +808,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll
               for (int e = 0; e < 8; ++e) oacc[e] = fmaf(pw, vf8[e], oacc[e]);
             }
-            if (t == grp - 1 && have_next) {             // ... and its V
-#pragma unroll
-              for (int ps = 0; ps < 4; ++ps) {
-                const int p = ps * PPB + warp * PPW + pgrp;
-                vreg[ps] = make_uint4(0u, 0u, 0u, 0u);
-                if (p < nxt.cnt && nxt.p_lo + p < nxt.fresh_lo)
-                  vreg[ps] = __ldcg(reinterpret_cast<const uint4*>(A.vc + nxt.cache_off + (size_t)(nxt.p_lo + p) * A.hd + sub * 8));
-              }
-            }
+            if (t == grp - 1 && have_next) issue_loads(nxt, kreg, vreg, false, true);   // ... and the V registers
 #pragma unroll 1
             for (int o = LPR; o < 32; o <<= 1) {
               sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -831,87 +816,133 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               for (int e = 0; e < 8; ++e) oacc[e] += __shfl_xor_sync(0xffffffffu, oacc[e], o);
             }
             if (pgrp == 0) {
+              // accumulate into the warp's running state of this segment (only this warp touches it)
+              float* so_w = s_o + ((size_t)warp * grp + t) * A.hd + sub * 8;
+              float m_old = -INFINITY, l_old = 0.0f;
+              if (!seg_start) { m_old = S.red[warp][t]; l_old = S.red2[warp][t]; }
+              const float M = fmaxf(m_old, mx);
+              const float f_old = (m_old > -INFINITY) ? expf(m_old - M) : 0.0f;
+              const float f_new = (mx > -INFINITY) ? expf(mx - M) : 0.0f;
 #pragma unroll
-              for (int e = 0; e < 8; ++e) s_o[((size_t)warp * grp + t) * A.hd + sub * 8 + e] = oacc[e];
-              if (sub == 0) { S.red[warp][t] = mx; S.red2[warp][t] = sum; }
+              for (int e = 0; e < 8; ++e) so_w[e] = (seg_start ? 0.0f : so_w[e] * f_old) + oacc[e] * f_new;
+              if (sub == 0) { S.red[warp][t] = M; S.red2[warp][t] = l_old * f_old + sum * f_new; }
             }
+            __syncwarp();
           }
-          __syncthreads();
           TSEC(1);
-          // ---- merge the warps (in warp order) and the fresh positions ----
-          const bool single = nsplit == 1;
+          if (seg_end) {
+            const int seg_lo = seg_first_split * split_len, seg_hi = p_lo + cnt;     // positions covered by the segment
+            // scores of the fresh positions that fall into this segment, from the staged k
 #pragma unroll 1
-          for (int idx = tid; idx < grp * A.hd; idx += kPT) {
-            const int t = idx / A.hd, dd = idx - t * A.hd;
-            float M = -INFINITY;
-#pragma unroll
-            for (int w2 = 0; w2 < kPW; ++w2) M = fmaxf(M, S.red[w2][t]);
-            for (int j = 0; j < n_fresh; ++j) M = fmaxf(M, S.sc[t][j]);
-            float v = 0.0f, l = 0.0f;
-#pragma unroll
-            for (int w2 = 0; w2 < kPW; ++w2) {
-              const float mw = S.red[w2][t];
-              const float f = (mw > -INFINITY) ? expf(mw - M) : 0.0f;
-              v = fmaf(f, s_o[((size_t)w2 * grp + t) * A.hd + dd], v);
-              l = fmaf(f, S.red2[w2][t], l);
+            for (int combo = warp; combo < grp * n_fresh; combo += kPW) {
+              const int t = combo / n_fresh, j = combo - t * n_fresh;
+              float dd = 0.0f;
+#pragma unroll 1
+              for (int i = lane; i < A.hd; i += 32) dd = fmaf(S.kf[j][i], S.q[t][i], dd);
+              dd = warp_sum_f32(dd);
+              const int pj = pos - j;
+              if (lane == 0) S.sc[t][j] = (pj >= seg_lo && pj < seg_hi) ? dd * A.attn_scale : -INFINITY;
             }
-            for (int j = 0; j < n_fresh; ++j) {
-              const float sf = S.sc[t][j];
-              if (sf > -INFINITY) { const float f = expf(sf - M); v = fmaf(f, S.vf[j][dd], v); l += f; }
-            }
-            const int head = gk * grp + t;
-            if (single) {
-              A.attn_out[(size_t)s * HD + head * A.hd + dd] = v / l;
-            } else {
-              const size_t pi = ((size_t)s * A.H + head) * A.max_splits + split;
-              A.part_o[pi * A.hd + dd] = v;
-              if (dd == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
-            }
-          }
-          TSEC(2);
-          if (!single) {
-            // the CTA that finishes the last split of a (slot, kv head) merges them in split order
-            __threadfence();
             __syncthreads();
-            if (tid == 0) S.flag = (atomicAdd(A.tickets + s * A.Hkv + gk, 1) == nsplit - 1);
-            __syncthreads();
-            if (S.flag) {
+            // ---- merge the warps (in warp order) and the fresh positions ----
+            const bool whole = seg_first_split == 0 && split == nsplit - 1;
+#pragma unroll 1
+            for (int idx = tid; idx < grp * A.hd; idx += kPT) {
+              const int t = idx / A.hd, dd = idx - t * A.hd;
+              float M = -INFINITY;
+#pragma unroll
+              for (int w2 = 0; w2 < kPW; ++w2) M = fmaxf(M, S.red[w2][t]);
+              for (int j = 0; j < n_fresh; ++j) M = fmaxf(M, S.sc[t][j]);
+              float v = 0.0f, l = 0.0f;
+#pragma unroll
+              for (int w2 = 0; w2 < kPW; ++w2) {
+                const float mw = S.red[w2][t];
+                const float f = (mw > -INFINITY) ? expf(mw - M) : 0.0f;
+                v = fmaf(f, s_o[((size_t)w2 * grp + t) * A.hd + dd], v);
+                l = fmaf(f, S.red2[w2][t], l);
+              }
+              for (int j = 0; j < n_fresh; ++j) {
+                const float sf = S.sc[t][j];
+                if (sf > -INFINITY) { const float f = expf(sf - M); v = fmaf(f, S.vf[j][dd], v); l += f; }
+              }
+              const int head = gk * grp + t;
+              if (whole) {
+                A.attn_out[(size_t)s * HD + head * A.hd + dd] = v / l;
+              } else {
+                const size_t pi = ((size_t)s * A.H + head) * A.max_splits + seg_first_split;
+                A.part_o[pi * A.hd + dd] = v;
+                if (dd == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
+              }
+            }
+            TSEC(2);
+            if (!whole) {
+              // the pair's chunks [g0, g0 + nsplit) are spread over the CTAs c_a .. c_b, one segment each
+              // (CTAs without chunks excepted); the CTA whose ticket completes the pair merges the segments
+              // in CTA order.  S.segfirst[j] = first split of CTA c_a + j's segment, or -1.
+              const int c_a = ((cur.g0 + 1) * NC - 1) / T, c_b = ((cur.g0 + nsplit) * NC - 1) / T;
+              const int n_c = c_b - c_a + 1;
+#pragma unroll 1
+              for (int j = tid; j < n_c; j += kPT) {
+                const int lo_c = (c_a + j) * T / NC, hi_c = (c_a + j + 1) * T / NC;
+                S.segfirst[j] = (lo_c < hi_c) ? max(lo_c, cur.g0) - cur.g0 : -1;
+              }
               __threadfence();
+              __syncthreads();
+              if (tid == 0) {
+                int n_seg = 0;
 #pragma unroll 1
-              for (int t = warp; t < grp; t += kPW) {      // rescaling factors of the splits, one warp per head
-                const size_t base = ((size_t)s * A.H + gk * grp + t) * A.max_splits;
-                float M = -INFINITY;
-#pragma unroll 1
-                for (int j = lane; j < nsplit; j += 32) M = fmaxf(M, __ldcg(A.part_ml + (base + j) * 2));
-                M = warp_max_f32(M);
-                float den = 0.0f;
-#pragma unroll 1
-                for (int j = lane; j < nsplit; j += 32) {
-                  const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + j) * 2));
-                  const float f = expf(ml.x - M);
-                  S.sc[t][j] = f;
-                  den = fmaf(f, ml.y, den);
-                }
-                den = warp_sum_f32(den);
-                if (lane == 0) S.l_[t] = den;
+                for (int j = 0; j < n_c; ++j) n_seg += S.segfirst[j] >= 0;
+                S.flag = (atomicAdd(A.tickets + s * A.Hkv + gk, 1) == n_seg - 1);
               }
               __syncthreads();
+              if (S.flag) {
+                __threadfence();
 #pragma unroll 1
-              for (int idx = tid; idx < grp * A.hd; idx += kPT) {
-                const int t = idx / A.hd, dd = idx - t * A.hd;
-                const int head = gk * grp + t;
-                const size_t base = ((size_t)s * A.H + head) * A.max_splits;
-                float num = 0.0f;
-#pragma unroll 4
-                for (int j = 0; j < nsplit; ++j) num = fmaf(S.sc[t][j], __ldcg(A.part_o + (base + j) * A.hd + dd), num);
-                A.attn_out[(size_t)s * HD + head * A.hd + dd] = num / S.l_[t];
+                for (int t = warp; t < grp; t += kPW) {      // rescaling factors of the segments, one warp per head
+                  const size_t base = ((size_t)s * A.H + gk * grp + t) * A.max_splits;
+                  float M = -INFINITY;
+#pragma unroll 1
+                  for (int j = lane; j < n_c; j += 32) {
+                    const int first = S.segfirst[j];
+                    if (first >= 0) M = fmaxf(M, __ldcg(A.part_ml + (base + first) * 2));
+                  }
+                  M = warp_max_f32(M);
+                  float den = 0.0f;
+#pragma unroll 1
+                  for (int j = lane; j < n_c; j += 32) {
+                    const int first = S.segfirst[j];
+                    float f = 0.0f;
+                    if (first >= 0) {
+                      const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + first) * 2));
+                      f = expf(ml.x - M);
+                      den = fmaf(f, ml.y, den);
+                    }
+                    S.sc[t][j] = f;
+                  }
+                  den = warp_sum_f32(den);
+                  if (lane == 0) S.l_[t] = den;
+                }
+                __syncthreads();
+#pragma unroll 1
+                for (int idx = tid; idx < grp * A.hd; idx += kPT) {
+                  const int t = idx / A.hd, dd = idx - t * A.hd;
+                  const int head = gk * grp + t;
+                  const size_t base = ((size_t)s * A.H + head) * A.max_splits;
+                  float num = 0.0f;
+#pragma unroll 2
+                  for (int j = 0; j < n_c; ++j) {
+                    const int first = S.segfirst[j];
+                    if (first >= 0) num = fmaf(S.sc[t][j], __ldcg(A.part_o + (base + first) * A.hd + dd), num);
+                  }
+                  A.attn_out[(size_t)s * HD + head * A.hd + dd] = num / S.l_[t];
+                }
+                if (tid == 0) A.tickets[s * A.Hkv + gk] = 0;
               }
-              if (tid == 0) A.tickets[s * A.Hkv + gk] = 0;
             }
+            __syncthreads();
+            TSEC(3);
           }
-          __syncthreads();
-          TSEC(3);
-          cur = nxt; have = have_next; item += NC;
+          cur = nxt;
         }
         GRID_SYNC();
       }
