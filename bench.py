@@ -484,11 +484,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--trace", default=None, help="write the persistent kernel's phase timeline of one round to this file")
+    ap.add_argument("--requests", type=int, default=0, help="override the workload's number of concurrent requests (profiling aid)")
     ap.add_argument("--path", default="auto", choices=["auto", "per-op"], help="drafting path (per-op forces one kernel per operation)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     wl = W.WORKLOADS[args.config]
+    if args.requests > 0:
+        wl = wl.replace(n_requests=args.requests, name=f"{wl.name}[B={args.requests}]")
     if args.impl == "reference":
         run_reference(args, wl)
     else:

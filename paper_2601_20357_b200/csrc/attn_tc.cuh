@@ -1,0 +1,379 @@
+// Decode attention over bf16 K,V caches for MANY (slot, KV head) pairs in one launch (the drafting
+// step of Algorithm 1 with many rows: every slot attends over its own row's cache).
+//
+// The work is bound by reading the caches once, so the kernel is built around keeping HBM busy:
+//   * a fixed grid of CTAs, each walking a CONTIGUOUS range of the 128-position chunks of all
+//     (slot, KV head) caches in (slot, head, position) order;
+//   * a chunk of K and of V is one TMA tile each (cp.async.bulk.tensor, 128 rows x 64 dims, 128-byte
+//     swizzle), landing in a ring of shared-memory stages several chunks ahead of the arithmetic and
+//     signalling an mbarrier: the bytes in flight live in shared memory, not in registers;
+//   * the arithmetic runs on the tensor cores (mma.sync m16n8k16): rows of the A operand are the
+//     query heads that share the KV head (at most 8 of 16 rows are used: the contraction is far
+//     from the tensor roofline, the point is to keep the issue slots free).  q and the softmax
+//     weights are split into a bf16 head and a bf16 remainder (two products each), K and V are bf16
+//     already, so products are exact to ~2^-17 relative and the sums are fp32;
+//   * a warp owns 16 positions of every chunk and carries its own running (max, sum, output) in
+//     registers across the chunks of a segment (the part of one cache that this CTA owns).  The
+//     warps run free of one another: each waits for a stage on its own, the LAST warp to finish
+//     with a stage refills it (TMA of the chunk n_stages ahead), and the last warp to finish a
+//     segment combines the eight states and writes the result, while the others are already in
+//     the next segment.  q of a cache rides along with the first tile of its segment (one more
+//     bulk copy onto the same mbarrier);
+//   * segments of a cache that spans several CTAs are combined by the warp that finishes last
+//     (ticket), in CTA order, reading the partial results from L2;
+//   * exponentials are taken in base 2 (scores pre-multiplied by log2 e, ex2.approx: relative
+//     error 2^-22).
+// Rows past a slot's position inside the last tile are masked (score -inf, weight 0); the caches are
+// zero-initialised and only ever hold finite values, so the masked V rows contribute exactly 0.
+// Waits on the copies are bounded (error bit 16 in *err; the CTA stops and drains).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "forward_kernels.cuh"
+#include "round_kernel.cuh"
+
+namespace tabed {
+
+constexpr int kAtcThreads = 256;
+constexpr int kAtcWarps = kAtcThreads / 32;
+constexpr int kAtcSplit = 128;               // positions per chunk = rows of a TMA tile
+constexpr int kAtcHd = 64;                   // head size served by this kernel
+constexpr int kAtcTile = kAtcSplit * kAtcHd * 2;   // bytes of one K (or V) tile
+constexpr int kAtcMaxStages = 8;
+constexpr int kAtcMaxCtas = 1024;
+constexpr int kAtcMaxSlots = 512;
+constexpr unsigned kAtcMaxDynSmem = 220u * 1024u;   // dynamic shared memory of a CTA that has the SM to itself (static: ~3 KB)
+
+struct AttnTcArgs {
+  const float* qkv;                          // [n_slots][qkv_w] rotated q (k, v already in the caches)
+  const SlotDesc* slots;
+  int n_slots, H, Hkv, layer, L, cap, qkv_w;
+  float *part_o, *part_ml;                   // [n_slots][H][max_splits][hd], [..][2] segment partials
+  int max_splits;
+  int* tickets;                              // [n_slots][Hkv], zero on entry and on exit
+  float* out;                                // [n_slots][H][hd]
+  float scale;
+  int* err;
+  int n_stages;
+};
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// x = hi + lo with hi, lo bf16 (lo the rounded remainder); returns them packed for two values
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const float h0 = round_bf16(x0), h1 = round_bf16(x1);
+  hi = pack_bf16(h0, h1);
+  lo = pack_bf16(x0 - h0, x1 - h1);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(kAtcThreads, 2)
+k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const AttnTcArgs A) {
+  constexpr int HD = kAtcHd, NW = kAtcWarps, SPLIT = kAtcSplit;
+  constexpr unsigned FULL = 0xffffffffu;
+  const int H = A.H, Hkv = A.Hkv, grp = H / Hkv, NC = gridDim.x, cta = blockIdx.x, n_slots = A.n_slots;
+  const int n_stages = A.n_stages;
+  const SlotDesc* __restrict__ slots = A.slots;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t4 = lane & 3;
+  extern __shared__ unsigned char atc_raw[];
+  unsigned char* stage0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(atc_raw) + 1023) & ~(uintptr_t)1023);
+  float* sq = reinterpret_cast<float*>(stage0 + (size_t)n_stages * 2 * kAtcTile);   // [n_stages][grp][HD] q beside its stage
+  float* so = sq + (size_t)n_stages * grp * HD;                                     // [n_stages][NW][grp][HD] states of a segment
+  float* sm = so + (size_t)n_stages * NW * grp * HD;                                // [n_stages][NW][grp] running maxima (base 2)
+  float* sl = sm + n_stages * NW * grp;                                             // [n_stages][NW][grp] running sums
+  __shared__ uint64_t full[kAtcMaxStages];
+  __shared__ int s_done[kAtcMaxStages];         // warps that have finished with a stage
+  __shared__ int s_seg[kAtcMaxStages];          // warps that have finished a segment (ring of n_stages segments)
+  __shared__ int s_pref[kAtcMaxSlots + 1];
+  __shared__ int s_start;
+  if (tid == 0) {
+    for (int i = 0; i < n_stages; ++i) { mbar_init(&full[i], 1); s_done[i] = 0; s_seg[i] = 0; }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // chunks before every slot (prefix sums), built by the whole CTA
+  for (int i = tid; i < n_slots; i += kAtcThreads)
+    s_pref[i + 1] = slots[i].active ? Hkv * ((slots[i].pos + SPLIT) / SPLIT) : 0;
+  __syncthreads();
+  if (warp == 0) {
+    int carry = 0;
+    for (int base = 0; base < n_slots; base += 32) {
+      int v = (base + lane < n_slots) ? s_pref[base + lane + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(FULL, v, o); if (lane >= o) v += n; }
+      if (base + lane < n_slots) s_pref[base + lane + 1] = carry + v;
+      carry += __shfl_sync(FULL, v, 31);
+    }
+    if (lane == 0) s_pref[0] = 0;
+  }
+  __syncthreads();
+  const int T = s_pref[n_slots];
+  const int g_lo = (int)((long long)cta * T / NC), g_hi = (int)((long long)(cta + 1) * T / NC);
+  for (int i = tid; i < n_slots; i += kAtcThreads)
+    if (s_pref[i] <= g_lo && g_lo < s_pref[i + 1]) s_start = i;
+  struct Walk { int s, gk, split, nsplit, row, pos; };
+  auto advance = [&](Walk& w) {                      // to the next chunk in (slot, head, position) order
+    w.split++;
+    if (w.split == w.nsplit) {
+      w.split = 0; w.gk++;
+      if (w.gk == Hkv) {
+        w.gk = 0;
+        do { w.s++; } while (w.s < n_slots && !slots[w.s].active);
+        if (w.s < n_slots) { w.row = slots[w.s].row; w.pos = slots[w.s].pos; }
+        w.nsplit = (w.pos + SPLIT) / SPLIT;
+      }
+    }
+  };
+  // one thread: the two TMA tiles of chunk `w` into stage `st`; q of the cache with the first chunk of a segment
+  auto issue = [&](const Walk& w, int st, bool first) {
+    const int y = ((w.row * A.L + A.layer) * Hkv + w.gk) * A.cap + w.split * SPLIT;
+    const uint32_t dst = smem_u32(stage0 + (size_t)st * 2 * kAtcTile), bar = smem_u32(&full[st]);
+    const bool with_q = first || w.split == 0;
+    const unsigned qbytes = (unsigned)grp * HD * 4u;
+    mbar_expect_tx(&full[st], 2u * kAtcTile + (with_q ? qbytes : 0u));
+    tma_load_2d(dst, &tm_k, 0, y, bar);
+    tma_load_2d(dst + kAtcTile, &tm_v, 0, y, bar);
+    if (with_q) bulk_g2s(sq + (size_t)st * grp * HD, A.qkv + (size_t)w.s * A.qkv_w + (size_t)w.gk * grp * HD, qbytes, &full[st]);
+  };
+  __syncthreads();
+  // cur: the chunk a warp works on; ahead: the chunk n_stages later (the one that refills cur's stage)
+  Walk cur{0, 0, 0, 1, 0, 0}, ahead{0, 0, 0, 1, 0, 0};
+  if (g_lo < g_hi) {
+    const int rem = g_lo - s_pref[s_start];
+    cur.s = s_start;
+    cur.row = slots[s_start].row; cur.pos = slots[s_start].pos;
+    cur.nsplit = (cur.pos + SPLIT) / SPLIT;
+    cur.gk = rem / cur.nsplit;
+    cur.split = rem - cur.gk * cur.nsplit;
+    ahead = cur;
+    for (int i = 0; i < n_stages; ++i) {
+      if (tid == 0 && g_lo + i < g_hi) issue(ahead, i, i == 0);
+      if (g_lo + i + 1 < g_hi) advance(ahead);
+    }
+  }
+  // per-warp running state of the current segment (row g of the accumulators = head g of the group)
+  uint32_t qh[4][2], ql[4][2];                  // A fragments of q (rows 8..15 are zero)
+  float o[8][4];
+  float m_run = -INFINITY, l_run = 0.0f;        // maximum in base-2 units
+  int seg_first_split = 0, st = 0, seg_buf = 0;
+  unsigned phase = 0;
+  const float scale2 = A.scale * 1.4426950408889634f;
+  const int r8 = lane & 7, ti = lane >> 3;
+#pragma unroll 1
+  for (int gi = g_lo; gi < g_hi; ++gi) {
+    const int split = cur.split, nsplit = cur.nsplit;
+    const int cnt = min(SPLIT, cur.pos + 1 - split * SPLIT);
+    const bool have_next = gi + 1 < g_hi;
+    const bool seg_start = (gi == g_lo) || split == 0;
+    const bool seg_end = !have_next || split == nsplit - 1;
+    {
+      // every warp waits for the tiles on its own (also a warp without positions in this chunk: the
+      // parity test is only valid for a warp that has seen every earlier phase complete)
+      unsigned spins = 0;
+      while (!mbar_try_wait(&full[st], phase)) {
+        if (++spins > (1u << 20)) { if (lane == 0) atomicOr(A.err, 16); break; }     // reported; results are void
+        if (spins > 4096) __nanosleep(64);
+      }
+    }
+    if (seg_start) {
+      seg_first_split = split;
+      m_run = -INFINITY; l_run = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
+      const float* qrow = sq + ((size_t)st * grp + g) * HD;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        float2 a = make_float2(0.0f, 0.0f), b = make_float2(0.0f, 0.0f);
+        if (g < grp) {
+          a = *reinterpret_cast<const float2*>(qrow + kk * 16 + 2 * t4);
+          b = *reinterpret_cast<const float2*>(qrow + kk * 16 + 8 + 2 * t4);
+        }
+        split_bf16x2(a.x, a.y, qh[kk][0], ql[kk][0]);
+        split_bf16x2(b.x, b.y, qh[kk][1], ql[kk][1]);
+      }
+    }
+    if (warp * 16 < cnt) {
+      const uint32_t kst = smem_u32(stage0 + (size_t)st * 2 * kAtcTile), vst = kst + kAtcTile;
+      // scores of 16 positions: two n-tiles of 8, k = 64 dims in 4 steps; the products with the head and
+      // with the remainder of q accumulate separately (shorter dependent chains)
+      float sc[2][4], sr[2][4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.0f;
+        sr[j][0] = sr[j][1] = sr[j][2] = sr[j][3] = 0.0f;
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t a0h[4] = {qh[2 * half][0], 0u, qh[2 * half][1], 0u}, a0l[4] = {ql[2 * half][0], 0u, ql[2 * half][1], 0u};
+        const uint32_t a1h[4] = {qh[2 * half + 1][0], 0u, qh[2 * half + 1][1], 0u}, a1l[4] = {ql[2 * half + 1][0], 0u, ql[2 * half + 1][1], 0u};
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          uint32_t kb[4];
+          ldsm_x4(kb, kst + (uint32_t)(warp * 16 + j * 8 + r8) * 128u + (uint32_t)(((half * 4 + ti) ^ r8) << 4));
+          const uint32_t b0[2] = {kb[0], kb[1]}, b1[2] = {kb[2], kb[3]};
+          mma_bf16(sc[j], a0h, b0); mma_bf16(sr[j], a0l, b0);
+          mma_bf16(sc[j], a1h, b1); mma_bf16(sr[j], a1l, b1);
+        }
+      }
+      // softmax over the warp's 16 positions (row g lives in the 4 lanes of a quad), base 2
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          sc[j][e] = (sc[j][e] + sr[j][e]) * scale2;
+          if (cnt < SPLIT && warp * 16 + j * 8 + 2 * t4 + e >= cnt) sc[j][e] = -INFINITY;
+          mx = fmaxf(mx, sc[j][e]);
+        }
+      mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
+      if (__any_sync(FULL, mx > m_run)) {          // the running maximum moves: rescale what has been gathered
+        const float m_new = fmaxf(m_run, mx);
+        const float f_old = ex2_approx(m_run - m_new);
+        l_run *= f_old;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { o[j][0] *= f_old; o[j][1] *= f_old; }
+        m_run = m_new;
+      }
+      float pw[2][2];
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) { pw[j][e] = ex2_approx(sc[j][e] - m_run); l_run += pw[j][e]; }
+      uint32_t ph[4] = {0u, 0u, 0u, 0u}, pl[4] = {0u, 0u, 0u, 0u};
+      split_bf16x2(pw[0][0], pw[0][1], ph[0], pl[0]);
+      split_bf16x2(pw[1][0], pw[1][1], ph[2], pl[2]);
+      // output += P V: k = the 16 positions, n = 64 dims in 8 tiles (V tiles transposed on load)
+      const uint32_t vrow = vst + (uint32_t)(warp * 16 + (ti & 1) * 8 + r8) * 128u;
+#pragma unroll
+      for (int jn = 0; jn < 8; jn += 2) {
+        uint32_t vb[4];
+        ldsm_x4_trans(vb, vrow + (uint32_t)(((jn + (ti >> 1)) ^ r8) << 4));
+        const uint32_t b0[2] = {vb[0], vb[1]}, b1[2] = {vb[2], vb[3]};
+        mma_bf16(o[jn], ph, b0); mma_bf16(o[jn + 1], ph, b1);
+        mma_bf16(o[jn], pl, b0); mma_bf16(o[jn + 1], pl, b1);
+      }
+    }
+    // the last warp to finish with the stage refills it (the mma above have consumed every ldmatrix result)
+    __syncwarp();
+    if (lane == 0) {
+      if (atomicAdd(&s_done[st], 1) == NW - 1) {
+        s_done[st] = 0;
+        if (gi + n_stages < g_hi) issue(ahead, st, false);
+      }
+    }
+    if (gi + n_stages + 1 < g_hi) advance(ahead);
+    if (++st == n_stages) { st = 0; phase ^= 1u; }
+    if (seg_end) {
+      // this warp's state -> shared memory; the last warp to get here combines the eight states
+      float l_tot = l_run + __shfl_xor_sync(FULL, l_run, 1);
+      l_tot += __shfl_xor_sync(FULL, l_tot, 2);
+      float* so_b = so + (size_t)seg_buf * NW * grp * HD;
+      float* sm_b = sm + seg_buf * NW * grp;
+      float* sl_b = sl + seg_buf * NW * grp;
+      if (g < grp) {
+        float* dst = so_b + ((size_t)warp * grp + g) * HD + 2 * t4;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) *reinterpret_cast<float2*>(dst + 8 * j) = make_float2(o[j][0], o[j][1]);
+        if (t4 == 0) { sm_b[warp * grp + g] = m_run; sl_b[warp * grp + g] = l_tot; }
+      }
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) {
+        __threadfence_block();
+        last = atomicAdd(&s_seg[seg_buf], 1) == NW - 1;
+        if (last) { s_seg[seg_buf] = 0; __threadfence_block(); }
+      }
+      last = __shfl_sync(FULL, last, 0);
+      if (last) {
+        const int s = cur.s, gk = cur.gk;
+        const bool whole = seg_first_split == 0 && split == nsplit - 1;
+        const int g0 = gi - split;                 // first chunk of this cache
+        int n_c = 0, c_a = 0;
+        if (!whole) {
+          c_a = (int)((((long long)g0 + 1) * NC - 1) / T);
+          n_c = (int)((((long long)g0 + nsplit) * NC - 1) / T) - c_a + 1;
+        }
+        // first split of CTA (c_a + j)'s segment of this cache, or -1 when that CTA has no chunk at all
+        auto seg_of = [&](int j) {
+          const int lo_c = (int)((long long)(c_a + j) * T / NC), hi_c = (int)((long long)(c_a + j + 1) * T / NC);
+          return (lo_c < hi_c) ? max(lo_c, g0) - g0 : -1;
+        };
+#pragma unroll 1
+        for (int t = 0; t < grp; ++t) {
+          float M = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < NW; ++w) M = fmaxf(M, sm_b[w * grp + t]);
+          float2 v = make_float2(0.0f, 0.0f);
+          float l = 0.0f;
+#pragma unroll
+          for (int w = 0; w < NW; ++w) {
+            const float f = ex2_approx(sm_b[w * grp + t] - M);      // 0 for a warp that saw no position
+            const float2 x = *reinterpret_cast<const float2*>(so_b + ((size_t)w * grp + t) * HD + 2 * lane);
+            v.x = fmaf(f, x.x, v.x); v.y = fmaf(f, x.y, v.y);
+            l = fmaf(f, sl_b[w * grp + t], l);
+          }
+          const int head = gk * grp + t;
+          if (whole) {
+            *reinterpret_cast<float2*>(A.out + ((size_t)s * H + head) * HD + 2 * lane) = make_float2(v.x / l, v.y / l);
+          } else {
+            const size_t pi = ((size_t)s * H + head) * A.max_splits + seg_first_split;
+            *reinterpret_cast<float2*>(A.part_o + pi * HD + 2 * lane) = v;
+            if (lane == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
+          }
+        }
+        if (!whole) {
+          __syncwarp();
+          int fin = 0;
+          if (lane == 0) {
+            __threadfence();                       // the warp's partial results before the ticket
+            int n_seg = 0;
+            for (int j = 0; j < n_c; ++j) n_seg += seg_of(j) >= 0;
+            fin = atomicAdd(A.tickets + s * Hkv + gk, 1) == n_seg - 1;
+            if (fin) __threadfence();
+          }
+          fin = __shfl_sync(FULL, fin, 0);
+          if (fin) {                               // every segment of the cache is in L2: combine them in CTA order
+#pragma unroll 1
+            for (int t = 0; t < grp; ++t) {
+              const int head = gk * grp + t;
+              const size_t base = ((size_t)s * H + head) * A.max_splits;
+              float M = -INFINITY;
+              for (int j = 0; j < n_c; ++j) { const int f0 = seg_of(j); if (f0 >= 0) M = fmaxf(M, __ldcg(A.part_ml + (base + f0) * 2)); }
+              float2 num = make_float2(0.0f, 0.0f);
+              float den = 0.0f;
+              for (int j = 0; j < n_c; ++j) {
+                const int f0 = seg_of(j);
+                if (f0 < 0) continue;
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + f0) * 2));
+                const float f = ex2_approx(ml.x - M);
+                const float2 x = __ldcg(reinterpret_cast<const float2*>(A.part_o + (base + f0) * HD + 2 * lane));
+                num.x = fmaf(f, x.x, num.x); num.y = fmaf(f, x.y, num.y);
+                den = fmaf(f, ml.y, den);
+              }
+              *reinterpret_cast<float2*>(A.out + ((size_t)s * H + head) * HD + 2 * lane) = make_float2(num.x / den, num.y / den);
+            }
+            if (lane == 0) A.tickets[s * Hkv + gk] = 0;
+          }
+        }
+      }
+      if (++seg_buf == n_stages) seg_buf = 0;
+    }
+    if (have_next) advance(cur);
+  }
+}
+
+}  // namespace tabed

@@ -18,6 +18,7 @@
 #include "decide_kernels.cuh"
 #include "round_kernel.cuh"
 #include "gemm_tc.cuh"
+#include "attn_tc.cuh"
 
 using namespace tabed;
 
@@ -79,6 +80,9 @@ struct tabed_handle {
   LayerW* layer_tab = nullptr;
   float *xa = nullptr, *x1 = nullptr;
   int* tickets = nullptr; unsigned* bar = nullptr; float* ssq = nullptr;
+  // tensor-core streaming attention of the per-operation paths (bf16 caches, head size 64)
+  int* attn_tickets = nullptr; int n_sm = 0;
+  bool atc_ok = false; CUtensorMap tm_k, tm_v;
   unsigned char* packed = nullptr;
   uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
   unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false;
@@ -200,6 +204,30 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
     auto part = k_attn_split_bf16<HD>;
     static bool attr_set = false;
     if (!attr_set) { cudaFuncSetAttribute(part, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr_set = true; }
+    if constexpr (HD == kAtcHd) {
+      if (h->atc_ok && n_slots <= kAtcMaxSlots) {
+        // fixed grid of streaming CTAs, contiguous chunk ranges, TMA-fed tensor-core arithmetic, in-kernel merge
+        // two CTAs per SM with three stages each when the shared memory allows, else one CTA with a deeper ring
+        // per stage: the K and V tiles, q of the cache, and one set of the eight warps' states
+        const size_t per_stage = 2 * (size_t)kAtcTile + ((size_t)grp * HD + (size_t)kAtcWarps * grp * (HD + 2)) * sizeof(float);
+        int n_ctas = std::min(kAtcMaxCtas, 2 * h->n_sm), n_stages = 3;
+        if (1024 + n_stages * per_stage > 108u * 1024u) {
+          n_ctas = std::min(kAtcMaxCtas, h->n_sm);
+          n_stages = (int)std::min<size_t>(kAtcMaxStages, (kAtcMaxDynSmem - 1024u) / per_stage);
+        }
+        if (n_stages >= 3) {
+          const size_t smem2 = 1024 + n_stages * per_stage;
+          static bool attr2_set = false;
+          if (!attr2_set) { cudaFuncSetAttribute(k_attn_tc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtcMaxDynSmem); attr2_set = true; }
+          AttnTcArgs a;
+          a.qkv = h->qkv; a.slots = h->slots; a.n_slots = n_slots; a.H = h->H; a.Hkv = h->Hkv; a.layer = layer; a.L = h->L;
+          a.cap = h->cap; a.qkv_w = h->qkv_w; a.part_o = h->part_o; a.part_ml = h->part_ml; a.max_splits = h->max_splits;
+          a.tickets = h->attn_tickets; a.out = h->attn_out; a.scale = 1.0f / sqrtf((float)h->hd); a.err = h->err; a.n_stages = n_stages;
+          TABED_LAUNCH(h, k_attn_tc_bf16, n_ctas, kAtcThreads, smem2, h->tm_k, h->tm_v, a);
+          return;
+        }
+      }
+    }
     if (smem <= 96 * 1024) {
       TABED_LAUNCH(h, part, dim3(splits, h->Hkv, n_slots), kAttnBwThreads, smem, h->qkv, h->slots, h->H, h->Hkv,
                    reinterpret_cast<const __nv_bfloat16*>(h->kc), reinterpret_cast<const __nv_bfloat16*>(h->vc), layer, h->L, h->cap,
@@ -694,6 +722,32 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
     A(&h->x, 2 * R * h->d); A(&h->qkv, 2 * R * h->qkv_w); A(&h->attn_out, 2 * R * h->H * h->hd); A(&h->mid, 2 * R * h->F);
     A(&h->part_o, 2 * R * h->H * (size_t)h->max_splits * h->hd); A(&h->part_ml, 2 * R * h->H * (size_t)h->max_splits * 2);
     A(&h->logits_own, G * R * V);
+    A(&h->attn_tickets, 2 * R * h->Hkv);
+    { cudaDeviceProp pr; if (cudaGetDeviceProperties(&pr, c.device) == cudaSuccess) h->n_sm = pr.multiProcessorCount; }
+    if (c.dtype == TABED_DTYPE_BF16 && h->hd == kAtcHd && h->H / h->Hkv <= kMaxGroup && rc == TABED_OK) {
+      // TMA descriptors of the caches seen as [all rows of all (row, layer, head)][64] bf16, tiles of 128 rows, 128-byte swizzle
+      typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      const unsigned long long n_rows = (unsigned long long)R * h->L * h->Hkv * (unsigned long long)h->cap;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess && fn &&
+          qres == cudaDriverEntryPointSuccess && n_rows < (1ull << 31)) {
+        const cuuint64_t dims[2] = {(cuuint64_t)kAtcHd, (cuuint64_t)n_rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)kAtcHd * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kAtcHd, (cuuint32_t)kAtcSplit};
+        const cuuint32_t estr[2] = {1, 1};
+        EncodeFn enc = reinterpret_cast<EncodeFn>(fn);
+        const CUresult r1 = enc(&h->tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->kc, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        const CUresult r2 = enc(&h->tm_v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->vc, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        h->atc_ok = (r1 == CUDA_SUCCESS && r2 == CUDA_SUCCESS);
+      } else {
+        cudaGetLastError();
+      }
+    }
     A(&h->rope_cos, (size_t)h->cap * (h->hd / 2)); A(&h->rope_sin, (size_t)h->cap * (h->hd / 2));
     if (rc == TABED_OK) {
       const int half = h->hd / 2;
