@@ -75,3 +75,44 @@ def test_tensor_path_agrees_with_per_operation_path():
     assert np.max(np.abs(la - lb)) <= H.LOGIT_TOL["bf16"]
     H.check_error_flag(a.gpu)
     a.gpu.destroy(); b.gpu.destroy()
+
+
+# ------------------------------------------------------------------------------------------------
+# TMA / tensor-core attention of the per-operation paths (bf16 caches, head size 64)
+# ------------------------------------------------------------------------------------------------
+def wl_attn(*, heads, kv_heads, d, prefixes, cap, B=1, cid=90, gamma=3, sigma=0.3, layers=2):
+    m = len(prefixes)
+    # vocabulary 8000: with a few thousand words the largest probabilities are so large that one bf16 ulp in
+    # a cache entry (the checker rounds fp64 values, the kernels fp32 ones) moves them by more than 1e-5
+    cfg = W.DrafterCfg(layers, d, heads, kv_heads, 512, 8000, "bf16")
+    alpha = tuple([1.0 / m] * m)
+    return W.Workload(name=f"attn{cid}", config_id=cid, drafter=cfg, n_inputs=m, n_requests=B, gamma=gamma, window_h=4,
+                      rounds=4, policy=W.POLICY_SOFTMAX_INV_ERR if m != 2 else W.POLICY_GRID_MT, prefixes=prefixes,
+                      kv_capacity=cap, alpha=alpha, sigma_schedule=((0, sigma),))
+
+
+@pytest.mark.parametrize("heads,kv_heads,d", [(4, 2, 256), (8, 2, 512), (14, 2, 896)])
+def test_attention_caches_spread_over_many_ctas(heads, kv_heads, d):
+    """Per-operation path, few rows with long caches: fewer chunks of 128 positions than CTAs, so every
+    cache longer than one chunk is cut into one-chunk segments on different CTAs (with idle CTAs in
+    between) and put together by the last warp to finish (ticket).  Ragged last chunks (700 % 128, 130 %
+    128), a cache shorter than one chunk, groups of 2, 4 and 7 query heads per KV head."""
+    wl = wl_attn(heads=heads, kv_heads=kv_heads, d=d, cap=1024, cid=90 + heads,
+                 prefixes=((("tokens", 700),), (("tokens", 130),), (("embeds", 37), ("tokens", 9))))
+    pair = H.build_pair(wl)
+    pair.gpu.select_path(TB.PATH_PER_OP)
+    for rnd in range(3):
+        H.lockstep_round(pair, rnd, override=True)
+    pair.gpu.destroy()
+
+
+def test_attention_many_rows_several_chunks_each():
+    """Tensor-core path, 36 rows with 2 to 4 chunks per cache: segments that start and end inside a CTA's
+    range next to caches that straddle two CTAs; two pending tokens for some requests (inactive slots)."""
+    wl = wl_attn(heads=4, kv_heads=2, d=256, cap=512, B=12, cid=97, sigma=0.05, gamma=2,
+                 prefixes=((("tokens", 390),), (("tokens", 260),), (("embeds", 120), ("tokens", 30))))
+    pair = H.build_pair(wl)
+    assert pair.gpu.current_path() == TB.PATH_TENSOR_CORE
+    for rnd in range(3):
+        H.lockstep_round(pair, rnd, override=True)
+    pair.gpu.destroy()
