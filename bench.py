@@ -320,8 +320,12 @@ def run_ours(args, wl):
     torch.cuda.synchronize(device)
     launches0 = g.launch_count()
     persistent = g.current_path() == TB.PATH_PERSISTENT
-    top_cls, top_name, top_kernel = ((TB.PROF_DRAFT_ROUND, "draft_round", "k_draft_round (persistent: gamma decoder steps + ensemble)")
-                                     if persistent else (TB.PROF_LM_HEAD, "lm_head", "k_gemv (LM head)"))
+    if persistent:
+        top_cls, top_name, top_kernel = TB.PROF_DRAFT_ROUND, "draft_round", "k_draft_round (persistent: gamma decoder steps + ensemble)"
+    elif g.current_path() == TB.PATH_TENSOR_CORE:
+        top_cls, top_name, top_kernel = TB.PROF_ATTENTION, "attention", "k_attn_tc_bf16 (decode attention of all rows over their bf16 K,V caches)"
+    else:
+        top_cls, top_name, top_kernel = TB.PROF_LM_HEAD, "lm_head", "k_gemv (LM head)"
     g.profile_begin(top_cls)
     sampler.mark_begin()
     wall0 = time.perf_counter()

@@ -576,11 +576,11 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
       }
       const size_t elems = (size_t)n_slots * h->qkv_w;
       TABED_LAUNCH(h, k_sum_slabs, (unsigned)((elems / 4 + 255) / 256), 256, 0, h->tc_pq, h->tck[KIND_QKV].ks, S2 * h->qkv_w, elems, h->qkv);
-    }
-    {
-      ProfScope ps(h, TABED_PROF_ATTENTION);
       TABED_LAUNCH(h, k_rope_append<bf>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos, h->rope_sin,
                    reinterpret_cast<bf*>(h->kc), reinterpret_cast<bf*>(h->vc), l, h->L, h->cap);
+    }
+    {
+      ProfScope ps(h, TABED_PROF_ATTENTION);       // the attention kernel(s) alone on this path
       launch_attention_t<bf>(h, l, n_slots, max_pos);
     }
     {
