@@ -410,7 +410,7 @@ def run_ours(args, wl):
         g.state_import(snap)
         for r in range(Wm):
             one_round(r)
-        g.debug_trace(True)
+        g.debug_trace(True, args.trace_cta)
         flush.zero_()
         g.draft_round(u[Wm][0], toks)
         torch.cuda.synchronize(device)
@@ -423,8 +423,8 @@ def run_ours(args, wl):
         names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "gateup", "down")] + ["lm_head", "expsum", "mix"]
         mhz = float(clocks.get("sm_mhz") or 1965.0)
         with open(args.trace, "w") as f:
-            f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA 0): us from the previous grid barrier to this one,\n"
-                    f"# then CTA 0's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
+            f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA {args.trace_cta}): us from the previous grid barrier to this one,\n"
+                    f"# then that CTA's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
                     f"# (attention phases: load+stage q/k/v, scores+softmax, PV+write, split merge, -, barrier)\n")
             prev = None
             for st in range(G):
@@ -492,6 +492,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--trace", default=None, help="write the persistent kernel's phase timeline of one round to this file")
+    ap.add_argument("--trace-cta", type=int, default=0, help="the CTA whose phase timeline --trace records")
     ap.add_argument("--requests", type=int, default=0, help="override the workload's number of concurrent requests (profiling aid)")
     ap.add_argument("--path", default="auto", choices=["auto", "per-op"], help="drafting path (per-op forces one kernel per operation)")
     args = ap.parse_args()

@@ -207,9 +207,10 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
 int tabed_select_path(tabed_handle* h, int32_t path);
 int tabed_current_path(const tabed_handle* h);
 
-/* Switch the phase timeline of the persistent kernel on or off: when on, CTA 0 stores one record of
+/* Switch the phase timeline of the persistent kernel off (on = 0) or on (on = 1 + the index of the CTA
+ * that records; CTA 0 if the grid is smaller): when on, that CTA stores one record of
  * 8 words per grid barrier into TABED_VIEW_TRACE (first index = drafting step): [0] the GPU's
- * nanosecond timer after the barrier; [1..6] SM clock cycles that CTA 0 spent since the previous
+ * nanosecond timer after the barrier; [1..6] SM clock cycles that that CTA spent since the previous
  * barrier resolving and staging activations, waiting for weight tiles, in the tensor-core products,
  * issuing weight copies, in epilogues (or, for the phases without weights, in all of the phase), and
  * in the barrier itself; [7] unused.  Barrier order within a step: per layer QKV, attention, O,

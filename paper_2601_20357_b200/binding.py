@@ -311,8 +311,8 @@ class Tabed:
             raise TabedError(rc, "tabed_current_path")
         return rc
 
-    def debug_trace(self, on: bool) -> None:
-        _check(lib().tabed_debug_trace(self._h, 1 if on else 0), "tabed_debug_trace")
+    def debug_trace(self, on: bool, cta: int = 0) -> None:
+        _check(lib().tabed_debug_trace(self._h, 1 + int(cta) if on else 0), "tabed_debug_trace")
 
     def launch_count(self) -> int:
         return int(lib().tabed_launch_count(self._h))

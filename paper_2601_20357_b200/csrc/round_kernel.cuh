@@ -102,7 +102,7 @@ struct RoundArgs {
   int bar_sel;
   int* err;
   unsigned long long* trace;            // optional [G][trace_stride][kTraceRec] phase timeline
-  int trace_stride;
+  int trace_stride, trace_cta;          // the CTA that records
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -253,6 +253,26 @@ __device__ __forceinline__ bool wait_full(PShared& S, int slot, unsigned parity,
 // Grid-wide barrier on a counter that only grows during a launch.  (One flag per CTA polled by all
 // CTAs in parallel was measured 3-4x slower: 148 x 148 concurrent polls saturate the L2 slice.)
 // Returns false if the wait ran out.
+// The barrier in two halves, for work that may overlap the wait (loads that do not depend on the
+// other CTAs are requested between the halves: a fence would wait for them).
+__device__ __forceinline__ void grid_barrier_arrive(unsigned* bar) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(bar, 1u);
+  }
+}
+__device__ __noinline__ bool grid_barrier_wait(PShared& S, unsigned* bar, unsigned target, int* err) {
+  if (threadIdx.x == 0) {
+    unsigned spins = 0;
+    while ((int)(ld_acquire_u32(bar) - target) < 0) {
+      if (++spins > kSpinLimit) { atomicOr(err, PERR_BARRIER); S.dead = 1; break; }
+      if (spins > 4096) __nanosleep(64);
+    }
+  }
+  __syncthreads();
+  return S.dead == 0;
+}
 __device__ __noinline__ bool grid_barrier(PShared& S, unsigned* bar, unsigned target, int* err) {
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -391,7 +411,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   // [0] nanosecond timer after the barrier, [1..6] clock cycles spent since the previous barrier in
   // staging activations, waiting for weight tiles, mma+partials, issuing copies + epilogue (for
   // attention: its four sections in slots 1-4), everything else, and in the barrier itself
-  const bool tr_on = TRACE && A.trace != nullptr && cta == 0 && tid == 0;
+  const bool tr_on = TRACE && A.trace != nullptr && cta == (A.trace_cta < NC ? A.trace_cta : 0) && tid == 0;
   long long t_sec[6] = {0, 0, 0, 0, 0, 0};
   long long t_mark = 0;
 #define TSEC(k)                                       \
@@ -401,6 +421,16 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       t_sec[k] += t_now - t_mark;                     \
       t_mark = t_now;                                 \
     }                                                 \
+  } while (0)
+#define GRID_SYNC_TAIL()                                                   \
+  do {                                                                     \
+    TSEC(5);                                                               \
+    if (TRACE && tr_on && trace_n < A.trace_stride) {                      \
+      unsigned long long* rec = A.trace + ((size_t)step * A.trace_stride + trace_n++) * kTraceRec; \
+      rec[0] = global_timer();                                             \
+      for (int k = 0; k < 6; ++k) { rec[1 + k] = (unsigned long long)t_sec[k]; t_sec[k] = 0; }     \
+    }                                                                      \
+    if (!alive) goto drain;                                                \
   } while (0)
 #define GRID_SYNC()                                                        \
   do {                                                                     \
@@ -536,12 +566,74 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         }
         __syncthreads();
       } else if (kind == KIND_O && ka < kb) {
-        // ---- stage the attention output, whole rows ------------------------------------------------
+        // ---- stage the attention output, whole rows: put every pair's partial results together -----
+        // n_seg of a pair (see the attention phase): the CTAs its chunks fall on, or its chunks.
+        {
+          const int split_len = A.split_len;
+          int Ta = 0;
+#pragma unroll 1
+          for (int s = 0; s < n_in; ++s)
+            if (S.slot[s].active) Ta += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
+#pragma unroll 1
+          for (int c2 = tid; c2 < n_in * A.Hkv; c2 += kPT) {
+            const int s = c2 / A.Hkv, gk = c2 - s * A.Hkv;
+            int n_seg = 0;
+            if (S.slot[s].active) {
+              const int nsplit = (S.slot[s].pos + split_len) / split_len;
+              n_seg = nsplit;
+              if (Ta >= NC) {
+                int g0 = gk * nsplit;
+                for (int s2 = 0; s2 < s; ++s2)
+                  if (S.slot[s2].active) g0 += A.Hkv * ((S.slot[s2].pos + split_len) / split_len);
+                n_seg = ((g0 + nsplit) * NC - 1) / Ta - ((g0 + 1) * NC - 1) / Ta + 1;
+              }
+            }
+            S.segfirst[c2] = n_seg;
+          }
+          __syncthreads();
+        }
         const int nvec = g.kchunk >> 2;
 #pragma unroll 1
         for (int idx = tid; idx < n_in * nvec; idx += kPT) {
           const int s = idx / nvec, j = (idx - s * nvec) << 2;
-          const float4 v = __ldcg(reinterpret_cast<const float4*>(A.attn_out + (size_t)s * HD + j));
+          const int head = j / A.hd, dd = j - head * A.hd;
+          const int n_seg = S.segfirst[s * A.Hkv + head / grp];
+          const size_t base = ((size_t)s * A.H + head) * A.max_splits;
+          float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+          if (n_seg == 1) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + base * 2));
+            const float4 x = __ldcg(reinterpret_cast<const float4*>(A.part_o + base * A.hd + dd));
+            const float r = 1.0f / ml.y;
+            v = make_float4(x.x * r, x.y * r, x.z * r, x.w * r);
+          } else if (n_seg > 1) {
+            // running maximum over the partial results in their fixed order (4 at a time in flight)
+            float M = -INFINITY, den = 0.0f;
+#pragma unroll 1
+            for (int j0 = 0; j0 < n_seg; j0 += 4) {
+              float2 ml[4];
+              float4 x[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const bool ok = j0 + q < n_seg;
+                ml[q] = ok ? __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + j0 + q) * 2)) : make_float2(-INFINITY, 0.0f);
+                x[q] = ok ? __ldcg(reinterpret_cast<const float4*>(A.part_o + (base + j0 + q) * A.hd + dd)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+              }
+              float Mn = M;
+#pragma unroll
+              for (int q = 0; q < 4; ++q) Mn = fmaxf(Mn, ml[q].x);
+              const float fo = (M > -INFINITY) ? expf(M - Mn) : 0.0f;
+              v.x *= fo; v.y *= fo; v.z *= fo; v.w *= fo; den *= fo;
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float f = (ml[q].x > -INFINITY) ? expf(ml[q].x - Mn) : 0.0f;
+                v.x = fmaf(f, x[q].x, v.x); v.y = fmaf(f, x[q].y, v.y); v.z = fmaf(f, x[q].z, v.z); v.w = fmaf(f, x[q].w, v.w);
+                den = fmaf(f, ml[q].y, den);
+              }
+              M = Mn;
+            }
+            const float r = 1.0f / den;
+            v.x *= r; v.y *= r; v.z *= r; v.w *= r;
+          }
           uint2 pk;
           pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
           *reinterpret_cast<uint2*>(act + s * apitch + j) = pk;
@@ -669,8 +761,6 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         __syncthreads();
         if (tid < R && S.lmmax[tid] != 0u) atomicMax(A.rowmax + step * R + tid, S.lmmax[tid]);
       }
-      GRID_SYNC();
-
       // ---- attention over the rows' caches (after the QKV phase) -----------------------------------
       // The caches of all (slot, KV head) pairs are cut into chunks of split_len positions; the chunks, in
       // (slot, head, position) order, are dealt to the CTAs in contiguous ranges, so a CTA walks along one
@@ -679,50 +769,64 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       // chunks of a segment (= the part of one pair's cache this CTA owns): no block-wide exchange per
       // chunk, the next chunk's K and V are requested as soon as the registers are free.  At the end of
       // a segment the 16 warps are merged (plus the positions produced in this very phase, which come
-      // from the QKV output, not from the cache); pairs that span several CTAs are combined by the CTA
-      // that finishes last (ticket), in segment order.
+      // from the QKV output, not from the cache) into ONE partial result (max, sum, un-normalised
+      // output) per head; the partial results of a pair are put together by the O-projection phase
+      // while it stages its input (every CTA needs all of it anyway), so this phase ends without a
+      // second exchange between CTAs.
+      // The cached positions do not depend on the QKV phase (its positions come from the QKV output),
+      // so the first chunk's K and V are requested BEFORE the grid barrier and arrive while it is taken.
+      const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
+      const int PPW = 32 / LPR, PPB = kPW * PPW;     // positions per warp / per CTA pass
+      const int sub = lane % LPR, pgrp = lane / LPR;
+      // chunks of split_len positions (4 register passes of the CTA); short caches give fewer chunks than
+      // CTAs - shorter chunks were measured slower there (the phase is latency-bound)
+      const int split_len = A.split_len;
+      struct Walk { int s, gk, split, nsplit, g0; };          // g0 = global index of the pair's first chunk
+      auto seek = [&](int g, Walk& w) {
+        int s = 0, rem = g, acc = 0, nsplit = 0;
+#pragma unroll 1
+        for (; s < ns; ++s) {
+          nsplit = S.slot[s].active ? (S.slot[s].pos + split_len) / split_len : 0;
+          if (rem < A.Hkv * nsplit) break;
+          rem -= A.Hkv * nsplit; acc += A.Hkv * nsplit;
+        }
+        w.s = s; w.nsplit = nsplit; w.gk = nsplit ? rem / nsplit : 0; w.split = nsplit ? rem - w.gk * nsplit : 0;
+        w.g0 = acc + w.gk * nsplit;
+      };
+      auto issue_loads = [&](const Walk& w, uint4 (&kr)[4], uint4 (&vr)[4], bool want_k, bool want_v) {
+        const int pos = S.slot[w.s].pos;
+        const int p_lo = w.split * split_len, cnt = min(split_len, pos + 1 - p_lo);
+        const int fresh_lo = pos - (w.s >= R ? 1 : 0);
+        const size_t off = ((((size_t)S.slot[w.s].row * A.L + layer) * A.Hkv + w.gk) * A.cap) * A.hd;
+#pragma unroll
+        for (int ps = 0; ps < 4; ++ps) {
+          const int p = ps * PPB + warp * PPW + pgrp;
+          const bool ok = p < cnt && p_lo + p < fresh_lo;
+          if (want_k) kr[ps] = ok ? __ldcg(reinterpret_cast<const uint4*>(A.kc + off + (size_t)(p_lo + p) * A.hd + sub * 8)) : make_uint4(0u, 0u, 0u, 0u);
+          if (want_v) vr[ps] = ok ? __ldcg(reinterpret_cast<const uint4*>(A.vc + off + (size_t)(p_lo + p) * A.hd + sub * 8)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      };
+      uint4 kreg[4], vreg[4];
+      Walk cur{0, 0, 0, 0, 0}, nxt{0, 0, 0, 0, 0};
+      int T = 0, g_lo = 0, g_hi = 0;
       if (kind == KIND_QKV) {
-        const int LPR = A.hd >> 3;                     // lanes per cache row (8 bf16 per 16-byte load)
-        const int PPW = 32 / LPR, PPB = kPW * PPW;     // positions per warp / per CTA pass
-        const int sub = lane % LPR, pgrp = lane / LPR;
-        // chunks of split_len positions (4 register passes of the CTA); short caches give fewer chunks than
-        // CTAs - shorter chunks were measured slower there (more segments to merge, the phase is latency-bound)
-        const int split_len = A.split_len;
-        int T = 0;
 #pragma unroll 1
         for (int s = 0; s < ns; ++s)
           if (S.slot[s].active) T += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
         // (T <= 8 slots x 64 heads x 256 chunks, so c * T stays far below 2^31)
-        const int g_lo = cta * T / NC, g_hi = (cta + 1) * T / NC;
-        // walker over (slot, head, split) in global chunk order
-        struct Walk { int s, gk, split, nsplit, g0; };          // g0 = global index of the pair's first chunk
-        auto seek = [&](int g, Walk& w) {
-          int s = 0, rem = g, acc = 0, nsplit = 0;
-#pragma unroll 1
-          for (; s < ns; ++s) {
-            nsplit = S.slot[s].active ? (S.slot[s].pos + split_len) / split_len : 0;
-            if (rem < A.Hkv * nsplit) break;
-            rem -= A.Hkv * nsplit; acc += A.Hkv * nsplit;
-          }
-          w.s = s; w.nsplit = nsplit; w.gk = nsplit ? rem / nsplit : 0; w.split = nsplit ? rem - w.gk * nsplit : 0;
-          w.g0 = acc + w.gk * nsplit;
-        };
-        auto issue_loads = [&](const Walk& w, uint4 (&kr)[4], uint4 (&vr)[4], bool want_k, bool want_v) {
-          const int pos = S.slot[w.s].pos;
-          const int p_lo = w.split * split_len, cnt = min(split_len, pos + 1 - p_lo);
-          const int fresh_lo = pos - (w.s >= R ? 1 : 0);
-          const size_t off = ((((size_t)S.slot[w.s].row * A.L + layer) * A.Hkv + w.gk) * A.cap) * A.hd;
-#pragma unroll
-          for (int ps = 0; ps < 4; ++ps) {
-            const int p = ps * PPB + warp * PPW + pgrp;
-            const bool ok = p < cnt && p_lo + p < fresh_lo;
-            if (want_k) kr[ps] = ok ? __ldcg(reinterpret_cast<const uint4*>(A.kc + off + (size_t)(p_lo + p) * A.hd + sub * 8)) : make_uint4(0u, 0u, 0u, 0u);
-            if (want_v) vr[ps] = ok ? __ldcg(reinterpret_cast<const uint4*>(A.vc + off + (size_t)(p_lo + p) * A.hd + sub * 8)) : make_uint4(0u, 0u, 0u, 0u);
-          }
-        };
-        uint4 kreg[4], vreg[4];
-        Walk cur{0, 0, 0, 0, 0}, nxt{0, 0, 0, 0, 0};
-        if (g_lo < g_hi) { seek(g_lo, cur); issue_loads(cur, kreg, vreg, true, true); }
+        g_lo = cta * T / NC; g_hi = (cta + 1) * T / NC;
+        if (g_lo < g_hi) seek(g_lo, cur);
+        TSEC(4);
+        bar_target += (unsigned)NC;
+        grid_barrier_arrive(bar);
+        if (g_lo < g_hi) issue_loads(cur, kreg, vreg, true, true);
+        alive = grid_barrier_wait(S, bar, bar_target, A.err);
+        GRID_SYNC_TAIL();
+      } else {
+        GRID_SYNC();
+      }
+
+      if (kind == KIND_QKV) {
         int seg_first_split = 0;
 #pragma unroll 1
         for (int g = g_lo; g < g_hi; ++g) {
@@ -844,8 +948,10 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               if (lane == 0) S.sc[t][j] = (pj >= seg_lo && pj < seg_hi) ? dd * A.attn_scale : -INFINITY;
             }
             __syncthreads();
-            // ---- merge the warps (in warp order) and the fresh positions ----
-            const bool whole = seg_first_split == 0 && split == nsplit - 1;
+            // ---- merge the warps (in warp order) and the fresh positions into the segment's partial result ----
+            // Its place among the pair's partial results: with at least as many chunks as CTAs every CTA owns
+            // chunks, so the segments of a pair sit on consecutive CTAs; with fewer, a segment is one chunk.
+            const int ord = (T >= NC) ? cta - ((cur.g0 + 1) * NC - 1) / T : split;
 #pragma unroll 1
             for (int idx = tid; idx < grp * A.hd; idx += kPT) {
               const int t = idx / A.hd, dd = idx - t * A.hd;
@@ -866,79 +972,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
                 if (sf > -INFINITY) { const float f = expf(sf - M); v = fmaf(f, S.vf[j][dd], v); l += f; }
               }
               const int head = gk * grp + t;
-              if (whole) {
-                A.attn_out[(size_t)s * HD + head * A.hd + dd] = v / l;
-              } else {
-                const size_t pi = ((size_t)s * A.H + head) * A.max_splits + seg_first_split;
-                A.part_o[pi * A.hd + dd] = v;
-                if (dd == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
-              }
+              const size_t pi = ((size_t)s * A.H + head) * A.max_splits + ord;
+              A.part_o[pi * A.hd + dd] = v;
+              if (dd == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
             }
             TSEC(2);
-            if (!whole) {
-              // the pair's chunks [g0, g0 + nsplit) are spread over the CTAs c_a .. c_b, one segment each
-              // (CTAs without chunks excepted); the CTA whose ticket completes the pair merges the segments
-              // in CTA order.  S.segfirst[j] = first split of CTA c_a + j's segment, or -1.
-              const int c_a = ((cur.g0 + 1) * NC - 1) / T, c_b = ((cur.g0 + nsplit) * NC - 1) / T;
-              const int n_c = c_b - c_a + 1;
-#pragma unroll 1
-              for (int j = tid; j < n_c; j += kPT) {
-                const int lo_c = (c_a + j) * T / NC, hi_c = (c_a + j + 1) * T / NC;
-                S.segfirst[j] = (lo_c < hi_c) ? max(lo_c, cur.g0) - cur.g0 : -1;
-              }
-              __threadfence();
-              __syncthreads();
-              if (tid == 0) {
-                int n_seg = 0;
-#pragma unroll 1
-                for (int j = 0; j < n_c; ++j) n_seg += S.segfirst[j] >= 0;
-                S.flag = (atomicAdd(A.tickets + s * A.Hkv + gk, 1) == n_seg - 1);
-              }
-              __syncthreads();
-              if (S.flag) {
-                __threadfence();
-#pragma unroll 1
-                for (int t = warp; t < grp; t += kPW) {      // rescaling factors of the segments, one warp per head
-                  const size_t base = ((size_t)s * A.H + gk * grp + t) * A.max_splits;
-                  float M = -INFINITY;
-#pragma unroll 1
-                  for (int j = lane; j < n_c; j += 32) {
-                    const int first = S.segfirst[j];
-                    if (first >= 0) M = fmaxf(M, __ldcg(A.part_ml + (base + first) * 2));
-                  }
-                  M = warp_max_f32(M);
-                  float den = 0.0f;
-#pragma unroll 1
-                  for (int j = lane; j < n_c; j += 32) {
-                    const int first = S.segfirst[j];
-                    float f = 0.0f;
-                    if (first >= 0) {
-                      const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + first) * 2));
-                      f = expf(ml.x - M);
-                      den = fmaf(f, ml.y, den);
-                    }
-                    S.sc[t][j] = f;
-                  }
-                  den = warp_sum_f32(den);
-                  if (lane == 0) S.l_[t] = den;
-                }
-                __syncthreads();
-#pragma unroll 1
-                for (int idx = tid; idx < grp * A.hd; idx += kPT) {
-                  const int t = idx / A.hd, dd = idx - t * A.hd;
-                  const int head = gk * grp + t;
-                  const size_t base = ((size_t)s * A.H + head) * A.max_splits;
-                  float num = 0.0f;
-#pragma unroll 2
-                  for (int j = 0; j < n_c; ++j) {
-                    const int first = S.segfirst[j];
-                    if (first >= 0) num = fmaf(S.sc[t][j], __ldcg(A.part_o + (base + first) * A.hd + dd), num);
-                  }
-                  A.attn_out[(size_t)s * HD + head * A.hd + dd] = num / S.l_[t];
-                }
-                if (tid == 0) A.tickets[s * A.Hkv + gk] = 0;
-              }
-            }
             __syncthreads();
             TSEC(3);
           }

@@ -85,7 +85,7 @@ struct tabed_handle {
   bool atc_ok = false; CUtensorMap tm_k, tm_v;
   unsigned char* packed = nullptr;
   uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
-  unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false;
+  unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false; int trace_cta = 0;
   // tensor-core projections for many rows (bf16 drafter, more than 8 slots per step)
   bool tc_ok = false;
   struct TcKind { int rows, K, m_tiles, k_chunks, ks, cps; size_t bytes; };
@@ -464,7 +464,7 @@ int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_
   (void)max_pos;
   A.split_len = (h->hd <= 64) ? 256 : 128;          // positions per attention item: 4 register passes of the CTA
   A.bar_sel = (int)(h->launches_persist & 1u);
-  A.trace = h->trace_on ? h->trace : nullptr;
+  A.trace = h->trace_on ? h->trace : nullptr; A.trace_cta = h->trace_cta;
   void* args[] = {&A};
   const void* kern = h->trace_on ? (const void*)k_draft_round<true> : (const void*)k_draft_round<false>;
   if (cudaLaunchCooperativeKernel(kern, dim3(h->n_cta), dim3(kPT), args, h->persist_smem, h->stream) != cudaSuccess)
@@ -1071,6 +1071,7 @@ int tabed_debug_trace(tabed_handle* h, int32_t on) {
   if (!h) return TABED_ERR_NULL_PTR;
   if (!h->persist_ok) return TABED_ERR_UNSUPPORTED;
   h->trace_on = on != 0;
+  h->trace_cta = on > 0 ? on - 1 : 0;
   return TABED_OK;
 }
 
