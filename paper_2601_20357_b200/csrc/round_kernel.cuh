@@ -171,7 +171,7 @@ struct PShared {
   uint32_t ulist[kMaxUnits];            // this CTA's units of one decoder step, in consumption order
   uint16_t pstart[kMaxPhase + 1];       // first entry of every phase in ulist
   float sc[kMaxGroup][kAttnSplitMax];
-  float q[kMaxGroup][128];
+  alignas(16) float q[kMaxGroup][128];
   float kf[2][128], vf[2][128];
   float red[kPW][kPSlots];
   float red2[kPW][kPSlots];
@@ -185,6 +185,7 @@ struct PShared {
   PSlot slot[kPSlots];
   int lm_src[kPSlots];
   int segfirst[kPT];
+  int att[8];                           // attention geometry of the step: T, g_lo, g_hi, then this CTA's first chunk (s, gk, split, nsplit, g0)
   int tok[kPSlots];
   int dead, flag, result, chunk;
   unsigned long long thr;
@@ -481,6 +482,30 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       }
     }
     __syncthreads();
+    if (tid == 0) {
+      // chunks of split_len positions of all (slot, KV head) caches in (slot, head, position) order; this CTA's
+      // contiguous range of them and where it starts (the same for every layer of the step)
+      const int sl = A.split_len;
+      int T = 0;
+#pragma unroll 1
+      for (int s = 0; s < ns; ++s)
+        if (S.slot[s].active) T += A.Hkv * ((S.slot[s].pos + sl) / sl);
+      // (T <= 8 slots x 64 heads x 256 chunks, so c * T stays far below 2^31)
+      const int lo = cta * T / NC, hi = (cta + 1) * T / NC;
+      int s = 0, rem = lo, acc = 0, nsplit = 0;
+      if (lo < hi) {
+#pragma unroll 1
+        for (; s < ns; ++s) {
+          nsplit = S.slot[s].active ? (S.slot[s].pos + sl) / sl : 0;
+          if (rem < A.Hkv * nsplit) break;
+          rem -= A.Hkv * nsplit; acc += A.Hkv * nsplit;
+        }
+      }
+      const int gk = nsplit ? rem / nsplit : 0;
+      S.att[0] = T; S.att[1] = lo; S.att[2] = hi; S.att[3] = s; S.att[4] = gk; S.att[5] = nsplit ? rem - gk * nsplit : 0;
+      S.att[6] = nsplit; S.att[7] = acc + gk * nsplit;
+    }
+    __syncthreads();
 
 #pragma unroll 1
     for (int phase = 0; phase < n_phase; ++phase) {
@@ -567,73 +592,51 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         __syncthreads();
       } else if (kind == KIND_O && ka < kb) {
         // ---- stage the attention output, whole rows: put every pair's partial results together -----
-        // n_seg of a pair (see the attention phase): the CTAs its chunks fall on, or its chunks.
-        {
-          const int split_len = A.split_len;
-          int Ta = 0;
-#pragma unroll 1
-          for (int s = 0; s < n_in; ++s)
-            if (S.slot[s].active) Ta += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
-#pragma unroll 1
-          for (int c2 = tid; c2 < n_in * A.Hkv; c2 += kPT) {
-            const int s = c2 / A.Hkv, gk = c2 - s * A.Hkv;
-            int n_seg = 0;
-            if (S.slot[s].active) {
-              const int nsplit = (S.slot[s].pos + split_len) / split_len;
-              n_seg = nsplit;
-              if (Ta >= NC) {
-                int g0 = gk * nsplit;
-                for (int s2 = 0; s2 < s; ++s2)
-                  if (S.slot[s2].active) g0 += A.Hkv * ((S.slot[s2].pos + split_len) / split_len);
-                n_seg = ((g0 + nsplit) * NC - 1) / Ta - ((g0 + 1) * NC - 1) / Ta + 1;
-              }
-            }
-            S.segfirst[c2] = n_seg;
-          }
-          __syncthreads();
-        }
+        // The first four partial results of a pair are requested together with their count (entries past the
+        // count are ignored), so the common case costs one round trip to L2.
         const int nvec = g.kchunk >> 2;
+        const int spec = A.max_splits < 4 ? A.max_splits : 4;
 #pragma unroll 1
         for (int idx = tid; idx < n_in * nvec; idx += kPT) {
           const int s = idx / nvec, j = (idx - s * nvec) << 2;
           const int head = j / A.hd, dd = j - head * A.hd;
-          const int n_seg = S.segfirst[s * A.Hkv + head / grp];
           const size_t base = ((size_t)s * A.H + head) * A.max_splits;
+          float2 ml[4];
+          float4 x[4];
+          const int n_seg = S.slot[s].active ? __ldcg(A.tickets + s * A.Hkv + head / grp) : 0;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            ml[q] = q < spec ? __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + q) * 2)) : make_float2(-INFINITY, 0.0f);
+            x[q] = q < spec ? __ldcg(reinterpret_cast<const float4*>(A.part_o + (base + q) * A.hd + dd)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+          }
           float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-          if (n_seg == 1) {
-            const float2 ml = __ldcg(reinterpret_cast<const float2*>(A.part_ml + base * 2));
-            const float4 x = __ldcg(reinterpret_cast<const float4*>(A.part_o + base * A.hd + dd));
-            const float r = 1.0f / ml.y;
-            v = make_float4(x.x * r, x.y * r, x.z * r, x.w * r);
-          } else if (n_seg > 1) {
-            // running maximum over the partial results in their fixed order (4 at a time in flight)
-            float M = -INFINITY, den = 0.0f;
+          float M = -INFINITY, den = 0.0f;
 #pragma unroll 1
-            for (int j0 = 0; j0 < n_seg; j0 += 4) {
-              float2 ml[4];
-              float4 x[4];
+          for (int j0 = 0; j0 < n_seg; j0 += 4) {        // running maximum over the partial results in their fixed order
+            if (j0 > 0) {
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
                 const bool ok = j0 + q < n_seg;
                 ml[q] = ok ? __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + j0 + q) * 2)) : make_float2(-INFINITY, 0.0f);
                 x[q] = ok ? __ldcg(reinterpret_cast<const float4*>(A.part_o + (base + j0 + q) * A.hd + dd)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
               }
-              float Mn = M;
+            }
+            float Mn = M;
 #pragma unroll
-              for (int q = 0; q < 4; ++q) Mn = fmaxf(Mn, ml[q].x);
-              const float fo = (M > -INFINITY) ? expf(M - Mn) : 0.0f;
-              v.x *= fo; v.y *= fo; v.z *= fo; v.w *= fo; den *= fo;
+            for (int q = 0; q < 4; ++q) if (j0 + q < n_seg) Mn = fmaxf(Mn, ml[q].x);
+            const float fo = (M > -INFINITY) ? expf(M - Mn) : 0.0f;
+            v.x *= fo; v.y *= fo; v.z *= fo; v.w *= fo; den *= fo;
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const float f = (ml[q].x > -INFINITY) ? expf(ml[q].x - Mn) : 0.0f;
+            for (int q = 0; q < 4; ++q) {
+              if (j0 + q < n_seg && ml[q].x > -INFINITY) {
+                const float f = expf(ml[q].x - Mn);
                 v.x = fmaf(f, x[q].x, v.x); v.y = fmaf(f, x[q].y, v.y); v.z = fmaf(f, x[q].z, v.z); v.w = fmaf(f, x[q].w, v.w);
                 den = fmaf(f, ml[q].y, den);
               }
-              M = Mn;
             }
-            const float r = 1.0f / den;
-            v.x *= r; v.y *= r; v.z *= r; v.w *= r;
+            M = Mn;
           }
+          if (n_seg > 0) { const float r = 1.0f / den; v.x *= r; v.y *= r; v.z *= r; v.w *= r; }
           uint2 pk;
           pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
           *reinterpret_cast<uint2*>(act + s * apitch + j) = pk;
@@ -793,11 +796,29 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         w.s = s; w.nsplit = nsplit; w.gk = nsplit ? rem / nsplit : 0; w.split = nsplit ? rem - w.gk * nsplit : 0;
         w.g0 = acc + w.gk * nsplit;
       };
+      // Head size 64 with chunks of 256 positions runs on the tensor cores: a warp owns 16 positions of the chunk and
+      // loads K and V straight into mma fragments.  The order of the summed index of a product is free, so the
+      // 64 dims of q.k are dealt to the k-steps such that lane (g, t) needs the 16-byte pieces t and t + 4 of row g
+      // of a K n-tile; in P.V the output column (n-tile j, column g) stands for dim 8 g + j, so the lane needs
+      // piece g of the four positions 2t, 2t+1, 8+2t, 9+2t (pairs of positions are interleaved with byte permutes).
+      const bool mma_path = (A.hd == 64) && (split_len == kPW * 16);
+      const int gq = lane >> 2, t4 = lane & 3;
       auto issue_loads = [&](const Walk& w, uint4 (&kr)[4], uint4 (&vr)[4], bool want_k, bool want_v) {
         const int pos = S.slot[w.s].pos;
         const int p_lo = w.split * split_len, cnt = min(split_len, pos + 1 - p_lo);
         const int fresh_lo = pos - (w.s >= R ? 1 : 0);
         const size_t off = ((((size_t)S.slot[w.s].row * A.L + layer) * A.Hkv + w.gk) * A.cap) * A.hd;
+        if (mma_path) {
+          const int lim = min(cnt, fresh_lo - p_lo);                   // cached positions of the chunk: [0, lim)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int pk = warp * 16 + (i >> 1) * 8 + gq;                // K: n-tile i/2, row g; piece t or t + 4
+            const int pv = warp * 16 + (i >> 1) * 8 + 2 * t4 + (i & 1);   // V: positions 2t, 2t+1, 8+2t, 9+2t; piece g
+            if (want_k) kr[i] = pk < lim ? __ldcg(reinterpret_cast<const uint4*>(A.kc + off + (size_t)(p_lo + pk) * 64 + (t4 + 4 * (i & 1)) * 8)) : make_uint4(0u, 0u, 0u, 0u);
+            if (want_v) vr[i] = pv < lim ? __ldcg(reinterpret_cast<const uint4*>(A.vc + off + (size_t)(p_lo + pv) * 64 + gq * 8)) : make_uint4(0u, 0u, 0u, 0u);
+          }
+          return;
+        }
 #pragma unroll
         for (int ps = 0; ps < 4; ++ps) {
           const int p = ps * PPB + warp * PPW + pgrp;
@@ -810,12 +831,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       Walk cur{0, 0, 0, 0, 0}, nxt{0, 0, 0, 0, 0};
       int T = 0, g_lo = 0, g_hi = 0;
       if (kind == KIND_QKV) {
-#pragma unroll 1
-        for (int s = 0; s < ns; ++s)
-          if (S.slot[s].active) T += A.Hkv * ((S.slot[s].pos + split_len) / split_len);
-        // (T <= 8 slots x 64 heads x 256 chunks, so c * T stays far below 2^31)
-        g_lo = cta * T / NC; g_hi = (cta + 1) * T / NC;
-        if (g_lo < g_hi) seek(g_lo, cur);
+        T = S.att[0]; g_lo = S.att[1]; g_hi = S.att[2];
+        cur.s = S.att[3]; cur.gk = S.att[4]; cur.split = S.att[5]; cur.nsplit = S.att[6]; cur.g0 = S.att[7];
         TSEC(4);
         bar_target += (unsigned)NC;
         grid_barrier_arrive(bar);
@@ -876,6 +893,95 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               A.vc[off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
             }
           }
+          if (mma_path) {
+            // ---- per warp: scores, softmax, P V of its 16 positions for all heads of the group at once ----
+            const int lim = min(cnt, fresh_lo - p_lo);
+            uint32_t qa[4][2];
+            {
+              const float* qr = S.q[gq < grp ? gq : 0];
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const int d0 = (kk < 2 ? 0 : 32) + 8 * t4 + 4 * (kk & 1);
+                const float2 x = *reinterpret_cast<const float2*>(qr + d0), y = *reinterpret_cast<const float2*>(qr + d0 + 2);
+                qa[kk][0] = gq < grp ? pack_bf16(x.x, x.y) : 0u;      // q is bf16-valued already
+                qa[kk][1] = gq < grp ? pack_bf16(y.x, y.y) : 0u;
+              }
+            }
+            float sc2[2][4];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              sc2[j][0] = sc2[j][1] = sc2[j][2] = sc2[j][3] = 0.0f;
+              const uint32_t kw[8] = {kreg[2 * j].x, kreg[2 * j].y, kreg[2 * j].z, kreg[2 * j].w,
+                                      kreg[2 * j + 1].x, kreg[2 * j + 1].y, kreg[2 * j + 1].z, kreg[2 * j + 1].w};
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint32_t af[4] = {qa[kk][0], 0u, qa[kk][1], 0u}, bfr[2] = {kw[2 * kk], kw[2 * kk + 1]};
+                mma_bf16(sc2[j], af, bfr);
+              }
+            }
+            if (have_next) issue_loads(nxt, kreg, vreg, true, false);   // K registers are free
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                sc2[j][e] = (warp * 16 + j * 8 + 2 * t4 + e < lim) ? sc2[j][e] * A.attn_scale : -INFINITY;
+                mx = fmaxf(mx, sc2[j][e]);
+              }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            float pw[2][2], sum = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+              for (int e = 0; e < 2; ++e) { pw[j][e] = (sc2[j][e] > -INFINITY) ? __expf(sc2[j][e] - mx) : 0.0f; sum += pw[j][e]; }
+            // the weights as a bf16 head and a bf16 remainder: two products, fp32 sums
+            uint32_t ph[4] = {0u, 0u, 0u, 0u}, pl[4] = {0u, 0u, 0u, 0u};
+            {
+              const float h00 = round_bf16(pw[0][0]), h01 = round_bf16(pw[0][1]), h10 = round_bf16(pw[1][0]), h11 = round_bf16(pw[1][1]);
+              ph[0] = pack_bf16(h00, h01); pl[0] = pack_bf16(pw[0][0] - h00, pw[0][1] - h01);
+              ph[2] = pack_bf16(h10, h11); pl[2] = pack_bf16(pw[1][0] - h10, pw[1][1] - h11);
+            }
+            float oc[8][4];
+            {
+              const uint32_t va[4] = {vreg[0].x, vreg[0].y, vreg[0].z, vreg[0].w}, vb[4] = {vreg[1].x, vreg[1].y, vreg[1].z, vreg[1].w};
+              const uint32_t vc2[4] = {vreg[2].x, vreg[2].y, vreg[2].z, vreg[2].w}, vd[4] = {vreg[3].x, vreg[3].y, vreg[3].z, vreg[3].w};
+#pragma unroll
+              for (int jn = 0; jn < 8; ++jn) {
+                oc[jn][0] = oc[jn][1] = oc[jn][2] = oc[jn][3] = 0.0f;
+                const unsigned sel = (jn & 1) ? 0x7632u : 0x5410u;
+                const uint32_t bfr[2] = {__byte_perm(va[jn >> 1], vb[jn >> 1], sel), __byte_perm(vc2[jn >> 1], vd[jn >> 1], sel)};
+                mma_bf16(oc[jn], ph, bfr);
+                mma_bf16(oc[jn], pl, bfr);
+              }
+            }
+            if (have_next) issue_loads(nxt, kreg, vreg, false, true);   // ... and the V registers
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            if (gq < grp) {
+              // accumulate into the warp's running state of this segment: lane t of the quad holds dims 16t .. 16t+15
+              float* so_w = s_o + ((size_t)warp * grp + gq) * 64 + 16 * t4;
+              float m_old = -INFINITY, l_old = 0.0f;
+              if (!seg_start) { m_old = S.red[warp][gq]; l_old = S.red2[warp][gq]; }
+              const float M = fmaxf(m_old, mx);
+              const float f_old = (m_old > -INFINITY) ? __expf(m_old - M) : 0.0f;
+              const float f_new = (mx > -INFINITY) ? __expf(mx - M) : 0.0f;
+#pragma unroll
+              for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int q4 = 0; q4 < 2; ++q4) {
+                  float4 c4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                  float4* pp = reinterpret_cast<float4*>(so_w + 8 * hf + 4 * q4);
+                  if (!seg_start) { c4 = *pp; c4.x *= f_old; c4.y *= f_old; c4.z *= f_old; c4.w *= f_old; }
+                  c4.x = fmaf(oc[4 * q4 + 0][hf], f_new, c4.x); c4.y = fmaf(oc[4 * q4 + 1][hf], f_new, c4.y);
+                  c4.z = fmaf(oc[4 * q4 + 2][hf], f_new, c4.z); c4.w = fmaf(oc[4 * q4 + 3][hf], f_new, c4.w);
+                  *pp = c4;
+                }
+              __syncwarp(__activemask());
+              if (t4 == 0) { S.red[warp][gq] = M; S.red2[warp][gq] = l_old * f_old + sum * f_new; }
+            }
+            __syncwarp();
+          } else
           // ---- per warp: scores, softmax, P V over its cached positions of this chunk, head by head ----
 #pragma unroll 1
           for (int t = 0; t < grp; ++t) {
@@ -951,7 +1057,10 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             // ---- merge the warps (in warp order) and the fresh positions into the segment's partial result ----
             // Its place among the pair's partial results: with at least as many chunks as CTAs every CTA owns
             // chunks, so the segments of a pair sit on consecutive CTAs; with fewer, a segment is one chunk.
-            const int ord = (T >= NC) ? cta - ((cur.g0 + 1) * NC - 1) / T : split;
+            const int c_first = ((cur.g0 + 1) * NC - 1) / T;
+            const int ord = (T >= NC) ? cta - c_first : split;
+            if (ord == 0 && tid == 0)                  // how many partial results the pair has (read by the O-projection phase)
+              A.tickets[s * A.Hkv + gk] = (T >= NC) ? ((cur.g0 + nsplit) * NC - 1) / T - c_first + 1 : nsplit;
 #pragma unroll 1
             for (int idx = tid; idx < grp * A.hd; idx += kPT) {
               const int t = idx / A.hd, dd = idx - t * A.hd;
