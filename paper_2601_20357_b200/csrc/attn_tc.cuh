@@ -89,6 +89,7 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int n_stages = A.n_stages;
   const SlotDesc* __restrict__ slots = A.slots;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t4 = lane & 3;
+  pdl_trigger();
   extern __shared__ unsigned char atc_raw[];
   unsigned char* stage0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(atc_raw) + 1023) & ~(uintptr_t)1023);
   float* sq = reinterpret_cast<float*>(stage0 + (size_t)n_stages * 2 * kAtcTile);   // [n_stages][grp][HD] q beside its stage
@@ -104,6 +105,7 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     for (int i = 0; i < n_stages; ++i) { mbar_init(&full[i], 1); s_done[i] = 0; s_seg[i] = 0; }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  pdl_wait();                                   // the slot table, q and the appended K, V come from the kernels before
   // chunks before every slot (prefix sums), built by the whole CTA
   for (int i = tid; i < n_slots; i += kAtcThreads)
     s_pref[i + 1] = slots[i].active ? Hkv * ((slots[i].pos + SPLIT) / SPLIT) : 0;

@@ -20,6 +20,14 @@ struct SlotDesc { int row; int pos; int active; int pad; };
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
+// Programmatic dependent launch (kernels of a chain launched with the stream-serialization attribute):
+// pdl_trigger lets the next kernel of the stream be scheduled while this one still runs; pdl_wait blocks
+// until every kernel before this one has completed and its writes are visible.  A kernel must not touch
+// memory that other kernels write, or that they may still read, before pdl_wait.  Both are no-ops in a
+// kernel launched without the attribute.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
   static constexpr int kPerVec = 4;                      // elements per 16-byte load
@@ -65,6 +73,8 @@ struct StepArgs {
 // grid: number of slots of the step; block 128
 template <typename T>
 __global__ void k_begin_step(StepArgs A, const T* __restrict__ embed) {
+  pdl_trigger();
+  pdl_wait();
   const int s = blockIdx.x;
   int row, pos, active = 1, tok = -1;
   const float* src_embed = nullptr;
@@ -284,6 +294,8 @@ template <typename T>
 __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restrict__ slots, int H, int Hkv, int hd,
                               const float* __restrict__ rope_cos, const float* __restrict__ rope_sin,
                               T* __restrict__ kc, T* __restrict__ vc, int layer, int L, int cap) {
+  pdl_trigger();
+  pdl_wait();
   const int s = blockIdx.x;
   const SlotDesc sd = slots[s];
   if (!sd.active) return;

@@ -75,11 +75,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (G.slots) {
-    int any = 0;
-    for (int s = tid; s < G.n_slots; s += kTcThreads) any |= G.slots[s].active;
-    if (!__syncthreads_or(any)) return;
-  }
+  pdl_trigger();
   const int m_tile = blockIdx.x / G.ks, split = blockIdx.x - m_tile * G.ks;
   const int c_lo = split * G.cps, c_hi = min(c_lo + G.cps, G.k_chunks), n_ch = c_hi - c_lo;
   const size_t a_bytes = tc_block_bytes(kTcM), b_bytes = tc_block_bytes(G.n_pad);
@@ -101,19 +97,48 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = s_tmem;
+  const unsigned char* a_src = G.a_packed + ((size_t)m_tile * G.k_chunks + c_lo) * a_bytes;
+  const unsigned char* b_src = G.b_packed + (size_t)c_lo * b_bytes;
+  const int pre = n_ch < n_stages ? n_ch : n_stages;
+  // The weights do not depend on the kernels before this one: their first stages are requested before
+  // the wait on those kernels (transaction bytes announced without an arrival, so a stage's barrier
+  // cannot complete before its activations have been requested too).
+  if (tid == 0) {
+    for (int c = 0; c < pre; ++c) {
+      asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_full[c])), "r"((unsigned)a_bytes) : "memory");
+      bulk_g2s(tc_smem + (size_t)c * (a_bytes + b_bytes), a_src + (size_t)c * a_bytes, (unsigned)a_bytes, &s_full[c]);
+    }
+  }
+  pdl_wait();
+  {
+    int any = 1;
+    if (G.slots) {
+      any = 0;
+      for (int s = tid; s < G.n_slots; s += kTcThreads) any |= G.slots[s].active;
+    }
+    if (!__syncthreads_or(any)) {
+      // nobody needs this pass: let the weight copies land, give the tensor memory back, leave
+      if (tid == 0) {
+        for (int c = 0; c < pre; ++c) {
+          mbar_expect_tx(&s_full[c], 0u);
+          unsigned spins = 0;
+          while (!mbar_try_wait(&s_full[c], 0) && ++spins < (1u << 20)) __nanosleep(32);
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();
+      if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
+      return;
+    }
+  }
 
   if (tid == 0 && n_ch > 0) {
     // instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N and M
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(G.n_pad >> 3) << 17) | ((uint32_t)(kTcM >> 4) << 24);
-    const unsigned char* a_src = G.a_packed + ((size_t)m_tile * G.k_chunks + c_lo) * a_bytes;
-    const unsigned char* b_src = G.b_packed + (size_t)c_lo * b_bytes;
     bool ok = true;
-    const int pre = n_ch < n_stages ? n_ch : n_stages;
     for (int c = 0; c < pre; ++c) {
-      unsigned char* st = tc_smem + (size_t)c * (a_bytes + b_bytes);
-      mbar_expect_tx(&s_full[c], (unsigned)(a_bytes + b_bytes));
-      bulk_g2s(st, a_src + (size_t)c * a_bytes, (unsigned)a_bytes, &s_full[c]);
-      bulk_g2s(st + a_bytes, b_src + (size_t)c * b_bytes, (unsigned)b_bytes, &s_full[c]);
+      mbar_expect_tx(&s_full[c], (unsigned)b_bytes);
+      bulk_g2s(tc_smem + (size_t)c * (a_bytes + b_bytes) + a_bytes, b_src + (size_t)c * b_bytes, (unsigned)b_bytes, &s_full[c]);
     }
     int issued = pre;
     for (int c = 0; c < n_ch && ok; ++c) {
@@ -224,6 +249,8 @@ __global__ void k_pack_tc(const __nv_bfloat16* __restrict__ w0, int rows0, const
 // grid (k_chunks), block 256.
 __global__ void k_prep_act(const float* __restrict__ x, int stride, int n, int n_pad, int K, const float* __restrict__ row_scale,
                            const __nv_bfloat16* __restrict__ gain, unsigned char* __restrict__ dst) {
+  pdl_trigger();
+  pdl_wait();
   const int kc = blockIdx.x;
   unsigned char* blk = dst + (size_t)kc * tc_block_bytes(n_pad);
   for (int idx = threadIdx.x; idx < n_pad * (kTcKC / 8); idx += blockDim.x) {
@@ -259,6 +286,8 @@ struct PrepRowArgs {
   unsigned char* dst;                    // [k_chunks] blocks of n_pad rows
 };
 __global__ void __launch_bounds__(256) k_prep_row(const PrepRowArgs P) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x, tid = threadIdx.x;
   const int s = P.src_slot ? P.src_slot[P.slot0 + r] : P.slot0 + r;
   if (P.slots && !P.slots[s].active) return;
@@ -321,6 +350,8 @@ __global__ void __launch_bounds__(256) k_prep_row(const PrepRowArgs P) {
 // grid (k_chunks of F, slots of the group), block 16 (one thread per 8 columns of the chunk).
 __global__ void k_swiglu_prep(const float* __restrict__ partial, int ks, size_t slab, int F, const SlotDesc* __restrict__ slots,
                               int slot0, int n_pad, unsigned char* __restrict__ dst) {
+  pdl_trigger();
+  pdl_wait();
   const int kc = blockIdx.x, r = blockIdx.y, k8 = threadIdx.x;
   const int s = slot0 + r;
   if (slots && !slots[s].active) return;
@@ -345,6 +376,8 @@ __global__ void k_swiglu_prep(const float* __restrict__ partial, int ks, size_t 
 
 // out[i] = sum over the k-split slabs (fixed order); grid over elems.
 __global__ void k_sum_slabs(const float* __restrict__ part, int ks, size_t slab, size_t elems, float* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= elems) return;
   float4 v = make_float4(0.f, 0.f, 0.f, 0.f);

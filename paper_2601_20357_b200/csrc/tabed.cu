@@ -10,6 +10,7 @@
 #include <mutex>
 #include <new>
 #include <type_traits>
+#include <utility>
 #include <vector>
 
 #include "../../include/tabed.h"
@@ -124,6 +125,21 @@ struct ProfScope {
     (h)->launches++;                                                  \
   } while (0)
 
+// Launch as a programmatic dependent of the kernel before it in the stream (the kernel calls pdl_wait before it
+// touches anything dynamic): launch latency and prologue overlap the predecessor's tail.
+template <typename... KArgs, typename... Args>
+void launch_pdl(tabed_handle* h, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = h->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
+  h->launches++;
+}
+#define TABED_LAUNCH_PDL(h, kern, grid, block, smem, ...) launch_pdl((h), (kern), dim3(grid), dim3(block), (smem), __VA_ARGS__)
+
 template <typename T>
 int dev_alloc(tabed_handle* h, T** out, size_t count, bool zero = true) {
   void* ptr = nullptr;
@@ -223,7 +239,7 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
           a.qkv = h->qkv; a.slots = h->slots; a.n_slots = n_slots; a.H = h->H; a.Hkv = h->Hkv; a.layer = layer; a.L = h->L;
           a.cap = h->cap; a.qkv_w = h->qkv_w; a.part_o = h->part_o; a.part_ml = h->part_ml; a.max_splits = h->max_splits;
           a.tickets = h->attn_tickets; a.out = h->attn_out; a.scale = 1.0f / sqrtf((float)h->hd); a.err = h->err; a.n_stages = n_stages;
-          TABED_LAUNCH(h, k_attn_tc_bf16, n_ctas, kAtcThreads, smem2, h->tm_k, h->tm_v, a);
+          TABED_LAUNCH_PDL(h, k_attn_tc_bf16, n_ctas, kAtcThreads, smem2, h->tm_k, h->tm_v, a);
           return;
         }
       }
@@ -545,7 +561,7 @@ void launch_gemm_tc(tabed_handle* h, int kind, int layer, int n, float* partial,
   G.rows_total = t.rows; G.rows_valid = rows_valid; G.n_pad = (n + 15) / 16 * 16; G.n_slots = n;
   G.k_chunks = t.k_chunks; G.ks = t.ks; G.cps = t.cps; G.err = h->err;
   const size_t smem = (size_t)tc_stages(G.n_pad) * (tc_block_bytes(kTcM) + tc_block_bytes(G.n_pad)) + 1024;
-  TABED_LAUNCH(h, k_gemm_tc, t.m_tiles * t.ks, kTcThreads, smem, G);
+  TABED_LAUNCH_PDL(h, k_gemm_tc, t.m_tiles * t.ks, kTcThreads, smem, G);
 }
 
 // One shared-weight decoder step over `n_slots` slots with the projections on the tensor cores.
@@ -554,7 +570,7 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
   sa.R = h->R; sa.m = h->m; sa.d = h->d; sa.G = h->G;
   sa.kv_len = h->kv_len; sa.pending = h->pending;
   sa.slots = h->slots; sa.last_slot = h->last_slot; sa.x = h->x; sa.err = h->err; sa.kv_capacity = h->cap;
-  TABED_LAUNCH(h, k_begin_step<bf>, n_slots, 128, 0, sa, reinterpret_cast<const bf*>(h->embed));
+  TABED_LAUNCH_PDL(h, k_begin_step<bf>, n_slots, 128, 0, sa, reinterpret_cast<const bf*>(h->embed));
   const size_t S2 = 2 * (size_t)h->R;
   const int d = h->d, HD = h->H * h->hd, F = h->F;
   struct Grp { int s0, n; };
@@ -565,7 +581,7 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
     P.x = h->x; P.d = d; P.partial = partial; P.ks = partial ? ks : 0; P.slab = slab; P.src_slot = src; P.slots = slots;
     P.gain = reinterpret_cast<const bf*>(gain); P.eps = h->cfg.rms_eps; P.slot0 = g.s0; P.n = g.n; P.n_pad = (g.n + 15) / 16 * 16;
     P.write_back = write_back; P.dst = h->tc_act;
-    TABED_LAUNCH(h, k_prep_row, g.n, 256, 0, P);
+    TABED_LAUNCH_PDL(h, k_prep_row, g.n, 256, 0, P);
   };
   for (int l = 0; l < h->L; ++l) {
     {
@@ -575,8 +591,8 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
         launch_gemm_tc(h, KIND_QKV, l, g.n, h->tc_pq + (size_t)g.s0 * h->qkv_w, S2 * h->qkv_w, h->slots + g.s0, h->qkv_w);
       }
       const size_t elems = (size_t)n_slots * h->qkv_w;
-      TABED_LAUNCH(h, k_sum_slabs, (unsigned)((elems / 4 + 255) / 256), 256, 0, h->tc_pq, h->tck[KIND_QKV].ks, S2 * h->qkv_w, elems, h->qkv);
-      TABED_LAUNCH(h, k_rope_append<bf>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos, h->rope_sin,
+      TABED_LAUNCH_PDL(h, k_sum_slabs, (unsigned)((elems / 4 + 255) / 256), 256, 0, h->tc_pq, h->tck[KIND_QKV].ks, S2 * h->qkv_w, elems, h->qkv);
+      TABED_LAUNCH_PDL(h, k_rope_append<bf>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos, h->rope_sin,
                    reinterpret_cast<bf*>(h->kc), reinterpret_cast<bf*>(h->vc), l, h->L, h->cap);
     }
     {
@@ -587,7 +603,7 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
       ProfScope ps(h, TABED_PROF_OPROJ);
       for (const Grp& g : groups) {
         const int n_pad = (g.n + 15) / 16 * 16;
-        TABED_LAUNCH(h, k_prep_act, h->tck[KIND_O].k_chunks, 256, 0, h->attn_out + (size_t)g.s0 * HD, HD, g.n, n_pad, HD,
+        TABED_LAUNCH_PDL(h, k_prep_act, h->tck[KIND_O].k_chunks, 256, 0, h->attn_out + (size_t)g.s0 * HD, HD, g.n, n_pad, HD,
                      (const float*)nullptr, (const bf*)nullptr, h->tc_act);
         launch_gemm_tc(h, KIND_O, l, g.n, h->tc_po + (size_t)g.s0 * d, S2 * d, h->slots + g.s0, d);
       }
@@ -603,7 +619,7 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
       ProfScope ps(h, TABED_PROF_DOWN);
       for (const Grp& g : groups) {
         const int n_pad = (g.n + 15) / 16 * 16;
-        TABED_LAUNCH(h, k_swiglu_prep, dim3(h->tck[KIND_DN].k_chunks, g.n), kTcKC / 8, 0, h->tc_pgu, h->tck[KIND_GU].ks, S2 * 2 * F, F,
+        TABED_LAUNCH_PDL(h, k_swiglu_prep, dim3(h->tck[KIND_DN].k_chunks, g.n), kTcKC / 8, 0, h->tc_pgu, h->tck[KIND_GU].ks, S2 * 2 * F, F,
                      h->slots, g.s0, n_pad, h->tc_act);
         launch_gemm_tc(h, KIND_DN, l, g.n, h->tc_pd + (size_t)g.s0 * d, S2 * d, h->slots + g.s0, d);
       }
