@@ -4,6 +4,7 @@
 // warp-shuffle reductions, integer atomics for the cross-CTA sums (exact, order-free).
 #pragma once
 #include "exact_math.cuh"
+#include "forward_kernels.cuh"
 
 namespace tabed {
 
@@ -55,6 +56,8 @@ __device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v
 // grid (chunks, rows).  rowmax_enc[row] must be zeroed beforehand.
 __global__ void __launch_bounds__(kDecThreads)
 k_rowmax(const float* __restrict__ logits, int V, long long row_stride, uint32_t* __restrict__ rowmax_enc) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.y;
   const float* x = logits + (long long)row * row_stride;
   const bool vec = ((V & 3) == 0) && ((row_stride & 3) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
@@ -80,6 +83,8 @@ k_rowmax(const float* __restrict__ logits, int V, long long row_stride, uint32_t
 __global__ void __launch_bounds__(kDecThreads)
 k_expsum(const float* __restrict__ logits, int V, long long row_stride,
          const uint32_t* __restrict__ rowmax_enc, unsigned long long* __restrict__ rowsum) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.y;
   const float* x = logits + (long long)row * row_stride;
   const bool vec = ((V & 3) == 0) && ((row_stride & 3) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
@@ -101,6 +106,8 @@ __global__ void __launch_bounds__(kDecThreads)
 k_normalize(const float* __restrict__ logits, int V, long long row_stride,
             const uint32_t* __restrict__ rowmax_enc, const unsigned long long* __restrict__ rowsum,
             float* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.y;
   const float* x = logits + (long long)row * row_stride;
   float* o = out + (long long)row * V;
@@ -126,6 +133,8 @@ k_mix(const float* __restrict__ logits, int V, int m, const float* __restrict__ 
       float* __restrict__ qk_out, long long qk_req_stride,
       float* __restrict__ q_out, long long q_req_stride,
       unsigned long long* __restrict__ chunk_mass, ChunkBest* __restrict__ chunk_best, int n_chunks, int greedy) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.y;
   const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
   const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
@@ -197,6 +206,8 @@ __device__ __forceinline__ float resid_val(float p, float q) { return fmaxf(0.0f
 
 template <int SRC>
 __global__ void __launch_bounds__(kDecThreads) k_select(SelectArgs A) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.x;
   const int tid = threadIdx.x;
   __shared__ unsigned long long s_thr, s_scan[kDecThreads / 32], s_total;
@@ -329,6 +340,8 @@ __global__ void k_accept(int B, int G, int V, const float* __restrict__ p, const
                          long long q_req_stride, const int* __restrict__ tokens,
                          const float* __restrict__ u_accept, const ChunkBest* __restrict__ p_best,
                          int n_chunks, int greedy, int* __restrict__ n_accept, int* __restrict__ out_n_accept) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   int a = 0;
@@ -356,6 +369,8 @@ __global__ void k_accept(int B, int G, int V, const float* __restrict__ p, const
 // per-chunk argmax of every target row (greedy verification); grid (chunks, B*(G+1))
 __global__ void __launch_bounds__(kDecThreads)
 k_row_best(const float* __restrict__ p, int V, int n_chunks, ChunkBest* __restrict__ best) {
+  pdl_trigger();
+  pdl_wait();
   const int row = blockIdx.y;
   const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
   float a[kPerThread];
@@ -384,6 +399,8 @@ k_row_best(const float* __restrict__ p, int V, int n_chunks, ChunkBest* __restri
 __global__ void __launch_bounds__(kDecThreads)
 k_resid_chunks(int V, int G, const float* __restrict__ p, const float* __restrict__ q, long long q_req_stride,
                const int* __restrict__ n_accept, unsigned long long* __restrict__ chunk_mass, int n_chunks) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.y;
   const int a = n_accept[b];
   const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
@@ -411,6 +428,8 @@ __global__ void __launch_bounds__(kDecThreads)
 k_deviation(int V, int G, int m, int n_dev, int grid_policy, int tvd,
             const float* __restrict__ p, const float* __restrict__ qk, const int* __restrict__ n_accept,
             long long* __restrict__ dev) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.z, i = blockIdx.y;
   const int a = n_accept[b];
   if (i > min(a, G - 1)) return;
@@ -498,6 +517,8 @@ struct PolicyArgs {
 };
 
 __global__ void k_policy(PolicyArgs A) {
+  pdl_trigger();
+  pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= A.B) return;
   const int a = A.n_accept[b];

@@ -335,16 +335,16 @@ void run_ensemble(tabed_handle* h, const float* logits, const float* w, const fl
   cudaMemsetAsync(h->rowmax, 0, sizeof(uint32_t) * h->R, h->stream);
   cudaMemsetAsync(h->rowsum, 0, sizeof(unsigned long long) * h->R, h->stream);
   const dim3 grid_rows(h->n_chunks, h->R), grid_req(h->n_chunks, h->B);
-  TABED_LAUNCH(h, k_rowmax, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax);
-  TABED_LAUNCH(h, k_expsum, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
-  TABED_LAUNCH(h, k_mix, grid_req, kDecThreads, 0, logits, h->V, h->m, w, h->rowmax, h->rowsum, qk_out, qk_stride,
+  TABED_LAUNCH_PDL(h, k_rowmax, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax);
+  TABED_LAUNCH_PDL(h, k_expsum, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
+  TABED_LAUNCH_PDL(h, k_mix, grid_req, kDecThreads, 0, logits, h->V, h->m, w, h->rowmax, h->rowsum, qk_out, qk_stride,
                q_out, q_stride, h->chunk_mass, h->chunk_best, h->n_chunks, greedy);
   SelectArgs s{};
   s.V = h->V; s.n_chunks = h->n_chunks; s.G = h->G; s.greedy = greedy;
   s.q = q_out; s.q_req_stride = q_stride; s.u = u; s.u_stride = u_stride;
   s.chunk_mass = h->chunk_mass; s.chunk_best = h->chunk_best;
   s.out0 = y0; s.out0_stride = y0_stride; s.out1 = y1; s.out1_stride = y1_stride; s.err = h->err;
-  TABED_LAUNCH(h, k_select<0>, h->B, kDecThreads, 0, s);
+  TABED_LAUNCH_PDL(h, k_select<0>, h->B, kDecThreads, 0, s);
 }
 
 // ---- persistent drafting-round kernel: geometry and set-up -----------------------------------------
@@ -964,20 +964,20 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   cudaMemsetAsync(h->rowmax, 0, sizeof(uint32_t) * rows, h->stream);
   cudaMemsetAsync(h->rowsum, 0, sizeof(unsigned long long) * rows, h->stream);
   const dim3 grid_rows(h->n_chunks, rows), grid_req(h->n_chunks, h->B);
-  TABED_LAUNCH(h, k_rowmax, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax);
-  TABED_LAUNCH(h, k_expsum, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
-  TABED_LAUNCH(h, k_normalize, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum, h->p);
+  TABED_LAUNCH_PDL(h, k_rowmax, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax);
+  TABED_LAUNCH_PDL(h, k_expsum, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
+  TABED_LAUNCH_PDL(h, k_normalize, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum, h->p);
   if (greedy) TABED_LAUNCH(h, k_row_best, grid_rows, kDecThreads, 0, h->p, h->V, h->n_chunks, h->chunk_best);
-  TABED_LAUNCH(h, k_accept, (h->B + 127) / 128, 128, 0, h->B, h->G, h->V, h->p, h->q, GV, h->tokens, u_accept,
+  TABED_LAUNCH_PDL(h, k_accept, (h->B + 127) / 128, 128, 0, h->B, h->G, h->V, h->p, h->q, GV, h->tokens, u_accept,
                h->chunk_best, h->n_chunks, greedy, h->n_accept, out_n_accept);
   if (!greedy)
-    TABED_LAUNCH(h, k_resid_chunks, grid_req, kDecThreads, 0, h->V, h->G, h->p, h->q, GV, h->n_accept, h->chunk_mass, h->n_chunks);
+    TABED_LAUNCH_PDL(h, k_resid_chunks, grid_req, kDecThreads, 0, h->V, h->G, h->p, h->q, GV, h->n_accept, h->chunk_mass, h->n_chunks);
   SelectArgs s{};
   s.V = h->V; s.n_chunks = h->n_chunks; s.G = h->G; s.greedy = greedy;
   s.q = h->q; s.q_req_stride = GV; s.p = h->p; s.n_accept = h->n_accept; s.u = u_resid; s.u_stride = 1;
   s.chunk_mass = h->chunk_mass; s.chunk_best = h->chunk_best;
   s.out0 = h->next_token; s.out0_stride = 1; s.out1 = out_next_token; s.out1_stride = 1; s.err = h->err;
-  TABED_LAUNCH(h, k_select<1>, h->B, kDecThreads, 0, s);
+  TABED_LAUNCH_PDL(h, k_select<1>, h->B, kDecThreads, 0, s);
   h->phase = PH_VERIFIED;
   return check_cuda();
 }
@@ -988,7 +988,7 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
   DeviceGuard guard(h->cfg.device);
   const int tvd = h->cfg.distance == TABED_DIST_TVD;
   ProfScope* ps = new ProfScope(h, TABED_PROF_UPDATE);
-  TABED_LAUNCH(h, k_deviation, dim3(h->n_chunks, h->G, h->B), kDecThreads, 0, h->V, h->G, h->m, h->n_dev,
+  TABED_LAUNCH_PDL(h, k_deviation, dim3(h->n_chunks, h->G, h->B), kDecThreads, 0, h->V, h->G, h->m, h->n_dev,
                  h->cfg.policy == TABED_POLICY_GRID_MT ? 1 : 0, tvd, h->p, h->qk, h->n_accept, h->dev);
   PolicyArgs a{};
   a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
@@ -997,7 +997,7 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
   a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
   a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
   a.pending = h->pending; a.out_w = out_w; a.out_argmax = out_w_argmax;
-  TABED_LAUNCH(h, k_policy, (h->B + 127) / 128, 128, 0, a);
+  TABED_LAUNCH_PDL(h, k_policy, (h->B + 127) / 128, 128, 0, a);
   delete ps;
   if (h->has_drafter && h->round_has_forward) for (int& v : h->len_ub) v = std::min(v + h->G + 1, h->cap);
   h->phase = PH_IDLE;
