@@ -78,11 +78,11 @@ __global__ void k_begin_step(StepArgs A, const T* __restrict__ embed) {
   const int s = blockIdx.x;
   int row, pos, active = 1, tok = -1;
   const float* src_embed = nullptr;
-  if (A.mode == STEP_PREFILL) {
+  if (A.mode == STEP_PREFILL) {                    // slot s = position prefill_off + s of the row's new prefix
     row = A.prefill_row;
-    pos = A.kv_len[row] + A.prefill_off;
-    if (A.prefill_tokens) tok = A.prefill_tokens[A.prefill_off];
-    else src_embed = A.prefill_embeds + (long long)A.prefill_off * A.d;
+    pos = A.kv_len[row] + A.prefill_off + s;
+    if (A.prefill_tokens) tok = A.prefill_tokens[A.prefill_off + s];
+    else src_embed = A.prefill_embeds + (long long)(A.prefill_off + s) * A.d;
   } else {
     row = s % A.R;
     const int b = row / A.m;

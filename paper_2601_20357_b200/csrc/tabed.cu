@@ -88,7 +88,9 @@ struct tabed_handle {
   uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
   unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false; int trace_cta = 0;
   // tensor-core projections for many rows (bf16 drafter, more than 8 slots per step)
-  bool tc_ok = false;
+  bool tc_ok = false;                        // tcgen05 projections are set up (prefill in chunks; drafting when tc_auto)
+  bool tc_auto = false;                      // ... and are the automatic choice for drafting (16 or more rows)
+  int slot_cap = 0;                          // slots the step buffers hold: 2R, or a prefill chunk if that is more
   struct TcKind { int rows, K, m_tiles, k_chunks, ks, cps; size_t bytes; };
   TcKind tck[5]{};                  // KIND_QKV, KIND_O, KIND_GU (gate|up rows), KIND_DN, KIND_LM
   unsigned char* tc_w = nullptr;    // [L][QKV | O | GU | DN] then LM, operand blocks of k_pack_tc
@@ -494,7 +496,7 @@ int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_
 int setup_tc(tabed_handle* h) {
   const tabed_config& c = h->cfg;
   h->tc_ok = false;
-  if (c.dtype != TABED_DTYPE_BF16 || h->persist_ok || h->R < 16 || h->d % 8 || h->F % 8 || (h->H * h->hd) % 8) return TABED_OK;
+  if (c.dtype != TABED_DTYPE_BF16 || h->slot_cap < kPrefillChunk || h->d % 8 || h->F % 8 || (h->H * h->hd) % 8) return TABED_OK;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return TABED_ERR_CUDA;
   if (prop.major < 10) return TABED_OK;
@@ -517,7 +519,7 @@ int setup_tc(tabed_handle* h) {
   h->tc_off[KIND_DN] = h->tc_off[KIND_GU] + h->tck[KIND_GU].bytes;
   h->tc_layer_stride = h->tc_off[KIND_DN] + h->tck[KIND_DN].bytes;
   h->tc_off[KIND_LM] = h->tc_layer_stride * h->L;
-  const int n_pad_max = (std::min(2 * h->R, kTcMaxN) + 15) / 16 * 16;
+  const int n_pad_max = (std::min(h->slot_cap, kTcMaxN) + 15) / 16 * 16;
   h->tc_smem = 0;
   for (int np = 16; np <= n_pad_max; np += 16)
     h->tc_smem = std::max(h->tc_smem, (size_t)tc_stages(np) * (tc_block_bytes(kTcM) + tc_block_bytes(np)) + 1024);
@@ -525,7 +527,7 @@ int setup_tc(tabed_handle* h) {
   if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->tc_smem) != cudaSuccess) return TABED_ERR_CUDA;
   int rc = TABED_OK;
   auto A2 = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count, false); };
-  const size_t S2 = 2 * (size_t)h->R;
+  const size_t S2 = (size_t)h->slot_cap;
   int kc_max = 0;
   for (int k = 0; k < 5; ++k) kc_max = std::max(kc_max, h->tck[k].k_chunks);
   A2(&h->tc_w, h->tc_off[KIND_LM] + h->tck[KIND_LM].bytes);
@@ -549,6 +551,7 @@ int setup_tc(tabed_handle* h) {
   }
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
   h->tc_ok = true;
+  h->tc_auto = !h->persist_ok && h->R >= 16;
   return TABED_OK;
 }
 
@@ -571,7 +574,7 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
   sa.kv_len = h->kv_len; sa.pending = h->pending;
   sa.slots = h->slots; sa.last_slot = h->last_slot; sa.x = h->x; sa.err = h->err; sa.kv_capacity = h->cap;
   TABED_LAUNCH_PDL(h, k_begin_step<bf>, n_slots, 128, 0, sa, reinterpret_cast<const bf*>(h->embed));
-  const size_t S2 = 2 * (size_t)h->R;
+  const size_t S2 = (size_t)h->slot_cap;
   const int d = h->d, HD = h->H * h->hd, F = h->F;
   struct Grp { int s0, n; };
   std::vector<Grp> groups;                       // up to 256 slots share one pass over the weights
@@ -636,6 +639,11 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
 }
 
 int check_cuda() { return cudaGetLastError() == cudaSuccess ? TABED_OK : TABED_ERR_CUDA; }
+
+// drafting steps outside the persistent kernel: tensor-core projections when chosen (or automatic with many rows)
+bool use_tc(const tabed_handle* h) {
+  return h->tc_ok && (h->path_sel == TABED_PATH_TENSOR_CORE || (h->path_sel == TABED_PATH_AUTO && h->tc_auto));
+}
 
 int max_len_ub(const tabed_handle* h) {
   int mx = 0;
@@ -734,11 +742,15 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
     unsigned char *kcb = nullptr, *vcb = nullptr;
     A(&kcb, kv_elems * h->esz); A(&vcb, kv_elems * h->esz);
     h->kc = kcb; h->vc = vcb;
-    A(&h->kv_len, R); A(&h->slots, 2 * R); A(&h->last_slot, R);
-    A(&h->x, 2 * R * h->d); A(&h->qkv, 2 * R * h->qkv_w); A(&h->attn_out, 2 * R * h->H * h->hd); A(&h->mid, 2 * R * h->F);
-    A(&h->part_o, 2 * R * h->H * (size_t)h->max_splits * h->hd); A(&h->part_ml, 2 * R * h->H * (size_t)h->max_splits * 2);
+    // step buffers: 2R slots for drafting; a bf16 drafter is prefilled in chunks of kPrefillChunk positions
+    // (one slot per position) through the tensor-core kernels, which needs that many
+    const size_t SC = (c.dtype == TABED_DTYPE_BF16) ? std::max<size_t>(2 * R, kPrefillChunk) : 2 * R;
+    h->slot_cap = (int)SC;
+    A(&h->kv_len, R); A(&h->slots, SC); A(&h->last_slot, R);
+    A(&h->x, SC * h->d); A(&h->qkv, SC * h->qkv_w); A(&h->attn_out, SC * h->H * h->hd); A(&h->mid, SC * h->F);
+    A(&h->part_o, SC * h->H * (size_t)h->max_splits * h->hd); A(&h->part_ml, SC * h->H * (size_t)h->max_splits * 2);
     A(&h->logits_own, G * R * V);
-    A(&h->attn_tickets, 2 * R * h->Hkv);
+    A(&h->attn_tickets, SC * h->Hkv);
     { cudaDeviceProp pr; if (cudaGetDeviceProperties(&pr, c.device) == cudaSuccess) h->n_sm = pr.multiProcessorCount; }
     if (c.dtype == TABED_DTYPE_BF16 && h->hd == kAtcHd && h->H / h->Hkv <= kMaxGroup && rc == TABED_OK) {
       // TMA descriptors of the caches seen as [all rows of all (row, layer, head)][64] bf16, tiles of 128 rows, 128-byte swizzle
@@ -837,11 +849,23 @@ static int prefill_common(tabed_handle* h, int32_t row, const int32_t* tokens, c
   if (row < 0 || row >= h->R || len < 1) return TABED_ERR_INVALID_ARG;
   if (h->len_ub[row] + len > h->cap) return TABED_ERR_KV_OVERFLOW;
   DeviceGuard guard(h->cfg.device);
-  for (int t = 0; t < len; ++t) {
-    StepArgs sa{};
-    sa.mode = STEP_PREFILL; sa.prefill_row = row; sa.prefill_off = t;
-    sa.prefill_tokens = tokens; sa.prefill_embeds = embeds;
-    run_step(h, sa, 1, h->len_ub[row] + t + 1, nullptr);
+  if (h->tc_ok && h->path_sel != TABED_PATH_PER_OP) {
+    // chunks of positions as slots of one weight pass: the projections are dense contractions (tcgen05), every
+    // slot attends over the row's cache up to its own position (all K, V of the chunk are appended first)
+    for (int t = 0; t < len; t += kPrefillChunk) {
+      const int n = std::min(kPrefillChunk, len - t);
+      StepArgs sa{};
+      sa.mode = STEP_PREFILL; sa.prefill_row = row; sa.prefill_off = t;
+      sa.prefill_tokens = tokens; sa.prefill_embeds = embeds;
+      run_step_tc(h, sa, n, h->len_ub[row] + t + n, nullptr);
+    }
+  } else {
+    for (int t = 0; t < len; ++t) {
+      StepArgs sa{};
+      sa.mode = STEP_PREFILL; sa.prefill_row = row; sa.prefill_off = t;
+      sa.prefill_tokens = tokens; sa.prefill_embeds = embeds;
+      run_step(h, sa, 1, h->len_ub[row] + t + 1, nullptr);
+    }
   }
   TABED_LAUNCH(h, k_advance_len, (h->R + 127) / 128, 128, 0, h->kv_len, h->R, row, len);
   h->len_ub[row] += len;
@@ -882,7 +906,7 @@ int tabed_decode_step(tabed_handle* h, const int32_t* tok, float* out_logits) {
   DeviceGuard guard(h->cfg.device);
   StepArgs sa{};
   sa.mode = STEP_FREE; sa.tokens = tok;
-  if (h->tc_ok && h->path_sel != TABED_PATH_PER_OP) run_step_tc(h, sa, h->R, max_len_ub(h) + 1, out_logits);
+  if (use_tc(h)) run_step_tc(h, sa, h->R, max_len_ub(h) + 1, out_logits);
   else run_step(h, sa, h->R, max_len_ub(h) + 1, out_logits);
   TABED_LAUNCH(h, k_advance_len, (h->R + 127) / 128, 128, 0, h->kv_len, h->R, -1, 1);
   for (int& v : h->len_ub) v += 1;
@@ -907,7 +931,7 @@ static int draft_common(tabed_handle* h, const float* ext_logits, const float* u
   if (fwd && max_len_ub(h) + 2 + h->G - 1 > h->cap) return TABED_ERR_KV_OVERFLOW;
   DeviceGuard guard(h->cfg.device);
   const long long RV = (long long)h->R * h->V, GV = (long long)h->G * h->V;
-  if (fwd && h->persist_ok && h->path_sel != 1) {
+  if (fwd && h->persist_ok && (h->path_sel == TABED_PATH_AUTO || h->path_sel == TABED_PATH_PERSISTENT)) {
     // the whole round (gamma decoder steps, each with its ensemble + draw) in one cooperative launch
     {
       ProfScope ps(h, TABED_PROF_DRAFT_ROUND);
@@ -926,7 +950,7 @@ static int draft_common(tabed_handle* h, const float* ext_logits, const float* u
       StepArgs sa{};
       sa.mode = (i == 0) ? STEP_ROUND_FIRST : STEP_ROUND_NEXT; sa.step = i; sa.tokens = h->tokens;
       float* own = h->logits_own + i * RV;
-      if (h->tc_ok && h->path_sel != TABED_PATH_PER_OP) run_step_tc(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
+      if (use_tc(h)) run_step_tc(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
       else run_step(h, sa, i == 0 ? 2 * h->R : h->R, max_len_ub(h) + 2 + i, own);
       lg = h->logits_override ? h->logits_override + i * RV : own;
     } else {
@@ -1080,7 +1104,9 @@ int tabed_select_path(tabed_handle* h, int32_t path) {
 int tabed_current_path(const tabed_handle* h) {
   if (!h) return TABED_ERR_NULL_PTR;
   if (h->path_sel == TABED_PATH_PER_OP) return TABED_PATH_PER_OP;
-  return h->persist_ok ? TABED_PATH_PERSISTENT : (h->tc_ok ? TABED_PATH_TENSOR_CORE : TABED_PATH_PER_OP);
+  if (h->path_sel == TABED_PATH_TENSOR_CORE) return TABED_PATH_TENSOR_CORE;
+  if (h->path_sel == TABED_PATH_PERSISTENT) return TABED_PATH_PERSISTENT;
+  return h->persist_ok ? TABED_PATH_PERSISTENT : (h->tc_auto ? TABED_PATH_TENSOR_CORE : TABED_PATH_PER_OP);
 }
 
 int tabed_debug_trace(tabed_handle* h, int32_t on) {

@@ -53,12 +53,16 @@ class Pair:
     orc: TabedOracle
 
 
-def build_pair(wl: W.Workload, kv_lengths: Optional[np.ndarray] = None) -> Pair:
-    """Drafter-backed handle and checker with identical weights, prefixes / synthetic caches, pending tokens."""
+def build_pair(wl: W.Workload, kv_lengths: Optional[np.ndarray] = None, prefill_path: Optional[int] = None) -> Pair:
+    """Drafter-backed handle and checker with identical weights, prefixes / synthetic caches, pending tokens.
+    prefill_path: path selected while the prompts are fed (None = the library's choice: chunks of positions
+    through the tensor-core kernels for a bf16 drafter); the automatic choice is restored afterwards."""
     weights = W.make_weights(wl)
     orc = make_oracle(wl, OracleDrafter(wl.drafter, weights))
     wdev = TB.weights_to_device(wl.drafter, weights, DEV)
     gpu = make_gpu(wl, wdev)
+    if prefill_path is not None:
+        gpu.select_path(prefill_path)
     tdt = torch.float32 if wl.drafter.dtype == "fp32" else torch.bfloat16
     if wl.synthetic_kv_len is not None:
         lens = kv_lengths if kv_lengths is not None else W.synthetic_kv_lengths(wl)
@@ -76,6 +80,8 @@ def build_pair(wl: W.Workload, kv_lengths: Optional[np.ndarray] = None) -> Pair:
                         gpu.prefill_tokens(row, t(seg.data))
                     else:
                         gpu.prefill_embeds(row, t(seg.data))
+    if prefill_path is not None:
+        gpu.select_path(TB.PATH_AUTO)
     pend = W.initial_pending(wl)
     orc.set_pending(pend)
     tok = np.zeros((wl.n_requests, 2), np.int32)

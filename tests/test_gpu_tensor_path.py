@@ -116,3 +116,35 @@ def test_attention_many_rows_several_chunks_each():
     for rnd in range(3):
         H.lockstep_round(pair, rnd, override=True)
     pair.gpu.destroy()
+
+
+# ------------------------------------------------------------------------------------------------
+# prompts fed in chunks of 128 positions through the tensor-core kernels
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("heads,kv_heads,d", [(4, 2, 256), (8, 2, 256)])
+def test_chunked_prefill_matches_position_by_position_prefill(heads, kv_heads, d):
+    """The same prompts (700 tokens = 5 full chunks + 60; 130 = one chunk + 2; 37 embeddings + 9 tokens) fed as
+    chunks of positions (tcgen05 projections, every position attending up to itself) and one position at a
+    time (per-operation kernels): both handles then follow the checker in lock step, and their first
+    drafting step agrees within the bf16 bound.  Head sizes 64 (TMA attention) and 32 (split kernels)."""
+    wl = wl_attn(heads=heads, kv_heads=kv_heads, d=d, cap=1024, cid=120 + heads,
+                 prefixes=((("tokens", 700),), (("tokens", 130),), (("embeds", 37), ("tokens", 9))))
+    a = H.build_pair(wl)
+    b = H.build_pair(wl, prefill_path=TB.PATH_PER_OP)
+    ud, _, _ = W.round_uniforms(wl, 0)
+    toks = torch.empty((1, wl.gamma), dtype=torch.int32, device=H.DEV)
+    for p in (a, b):
+        p.gpu.select_path(TB.PATH_PER_OP)
+    a.gpu.draft_round(H.t(ud), toks)
+    b.gpu.draft_round(H.t(ud), toks.clone())
+    torch.cuda.synchronize()
+    la = a.gpu.debug_view(TB.VIEW_LOGITS)[0].cpu().numpy()
+    lb = b.gpu.debug_view(TB.VIEW_LOGITS)[0].cpu().numpy()
+    assert np.max(np.abs(la - lb)) <= H.LOGIT_TOL["bf16"]
+    H.check_error_flag(a.gpu); H.check_error_flag(b.gpu)
+    a.gpu.destroy(); b.gpu.destroy()
+    for path in (None, TB.PATH_PER_OP):
+        pair = H.build_pair(wl, prefill_path=path)
+        for rnd in range(2):
+            H.lockstep_round(pair, rnd, override=True)
+        pair.gpu.destroy()
