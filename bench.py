@@ -190,7 +190,40 @@ def run_reference(args, wl):
 # --------------------------------------------------------------------------------------------------
 # CUDA arm
 # --------------------------------------------------------------------------------------------------
-def gpu_setup(wl, device):
+def run_prefill(args, wl):
+    """Feeding the prompts (not part of a round; the caches it leaves are what the rounds read): one JSON line with
+    the tokens per second of both ways of feeding them, on a fresh handle each."""
+    import torch
+    from paper_2601_20357_b200 import binding as TB
+    if wl.synthetic_kv_len is not None or wl.drafter.dtype != "bf16":
+        print(json.dumps({"metric": "prefill_tokens_per_sec", "unavailable": "the workload's caches are loaded, not computed, "
+                          "or its drafter is fp32 (fed one position at a time only)"}), flush=True)
+        return
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    res = {}
+    for name, path in (("chunks_of_128_positions_tcgen05", None), ("one_position_at_a_time", TB.PATH_PER_OP)):
+        best = None
+        for rep in range(3):
+            tms = []
+            g = gpu_setup(wl, device, prefill_path=path, prefill_times=tms)
+            g.destroy()
+            best = tms[0] if best is None or tms[0][1] < best[1] else best
+        res[name] = {"tokens": best[0], "ms": best[1], "tokens_per_sec": best[0] / (best[1] / 1000.0)}
+    c = wl.drafter
+    layer_w = c.n_layers * (c.d_model * (c.n_heads + 2 * c.n_kv_heads) * (c.d_model // c.n_heads) + c.n_heads * (c.d_model // c.n_heads) * c.d_model
+                            + 3 * c.d_model * c.d_ffn) * 2
+    print(json.dumps({"metric": "prefill_tokens_per_sec", "value": res["chunks_of_128_positions_tcgen05"]["tokens_per_sec"],
+                      "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True, "data": "synthetic",
+                      "config": {"workload": wl.name, "rows": wl.n_rows, "prompt_tokens": res["chunks_of_128_positions_tcgen05"]["tokens"]},
+                      "ways": res, "layer_weight_bytes_per_chunk": int(layer_w),
+                      "note": "best of 3 fresh handles each, CUDA events around the feeding calls; a chunk reads the layers' "
+                              "weights once for 128 positions"}), flush=True)
+
+
+def gpu_setup(wl, device, prefill_path=None, prefill_times=None):
+    """prefill_path: path forced while the prompts are fed (None: the library's choice); prefill_times: a list that
+    receives (tokens, milliseconds) of the prompt feeding, timed with CUDA events."""
     import torch
     from paper_2601_20357_b200 import binding as TB
     weights = TB.weights_to_device(wl.drafter, W.make_weights(wl), device)
@@ -206,13 +239,24 @@ def gpu_setup(wl, device):
             k, v = W.make_synthetic_kv(wl, row, int(lens[row]))
             g.load_prefix_kv(row, dev(k, tdt), dev(v, tdt))
     else:
-        for b in range(wl.n_requests):
-            for k, segs in enumerate(W.make_prefixes(wl, b)):
-                for seg in segs:
-                    if seg.kind == "tokens":
-                        g.prefill_tokens(b * wl.n_inputs + k, dev(seg.data))
-                    else:
-                        g.prefill_embeds(b * wl.n_inputs + k, dev(seg.data))
+        if prefill_path is not None:
+            g.select_path(prefill_path)
+        feed = [(b * wl.n_inputs + k, seg.kind, dev(seg.data)) for b in range(wl.n_requests)
+                for k, segs in enumerate(W.make_prefixes(wl, b)) for seg in segs]
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for row, kind, data in feed:
+            if kind == "tokens":
+                g.prefill_tokens(row, data)
+            else:
+                g.prefill_embeds(row, data)
+        e1.record()
+        torch.cuda.synchronize(device)
+        if prefill_times is not None:
+            prefill_times.append((int(sum(x[2].shape[0] for x in feed)), float(e0.elapsed_time(e1))))
+        if prefill_path is not None:
+            g.select_path(TB.PATH_AUTO)
     tok = np.zeros((wl.n_requests, 2), np.int32)
     tok[:, 0] = W.initial_pending(wl)
     g.set_pending(dev(tok), dev(np.ones(wl.n_requests, np.int32)))
@@ -494,6 +538,9 @@ def main():
     ap.add_argument("--trace", default=None, help="write the persistent kernel's phase timeline of one round to this file")
     ap.add_argument("--trace-cta", type=int, default=0, help="the CTA whose phase timeline --trace records")
     ap.add_argument("--requests", type=int, default=0, help="override the workload's number of concurrent requests (profiling aid)")
+    ap.add_argument("--prefill", action="store_true",
+                    help="time the feeding of the workload's prompts instead of rounds: chunks of positions through the "
+                         "tensor-core kernels (the library's choice for bf16) and one position at a time")
     ap.add_argument("--path", default="auto", choices=["auto", "per-op"], help="drafting path (per-op forces one kernel per operation)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -503,6 +550,8 @@ def main():
         wl = wl.replace(n_requests=args.requests, name=f"{wl.name}[B={args.requests}]")
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.prefill:
+        run_prefill(args, wl)
     else:
         run_ours(args, wl)
 
