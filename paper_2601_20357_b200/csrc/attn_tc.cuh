@@ -33,6 +33,7 @@
 #include <stdint.h>
 
 #include "forward_kernels.cuh"
+#include "gemm_tc.cuh"
 #include "round_kernel.cuh"
 
 namespace tabed {
@@ -54,7 +55,9 @@ struct AttnTcArgs {
   float *part_o, *part_ml;                   // [n_slots][H][max_splits][hd], [..][2] segment partials
   int max_splits;
   int* tickets;                              // [n_slots][Hkv], zero on entry and on exit
-  float* out;                                // [n_slots][H][hd]
+  float* out;                                // [n_slots][H][hd]; unused when act_out is given
+  unsigned char* act_out;                    // or null: the output as the bf16 B operand of the next projection
+  int act_npad;                              //   (core-matrix layout of k_gemm_tc for act_npad slots, K = H * hd)
   float scale;
   int* err;
   int n_stages;
@@ -149,6 +152,17 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     tma_load_2d(dst, &tm_k, 0, y, bar);
     tma_load_2d(dst + kAtcTile, &tm_v, 0, y, bar);
     if (with_q) bulk_g2s(sq + (size_t)st * grp * HD, A.qkv + (size_t)w.s * A.qkv_w + (size_t)w.gk * grp * HD, qbytes, &full[st]);
+  };
+  // a lane's two output dims of (slot, head): fp32 rows, or straight into the next projection's operand blocks
+  auto store_out = [&](int s, int head, float x0, float x1) {
+    if (A.act_out) {
+      const int k = head * HD + 2 * lane;          // column of the projection's input
+      unsigned char* blk = A.act_out + (size_t)(k / kTcKC) * tc_block_bytes(A.act_npad);
+      *reinterpret_cast<uint32_t*>(blk + ((size_t)((k % kTcKC) >> 3) * (A.act_npad >> 3) + (s >> 3)) * 128 + (s & 7) * 16 + (k & 7) * 2) =
+          pack_bf16(x0, x1);
+    } else {
+      *reinterpret_cast<float2*>(A.out + ((size_t)s * H + head) * HD + 2 * lane) = make_float2(x0, x1);
+    }
   };
   __syncthreads();
   // cur: the chunk a warp works on; ahead: the chunk n_stages later (the one that refills cur's stage)
@@ -330,7 +344,7 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
           const int head = gk * grp + t;
           if (whole) {
-            *reinterpret_cast<float2*>(A.out + ((size_t)s * H + head) * HD + 2 * lane) = make_float2(v.x / l, v.y / l);
+            store_out(s, head, v.x / l, v.y / l);
           } else {
             const size_t pi = ((size_t)s * H + head) * A.max_splits + seg_first_split;
             *reinterpret_cast<float2*>(A.part_o + pi * HD + 2 * lane) = v;
@@ -366,7 +380,7 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 num.x = fmaf(f, x.x, num.x); num.y = fmaf(f, x.y, num.y);
                 den = fmaf(f, ml.y, den);
               }
-              *reinterpret_cast<float2*>(A.out + ((size_t)s * H + head) * HD + 2 * lane) = make_float2(num.x / den, num.y / den);
+              store_out(s, head, num.x / den, num.y / den);
             }
             if (lane == 0) A.tickets[s * Hkv + gk] = 0;
           }

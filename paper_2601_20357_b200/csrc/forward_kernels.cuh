@@ -291,9 +291,11 @@ __global__ void __launch_bounds__(kGemvThreads) k_gemv(GemvArgs A) {
 // Cache layout [R][L][Hkv][cap][hd].   grid (slots), block 128.
 // ------------------------------------------------------------------------------------------------
 template <typename T>
+// part != nullptr: the QKV projection is still ks split-K slabs [ks][slab], summed here in slab order.
 __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restrict__ slots, int H, int Hkv, int hd,
                               const float* __restrict__ rope_cos, const float* __restrict__ rope_sin,
-                              T* __restrict__ kc, T* __restrict__ vc, int layer, int L, int cap) {
+                              T* __restrict__ kc, T* __restrict__ vc, int layer, int L, int cap,
+                              const float* __restrict__ part = nullptr, int ks = 0, size_t slab = 0) {
   pdl_trigger();
   pdl_wait();
   const int s = blockIdx.x;
@@ -301,13 +303,26 @@ __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restric
   if (!sd.active) return;
   const int half = hd >> 1;
   float* row = qkv + (long long)s * (H + 2 * Hkv) * hd;
+  const float* prow = part ? part + (long long)s * (H + 2 * Hkv) * hd : nullptr;
+  auto value = [&](int col) {
+    if (!prow) return row[col];
+    float v = 0.0f;
+    int k = 0;
+    for (; k + 4 <= ks; k += 4) {                  // four slabs in flight, summed in slab order
+      const float a0 = prow[(size_t)k * slab + col], a1 = prow[(size_t)(k + 1) * slab + col];
+      const float a2 = prow[(size_t)(k + 2) * slab + col], a3 = prow[(size_t)(k + 3) * slab + col];
+      v += a0; v += a1; v += a2; v += a3;
+    }
+    for (; k < ks; ++k) v += prow[(size_t)k * slab + col];
+    return v;
+  };
   const float* c = rope_cos + (long long)sd.pos * half;
   const float* sn = rope_sin + (long long)sd.pos * half;
   // q heads and k heads: (H + Hkv) * half pairs
   for (int idx = threadIdx.x; idx < (H + Hkv) * half; idx += blockDim.x) {
     const int head = idx / half, i = idx - head * half;
     float* p = row + head * hd;
-    const float x1 = p[i], x2 = p[i + half];
+    const float x1 = value(head * hd + i), x2 = value(head * hd + i + half);
     const float r1 = x1 * c[i] - x2 * sn[i];
     const float r2 = x2 * c[i] + x1 * sn[i];
     if (head < H) {
@@ -321,7 +336,7 @@ __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restric
   for (int idx = threadIdx.x; idx < Hkv * hd; idx += blockDim.x) {
     const int g = idx / hd, i = idx - g * hd;
     T* dst = vc + ((((long long)sd.row * L + layer) * Hkv + g) * cap + sd.pos) * hd;
-    Elem<T>::store(dst + i, row[(H + Hkv) * hd + idx]);
+    Elem<T>::store(dst + i, value((H + Hkv) * hd + idx));
   }
 }
 

@@ -21,7 +21,9 @@
 //   * four warp groups work on four units at a time (mma.sync m16n8k16, bf16 x bf16 -> fp32:
 //     16 weight rows x up to 8 slots).  The contraction is HBM-bound (<= 8 flop per weight byte);
 //     the tensor pipe only keeps the ALUs off the critical path;
-//   * an attention item issues all its loads (K, V, q) before it uses any;
+//   * attention: a CTA walks a contiguous range of cache chunks; its first chunk's K, V are requested
+//     between the two halves of the grid barrier; head size 64 runs on mma fragments loaded straight
+//     from global memory; the partial results of a cache are put together by the next phase's staging;
 //   * all cross-CTA data is read with ld.global.cg (L2) because L1 is not coherent across SMs;
 //   * loops are deliberately not unrolled except the few hot ones: every phase runs its code once,
 //     so unrolling buys nothing and only inflates the instruction footprint.
@@ -84,7 +86,7 @@ struct RoundArgs {
   float *qkv, *mid, *attn_out;          // [8][qkv_w], [8][F], [8][H*hd]
   float *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2]
   int max_splits;
-  int* tickets;                         // [8][Hkv]
+  int* tickets;                         // [8][Hkv] partial attention results of a (slot, KV head) pair in the current layer
   // ensemble
   float* logits_own;                    // [G][R][V]
   const float* logits_override;         // or null

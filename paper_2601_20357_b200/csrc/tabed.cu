@@ -211,8 +211,10 @@ void launch_gemv(tabed_handle* h, const GemvArgs& a, int epi, int ns) {
   else { if (f32) launch_gemv_ns<float, EPI_SWIGLU>(h, a, ns); else launch_gemv_ns<__nv_bfloat16, EPI_SWIGLU>(h, a, ns); }
 }
 
+// act_out != null (and *wrote_act given): the caller wants the output as the next projection's bf16 operand blocks;
+// the kernel that can do that sets *wrote_act, otherwise the fp32 rows in h->attn_out are the result.
 template <typename T, int HD>
-void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
+void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos, unsigned char* act_out, int act_npad, bool* wrote_act) {
   if constexpr (std::is_same<T, __nv_bfloat16>::value) {
     // bandwidth-oriented kernel: all K, V loads of a split in flight at once
     const int split_len = attn_bw_split_len(HD);
@@ -240,8 +242,10 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
           AttnTcArgs a;
           a.qkv = h->qkv; a.slots = h->slots; a.n_slots = n_slots; a.H = h->H; a.Hkv = h->Hkv; a.layer = layer; a.L = h->L;
           a.cap = h->cap; a.qkv_w = h->qkv_w; a.part_o = h->part_o; a.part_ml = h->part_ml; a.max_splits = h->max_splits;
+          a.act_out = act_out; a.act_npad = act_npad;
           a.tickets = h->attn_tickets; a.out = h->attn_out; a.scale = 1.0f / sqrtf((float)h->hd); a.err = h->err; a.n_stages = n_stages;
           TABED_LAUNCH_PDL(h, k_attn_tc_bf16, n_ctas, kAtcThreads, smem2, h->tm_k, h->tm_v, a);
+          if (wrote_act) *wrote_act = act_out != nullptr;
           return;
         }
       }
@@ -268,11 +272,13 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos) {
 }
 
 template <typename T>
-void launch_attention_t(tabed_handle* h, int layer, int n_slots, int max_pos) {
+void launch_attention_t(tabed_handle* h, int layer, int n_slots, int max_pos, unsigned char* act_out = nullptr, int act_npad = 0,
+                        bool* wrote_act = nullptr) {
+  if (wrote_act) *wrote_act = false;
   switch (h->hd) {
-    case 32: launch_attention_hd<T, 32>(h, layer, n_slots, max_pos); break;
-    case 64: launch_attention_hd<T, 64>(h, layer, n_slots, max_pos); break;
-    default: launch_attention_hd<T, 128>(h, layer, n_slots, max_pos); break;
+    case 32: launch_attention_hd<T, 32>(h, layer, n_slots, max_pos, act_out, act_npad, wrote_act); break;
+    case 64: launch_attention_hd<T, 64>(h, layer, n_slots, max_pos, act_out, act_npad, wrote_act); break;
+    default: launch_attention_hd<T, 128>(h, layer, n_slots, max_pos, act_out, act_npad, wrote_act); break;
   }
 }
 
@@ -593,20 +599,24 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
         prep_row(g, l == 0 ? nullptr : h->tc_pd, h->tck[KIND_DN].ks, S2 * d, 1, h->norm1[l], nullptr, h->slots);
         launch_gemm_tc(h, KIND_QKV, l, g.n, h->tc_pq + (size_t)g.s0 * h->qkv_w, S2 * h->qkv_w, h->slots + g.s0, h->qkv_w);
       }
-      const size_t elems = (size_t)n_slots * h->qkv_w;
-      TABED_LAUNCH_PDL(h, k_sum_slabs, (unsigned)((elems / 4 + 255) / 256), 256, 0, h->tc_pq, h->tck[KIND_QKV].ks, S2 * h->qkv_w, elems, h->qkv);
-      TABED_LAUNCH_PDL(h, k_rope_append<bf>, n_slots, 128, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos, h->rope_sin,
-                   reinterpret_cast<bf*>(h->kc), reinterpret_cast<bf*>(h->vc), l, h->L, h->cap);
+      // the split-K slabs of the projection are summed by the kernel that rotates q, k and appends k, v
+      TABED_LAUNCH_PDL(h, k_rope_append<bf>, n_slots, 512, 0, h->qkv, h->slots, h->H, h->Hkv, h->hd, h->rope_cos, h->rope_sin,
+                   reinterpret_cast<bf*>(h->kc), reinterpret_cast<bf*>(h->vc), l, h->L, h->cap,
+                   (const float*)h->tc_pq, h->tck[KIND_QKV].ks, S2 * h->qkv_w);
     }
+    bool attn_wrote_act = false;
     {
       ProfScope ps(h, TABED_PROF_ATTENTION);       // the attention kernel(s) alone on this path
-      launch_attention_t<bf>(h, l, n_slots, max_pos);
+      // one slot group: the attention kernel can leave its output as the O projection's operand blocks
+      const bool one = groups.size() == 1;
+      launch_attention_t<bf>(h, l, n_slots, max_pos, one ? h->tc_act : nullptr, one ? (groups[0].n + 15) / 16 * 16 : 0, &attn_wrote_act);
     }
     {
       ProfScope ps(h, TABED_PROF_OPROJ);
       for (const Grp& g : groups) {
         const int n_pad = (g.n + 15) / 16 * 16;
-        TABED_LAUNCH_PDL(h, k_prep_act, h->tck[KIND_O].k_chunks, 256, 0, h->attn_out + (size_t)g.s0 * HD, HD, g.n, n_pad, HD,
+        if (!attn_wrote_act)
+          TABED_LAUNCH_PDL(h, k_prep_act, h->tck[KIND_O].k_chunks, 256, 0, h->attn_out + (size_t)g.s0 * HD, HD, g.n, n_pad, HD,
                      (const float*)nullptr, (const bf*)nullptr, h->tc_act);
         launch_gemm_tc(h, KIND_O, l, g.n, h->tc_po + (size_t)g.s0 * d, S2 * d, h->slots + g.s0, d);
       }
