@@ -83,7 +83,7 @@ struct RoundArgs {
   // activations exchanged through L2
   float *xa, *x1;                       // [8][d] residual entering a layer / after its attention block
   float* ssq;                           // [d/16][8] sums of squares of the last residual, per 16-row tile
-  float *qkv, *mid, *attn_out;          // [8][qkv_w], [8][F], [8][H*hd]
+  float *qkv, *mid, *attn_out;          // [8][qkv_w], [8][F] (holds bf16 values here), [8][H*hd]
   float *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2]
   int max_splits;
   int* tickets;                         // [8][Hkv] partial attention results of a (slot, KV head) pair in the current layer
@@ -658,19 +658,19 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         int u = 0, sub = 0;
         if (has) { u = (int)(S.ulist[k - (unsigned)step * per_step] >> 10); sub = u % g.nsub; }
         if (kind == KIND_DN) {
-          // stage this round's chunks of the gated product: area of group w <- columns of its sub-unit
-          const int nvec = g.kchunk >> 2;
+          // stage this round's chunks of the gated product (left as bf16 by the gate/up epilogue): area of
+          // group w <- columns of its sub-unit, 16 bytes at a time
+          const int nvec = g.kchunk >> 3;
+          const __nv_bfloat16* midb = reinterpret_cast<const __nv_bfloat16*>(A.mid);
 #pragma unroll 1
           for (int idx = tid; idx < kWG * n_in * nvec; idx += kPT) {
             const int w2 = idx / (n_in * nvec), r2 = idx - w2 * (n_in * nvec);
-            const int s = r2 / nvec, j = (r2 - s * nvec) << 2;
+            const int s = r2 / nvec, j = (r2 - s * nvec) << 3;
             const unsigned kq = k0 + (unsigned)w2;
             if (kq < kb) {
               const int sq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10) % g.nsub;
-              const float4 v = __ldcg(reinterpret_cast<const float4*>(A.mid + (size_t)s * A.F + (size_t)sq * g.kchunk + j));
-              uint2 pk;
-              pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
-              *reinterpret_cast<uint2*>(act + w2 * area_elems + s * apitch + j) = pk;
+              const uint4 v = __ldcg(reinterpret_cast<const uint4*>(midb + (size_t)s * A.F + (size_t)sq * g.kchunk + j));
+              *reinterpret_cast<uint4*>(act + w2 * area_elems + s * apitch + j) = v;
             }
           }
           __syncthreads();
@@ -735,7 +735,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           if (kind == KIND_GU) {
             const float up = __shfl_down_sync(0xffffffffu, v, 8);
-            if (lead && r < 8 && slot_on) A.mid[(size_t)n * A.F + tile * 8 + r] = v / (1.0f + expf(-v)) * up;
+            if (lead && r < 8 && slot_on)            // bf16: the down projection rounds its input to bf16 anyway
+              reinterpret_cast<__nv_bfloat16*>(A.mid)[(size_t)n * A.F + tile * 8 + r] = __float2bfloat16_rn(v / (1.0f + expf(-v)) * up);
           } else if (kind == KIND_LM) {
             if (lead && slot_on && o < V) {
               A.logits_own[((size_t)step * R + n) * V + o] = v;
