@@ -519,34 +519,48 @@ struct PolicyArgs {
 __global__ void k_policy(PolicyArgs A) {
   pdl_trigger();
   pdl_wait();
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  // one warp per request: lane kd carries deviation index kd through the window (its running sum stays in a
+  // register, the loads of the positions are independent), then lane 0 applies the policy in its fixed order
+  const int b = blockIdx.x, lane = threadIdx.x;
   if (b >= A.B) return;
   const int a = A.n_accept[b];
   const int last = min(a, A.G - 1);
-  long long* run = A.running + (long long)b * kMaxDev;
-  for (int i = 0; i <= last; ++i) {
-    long long* d = A.dev + ((long long)b * A.G + i) * kMaxDev;
-    if (A.h > 0) {
-      long long* slot = A.ring + ((long long)b * A.h + A.ring_head[b]) * kMaxDev;
-      const bool full = A.ring_count[b] == A.h;
-      for (int kd = 0; kd < A.n_dev; ++kd) {
-        if (full) run[kd] -= slot[kd];
-        slot[kd] = d[kd];
-        run[kd] += d[kd];
+  long long r = 0;
+  {
+    long long* run = A.running + (long long)b * kMaxDev;
+    const bool on = lane < A.n_dev;
+    if (on) r = run[lane];
+    int head = A.h > 0 ? A.ring_head[b] : 0, count = A.h > 0 ? A.ring_count[b] : 0;
+    for (int i = 0; i <= last; ++i) {
+      const long long dv = on ? A.dev[((long long)b * A.G + i) * kMaxDev + lane] : 0;
+      if (A.h > 0) {
+        long long* slot = A.ring + ((long long)b * A.h + head) * kMaxDev;
+        const bool full = count == A.h;
+        if (on) {
+          if (full) r -= slot[lane];
+          slot[lane] = dv;
+        }
+        head = (head + 1) % A.h;
+        if (!full) count += 1;
       }
-      A.ring_head[b] = (A.ring_head[b] + 1) % A.h;
-      if (!full) A.ring_count[b] += 1;
-    } else {
-      for (int kd = 0; kd < A.n_dev; ++kd) run[kd] += d[kd];
+      r += dv;
     }
-    A.pushed[b] += 1;
+    if (on) run[lane] = r;
+    if (lane == 0) {
+      if (A.h > 0) { A.ring_head[b] = head; A.ring_count[b] = count; }
+      A.pushed[b] += last + 1;
+    }
+    for (int i = lane; i < A.G * kMaxDev; i += 32) A.dev[(long long)b * A.G * kMaxDev + i] = 0;
   }
-  for (int i = 0; i < A.G; ++i)
-    for (int kd = 0; kd < kMaxDev; ++kd) A.dev[((long long)b * A.G + i) * kMaxDev + kd] = 0;
+  long long run[kMaxDev];
+#pragma unroll
+  for (int kd = 0; kd < kMaxDev; ++kd) run[kd] = __shfl_sync(0xffffffffu, r, kd);
+  if (lane != 0) return;
+  const int pushed = A.pushed[b];
 
   float* w = A.w + (long long)b * A.m;
   const float fx_scale = A.tvd ? 4.547473508864641e-13f : kMassInv;     // 2^-41 or 2^-40
-  if (A.policy == 0 || A.pushed[b] == 0) {
+  if (A.policy == 0 || pushed == 0) {
     const float s = __fdiv_rn(1.0f, (float)A.m);
     for (int k = 0; k < A.m; ++k) w[k] = s;
   } else if (A.policy == 1) {

@@ -1031,7 +1031,7 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
   a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
   a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
   a.pending = h->pending; a.out_w = out_w; a.out_argmax = out_w_argmax;
-  TABED_LAUNCH_PDL(h, k_policy, (h->B + 127) / 128, 128, 0, a);
+  TABED_LAUNCH_PDL(h, k_policy, h->B, 32, 0, a);
   delete ps;
   if (h->has_drafter && h->round_has_forward) for (int& v : h->len_ub) v = std::min(v + h->G + 1, h->cap);
   h->phase = PH_IDLE;
