@@ -210,6 +210,23 @@ def run_prefill(args, wl):
             g.destroy()
             best = tms[0] if best is None or tms[0][1] < best[1] else best
         res[name] = {"tokens": best[0], "ms": best[1], "tokens_per_sec": best[0] / (best[1] / 1000.0)}
+    # the pooled image prefix (2 x 2 average of a 24 x 24 token grid in the drafter's embedding width)
+    g = gpu_setup(wl, device)
+    x = torch.randn((576, wl.drafter.d_model), device=device)
+    y = torch.empty((144, wl.drafter.d_model), device=device)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+    for i in range(23):
+        flush.zero_()
+        if i >= 3:
+            evs[i - 3][0].record()
+        g.pool_embeds(x, 24, 24, y)
+        if i >= 3:
+            evs[i - 3][1].record()
+    torch.cuda.synchronize(device)
+    pool_us = 1000.0 * float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    pool_bytes = (576 + 144) * wl.drafter.d_model * 4
+    g.destroy()
     c = wl.drafter
     layer_w = c.n_layers * (c.d_model * (c.n_heads + 2 * c.n_kv_heads) * (c.d_model // c.n_heads) + c.n_heads * (c.d_model // c.n_heads) * c.d_model
                             + 3 * c.d_model * c.d_ffn) * 2
@@ -217,6 +234,8 @@ def run_prefill(args, wl):
                       "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True, "data": "synthetic",
                       "config": {"workload": wl.name, "rows": wl.n_rows, "prompt_tokens": res["chunks_of_128_positions_tcgen05"]["tokens"]},
                       "ways": res, "layer_weight_bytes_per_chunk": int(layer_w),
+                      "pool_2x2": {"tokens_in": 576, "tokens_out": 144, "avg_us": pool_us, "bytes": int(pool_bytes),
+                                   "gbs": pool_bytes / (pool_us * 1e-6) / 1e9, "note": "k_pool2x2, 20 launches, L2 flushed before each"},
                       "note": "best of 3 fresh handles each, CUDA events around the feeding calls; a chunk reads the layers' "
                               "weights once for 128 positions"}), flush=True)
 

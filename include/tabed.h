@@ -144,6 +144,14 @@ int tabed_load_prefix_kv(tabed_handle* h, int32_t row, const void* k, const void
 int tabed_prefill_tokens(tabed_handle* h, int32_t row, const int32_t* tokens, int32_t len);
 int tabed_prefill_embeds(tabed_handle* h, int32_t row, const float* embeds, int32_t len);
 
+/* Pooled multimodal drafting input (Sec. 5, "Pooled Multimodal Drafting (P)"): the visual tokens of one image,
+ * in: float [grid_h * grid_w][d] on the device (row-major 2-D arrangement, 24 x 24 in the paper's default), are
+ * averaged over every 2 x 2 block of tokens, feature by feature: out float [(grid_h/2) * (grid_w/2)][d] on the
+ * device (576 -> 144 tokens), the correctly rounded mean of the four values.  The caller owns both buffers (they must
+ * not be the same); the result is a prefix for tabed_prefill_embeds once it is in the drafter's embedding space.  Runs on the handle's
+ * stream.  Errors: NULL_PTR, INVALID_ARG (a grid side odd or < 2, d < 1, in == out). */
+int tabed_pool_embeds(tabed_handle* h, const float* in, int32_t grid_h, int32_t grid_w, int32_t d, float* out);
+
 /* Set the verified-but-not-yet-consumed token(s) of every request: tok int32 [B][2],
  * cnt int32 [B] with values 1 or 2.  Normally only needed once, before the first round. */
 int tabed_set_pending(tabed_handle* h, const int32_t* tok, const int32_t* cnt);

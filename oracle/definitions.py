@@ -92,6 +92,21 @@ def policy_grid(p_window, qk_window, n_grid: int = 10):
     return j_star, cands[j_star], G
 
 
+def pool_image_tokens_2x2(x: np.ndarray, grid_h: int, grid_w: int) -> np.ndarray:
+    """Pooled multimodal drafting input (Sec. 5, "Pooled Multimodal Drafting (P)"): the visual tokens keep their 2-D
+    arrangement (row-major grid_h x grid_w, 24 x 24 = 576 in the paper's default) and every 2 x 2 block of tokens is
+    replaced by its average, feature by feature: 576 -> 144 tokens.  x: [grid_h * grid_w][d]; returns
+    [(grid_h / 2) * (grid_w / 2)][d] fp32 (the mean is taken in fp64 and rounded once)."""
+    if grid_h % 2 or grid_w % 2 or x.shape[0] != grid_h * grid_w:
+        raise ValueError("the token grid must have even sides and match the number of tokens")
+    g = np.asarray(x, dtype=np.float64).reshape(grid_h, grid_w, -1)
+    out = np.empty((grid_h // 2, grid_w // 2, g.shape[2]), dtype=np.float64)
+    for i in range(grid_h // 2):
+        for j in range(grid_w // 2):
+            out[i, j] = (g[2 * i, 2 * j] + g[2 * i, 2 * j + 1] + g[2 * i + 1, 2 * j] + g[2 * i + 1, 2 * j + 1]) / 4.0
+    return out.reshape(-1, g.shape[2]).astype(np.float32)
+
+
 def expected_speedup(block_efficiency: float, gamma: int, latency_ratio: float) -> float:
     """Eq. 1: tau / (gamma * T_q/T_p + 1)."""
     return block_efficiency / (gamma * latency_ratio + 1.0)

@@ -29,7 +29,7 @@ MAX_DEV = 11
 
 EXPORTS = [
     "tabed_init", "tabed_destroy", "tabed_strerror", "tabed_load_prefix_kv", "tabed_prefill_tokens",
-    "tabed_prefill_embeds", "tabed_set_pending", "tabed_decode_step", "tabed_ensemble_step",
+    "tabed_prefill_embeds", "tabed_pool_embeds", "tabed_set_pending", "tabed_decode_step", "tabed_ensemble_step",
     "tabed_draft_round", "tabed_draft_round_logits", "tabed_verify", "tabed_update_weights",
     "tabed_round_host", "tabed_debug_view", "tabed_debug_override_logits", "tabed_state_export", "tabed_state_import",
     "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end", "tabed_ensemble_step_static",
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
         L.tabed_load_prefix_kv.argtypes = [vp, i32, vp, vp, i32]
         L.tabed_prefill_tokens.argtypes = [vp, i32, vp, i32]
         L.tabed_prefill_embeds.argtypes = [vp, i32, vp, i32]
+        L.tabed_pool_embeds.argtypes = [vp, vp, i32, i32, i32, vp]
         L.tabed_set_pending.argtypes = [vp, vp, vp]
         L.tabed_decode_step.argtypes = [vp, vp, vp]
         L.tabed_ensemble_step.argtypes = [vp] + [vp] * 6
@@ -205,6 +206,11 @@ class Tabed:
     def prefill_embeds(self, row: int, embeds: torch.Tensor) -> None:
         _check(lib().tabed_prefill_embeds(self._h, row, _ptr(embeds, torch.float32, None, "embeds", self.device),
                                           embeds.shape[0]), "tabed_prefill_embeds")
+
+    def pool_embeds(self, tokens: torch.Tensor, grid_h: int, grid_w: int, out: torch.Tensor) -> None:
+        d = tokens.shape[1]
+        _check(lib().tabed_pool_embeds(self._h, _ptr(tokens, torch.float32, grid_h * grid_w * d, "tokens", self.device), grid_h, grid_w, d,
+                                       _ptr(out, torch.float32, (grid_h // 2) * (grid_w // 2) * d, "out", self.device)), "tabed_pool_embeds")
 
     def set_pending(self, tok: torch.Tensor, cnt: torch.Tensor) -> None:
         _check(lib().tabed_set_pending(self._h, _ptr(tok, torch.int32, self.B * 2, "tok", self.device),

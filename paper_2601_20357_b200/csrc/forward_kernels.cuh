@@ -116,6 +116,19 @@ __global__ void k_begin_step(StepArgs A, const T* __restrict__ embed) {
   }
 }
 
+// Pooled multimodal drafting input (Sec. 5, "Pooled Multimodal Drafting (P)"): visual tokens on a row-major
+// grid_h x grid_w grid, every 2 x 2 block replaced by its average.  The sum of four fp32 values is exact in
+// fp64, so the result is the correctly rounded mean.  grid (grid_h/2 * grid_w/2), any block size.
+__global__ void k_pool2x2(const float* __restrict__ in, int grid_w, int d, float* __restrict__ out) {
+  const int ow = grid_w >> 1;
+  const int oi = blockIdx.x / ow, oj = blockIdx.x - oi * ow;
+  const float* r0 = in + ((size_t)(2 * oi) * grid_w + 2 * oj) * d;
+  const float* r1 = r0 + (size_t)grid_w * d;
+  float* o = out + (size_t)blockIdx.x * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    o[i] = (float)((((double)r0[i] + (double)r0[d + i]) + ((double)r1[i] + (double)r1[d + i])) * 0.25);
+}
+
 // advance committed lengths by one (STEP_FREE: all rows; STEP_PREFILL handled on the host side
 // by a single add at the end)
 __global__ void k_advance_len(int* kv_len, int R, int row_only, int by) {

@@ -889,6 +889,14 @@ int tabed_prefill_embeds(tabed_handle* h, int32_t row, const float* embeds, int3
   return prefill_common(h, row, nullptr, embeds, len);
 }
 
+int tabed_pool_embeds(tabed_handle* h, const float* in, int32_t grid_h, int32_t grid_w, int32_t d, float* out) {
+  if (!h || !in || !out) return TABED_ERR_NULL_PTR;
+  if (grid_h < 2 || grid_w < 2 || (grid_h & 1) || (grid_w & 1) || d < 1 || in == out) return TABED_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  TABED_LAUNCH(h, k_pool2x2, (grid_h / 2) * (grid_w / 2), 256, 0, in, grid_w, d, out);
+  return check_cuda();
+}
+
 int tabed_set_pending(tabed_handle* h, const int32_t* tok, const int32_t* cnt) {
   if (!h || !tok || !cnt) return TABED_ERR_NULL_PTR;
   if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;

@@ -304,3 +304,23 @@ def test_ensemble_step_is_stateless_and_matches_checker():
         assert np.array_equal(qk[b].cpu().numpy(), qk_o) and np.array_equal(q[b].cpu().numpy(), q_o)
         assert int(y[b]) == X.draw(X.masses(q_o), u[b])
     g.destroy()
+
+
+# --------------------------------------------------------------------------------------------------
+# Pooled multimodal drafting input (Sec. 5): 2 x 2 average pooling of the visual tokens
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("gh,gw,d", [(24, 24, 768), (2, 2, 1), (6, 4, 130), (48, 2, 33)])
+def test_pool_embeds_bit_exact(gh, gw, d):
+    """The mean of four fp32 values rounded once: bitwise equal to the checker's."""
+    from oracle.definitions import pool_image_tokens_2x2
+    g = H.make_gpu(W.TINY)
+    rng = np.random.default_rng(100 + gh + d)
+    x = (rng.standard_normal((gh * gw, d)) * rng.choice([1e-3, 1.0, 1e3], size=(gh * gw, 1))).astype(np.float32)
+    out = torch.full(((gh // 2) * (gw // 2), d), float("nan"), device=H.DEV)
+    g.pool_embeds(H.t(x), gh, gw, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), pool_image_tokens_2x2(x, gh, gw))
+    with pytest.raises(TB.TabedError) as e:
+        g.pool_embeds(H.t(np.zeros((12, 4), np.float32)), 3, 4, torch.empty((2, 4), device=H.DEV))
+    assert e.value.code == -1
+    g.destroy()

@@ -277,3 +277,43 @@ def test_tiny_workload_free_run_smoke():
         acc.append(int(a[0]))
         assert abs(float(w.sum()) - 1) < 1e-6 and 0 <= a[0] <= wl.gamma and 0 <= z[0] < wl.drafter.vocab
     assert o.count[0] == sum(min(a, wl.gamma - 1) + 1 for a in acc)
+
+
+# --------------------------------------------------------------------------------------------------
+# Pooled multimodal drafting input (Sec. 5): 2 x 2 average pooling of the visual tokens' grid
+# --------------------------------------------------------------------------------------------------
+def test_pool_2x2_against_library_pooling():
+    """torch's avg_pool2d (an independent routine) on the same grid, features as channels."""
+    import torch
+    from oracle.definitions import pool_image_tokens_2x2
+    rng = np.random.default_rng(5)
+    for gh, gw, d in ((24, 24, 32), (2, 2, 5), (6, 4, 7)):
+        x = rng.standard_normal((gh * gw, d)).astype(np.float32)
+        got = pool_image_tokens_2x2(x, gh, gw)
+        ref = torch.nn.functional.avg_pool2d(torch.from_numpy(x).double().reshape(gh, gw, d).permute(2, 0, 1)[None], 2)[0]
+        ref = ref.permute(1, 2, 0).reshape(-1, d).numpy()
+        assert got.shape == ((gh // 2) * (gw // 2), d) and got.dtype == np.float32
+        assert np.max(np.abs(got.astype(np.float64) - ref)) <= 1e-7 * max(1.0, np.max(np.abs(ref)))
+
+
+def test_pool_2x2_closed_forms_and_token_count():
+    from oracle.definitions import pool_image_tokens_2x2
+    # the paper's default: 576 visual tokens -> 144
+    assert pool_image_tokens_2x2(np.zeros((576, 3), np.float32), 24, 24).shape == (144, 3)
+    # a constant grid stays constant; a ramp over rows/columns gives the block centres
+    assert np.array_equal(pool_image_tokens_2x2(np.full((16, 2), 1.25, np.float32), 4, 4), np.full((4, 2), 1.25, np.float32))
+    ii, jj = np.meshgrid(np.arange(4), np.arange(6), indexing="ij")
+    x = np.stack([ii.ravel(), jj.ravel(), (10 * ii + jj).ravel()], axis=1).astype(np.float32)
+    got = pool_image_tokens_2x2(x, 4, 6).reshape(2, 3, 3)
+    for i in range(2):
+        for j in range(3):
+            assert np.allclose(got[i, j], [2 * i + 0.5, 2 * j + 0.5, 10 * (2 * i + 0.5) + 2 * j + 0.5])
+    # a transposed grid (rows and columns swapped) must give a different result for a non-symmetric input:
+    # the pooling follows the row-major arrangement
+    assert not np.array_equal(pool_image_tokens_2x2(x, 4, 6), pool_image_tokens_2x2(x, 6, 4))
+    # one block only sees its own four tokens
+    x = np.zeros((16, 1), np.float32); x[5] = 4.0          # token (1, 1) -> block (0, 0)
+    assert np.array_equal(pool_image_tokens_2x2(x, 4, 4).ravel(), np.array([1, 0, 0, 0], np.float32))
+    for bad in ((3, 4), (4, 3)):
+        with pytest.raises(ValueError):
+            pool_image_tokens_2x2(np.zeros((12, 1), np.float32), *bad)
