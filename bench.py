@@ -411,12 +411,8 @@ def run_ours(args, wl):
     clocks = sampler.stop()
     launches = g.launch_count() - launches0
     per_round = np.array([s.elapsed_time(e) for s, e in ev])
-    dev_ms = float(per_round.sum())
-    if dist is not None:
-        tt = torch.tensor([dev_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        dev_ms = float(tt.item())
-    value = world * B * K / (dev_ms / 1000.0)
+    from paper_2601_20357_b200.replicas import whole_job
+    dev_ms, _, value = whole_job(float(per_round.sum()), B * K, dist, device)     # slowest rank's time, all ranks' rounds
 
     peak, peak_kind = read_peaks()
     cb = class_bytes(wl, kv_tokens_total, mean_accept)
