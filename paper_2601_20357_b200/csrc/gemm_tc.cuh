@@ -375,18 +375,4 @@ __global__ void k_swiglu_prep(const float* __restrict__ partial, int ks, size_t 
   *reinterpret_cast<uint4*>(dst + (size_t)kc * tc_block_bytes(n_pad) + ((size_t)k8 * (n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
 }
 
-// out[i] = sum over the k-split slabs (fixed order); grid over elems.
-__global__ void k_sum_slabs(const float* __restrict__ part, int ks, size_t slab, size_t elems, float* __restrict__ out) {
-  pdl_trigger();
-  pdl_wait();
-  const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (i >= elems) return;
-  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int k = 0; k < ks; ++k) {
-    const float4 a = *reinterpret_cast<const float4*>(part + (size_t)k * slab + i);
-    v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
-  }
-  *reinterpret_cast<float4*>(out + i) = v;
-}
-
 }  // namespace tabed
