@@ -482,6 +482,7 @@ def run_ours(args, wl):
         names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "gateup", "down")] + ["lm_head", "expsum", "mix"]
         mhz = float(clocks.get("sm_mhz") or 1965.0)
         with open(args.trace, "w") as f:
+            f.write("# made by: python " + " ".join(a if a != args.trace else "<this file>" for a in sys.argv) + "\n")
             f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA {args.trace_cta}): us from the previous grid barrier to this one,\n"
                     f"# then that CTA's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
                     f"# (attention phases: load+stage q/k/v, scores+softmax, PV+write, split merge, -, barrier)\n")
