@@ -197,25 +197,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   if (done_ok) {
     const int row = m_tile * kTcM + warp * 32 + lane;
     float* out = G.partial + (size_t)split * G.slab + row;
-#pragma unroll 1
-    for (int c0 = 0; c0 < G.n_pad; c0 += 16) {
-      uint32_t v[16];
-      if (n_ch > 0) {
-        const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
-        asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                       "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-                     : "r"(taddr));
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      } else {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = 0u;
-      }
+    // two loads of 16 columns in flight: the next one is requested before the current one is stored
+    auto ld16 = [&](uint32_t (&v)[16], int c0) {
+      const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+      asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                   : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                     "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                   : "r"(taddr));
+    };
+    auto st16 = [&](const uint32_t (&v)[16], int c0) {
       if (row < G.rows_valid) {
 #pragma unroll
         for (int j = 0; j < 16; ++j)
           if (c0 + j < G.n_slots) out[(size_t)(c0 + j) * G.rows_total] = __uint_as_float(v[j]);
       }
+    };
+    if (n_ch > 0) {
+      uint32_t va[16], vb[16];
+      ld16(va, 0);
+#pragma unroll 1
+      for (int c0 = 0; c0 < G.n_pad; c0 += 32) {
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        const bool more = c0 + 16 < G.n_pad;
+        if (more) ld16(vb, c0 + 16);
+        st16(va, c0);
+        if (more) {
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (c0 + 32 < G.n_pad) ld16(va, c0 + 32);
+          st16(vb, c0 + 16);
+        }
+      }
+    } else {
+      if (row < G.rows_valid)
+        for (int c = 0; c < G.n_slots; ++c) out[(size_t)c * G.rows_total] = 0.0f;
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
