@@ -25,7 +25,7 @@ DEV = torch.device("cuda", 0)
 # Probabilities are ~1/V, so the 1e-5 absolute bar on them is met with a wide margin either way.
 LOGIT_TOL = {"fp32": 2e-5, "bf16": 6e-2}
 LOGIT_MEAN_TOL = {"fp32": 2e-6, "bf16": 1e-2}
-PROB_TOL = 1e-5           # spec tolerance on probabilities
+PROB_TOL = 1e-5           # tolerance on probabilities (the bar the library is built to)
 
 
 def t(a: np.ndarray, dtype=None) -> torch.Tensor:
