@@ -315,10 +315,21 @@ __global__ void __launch_bounds__(256) k_prep_row(const PrepRowArgs P) {
     float f[8];
     const float4 a = *reinterpret_cast<const float4*>(xr + k), b = *reinterpret_cast<const float4*>(xr + k + 4);
     f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
-    for (int q = 0; q < P.ks; ++q) {
-      const float* pp = P.partial + (size_t)q * P.slab + (size_t)s * P.d + k;
-      const float4 c = *reinterpret_cast<const float4*>(pp), e = *reinterpret_cast<const float4*>(pp + 4);
-      f[0] += c.x; f[1] += c.y; f[2] += c.z; f[3] += c.w; f[4] += e.x; f[5] += e.y; f[6] += e.z; f[7] += e.w;
+    for (int q0 = 0; q0 < P.ks; q0 += 4) {          // four slabs in flight, added in slab order
+      float4 c[4], e[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool ok = q0 + j < P.ks;
+        const float* pp = P.partial + (size_t)(ok ? q0 + j : 0) * P.slab + (size_t)s * P.d + k;
+        c[j] = ok ? *reinterpret_cast<const float4*>(pp) : make_float4(0.f, 0.f, 0.f, 0.f);
+        e[j] = ok ? *reinterpret_cast<const float4*>(pp + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (q0 + j < P.ks) {
+          f[0] += c[j].x; f[1] += c[j].y; f[2] += c[j].z; f[3] += c[j].w; f[4] += e[j].x; f[5] += e[j].y; f[6] += e[j].z; f[7] += e[j].w;
+        }
+      }
     }
     if (P.write_back && P.ks > 0) {
       *reinterpret_cast<float4*>(xr + k) = make_float4(f[0], f[1], f[2], f[3]);
