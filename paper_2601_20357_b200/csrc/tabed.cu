@@ -513,7 +513,7 @@ int setup_tc(tabed_handle* h) {
     tabed_handle::TcKind& t = h->tck[k];
     t.rows = rows[k]; t.K = Ks[k];
     t.m_tiles = (t.rows + kTcM - 1) / kTcM; t.k_chunks = (t.K + kTcKC - 1) / kTcKC;
-    int ks = std::max(1, std::min(t.k_chunks, (n_sm + t.m_tiles - 1) / t.m_tiles));
+    int ks = std::max(1, std::min(std::min(t.k_chunks, 8), (n_sm + t.m_tiles - 1) / t.m_tiles));   // at most 8 slabs to sum
     if (k == KIND_LM) ks = 1;                       // logits are stored directly
     t.cps = (t.k_chunks + ks - 1) / ks;
     t.ks = (t.k_chunks + t.cps - 1) / t.cps;
