@@ -148,3 +148,20 @@ def test_chunked_prefill_matches_position_by_position_prefill(heads, kv_heads, d
         for rnd in range(2):
             H.lockstep_round(pair, rnd, override=True)
         pair.gpu.destroy()
+
+
+def test_tensor_path_forced_on_few_rows():
+    """The tensor-core kernels are set up for every bf16 drafter (they feed the prompts); forcing them for the
+    drafting steps of a 3-row workload (6 slots padded to 16 MMA columns, half of them inactive most rounds)
+    must follow the checker like the automatic choice does."""
+    wl = wl_attn(heads=4, kv_heads=2, d=256, cap=512, cid=131, sigma=0.05, gamma=3,
+                 prefixes=((("tokens", 150),), (("tokens", 40),), (("embeds", 20), ("tokens", 3))))
+    pair = H.build_pair(wl)
+    assert pair.gpu.current_path() == TB.PATH_PERSISTENT
+    pair.gpu.select_path(TB.PATH_TENSOR_CORE)
+    assert pair.gpu.current_path() == TB.PATH_TENSOR_CORE
+    for rnd in range(4):
+        H.lockstep_round(pair, rnd, override=True)
+    pair.gpu.select_path(TB.PATH_AUTO)
+    H.lockstep_round(pair, 4, override=True)         # and back on the persistent kernel, same caches
+    pair.gpu.destroy()
