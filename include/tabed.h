@@ -79,16 +79,19 @@ extern "C" {
                                                            (tabed_debug_trace): one record per grid barrier */
 
 /* How tabed_draft_round runs Algorithm 1 (tabed_select_path).  Results obey the same contract on
- * both paths: identical integer decisions for identical logits; logits agree within the forward
- * pass's floating-point tolerance (summation order differs). */
+ * every path: identical integer decisions for identical logits; logits agree within the forward
+ * pass's floating-point tolerance (summation order differs).  The selection also governs how
+ * tabed_prefill_* feed a prompt: with TABED_PATH_PER_OP one position at a time, otherwise (bf16
+ * drafter) in chunks of 128 positions through the tensor-core kernels. */
 #define TABED_PATH_AUTO        0   /* persistent kernel if the drafter qualifies, else tensor-core
-                                      projections if it qualifies, else per-operation                   */
+                                      projections with 16 or more rows, else per-operation               */
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
 #define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, 2*B*m <= 8
                                       slots, d_model <= 2048 and a multiple of 16, d_ffn a multiple of 16,
                                       (H/Hkv)*head_dim <= 512, <= 64 layers, kv_capacity <= 32768        */
 #define TABED_PATH_TENSOR_CORE 3   /* one kernel per operation with the projections as tcgen05 contractions
-                                      over all rows: bf16 drafter, B*m >= 16 rows, not persistent-eligible */
+                                      over all rows: any bf16 drafter with d_model, d_ffn, H*head_dim
+                                      multiples of 8 (the automatic choice from 16 rows on)               */
 
 typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
 
@@ -137,8 +140,8 @@ const char* tabed_strerror(int code);
  * sets the row's committed length to len.  Errors: INVALID_ARG (row / len out of range). */
 int tabed_load_prefix_kv(tabed_handle* h, int32_t row, const void* k, const void* v, int32_t len);
 
-/* Consume a prompt prefix into one row's cache by running the drafter over it position by
- * position (Algorithm 1's prefix x^(k)).  tokens: int32 [len]; embeds: float [len][d] (projected
+/* Consume a prompt prefix into one row's cache by running the drafter over it (Algorithm 1's
+ * prefix x^(k)): causal attention, position by position or in chunks of positions (see TABED_PATH_*).  tokens: int32 [len]; embeds: float [len][d] (projected
  * image tokens enter as embeddings).  Appends at the row's committed length.
  * Errors: INVALID_ARG, KV_OVERFLOW, BAD_STATE (handle without drafter). */
 int tabed_prefill_tokens(tabed_handle* h, int32_t row, const int32_t* tokens, int32_t len);
