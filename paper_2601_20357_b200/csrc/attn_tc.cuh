@@ -96,16 +96,21 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   extern __shared__ unsigned char atc_raw[];
   unsigned char* stage0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(atc_raw) + 1023) & ~(uintptr_t)1023);
   float* sq = reinterpret_cast<float*>(stage0 + (size_t)n_stages * 2 * kAtcTile);   // [n_stages][grp][HD] q beside its stage
-  float* so = sq + (size_t)n_stages * grp * HD;                                     // [n_stages][NW][grp][HD] states of a segment
-  float* sm = so + (size_t)n_stages * NW * grp * HD;                                // [n_stages][NW][grp] running maxima (base 2)
-  float* sl = sm + n_stages * NW * grp;                                             // [n_stages][NW][grp] running sums
+  // The warps' states of a segment go through a ring of n_stages + 1 buffers: a warp can be n_stages chunks (hence
+  // segments) ahead of the slowest one - the refill of a stage waits for all warps' reads, not for their segment
+  // ends - and must not touch the buffer that warp's segment is still being combined from.
+  const int n_segbuf = n_stages + 1;
+  float* so = sq + (size_t)n_stages * grp * HD;                                     // [n_segbuf][NW][grp][HD] states of a segment
+  float* sm = so + (size_t)n_segbuf * NW * grp * HD;                                // [n_segbuf][NW][grp] running maxima (base 2)
+  float* sl = sm + n_segbuf * NW * grp;                                             // [n_segbuf][NW][grp] running sums
   __shared__ uint64_t full[kAtcMaxStages];
   __shared__ int s_done[kAtcMaxStages];         // warps that have finished with a stage
-  __shared__ int s_seg[kAtcMaxStages];          // warps that have finished a segment (ring of n_stages segments)
+  __shared__ int s_seg[kAtcMaxStages + 1];      // warps that have finished a segment (ring of n_stages + 1 segments)
   __shared__ int s_pref[kAtcMaxSlots + 1];
   __shared__ int s_start;
   if (tid == 0) {
-    for (int i = 0; i < n_stages; ++i) { mbar_init(&full[i], 1); s_done[i] = 0; s_seg[i] = 0; }
+    for (int i = 0; i < n_stages; ++i) { mbar_init(&full[i], 1); s_done[i] = 0; }
+    for (int i = 0; i <= n_stages; ++i) s_seg[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   pdl_wait();                                   // the slot table, q and the appended K, V come from the kernels before
@@ -386,7 +391,7 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           }
         }
       }
-      if (++seg_buf == n_stages) seg_buf = 0;
+      if (++seg_buf == n_segbuf) seg_buf = 0;
     }
     if (have_next) advance(cur);
   }

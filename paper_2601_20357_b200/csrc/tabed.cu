@@ -229,14 +229,15 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos, u
         // fixed grid of streaming CTAs, contiguous chunk ranges, TMA-fed tensor-core arithmetic, in-kernel merge
         // two CTAs per SM with three stages each when the shared memory allows, else one CTA with a deeper ring
         // per stage: the K and V tiles, q of the cache, and one set of the eight warps' states
-        const size_t per_stage = 2 * (size_t)kAtcTile + ((size_t)grp * HD + (size_t)kAtcWarps * grp * (HD + 2)) * sizeof(float);
+        const size_t seg_state = (size_t)kAtcWarps * grp * (HD + 2) * sizeof(float);      // the eight warps' states of a segment
+        const size_t per_stage = 2 * (size_t)kAtcTile + (size_t)grp * HD * sizeof(float) + seg_state;
         int n_ctas = std::min(kAtcMaxCtas, 2 * h->n_sm), n_stages = 3;
-        if (1024 + n_stages * per_stage > 108u * 1024u) {
+        if (1024 + n_stages * per_stage + seg_state > 108u * 1024u) {
           n_ctas = std::min(kAtcMaxCtas, h->n_sm);
-          n_stages = (int)std::min<size_t>(kAtcMaxStages, (kAtcMaxDynSmem - 1024u) / per_stage);
+          n_stages = (int)std::min<size_t>(kAtcMaxStages, (kAtcMaxDynSmem - 1024u - seg_state) / per_stage);
         }
         if (n_stages >= 3) {
-          const size_t smem2 = 1024 + n_stages * per_stage;
+          const size_t smem2 = 1024 + n_stages * per_stage + seg_state;       // one more set of states than stages
           static bool attr2_set = false;
           if (!attr2_set) { cudaFuncSetAttribute(k_attn_tc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtcMaxDynSmem); attr2_set = true; }
           AttnTcArgs a;
