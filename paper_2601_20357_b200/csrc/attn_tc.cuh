@@ -14,10 +14,11 @@
 //     already, so products are exact to ~2^-17 relative and the sums are fp32;
 //   * a warp owns 16 positions of every chunk and carries its own running (max, sum, output) in
 //     registers across the chunks of a segment (the part of one cache that this CTA owns).  The
-//     warps run free of one another: each waits for a stage on its own, the LAST warp to finish
-//     with a stage refills it (TMA of the chunk n_stages ahead), and the last warp to finish a
-//     segment combines the eight states and writes the result, while the others are already in
-//     the next segment.  q of a cache rides along with the first tile of its segment (one more
+//     warps run free of one another: each waits for a stage's "full" mbarrier on its own and
+//     reports the stage read on its "empty" mbarrier (no answer needed); the warps take turns at
+//     waiting for all eight reports and refilling the stage (TMA of the chunk n_stages ahead);
+//     the last warp to finish a segment combines the eight states and writes the result, while
+//     the others are already in the next segment.  q of a cache rides along with the first tile of its segment (one more
 //     bulk copy onto the same mbarrier);
 //   * segments of a cache that spans several CTAs are combined by the warp that finishes last
 //     (ticket), in CTA order, reading the partial results from L2;
@@ -104,12 +105,12 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   float* sm = so + (size_t)n_segbuf * NW * grp * HD;                                // [n_segbuf][NW][grp] running maxima (base 2)
   float* sl = sm + n_segbuf * NW * grp;                                             // [n_segbuf][NW][grp] running sums
   __shared__ uint64_t full[kAtcMaxStages];
-  __shared__ int s_done[kAtcMaxStages];         // warps that have finished with a stage
+  __shared__ uint64_t empty[kAtcMaxStages];     // a stage's tiles have been read by all eight warps
   __shared__ int s_seg[kAtcMaxStages + 1];      // warps that have finished a segment (ring of n_stages + 1 segments)
   __shared__ int s_pref[kAtcMaxSlots + 1];
   __shared__ int s_start;
   if (tid == 0) {
-    for (int i = 0; i < n_stages; ++i) { mbar_init(&full[i], 1); s_done[i] = 0; }
+    for (int i = 0; i < n_stages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], NW); }
     for (int i = 0; i <= n_stages; ++i) s_seg[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -146,6 +147,14 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         w.nsplit = (w.pos + SPLIT) / SPLIT;
       }
     }
+  };
+  auto seek = [&](int g, Walk& w) {                 // the (slot, head, split) of global chunk g < T
+    int lo = 0, hi = n_slots;
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_pref[mid] <= g) lo = mid; else hi = mid; }
+    w.s = lo; w.row = slots[lo].row; w.pos = slots[lo].pos;
+    w.nsplit = (w.pos + SPLIT) / SPLIT;
+    const int rem = g - s_pref[lo];
+    w.gk = rem / w.nsplit; w.split = rem - w.gk * w.nsplit;
   };
   // one thread: the two TMA tiles of chunk `w` into stage `st`; q of the cache with the first chunk of a segment
   auto issue = [&](const Walk& w, int st, bool first) {
@@ -288,15 +297,23 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         mma_bf16(o[jn], pl, b0); mma_bf16(o[jn + 1], pl, b1);
       }
     }
-    // the last warp to finish with the stage refills it (the mma above have consumed every ldmatrix result)
+    // (the mma above have consumed every ldmatrix result)
+    // every warp reports the stage read (no answer needed); the warps take turns at waiting for all eight
+    // reports and refilling the stage with the chunk n_stages ahead
     __syncwarp();
-    if (lane == 0) {
-      if (atomicAdd(&s_done[st], 1) == NW - 1) {
-        s_done[st] = 0;
-        if (gi + n_stages < g_hi) issue(ahead, st, false);
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&empty[st])) : "memory");
+    if (((gi - g_lo) & (NW - 1)) == warp && gi + n_stages < g_hi) {
+      seek(gi + n_stages, ahead);
+      if (lane == 0) {
+        unsigned spins = 0;
+        while (!mbar_try_wait(&empty[st], phase)) {
+          if (++spins > (1u << 20)) { atomicOr(A.err, 16); break; }      // reported; the round's results are void
+          if (spins > 4096) __nanosleep(64);
+        }
+        issue(ahead, st, false);
       }
+      __syncwarp();
     }
-    if (gi + n_stages + 1 < g_hi) advance(ahead);
     if (++st == n_stages) { st = 0; phase ^= 1u; }
     if (seg_end) {
       // this warp's state -> shared memory; the last warp to get here combines the eight states
