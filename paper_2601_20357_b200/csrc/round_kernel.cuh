@@ -51,7 +51,7 @@ constexpr int kPPer = kChunk / kPT;      // vocabulary elements per thread and c
 constexpr int kPMaxD = 2048;             // d_model bound
 constexpr int kTraceRec = 8;             // words per record of the phase timeline
 constexpr int kPMaxL = 64;               // layers (their pointer table lives in shared memory)
-constexpr int kMaxUnits = 3072;          // units of one CTA in one decoder step
+constexpr int kMaxUnits = 1024;          // units of one CTA in one decoder step (config 3 needs 168)
 constexpr int kMaxPhase = 4 * kPMaxL + 1;
 
 enum { KIND_QKV = 0, KIND_O = 1, KIND_GU = 2, KIND_DN = 3, KIND_LM = 4 };
@@ -172,7 +172,7 @@ struct PShared {
   LayerW layers[kPMaxL];
   uint32_t ulist[kMaxUnits];            // this CTA's units of one decoder step, in consumption order
   uint16_t pstart[kMaxPhase + 1];       // first entry of every phase in ulist
-  float sc[kMaxGroup][kAttnSplitMax];
+  float sc[kMaxGroup][4];               // scores of the positions produced in this very phase (at most 2)
   alignas(16) float q[kMaxGroup][128];
   float kf[2][128], vf[2][128];
   float red[kPW][kPSlots];
@@ -186,7 +186,6 @@ struct PShared {
   float m_[kMaxGroup], l_[kMaxGroup];
   PSlot slot[kPSlots];
   int lm_src[kPSlots];
-  int segfirst[kPT];
   int att[8];                           // attention geometry of the step: T, g_lo, g_hi, then this CTA's first chunk (s, gk, split, nsplit, g0)
   int tok[kPSlots];
   int dead, flag, result, chunk;
