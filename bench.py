@@ -202,7 +202,7 @@ def run_prefill(args, wl):
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
     res = {}
-    for name, path in (("chunks_of_128_positions_tcgen05", None), ("one_position_at_a_time", TB.PATH_PER_OP)):
+    for name, path in (("chunks_of_256_positions_tcgen05", None), ("one_position_at_a_time", TB.PATH_PER_OP)):
         best = None
         for rep in range(3):
             tms = []
@@ -230,14 +230,14 @@ def run_prefill(args, wl):
     c = wl.drafter
     layer_w = c.n_layers * (c.d_model * (c.n_heads + 2 * c.n_kv_heads) * (c.d_model // c.n_heads) + c.n_heads * (c.d_model // c.n_heads) * c.d_model
                             + 3 * c.d_model * c.d_ffn) * 2
-    print(json.dumps({"metric": "prefill_tokens_per_sec", "value": res["chunks_of_128_positions_tcgen05"]["tokens_per_sec"],
+    print(json.dumps({"metric": "prefill_tokens_per_sec", "value": res["chunks_of_256_positions_tcgen05"]["tokens_per_sec"],
                       "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True, "data": "synthetic",
-                      "config": {"workload": wl.name, "rows": wl.n_rows, "prompt_tokens": res["chunks_of_128_positions_tcgen05"]["tokens"]},
+                      "config": {"workload": wl.name, "rows": wl.n_rows, "prompt_tokens": res["chunks_of_256_positions_tcgen05"]["tokens"]},
                       "ways": res, "layer_weight_bytes_per_chunk": int(layer_w),
                       "pool_2x2": {"tokens_in": 576, "tokens_out": 144, "avg_us": pool_us, "bytes": int(pool_bytes),
                                    "gbs": pool_bytes / (pool_us * 1e-6) / 1e9, "note": "k_pool2x2, 20 launches, L2 flushed before each"},
                       "note": "best of 3 fresh handles each, CUDA events around the feeding calls; a chunk reads the layers' "
-                              "weights once for 128 positions"}), flush=True)
+                              "weights once for 256 positions"}), flush=True)
 
 
 def gpu_setup(wl, device, prefill_path=None, prefill_times=None):

@@ -82,7 +82,7 @@ extern "C" {
  * every path: identical integer decisions for identical logits; logits agree within the forward
  * pass's floating-point tolerance (summation order differs).  The selection also governs how
  * tabed_prefill_* feed a prompt: with TABED_PATH_PER_OP one position at a time, otherwise (bf16
- * drafter) in chunks of 128 positions through the tensor-core kernels. */
+ * drafter) in chunks of 256 positions through the tensor-core kernels. */
 #define TABED_PATH_AUTO        0   /* persistent kernel if the drafter qualifies, else tensor-core
                                       projections with 16 or more rows, else per-operation               */
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */

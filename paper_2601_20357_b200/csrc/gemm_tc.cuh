@@ -30,7 +30,7 @@ constexpr int kTcM = 128;          // weight rows per tile (MMA M)
 constexpr int kTcKC = 128;         // input columns per pipeline stage
 constexpr int kTcStages = 3;        // pipeline stages (2 when more than 128 slots share the shared memory)
 constexpr int kTcThreads = 128;
-constexpr int kPrefillChunk = 128;        // positions of one row prefilled as slots of one weight pass
+constexpr int kPrefillChunk = 256;        // positions of one row prefilled as slots of one weight pass
 constexpr int kTcMaxN = 256;       // slots per launch (MMA N is their count rounded up to 16)
 __host__ __device__ inline int tc_stages(int n_pad) { return n_pad > 128 ? 2 : kTcStages; }
 

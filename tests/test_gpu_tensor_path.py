@@ -119,11 +119,11 @@ def test_attention_many_rows_several_chunks_each():
 
 
 # ------------------------------------------------------------------------------------------------
-# prompts fed in chunks of 128 positions through the tensor-core kernels
+# prompts fed in chunks of 256 positions through the tensor-core kernels
 # ------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("heads,kv_heads,d", [(4, 2, 256), (8, 2, 256)])
 def test_chunked_prefill_matches_position_by_position_prefill(heads, kv_heads, d):
-    """The same prompts (700 tokens = 5 full chunks + 60; 130 = one chunk + 2; 37 embeddings + 9 tokens) fed as
+    """The same prompts (700 tokens = 2 full chunks + 188; 130 and 37 embeddings + 9 tokens: short chunks) fed as
     chunks of positions (tcgen05 projections, every position attending up to itself) and one position at a
     time (per-operation kernels): both handles then follow the checker in lock step, and their first
     drafting step agrees within the bf16 bound.  Head sizes 64 (TMA attention) and 32 (split kernels)."""
