@@ -330,6 +330,8 @@ def run_ours(args, wl):
     g = gpu_setup(wl, device)
     if args.path == "per-op":
         g.select_path(TB.PATH_PER_OP)
+    elif args.path == "tensor-core":
+        g.select_path(TB.PATH_TENSOR_CORE)
     snap = g.state_export()
     alpha = torch.from_numpy(W.request_alpha(wl)).to(device)
     gen = torch.Generator(device=device)
@@ -557,7 +559,8 @@ def main():
     ap.add_argument("--prefill", action="store_true",
                     help="time the feeding of the workload's prompts instead of rounds: chunks of positions through the "
                          "tensor-core kernels (the library's choice for bf16) and one position at a time")
-    ap.add_argument("--path", default="auto", choices=["auto", "per-op"], help="drafting path (per-op forces one kernel per operation)")
+    ap.add_argument("--path", default="auto", choices=["auto", "per-op", "tensor-core"],
+                    help="drafting path (per-op forces one kernel per operation, tensor-core the tcgen05 projections)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -84,14 +84,15 @@ extern "C" {
  * tabed_prefill_* feed a prompt: with TABED_PATH_PER_OP one position at a time, otherwise (bf16
  * drafter) in chunks of 256 positions through the tensor-core kernels. */
 #define TABED_PATH_AUTO        0   /* persistent kernel if the drafter qualifies, else tensor-core
-                                      projections with 16 or more rows, else per-operation               */
+                                      projections if it qualifies, else per-operation                    */
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
 #define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, 2*B*m <= 8
                                       slots, d_model <= 2048 and a multiple of 16, d_ffn a multiple of 16,
                                       (H/Hkv)*head_dim <= 512, <= 64 layers, kv_capacity <= 32768        */
 #define TABED_PATH_TENSOR_CORE 3   /* one kernel per operation with the projections as tcgen05 contractions
                                       over all rows: any bf16 drafter with d_model, d_ffn, H*head_dim
-                                      multiples of 8 (the automatic choice from 16 rows on)               */
+                                      multiples of 8 (the automatic choice when the persistent kernel
+                                      does not take the shape, i.e. more than 4 rows)                     */
 
 typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
 

@@ -89,7 +89,7 @@ struct tabed_handle {
   unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false; int trace_cta = 0;
   // tensor-core projections for many rows (bf16 drafter, more than 8 slots per step)
   bool tc_ok = false;                        // tcgen05 projections are set up (prefill in chunks; drafting when tc_auto)
-  bool tc_auto = false;                      // ... and are the automatic choice for drafting (16 or more rows)
+  bool tc_auto = false;                      // ... and are the automatic choice for drafting (no persistent kernel)
   int slot_cap = 0;                          // slots the step buffers hold: 2R, or a prefill chunk if that is more
   struct TcKind { int rows, K, m_tiles, k_chunks, ks, cps; size_t bytes; };
   TcKind tck[5]{};                  // KIND_QKV, KIND_O, KIND_GU (gate|up rows), KIND_DN, KIND_LM
@@ -558,7 +558,7 @@ int setup_tc(tabed_handle* h) {
   }
   if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
   h->tc_ok = true;
-  h->tc_auto = !h->persist_ok && h->R >= 16;
+  h->tc_auto = !h->persist_ok;            // measured faster than one kernel per operation from 6 rows on (1.46 vs 2.20 ms)
   return TABED_OK;
 }
 
