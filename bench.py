@@ -407,6 +407,9 @@ def run_ours(args, wl):
     torch.cuda.synchronize(device)
     wall = time.perf_counter() - wall0
     sampler.mark_end()
+    dev_err = int(g.debug_view(TB.VIEW_ERROR_FLAG).cpu()[0])
+    if dev_err != 0:                        # a bounded wait ran out or a cache overflowed: the timing means nothing
+        raise RuntimeError(f"device-side error flag {dev_err} after the timed rounds")
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(device)
