@@ -1228,9 +1228,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll 1
         for (int c0 = 0; c0 < n_chunks; c0 += kPT) {
           const unsigned long long mine = (c0 + tid < n_chunks) ? __ldcg(cm + c0 + tid) : 0ull;
+          if (n_chunks <= kPT && tid < n_chunks) S.cm[tid] = mine;       // one trip to L2 serves the sum and the walk
           T += block_sum_u64_p(mine, S);
         }
-        if (n_chunks <= kPT && tid < n_chunks) S.cm[tid] = __ldcg(cm + tid);
         __syncthreads();
         if (tid == 0) {
           S.result = 0x7fffffff;
