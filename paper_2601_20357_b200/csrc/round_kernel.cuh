@@ -483,7 +483,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       }
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid == kPT - 32) {
+      // (a thread of the last warp, off the path of the staging that follows; the result is first read at the end of
+      // the QKV phase, several block-wide barriers later)
       // chunks of split_len positions of all (slot, KV head) caches in (slot, head, position) order; this CTA's
       // contiguous range of them and where it starts (the same for every layer of the step)
       const int sl = A.split_len;
@@ -506,7 +508,6 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       S.att[0] = T; S.att[1] = lo; S.att[2] = hi; S.att[3] = s; S.att[4] = gk; S.att[5] = nsplit ? rem - gk * nsplit : 0;
       S.att[6] = nsplit; S.att[7] = acc + gk * nsplit;
     }
-    __syncthreads();
 
 #pragma unroll 1
     for (int phase = 0; phase < n_phase; ++phase) {
@@ -833,11 +834,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       Walk cur{0, 0, 0, 0, 0}, nxt{0, 0, 0, 0, 0};
       int T = 0, g_lo = 0, g_hi = 0;
       if (kind == KIND_QKV) {
-        T = S.att[0]; g_lo = S.att[1]; g_hi = S.att[2];
-        cur.s = S.att[3]; cur.gk = S.att[4]; cur.split = S.att[5]; cur.nsplit = S.att[6]; cur.g0 = S.att[7];
         TSEC(4);
         bar_target += (unsigned)NC;
-        grid_barrier_arrive(bar);
+        grid_barrier_arrive(bar);                 // (its block-wide barrier also orders the geometry written at step start)
+        T = S.att[0]; g_lo = S.att[1]; g_hi = S.att[2];
+        cur.s = S.att[3]; cur.gk = S.att[4]; cur.split = S.att[5]; cur.nsplit = S.att[6]; cur.g0 = S.att[7];
         if (g_lo < g_hi) issue_loads(cur, kreg, vreg, true, true);
         alive = grid_barrier_wait(S, bar, bar_target, A.err);
         GRID_SYNC_TAIL();
