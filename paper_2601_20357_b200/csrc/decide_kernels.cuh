@@ -342,12 +342,13 @@ __global__ void k_accept(int B, int G, int V, const float* __restrict__ p, const
                          int n_chunks, int greedy, int* __restrict__ n_accept, int* __restrict__ out_n_accept) {
   pdl_trigger();
   pdl_wait();
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  // one warp per request, lane a decides position a (all positions' loads in flight together); the accepted
+  // prefix ends at the first lane that says no.  grid (B), block 32; G <= 32.
+  const int b = blockIdx.x, a = threadIdx.x;
   if (b >= B) return;
-  int a = 0;
-  for (; a < G; ++a) {
+  bool ok = true;
+  if (a < G) {
     const int y = tokens[b * G + a];
-    bool ok;
     if (greedy) {
       // argmax of p_a from the per-chunk bests
       float bv = -1.0f; int bi = 0x7fffffff;
@@ -360,10 +361,13 @@ __global__ void k_accept(int B, int G, int V, const float* __restrict__ p, const
       const float qy = q[(long long)b * q_req_stride + (long long)a * V + y];
       ok = (py >= qy) || (__fmul_rn(u_accept[b * G + a], qy) < py);
     }
-    if (!ok) break;
   }
-  n_accept[b] = a;
-  if (out_n_accept) out_n_accept[b] = a;
+  const unsigned no = ~__ballot_sync(0xffffffffu, ok);
+  const int n = no ? min(G, __ffs(no) - 1) : G;
+  if (a == 0) {
+    n_accept[b] = n;
+    if (out_n_accept) out_n_accept[b] = n;
+  }
 }
 
 // per-chunk argmax of every target row (greedy verification); grid (chunks, B*(G+1))

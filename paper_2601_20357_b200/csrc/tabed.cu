@@ -1011,7 +1011,7 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   TABED_LAUNCH_PDL(h, k_expsum, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
   TABED_LAUNCH_PDL(h, k_normalize, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum, h->p);
   if (greedy) TABED_LAUNCH(h, k_row_best, grid_rows, kDecThreads, 0, h->p, h->V, h->n_chunks, h->chunk_best);
-  TABED_LAUNCH_PDL(h, k_accept, (h->B + 127) / 128, 128, 0, h->B, h->G, h->V, h->p, h->q, GV, h->tokens, u_accept,
+  TABED_LAUNCH_PDL(h, k_accept, h->B, 32, 0, h->B, h->G, h->V, h->p, h->q, GV, h->tokens, u_accept,
                h->chunk_best, h->n_chunks, greedy, h->n_accept, out_n_accept);
   if (!greedy)
     TABED_LAUNCH_PDL(h, k_resid_chunks, grid_req, kDecThreads, 0, h->V, h->G, h->p, h->q, GV, h->n_accept, h->chunk_mass, h->n_chunks);
