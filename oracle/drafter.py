@@ -36,15 +36,38 @@ def round_bf16(x: np.ndarray) -> np.ndarray:
 
 
 class RowCache:
-    """K and V of one row: [L][Hkv][cap][hd] float64, `length` valid positions."""
+    """K and V of one row: [L][Hkv][positions][hd], `length` valid positions, at most `capacity`.
 
-    def __init__(self, n_layers: int, n_kv_heads: int, head_dim: int, capacity: int):
-        self.k = np.zeros((n_layers, n_kv_heads, capacity, head_dim))
-        self.v = np.zeros((n_layers, n_kv_heads, capacity, head_dim))
+    Storage only: the arrays hold the positions in use (they grow as the row grows) instead of the whole
+    capacity, and the values of a bf16 drafter - bf16 numbers, which float32 holds exactly - are kept
+    as float32; every product and sum that reads them is taken in float64 as before."""
+
+    def __init__(self, n_layers: int, n_kv_heads: int, head_dim: int, capacity: int, dtype=np.float64):
+        self.shape = (n_layers, n_kv_heads, head_dim)
+        self.capacity = capacity
+        self.dtype = dtype
+        self.k = np.zeros((n_layers, n_kv_heads, 0, head_dim), dtype)
+        self.v = np.zeros((n_layers, n_kv_heads, 0, head_dim), dtype)
         self.length = 0
+
+    def reserve(self, n: int) -> None:
+        """Make room for positions [0, n)."""
+        if n > self.capacity:
+            raise ValueError("row cache capacity exceeded")
+        have = self.k.shape[2]
+        if n <= have:
+            return
+        room = min(self.capacity, max(n, have + have // 2 + 16))
+        L, Hkv, hd = self.shape
+        for name in ("k", "v"):
+            old = getattr(self, name)
+            new = np.zeros((L, Hkv, room, hd), self.dtype)
+            new[:, :, :have] = old
+            setattr(self, name, new)
 
     def load(self, k: np.ndarray, v: np.ndarray) -> None:
         n = k.shape[2]
+        self.reserve(n)
         self.k[:, :, :n] = k
         self.v[:, :, :n] = v
         self.length = n
@@ -70,7 +93,7 @@ class OracleDrafter:
 
     def new_cache(self, capacity: int) -> RowCache:
         c = self.cfg
-        return RowCache(c.n_layers, c.n_kv_heads, c.head_dim, capacity)
+        return RowCache(c.n_layers, c.n_kv_heads, c.head_dim, capacity, np.float32 if self.bf16 else np.float64)
 
     def rmsnorm(self, x: np.ndarray, g: np.ndarray) -> np.ndarray:
         ms = np.mean(x * x, axis=-1, keepdims=True)
@@ -94,6 +117,7 @@ class OracleDrafter:
         H, Hkv, hd = c.n_heads, c.n_kv_heads, c.head_dim
         grp = H // Hkv
         p0 = cache.length
+        cache.reserve(p0 + T)
         pos = np.arange(p0, p0 + T)
         x = np.asarray(x, np.float64).copy()
         # causal mask: new position t sees cached [0, p0) and new [0, t]

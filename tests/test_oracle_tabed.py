@@ -142,6 +142,39 @@ def test_grid_policy_matches_definition_and_endpoints():
         assert abs(we[0] - e0) < 2e-5 and abs(we[10] - e1) < 2e-5 and we.min() <= min(we[0], we[10])
 
 
+@pytest.mark.parametrize("h", [0, 3])
+def test_tvd_softmax_policy_matches_definitions(h):
+    """Sec. 4.1 with the total-variation distance, App. B softmax(1/e) policy: the weights of the round
+    machine equal the fp64 definition applied to the fp64 TVD sums over the window.  The window error
+    is 1/2 sum |p - q| (a factor-of-two slip in its fixed-point scale doubles every e, halves every
+    1/e and moves the weights far outside the tolerance)."""
+    rng = np.random.default_rng(21)
+    G, V, m = 3, 400, 3
+    o = mk(m=m, B=1, gamma=G, h=h, V=V, distance=W.DIST_TVD)
+    hist = []
+    moved = 0.0
+    for rnd in range(5):
+        # drafters at different distances from the target so that the three errors are well separated
+        base = rng.standard_normal((G, 1, 1, V)).astype(F)
+        lg = (base + np.array([0.3, 0.9, 1.8], F)[None, None, :, None] * rng.standard_normal((G, 1, m, V))).astype(F)
+        o.draft_round_logits(lg, lat(rng, (1, G)))
+        tl = np.concatenate([base[:, :, 0, :], base[-1:, :, 0, :]], axis=0).transpose(1, 0, 2).astype(F)
+        a, _ = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+        for i in range(min(int(a[0]), G - 1) + 1):
+            hist.append([D.total_variation(o.p[0, i], o.qk[0, i, k]) for k in range(m)])
+        w, am = o.update_weights()
+        win = hist[-h:] if h > 0 else hist
+        e_def = np.sum(win, axis=0)
+        assert np.all(e_def > 0) and np.all(e_def <= len(win))                       # each TVD lies in [0, 1]
+        np.testing.assert_allclose(o.window_error(0), e_def, atol=1e-5)
+        np.testing.assert_allclose([float(X.fixed_to_float(int(t), True)) for t in o.running[0]], e_def, atol=1e-5)
+        w_def = D.policy_softmax_inv_err(e_def)
+        np.testing.assert_allclose(w[0], w_def, atol=2e-5)
+        assert am[0] == int(np.argmax(w_def))
+        moved = max(moved, float(np.max(np.abs(w_def - D.policy_softmax_inv_err(2.0 * e_def)))))
+    assert moved > 1e-2          # the test has the resolution to see a doubled error
+
+
 def test_window_h1_depends_only_on_last_verified_position():
     """App. B: h = 1 uses only the ground truth of the previous decoding step."""
     rng = np.random.default_rng(6)
