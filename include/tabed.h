@@ -18,6 +18,14 @@
  *   - The caller owns weights, inputs and outputs (weights must outlive the handle).  The library
  *     owns KV caches, the window ring, the per-round q / q^(k) / p buffers and all scratch, all
  *     allocated in tabed_init and released in tabed_destroy; no call in between allocates.
+ *   - Alignment: every drafter weight pointer (tabed_weights) must be 16-byte aligned (the projection
+ *     kernels read them with 128-bit loads; tabed_init rejects others with TABED_ERR_INVALID_ARG).
+ *     Other array arguments need only their element's natural alignment: 16-byte aligned pointers
+ *     take the 128-bit paths, others (e.g. offset views) the element-wise ones, with identical results.
+ *   - Device-side failures (a bounded wait that ran out, a cache position beyond kv_capacity, a
+ *     distribution without mass) set bits in an error word on the device.  tabed_round_host, which
+ *     synchronises anyway, returns the matching code (TABED_ERR_TIMEOUT / _KV_OVERFLOW / _NUMERIC) and
+ *     clears the word; after the asynchronous calls use tabed_last_device_error.
  *   - Layouts are row-major with the last index fastest.  B = n_requests, m = n_inputs,
  *     R = B*m rows (row = request*m + input), V = vocab, G = gamma.
  *   - Uniforms are caller-supplied floats on the lattice u = (k + 1/2) * 2^-23, 0 <= k < 2^23.
@@ -46,6 +54,7 @@ extern "C" {
 #define TABED_ERR_CUDA         -5
 #define TABED_ERR_TIMEOUT      -6
 #define TABED_ERR_UNSUPPORTED  -7
+#define TABED_ERR_NUMERIC      -8   /* a distribution had no mass to draw from (non-finite logits) */
 
 #define TABED_DTYPE_FP32 0      /* fp32 weights and KV cache, no intermediate rounding          */
 #define TABED_DTYPE_BF16 1      /* bf16 weights and KV cache, fp32 accumulation, matmul inputs
@@ -212,6 +221,25 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
                      int32_t* out_n_accept, int32_t* out_next_token, float* out_w,
                      int32_t* out_w_argmax);
 
+/* Synchronises the stream and returns the code of the device-side failures recorded since the last call
+ * (TABED_OK if none; TABED_ERR_TIMEOUT: a bounded wait of a kernel ran out, its results are void;
+ * TABED_ERR_KV_OVERFLOW: a row reached kv_capacity; TABED_ERR_NUMERIC: a distribution had no mass), then
+ * clears the record.  For use after the asynchronous calls, whose return codes only cover the host side. */
+int tabed_last_device_error(tabed_handle* h);
+
+/* Reads the rows' committed cache lengths and the pending-token counts back (synchronises the stream) so that
+ * the host-side overflow check of tabed_draft_round, which otherwise assumes that every round kept its
+ * maximum of gamma + 1 positions per row, works on exact lengths again.  tabed_round_host keeps them exact
+ * by itself.  Errors: BAD_STATE (mid-round), CUDA. */
+int tabed_sync_lengths(tabed_handle* h);
+
+/* Test aid for the failure path of the device-side waits: launches ONE CTA that takes the persistent
+ * kernel's grid barrier with an arrival count nobody else completes, so that its bounded wait (about
+ * 2^21 polls, a fraction of a second) runs out, records the failure and returns by itself - the GPU keeps
+ * answering.  Returns what tabed_last_device_error then reports (TABED_ERR_TIMEOUT).
+ * Errors: UNSUPPORTED (handle without the persistent kernel), CUDA. */
+int tabed_debug_barrier_timeout(tabed_handle* h);
+
 /* Choose the drafting path (TABED_PATH_*).  Errors: UNSUPPORTED (TABED_PATH_PERSISTENT on a drafter
  * that does not qualify; likewise TABED_PATH_TENSOR_CORE), BAD_STATE (mid-round), INVALID_ARG.
  * tabed_current_path returns the path the next tabed_draft_round will take: TABED_PATH_PER_OP,
@@ -257,12 +285,16 @@ int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* byte
  * step); make that first call before any stream capture begins.
  * All calls on one device share the one scratch array, which keeps the last call's contents (the
  * call clears what has to start at zero): two calls whose kernels overlap on the GPU, e.g. on
- * different streams, race.  Serialise them on one stream or with events. */
+ * different streams, race.  Serialise them on one stream or with events.
+ * A distribution without mass (non-finite logits) gives token 0 and is recorded in the scratch array;
+ * tabed_static_last_error(device, stream) synchronises that stream, returns TABED_ERR_NUMERIC if one was
+ * recorded since its last call (else TABED_OK) and clears the record; it allocates nothing either. */
 #define TABED_STATIC_MAX_ROWS   1024
 #define TABED_STATIC_MAX_CHUNKS 8192
 int tabed_ensemble_step_static(const float* logits, const float* w, const float* u, int32_t n_requests,
                                int32_t n_inputs, int32_t vocab, int32_t sample_mode, int32_t device,
                                void* stream, int32_t* y, float* q, float* qk);
+int tabed_static_last_error(int32_t device, void* stream);
 
 /* Stand-alone run of the tensor-core projection used for many shared-weight rows (Sec. 4.1 "batched
  * inference": all rows share the parameters, so a projection is one weights x rows contraction):

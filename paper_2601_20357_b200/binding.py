@@ -16,6 +16,7 @@ import torch
 from . import build as _build
 
 OK = 0
+ERR_INVALID_ARG, ERR_NULL_PTR, ERR_BAD_STATE, ERR_KV_OVERFLOW, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_NUMERIC = range(-1, -9, -1)
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR = 0, 1, 2
 DIST_KL, DIST_TVD = 0, 1
@@ -34,6 +35,7 @@ EXPORTS = [
     "tabed_round_host", "tabed_debug_view", "tabed_debug_override_logits", "tabed_state_export", "tabed_state_import",
     "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end", "tabed_ensemble_step_static",
     "tabed_select_path", "tabed_current_path", "tabed_debug_trace", "tabed_debug_gemm_tc",
+    "tabed_last_device_error", "tabed_sync_lengths", "tabed_debug_barrier_timeout", "tabed_static_last_error",
 ]
 
 
@@ -104,6 +106,10 @@ def lib() -> C.CDLL:
         L.tabed_current_path.argtypes = [vp]
         L.tabed_debug_trace.argtypes = [vp, i32]
         L.tabed_debug_gemm_tc.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, vp]
+        L.tabed_last_device_error.argtypes = [vp]
+        L.tabed_sync_lengths.argtypes = [vp]
+        L.tabed_debug_barrier_timeout.argtypes = [vp]
+        L.tabed_static_last_error.argtypes = [i32, vp]
         L.tabed_launch_count.argtypes = [vp]
         L.tabed_launch_count.restype = C.c_int64
         for name in EXPORTS:
@@ -320,6 +326,16 @@ class Tabed:
     def debug_trace(self, on: bool, cta: int = 0) -> None:
         _check(lib().tabed_debug_trace(self._h, 1 + int(cta) if on else 0), "tabed_debug_trace")
 
+    def last_device_error(self) -> int:
+        """Return code of the device-side failures recorded since the last call (0 if none); clears the record."""
+        return int(lib().tabed_last_device_error(self._h))
+
+    def sync_lengths(self) -> None:
+        _check(lib().tabed_sync_lengths(self._h), "tabed_sync_lengths")
+
+    def debug_barrier_timeout(self) -> int:
+        return int(lib().tabed_debug_barrier_timeout(self._h))
+
     def launch_count(self) -> int:
         return int(lib().tabed_launch_count(self._h))
 
@@ -342,6 +358,11 @@ def debug_gemm_tc(w: torch.Tensor, act: torch.Tensor, ks: int = 1) -> torch.Tens
     _check(lib().tabed_debug_gemm_tc(_ptr(w, torch.bfloat16, rows * K, "w", w.device), _ptr(act, torch.float32, n * K, "act", w.device),
                                      rows, K, n, ks, out.data_ptr(), w.device.index or 0, None), "tabed_debug_gemm_tc")
     return out
+
+
+def static_last_error(device: int = 0, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """tabed_static_last_error: code of a failure recorded by tabed_ensemble_step_static on `device` (0 if none)."""
+    return int(lib().tabed_static_last_error(device, stream.cuda_stream if stream is not None else None))
 
 
 def ensemble_step_static(logits: torch.Tensor, w: torch.Tensor, u: torch.Tensor, y: torch.Tensor, q: torch.Tensor,

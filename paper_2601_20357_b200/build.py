@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libtabed_b200.so")
 SOURCES = ["tabed.cu"]
-HEADERS = ["exact_math.cuh", "forward_kernels.cuh", "decide_kernels.cuh", "round_kernel.cuh", "gemm_tc.cuh", "attn_tc.cuh", os.path.join("..", "..", "include", "tabed.h")]
+HEADERS = ["exact_math.cuh", "forward_kernels.cuh", "decide_kernels.cuh", "round_kernel.cuh", "gemm_tc.cuh", "attn_tc.cuh", "request_kernels.cuh", os.path.join("..", "..", "include", "tabed.h")]
 
 
 def _stale() -> bool:

@@ -101,27 +101,6 @@ k_expsum(const float* __restrict__ logits, int V, long long row_stride,
   if (threadIdx.x == 0 && s) atomicAdd(rowsum + row, s);
 }
 
-// ---- softmax pass 3 (target rows): p = e / S ----------------------------------------------------
-__global__ void __launch_bounds__(kDecThreads)
-k_normalize(const float* __restrict__ logits, int V, long long row_stride,
-            const uint32_t* __restrict__ rowmax_enc, const unsigned long long* __restrict__ rowsum,
-            float* __restrict__ out) {
-  pdl_trigger();
-  pdl_wait();
-  const int row = blockIdx.y;
-  const float* x = logits + (long long)row * row_stride;
-  float* o = out + (long long)row * V;
-  const bool vec = ((V & 3) == 0) && ((row_stride & 3) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
-  const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
-  const float mx = ord_decode(rowmax_enc[row]);
-  const float S = norm_of(rowsum[row]);
-  float a[kPerThread];
-  load8(x, v0, V, vec, -INFINITY, a);
-#pragma unroll
-  for (int j = 0; j < kPerThread; ++j) a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx)), S);
-  store8(o, v0, V, (V & 3) == 0, a);
-}
-
 // ---- ensemble mix: q^(k) = e/S_k, q = sum_k w_k q^(k), chunk masses (or chunk argmax) -----------
 // grid (chunks, B).  logits [B][m][V] (row = b*m + k), w [B][m].
 // qk_out [b][..]: pitch qk_req_stride between requests, V between drafters; q_out pitch q_req_stride.
@@ -152,9 +131,12 @@ k_mix(const float* __restrict__ logits, int V, int m, const float* __restrict__ 
       const float t = __fmul_rn(wk, a[j]);
       acc[j] = (k == 0) ? t : __fadd_rn(acc[j], t);
     }
-    if (qk_out) store8(qk_out + (long long)b * qk_req_stride + (long long)k * V, v0, V, (V & 3) == 0 && (qk_req_stride & 3) == 0, a);
+    // (vector stores only to 16-byte aligned outputs: the caller's q / qk pointers may be offset views)
+    if (qk_out) store8(qk_out + (long long)b * qk_req_stride + (long long)k * V, v0, V,
+                       (V & 3) == 0 && (qk_req_stride & 3) == 0 && (reinterpret_cast<uintptr_t>(qk_out) & 15) == 0, a);
   }
-  if (q_out) store8(q_out + (long long)b * q_req_stride, v0, V, (V & 3) == 0 && (q_req_stride & 3) == 0, acc);
+  if (q_out) store8(q_out + (long long)b * q_req_stride, v0, V,
+                    (V & 3) == 0 && (q_req_stride & 3) == 0 && (reinterpret_cast<uintptr_t>(q_out) & 15) == 0, acc);
   if (!greedy) {
     unsigned long long s = 0;
 #pragma unroll
@@ -334,182 +316,12 @@ __global__ void __launch_bounds__(kDecThreads) k_select(SelectArgs A) {
   }
 }
 
-// ---- verification: sequential acceptance (Sec. 3 item 3) -----------------------------------------
-// one thread per request
-__global__ void k_accept(int B, int G, int V, const float* __restrict__ p, const float* __restrict__ q,
-                         long long q_req_stride, const int* __restrict__ tokens,
-                         const float* __restrict__ u_accept, const ChunkBest* __restrict__ p_best,
-                         int n_chunks, int greedy, int* __restrict__ n_accept, int* __restrict__ out_n_accept) {
-  pdl_trigger();
-  pdl_wait();
-  // one warp per request, lane a decides position a (all positions' loads in flight together); the accepted
-  // prefix ends at the first lane that says no.  grid (B), block 32; G <= 32.
-  const int b = blockIdx.x, a = threadIdx.x;
-  if (b >= B) return;
-  bool ok = true;
-  if (a < G) {
-    const int y = tokens[b * G + a];
-    if (greedy) {
-      // argmax of p_a from the per-chunk bests
-      float bv = -1.0f; int bi = 0x7fffffff;
-      const ChunkBest* cb = p_best + ((long long)b * (G + 1) + a) * n_chunks;
-      for (int c = 0; c < n_chunks; ++c)
-        if (cb[c].val > bv || (cb[c].val == bv && cb[c].idx < bi)) { bv = cb[c].val; bi = cb[c].idx; }
-      ok = (bi == y);
-    } else {
-      const float py = p[((long long)b * (G + 1) + a) * V + y];
-      const float qy = q[(long long)b * q_req_stride + (long long)a * V + y];
-      ok = (py >= qy) || (__fmul_rn(u_accept[b * G + a], qy) < py);
-    }
-  }
-  const unsigned no = ~__ballot_sync(0xffffffffu, ok);
-  const int n = no ? min(G, __ffs(no) - 1) : G;
-  if (a == 0) {
-    n_accept[b] = n;
-    if (out_n_accept) out_n_accept[b] = n;
-  }
-}
-
-// per-chunk argmax of every target row (greedy verification); grid (chunks, B*(G+1))
-__global__ void __launch_bounds__(kDecThreads)
-k_row_best(const float* __restrict__ p, int V, int n_chunks, ChunkBest* __restrict__ best) {
-  pdl_trigger();
-  pdl_wait();
-  const int row = blockIdx.y;
-  const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
-  float a[kPerThread];
-  load8(p + (long long)row * V, v0, V, (V & 3) == 0, -1.0f, a);
-  float bv = -1.0f; int bi = 0x7fffffff;
-#pragma unroll
-  for (int j = 0; j < kPerThread; ++j) if (v0 + j < V && a[j] > bv) { bv = a[j]; bi = v0 + j; }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-    if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-  }
-  __shared__ float shv[kDecThreads / 32];
-  __shared__ int shi[kDecThreads / 32];
-  if ((threadIdx.x & 31) == 0) { shv[threadIdx.x >> 5] = bv; shi[threadIdx.x >> 5] = bi; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int i = 1; i < kDecThreads / 32; ++i)
-      if (shv[i] > bv || (shv[i] == bv && shi[i] < bi)) { bv = shv[i]; bi = shi[i]; }
-    best[(long long)row * n_chunks + blockIdx.x] = ChunkBest{bv, bi};
-  }
-}
-
-// chunk masses of the replacement / bonus distribution; grid (chunks, B)
-__global__ void __launch_bounds__(kDecThreads)
-k_resid_chunks(int V, int G, const float* __restrict__ p, const float* __restrict__ q, long long q_req_stride,
-               const int* __restrict__ n_accept, unsigned long long* __restrict__ chunk_mass, int n_chunks) {
-  pdl_trigger();
-  pdl_wait();
-  const int b = blockIdx.y;
-  const int a = n_accept[b];
-  const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
-  const bool vec = (V & 3) == 0;
-  float pa[kPerThread], qa[kPerThread];
-  load8(p + ((long long)b * (G + 1) + a) * V, v0, V, vec, 0.0f, pa);
-  unsigned long long s = 0;
-  if (a < G) {
-    load8(q + (long long)b * q_req_stride + (long long)a * V, v0, V, vec && (q_req_stride & 3) == 0, 0.0f, qa);
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) if (v0 + j < V) s += mass_of(resid_val(pa[j], qa[j]));
-  } else {
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) if (v0 + j < V) s += mass_of(pa[j]);
-  }
-  __shared__ unsigned long long sh[kDecThreads / 32];
-  s = block_sum_u64(s, sh);
-  if (threadIdx.x == 0) chunk_mass[(long long)b * n_chunks + blockIdx.x] = s;
-}
-
-// ---- deviation of every drafter (or grid candidate) from the target (Sec. 4.1) -------------------
-// grid (chunks, G, B); positions i > min(a, G-1) exit.  dev[b][i][kd] (int64, zeroed beforehand)
-// accumulates trunc(term * 2^40): KL term p (ln p - ln max(q, FLT_MIN)); TVD term |p - q|.
-__global__ void __launch_bounds__(kDecThreads)
-k_deviation(int V, int G, int m, int n_dev, int grid_policy, int tvd,
-            const float* __restrict__ p, const float* __restrict__ qk, const int* __restrict__ n_accept,
-            long long* __restrict__ dev) {
-  pdl_trigger();
-  pdl_wait();
-  const int b = blockIdx.z, i = blockIdx.y;
-  const int a = n_accept[b];
-  if (i > min(a, G - 1)) return;
-  const int v0 = blockIdx.x * kChunk + threadIdx.x * kPerThread;
-  const bool vec = (V & 3) == 0;
-  float pv[kPerThread], lp[kPerThread];
-  load8(p + ((long long)b * (G + 1) + i) * V, v0, V, vec, 0.0f, pv);
-  if (!tvd) {
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
-  }
-  long long acc[kMaxDev];
-#pragma unroll
-  for (int kd = 0; kd < kMaxDev; ++kd) acc[kd] = 0;
-  const float* qbase = qk + ((long long)b * G + i) * m * V;
-  if (!grid_policy) {
-    for (int k = 0; k < m; ++k) {
-      float qv[kPerThread];
-      load8(qbase + (long long)k * V, v0, V, vec, 0.0f, qv);
-      long long s = 0;
-#pragma unroll
-      for (int j = 0; j < kPerThread; ++j) {
-        if (v0 + j >= V) continue;
-        float t;
-        if (tvd) t = fabsf(__fsub_rn(pv[j], qv[j]));
-        else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(qv[j], kFltMin)))) : 0.0f;
-        s += __float2ll_rz(__fmul_rn(t, kMassScale));
-      }
-#pragma unroll
-      for (int kd = 0; kd < kMaxInputs; ++kd) acc[kd] = (kd == k) ? s : acc[kd];
-    }
-  } else {
-    float q0[kPerThread], q1[kPerThread];
-    load8(qbase, v0, V, vec, 0.0f, q0);
-    load8(qbase + V, v0, V, vec, 0.0f, q1);
-#pragma unroll
-    for (int jc = 0; jc < kGridCand; ++jc) {
-      const float c1 = __fdiv_rn((float)jc, 10.0f);
-      const float c0 = __fsub_rn(1.0f, c1);
-      long long s = 0;
-#pragma unroll
-      for (int j = 0; j < kPerThread; ++j) {
-        if (v0 + j >= V) continue;
-        const float mix = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
-        float t;
-        if (tvd) t = fabsf(__fsub_rn(pv[j], mix));
-        else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(mix, kFltMin)))) : 0.0f;
-        s += __float2ll_rz(__fmul_rn(t, kMassScale));
-      }
-      acc[jc] = s;
-    }
-  }
-  __shared__ long long sh[kDecThreads / 32][kMaxDev];
-  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
-#pragma unroll
-  for (int kd = 0; kd < kMaxDev; ++kd) {
-    if (kd < n_dev) {
-      const long long t = warp_sum_i64(acc[kd]);
-      if (l == 0) sh[w][kd] = t;
-    }
-  }
-  __syncthreads();
-  if (threadIdx.x < n_dev) {
-    long long t = 0;
-    for (int i2 = 0; i2 < kDecThreads / 32; ++i2) t += sh[i2][threadIdx.x];
-    if (t) atomicAdd(reinterpret_cast<unsigned long long*>(dev + ((long long)b * G + i) * kMaxDev + threadIdx.x),
-                     (unsigned long long)t);
-  }
-}
-
 // ---- window push, policy, commit (Algorithm 1 steps 2-3; App. B) -----------------------------------
 struct PolicyArgs {
   int B, G, m, n_dev, h, policy, tvd;
   float tau;
   const int* n_accept; const int* next_token; const int* tokens;   // [B], [B], [B][G]
-  long long* dev;            // [B][G][kMaxDev], re-zeroed here
+  long long* dev;            // unused (the deviation sums travel through shared memory)
   long long* ring;           // [B][h][kMaxDev]
   int* ring_head; int* ring_count; long long* pushed;              // [B]
   long long* running;        // [B][kMaxDev]
@@ -519,91 +331,5 @@ struct PolicyArgs {
   int* pending;              // [B][3] {cnt, tok0, tok1}
   float* out_w; int* out_argmax;
 };
-
-__global__ void k_policy(PolicyArgs A) {
-  pdl_trigger();
-  pdl_wait();
-  // one warp per request: lane kd carries deviation index kd through the window (its running sum stays in a
-  // register, the loads of the positions are independent), then lane 0 applies the policy in its fixed order
-  const int b = blockIdx.x, lane = threadIdx.x;
-  if (b >= A.B) return;
-  const int a = A.n_accept[b];
-  const int last = min(a, A.G - 1);
-  long long r = 0;
-  {
-    long long* run = A.running + (long long)b * kMaxDev;
-    const bool on = lane < A.n_dev;
-    if (on) r = run[lane];
-    int head = A.h > 0 ? A.ring_head[b] : 0, count = A.h > 0 ? A.ring_count[b] : 0;
-    for (int i = 0; i <= last; ++i) {
-      const long long dv = on ? A.dev[((long long)b * A.G + i) * kMaxDev + lane] : 0;
-      if (A.h > 0) {
-        long long* slot = A.ring + ((long long)b * A.h + head) * kMaxDev;
-        const bool full = count == A.h;
-        if (on) {
-          if (full) r -= slot[lane];
-          slot[lane] = dv;
-        }
-        head = (head + 1) % A.h;
-        if (!full) count += 1;
-      }
-      r += dv;
-    }
-    if (on) run[lane] = r;
-    if (lane == 0) {
-      if (A.h > 0) { A.ring_head[b] = head; A.ring_count[b] = count; }
-      A.pushed[b] += last + 1;
-    }
-    for (int i = lane; i < A.G * kMaxDev; i += 32) A.dev[(long long)b * A.G * kMaxDev + i] = 0;
-  }
-  long long run[kMaxDev];
-#pragma unroll
-  for (int kd = 0; kd < kMaxDev; ++kd) run[kd] = __shfl_sync(0xffffffffu, r, kd);
-  if (lane != 0) return;
-  const int pushed = A.pushed[b];
-
-  float* w = A.w + (long long)b * A.m;
-  const float fx_scale = A.tvd ? 4.547473508864641e-13f : kMassInv;     // 2^-41 or 2^-40
-  if (A.policy == 0 || pushed == 0) {
-    const float s = __fdiv_rn(1.0f, (float)A.m);
-    for (int k = 0; k < A.m; ++k) w[k] = s;
-  } else if (A.policy == 1) {
-    int js = 0;
-    for (int j = 1; j < kGridCand; ++j) if (run[j] < run[js]) js = j;
-    A.grid_j[b] = js;
-    const float c1 = __fdiv_rn((float)js, 10.0f);
-    w[0] = __fsub_rn(1.0f, c1);
-    w[1] = c1;
-  } else {
-    float s[8], x[8];
-    float smax = -INFINITY;
-    for (int k = 0; k < A.m; ++k) {
-      const float e = __fmul_rn(__ll2float_rn(run[k]), fx_scale);
-      s[k] = __fdiv_rn(1.0f, fmaxf(e, __uint_as_float(0x322BCC77u)));   // 1e-8
-      smax = fmaxf(smax, s[k]);
-    }
-    float tot = 0.0f;
-    for (int k = 0; k < A.m; ++k) {
-      x[k] = xexp(__fdiv_rn(__fsub_rn(s[k], smax), A.tau));
-      tot = (k == 0) ? x[0] : __fadd_rn(tot, x[k]);
-    }
-    for (int k = 0; k < A.m; ++k) w[k] = __fdiv_rn(x[k], tot);
-  }
-  int am = 0;
-  for (int k = 1; k < A.m; ++k) if (w[k] > w[am]) am = k;
-  if (A.out_w) for (int k = 0; k < A.m; ++k) A.out_w[(long long)b * A.m + k] = w[k];
-  if (A.out_argmax) A.out_argmax[b] = am;
-
-  // commit: caches keep the pending token(s) and the accepted drafts that were fed
-  int* pend = A.pending + b * 3;
-  const int cnt = pend[0];
-  if (A.kv_len) {
-    const int keep = cnt + (a < A.G ? a : A.G - 1);
-    for (int k = 0; k < A.m; ++k) A.kv_len[b * A.m + k] += keep;
-  }
-  const int z = A.next_token[b];
-  if (a < A.G) { pend[0] = 1; pend[1] = z; pend[2] = 0; }
-  else { pend[0] = 2; pend[1] = A.tokens[b * A.G + A.G - 1]; pend[2] = z; }
-}
 
 }  // namespace tabed

@@ -1,0 +1,650 @@
+// One thread-block CLUSTER per request for the three vocabulary-wide stages of a round:
+//   k_ensemble_req : Algorithm 1 steps 6-7   (softmax of the m drafter rows, weighted average, draw)
+//   k_verify_req   : Sec. 3 item 3           (target softmax, sequential acceptance, residual / bonus draw)
+//   k_update_req   : Sec. 4.1, App. B        (deviation of every drafter over the verified positions, window
+//                                             push, policy, cache commit)
+// Each stage is ONE launch with no scratch in global memory and no spin-wait: the vocabulary is cut into
+// one contiguous slice per CTA of the cluster; every vocabulary-wide quantity (row maxima, integer mass
+// sums, per-slice masses, accept flags, deviation sums) is exchanged through distributed shared memory and
+// ordered by the hardware cluster barrier.  A row is read from HBM once; the later passes of the exact
+// softmax (maximum -> integer sum of masses -> quotient) re-read the CTA's own slice, which L1/L2 still hold.
+// Loads are 128-bit where the row pitch allows, reductions are warp shuffles.  All decision arithmetic is
+// the order-independent specification of exact_math.cuh, so the results do not depend on the cluster size.
+#pragma once
+#include <cooperative_groups.h>
+
+#include "decide_kernels.cuh"
+#include "exact_math.cuh"
+#include "forward_kernels.cuh"
+
+namespace tabed {
+
+namespace cg = cooperative_groups;
+
+constexpr int kReqThreads = 512;
+constexpr int kReqWarps = kReqThreads / 32;
+constexpr int kReqMaxCluster = 16;          // CTAs per cluster (16 needs the non-portable opt-in, 8 is portable)
+constexpr int kReqMaxRows = 17;             // rows of one request handled together: gamma + 1 <= 17, m <= 8
+constexpr int kReqStep = kReqThreads * 4;   // vocabulary elements one pass of the CTA covers
+
+struct ReqCtx {
+  unsigned CS, rank;
+  int tid, lane, warp;
+  int v_lo, v_hi;                           // this CTA's slice of the vocabulary
+};
+
+__device__ __forceinline__ void req_ld4(const float* __restrict__ row, int v, int v_hi, bool vec, float fill, float (&x)[4]) {
+  if (vec && v + 4 <= v_hi) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(row + v));
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) x[j] = (v + j < v_hi) ? __ldg(row + v + j) : fill;
+  }
+}
+// coherent variant for data this very kernel has written (p)
+__device__ __forceinline__ void req_ld4_rw(const float* row, int v, int v_hi, bool vec, float fill, float (&x)[4]) {
+  if (vec && v + 4 <= v_hi) {
+    const float4 a = *reinterpret_cast<const float4*>(row + v);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) x[j] = (v + j < v_hi) ? row[v + j] : fill;
+  }
+}
+__device__ __forceinline__ void req_st4(float* __restrict__ row, int v, int v_hi, bool vec, const float (&x)[4]) {
+  if (vec && v + 4 <= v_hi) {
+    *reinterpret_cast<float4*>(row + v) = make_float4(x[0], x[1], x[2], x[3]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) if (v + j < v_hi) row[v + j] = x[j];
+  }
+}
+__device__ __forceinline__ bool req_vec_ok(const void* base, long long pitch_elems) {
+  return (pitch_elems & 3) == 0 && (reinterpret_cast<uintptr_t>(base) & 15) == 0;
+}
+
+struct ReqBest { float val; int idx; };
+__device__ __forceinline__ void best_merge(ReqBest& a, const ReqBest& o) {
+  if (o.val > a.val || (o.val == a.val && o.idx < a.idx)) a = o;
+}
+
+// Shared state of the softmax passes: per-warp partials, then one entry per (CTA of the cluster, row).
+struct ReqShared {
+  float red_f[kReqWarps][kReqMaxRows];
+  unsigned long long red_u[kReqWarps][kReqMaxRows];
+  ReqBest red_b[kReqWarps][kReqMaxRows];
+  float all_max[kReqMaxCluster][kReqMaxRows];
+  unsigned long long all_sum[kReqMaxCluster][kReqMaxRows];
+  ReqBest all_best[kReqMaxCluster][kReqMaxRows];
+  unsigned long long all_mass[2][kReqMaxCluster];
+  unsigned long long scan[kReqWarps];
+  int ok[kReqMaxRows];
+  int result;
+};
+
+// Row maxima of `rows` rows (row i at base + i * pitch) over this CTA's slice, gathered over the cluster:
+// afterwards S.all_max[r][i] holds CTA r's maximum of row i in every CTA.  Four rows' loads are in flight together.
+__device__ __forceinline__ void req_row_maxima(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, const float* __restrict__ base,
+                                               long long pitch, int rows, bool vec) {
+#pragma unroll 1
+  for (int i0 = 0; i0 < rows; i0 += 4) {
+    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 2
+    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      float x[4][4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + j < rows) req_ld4(base + (long long)(i0 + j) * pitch, v, c.v_hi, vec, -INFINITY, x[j]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + j < rows) mx[j] = fmaxf(fmaxf(mx[j], fmaxf(x[j][0], x[j][1])), fmaxf(x[j][2], x[j][3]));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float w = warp_max_f32(mx[j]);
+      if (c.lane == 0 && i0 + j < rows) S.red_f[c.warp][i0 + j] = w;
+    }
+  }
+  __syncthreads();
+  if (c.tid < rows) {
+    float v = S.red_f[0][c.tid];
+#pragma unroll
+    for (int w = 1; w < kReqWarps; ++w) v = fmaxf(v, S.red_f[w][c.tid]);
+    for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.all_max[0][0], r)[c.rank * kReqMaxRows + c.tid] = v;
+  }
+  cluster.sync();
+}
+__device__ __forceinline__ float req_max_of(const ReqCtx& c, const ReqShared& S, int row) {
+  float v = S.all_max[0][row];
+  for (unsigned r = 1; r < c.CS; ++r) v = fmaxf(v, S.all_max[r][row]);
+  return v;
+}
+
+// Integer sums of the exp masses of the rows (softmax normalisers), gathered over the cluster.
+__device__ __forceinline__ void req_row_sums(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, const float* __restrict__ base,
+                                             long long pitch, int rows, bool vec) {
+#pragma unroll 1
+  for (int i0 = 0; i0 < rows; i0 += 2) {
+    unsigned long long sm[2] = {0ull, 0ull};
+    float mx[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) mx[j] = (i0 + j < rows) ? req_max_of(c, S, i0 + j) : 0.0f;
+#pragma unroll 2
+    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      float x[2][4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+        if (i0 + j < rows) req_ld4(base + (long long)(i0 + j) * pitch, v, c.v_hi, vec, -INFINITY, x[j]);
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        if (i0 + j >= rows) continue;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) if (v + e < c.v_hi) sm[j] += mass_of(xexp(__fsub_rn(x[j][e], mx[j])));
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const unsigned long long w = warp_sum_u64(sm[j]);
+      if (c.lane == 0 && i0 + j < rows) S.red_u[c.warp][i0 + j] = w;
+    }
+  }
+  __syncthreads();
+  if (c.tid < rows) {
+    unsigned long long v = 0;
+#pragma unroll
+    for (int w = 0; w < kReqWarps; ++w) v += S.red_u[w][c.tid];
+    for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.all_sum[0][0], r)[c.rank * kReqMaxRows + c.tid] = v;
+  }
+  cluster.sync();
+}
+__device__ __forceinline__ float req_norm_of(const ReqCtx& c, const ReqShared& S, int row) {
+  unsigned long long t = 0;
+  for (unsigned r = 0; r < c.CS; ++r) t += S.all_sum[r][row];
+  return norm_of(t);
+}
+
+// This CTA's mass of one distribution (block sum), gathered into S.all_mass[which][rank] of every CTA.
+// Ends with the cluster barrier.
+__device__ __forceinline__ void req_gather_mass(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, unsigned long long mine, int which) {
+  mine = warp_sum_u64(mine);
+  if (c.lane == 0) S.scan[c.warp] = mine;
+  __syncthreads();
+  if (c.tid == 0) {
+    unsigned long long t = 0;
+#pragma unroll
+    for (int w = 0; w < kReqWarps; ++w) t += S.scan[w];
+    for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.all_mass[0][0], r)[which * kReqMaxCluster + c.rank] = t;
+  }
+  cluster.sync();
+}
+
+// Inverse-CDF draw on the masses gathered in S.all_mass[which]: the CTA whose slice holds the threshold walks
+// it (block-wide prefix sums, 4 consecutive elements per thread) and returns the token through `found`
+// (true in every thread of that CTA only).  mass_at(v) gives the integer mass of element v of the slice.
+template <typename MassAt>
+__device__ __forceinline__ bool req_draw(const ReqCtx& c, ReqShared& S, int which, float u, MassAt mass_at, int* token, int* status) {
+  unsigned long long T = 0;
+  for (unsigned r = 0; r < c.CS; ++r) T += S.all_mass[which][r];
+  *status = 0;
+  if (T == 0ull) { *status = 1; return false; }               // no mass (caller decides: fall back or report)
+  unsigned long long thr = draw_threshold(u, T);
+  unsigned owner = 0;
+  for (; owner + 1 < c.CS; ++owner) {
+    const unsigned long long mr = S.all_mass[which][owner];
+    if (thr < mr) break;
+    thr -= mr;
+  }
+  if (owner != c.rank) return false;
+  if (c.tid == 0) S.result = 0x7fffffff;
+  __syncthreads();
+  unsigned long long carry = 0;
+#pragma unroll 1
+  for (int v0 = c.v_lo; v0 < c.v_hi; v0 += kReqStep) {
+    const int v = v0 + c.tid * 4;
+    unsigned long long mloc[4], tsum = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { mloc[j] = (v + j < c.v_hi) ? mass_at(v + j) : 0ull; tsum += mloc[j]; }
+    unsigned long long incl = tsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (c.lane >= o) incl += t;
+    }
+    if (c.lane == 31) S.scan[c.warp] = incl;
+    __syncthreads();
+    unsigned long long wpre = 0, ctot = 0;
+#pragma unroll
+    for (int i = 0; i < kReqWarps; ++i) { if (i < c.warp) wpre += S.scan[i]; ctot += S.scan[i]; }
+    unsigned long long run = carry + wpre + incl - tsum;
+    if (run <= thr) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        run += mloc[j];
+        if (run > thr && mloc[j] != 0ull) { atomicMin(&S.result, v + j); break; }
+      }
+    }
+    carry += ctot;
+    __syncthreads();
+    if (S.result != 0x7fffffff) break;
+  }
+  const int y = S.result;
+  if (y == 0x7fffffff) { *status = 2; *token = 0; }           // cannot happen for consistent masses; reported
+  else *token = y;
+  return true;
+}
+
+__device__ __forceinline__ ReqCtx req_ctx(cg::cluster_group& cluster, int V, int slice) {
+  ReqCtx c;
+  c.CS = cluster.num_blocks(); c.rank = cluster.block_rank();
+  c.tid = threadIdx.x; c.lane = c.tid & 31; c.warp = c.tid >> 5;
+  c.v_lo = min(V, (int)c.rank * slice); c.v_hi = min(V, c.v_lo + slice);
+  return c;
+}
+
+// per-thread best of a value over the slice -> block -> gathered over the cluster into S.all_best[r][row]
+__device__ __forceinline__ void req_gather_best(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, ReqBest mine, int row, bool last_row) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    ReqBest other;
+    other.val = __shfl_xor_sync(0xffffffffu, mine.val, o);
+    other.idx = __shfl_xor_sync(0xffffffffu, mine.idx, o);
+    best_merge(mine, other);
+  }
+  if (c.lane == 0) S.red_b[c.warp][row] = mine;
+  if (!last_row) return;
+  __syncthreads();
+  if (c.tid <= row) {
+    ReqBest v = S.red_b[0][c.tid];
+#pragma unroll
+    for (int w = 1; w < kReqWarps; ++w) best_merge(v, S.red_b[w][c.tid]);
+    for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.all_best[0][0], r)[c.rank * kReqMaxRows + c.tid] = v;
+  }
+}
+__device__ __forceinline__ int req_best_of(const ReqCtx& c, const ReqShared& S, int row) {
+  ReqBest v = S.all_best[0][row];
+  for (unsigned r = 1; r < c.CS; ++r) best_merge(v, S.all_best[r][row]);
+  return v.idx;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Algorithm 1 steps 6-7 for one request per cluster.  logits [B][m][V] (row = b*m + k).
+// ------------------------------------------------------------------------------------------------
+struct EnsembleArgs {
+  int V, m, greedy, slice;
+  const float* logits;
+  const float* w;                               // [B][m]
+  const float* u; int u_stride;                 // u[b * u_stride]
+  float* qk_out; long long qk_req_stride;       // optional [b][k][V]
+  float* q_out; long long q_req_stride;         // required (the draw re-reads it)
+  int* out0; int out0_stride;                   // y[b * out0_stride]
+  int* out1; int out1_stride;                   // optional second copy
+  int* err;
+};
+
+__global__ void __launch_bounds__(kReqThreads) k_ensemble_req(const EnsembleArgs A) {
+  pdl_trigger();
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ ReqShared S;
+  const ReqCtx c = req_ctx(cluster, A.V, A.slice);
+  const int b = blockIdx.x / c.CS, m = A.m, V = A.V;
+  pdl_wait();
+  const float* lg = A.logits + (long long)b * m * V;
+  const bool vec = req_vec_ok(A.logits, V);
+  req_row_maxima(cluster, c, S, lg, V, m, vec);
+  req_row_sums(cluster, c, S, lg, V, m, vec);
+  float mx[kMaxInputs], sn[kMaxInputs], wk[kMaxInputs];
+#pragma unroll
+  for (int k = 0; k < kMaxInputs; ++k) {
+    mx[k] = k < m ? req_max_of(c, S, k) : 0.0f;
+    sn[k] = k < m ? req_norm_of(c, S, k) : 1.0f;
+    wk[k] = k < m ? A.w[b * m + k] : 0.0f;
+  }
+  float* q_row = A.q_out + (long long)b * A.q_req_stride;
+  float* qk_b = A.qk_out ? A.qk_out + (long long)b * A.qk_req_stride : nullptr;
+  const bool vec_q = req_vec_ok(A.q_out, A.q_req_stride) && (V & 3) == 0;
+  const bool vec_qk = A.qk_out && req_vec_ok(A.qk_out, A.qk_req_stride) && (V & 3) == 0;
+  unsigned long long mass = 0;
+  ReqBest best{-1.0f, 0x7fffffff};
+#pragma unroll 1
+  for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+    float acc[4];
+    float nxt[4];
+    req_ld4(lg, v, c.v_hi, vec, -INFINITY, nxt);
+#pragma unroll
+    for (int k = 0; k < kMaxInputs; ++k) {
+      if (k >= m) break;
+      float a[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) a[j] = nxt[j];
+      if (k + 1 < m) req_ld4(lg + (long long)(k + 1) * V, v, c.v_hi, vec, -INFINITY, nxt);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx[k])), sn[k]);
+        const float t = __fmul_rn(wk[k], a[j]);
+        acc[j] = (k == 0) ? t : __fadd_rn(acc[j], t);
+      }
+      if (qk_b) req_st4(qk_b + (long long)k * V, v, c.v_hi, vec_qk, a);
+    }
+    req_st4(q_row, v, c.v_hi, vec_q, acc);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (v + j >= c.v_hi) continue;
+      if (A.greedy) { if (acc[j] > best.val) { best.val = acc[j]; best.idx = v + j; } }
+      else mass += mass_of(acc[j]);
+    }
+  }
+  int y = 0, status = 0;
+  bool mine = false;
+  if (A.greedy) {
+    req_gather_best(cluster, c, S, best, 0, true);
+    cluster.sync();
+    y = req_best_of(c, S, 0);
+    mine = c.rank == 0;
+  } else {
+    req_gather_mass(cluster, c, S, mass, 0);       // (its barriers also make this CTA's q slice visible to all its threads)
+    mine = req_draw(c, S, 0, A.u[b * A.u_stride], [&](int v) { return mass_of(q_row[v]); }, &y, &status);
+    if (status == 1 && c.rank == 0) { mine = true; y = 0; }
+  }
+  if (mine && c.tid == 0) {
+    if (status && A.err) atomicOr(A.err, status);
+    A.out0[b * A.out0_stride] = y;
+    if (A.out1) A.out1[b * A.out1_stride] = y;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sec. 3 item 3 for one request per cluster.
+// ------------------------------------------------------------------------------------------------
+struct VerifyArgs {
+  int V, G, greedy, slice;
+  const float* logits;                          // target [B][G+1][V]
+  const float* q; long long q_req_stride;       // ensembled [B][..][V], position pitch V
+  const int* tokens;                            // [B][G]
+  const float* u_accept;                        // [B][G]
+  const float* u_resid;                         // [B]
+  float* p;                                     // [B][G+1][V]
+  int *n_accept, *out_n_accept, *next_token, *out_next_token;
+  int* err;
+};
+
+__global__ void __launch_bounds__(kReqThreads) k_verify_req(const VerifyArgs A) {
+  pdl_trigger();
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ ReqShared S;
+  const ReqCtx c = req_ctx(cluster, A.V, A.slice);
+  const int b = blockIdx.x / c.CS, G = A.G, V = A.V, rows = G + 1;
+  pdl_wait();
+  const float* lg = A.logits + (long long)b * rows * V;
+  float* p_b = A.p + (long long)b * rows * V;
+  const float* q_b = A.q + (long long)b * A.q_req_stride;
+  const bool vec = req_vec_ok(A.logits, V), vec_p = (V & 3) == 0;
+  req_row_maxima(cluster, c, S, lg, V, rows, vec);
+  req_row_sums(cluster, c, S, lg, V, rows, vec);
+  // p = e / S for every row; in greedy mode also each row's argmax
+#pragma unroll 1
+  for (int i = 0; i < rows; ++i) {
+    const float mx = req_max_of(c, S, i), sn = req_norm_of(c, S, i);
+    ReqBest best{-1.0f, 0x7fffffff};
+#pragma unroll 2
+    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      float a[4];
+      req_ld4(lg + (long long)i * V, v, c.v_hi, vec, -INFINITY, a);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx)), sn);
+        if (A.greedy && v + j < c.v_hi && a[j] > best.val) { best.val = a[j]; best.idx = v + j; }
+      }
+      req_st4(p_b + (long long)i * V, v, c.v_hi, vec_p, a);
+    }
+    if (A.greedy) req_gather_best(cluster, c, S, best, i, i == rows - 1);
+  }
+  if (!A.greedy && c.tid < G) {
+    // position tid: the CTA whose slice holds the drafted token decides and tells every CTA
+    const int i = c.tid, y = A.tokens[b * G + i];
+    if (y >= c.v_lo && y < c.v_hi) {
+      const float py = __fdiv_rn(xexp(__fsub_rn(__ldg(lg + (long long)i * V + y), req_max_of(c, S, i))), req_norm_of(c, S, i));
+      const float qy = __ldg(q_b + (long long)i * V + y);
+      const int ok = (py >= qy) || (__fmul_rn(A.u_accept[b * G + i], qy) < py);
+      for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.ok[0], r)[i] = ok;
+    }
+  }
+  cluster.sync();
+  int a = 0;
+  if (A.greedy) { for (; a < G; ++a) if (req_best_of(c, S, a) != A.tokens[b * G + a]) break; }
+  else { for (; a < G; ++a) if (!S.ok[a]) break; }
+  if (c.rank == 0 && c.tid == 0) {
+    A.n_accept[b] = a;
+    if (A.out_n_accept) A.out_n_accept[b] = a;
+  }
+  int z = 0, status = 0;
+  bool mine = false;
+  if (A.greedy) {
+    z = req_best_of(c, S, a);
+    mine = c.rank == 0;
+  } else {
+    // replacement token from norm(max(0, p_a - q_a)) (from p_a if that has no mass); bonus token from p_G
+    const float* p_a = p_b + (long long)a * V;
+    const float* q_a = (a < G) ? q_b + (long long)a * V : nullptr;
+    const bool vec_qa = q_a && req_vec_ok(A.q, A.q_req_stride) && (V & 3) == 0;
+    unsigned long long mass = 0;
+#pragma unroll 2
+    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      float pa[4], qa[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+      req_ld4_rw(p_a, v, c.v_hi, vec_p, 0.0f, pa);
+      if (q_a) req_ld4(q_a, v, c.v_hi, vec_qa, 0.0f, qa);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) if (v + j < c.v_hi) mass += mass_of(q_a ? resid_val(pa[j], qa[j]) : pa[j]);
+    }
+    req_gather_mass(cluster, c, S, mass, 0);
+    const float u = A.u_resid[b];
+    mine = req_draw(c, S, 0, u, [&](int v) { return mass_of(q_a ? resid_val(p_a[v], __ldg(q_a + v)) : p_a[v]); }, &z, &status);
+    if (status == 1 && q_a) {
+      // residual without mass (p_a == q_a bitwise): draw from p_a itself.  Every CTA sees the same zero total.
+      mass = 0;
+#pragma unroll 2
+      for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+        float pa[4];
+        req_ld4_rw(p_a, v, c.v_hi, vec_p, 0.0f, pa);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) if (v + j < c.v_hi) mass += mass_of(pa[j]);
+      }
+      req_gather_mass(cluster, c, S, mass, 1);
+      mine = req_draw(c, S, 1, u, [&](int v) { return mass_of(p_a[v]); }, &z, &status);
+    }
+    if (status == 1 && c.rank == 0) { mine = true; z = 0; }
+  }
+  if (mine && c.tid == 0) {
+    if (status && A.err) atomicOr(A.err, status);
+    A.next_token[b] = z;
+    if (A.out_next_token) A.out_next_token[b] = z;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sec. 4.1 / App. B for one request per cluster: deviation sums of the verified positions, window push,
+// policy, cache commit.  The CTAs' fixed-point partial sums meet in CTA 0 of the cluster (integer sums:
+// order-free), whose first warp then runs the policy.
+// ------------------------------------------------------------------------------------------------
+struct UpdateArgs {
+  int V, slice, grid_policy;
+  const float* p;                 // [B][G+1][V]
+  const float* qk;                // [B][G][m][V]
+  PolicyArgs P;                   // P.dev unused
+};
+
+struct UpdShared {
+  long long red[kReqWarps][kMaxDev];
+  long long all_dev[kReqMaxCluster][kReqMaxRows - 1][kMaxDev];    // [CTA][position][deviation index], filled in CTA 0
+};
+
+__device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last, const UpdShared& U, unsigned CS);
+
+__global__ void __launch_bounds__(kReqThreads) k_update_req(const UpdateArgs A) {
+  pdl_trigger();
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ UpdShared U;
+  const ReqCtx c = req_ctx(cluster, A.V, A.slice);
+  const PolicyArgs& P = A.P;
+  const int b = blockIdx.x / c.CS, G = P.G, V = A.V, m = P.m, n_dev = P.n_dev, tvd = P.tvd;
+  pdl_wait();
+  const int a = P.n_accept[b];
+  const int last = min(a, G - 1);
+  const bool vec = (V & 3) == 0;
+  long long* mine_in_0 = cluster.map_shared_rank(&U.all_dev[0][0][0], 0) + (size_t)c.rank * (kReqMaxRows - 1) * kMaxDev;
+#pragma unroll 1
+  for (int i = 0; i <= last; ++i) {
+    const float* p_i = A.p + ((long long)b * (G + 1) + i) * V;
+    const float* qbase = A.qk + ((long long)b * G + i) * m * V;
+    long long acc[kMaxDev];
+#pragma unroll
+    for (int kd = 0; kd < kMaxDev; ++kd) acc[kd] = 0;
+#pragma unroll 1
+    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      float pv[4], lp[4];
+      req_ld4(p_i, v, c.v_hi, vec, 0.0f, pv);
+      if (!tvd) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
+      }
+      if (!A.grid_policy) {
+#pragma unroll
+        for (int k = 0; k < kMaxInputs; ++k) {
+          if (k >= m) break;
+          float qv[4];
+          req_ld4(qbase + (long long)k * V, v, c.v_hi, vec, 0.0f, qv);
+          long long s = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (v + j >= c.v_hi) continue;
+            float t;
+            if (tvd) t = fabsf(__fsub_rn(pv[j], qv[j]));
+            else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(qv[j], kFltMin)))) : 0.0f;
+            s += __float2ll_rz(__fmul_rn(t, kMassScale));
+          }
+          acc[k] += s;
+        }
+      } else {
+        float q0[4], q1[4];
+        req_ld4(qbase, v, c.v_hi, vec, 0.0f, q0);
+        req_ld4(qbase + V, v, c.v_hi, vec, 0.0f, q1);
+#pragma unroll
+        for (int jc = 0; jc < kGridCand; ++jc) {
+          const float c1 = __fdiv_rn((float)jc, 10.0f);
+          const float c0 = __fsub_rn(1.0f, c1);
+          long long s = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (v + j >= c.v_hi) continue;
+            const float mix = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
+            float t;
+            if (tvd) t = fabsf(__fsub_rn(pv[j], mix));
+            else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(mix, kFltMin)))) : 0.0f;
+            s += __float2ll_rz(__fmul_rn(t, kMassScale));
+          }
+          acc[jc] += s;
+        }
+      }
+    }
+    __syncthreads();                                  // the previous position's partials have been read
+#pragma unroll
+    for (int kd = 0; kd < kMaxDev; ++kd) {
+      if (kd < n_dev) {
+        const long long t = warp_sum_i64(acc[kd]);
+        if (c.lane == 0) U.red[c.warp][kd] = t;
+      }
+    }
+    __syncthreads();
+    if (c.tid < n_dev) {
+      long long t = 0;
+#pragma unroll
+      for (int w = 0; w < kReqWarps; ++w) t += U.red[w][c.tid];
+      mine_in_0[i * kMaxDev + c.tid] = t;
+    }
+  }
+  cluster.sync();
+  if (c.rank == 0 && c.warp == 0) policy_commit(P, b, c.lane, last, U, c.CS);
+}
+
+// One warp per request: lane kd carries deviation index kd through the window (its running sum stays in a
+// register), then lane 0 applies the policy in its fixed order and commits the caches and pending tokens.
+__device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last, const UpdShared& U, unsigned CS) {
+  const int a = A.n_accept[b];
+  long long r = 0;
+  {
+    long long* run = A.running + (long long)b * kMaxDev;
+    const bool on = lane < A.n_dev;
+    if (on) r = run[lane];
+    int head = A.h > 0 ? A.ring_head[b] : 0, count = A.h > 0 ? A.ring_count[b] : 0;
+    for (int i = 0; i <= last; ++i) {
+      long long dv = 0;
+      if (on) for (unsigned q = 0; q < CS; ++q) dv += U.all_dev[q][i][lane];
+      if (A.h > 0) {
+        long long* slot = A.ring + ((long long)b * A.h + head) * kMaxDev;
+        const bool full = count == A.h;
+        if (on) {
+          if (full) r -= slot[lane];
+          slot[lane] = dv;
+        }
+        head = (head + 1) % A.h;
+        if (!full) count += 1;
+      }
+      r += dv;
+    }
+    if (on) run[lane] = r;
+    if (lane == 0) {
+      if (A.h > 0) { A.ring_head[b] = head; A.ring_count[b] = count; }
+      A.pushed[b] += last + 1;
+    }
+  }
+  long long run[kMaxDev];
+#pragma unroll
+  for (int kd = 0; kd < kMaxDev; ++kd) run[kd] = __shfl_sync(0xffffffffu, r, kd);
+  if (lane != 0) return;
+  const long long pushed = A.pushed[b];
+
+  float* w = A.w + (long long)b * A.m;
+  const float fx_scale = A.tvd ? 4.547473508864641e-13f : kMassInv;     // 2^-41 or 2^-40
+  if (A.policy == 0 || pushed == 0) {
+    const float s = __fdiv_rn(1.0f, (float)A.m);
+    for (int k = 0; k < A.m; ++k) w[k] = s;
+  } else if (A.policy == 1) {
+    int js = 0;
+    for (int j = 1; j < kGridCand; ++j) if (run[j] < run[js]) js = j;
+    A.grid_j[b] = js;
+    const float c1 = __fdiv_rn((float)js, 10.0f);
+    w[0] = __fsub_rn(1.0f, c1);
+    w[1] = c1;
+  } else {
+    float s[8], x[8];
+    float smax = -INFINITY;
+    for (int k = 0; k < A.m; ++k) {
+      const float e = __fmul_rn(__ll2float_rn(run[k]), fx_scale);
+      s[k] = __fdiv_rn(1.0f, fmaxf(e, __uint_as_float(0x322BCC77u)));   // 1e-8
+      smax = fmaxf(smax, s[k]);
+    }
+    float tot = 0.0f;
+    for (int k = 0; k < A.m; ++k) {
+      x[k] = xexp(__fdiv_rn(__fsub_rn(s[k], smax), A.tau));
+      tot = (k == 0) ? x[0] : __fadd_rn(tot, x[k]);
+    }
+    for (int k = 0; k < A.m; ++k) w[k] = __fdiv_rn(x[k], tot);
+  }
+  int am = 0;
+  for (int k = 1; k < A.m; ++k) if (w[k] > w[am]) am = k;
+  if (A.out_w) for (int k = 0; k < A.m; ++k) A.out_w[(long long)b * A.m + k] = w[k];
+  if (A.out_argmax) A.out_argmax[b] = am;
+
+  // commit: caches keep the pending token(s) and the accepted drafts that were fed
+  int* pend = A.pending + b * 3;
+  const int cnt = pend[0];
+  if (A.kv_len) {
+    const int keep = cnt + (a < A.G ? a : A.G - 1);
+    for (int k = 0; k < A.m; ++k) A.kv_len[b * A.m + k] += keep;
+  }
+  const int z = A.next_token[b];
+  if (a < A.G) { pend[0] = 1; pend[1] = z; pend[2] = 0; }
+  else { pend[0] = 2; pend[1] = A.tokens[b * A.G + A.G - 1]; pend[2] = z; }
+}
+
+}  // namespace tabed

@@ -20,12 +20,15 @@
 #include "round_kernel.cuh"
 #include "gemm_tc.cuh"
 #include "attn_tc.cuh"
+#include "request_kernels.cuh"
 
 using namespace tabed;
 
 namespace {
 
 enum Phase { PH_IDLE = 0, PH_DRAFTED = 1, PH_VERIFIED = 2 };
+
+constexpr int kMaxDevices = 64;       // device ordinals the per-device tables below can hold
 
 struct DeviceGuard {
   int prev = -1; bool ok = true;
@@ -54,15 +57,15 @@ struct tabed_handle {
   float *rope_cos = nullptr, *rope_sin = nullptr;
   int *kv_len = nullptr, *pending = nullptr;
   float *w = nullptr;
-  long long *dev = nullptr, *ring = nullptr, *running = nullptr, *pushed = nullptr;
+  long long *ring = nullptr, *running = nullptr, *pushed = nullptr;
   int *ring_head = nullptr, *ring_count = nullptr, *grid_j = nullptr;
   SlotDesc* slots = nullptr; int* last_slot = nullptr;
   float *x = nullptr, *qkv = nullptr, *attn_out = nullptr, *mid = nullptr, *part_o = nullptr, *part_ml = nullptr;
   float *logits_own = nullptr, *qk = nullptr, *q = nullptr, *p = nullptr, *scratch_q = nullptr;
   int *tokens = nullptr, *n_accept = nullptr, *next_token = nullptr, *w_argmax = nullptr;
-  uint32_t* rowmax = nullptr; unsigned long long* rowsum = nullptr;
   unsigned long long* chunk_mass = nullptr; ChunkBest* chunk_best = nullptr;
   int* err = nullptr;
+  int cs_max = 8;                   // largest cluster the per-request kernels may use on this device (8 portable, 16 opt-in)
   // staging for the host-buffer entry point
   float *st_u_draft = nullptr, *st_u_accept = nullptr, *st_u_resid = nullptr, *st_target = nullptr;
   int* st_tokens = nullptr;
@@ -71,6 +74,8 @@ struct tabed_handle {
   bool round_has_forward = false;
   const float* logits_override = nullptr;   // tabed_debug_override_logits
   std::vector<int> len_ub;          // upper bound of every row's committed length
+  std::vector<int> pend_cnt;        // pending tokens of every request as the host last saw them
+  bool pend_known = false;          // ... and whether that is still what the device holds
   int64_t launches = 0;
   // persistent drafting-round kernel (bf16 drafters with at most kPSlots slots per step)
   bool persist_ok = false;
@@ -142,6 +147,32 @@ void launch_pdl(tabed_handle* h, void (*kern)(KArgs...), dim3 grid, dim3 block, 
 }
 #define TABED_LAUNCH_PDL(h, kern, grid, block, smem, ...) launch_pdl((h), (kern), dim3(grid), dim3(block), (smem), __VA_ARGS__)
 
+// One cluster of `cs` CTAs per request, as a programmatic dependent of the kernel before it in the stream.
+template <typename ArgT>
+void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_requests, int cs, const ArgT& args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(n_requests * cs)); cfg.blockDim = dim3(kReqThreads); cfg.dynamicSmemBytes = 0; cfg.stream = h->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 2;
+  cudaLaunchKernelEx(&cfg, kern, args);
+  h->launches++;
+}
+
+// CTAs per request cluster: as many as keep about two CTAs per SM busy over all requests, no finer than ~1024
+// vocabulary elements per CTA; slice = vocabulary elements per CTA (a multiple of 4, so that slices start on
+// 16-byte boundaries).
+int pick_cluster(const tabed_handle* h, int* slice) {
+  const int by_v = (h->V + 1023) / 1024, n_sm = h->n_sm > 0 ? h->n_sm : 148;
+  int cs = 1;
+  while (cs * 2 <= h->cs_max && (long long)h->B * cs * 2 <= 2ll * n_sm && cs < by_v) cs *= 2;
+  *slice = ((h->V + cs - 1) / cs + 3) & ~3;
+  return cs;
+}
+
 template <typename T>
 int dev_alloc(tabed_handle* h, T** out, size_t count, bool zero = true) {
   void* ptr = nullptr;
@@ -165,10 +196,10 @@ void launch_gemv_inst(tabed_handle* h, const GemvArgs& a, int n_chunks) {
   constexpr bool ROUND_IN = !std::is_same<T, float>::value;
   auto kern = k_gemv<T, NS, RPW, EPI, ROUND_IN>;
   const size_t smem = (size_t)NS * a.K * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {false};          // the attribute belongs to a (function, device) pair
+  if (!attr_set[h->cfg.device]) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    attr_set = true;
+    attr_set[h->cfg.device] = true;
   }
   const int n_out = (EPI == EPI_SWIGLU) ? a.rows0 : (a.rows0 + a.rows1 + a.rows2);
   const int n_groups = (n_out + RPW - 1) / RPW;
@@ -222,8 +253,8 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos, u
     const int grp = h->H / h->Hkv;
     const size_t smem = ((size_t)(kAttnBwThreads / 32) * grp * (HD + 2)) * sizeof(float);
     auto part = k_attn_split_bf16<HD>;
-    static bool attr_set = false;
-    if (!attr_set) { cudaFuncSetAttribute(part, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr_set = true; }
+    static bool attr_set[kMaxDevices] = {false};
+    if (!attr_set[h->cfg.device]) { cudaFuncSetAttribute(part, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024); attr_set[h->cfg.device] = true; }
     if constexpr (HD == kAtcHd) {
       if (h->atc_ok && n_slots <= kAtcMaxSlots) {
         // fixed grid of streaming CTAs, contiguous chunk ranges, TMA-fed tensor-core arithmetic, in-kernel merge
@@ -238,8 +269,8 @@ void launch_attention_hd(tabed_handle* h, int layer, int n_slots, int max_pos, u
         }
         if (n_stages >= 3) {
           const size_t smem2 = 1024 + n_stages * per_stage + seg_state;       // one more set of states than stages
-          static bool attr2_set = false;
-          if (!attr2_set) { cudaFuncSetAttribute(k_attn_tc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtcMaxDynSmem); attr2_set = true; }
+          static bool attr2_set[kMaxDevices] = {false};
+          if (!attr2_set[h->cfg.device]) { cudaFuncSetAttribute(k_attn_tc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAtcMaxDynSmem); attr2_set[h->cfg.device] = true; }
           AttnTcArgs a;
           a.qkv = h->qkv; a.slots = h->slots; a.n_slots = n_slots; a.H = h->H; a.Hkv = h->Hkv; a.layer = layer; a.L = h->L;
           a.cap = h->cap; a.qkv_w = h->qkv_w; a.part_o = h->part_o; a.part_ml = h->part_ml; a.max_splits = h->max_splits;
@@ -335,25 +366,18 @@ void run_step(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* log
   }
 }
 
-// Algorithm 1 steps 6-7 for all requests on logits [B][m][V].
+// Algorithm 1 steps 6-7 for all requests on logits [B][m][V]: one launch, one cluster per request.
 void run_ensemble(tabed_handle* h, const float* logits, const float* w, const float* u, int u_stride,
                   int* y0, int y0_stride, int* y1, int y1_stride, float* qk_out, long long qk_stride,
                   float* q_out, long long q_stride) {
-  const int greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
   ProfScope ps(h, TABED_PROF_ENSEMBLE);
-  cudaMemsetAsync(h->rowmax, 0, sizeof(uint32_t) * h->R, h->stream);
-  cudaMemsetAsync(h->rowsum, 0, sizeof(unsigned long long) * h->R, h->stream);
-  const dim3 grid_rows(h->n_chunks, h->R), grid_req(h->n_chunks, h->B);
-  TABED_LAUNCH_PDL(h, k_rowmax, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax);
-  TABED_LAUNCH_PDL(h, k_expsum, grid_rows, kDecThreads, 0, logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
-  TABED_LAUNCH_PDL(h, k_mix, grid_req, kDecThreads, 0, logits, h->V, h->m, w, h->rowmax, h->rowsum, qk_out, qk_stride,
-               q_out, q_stride, h->chunk_mass, h->chunk_best, h->n_chunks, greedy);
-  SelectArgs s{};
-  s.V = h->V; s.n_chunks = h->n_chunks; s.G = h->G; s.greedy = greedy;
-  s.q = q_out; s.q_req_stride = q_stride; s.u = u; s.u_stride = u_stride;
-  s.chunk_mass = h->chunk_mass; s.chunk_best = h->chunk_best;
-  s.out0 = y0; s.out0_stride = y0_stride; s.out1 = y1; s.out1_stride = y1_stride; s.err = h->err;
-  TABED_LAUNCH_PDL(h, k_select<0>, h->B, kDecThreads, 0, s);
+  EnsembleArgs a{};
+  const int cs = pick_cluster(h, &a.slice);
+  a.V = h->V; a.m = h->m; a.greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
+  a.logits = logits; a.w = w; a.u = u; a.u_stride = u_stride;
+  a.qk_out = qk_out; a.qk_req_stride = qk_stride; a.q_out = q_out; a.q_req_stride = q_stride;
+  a.out0 = y0; a.out0_stride = y0_stride; a.out1 = y1; a.out1_stride = y1_stride; a.err = h->err;
+  launch_request_clusters(h, k_ensemble_req, h->B, cs, a);
 }
 
 // ---- persistent drafting-round kernel: geometry and set-up -----------------------------------------
@@ -409,8 +433,10 @@ int setup_persistent(tabed_handle* h) {
   if (avail < u_bytes + (size_t)kWG * A.slot_bytes) return TABED_OK;      // a round needs kWG units in flight
   A.n_ring = (int)std::min<size_t>(kPRing, (avail - u_bytes) / A.slot_bytes);
   h->persist_smem = (size_t)A.n_ring * A.slot_bytes + u_bytes;
-  if (cudaFuncSetAttribute(k_draft_round<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess ||
-      cudaFuncSetAttribute(k_draft_round<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->persist_smem) != cudaSuccess)
+  // (the device's opt-in maximum, not this handle's own size: a later handle with a smaller ring must not lower it)
+  const int persist_attr = (int)((size_t)prop.sharedMemPerBlockOptin - fa.sharedSizeBytes);
+  if (cudaFuncSetAttribute(k_draft_round<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, persist_attr) != cudaSuccess ||
+      cudaFuncSetAttribute(k_draft_round<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, persist_attr) != cudaSuccess)
     return TABED_ERR_CUDA;
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_draft_round<true>, kPT, h->persist_smem) != cudaSuccess) return TABED_ERR_CUDA;
@@ -651,6 +677,27 @@ void run_step_tc(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* 
 
 int check_cuda() { return cudaGetLastError() == cudaSuccess ? TABED_OK : TABED_ERR_CUDA; }
 
+// Bits of the device-side error word -> return code (most severe first): a bounded wait that ran out, a cache
+// position beyond the capacity, a distribution without mass (non-finite logits) or a draw that found no token.
+int map_device_error(int bits) {
+  if (bits & (PERR_BARRIER | PERR_COPY)) return TABED_ERR_TIMEOUT;
+  if (bits & PERR_KV) return TABED_ERR_KV_OVERFLOW;
+  if (bits & 3) return TABED_ERR_NUMERIC;
+  return bits ? TABED_ERR_CUDA : TABED_OK;
+}
+
+// Copies the error word back, clears it on the device and synchronises the stream.
+int read_clear_device_error(int* err_dev, cudaStream_t st, int* bits_out) {
+  int bits = 0;
+  if (cudaMemcpyAsync(&bits, err_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemsetAsync(err_dev, 0, sizeof(int), st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return TABED_ERR_CUDA;
+  }
+  *bits_out = bits;
+  return TABED_OK;
+}
+
 // drafting steps outside the persistent kernel: tensor-core projections when chosen (or automatic with many rows)
 bool use_tc(const tabed_handle* h) {
   return h->tc_ok && (h->path_sel == TABED_PATH_TENSOR_CORE || (h->path_sel == TABED_PATH_AUTO && h->tc_auto));
@@ -677,6 +724,7 @@ const char* tabed_strerror(int code) {
     case TABED_ERR_CUDA: return "CUDA runtime error";
     case TABED_ERR_TIMEOUT: return "device-side wait ran out";
     case TABED_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TABED_ERR_NUMERIC: return "a distribution had no mass (non-finite logits)";
     default: return "unknown error code";
   }
 }
@@ -705,7 +753,16 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
       if (!wts->wq[l] || !wts->wk[l] || !wts->wv[l] || !wts->wo[l] || !wts->w_gate[l] || !wts->w_up[l] ||
           !wts->w_down[l] || !wts->norm1[l] || !wts->norm2[l])
         return TABED_ERR_NULL_PTR;
+    // the projection kernels read the drafter with 128-bit loads
+    auto misaligned = [](const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0; };
+    if (misaligned(wts->embed) || misaligned(wts->lm_head) || misaligned(wts->final_norm)) return TABED_ERR_INVALID_ARG;
+    for (int l = 0; l < c.n_layers; ++l)
+      if (misaligned(wts->wq[l]) || misaligned(wts->wk[l]) || misaligned(wts->wv[l]) || misaligned(wts->wo[l]) ||
+          misaligned(wts->w_gate[l]) || misaligned(wts->w_up[l]) || misaligned(wts->w_down[l]) || misaligned(wts->norm1[l]) ||
+          misaligned(wts->norm2[l]))
+        return TABED_ERR_INVALID_ARG;
   }
+  if (c.device >= kMaxDevices) return TABED_ERR_INVALID_ARG;
   int n_devices = 0;
   if (cudaGetDeviceCount(&n_devices) != cudaSuccess || c.device >= n_devices) { cudaGetLastError(); return TABED_ERR_CUDA; }
   DeviceGuard guard(c.device);
@@ -720,16 +777,36 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   h->ns = pick_ns(h->R);
   h->has_drafter = wts != nullptr;
   int rc = TABED_OK;
+  {
+    cudaDeviceProp pr;
+    if (cudaGetDeviceProperties(&pr, c.device) == cudaSuccess) h->n_sm = pr.multiProcessorCount;
+    // the per-request cluster kernels: clusters of 16 CTAs where the device can place one (non-portable size)
+    h->cs_max = 8;
+    if (cudaFuncSetAttribute(k_ensemble_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+        cudaFuncSetAttribute(k_verify_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+        cudaFuncSetAttribute(k_update_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(kReqMaxCluster); lc.blockDim = dim3(kReqThreads);
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = kReqMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at; lc.numAttrs = 1;
+      int n16 = 0;
+      bool ok = true;
+      for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_update_req})
+        ok = ok && cudaOccupancyMaxActiveClusters(&n16, fn, &lc) == cudaSuccess && n16 >= 1;
+      if (ok) h->cs_max = kReqMaxCluster;
+    }
+    cudaGetLastError();
+  }
   auto A = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count); };
   const size_t B = h->B, m = h->m, R = h->R, G = h->G, V = h->V;
   A(&h->w, B * m); A(&h->pending, B * 3);
-  A(&h->dev, B * G * kMaxDev); A(&h->ring, B * std::max(1, c.window_h) * kMaxDev); A(&h->running, B * kMaxDev);
+  A(&h->ring, B * std::max(1, c.window_h) * kMaxDev); A(&h->running, B * kMaxDev);
   A(&h->pushed, B); A(&h->ring_head, B); A(&h->ring_count, B); A(&h->grid_j, B);
   A(&h->qk, B * G * m * V); A(&h->q, B * G * V); A(&h->p, B * (G + 1) * V); A(&h->scratch_q, B * V);
   A(&h->tokens, B * G); A(&h->n_accept, B); A(&h->next_token, B); A(&h->w_argmax, B);
-  const size_t max_rows = std::max(R, B * (G + 1));
-  A(&h->rowmax, max_rows); A(&h->rowsum, max_rows);
-  A(&h->chunk_mass, B * h->n_chunks); A(&h->chunk_best, B * (G + 1) * h->n_chunks);
+  A(&h->chunk_mass, B * h->n_chunks); A(&h->chunk_best, B * h->n_chunks);
   A(&h->err, 1);
   A(&h->st_u_draft, B * G); A(&h->st_u_accept, B * G); A(&h->st_u_resid, B); A(&h->st_target, B * (G + 1) * V); A(&h->st_tokens, B * G);
   if (h->has_drafter) {
@@ -762,7 +839,6 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
     A(&h->part_o, SC * h->H * (size_t)h->max_splits * h->hd); A(&h->part_ml, SC * h->H * (size_t)h->max_splits * 2);
     A(&h->logits_own, G * R * V);
     A(&h->attn_tickets, SC * h->Hkv);
-    { cudaDeviceProp pr; if (cudaGetDeviceProperties(&pr, c.device) == cudaSuccess) h->n_sm = pr.multiProcessorCount; }
     if (c.dtype == TABED_DTYPE_BF16 && h->hd == kAtcHd && h->H / h->Hkv <= kMaxGroup && rc == TABED_OK) {
       // TMA descriptors of the caches seen as [all rows of all (row, layer, head)][64] bf16, tiles of 128 rows, 128-byte swizzle
       typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -819,6 +895,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
         cudaStreamSynchronize(h->stream) != cudaSuccess)
       rc = TABED_ERR_CUDA;
   }
+  h->pend_cnt.assign(B, 1); h->pend_known = true;
   if (rc != TABED_OK) { tabed_destroy(h); cudaGetLastError(); return rc; }
   *out = h;
   return TABED_OK;
@@ -915,6 +992,7 @@ int tabed_set_pending(tabed_handle* h, const int32_t* tok, const int32_t* cnt) {
   if (cudaMemcpyAsync(h->pending, pend.data(), pend.size() * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
       cudaStreamSynchronize(h->stream) != cudaSuccess)
     return TABED_ERR_CUDA;
+  h->pend_cnt = hc; h->pend_known = true;
   return TABED_OK;
 }
 
@@ -1000,27 +1078,16 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   if (!h || !target_logits || !u_accept || !u_resid || !out_n_accept || !out_next_token) return TABED_ERR_NULL_PTR;
   if (h->phase != PH_DRAFTED) return TABED_ERR_BAD_STATE;
   DeviceGuard guard(h->cfg.device);
-  const int greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
-  const int rows = h->B * (h->G + 1);
-  const long long GV = (long long)h->G * h->V;
   ProfScope ps(h, TABED_PROF_VERIFY);
-  cudaMemsetAsync(h->rowmax, 0, sizeof(uint32_t) * rows, h->stream);
-  cudaMemsetAsync(h->rowsum, 0, sizeof(unsigned long long) * rows, h->stream);
-  const dim3 grid_rows(h->n_chunks, rows), grid_req(h->n_chunks, h->B);
-  TABED_LAUNCH_PDL(h, k_rowmax, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax);
-  TABED_LAUNCH_PDL(h, k_expsum, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum);
-  TABED_LAUNCH_PDL(h, k_normalize, grid_rows, kDecThreads, 0, target_logits, h->V, (long long)h->V, h->rowmax, h->rowsum, h->p);
-  if (greedy) TABED_LAUNCH(h, k_row_best, grid_rows, kDecThreads, 0, h->p, h->V, h->n_chunks, h->chunk_best);
-  TABED_LAUNCH_PDL(h, k_accept, h->B, 32, 0, h->B, h->G, h->V, h->p, h->q, GV, h->tokens, u_accept,
-               h->chunk_best, h->n_chunks, greedy, h->n_accept, out_n_accept);
-  if (!greedy)
-    TABED_LAUNCH_PDL(h, k_resid_chunks, grid_req, kDecThreads, 0, h->V, h->G, h->p, h->q, GV, h->n_accept, h->chunk_mass, h->n_chunks);
-  SelectArgs s{};
-  s.V = h->V; s.n_chunks = h->n_chunks; s.G = h->G; s.greedy = greedy;
-  s.q = h->q; s.q_req_stride = GV; s.p = h->p; s.n_accept = h->n_accept; s.u = u_resid; s.u_stride = 1;
-  s.chunk_mass = h->chunk_mass; s.chunk_best = h->chunk_best;
-  s.out0 = h->next_token; s.out0_stride = 1; s.out1 = out_next_token; s.out1_stride = 1; s.err = h->err;
-  TABED_LAUNCH_PDL(h, k_select<1>, h->B, kDecThreads, 0, s);
+  VerifyArgs a{};
+  const int cs = pick_cluster(h, &a.slice);
+  a.V = h->V; a.G = h->G; a.greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
+  a.logits = target_logits; a.q = h->q; a.q_req_stride = (long long)h->G * h->V; a.tokens = h->tokens;
+  a.u_accept = u_accept; a.u_resid = u_resid; a.p = h->p;
+  a.n_accept = h->n_accept; a.out_n_accept = out_n_accept == h->n_accept ? nullptr : out_n_accept;
+  a.next_token = h->next_token; a.out_next_token = out_next_token == h->next_token ? nullptr : out_next_token;
+  a.err = h->err;
+  launch_request_clusters(h, k_verify_req, h->B, cs, a);
   h->phase = PH_VERIFIED;
   return check_cuda();
 }
@@ -1030,19 +1097,24 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
   if (h->phase != PH_VERIFIED) return TABED_ERR_BAD_STATE;
   DeviceGuard guard(h->cfg.device);
   const int tvd = h->cfg.distance == TABED_DIST_TVD;
-  ProfScope* ps = new ProfScope(h, TABED_PROF_UPDATE);
-  TABED_LAUNCH_PDL(h, k_deviation, dim3(h->n_chunks, h->G, h->B), kDecThreads, 0, h->V, h->G, h->m, h->n_dev,
-                 h->cfg.policy == TABED_POLICY_GRID_MT ? 1 : 0, tvd, h->p, h->qk, h->n_accept, h->dev);
-  PolicyArgs a{};
-  a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
-  a.tau = h->cfg.tau; a.n_accept = h->n_accept; a.next_token = h->next_token; a.tokens = h->tokens;
-  a.dev = h->dev; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
-  a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
-  a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
-  a.pending = h->pending; a.out_w = out_w; a.out_argmax = out_w_argmax;
-  TABED_LAUNCH_PDL(h, k_policy, h->B, 32, 0, a);
-  delete ps;
+  {
+    ProfScope ps(h, TABED_PROF_UPDATE);
+    UpdateArgs u{};
+    const int cs = pick_cluster(h, &u.slice);
+    u.V = h->V; u.grid_policy = h->cfg.policy == TABED_POLICY_GRID_MT ? 1 : 0; u.p = h->p; u.qk = h->qk;
+    PolicyArgs& a = u.P;
+    a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
+    a.tau = h->cfg.tau; a.n_accept = h->n_accept; a.next_token = h->next_token; a.tokens = h->tokens;
+    a.dev = nullptr; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
+    a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
+    a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
+    a.pending = h->pending; a.out_w = out_w; a.out_argmax = out_w_argmax;
+    launch_request_clusters(h, k_update_req, h->B, cs, u);
+  }
+  // the host has not seen the accept counts: the bound grows by the most a round can keep (tabed_round_host and
+  // tabed_sync_lengths replace it by the exact lengths)
   if (h->has_drafter && h->round_has_forward) for (int& v : h->len_ub) v = std::min(v + h->G + 1, h->cap);
+  h->pend_known = false;
   h->phase = PH_IDLE;
   return check_cuda();
 }
@@ -1061,6 +1133,8 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
       cudaMemcpyAsync(h->st_u_resid, u_resid, (size_t)h->B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(h->st_target, target_logits, (size_t)h->B * (h->G + 1) * h->V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return TABED_ERR_CUDA;
+  const std::vector<int> len_before = h->len_ub, cnt_before = h->pend_cnt;
+  const bool known_before = h->pend_known;
   // outputs land in library buffers first (tokens / n_accept / next_token / w / w_argmax)
   int rc = tabed_draft_round(h, h->st_u_draft, h->st_tokens, nullptr);
   if (rc != TABED_OK) return rc;
@@ -1072,9 +1146,72 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
       cudaMemcpyAsync(out_n_accept, h->n_accept, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaMemcpyAsync(out_next_token, h->next_token, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       (out_w && cudaMemcpyAsync(out_w, h->w, (size_t)h->B * h->m * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) ||
-      (out_w_argmax && cudaMemcpyAsync(out_w_argmax, h->w_argmax, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) ||
-      cudaStreamSynchronize(st) != cudaSuccess)
+      (out_w_argmax && cudaMemcpyAsync(out_w_argmax, h->w_argmax, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess))
     return TABED_ERR_CUDA;
+  // the device-side error word comes back with the results (this call synchronises anyway)
+  int bits = 0;
+  rc = read_clear_device_error(h->err, st, &bits);
+  if (rc != TABED_OK) return rc;
+  if (bits) { h->pend_known = false; return map_device_error(bits); }
+  if (known_before) {
+    // exact lengths: a row keeps its pending token(s) and the accepted drafts that were fed
+    for (int b = 0; b < h->B; ++b) {
+      const int a = out_n_accept[b], keep = cnt_before[b] + std::min(a, h->G - 1);
+      for (int k = 0; k < h->m; ++k) h->len_ub[b * h->m + k] = std::min(len_before[b * h->m + k] + keep, h->cap);
+      h->pend_cnt[b] = (a >= h->G) ? 2 : 1;
+    }
+    h->pend_known = true;
+  }
+  return TABED_OK;
+}
+
+namespace {
+// One CTA takes the grid barrier against a target that needs a second arrival: the bounded wait runs out,
+// the error bit is set and the kernel returns.
+__global__ void __launch_bounds__(kPT) k_barrier_probe(unsigned* bar, int* err) {
+  __shared__ PShared S;
+  if (threadIdx.x == 0) S.dead = 0;
+  __syncthreads();
+  const unsigned base = *bar;
+  grid_barrier(S, bar, base + 2u, err);
+}
+}  // namespace
+
+int tabed_debug_barrier_timeout(tabed_handle* h) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (!h->persist_ok) return TABED_ERR_UNSUPPORTED;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  DeviceGuard guard(h->cfg.device);
+  // (the counter of the launch after next: this launch's own counter is reset by the next persistent launch)
+  unsigned* bar = h->bar + (h->launches_persist & 1u);
+  k_barrier_probe<<<1, kPT, 0, h->stream>>>(bar, h->err);
+  h->launches++;
+  if (cudaMemsetAsync(bar, 0, sizeof(unsigned), h->stream) != cudaSuccess) { cudaGetLastError(); return TABED_ERR_CUDA; }
+  return tabed_last_device_error(h);
+}
+
+int tabed_last_device_error(tabed_handle* h) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  DeviceGuard guard(h->cfg.device);
+  int bits = 0;
+  const int rc = read_clear_device_error(h->err, h->stream, &bits);
+  return rc != TABED_OK ? rc : map_device_error(bits);
+}
+
+int tabed_sync_lengths(tabed_handle* h) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
+  DeviceGuard guard(h->cfg.device);
+  std::vector<int> lens(h->has_drafter ? h->R : 0), pend((size_t)h->B * 3);
+  if ((h->has_drafter && cudaMemcpyAsync(lens.data(), h->kv_len, lens.size() * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) ||
+      cudaMemcpyAsync(pend.data(), h->pending, pend.size() * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return TABED_ERR_CUDA;
+  }
+  for (size_t r = 0; r < lens.size(); ++r) h->len_ub[r] = lens[r];
+  for (int b = 0; b < h->B; ++b) h->pend_cnt[b] = pend[(size_t)b * 3];
+  h->pend_known = true;
   return TABED_OK;
 }
 
@@ -1207,6 +1344,33 @@ int tabed_state_import(tabed_handle* h, const void* host, size_t bytes) {
   if (hdr[0] != 0x7ABED || hdr[1] != h->B || hdr[2] != h->m || hdr[3] != h->cfg.window_h ||
       hdr[4] != (h->has_drafter ? 1 : 0) || hdr[5] != h->R)
     return TABED_ERR_INVALID_ARG;
+  {
+    // every field that indexes memory on the device is range-checked on the host copy first: a stale or corrupt
+    // snapshot is rejected without touching the device state
+    const size_t B = h->B, hh = std::max(1, h->cfg.window_h);
+    const unsigned char* q = in;
+    q += B * h->m * 4;                                                   // w
+    const int32_t* pend = reinterpret_cast<const int32_t*>(q); q += B * 3 * 4;
+    q += B * hh * kMaxDev * 8 + B * kMaxDev * 8;                         // ring, running sums
+    const unsigned char* pushed_raw = q; q += B * 8;                     // (64-bit fields may sit at any 4-byte offset: copied out)
+    const int32_t* ring_head = reinterpret_cast<const int32_t*>(q); q += B * 4;
+    const int32_t* ring_count = reinterpret_cast<const int32_t*>(q); q += B * 4;
+    const int32_t* grid_j = reinterpret_cast<const int32_t*>(q); q += B * 4;
+    for (size_t b = 0; b < B; ++b) {
+      const int cnt = pend[b * 3];
+      if (cnt < 1 || cnt > 2) return TABED_ERR_INVALID_ARG;
+      for (int j = 0; j < cnt; ++j) if (pend[b * 3 + 1 + j] < 0 || pend[b * 3 + 1 + j] >= h->V) return TABED_ERR_INVALID_ARG;
+      long long pushed_b;
+      memcpy(&pushed_b, pushed_raw + b * 8, 8);
+      if (pushed_b < 0 || ring_head[b] < 0 || ring_head[b] >= (int)hh || ring_count[b] < 0 || ring_count[b] > h->cfg.window_h ||
+          grid_j[b] < -1 || grid_j[b] >= kGridCand)
+        return TABED_ERR_INVALID_ARG;
+    }
+    if (h->has_drafter) {
+      const int32_t* lens = reinterpret_cast<const int32_t*>(q);
+      for (int r = 0; r < h->R; ++r) if (lens[r] < 0 || lens[r] > h->cap) return TABED_ERR_INVALID_ARG;
+    }
+  }
   DeviceGuard guard(h->cfg.device);
   for (const auto& s : parts) {
     if (cudaMemcpyAsync(s.ptr, in, s.bytes, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return TABED_ERR_CUDA;
@@ -1215,10 +1379,12 @@ int tabed_state_import(tabed_handle* h, const void* host, size_t bytes) {
   if (cudaStreamSynchronize(h->stream) != cudaSuccess) return TABED_ERR_CUDA;
   if (h->has_drafter) {
     const int32_t* lens = reinterpret_cast<const int32_t*>(in - (size_t)h->R * 4);
-    for (int r = 0; r < h->R; ++r) {
-      if (lens[r] < 0 || lens[r] > h->cap) return TABED_ERR_INVALID_ARG;
-      h->len_ub[r] = lens[r];
-    }
+    for (int r = 0; r < h->R; ++r) h->len_ub[r] = lens[r];
+  }
+  {
+    const int32_t* pend = reinterpret_cast<const int32_t*>(reinterpret_cast<const unsigned char*>(host) + 6 * sizeof(int32_t) + (size_t)h->B * h->m * 4);
+    for (int b = 0; b < h->B; ++b) h->pend_cnt[b] = pend[(size_t)b * 3];
+    h->pend_known = true;
   }
   return TABED_OK;
 }
@@ -1296,10 +1462,33 @@ static_assert(sizeof(ChunkBest) == 8, "scratch layout assumes 8-byte ChunkBest")
 static __device__ __align__(256) unsigned char g_tabed_static_scratch[kStaticBytes];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 unsigned char* g_static_ptr[kMaxDevices] = {nullptr};
 }  // namespace
+
+namespace {
+// device address of the static scratch on `device` (which must be current); looked up once per device
+unsigned char* static_scratch_base(int device) {
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[device]) {
+    void* sym = nullptr;
+    if (cudaGetSymbolAddress(&sym, g_tabed_static_scratch) != cudaSuccess || !sym) { cudaGetLastError(); return nullptr; }
+    g_static_ptr[device] = reinterpret_cast<unsigned char*>(sym);
+  }
+  return g_static_ptr[device];
+}
+}  // namespace
+
+int tabed_static_last_error(int32_t device, void* stream) {
+  if (device < 0 || device >= kMaxDevices) return TABED_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return TABED_ERR_CUDA;
+  unsigned char* base = static_scratch_base(device);
+  if (!base) return TABED_ERR_CUDA;
+  int bits = 0;
+  const int rc = read_clear_device_error(reinterpret_cast<int*>(base + kStaticErrOff), reinterpret_cast<cudaStream_t>(stream), &bits);
+  return rc != TABED_OK ? rc : map_device_error(bits);
+}
 
 int tabed_ensemble_step_static(const float* logits, const float* w, const float* u, int32_t n_requests,
                                int32_t n_inputs, int32_t vocab, int32_t sample_mode, int32_t device, void* stream,
@@ -1314,16 +1503,8 @@ int tabed_ensemble_step_static(const float* logits, const float* w, const float*
     return TABED_ERR_UNSUPPORTED;                       // beyond the fixed scratch: use a handle instead
   DeviceGuard guard(device);
   if (!guard.ok) return TABED_ERR_CUDA;
-  unsigned char* base = nullptr;
-  {
-    std::lock_guard<std::mutex> lock(g_static_mutex);
-    if (!g_static_ptr[device]) {                        // once per device, with that device current
-      void* sym = nullptr;
-      if (cudaGetSymbolAddress(&sym, g_tabed_static_scratch) != cudaSuccess || !sym) { cudaGetLastError(); return TABED_ERR_CUDA; }
-      g_static_ptr[device] = reinterpret_cast<unsigned char*>(sym);
-    }
-    base = g_static_ptr[device];
-  }
+  unsigned char* base = static_scratch_base(device);    // once per device, with that device current
+  if (!base) return TABED_ERR_CUDA;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint32_t* rowmax = reinterpret_cast<uint32_t*>(base + kStaticRowMaxOff);
   unsigned long long* rowsum = reinterpret_cast<unsigned long long*>(base + kStaticRowSumOff);

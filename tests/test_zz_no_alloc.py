@@ -42,6 +42,13 @@ def test_static_entry_point_matches_handle_entry_point_twice(B, m, V, mode):
         torch.cuda.synchronize()
         assert torch.equal(y0, y1)
         assert torch.equal(q0, q1) and torch.equal(qk0, qk1)      # tolerance 0: bitwise, as in the other tests
+        # ... and against the CPU checker itself, not only against the other entry point
+        from oracle import exact32 as X
+        lg_h, w_h, u_h = logits.cpu().numpy(), w.cpu().numpy(), u.cpu().numpy()
+        for b in range(B):
+            qk_o = X.softmax_exact(lg_h[b]); q_o = X.ensemble_exact(qk_o, w_h[b])
+            assert np.array_equal(qk1[b].cpu().numpy(), qk_o) and np.array_equal(q1[b].cpu().numpy(), q_o)
+            assert int(y1[b]) == (X.argmax_lowest(q_o) if mode == 1 else X.draw(X.masses(q_o), u_h[b]))
     h.destroy()
 
 
