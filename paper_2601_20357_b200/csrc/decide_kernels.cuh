@@ -321,7 +321,7 @@ struct PolicyArgs {
   int B, G, m, n_dev, h, policy, tvd;
   float tau;
   const int* n_accept; const int* next_token; const int* tokens;   // [B], [B], [B][G]
-  long long* dev;            // unused (the deviation sums travel through shared memory)
+  long long* dev;            // [B][G][kMaxDev] deviation sums of the round's verified positions
   long long* ring;           // [B][h][kMaxDev]
   int* ring_head; int* ring_count; long long* pushed;              // [B]
   long long* running;        // [B][kMaxDev]

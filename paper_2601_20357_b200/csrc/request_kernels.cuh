@@ -1,12 +1,17 @@
-// One thread-block CLUSTER per request for the three vocabulary-wide stages of a round:
+// Thread-block CLUSTERS for the three vocabulary-wide stages of a round, ONE launch each:
 //   k_ensemble_req : Algorithm 1 steps 6-7   (softmax of the m drafter rows, weighted average, draw)
+//                    one cluster per request
 //   k_verify_req   : Sec. 3 item 3           (target softmax, sequential acceptance, residual / bonus draw)
+//                    one cluster per (request, position): the softmax of the G + 1 target rows runs on all of
+//                    them at once; the cluster that finishes a request last (a ticket) takes its acceptance
+//                    prefix and draws the replacement / bonus token
 //   k_update_req   : Sec. 4.1, App. B        (deviation of every drafter over the verified positions, window
 //                                             push, policy, cache commit)
-// Each stage is ONE launch with no scratch in global memory and no spin-wait: the vocabulary is cut into
-// one contiguous slice per CTA of the cluster; every vocabulary-wide quantity (row maxima, integer mass
-// sums, per-slice masses, accept flags, deviation sums) is exchanged through distributed shared memory and
-// ordered by the hardware cluster barrier.  A row is read from HBM once; the later passes of the exact
+//                    one cluster per (request, verified position); the last one of a request runs the policy
+// No spin-wait anywhere: the vocabulary is cut into one contiguous slice per CTA of the cluster; every
+// vocabulary-wide quantity (row maxima, integer mass sums, per-slice masses, deviation sums) is exchanged
+// through distributed shared memory and ordered by the hardware cluster barrier; clusters of one request meet
+// through a ticket counter (taken after a fence, reset by the last arriver, so no memset is needed).  A row is read from HBM once; the later passes of the exact
 // softmax (maximum -> integer sum of masses -> quotient) re-read the CTA's own slice, which L1/L2 still hold.
 // Loads are 128-bit where the row pitch allows, reductions are warp shuffles.  All decision arithmetic is
 // the order-independent specification of exact_math.cuh, so the results do not depend on the cluster size.
@@ -90,7 +95,7 @@ __device__ __forceinline__ void req_row_maxima(cg::cluster_group& cluster, const
 #pragma unroll 1
   for (int i0 = 0; i0 < rows; i0 += 4) {
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 2
+#pragma unroll 4
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float x[4][4];
 #pragma unroll
@@ -130,7 +135,7 @@ __device__ __forceinline__ void req_row_sums(cg::cluster_group& cluster, const R
     float mx[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) mx[j] = (i0 + j < rows) ? req_max_of(c, S, i0 + j) : 0.0f;
-#pragma unroll 2
+#pragma unroll 4
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float x[2][4];
 #pragma unroll
@@ -179,11 +184,21 @@ __device__ __forceinline__ void req_gather_mass(cg::cluster_group& cluster, cons
   cluster.sync();
 }
 
-// Inverse-CDF draw on the masses gathered in S.all_mass[which]: the CTA whose slice holds the threshold walks
-// it (block-wide prefix sums, 4 consecutive elements per thread) and returns the token through `found`
-// (true in every thread of that CTA only).  mass_at(v) gives the integer mass of element v of the slice.
+// For the draw every thread owns a CONTIGUOUS range of the slice (so that a prefix over the threads is a prefix
+// over the vocabulary): [t_lo, t_hi), a multiple of 4 elements long.
+__device__ __forceinline__ void req_thread_range(const ReqCtx& c, int slice, int* t_lo, int* t_hi) {
+  const int per = ((slice + kReqThreads - 1) / kReqThreads + 3) & ~3;
+  *t_lo = min(c.v_hi, c.v_lo + c.tid * per);
+  *t_hi = min(c.v_hi, *t_lo + per);
+}
+
+// Inverse-CDF draw on the masses gathered in S.all_mass[which] (tmass = this thread's mass over its range):
+// the CTA whose slice holds the threshold finds the thread whose range holds it (one block-wide prefix sum),
+// and that thread walks its range.  Returns true in every thread of that CTA only, with the token in *token.
+// mass_at(v) gives the integer mass of element v.
 template <typename MassAt>
-__device__ __forceinline__ bool req_draw(const ReqCtx& c, ReqShared& S, int which, float u, MassAt mass_at, int* token, int* status) {
+__device__ __forceinline__ bool req_draw(const ReqCtx& c, ReqShared& S, int which, float u, unsigned long long tmass, int t_lo, int t_hi,
+                                         MassAt mass_at, int* token, int* status) {
   unsigned long long T = 0;
   for (unsigned r = 0; r < c.CS; ++r) T += S.all_mass[which][r];
   *status = 0;
@@ -196,38 +211,28 @@ __device__ __forceinline__ bool req_draw(const ReqCtx& c, ReqShared& S, int whic
     thr -= mr;
   }
   if (owner != c.rank) return false;
+  unsigned long long incl = tmass;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (c.lane >= o) incl += t;
+  }
+  __syncthreads();                                             // (S.scan was read by the gather before)
+  if (c.lane == 31) S.scan[c.warp] = incl;
   if (c.tid == 0) S.result = 0x7fffffff;
   __syncthreads();
-  unsigned long long carry = 0;
+  unsigned long long run = incl - tmass;
+#pragma unroll
+  for (int i = 0; i < kReqWarps; ++i) if (i < c.warp) run += S.scan[i];
+  if (run <= thr && thr < run + tmass) {
 #pragma unroll 1
-  for (int v0 = c.v_lo; v0 < c.v_hi; v0 += kReqStep) {
-    const int v = v0 + c.tid * 4;
-    unsigned long long mloc[4], tsum = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { mloc[j] = (v + j < c.v_hi) ? mass_at(v + j) : 0ull; tsum += mloc[j]; }
-    unsigned long long incl = tsum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (c.lane >= o) incl += t;
+    for (int v = t_lo; v < t_hi; ++v) {
+      const unsigned long long mv = mass_at(v);
+      run += mv;
+      if (run > thr && mv != 0ull) { S.result = v; break; }
     }
-    if (c.lane == 31) S.scan[c.warp] = incl;
-    __syncthreads();
-    unsigned long long wpre = 0, ctot = 0;
-#pragma unroll
-    for (int i = 0; i < kReqWarps; ++i) { if (i < c.warp) wpre += S.scan[i]; ctot += S.scan[i]; }
-    unsigned long long run = carry + wpre + incl - tsum;
-    if (run <= thr) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        run += mloc[j];
-        if (run > thr && mloc[j] != 0ull) { atomicMin(&S.result, v + j); break; }
-      }
-    }
-    carry += ctot;
-    __syncthreads();
-    if (S.result != 0x7fffffff) break;
   }
+  __syncthreads();
   const int y = S.result;
   if (y == 0x7fffffff) { *status = 2; *token = 0; }           // cannot happen for consistent masses; reported
   else *token = y;
@@ -282,7 +287,7 @@ struct EnsembleArgs {
   int* err;
 };
 
-__global__ void __launch_bounds__(kReqThreads) k_ensemble_req(const EnsembleArgs A) {
+__global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleArgs A) {
   pdl_trigger();
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ ReqShared S;
@@ -327,11 +332,9 @@ __global__ void __launch_bounds__(kReqThreads) k_ensemble_req(const EnsembleArgs
       if (qk_b) req_st4(qk_b + (long long)k * V, v, c.v_hi, vec_qk, a);
     }
     req_st4(q_row, v, c.v_hi, vec_q, acc);
+    if (A.greedy) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (v + j >= c.v_hi) continue;
-      if (A.greedy) { if (acc[j] > best.val) { best.val = acc[j]; best.idx = v + j; } }
-      else mass += mass_of(acc[j]);
+      for (int j = 0; j < 4; ++j) if (v + j < c.v_hi && acc[j] > best.val) { best.val = acc[j]; best.idx = v + j; }
     }
   }
   int y = 0, status = 0;
@@ -342,8 +345,19 @@ __global__ void __launch_bounds__(kReqThreads) k_ensemble_req(const EnsembleArgs
     y = req_best_of(c, S, 0);
     mine = c.rank == 0;
   } else {
-    req_gather_mass(cluster, c, S, mass, 0);       // (its barriers also make this CTA's q slice visible to all its threads)
-    mine = req_draw(c, S, 0, A.u[b * A.u_stride], [&](int v) { return mass_of(q_row[v]); }, &y, &status);
+    // masses of q over each thread's contiguous range (the slice was just written by this CTA: L1/L2 hold it)
+    __syncthreads();
+    int t_lo, t_hi;
+    req_thread_range(c, A.slice, &t_lo, &t_hi);
+#pragma unroll 4
+    for (int v = t_lo; v < t_hi; v += 4) {
+      float x[4];
+      req_ld4_rw(q_row, v, t_hi, vec_q, 0.0f, x);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(x[j]);
+    }
+    req_gather_mass(cluster, c, S, mass, 0);
+    mine = req_draw(c, S, 0, A.u[b * A.u_stride], mass, t_lo, t_hi, [&](int v) { return mass_of(q_row[v]); }, &y, &status);
     if (status == 1 && c.rank == 0) { mine = true; y = 0; }
   }
   if (mine && c.tid == 0) {
@@ -353,8 +367,23 @@ __global__ void __launch_bounds__(kReqThreads) k_ensemble_req(const EnsembleArgs
   }
 }
 
+// A cluster reports that its part of request b is in global memory and learns whether it is the last of
+// `n_parts`: the block barrier (the caller's cluster barrier) orders the cluster's stores before the fence of
+// CTA 0's first thread, which takes the ticket; the last arriver resets it.  Ends with a cluster barrier; the
+// answer is the same in every thread of the cluster.
+__device__ __forceinline__ bool req_last_of_request(cg::cluster_group& cluster, const ReqCtx& c, int* flag_smem, int* ticket, int n_parts) {
+  if (c.rank == 0 && c.tid == 0) {
+    __threadfence();
+    const int last = atomicAdd(ticket, 1) == n_parts - 1;
+    if (last) { *ticket = 0; __threadfence(); }
+    for (unsigned r = 0; r < c.CS; ++r) *cluster.map_shared_rank(flag_smem, r) = last;
+  }
+  cluster.sync();
+  return *flag_smem != 0;
+}
+
 // ------------------------------------------------------------------------------------------------
-// Sec. 3 item 3 for one request per cluster.
+// Sec. 3 item 3.  grid: B * (G + 1) clusters; cluster (b, i) owns target row i of request b.
 // ------------------------------------------------------------------------------------------------
 struct VerifyArgs {
   int V, G, greedy, slice;
@@ -364,32 +393,35 @@ struct VerifyArgs {
   const float* u_accept;                        // [B][G]
   const float* u_resid;                         // [B]
   float* p;                                     // [B][G+1][V]
+  int* row_flag;                                // [B][G+1] scratch: accept flag of position i (greedy: argmax of p_i)
+  int* ticket;                                  // [B] scratch, zero between launches
   int *n_accept, *out_n_accept, *next_token, *out_next_token;
   int* err;
 };
 
-__global__ void __launch_bounds__(kReqThreads) k_verify_req(const VerifyArgs A) {
+__global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs A) {
   pdl_trigger();
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ ReqShared S;
+  __shared__ int s_last;
   const ReqCtx c = req_ctx(cluster, A.V, A.slice);
-  const int b = blockIdx.x / c.CS, G = A.G, V = A.V, rows = G + 1;
+  const int G = A.G, V = A.V, rows = G + 1;
+  const int unit = blockIdx.x / c.CS, b = unit / rows, i = unit - b * rows;
   pdl_wait();
-  const float* lg = A.logits + (long long)b * rows * V;
+  const float* lg = A.logits + ((long long)b * rows + i) * V;
   float* p_b = A.p + (long long)b * rows * V;
   const float* q_b = A.q + (long long)b * A.q_req_stride;
   const bool vec = req_vec_ok(A.logits, V), vec_p = (V & 3) == 0;
-  req_row_maxima(cluster, c, S, lg, V, rows, vec);
-  req_row_sums(cluster, c, S, lg, V, rows, vec);
-  // p = e / S for every row; in greedy mode also each row's argmax
-#pragma unroll 1
-  for (int i = 0; i < rows; ++i) {
-    const float mx = req_max_of(c, S, i), sn = req_norm_of(c, S, i);
+  req_row_maxima(cluster, c, S, lg, V, 1, vec);
+  req_row_sums(cluster, c, S, lg, V, 1, vec);
+  const float mx = req_max_of(c, S, 0), sn = req_norm_of(c, S, 0);
+  {
+    // p_i = e / S; in greedy mode also its argmax
     ReqBest best{-1.0f, 0x7fffffff};
-#pragma unroll 2
+#pragma unroll 4
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float a[4];
-      req_ld4(lg + (long long)i * V, v, c.v_hi, vec, -INFINITY, a);
+      req_ld4(lg, v, c.v_hi, vec, -INFINITY, a);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx)), sn);
@@ -397,22 +429,28 @@ __global__ void __launch_bounds__(kReqThreads) k_verify_req(const VerifyArgs A) 
       }
       req_st4(p_b + (long long)i * V, v, c.v_hi, vec_p, a);
     }
-    if (A.greedy) req_gather_best(cluster, c, S, best, i, i == rows - 1);
+    if (A.greedy) req_gather_best(cluster, c, S, best, 0, true);
   }
-  if (!A.greedy && c.tid < G) {
-    // position tid: the CTA whose slice holds the drafted token decides and tells every CTA
-    const int i = c.tid, y = A.tokens[b * G + i];
-    if (y >= c.v_lo && y < c.v_hi) {
-      const float py = __fdiv_rn(xexp(__fsub_rn(__ldg(lg + (long long)i * V + y), req_max_of(c, S, i))), req_norm_of(c, S, i));
+  cluster.sync();                                // the row is stored (and the bests gathered)
+  if (c.rank == 0 && c.tid == 0) {
+    int flag;
+    if (A.greedy) flag = req_best_of(c, S, 0);
+    else if (i < G) {
+      const int y = A.tokens[b * G + i];
+      const float py = __fdiv_rn(xexp(__fsub_rn(__ldg(lg + y), mx)), sn);          // the value stored in p_i[y]
       const float qy = __ldg(q_b + (long long)i * V + y);
-      const int ok = (py >= qy) || (__fmul_rn(A.u_accept[b * G + i], qy) < py);
-      for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.ok[0], r)[i] = ok;
-    }
+      flag = (py >= qy) || (__fmul_rn(A.u_accept[b * G + i], qy) < py);
+    } else flag = 1;
+    A.row_flag[b * rows + i] = flag;
   }
-  cluster.sync();
+  if (!req_last_of_request(cluster, c, &s_last, A.ticket + b, rows)) return;
+
+  // ---- the request's last cluster: acceptance prefix, replacement / bonus token -----------------------
   int a = 0;
-  if (A.greedy) { for (; a < G; ++a) if (req_best_of(c, S, a) != A.tokens[b * G + a]) break; }
-  else { for (; a < G; ++a) if (!S.ok[a]) break; }
+  for (; a < G; ++a) {
+    const int f = __ldcg(A.row_flag + b * rows + a);
+    if (A.greedy ? (f != A.tokens[b * G + a]) : (f == 0)) break;
+  }
   if (c.rank == 0 && c.tid == 0) {
     A.n_accept[b] = a;
     if (A.out_n_accept) A.out_n_accept[b] = a;
@@ -420,37 +458,45 @@ __global__ void __launch_bounds__(kReqThreads) k_verify_req(const VerifyArgs A) 
   int z = 0, status = 0;
   bool mine = false;
   if (A.greedy) {
-    z = req_best_of(c, S, a);
+    z = __ldcg(A.row_flag + b * rows + a);
     mine = c.rank == 0;
   } else {
-    // replacement token from norm(max(0, p_a - q_a)) (from p_a if that has no mass); bonus token from p_G
+    // replacement token from norm(max(0, p_a - q_a)) (from p_a if that has no mass); bonus token from p_G.
+    // p_a was written by another cluster of this launch: read through L2.
     const float* p_a = p_b + (long long)a * V;
     const float* q_a = (a < G) ? q_b + (long long)a * V : nullptr;
+    auto p_at = [&](int v) { return __ldcg(p_a + v); };
+    int t_lo, t_hi;
+    req_thread_range(c, A.slice, &t_lo, &t_hi);
+    auto ld_p4 = [&](int v, float (&x)[4]) {
+      if (vec_p && v + 4 <= t_hi) { const float4 t = __ldcg(reinterpret_cast<const float4*>(p_a + v)); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
+      else { for (int j = 0; j < 4; ++j) x[j] = (v + j < t_hi) ? __ldcg(p_a + v + j) : 0.0f; }
+    };
     const bool vec_qa = q_a && req_vec_ok(A.q, A.q_req_stride) && (V & 3) == 0;
     unsigned long long mass = 0;
-#pragma unroll 2
-    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+#pragma unroll 4
+    for (int v = t_lo; v < t_hi; v += 4) {
       float pa[4], qa[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      req_ld4_rw(p_a, v, c.v_hi, vec_p, 0.0f, pa);
-      if (q_a) req_ld4(q_a, v, c.v_hi, vec_qa, 0.0f, qa);
+      ld_p4(v, pa);
+      if (q_a) req_ld4(q_a, v, t_hi, vec_qa, 0.0f, qa);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) if (v + j < c.v_hi) mass += mass_of(q_a ? resid_val(pa[j], qa[j]) : pa[j]);
+      for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(q_a ? resid_val(pa[j], qa[j]) : pa[j]);
     }
     req_gather_mass(cluster, c, S, mass, 0);
     const float u = A.u_resid[b];
-    mine = req_draw(c, S, 0, u, [&](int v) { return mass_of(q_a ? resid_val(p_a[v], __ldg(q_a + v)) : p_a[v]); }, &z, &status);
+    mine = req_draw(c, S, 0, u, mass, t_lo, t_hi, [&](int v) { return mass_of(q_a ? resid_val(p_at(v), __ldg(q_a + v)) : p_at(v)); }, &z, &status);
     if (status == 1 && q_a) {
       // residual without mass (p_a == q_a bitwise): draw from p_a itself.  Every CTA sees the same zero total.
       mass = 0;
-#pragma unroll 2
-      for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+#pragma unroll 4
+      for (int v = t_lo; v < t_hi; v += 4) {
         float pa[4];
-        req_ld4_rw(p_a, v, c.v_hi, vec_p, 0.0f, pa);
+        ld_p4(v, pa);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) if (v + j < c.v_hi) mass += mass_of(pa[j]);
+        for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(pa[j]);
       }
       req_gather_mass(cluster, c, S, mass, 1);
-      mine = req_draw(c, S, 1, u, [&](int v) { return mass_of(p_a[v]); }, &z, &status);
+      mine = req_draw(c, S, 1, u, mass, t_lo, t_hi, [&](int v) { return mass_of(p_at(v)); }, &z, &status);
     }
     if (status == 1 && c.rank == 0) { mine = true; z = 0; }
   }
@@ -462,38 +508,40 @@ __global__ void __launch_bounds__(kReqThreads) k_verify_req(const VerifyArgs A) 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Sec. 4.1 / App. B for one request per cluster: deviation sums of the verified positions, window push,
-// policy, cache commit.  The CTAs' fixed-point partial sums meet in CTA 0 of the cluster (integer sums:
-// order-free), whose first warp then runs the policy.
+// Sec. 4.1 / App. B.  grid: B * G clusters; cluster (b, i) sums the deviations of position i (if it is a
+// verified one: i <= min(a, G-1)); the fixed-point partial sums of its CTAs meet in CTA 0 (integer sums:
+// order-free), which stores them; the last cluster of the request then runs the policy in one warp.
 // ------------------------------------------------------------------------------------------------
 struct UpdateArgs {
   int V, slice, grid_policy;
   const float* p;                 // [B][G+1][V]
   const float* qk;                // [B][G][m][V]
-  PolicyArgs P;                   // P.dev unused
+  int* ticket;                    // [B] scratch, zero between launches
+  PolicyArgs P;                   // P.dev: [B][G][kMaxDev] scratch (every verified entry is rewritten each round)
 };
 
 struct UpdShared {
   long long red[kReqWarps][kMaxDev];
-  long long all_dev[kReqMaxCluster][kReqMaxRows - 1][kMaxDev];    // [CTA][position][deviation index], filled in CTA 0
+  long long all_dev[kReqMaxCluster][kMaxDev];        // [CTA][deviation index], filled in CTA 0
 };
 
-__device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last, const UpdShared& U, unsigned CS);
+__device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last);
 
-__global__ void __launch_bounds__(kReqThreads) k_update_req(const UpdateArgs A) {
+__global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs A) {
   pdl_trigger();
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ UpdShared U;
+  __shared__ int s_last;
   const ReqCtx c = req_ctx(cluster, A.V, A.slice);
   const PolicyArgs& P = A.P;
-  const int b = blockIdx.x / c.CS, G = P.G, V = A.V, m = P.m, n_dev = P.n_dev, tvd = P.tvd;
+  const int G = P.G, V = A.V, m = P.m, n_dev = P.n_dev, tvd = P.tvd;
+  const int unit = blockIdx.x / c.CS, b = unit / G, i = unit - b * G;
   pdl_wait();
   const int a = P.n_accept[b];
   const int last = min(a, G - 1);
+  if (i > last) return;                             // (the whole cluster: position not verified)
   const bool vec = (V & 3) == 0;
-  long long* mine_in_0 = cluster.map_shared_rank(&U.all_dev[0][0][0], 0) + (size_t)c.rank * (kReqMaxRows - 1) * kMaxDev;
-#pragma unroll 1
-  for (int i = 0; i <= last; ++i) {
+  {
     const float* p_i = A.p + ((long long)b * (G + 1) + i) * V;
     const float* qbase = A.qk + ((long long)b * G + i) * m * V;
     long long acc[kMaxDev];
@@ -503,23 +551,25 @@ __global__ void __launch_bounds__(kReqThreads) k_update_req(const UpdateArgs A) 
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float pv[4], lp[4];
       req_ld4(p_i, v, c.v_hi, vec, 0.0f, pv);
-      if (!tvd) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
-      }
       if (!A.grid_policy) {
+        float qv[kMaxInputs][4];
+#pragma unroll
+        for (int k = 0; k < kMaxInputs; ++k)
+          if (k < m) req_ld4(qbase + (long long)k * V, v, c.v_hi, vec, 0.0f, qv[k]);
+        if (!tvd) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
+        }
 #pragma unroll
         for (int k = 0; k < kMaxInputs; ++k) {
           if (k >= m) break;
-          float qv[4];
-          req_ld4(qbase + (long long)k * V, v, c.v_hi, vec, 0.0f, qv);
           long long s = 0;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             if (v + j >= c.v_hi) continue;
             float t;
-            if (tvd) t = fabsf(__fsub_rn(pv[j], qv[j]));
-            else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(qv[j], kFltMin)))) : 0.0f;
+            if (tvd) t = fabsf(__fsub_rn(pv[j], qv[k][j]));
+            else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(qv[k][j], kFltMin)))) : 0.0f;
             s += __float2ll_rz(__fmul_rn(t, kMassScale));
           }
           acc[k] += s;
@@ -528,6 +578,10 @@ __global__ void __launch_bounds__(kReqThreads) k_update_req(const UpdateArgs A) 
         float q0[4], q1[4];
         req_ld4(qbase, v, c.v_hi, vec, 0.0f, q0);
         req_ld4(qbase + V, v, c.v_hi, vec, 0.0f, q1);
+        if (!tvd) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
+        }
 #pragma unroll
         for (int jc = 0; jc < kGridCand; ++jc) {
           const float c1 = __fdiv_rn((float)jc, 10.0f);
@@ -546,7 +600,6 @@ __global__ void __launch_bounds__(kReqThreads) k_update_req(const UpdateArgs A) 
         }
       }
     }
-    __syncthreads();                                  // the previous position's partials have been read
 #pragma unroll
     for (int kd = 0; kd < kMaxDev; ++kd) {
       if (kd < n_dev) {
@@ -559,16 +612,23 @@ __global__ void __launch_bounds__(kReqThreads) k_update_req(const UpdateArgs A) 
       long long t = 0;
 #pragma unroll
       for (int w = 0; w < kReqWarps; ++w) t += U.red[w][c.tid];
-      mine_in_0[i * kMaxDev + c.tid] = t;
+      cluster.map_shared_rank(&U.all_dev[0][0], 0)[c.rank * kMaxDev + c.tid] = t;
     }
   }
   cluster.sync();
-  if (c.rank == 0 && c.warp == 0) policy_commit(P, b, c.lane, last, U, c.CS);
+  if (c.rank == 0 && c.tid < n_dev) {
+    long long t = 0;
+    for (unsigned r = 0; r < c.CS; ++r) t += U.all_dev[r][c.tid];
+    P.dev[((long long)b * G + i) * kMaxDev + c.tid] = t;
+  }
+  __syncthreads();                                  // (CTA 0: the sums are stored before its first thread's fence)
+  if (!req_last_of_request(cluster, c, &s_last, A.ticket + b, last + 1)) return;
+  if (c.rank == 0 && c.warp == 0) policy_commit(P, b, c.lane, last);
 }
 
 // One warp per request: lane kd carries deviation index kd through the window (its running sum stays in a
 // register), then lane 0 applies the policy in its fixed order and commits the caches and pending tokens.
-__device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last, const UpdShared& U, unsigned CS) {
+__device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last) {
   const int a = A.n_accept[b];
   long long r = 0;
   {
@@ -577,8 +637,7 @@ __device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int la
     if (on) r = run[lane];
     int head = A.h > 0 ? A.ring_head[b] : 0, count = A.h > 0 ? A.ring_count[b] : 0;
     for (int i = 0; i <= last; ++i) {
-      long long dv = 0;
-      if (on) for (unsigned q = 0; q < CS; ++q) dv += U.all_dev[q][i][lane];
+      const long long dv = on ? __ldcg(A.dev + ((long long)b * A.G + i) * kMaxDev + lane) : 0;   // stored by this launch's clusters
       if (A.h > 0) {
         long long* slot = A.ring + ((long long)b * A.h + head) * kMaxDev;
         const bool full = count == A.h;

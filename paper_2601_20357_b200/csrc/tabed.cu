@@ -57,7 +57,8 @@ struct tabed_handle {
   float *rope_cos = nullptr, *rope_sin = nullptr;
   int *kv_len = nullptr, *pending = nullptr;
   float *w = nullptr;
-  long long *ring = nullptr, *running = nullptr, *pushed = nullptr;
+  long long *dev = nullptr, *ring = nullptr, *running = nullptr, *pushed = nullptr;
+  int *req_ticket = nullptr, *row_flag = nullptr;     // scratch of the per-request cluster kernels
   int *ring_head = nullptr, *ring_count = nullptr, *grid_j = nullptr;
   SlotDesc* slots = nullptr; int* last_slot = nullptr;
   float *x = nullptr, *qkv = nullptr, *attn_out = nullptr, *mid = nullptr, *part_o = nullptr, *part_ml = nullptr;
@@ -147,11 +148,11 @@ void launch_pdl(tabed_handle* h, void (*kern)(KArgs...), dim3 grid, dim3 block, 
 }
 #define TABED_LAUNCH_PDL(h, kern, grid, block, smem, ...) launch_pdl((h), (kern), dim3(grid), dim3(block), (smem), __VA_ARGS__)
 
-// One cluster of `cs` CTAs per request, as a programmatic dependent of the kernel before it in the stream.
+// `n_clusters` clusters of `cs` CTAs, as a programmatic dependent of the kernel before it in the stream.
 template <typename ArgT>
-void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_requests, int cs, const ArgT& args) {
+void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_clusters, int cs, const ArgT& args) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(n_requests * cs)); cfg.blockDim = dim3(kReqThreads); cfg.dynamicSmemBytes = 0; cfg.stream = h->stream;
+  cfg.gridDim = dim3((unsigned)(n_clusters * cs)); cfg.blockDim = dim3(kReqThreads); cfg.dynamicSmemBytes = 0; cfg.stream = h->stream;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -162,13 +163,13 @@ void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_requests
   h->launches++;
 }
 
-// CTAs per request cluster: as many as keep about two CTAs per SM busy over all requests, no finer than ~1024
+// CTAs per cluster: as many as keep about two CTAs per SM busy over all clusters, no finer than ~1024
 // vocabulary elements per CTA; slice = vocabulary elements per CTA (a multiple of 4, so that slices start on
 // 16-byte boundaries).
-int pick_cluster(const tabed_handle* h, int* slice) {
+int pick_cluster(const tabed_handle* h, int n_clusters, int* slice) {
   const int by_v = (h->V + 1023) / 1024, n_sm = h->n_sm > 0 ? h->n_sm : 148;
   int cs = 1;
-  while (cs * 2 <= h->cs_max && (long long)h->B * cs * 2 <= 2ll * n_sm && cs < by_v) cs *= 2;
+  while (cs * 2 <= h->cs_max && (long long)n_clusters * cs * 2 <= 3ll * n_sm && cs < by_v) cs *= 2;
   *slice = ((h->V + cs - 1) / cs + 3) & ~3;
   return cs;
 }
@@ -372,7 +373,7 @@ void run_ensemble(tabed_handle* h, const float* logits, const float* w, const fl
                   float* q_out, long long q_stride) {
   ProfScope ps(h, TABED_PROF_ENSEMBLE);
   EnsembleArgs a{};
-  const int cs = pick_cluster(h, &a.slice);
+  const int cs = pick_cluster(h, h->B, &a.slice);
   a.V = h->V; a.m = h->m; a.greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
   a.logits = logits; a.w = w; a.u = u; a.u_stride = u_stride;
   a.qk_out = qk_out; a.qk_req_stride = qk_stride; a.q_out = q_out; a.q_req_stride = q_stride;
@@ -802,7 +803,8 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   auto A = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count); };
   const size_t B = h->B, m = h->m, R = h->R, G = h->G, V = h->V;
   A(&h->w, B * m); A(&h->pending, B * 3);
-  A(&h->ring, B * std::max(1, c.window_h) * kMaxDev); A(&h->running, B * kMaxDev);
+  A(&h->dev, B * G * kMaxDev); A(&h->ring, B * std::max(1, c.window_h) * kMaxDev); A(&h->running, B * kMaxDev);
+  A(&h->req_ticket, 2 * B); A(&h->row_flag, B * (G + 1));
   A(&h->pushed, B); A(&h->ring_head, B); A(&h->ring_count, B); A(&h->grid_j, B);
   A(&h->qk, B * G * m * V); A(&h->q, B * G * V); A(&h->p, B * (G + 1) * V); A(&h->scratch_q, B * V);
   A(&h->tokens, B * G); A(&h->n_accept, B); A(&h->next_token, B); A(&h->w_argmax, B);
@@ -1080,14 +1082,15 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   DeviceGuard guard(h->cfg.device);
   ProfScope ps(h, TABED_PROF_VERIFY);
   VerifyArgs a{};
-  const int cs = pick_cluster(h, &a.slice);
+  const int cs = pick_cluster(h, h->B * (h->G + 1), &a.slice);
+  a.row_flag = h->row_flag; a.ticket = h->req_ticket;
   a.V = h->V; a.G = h->G; a.greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
   a.logits = target_logits; a.q = h->q; a.q_req_stride = (long long)h->G * h->V; a.tokens = h->tokens;
   a.u_accept = u_accept; a.u_resid = u_resid; a.p = h->p;
   a.n_accept = h->n_accept; a.out_n_accept = out_n_accept == h->n_accept ? nullptr : out_n_accept;
   a.next_token = h->next_token; a.out_next_token = out_next_token == h->next_token ? nullptr : out_next_token;
   a.err = h->err;
-  launch_request_clusters(h, k_verify_req, h->B, cs, a);
+  launch_request_clusters(h, k_verify_req, h->B * (h->G + 1), cs, a);
   h->phase = PH_VERIFIED;
   return check_cuda();
 }
@@ -1100,16 +1103,17 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
   {
     ProfScope ps(h, TABED_PROF_UPDATE);
     UpdateArgs u{};
-    const int cs = pick_cluster(h, &u.slice);
+    const int cs = pick_cluster(h, h->B * h->G, &u.slice);
+    u.ticket = h->req_ticket + h->B;
     u.V = h->V; u.grid_policy = h->cfg.policy == TABED_POLICY_GRID_MT ? 1 : 0; u.p = h->p; u.qk = h->qk;
     PolicyArgs& a = u.P;
     a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
     a.tau = h->cfg.tau; a.n_accept = h->n_accept; a.next_token = h->next_token; a.tokens = h->tokens;
-    a.dev = nullptr; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
+    a.dev = h->dev; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
     a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
     a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
     a.pending = h->pending; a.out_w = out_w; a.out_argmax = out_w_argmax;
-    launch_request_clusters(h, k_update_req, h->B, cs, u);
+    launch_request_clusters(h, k_update_req, h->B * h->G, cs, u);
   }
   // the host has not seen the accept counts: the bound grows by the most a round can keep (tabed_round_host and
   // tabed_sync_lengths replace it by the exact lengths)
