@@ -155,32 +155,56 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def time_oracle(wl, rounds, warmup=0):
+def oracle_sample(wl):
+    """The part of the workload one CPU step covers: whole rounds of the first requests, as many as keep a round
+    of the plain checker to a few seconds (rows x layers x width is what a round costs)."""
+    c = wl.drafter
+    cost_row = c.n_params_layers + c.n_params_head                   # multiply-accumulates per row and step
+    rows_max = max(wl.n_inputs, int(2.0e8 / cost_row) * wl.n_inputs)  # ~1-2 s of fp64 matrix-vector work per round
+    n_req = max(1, min(wl.n_requests, rows_max // wl.n_inputs))
+    return wl if n_req == wl.n_requests else wl.replace(n_requests=n_req)
+
+
+def time_oracle(wl, rounds, warmup=0, budget_s=None):
+    """Times `rounds` rounds (after `warmup`) of the checker; with a budget, stops early once it is used up.
+    Returns (request-rounds per second, seconds, rounds actually timed)."""
     orc = oracle_setup(wl)
     for r in range(warmup):
         oracle_round(orc, wl, r)
     t0 = time.perf_counter()
+    done = 0
     for r in range(warmup, warmup + rounds):
         oracle_round(orc, wl, r)
+        done += 1
+        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+            break
     dt = time.perf_counter() - t0
-    return wl.n_requests * rounds / dt, dt
+    return wl.n_requests * done / dt, dt, done
+
+
+def config_of(wl):
+    """The `config` object both arms print (identical keys and values for one workload)."""
+    return {"workload": wl.name, "n_inputs": wl.n_inputs, "n_requests": wl.n_requests, "rows": wl.n_rows, "gamma": wl.gamma,
+            "window_h": wl.window_h, "vocab": wl.drafter.vocab, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model}
 
 
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    value, dt = time_oracle(wl, args.steps, args.warmup)
+    sub = oracle_sample(wl)
+    warm = min(args.warmup, 2)
+    value, dt, done = time_oracle(sub, args.steps, warm, budget_s=150.0)
     cores = blas_threads()
+    what = (f"each step = one whole round of the first {sub.n_requests} of {wl.n_requests} requests ({sub.n_rows} rows, their full caches); "
+            f"{done} of {args.steps} steps timed after {warm} warm-up steps ({dt:.1f} s); value = requests x steps / time")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1000.0 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": 1000.0 * dt / max(done, 1), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "n_inputs": wl.n_inputs, "n_requests": wl.n_requests, "gamma": wl.gamma,
-                   "window_h": wl.window_h, "vocab": wl.drafter.vocab},
+        "config": config_of(wl),
         "drafted_tokens_per_sec": value * wl.gamma,
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{args.steps} rounds of {wl.name} after {args.warmup} warm-up rounds, every round whole"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -307,30 +331,23 @@ def class_bytes(wl, kv_tokens_total, mean_accept):
     return cb
 
 
-def run_ours(args, wl):
+def measure(wl, device, K, Wm, *, rank=0, dist=None, path="auto", breakdown=False, e2e_steps=0, trace=None, trace_cta=0,
+            clock_index=None):
+    """Sets the workload up on `device`, rehearses the rounds (to have the target stand-in's logits), then times K
+    rounds after Wm warm-up rounds, one CUDA-event pair per round, 256 MB written between rounds.  Returns a dict."""
     import torch
     from paper_2601_20357_b200 import binding as TB
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    device = torch.device("cuda", local)
-    torch.cuda.set_device(device)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=device)
-    K, Wm = args.steps, args.warmup
+    from paper_2601_20357_b200.replicas import whole_job
     total = K + Wm
     B, G, m, V = wl.n_requests, wl.gamma, wl.n_inputs, wl.drafter.vocab
     if wl.kv_capacity and wl.synthetic_kv_len is None:
-        need = max(sum(l for _, l in pre) for pre in wl.prefixes) + (total + args.e2e_steps + 24) * (G + 1) + 8
+        need = max(sum(l for _, l in pre) for pre in wl.prefixes) + (total + e2e_steps + 24) * (G + 1) + 8
         if need > wl.kv_capacity:
             wl = wl.replace(kv_capacity=need)
     g = gpu_setup(wl, device)
-    if args.path == "per-op":
+    if path == "per-op":
         g.select_path(TB.PATH_PER_OP)
-    elif args.path == "tensor-core":
+    elif path == "tensor-core":
         g.select_path(TB.PATH_TENSOR_CORE)
     snap = g.state_export()
     alpha = torch.from_numpy(W.request_alpha(wl)).to(device)
@@ -378,8 +395,9 @@ def run_ours(args, wl):
         g.verify(targets[r], u[r][1], u[r][2], a, z)
         g.update_weights(w, am)
 
-    sampler = ClockSampler(local)
-    sampler.start()
+    sampler = ClockSampler(clock_index) if clock_index is not None else None
+    if sampler:
+        sampler.start()
     for r in range(Wm):
         flush.zero_()
         one_round(r)
@@ -388,15 +406,17 @@ def run_ours(args, wl):
         dist.barrier()
     torch.cuda.synchronize(device)
     launches0 = g.launch_count()
-    persistent = g.current_path() == TB.PATH_PERSISTENT
+    cur_path = g.current_path()
+    persistent = cur_path == TB.PATH_PERSISTENT
     if persistent:
         top_cls, top_name, top_kernel = TB.PROF_DRAFT_ROUND, "draft_round", "k_draft_round (persistent: gamma decoder steps + ensemble)"
-    elif g.current_path() == TB.PATH_TENSOR_CORE:
+    elif cur_path == TB.PATH_TENSOR_CORE:
         top_cls, top_name, top_kernel = TB.PROF_ATTENTION, "attention", "k_attn_tc_bf16 (decode attention of all rows over their bf16 K,V caches)"
     else:
         top_cls, top_name, top_kernel = TB.PROF_LM_HEAD, "lm_head", "k_gemv (LM head)"
     g.profile_begin(top_cls)
-    sampler.mark_begin()
+    if sampler:
+        sampler.mark_begin()
     wall0 = time.perf_counter()
     for i in range(K):
         flush.zero_()                       # the target model's pass between rounds evicts L2 in deployment
@@ -406,27 +426,42 @@ def run_ours(args, wl):
     head_ms, head_n = g.profile_end()       # synchronises the stream
     torch.cuda.synchronize(device)
     wall = time.perf_counter() - wall0
-    sampler.mark_end()
-    dev_err = int(g.debug_view(TB.VIEW_ERROR_FLAG).cpu()[0])
+    if sampler:
+        sampler.mark_end()
+    dev_err = g.last_device_error()
     if dev_err != 0:                        # a bounded wait ran out or a cache overflowed: the timing means nothing
-        raise RuntimeError(f"device-side error flag {dev_err} after the timed rounds")
+        raise RuntimeError(f"device-side error {dev_err} after the timed rounds of {wl.name}")
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(device)
-    clocks = sampler.stop()
+    clocks = sampler.stop() if sampler else None
     launches = g.launch_count() - launches0
     per_round = np.array([s.elapsed_time(e) for s, e in ev])
-    from paper_2601_20357_b200.replicas import whole_job
     dev_ms, _, value = whole_job(float(per_round.sum()), B * K, dist, device)     # slowest rank's time, all ranks' rounds
 
     peak, peak_kind = read_peaks()
     cb = class_bytes(wl, kv_tokens_total, mean_accept)
     head_dur = head_ms / max(head_n, 1)
     head_gbs = cb[top_name] / (head_dur * 1e-3) / 1e9
+    round_bytes = int(cb["draft_round"] + cb["verify"] + cb["update"])
+    res = {
+        "wl": wl, "value": value, "dev_ms": dev_ms, "ms_per_step": dev_ms / K, "mean_accept": mean_accept, "wall": wall,
+        "launches": int(launches), "clocks": clocks, "path": {TB.PATH_PERSISTENT: "persistent", TB.PATH_TENSOR_CORE: "tensor-core projections",
+                                                            TB.PATH_PER_OP: "per-operation"}[cur_path],
+        "roofline": {"kernel": top_kernel, "bound": "hbm", "achieved": head_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": head_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": (NCU_TRAFFIC.get((wl.name, top_name)) or {}).get("bytes"),
+                     "traffic_note": NCU_TRAFFIC.get((wl.name, top_name)),
+                     "avg_us": 1000.0 * head_dur, "launches_timed": head_n, "bytes_per_launch": int(cb[top_name]),
+                     "share_of_round": head_ms / K / (dev_ms / K)},
+        "round_roofline": {"bytes_per_round": round_bytes, "achieved_gbs": round_bytes / (dev_ms / K * 1e-3) / 1e9,
+                           "frac": round_bytes / (dev_ms / K * 1e-3) / 1e9 / peak,
+                           "note": "algorithmic bytes of one round / measured round time / peak"},
+        "kernels": {}, "e2e": None,
+    }
 
     # ---- per-class breakdown (separate untimed-for-the-headline passes over the same rounds) ----
-    kernels = {}
-    if rank == 0 and not args.no_breakdown:
+    if rank == 0 and breakdown:
         names = ["qkv", "attention", "oproj", "gateup", "down", "lm_head", "ensemble", "verify", "update", "draft_round"]
         nb = min(K, 12)
         for cls, nm in enumerate(names):
@@ -441,15 +476,14 @@ def run_ours(args, wl):
                 one_round(Wm + i)
             ms, n = g.profile_end()
             dur = ms / max(n, 1)
-            kernels[nm] = {"intervals_per_round": n / nb, "avg_us": 1000.0 * dur, "bytes": int(cb[nm]),
-                           "gbs": cb[nm] / (dur * 1e-3) / 1e9 if dur > 0 else None,
-                           "frac_of_peak": cb[nm] / (dur * 1e-3) / 1e9 / peak if dur > 0 else None,
-                           "share_of_round": ms / nb / float(per_round.mean())}
+            res["kernels"][nm] = {"intervals_per_round": n / nb, "avg_us": 1000.0 * dur, "bytes": int(cb[nm]),
+                                  "gbs": cb[nm] / (dur * 1e-3) / 1e9 if dur > 0 else None,
+                                  "frac_of_peak": cb[nm] / (dur * 1e-3) / 1e9 / peak if dur > 0 else None,
+                                  "share_of_round": ms / nb / float(per_round.mean())}
 
     # ---- end to end through the host-buffer entry point ----
-    e2e = None
-    if rank == 0 and args.e2e_steps > 0:
-        ne = min(args.e2e_steps, K)
+    if rank == 0 and e2e_steps > 0:
+        ne = min(e2e_steps, K)
         g.state_import(snap)
         for r in range(Wm):
             one_round(r)
@@ -466,15 +500,16 @@ def run_ours(args, wl):
             g.round_host(hu[i][0], hu[i][1], hu[i][2], hu[i][3], h_toks, h_a, h_z, h_w, h_am)
         dt = time.perf_counter() - t0
         h2d = sum(x.numel() * x.element_size() for x in hu[0])
-        d2h = sum(x.numel() * x.element_size() for x in (h_toks, h_a, h_z, h_am, h_w))
-        e2e = {"value": B * ne / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-               "steps": ne, "note": "tabed_round_host, pinned host buffers, L2 not flushed between rounds"}
+        d2h = sum(x.numel() * x.element_size() for x in (h_toks, h_a, h_z, h_am, h_w)) + 4
+        res["e2e"] = {"value": B * ne / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                      "steps": ne, "note": "tabed_round_host, pinned host buffers, L2 not flushed between rounds; the device-side "
+                                           "error word is read back with the results"}
 
-    if rank == 0 and args.trace and persistent:
+    if rank == 0 and trace and persistent:
         g.state_import(snap)
         for r in range(Wm):
             one_round(r)
-        g.debug_trace(True, args.trace_cta)
+        g.debug_trace(True, trace_cta)
         flush.zero_()
         g.draft_round(u[Wm][0], toks)
         torch.cuda.synchronize(device)
@@ -482,65 +517,97 @@ def run_ours(args, wl):
         tr = g.debug_view(TB.VIEW_TRACE).cpu().numpy().astype(np.int64)
         g.verify(targets[Wm], u[Wm][1], u[Wm][2], a, z)
         g.update_weights(w, am)
-        L = wl.drafter.n_layers
-        nb_step = 5 * L + 3
-        names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "gateup", "down")] + ["lm_head", "expsum", "mix"]
-        mhz = float(clocks.get("sm_mhz") or 1965.0)
-        with open(args.trace, "w") as f:
-            f.write("# made by: python " + " ".join(a if a != args.trace else "<this file>" for a in sys.argv) + "\n")
-            f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA {args.trace_cta}): us from the previous grid barrier to this one,\n"
-                    f"# then that CTA's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
-                    f"# (attention phases: load+stage q/k/v, scores+softmax, PV+write, split merge, -, barrier)\n")
-            prev = None
-            for st in range(G):
-                for j in range(nb_step):
-                    tcur = int(tr[st, j, 0])
-                    secs = " ".join(f"{int(c) / mhz:7.2f}" for c in tr[st, j, 1:7])
-                    f.write(f"step {st} {names_b[j]:>12s} {((tcur - prev) / 1000.0 if prev is not None else 0.0):8.2f}   {secs}\n")
-                    prev = tcur
-            f.write(f"# first barrier to last barrier: {(int(tr[G - 1, nb_step - 1, 0]) - int(tr[0, 0, 0])) / 1000.0:.1f} us\n")
+        write_trace(trace, trace_cta, wl, tr, float((clocks or {}).get("sm_mhz") or 1965.0))
+    g.destroy()
+    del targets, flush
+    torch.cuda.empty_cache()
+    return res
 
+
+def write_trace(path, cta, wl, tr, mhz):
+    L, G = wl.drafter.n_layers, wl.gamma
+    nb_step = 5 * L + 3
+    names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "gateup", "down")] + ["lm_head", "expsum", "mix"]
+    with open(path, "w") as f:
+        f.write("# made by: python " + " ".join(a if a != path else "<this file>" for a in sys.argv) + "\n")
+        f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA {cta}): us from the previous grid barrier to this one,\n"
+                f"# then that CTA's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
+                f"# (attention phases: load+stage q/k/v, scores+softmax, PV+write, split merge, -, barrier)\n")
+        prev = None
+        for st in range(G):
+            for j in range(nb_step):
+                tcur = int(tr[st, j, 0])
+                secs = " ".join(f"{int(c) / mhz:7.2f}" for c in tr[st, j, 1:7])
+                f.write(f"step {st} {names_b[j]:>12s} {((tcur - prev) / 1000.0 if prev is not None else 0.0):8.2f}   {secs}\n")
+                prev = tcur
+        f.write(f"# first barrier to last barrier: {(int(tr[G - 1, nb_step - 1, 0]) - int(tr[0, 0, 0])) / 1000.0:.1f} us\n")
+
+
+def run_ours(args, wl):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+    K, Wm = args.steps, args.warmup
+    r = measure(wl, device, K, Wm, rank=rank, dist=dist, path=args.path, breakdown=not args.no_breakdown, e2e_steps=args.e2e_steps,
+                trace=args.trace, trace_cta=args.trace_cta, clock_index=local)
+    wl = r["wl"]
+    # ---- the other workloads of the paper's shape, a few dozen rounds each (one GPU only) ----
+    per_config = {}
+    if rank == 0 and world == 1 and not args.no_per_config and args.path == "auto":
+        for name in ("tiny", "llava_small", "large_vocab", "long_context", "batched_serving"):
+            if name == wl.name:
+                o = r
+            else:
+                o = measure(W.WORKLOADS[name], device, min(K, 30), 3)
+            per_config[name] = {
+                "ms_per_step": o["ms_per_step"], "rounds_per_sec": o["value"], "drafted_tokens_per_sec": o["value"] * o["wl"].gamma,
+                "block_efficiency": o["mean_accept"] + 1.0, "path": o["path"], "rows": o["wl"].n_rows,
+                "dominant_kernel": o["roofline"]["kernel"].split(" ")[0], "dominant_kernel_frac": o["roofline"]["frac"],
+                "dominant_kernel_us": o["roofline"]["avg_us"], "dominant_kernel_share_of_round": o["roofline"]["share_of_round"],
+                "round_frac": o["round_roofline"]["frac"], "bytes_per_round": o["round_roofline"]["bytes_per_round"]}
     if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
         return
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        n_cpu = args.cpu_rounds
-        v, dt = time_oracle(wl, n_cpu, 0)
+        sub = oracle_sample(wl)
+        v, dt, done = time_oracle(sub, args.cpu_rounds, 0, budget_s=25.0)
         cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-               "sample": f"first {n_cpu} rounds of {wl.name} (whole rounds, prefill untimed), {dt:.1f} s"}
+               "sample": f"first {done} whole rounds of the first {sub.n_requests} of {wl.n_requests} requests of {wl.name} "
+                         f"({sub.n_rows} rows, their full caches; prompt feeding / cache loading untimed), {dt:.1f} s; "
+                         "value = requests x rounds / time"}
+    G = wl.gamma
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 accumulate over bf16 weights/KV" if wl.drafter.dtype == "bf16" else "f32",
         "data": "synthetic",
-        "config": {"workload": wl.name, "n_inputs": m, "n_requests": B, "rows": wl.n_rows, "gamma": G,
-                   "window_h": wl.window_h, "vocab": V, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model,
-                   "l2": "256 MB written between rounds (stands for the target model's pass); rounds timed one by one "
-                         "with CUDA events", "parallelism": f"replicas x{world}",
-                   "path": {TB.PATH_PERSISTENT: "persistent", TB.PATH_TENSOR_CORE: "tensor-core projections",
-                            TB.PATH_PER_OP: "per-operation"}[g.current_path()]},
-        "drafted_tokens_per_sec": value * G,
-        "block_efficiency": mean_accept + 1.0,
-        "wall_ms_per_step_incl_flush": 1000.0 * wall / K,
-        "roofline": {"kernel": top_kernel, "bound": "hbm", "achieved": head_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": head_gbs / peak, "peak_kind": peak_kind,
-                     "traffic": (NCU_TRAFFIC.get((wl.name, top_name)) or {}).get("bytes"),
-                     "traffic_note": NCU_TRAFFIC.get((wl.name, top_name)),
-                     "avg_us": 1000.0 * head_dur, "launches_timed": head_n, "bytes_per_launch": int(cb[top_name])},
-        "round_roofline": {"bytes_per_round": int(cb["draft_round"] + cb["verify"] + cb["update"]),
-                           "note": "algorithmic bytes of one round / measured round time / peak"},
-        "kernels": kernels,
+        "config": config_of(wl),
+        "details": {"l2": "256 MB written between rounds (stands for the target model's pass); rounds timed one by one "
+                          "with CUDA events", "parallelism": f"replicas x{world}", "path": r["path"]},
+        "drafted_tokens_per_sec": r["value"] * G,
+        "block_efficiency": r["mean_accept"] + 1.0,
+        "wall_ms_per_step_incl_flush": 1000.0 * r["wall"] / K,
+        "roofline": r["roofline"],
+        "round_roofline": r["round_roofline"],
+        "kernels": r["kernels"],
+        "per_config": per_config,
         "cpu_baseline": cpu,
-        "e2e": e2e,
-        "gpu_launches": int(launches),
-        "clocks": clocks,
+        "e2e": r["e2e"],
+        "gpu_launches": r["launches"],
+        "clocks": r["clocks"],
         "context": PAPER_CONTEXT,
     }
-    rr = line["round_roofline"]
-    rr["achieved_gbs"] = rr["bytes_per_round"] / (dev_ms / K * 1e-3) / 1e9
-    rr["frac"] = rr["achieved_gbs"] / peak
     print(json.dumps(line), flush=True)
-    g.destroy()
     if dist is not None:
         dist.destroy_process_group()
 
@@ -548,12 +615,14 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="llava_small", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--config", default="batched_serving", choices=sorted(W.WORKLOADS),
+                    help="workload of the headline line (default: the largest single-GPU one, 32 requests x 3 inputs)")
     ap.add_argument("--e2e-steps", type=int, default=50)
-    ap.add_argument("--cpu-rounds", type=int, default=60)
+    ap.add_argument("--cpu-rounds", type=int, default=60, help="at most this many rounds of the CPU checker (and at most ~25 s)")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--trace", default=None, help="write the persistent kernel's phase timeline of one round to this file")

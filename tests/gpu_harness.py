@@ -16,15 +16,30 @@ from paper_2601_20357_b200 import workloads as W
 
 DEV = torch.device("cuda", 0)
 
-# |logit_gpu - logit_oracle|.  fp32 drafter: fp32 accumulation against fp64, ~1e-6 relative.
-# bf16 drafter: every matmul input is rounded to bf16; a value that the two sides compute ~1e-7 apart
-# can fall on different sides of a rounding boundary (one step = 2^-8 relative), and the cache of a
-# few hundred prefix positions holds ~10^6 such roundings, so the two forward passes differ like two
-# runs of the checker with a 1e-7 relative perturbation before every rounding: mean |dlogit| ~3e-3,
-# max ~2e-2 on the LLaVA-like config (tests/test_oracle_drafter.py measures this on a small model).
-# Probabilities are ~1/V, so the 1e-5 absolute bar on them is met with a wide margin either way.
-LOGIT_TOL = {"fp32": 2e-5, "bf16": 6e-2}
-LOGIT_MEAN_TOL = {"fp32": 2e-6, "bf16": 1e-2}
+# |logit_gpu - logit_oracle| in the lock-step rounds, where each side builds its own caches.
+# fp32 drafter: fp32 accumulation against fp64, ~1e-6 relative.  bf16 drafter: every matmul input is rounded to
+# bf16; a value that the two sides compute ~1e-7 apart can fall on different sides of a rounding boundary (one
+# step = 2^-8 relative), and the caches hold ~10^6 such roundings, so the two forward passes differ like two runs
+# of the checker with a 1e-7 relative perturbation before every rounding (tests/test_oracle_drafter.py measures
+# that on a small model).  How far depends on depth and width, so the bound is per workload: three times the
+# largest (max, mean) of |dlogit| observed on a B200 over all rounds of all tests of that workload.
+# tests/test_gpu_forward_tight.py has the sharper check (identical caches, one step).
+LOCKSTEP_OBSERVED = {
+    "tiny": (2.1e-7, 3.3e-8),               # 2 layers, d = 128, fp32
+    "llava_small": (1.7e-2, 2.1e-3),        # 4 layers, d = 768
+    "large_vocab": (4.0e-2, 4.0e-3),        # 12 layers, d = 896
+    "long_context": (1.6e-2, 1.9e-3),       # 4 layers, d = 768, 8192 cached positions
+    "batched_serving": (1.9e-2, 2.2e-3),    # 4 layers, d = 768, 96 rows
+}
+LOCKSTEP_OBSERVED_OTHER = {"fp32": (2.1e-7, 3.3e-8), "bf16": (1.2e-2, 1.6e-3)}     # the tests' two-layer drafters (d <= 896)
+
+
+def logit_tols(wl):
+    """(max, mean) bound on |dlogit| of a lock-step round of this workload."""
+    obs = LOCKSTEP_OBSERVED.get(wl.name.split("[")[0], LOCKSTEP_OBSERVED_OTHER[wl.drafter.dtype])
+    return 3.0 * obs[0], 3.0 * obs[1]
+
+
 PROB_TOL = 1e-5           # tolerance on probabilities (the bar the library is built to)
 
 
@@ -178,8 +193,10 @@ def lockstep_round(p: Pair, rnd: int, override: bool = True):
     own = g.debug_view(TB.VIEW_LOGITS).clone()
     diff = (own.cpu().numpy().astype(np.float64) - logits_o.astype(np.float64))
     dt = wl.drafter.dtype
-    assert np.max(np.abs(diff)) <= LOGIT_TOL[dt], f"logits max err {np.max(np.abs(diff))}"
-    assert np.mean(np.abs(diff)) <= LOGIT_MEAN_TOL[dt], f"logits mean err {np.mean(np.abs(diff))}"
+    print(f"LOCKSTEP {wl.name} {dt} round {rnd}: max |dlogit| {np.max(np.abs(diff)):.3e} mean {np.mean(np.abs(diff)):.3e}")
+    tol_max, tol_mean = logit_tols(wl)
+    assert np.max(np.abs(diff)) <= tol_max, f"logits max err {np.max(np.abs(diff))} > {tol_max}"
+    assert np.mean(np.abs(diff)) <= tol_mean, f"logits mean err {np.mean(np.abs(diff))} > {tol_mean}"
     qk_own = torch.empty((B, m, V), dtype=torch.float32, device=DEV)
     y_tmp = torch.empty(B, dtype=torch.int32, device=DEV)
     for i in range(G):

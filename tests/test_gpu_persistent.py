@@ -109,7 +109,7 @@ def test_free_run_matches_per_operation_path_on_first_round():
     torch.cuda.synchronize()
     la = a.gpu.debug_view(TB.VIEW_LOGITS)[0].cpu().numpy()
     lb = b.gpu.debug_view(TB.VIEW_LOGITS)[0].cpu().numpy()
-    assert np.max(np.abs(la - lb)) <= H.LOGIT_TOL["bf16"]
+    assert np.max(np.abs(la - lb)) <= 2 * H.logit_tols(wl)[0]        # two CUDA paths, each within the bound of the checker
     H.check_error_flag(a.gpu)
     # the in-kernel ensemble on the kernel's own logits (row maxima gathered by the LM-head epilogue)
     # equals, bit for bit, the stand-alone ensemble step applied to those logits
