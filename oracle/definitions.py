@@ -11,7 +11,8 @@ blocking, fusion or reordering:
 * KL divergence, total variation distance ... Sec. 4.1 (error e_t^j), TVD variant
 * acceptance probability, residual law ...... Sec. 3, item 3
 * emitted-token law of one SD position ...... Sec. 3 (distribution preserved)
-* weight policies ........................... App. B "Weight Sampling Policy"
+* weight policies ........................... App. B "Weight Sampling Policy"; hard labels (Sec. 4.1); Random
+                                              ablation (Sec. 5); TABED-AdaBoost (appendix)
 * expected walltime speedup ................. Eq. 1
 """
 from __future__ import annotations
@@ -90,6 +91,41 @@ def policy_grid(p_window, qk_window, n_grid: int = 10):
             G[j] += kl_divergence(p, ensemble(qk, w), q_floor=np.finfo(np.float32).tiny)
     j_star = int(np.argmin(G))
     return j_star, cands[j_star], G
+
+
+def policy_random(u: np.ndarray) -> np.ndarray:
+    """Non-negative, sum-to-one random weights (Sec. 5 "Effectiveness of Dynamic Weights", the Random ablation):
+    a point drawn uniformly from the simplex, w_k = g_k / sum_j g_j with g_k = -ln u_k, u_k uniform in (0, 1)."""
+    g = -np.log(np.asarray(u, np.float64))
+    return g / g.sum()
+
+
+def hard_label_matches(qk: np.ndarray, label: int, n_grid: int = 10) -> np.ndarray:
+    """Hard-label score of every grid candidate at one verified position (Sec. 4.1, "utilizing hard labels"): 1 if the
+    token the candidate's ensemble q^j = (1 - j/n) q^(1) + (j/n) q^(2) would emit (its most likely token, lowest id on
+    ties) is the verified token, else 0.  qk [2][V].  Returns [n_grid + 1]."""
+    return np.array([int(int(np.argmax(ensemble(qk, w))) == int(label)) for w in grid_candidates(n_grid)], np.int64)
+
+
+def policy_grid_hard(label_window, qk_window, n_grid: int = 10):
+    """argmax_j of the number of token matches over the window (lowest j on ties).  Returns (j*, w*, counts[j])."""
+    counts = np.zeros(n_grid + 1, np.int64)
+    for y, qk in zip(label_window, qk_window):
+        counts += hard_label_matches(qk, y, n_grid)
+    j_star = int(np.argmax(counts))
+    return j_star, grid_candidates(n_grid)[j_star], counts
+
+
+def policy_adaboost(errors: np.ndarray, n: int, vocab: int, c: float = 1.0) -> np.ndarray:
+    """TABED-AdaBoost (App. "TABED-AdaBoost: A Theoretically Grounded Variant"): w_m = ln(1/eps_m - 1) + C ln(K - 1) with
+    eps_m the error rate of drafting method m, here the smoothed fraction (errors_m + 1) / (n + 2) of the n verified
+    positions of the window at which the method's most likely token was not the verified token; K the vocabulary
+    size.  The ensemble needs non-negative weights that sum to one: negative values are cut at 0 and the rest is
+    normalised (equal weights if nothing is left)."""
+    eps = (np.asarray(errors, np.float64) + 1.0) / (n + 2.0)
+    w = np.maximum(np.log(1.0 / eps - 1.0) + c * np.log(vocab - 1.0), 0.0)
+    s = w.sum()
+    return w / s if s > 0 else np.full(len(w), 1.0 / len(w))
 
 
 def pool_image_tokens_2x2(x: np.ndarray, grid_h: int, grid_w: int) -> np.ndarray:

@@ -200,3 +200,40 @@ def policy_softmax_inv_err(e, tau=1.0) -> np.ndarray:
     for k in range(1, len(x)):
         tot = F(tot + x[k])
     return (x / tot).astype(F)
+
+
+def policy_random(u) -> np.ndarray:
+    """Random non-negative sum-to-one weights from uniforms on the lattice: g_k = -xlog(u_k), w_k = g_k / (((g_0 + g_1)
+    + g_2) + ...)."""
+    g = -xlog(np.asarray(u, F))
+    tot = g[0]
+    for k in range(1, len(g)):
+        tot = F(tot + g[k])
+    return (g / tot).astype(F)
+
+
+def grid_hard_matches(qk, label: int, n_grid: int = 10) -> np.ndarray:
+    """Per grid candidate j: 1 if argmax_v of the fp32 ensemble c0 q^(0) + c1 q^(1) (lowest id on ties) is `label`."""
+    return np.array([int(argmax_lowest(ensemble_exact(qk, grid_weight(j, n_grid))) == int(label)) for j in range(n_grid + 1)],
+                    np.int64)
+
+
+def drafter_errors(qk, label: int) -> np.ndarray:
+    """Per drafting method k: 1 if argmax_v q^(k)_v (lowest id on ties) is NOT `label`."""
+    return np.array([int(argmax_lowest(qk[k]) != int(label)) for k in range(len(qk))], np.int64)
+
+
+def policy_adaboost(errors, n: int, vocab: int, c=1.0) -> np.ndarray:
+    """w_k = max(0, xlog(1/eps_k - 1) + c * xlog(K - 1)) normalised; eps_k = (errors_k + 1) / (n + 2); every step one
+    rounded fp32 operation, the sum taken in k order; equal weights if every value is cut to 0."""
+    errors = np.asarray(errors, np.int64)
+    eps = (errors.astype(F) + F(1)) / F(F(n) + F(2))
+    a = F(1) / eps
+    t = xlog(a - F(1)) + F(F(c) * xlog(np.array([F(vocab - 1)], F))[0])
+    t = np.maximum(t, F(0)).astype(F)
+    tot = t[0]
+    for k in range(1, len(t)):
+        tot = F(tot + t[k])
+    if not tot > 0:
+        return policy_static(len(t))
+    return (t / tot).astype(F)

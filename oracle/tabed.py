@@ -26,7 +26,7 @@ from . import exact32 as x32
 
 F = np.float32
 
-POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR = 0, 1, 2
+POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR, POLICY_RANDOM, POLICY_GRID_HARD, POLICY_ADABOOST = 0, 1, 2, 3, 4, 5
 DIST_KL, DIST_TVD = 0, 1
 MODE_SAMPLE, MODE_GREEDY = 0, 1
 N_GRID = 10
@@ -39,11 +39,11 @@ class TabedOracle:
         self.m, self.B, self.gamma, self.h = n_inputs, n_requests, gamma, window_h
         self.policy, self.V = policy, vocab
         self.distance, self.mode, self.tau = distance, sample_mode, tau
-        if policy == POLICY_GRID_MT and n_inputs != 2:
-            raise ValueError("the grid policy is defined for two drafting methods")
+        if policy in (POLICY_GRID_MT, POLICY_GRID_HARD) and n_inputs != 2:
+            raise ValueError("the grid policies are defined for two drafting methods")
         self.w = np.tile(x32.policy_static(n_inputs), (n_requests, 1))          # [B][m]
         self.j_star = np.full(n_requests, -1, np.int32)
-        n_dev = (N_GRID + 1) if policy == POLICY_GRID_MT else n_inputs
+        n_dev = (N_GRID + 1) if policy in (POLICY_GRID_MT, POLICY_GRID_HARD) else n_inputs
         self.n_dev = n_dev
         self.window = [deque() for _ in range(n_requests)]      # entries: int64 [n_dev]
         self.running = np.zeros((n_requests, n_dev), np.int64)  # h == 0: all history
@@ -160,21 +160,32 @@ class TabedOracle:
         return self.n_accept, self.next_token
 
     # ---- Sec. 4.1 deviation; App. B policies; Algorithm 1 steps 2-3 --------------
-    def _deviation(self, p: np.ndarray, qk: np.ndarray) -> np.ndarray:
+    def _deviation(self, p: np.ndarray, qk: np.ndarray, label: int) -> np.ndarray:
+        """What one verified position contributes to the window: soft labels -> the distance of every drafter (or grid
+        candidate) from p; hard labels -> whether each grid candidate's most likely token is the verified token
+        (Sec. 4.1), or, for the AdaBoost variant, whether each drafter's most likely token is NOT it (its error)."""
+        if self.policy == POLICY_GRID_HARD:
+            return x32.grid_hard_matches(qk, label, N_GRID)
+        if self.policy == POLICY_ADABOOST:
+            return x32.drafter_errors(qk, label)
         dist = x32.tvd_fixed if self.distance == DIST_TVD else x32.kl_fixed
         if self.policy == POLICY_GRID_MT:
             return np.array([dist(p, x32.ensemble_exact(qk, x32.grid_weight(j, N_GRID)))
                              for j in range(N_GRID + 1)], np.int64)
         return np.array([dist(p, qk[k]) for k in range(self.m)], np.int64)
 
-    def update_weights(self):
+    def update_weights(self, u_policy=None):
         """Push the round's verified positions into the window, choose w* for the next block,
-        and advance the caches / pending tokens.  Returns (w [B][m], w_argmax [B])."""
+        and advance the caches / pending tokens.  u_policy [B][m]: uniforms of the Random policy.
+        Returns (w [B][m], w_argmax [B])."""
         G = self.gamma
+        self.u_policy = u_policy
         for b in range(self.B):
             a = int(self.n_accept[b])
             for i in range(min(a, G - 1) + 1):
-                dev = self._deviation(self.p[b, i], self.qk[b, i])
+                # the verified token of position i: the accepted draft, or the replacement at the rejected position
+                label = int(self.tokens[b, i]) if i < a else int(self.next_token[b])
+                dev = self._deviation(self.p[b, i], self.qk[b, i], label)
                 self.running[b] += dev
                 self.count[b] += 1
                 if self.h > 0:
@@ -194,8 +205,16 @@ class TabedOracle:
         return self.w.copy(), np.argmax(self.w, axis=1).astype(np.int32)
 
     def _policy(self, b: int) -> np.ndarray:
+        if self.policy == POLICY_RANDOM:
+            return x32.policy_random(self.u_policy[b])
         if self.policy == POLICY_STATIC or self.count[b] == 0:
             return x32.policy_static(self.m)
+        if self.policy == POLICY_GRID_HARD:
+            self.j_star[b] = int(np.argmax(self.running[b]))            # most matches, lowest j on ties
+            return x32.grid_weight(int(self.j_star[b]), N_GRID)
+        if self.policy == POLICY_ADABOOST:
+            n = len(self.window[b]) if self.h > 0 else int(self.count[b])
+            return x32.policy_adaboost(self.running[b], n, self.V, self.tau)   # tau holds the constant C
         tvd = self.distance == DIST_TVD
         if self.policy == POLICY_GRID_MT:
             self.j_star[b] = int(np.argmin(self.running[b]))            # lowest j on ties

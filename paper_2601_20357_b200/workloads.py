@@ -27,6 +27,9 @@ MASTER_SEED = 0x7ABED
 POLICY_STATIC = 0
 POLICY_GRID_MT = 1
 POLICY_SOFTMAX_INV_ERR = 2
+POLICY_RANDOM = 3
+POLICY_GRID_HARD = 4
+POLICY_ADABOOST = 5
 
 DIST_KL = 0
 DIST_TVD = 1
@@ -310,6 +313,11 @@ def round_uniforms(wl: Workload, rnd: int) -> Tuple[np.ndarray, np.ndarray, np.n
     G = wl.gamma
     return (np.ascontiguousarray(u[:, :G]), np.ascontiguousarray(u[:, G:2 * G]),
             np.ascontiguousarray(u[:, 2 * G]))
+
+
+def policy_uniforms(wl: Workload, rnd: int) -> np.ndarray:
+    """Uniforms of the Random weight policy for one round, [B][m], on the same lattice as the draws."""
+    return lattice_uniforms(substream(wl.config_id, "policy_uniforms", rnd), (wl.n_requests, wl.n_inputs))
 
 
 def request_alpha(wl: Workload) -> np.ndarray:

@@ -350,3 +350,91 @@ def test_pool_2x2_closed_forms_and_token_count():
     for bad in ((3, 4), (4, 3)):
         with pytest.raises(ValueError):
             pool_image_tokens_2x2(np.zeros((12, 1), np.float32), *bad)
+
+
+# ---------------------------------------------------------------- the other weight policies
+def test_random_policy_is_uniform_on_the_simplex():
+    """Sec. 5 "Effectiveness of Dynamic Weights": non-negative sum-to-one random weights.  A uniform point of the
+    simplex: every weight has mean 1/m and one coordinate follows Beta(1, m-1) (for two methods: uniform on (0, 1))."""
+    rng = np.random.default_rng(31)
+    for m in (2, 3, 5):
+        u = lat(rng, (4000, m))
+        w = np.stack([X.policy_random(u[i]) for i in range(len(u))]).astype(np.float64)
+        assert np.all(w >= 0) and np.allclose(w.sum(axis=1), 1.0, atol=1e-6)
+        np.testing.assert_allclose(w, np.stack([D.policy_random(u[i]) for i in range(len(u))]), atol=2e-6)
+        np.testing.assert_allclose(w.mean(axis=0), 1.0 / m, atol=0.02)
+        # marginal of one coordinate of a flat Dirichlet is Beta(1, m-1): P(w_0 <= x) = 1 - (1-x)^(m-1)
+        for x in (0.1, 0.3, 0.6):
+            assert abs(float((w[:, 0] <= x).mean()) - (1 - (1 - x) ** (m - 1))) < 0.03
+    o = mk(m=3, B=2, gamma=2, h=2, V=50, policy=W.POLICY_RANDOM)
+    lg = rand_logits(rng, 2, 2, 3, 50)
+    o.draft_round_logits(lg, lat(rng, (2, 2)))
+    o.verify(rng.standard_normal((2, 3, 50)).astype(F), lat(rng, (2, 2)), lat(rng, (2,)))
+    up = lat(rng, (2, 3))
+    w, am = o.update_weights(up)
+    assert np.array_equal(w[0], X.policy_random(up[0])) and np.array_equal(w[1], X.policy_random(up[1]))
+
+
+def test_hard_label_grid_selection_counts_token_matches():
+    """Sec. 4.1: with hard labels w* maximises the number of token matches over the window."""
+    rng = np.random.default_rng(32)
+    G, V = 3, 40
+    o = mk(m=2, B=1, gamma=G, h=0, V=V, policy=W.POLICY_GRID_HARD)
+    labels, qks = [], []
+    for rnd in range(5):
+        lg = rand_logits(rng, G, 1, 2, V, 2.0)
+        o.draft_round_logits(lg, lat(rng, (1, G)))
+        tl = np.concatenate([lg[:, :, 1, :], lg[-1:, :, 1, :]], axis=0).transpose(1, 0, 2)      # the target follows drafter 1
+        tl = (3.0 * tl + 0.5 * rng.standard_normal(tl.shape)).astype(F)
+        a, z = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+        for i in range(min(int(a[0]), G - 1) + 1):
+            labels.append(int(o.tokens[0, i]) if i < a[0] else int(z[0])); qks.append(o.qk[0, i].copy())
+        w, am = o.update_weights()
+        j_def, w_def, counts = D.policy_grid_hard(labels, qks)
+        assert np.array_equal(o.running[0], counts) and int(o.j_star[0]) == j_def
+        np.testing.assert_allclose(w[0], w_def, atol=1e-7)
+        assert counts.max() <= len(labels) and counts.min() >= 0
+    # one-sided cases: only drafter 0 ever points at the verified token -> j* = 0 (w = [1, 0]); only drafter 1 -> j* = 10
+    for good in (0, 1):
+        qk = np.full((2, V), 0.5 / (V - 1))
+        qk[good, 7] = 0.5; qk[1 - good, 9] = 0.5
+        qk /= qk.sum(axis=1, keepdims=True)
+        m_ = X.grid_hard_matches(qk.astype(F), 7)
+        assert m_[0 if good == 0 else 10] == 1 and m_[10 if good == 0 else 0] == 0
+        assert np.array_equal(m_, D.hard_label_matches(qk.astype(F), 7))
+        j, wj, _ = D.policy_grid_hard([7], [qk.astype(F)])
+        assert j == (0 if good == 0 else int(np.argmax(m_))) and wj[good] >= 0.5
+
+
+def test_adaboost_weights_follow_the_printed_formula():
+    """w_m = ln(1/eps_m - 1) + C ln(K - 1), normalised; the lower a method's error rate the larger its weight."""
+    K = 32000
+    w = X.policy_adaboost(np.array([2, 5, 9]), 10, K, 1.0).astype(np.float64)
+    eps = (np.array([2, 5, 9]) + 1.0) / 12.0
+    raw = np.log(1.0 / eps - 1.0) + np.log(K - 1.0)
+    np.testing.assert_allclose(w, raw / raw.sum(), atol=2e-6)
+    np.testing.assert_allclose(w, D.policy_adaboost(np.array([2, 5, 9]), 10, K, 1.0), atol=2e-6)
+    assert w[0] > w[1] > w[2] and abs(w.sum() - 1) < 1e-6 and np.all(w >= 0)
+    eq = X.policy_adaboost(np.array([3, 3, 3, 3]), 8, K, 1.0)
+    assert np.all(eq == eq[0]) and abs(float(eq[0]) - 0.25) < 1e-7
+    # C = 0 and a method that is wrong more often than right: its term is negative, cut at 0
+    w0 = X.policy_adaboost(np.array([1, 9]), 10, K, 0.0)
+    assert w0[1] == 0 and w0[0] == 1
+    assert np.array_equal(X.policy_adaboost(np.array([9, 9]), 10, K, 0.0), X.policy_static(2))
+    # inside the round machine: errors are counted against the verified tokens over the window
+    rng = np.random.default_rng(33)
+    G, V, m = 3, 60, 3
+    o = mk(m=m, B=1, gamma=G, h=4, V=V, policy=W.POLICY_ADABOOST, tau=1.0)
+    errs = []
+    for rnd in range(4):
+        lg = rand_logits(rng, G, 1, m, V, 2.0)
+        o.draft_round_logits(lg, lat(rng, (1, G)))
+        tl = np.concatenate([lg[:, :, 0, :], lg[-1:, :, 0, :]], axis=0).transpose(1, 0, 2)
+        tl = (3.0 * tl + 0.3 * rng.standard_normal(tl.shape)).astype(F)
+        a, z = o.verify(tl, lat(rng, (1, G)), lat(rng, (1,)))
+        for i in range(min(int(a[0]), G - 1) + 1):
+            label = int(o.tokens[0, i]) if i < a[0] else int(z[0])
+            errs.append([int(int(np.argmax(o.qk[0, i, k])) != label) for k in range(m)])
+        w, am = o.update_weights()
+        win = np.array(errs[-4:])
+        np.testing.assert_allclose(w[0], D.policy_adaboost(win.sum(axis=0), len(win), V, 1.0), atol=2e-6)
