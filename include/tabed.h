@@ -63,6 +63,15 @@ extern "C" {
 #define TABED_POLICY_STATIC          0   /* w_k = 1/m (the paper's Static baseline)              */
 #define TABED_POLICY_GRID_MT         1   /* m = 2: w^j = [1-j/10, j/10], j = 0..10, argmin error  */
 #define TABED_POLICY_SOFTMAX_INV_ERR 2   /* w = softmax(1/e^(1..m); tau)                          */
+#define TABED_POLICY_RANDOM          3   /* ablation of Sec. 5 ("Effectiveness of Dynamic Weights"): non-negative
+                                            sum-to-one random weights, a uniform point of the simplex drawn from
+                                            caller-supplied uniforms (tabed_set_policy_uniforms)     */
+#define TABED_POLICY_GRID_HARD       4   /* m = 2, hard labels (Sec. 4.1): the grid candidate whose most likely
+                                            token matched the verified token most often in the window  */
+#define TABED_POLICY_ADABOOST        5   /* appendix "TABED-AdaBoost": w_k = ln(1/eps_k - 1) + C ln(V - 1),
+                                            eps_k = (errors_k + 1) / (n + 2) over the n window positions (an error:
+                                            the drafter's most likely token is not the verified token), negative
+                                            values cut at 0, normalised; C = config.tau                */
 
 #define TABED_DIST_KL   0       /* D = KL(p || q)        */
 #define TABED_DIST_TVD  1       /* D = 1/2 sum |p - q|   */
@@ -117,7 +126,7 @@ typedef struct {
   int32_t policy;             /* TABED_POLICY_* */
   int32_t distance;           /* TABED_DIST_* */
   int32_t sample_mode;        /* TABED_MODE_* */
-  float   tau;                /* temperature of TABED_POLICY_SOFTMAX_INV_ERR, > 0 */
+  float   tau;                /* temperature of TABED_POLICY_SOFTMAX_INV_ERR; constant C of TABED_POLICY_ADABOOST; > 0 */
   int32_t kv_capacity;        /* tokens per row */
   int32_t device;             /* CUDA device ordinal */
   void*   stream;             /* cudaStream_t, caller-owned; NULL = legacy default stream */
@@ -138,7 +147,8 @@ typedef struct {
 /* Create a handle: validates the configuration, allocates every library-owned buffer, sets the
  * ensemble weights to 1/m (no history yet) and leaves every row cache empty.
  * Errors: NULL_PTR, INVALID_ARG (sizes out of range, head_dim not in {32,64,128}, d_model or
- * d_ffn not a multiple of 8, grid policy with m != 2), UNSUPPORTED, CUDA (allocation failed). */
+ * d_ffn not a multiple of 8, a grid policy with m != 2, a weight pointer that is not 16-byte aligned),
+ * UNSUPPORTED, CUDA (allocation failed). */
 int tabed_init(const tabed_config* cfg, const tabed_weights* weights, tabed_handle** out);
 
 /* Release everything tabed_init allocated.  NULL is accepted. */
@@ -211,6 +221,11 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
  * length += pending + (a < G ? a : G-1), pending <- {next_token} or {y_{G-1}, next_token}.
  * Outputs: out_w float [B][m], out_w_argmax int32 [B] (lowest index on ties); either may be NULL. */
 int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax);
+
+/* Uniforms of TABED_POLICY_RANDOM for the next tabed_update_weights: u_policy float [B][m] on the device, on
+ * the uniform lattice; the buffer must stay valid until that call has run.  w_k = g_k / sum_j g_j with
+ * g_k = -ln u_k.  tabed_update_weights returns TABED_ERR_BAD_STATE under that policy if none was ever set. */
+int tabed_set_policy_uniforms(tabed_handle* h, const float* u_policy);
 
 /* Host-buffer round: tabed_draft_round -> tabed_verify -> tabed_update_weights with HOST pointers
  * (pageable or pinned) for every argument, same shapes as above.  Copies the inputs to the

@@ -18,7 +18,7 @@ from . import build as _build
 OK = 0
 ERR_INVALID_ARG, ERR_NULL_PTR, ERR_BAD_STATE, ERR_KV_OVERFLOW, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_NUMERIC = range(-1, -9, -1)
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR = 0, 1, 2
+POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR, POLICY_RANDOM, POLICY_GRID_HARD, POLICY_ADABOOST = range(6)
 DIST_KL, DIST_TVD = 0, 1
 MODE_SAMPLE, MODE_GREEDY = 0, 1
 (VIEW_QK, VIEW_Q, VIEW_P, VIEW_LOGITS, VIEW_KV_LEN, VIEW_WEIGHTS, VIEW_WINDOW_SUM, VIEW_PENDING,
@@ -36,6 +36,7 @@ EXPORTS = [
     "tabed_launch_count", "tabed_profile_begin", "tabed_profile_end", "tabed_ensemble_step_static",
     "tabed_select_path", "tabed_current_path", "tabed_debug_trace", "tabed_debug_gemm_tc",
     "tabed_last_device_error", "tabed_sync_lengths", "tabed_debug_barrier_timeout", "tabed_static_last_error",
+    "tabed_set_policy_uniforms",
 ]
 
 
@@ -106,6 +107,7 @@ def lib() -> C.CDLL:
         L.tabed_current_path.argtypes = [vp]
         L.tabed_debug_trace.argtypes = [vp, i32]
         L.tabed_debug_gemm_tc.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, vp]
+        L.tabed_set_policy_uniforms.argtypes = [vp, vp]
         L.tabed_last_device_error.argtypes = [vp]
         L.tabed_sync_lengths.argtypes = [vp]
         L.tabed_debug_barrier_timeout.argtypes = [vp]
@@ -256,6 +258,11 @@ class Tabed:
                                   _ptr(u_resid, torch.float32, self.B, "u_resid", d),
                                   _ptr(out_n_accept, torch.int32, self.B, "out_n_accept", d),
                                   _ptr(out_next_token, torch.int32, self.B, "out_next_token", d)), "tabed_verify")
+
+    def set_policy_uniforms(self, u_policy: Optional[torch.Tensor]) -> None:
+        self._keep_u_policy = u_policy
+        _check(lib().tabed_set_policy_uniforms(self._h, _ptr(u_policy, torch.float32, self.R, "u_policy", self.device)),
+               "tabed_set_policy_uniforms")
 
     def update_weights(self, out_w=None, out_w_argmax=None) -> None:
         d = self.device

@@ -318,8 +318,9 @@ __global__ void __launch_bounds__(kDecThreads) k_select(SelectArgs A) {
 
 // ---- window push, policy, commit (Algorithm 1 steps 2-3; App. B) -----------------------------------
 struct PolicyArgs {
-  int B, G, m, n_dev, h, policy, tvd;
-  float tau;
+  int B, G, m, n_dev, h, policy, tvd, V;
+  float tau;                 // temperature of the softmax policy; the constant C of the AdaBoost policy
+  const float* u_policy;     // [B][m] uniforms of the random policy
   const int* n_accept; const int* next_token; const int* tokens;   // [B], [B], [B][G]
   long long* dev;            // [B][G][kMaxDev] deviation sums of the round's verified positions
   long long* ring;           // [B][h][kMaxDev]

@@ -514,6 +514,8 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
 // ------------------------------------------------------------------------------------------------
 struct UpdateArgs {
   int V, slice, grid_policy;
+  int hard;                       // 0: soft labels (distance sums); 1: hard labels - whether each grid candidate's most likely
+                                  // token is the verified token (matches); 2: whether each drafter's is NOT (errors)
   const float* p;                 // [B][G+1][V]
   const float* qk;                // [B][G][m][V]
   int* ticket;                    // [B] scratch, zero between launches
@@ -523,6 +525,8 @@ struct UpdateArgs {
 struct UpdShared {
   long long red[kReqWarps][kMaxDev];
   long long all_dev[kReqMaxCluster][kMaxDev];        // [CTA][deviation index], filled in CTA 0
+  ReqBest red_b[kReqWarps][kMaxDev];                 // hard labels: most likely token per candidate
+  ReqBest all_b[kReqMaxCluster][kMaxDev];
 };
 
 __device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last);
@@ -541,7 +545,70 @@ __global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs 
   const int last = min(a, G - 1);
   if (i > last) return;                             // (the whole cluster: position not verified)
   const bool vec = (V & 3) == 0;
-  {
+  if (A.hard) {
+    // most likely token (lowest id on ties) of every grid candidate's ensemble, or of every drafter
+    const float* qbase = A.qk + ((long long)b * G + i) * m * V;
+    ReqBest best[kMaxDev];
+#pragma unroll
+    for (int kd = 0; kd < kMaxDev; ++kd) best[kd] = ReqBest{-1.0f, 0x7fffffff};
+#pragma unroll 1
+    for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      if (A.grid_policy) {
+        float q0[4], q1[4];
+        req_ld4(qbase, v, c.v_hi, vec, 0.0f, q0);
+        req_ld4(qbase + V, v, c.v_hi, vec, 0.0f, q1);
+#pragma unroll
+        for (int jc = 0; jc < kGridCand; ++jc) {
+          const float c1 = __fdiv_rn((float)jc, 10.0f);
+          const float c0 = __fsub_rn(1.0f, c1);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float mix = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
+            if (v + j < c.v_hi && mix > best[jc].val) { best[jc].val = mix; best[jc].idx = v + j; }
+          }
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < kMaxInputs; ++k) {
+          if (k >= m) break;
+          float qv[4];
+          req_ld4(qbase + (long long)k * V, v, c.v_hi, vec, 0.0f, qv);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) if (v + j < c.v_hi && qv[j] > best[k].val) { best[k].val = qv[j]; best[k].idx = v + j; }
+        }
+      }
+    }
+#pragma unroll
+    for (int kd = 0; kd < kMaxDev; ++kd) {
+      if (kd < n_dev) {
+        ReqBest mine = best[kd];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          ReqBest other;
+          other.val = __shfl_xor_sync(0xffffffffu, mine.val, o);
+          other.idx = __shfl_xor_sync(0xffffffffu, mine.idx, o);
+          best_merge(mine, other);
+        }
+        if (c.lane == 0) U.red_b[c.warp][kd] = mine;
+      }
+    }
+    __syncthreads();
+    if (c.tid < n_dev) {
+      ReqBest t = U.red_b[0][c.tid];
+#pragma unroll
+      for (int w = 1; w < kReqWarps; ++w) best_merge(t, U.red_b[w][c.tid]);
+      cluster.map_shared_rank(&U.all_b[0][0], 0)[c.rank * kMaxDev + c.tid] = t;
+    }
+    cluster.sync();
+    if (c.rank == 0 && c.tid < n_dev) {
+      ReqBest t = U.all_b[0][c.tid];
+      for (unsigned r = 1; r < c.CS; ++r) best_merge(t, U.all_b[r][c.tid]);
+      // the verified token of position i: the accepted draft, or the replacement at the rejected position
+      const int label = (i < a) ? P.tokens[b * G + i] : P.next_token[b];
+      const int hit = t.idx == label;
+      P.dev[((long long)b * G + i) * kMaxDev + c.tid] = (A.hard == 1) ? hit : 1 - hit;
+    }
+  } else {
     const float* p_i = A.p + ((long long)b * (G + 1) + i) * V;
     const float* qbase = A.qk + ((long long)b * G + i) * m * V;
     long long acc[kMaxDev];
@@ -614,12 +681,12 @@ __global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs 
       for (int w = 0; w < kReqWarps; ++w) t += U.red[w][c.tid];
       cluster.map_shared_rank(&U.all_dev[0][0], 0)[c.rank * kMaxDev + c.tid] = t;
     }
-  }
-  cluster.sync();
-  if (c.rank == 0 && c.tid < n_dev) {
-    long long t = 0;
-    for (unsigned r = 0; r < c.CS; ++r) t += U.all_dev[r][c.tid];
-    P.dev[((long long)b * G + i) * kMaxDev + c.tid] = t;
+    cluster.sync();
+    if (c.rank == 0 && c.tid < n_dev) {
+      long long t = 0;
+      for (unsigned r = 0; r < c.CS; ++r) t += U.all_dev[r][c.tid];
+      P.dev[((long long)b * G + i) * kMaxDev + c.tid] = t;
+    }
   }
   __syncthreads();                                  // (CTA 0: the sums are stored before its first thread's fence)
   if (!req_last_of_request(cluster, c, &s_last, A.ticket + b, last + 1)) return;
@@ -664,12 +731,35 @@ __device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int la
 
   float* w = A.w + (long long)b * A.m;
   const float fx_scale = A.tvd ? 4.547473508864641e-13f : kMassInv;     // 2^-41 or 2^-40
-  if (A.policy == 0 || pushed == 0) {
+  if (A.policy == 3) {
+    // random point of the simplex from the caller's uniforms: g_k = -ln u_k, w_k = g_k / sum g
+    float g[8], tot = 0.0f;
+    for (int k = 0; k < A.m; ++k) {
+      g[k] = -xlog(A.u_policy[(long long)b * A.m + k]);
+      tot = (k == 0) ? g[0] : __fadd_rn(tot, g[k]);
+    }
+    for (int k = 0; k < A.m; ++k) w[k] = __fdiv_rn(g[k], tot);
+  } else if (A.policy == 0 || pushed == 0) {
     const float s = __fdiv_rn(1.0f, (float)A.m);
     for (int k = 0; k < A.m; ++k) w[k] = s;
-  } else if (A.policy == 1) {
+  } else if (A.policy == 5) {
+    // AdaBoost-style weights from the drafters' error counts over the n window positions
+    const long long n = A.h > 0 ? (long long)A.ring_count[b] : pushed;
+    const float den = __fadd_rn(__ll2float_rn(n), 2.0f);
+    const float lk = __fmul_rn(A.tau, xlog((float)(A.V - 1)));
+    float t[8], tot = 0.0f;
+    for (int k = 0; k < A.m; ++k) {
+      const float eps = __fdiv_rn(__fadd_rn(__ll2float_rn(run[k]), 1.0f), den);
+      t[k] = fmaxf(__fadd_rn(xlog(__fsub_rn(__fdiv_rn(1.0f, eps), 1.0f)), lk), 0.0f);
+      tot = (k == 0) ? t[0] : __fadd_rn(tot, t[k]);
+    }
+    if (tot > 0.0f) { for (int k = 0; k < A.m; ++k) w[k] = __fdiv_rn(t[k], tot); }
+    else { const float s = __fdiv_rn(1.0f, (float)A.m); for (int k = 0; k < A.m; ++k) w[k] = s; }
+  } else if (A.policy == 1 || A.policy == 4) {
+    // grid: least accumulated distance (soft labels) or most token matches (hard labels), lowest j on ties
     int js = 0;
-    for (int j = 1; j < kGridCand; ++j) if (run[j] < run[js]) js = j;
+    if (A.policy == 1) { for (int j = 1; j < kGridCand; ++j) if (run[j] < run[js]) js = j; }
+    else { for (int j = 1; j < kGridCand; ++j) if (run[j] > run[js]) js = j; }
     A.grid_j[b] = js;
     const float c1 = __fdiv_rn((float)js, 10.0f);
     w[0] = __fsub_rn(1.0f, c1);

@@ -74,6 +74,7 @@ struct tabed_handle {
   int phase = PH_IDLE;
   bool round_has_forward = false;
   const float* logits_override = nullptr;   // tabed_debug_override_logits
+  const float* u_policy = nullptr;          // tabed_set_policy_uniforms (random weight policy)
   std::vector<int> len_ub;          // upper bound of every row's committed length
   std::vector<int> pend_cnt;        // pending tokens of every request as the host last saw them
   bool pend_known = false;          // ... and whether that is still what the device holds
@@ -735,10 +736,10 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   *out = nullptr;
   const tabed_config& c = *cfg;
   if (c.vocab < 2 || c.n_inputs < 1 || c.n_inputs > TABED_MAX_INPUTS || c.n_requests < 1 || c.gamma < 1 ||
-      c.gamma > 16 || c.window_h < 0 || c.window_h > 64 || c.policy < 0 || c.policy > 2 || c.distance < 0 ||
+      c.gamma > 16 || c.window_h < 0 || c.window_h > 64 || c.policy < 0 || c.policy > TABED_POLICY_ADABOOST || c.distance < 0 ||
       c.distance > 1 || c.sample_mode < 0 || c.sample_mode > 1 || !(c.tau > 0.0f) || c.device < 0)
     return TABED_ERR_INVALID_ARG;
-  if (c.policy == TABED_POLICY_GRID_MT && c.n_inputs != 2) return TABED_ERR_INVALID_ARG;
+  if ((c.policy == TABED_POLICY_GRID_MT || c.policy == TABED_POLICY_GRID_HARD) && c.n_inputs != 2) return TABED_ERR_INVALID_ARG;
   if ((long long)c.n_requests * c.n_inputs > 4096) return TABED_ERR_UNSUPPORTED;
   if (wts) {
     if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 8 || c.kv_capacity < 1 ||
@@ -773,7 +774,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   if (!h) return TABED_ERR_CUDA;
   h->cfg = c; h->stream = reinterpret_cast<cudaStream_t>(c.stream);
   h->B = c.n_requests; h->m = c.n_inputs; h->R = h->B * h->m; h->G = c.gamma; h->V = c.vocab;
-  h->n_dev = (c.policy == TABED_POLICY_GRID_MT) ? kGridCand : h->m;
+  h->n_dev = (c.policy == TABED_POLICY_GRID_MT || c.policy == TABED_POLICY_GRID_HARD) ? kGridCand : h->m;
   h->n_chunks = (h->V + kChunk - 1) / kChunk;
   h->ns = pick_ns(h->R);
   h->has_drafter = wts != nullptr;
@@ -1098,6 +1099,7 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
 int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
   if (!h) return TABED_ERR_NULL_PTR;
   if (h->phase != PH_VERIFIED) return TABED_ERR_BAD_STATE;
+  if (h->cfg.policy == TABED_POLICY_RANDOM && !h->u_policy) return TABED_ERR_BAD_STATE;
   DeviceGuard guard(h->cfg.device);
   const int tvd = h->cfg.distance == TABED_DIST_TVD;
   {
@@ -1105,9 +1107,13 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
     UpdateArgs u{};
     const int cs = pick_cluster(h, h->B * h->G, &u.slice);
     u.ticket = h->req_ticket + h->B;
-    u.V = h->V; u.grid_policy = h->cfg.policy == TABED_POLICY_GRID_MT ? 1 : 0; u.p = h->p; u.qk = h->qk;
+    u.V = h->V;
+    u.grid_policy = (h->cfg.policy == TABED_POLICY_GRID_MT || h->cfg.policy == TABED_POLICY_GRID_HARD) ? 1 : 0;
+    u.hard = h->cfg.policy == TABED_POLICY_GRID_HARD ? 1 : (h->cfg.policy == TABED_POLICY_ADABOOST ? 2 : 0);
+    u.p = h->p; u.qk = h->qk;
     PolicyArgs& a = u.P;
     a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
+    a.V = h->V; a.u_policy = h->u_policy;
     a.tau = h->cfg.tau; a.n_accept = h->n_accept; a.next_token = h->next_token; a.tokens = h->tokens;
     a.dev = h->dev; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
     a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
@@ -1192,6 +1198,12 @@ int tabed_debug_barrier_timeout(tabed_handle* h) {
   h->launches++;
   if (cudaMemsetAsync(bar, 0, sizeof(unsigned), h->stream) != cudaSuccess) { cudaGetLastError(); return TABED_ERR_CUDA; }
   return tabed_last_device_error(h);
+}
+
+int tabed_set_policy_uniforms(tabed_handle* h, const float* u_policy) {
+  if (!h) return TABED_ERR_NULL_PTR;
+  h->u_policy = u_policy;
+  return TABED_OK;
 }
 
 int tabed_last_device_error(tabed_handle* h) {

@@ -130,7 +130,7 @@ def assert_decisions_equal(p: Pair, toks_g, a_g, z_g, w_g, am_g, bit_exact_float
         assert np.array_equal(g.debug_view(TB.VIEW_WINDOW_SUM).cpu().numpy()[:, :n_dev], o.running), "window sums"
     else:
         assert np.max(np.abs(wg - o.w)) <= 1e-5, "ensemble weights"
-    if o.policy == W.POLICY_GRID_MT:
+    if o.policy in (W.POLICY_GRID_MT, W.POLICY_GRID_HARD):
         assert np.array_equal(g.debug_view(TB.VIEW_GRID_J).cpu().numpy(), o.j_star), "grid j*"
     pend = g.debug_view(TB.VIEW_PENDING).cpu().numpy()
     for b in range(o.B):
@@ -147,7 +147,10 @@ def logits_round(p: Pair, rnd: int, logits: np.ndarray, target: Optional[np.ndar
     o.draft_round_logits(logits, ud)
     tl = target if target is not None else W.target_logits(wl, rnd, logits)
     o.verify(tl, ua, ur)
-    o_w, o_am = o.update_weights()
+    up = W.policy_uniforms(wl, rnd) if wl.policy == W.POLICY_RANDOM else None
+    o_w, o_am = o.update_weights(up)
+    if up is not None:
+        g.set_policy_uniforms(t(up))
     toks = torch.empty((wl.n_requests, wl.gamma), dtype=torch.int32, device=DEV)
     out_q = torch.empty((wl.n_requests, wl.gamma, wl.drafter.vocab), dtype=torch.float32, device=DEV)
     a = torch.empty(wl.n_requests, dtype=torch.int32, device=DEV)
@@ -178,7 +181,10 @@ def lockstep_round(p: Pair, rnd: int, override: bool = True):
     logits_o = o.logits.copy()
     tl = W.target_logits(wl, rnd, logits_o)
     o.verify(tl, ua, ur)
-    o.update_weights()
+    up = W.policy_uniforms(wl, rnd) if wl.policy == W.POLICY_RANDOM else None
+    o.update_weights(up)
+    if up is not None:
+        g.set_policy_uniforms(t(up))
     toks = torch.empty((B, G), dtype=torch.int32, device=DEV)
     a = torch.empty(B, dtype=torch.int32, device=DEV)
     z = torch.empty_like(a)

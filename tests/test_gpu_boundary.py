@@ -199,3 +199,25 @@ def test_host_round_keeps_exact_cache_lengths():
         n_async += 1
     assert n_async >= 15 and g.last_device_error() == 0
     g.destroy()
+
+
+def test_random_policy_needs_its_uniforms():
+    wl = W.TINY.replace(policy=W.POLICY_RANDOM)
+    g = H.make_gpu(wl)
+    B, G, V = wl.n_requests, wl.gamma, wl.drafter.vocab
+    u = torch.full((B, G), 0.5, device=H.DEV)
+    toks = torch.empty((B, G), dtype=torch.int32, device=H.DEV)
+    a = torch.empty(B, dtype=torch.int32, device=H.DEV)
+    g.draft_round_logits(torch.zeros((G, B, wl.n_inputs, V), device=H.DEV), u, toks)
+    g.verify(torch.zeros((B, G + 1, V), device=H.DEV), u, u[:, 0].contiguous(), a, a.clone())
+    with pytest.raises(TB.TabedError) as e:
+        g.update_weights()
+    assert e.value.code == TB.ERR_BAD_STATE
+    g.set_policy_uniforms(torch.full((B, wl.n_inputs), 0.25, device=H.DEV))
+    w = torch.empty((B, wl.n_inputs), device=H.DEV)
+    g.update_weights(w)
+    torch.cuda.synchronize()
+    assert torch.allclose(w, torch.full_like(w, 0.5)) and g.last_device_error() == 0
+    with pytest.raises(TB.TabedError):
+        TB.Tabed(n_inputs=3, n_requests=1, gamma=3, window_h=2, policy=TB.POLICY_GRID_HARD, vocab=100)
+    g.destroy()

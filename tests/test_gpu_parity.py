@@ -32,6 +32,13 @@ DECISION_CASES = {
     "tiny_tvd_softmax_all": (W.TINY, dict(distance=W.DIST_TVD, policy=W.POLICY_SOFTMAX_INV_ERR, window_h=0), 4),
     "tiny_static": (W.TINY, dict(policy=W.POLICY_STATIC), 3),
     "tiny_h1": (W.TINY, dict(window_h=1, policy=W.POLICY_SOFTMAX_INV_ERR), 5),
+    "tiny_random": (W.TINY, dict(policy=W.POLICY_RANDOM), 4),
+    "tiny_grid_hard": (W.TINY, dict(policy=W.POLICY_GRID_HARD), 6),
+    "tiny_grid_hard_all_greedy": (W.TINY, dict(policy=W.POLICY_GRID_HARD, window_h=0, sample_mode=W.MODE_GREEDY), 5),
+    "tiny_adaboost": (W.TINY, dict(policy=W.POLICY_ADABOOST), 6),
+    "llava_small_random": (W.LLAVA_SMALL, dict(policy=W.POLICY_RANDOM), 3),
+    "llava_small_adaboost_all": (W.LLAVA_SMALL, dict(policy=W.POLICY_ADABOOST, window_h=0, tau=0.5), 4),
+    "batched_serving_adaboost": (W.BATCHED_SERVING, dict(policy=W.POLICY_ADABOOST), 3),
     "llava_small": (W.LLAVA_SMALL, {}, 4),
     "large_vocab": (W.LARGE_VOCAB, {}, 3),
     "long_context": (W.LONG_CONTEXT, {}, 3),
