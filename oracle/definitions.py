@@ -128,6 +128,59 @@ def policy_adaboost(errors: np.ndarray, n: int, vocab: int, c: float = 1.0) -> n
     return w / s if s > 0 else np.full(len(w), 1.0 / len(w))
 
 
+# ---- token tree of width d (Sec. 5 "Verification: Integrating Token Tree") ---------------------------------
+# Reading (the paper names the method and the widths 2 and 3, not the construction): at every depth of the block the
+# drafter proposes d distinct candidate tokens, drawn from the ensembled q WITHOUT replacement; the first one (the
+# primary) is the token the chain continues with, the others are leaves.  The target tries the candidates of a depth
+# in order by recursive rejection sampling: candidate x is accepted with probability min(1, p'(x) / q'(x)); after a
+# rejection p' <- norm(max(0, p' - q')) and q' <- q' restricted to the tokens not yet tried, renormalised (the law of
+# the next candidate given the rejected ones); if every candidate is rejected the token is drawn from the last
+# residual.  The emitted token follows the target law p exactly (checked by enumeration in the tests).
+
+def tree_after_rejection(p: np.ndarray, q: np.ndarray, x: int):
+    """(p', q') after candidate x has been rejected at a depth."""
+    p = np.asarray(p, np.float64); q = np.asarray(q, np.float64)
+    p2 = residual_distribution(p, q)
+    q2 = q.copy(); q2[x] = 0.0
+    s = q2.sum()
+    return p2, (q2 / s if s > 0 else q2)
+
+
+def tree_depth_outcomes(p: np.ndarray, q: np.ndarray, d: int):
+    """Every outcome of one depth of a width-d tree with its probability: yields (prob, token, level) where level = c
+    if candidate c was accepted (0 = the primary) and level = -1 for a token drawn from the last residual.
+    Enumerates all ordered tuples of d distinct candidates (fewer if q runs out of support)."""
+    p = np.asarray(p, np.float64); q = np.asarray(q, np.float64)
+    out = []
+
+    def rec(pp, qq, prob, c):
+        if c == d or qq.sum() <= 0:
+            for z, pz in enumerate(pp):
+                if pz > 0:
+                    out.append((prob * pz, z, -1))
+            return
+        for x in range(len(qq)):
+            if qq[x] <= 0:
+                continue
+            acc = accept_probability(pp[x], qq[x])
+            if acc > 0:
+                out.append((prob * qq[x] * acc, x, c))
+            if acc < 1:
+                p2, q2 = tree_after_rejection(pp, qq, x)
+                rec(p2, q2, prob * qq[x] * (1 - acc), c + 1)
+
+    rec(p, q, 1.0, 0)
+    return out
+
+
+def tree_depth_emitted_law(p: np.ndarray, q: np.ndarray, d: int) -> np.ndarray:
+    """Law of the token emitted at one depth of a width-d tree (equals p)."""
+    law = np.zeros(len(p))
+    for prob, tok, _ in tree_depth_outcomes(p, q, d):
+        law[tok] += prob
+    return law
+
+
 def pool_image_tokens_2x2(x: np.ndarray, grid_h: int, grid_w: int) -> np.ndarray:
     """Pooled multimodal drafting input (Sec. 5, "Pooled Multimodal Drafting (P)"): the visual tokens keep their 2-D
     arrangement (row-major grid_h x grid_w, 24 x 24 = 576 in the paper's default) and every 2 x 2 block of tokens is

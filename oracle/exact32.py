@@ -237,3 +237,46 @@ def policy_adaboost(errors, n: int, vocab: int, c=1.0) -> np.ndarray:
     if not tot > 0:
         return policy_static(len(t))
     return (t / tot).astype(F)
+
+
+# ---- token tree of width d (Sec. 5 "Verification: Integrating Token Tree"; reading in oracle/definitions.py) ----
+
+def draw_candidates(q, u, greedy: bool = False) -> np.ndarray:
+    """d distinct candidate tokens of one depth, [d] int32 (-1 where q has no mass left): candidate c is drawn by the
+    inverse-CDF rule from the masses of q with the earlier candidates' masses set to 0 (sampling without replacement),
+    with uniform u[c]; greedy: the d most likely tokens in order (lowest id on ties)."""
+    q = np.asarray(q, F)
+    d = len(u)
+    out = np.full(d, -1, np.int32)
+    if greedy:
+        left = q.astype(np.float64).copy()
+        for c in range(min(d, len(q))):
+            out[c] = int(np.argmax(left))
+            left[out[c]] = -1.0
+        return out
+    m = masses(q).copy()
+    for c in range(d):
+        if int(m.sum(dtype=U64)) == 0:
+            break
+        out[c] = draw(m, u[c])
+        m[out[c]] = 0
+    return out
+
+
+def tree_after_rejection(p, q, x: int):
+    """(p', q', ok) after candidate x was rejected: r = max(0, p - q) (one rounded subtraction); p' = r / R with
+    R = float(sum of masses of r) * 2^-40; q' = q / Qn with Qn = float(sum of masses of q minus the mass of q_x) * 2^-40
+    and q'_x = 0.  ok is False when either sum of masses is 0 (nothing to refine: the caller stops trying candidates)."""
+    p = np.asarray(p, F); q = np.asarray(q, F)
+    r = np.maximum(F(0), p - q)
+    MR = int(masses(r).sum(dtype=U64))
+    mq = masses(q)
+    MQ = int(mq.sum(dtype=U64)) - int(mq[x])
+    if MR == 0 or MQ == 0:
+        return r, q, False
+    Rn = F(np.array(MR, dtype=U64).astype(F) * F(2.0 ** -MASS_BITS))
+    Qn = F(np.array(MQ, dtype=U64).astype(F) * F(2.0 ** -MASS_BITS))
+    p2 = (r / Rn).astype(F)
+    q2 = (q / Qn).astype(F)
+    q2[x] = F(0)
+    return p2, q2, True

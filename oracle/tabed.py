@@ -35,8 +35,9 @@ N_GRID = 10
 class TabedOracle:
     def __init__(self, *, n_inputs: int, n_requests: int, gamma: int, window_h: int,
                  policy: int, vocab: int, distance: int = DIST_KL, sample_mode: int = MODE_SAMPLE,
-                 tau: float = 1.0, drafter=None, kv_capacity: int = 0):
+                 tau: float = 1.0, drafter=None, kv_capacity: int = 0, tree_width: int = 1):
         self.m, self.B, self.gamma, self.h = n_inputs, n_requests, gamma, window_h
+        self.d = tree_width            # candidates per depth of the token tree (1: a plain chain)
         self.policy, self.V = policy, vocab
         self.distance, self.mode, self.tau = distance, sample_mode, tau
         if policy in (POLICY_GRID_MT, POLICY_GRID_HARD) and n_inputs != 2:
@@ -60,6 +61,14 @@ class TabedOracle:
         self.p = None           # [B][gamma+1][V] fp32
         self.n_accept = None
         self.next_token = None
+        self.cands = None       # [B][gamma][d] int32 candidates of every depth (column 0: the primary chain)
+        self.acc_prim = None    # [B] accepted primaries;  sib_tok [B]: the accepted sibling's token or -1
+        self.sib_tok = None
+
+    def n_target_rows(self) -> int:
+        """Rows of target logits per request: the primary chain's gamma + 1 positions, then one leaf per sibling
+        candidate, depth-major: row gamma + 1 + i * (d - 1) + (c - 1) follows sibling c of depth i."""
+        return self.gamma + 1 + self.gamma * (self.d - 1)
 
     # ---- drafter-side helpers -------------------------------------------------
     def prefill(self, row: int, segments) -> None:
@@ -92,9 +101,8 @@ class TabedOracle:
         qk = x32.softmax_exact(logits_bk)                      # [m][V]
         q = x32.ensemble_exact(qk, self.w[b])
         self.qk[b, i], self.q[b, i] = qk, q
-        if self.mode == MODE_GREEDY:
-            return x32.argmax_lowest(q)
-        return x32.draw(x32.masses(q), u)
+        self.cands[b, i] = x32.draw_candidates(q, np.atleast_1d(u), self.mode == MODE_GREEDY)
+        return int(self.cands[b, i, 0])
 
     def _begin_round(self):
         B, G, m, V = self.B, self.gamma, self.m, self.V
@@ -102,10 +110,13 @@ class TabedOracle:
         self.q = np.zeros((B, G, V), F)
         self.qk = np.zeros((B, G, m, V), F)
         self.logits = np.zeros((G, B, m, V), F)
+        self.cands = np.full((B, G, self.d), -1, np.int32)
 
     def draft_round(self, u_draft: np.ndarray):
-        """gamma batched drafter steps; returns (tokens [B][gamma], q [B][gamma][V])."""
+        """gamma batched drafter steps; returns (tokens [B][gamma], q [B][gamma][V]).  u_draft [B][gamma] (or
+        [B][gamma][d] with a token tree: one uniform per candidate)."""
         self._begin_round()
+        u_draft = np.asarray(u_draft).reshape(self.B, self.gamma, self.d)
         for b in range(self.B):
             pend = self.pending[b]
             assert 1 <= len(pend) <= 2
@@ -122,6 +133,7 @@ class TabedOracle:
     def draft_round_logits(self, logits: np.ndarray, u_draft: np.ndarray):
         """Steps 6-7 on caller-supplied drafter logits [gamma][B][m][V]; no forward pass."""
         self._begin_round()
+        u_draft = np.asarray(u_draft).reshape(self.B, self.gamma, self.d)
         self.logits = np.asarray(logits, F)
         for b in range(self.B):
             for i in range(self.gamma):
@@ -131,32 +143,64 @@ class TabedOracle:
     # ---- Sec. 3, item 3 ---------------------------------------------------------
     def verify(self, target_logits: np.ndarray, u_accept: np.ndarray, u_resid: np.ndarray):
         """Sequential acceptance and the replacement / bonus token.
-        target_logits [B][gamma+1][V] fp32.  Returns (n_accept [B], next_token [B])."""
-        B, G = self.B, self.gamma
-        self.p = x32.softmax_exact(np.asarray(target_logits, F))          # [B][G+1][V]
+        target_logits [B][n_target_rows()][V] fp32; u_accept [B][gamma] ([B][gamma][d] with a tree).
+        Returns (n_accept [B], next_token [B]); n_accept counts every accepted draft token (an accepted sibling too)."""
+        B, G, d = self.B, self.gamma, self.d
+        tl = np.asarray(target_logits, F)
+        u_accept = np.asarray(u_accept).reshape(B, G, d)
+        self.p = np.zeros((B, self.n_target_rows(), self.V), F)
+        self.p[:, :G + 1] = x32.softmax_exact(tl[:, :G + 1])              # the primary chain's positions
         self.n_accept = np.zeros(B, np.int32)
         self.next_token = np.zeros(B, np.int32)
+        self.acc_prim = np.zeros(B, np.int32)
+        self.sib_tok = np.full(B, -1, np.int32)
         for b in range(B):
-            a = 0
-            for i in range(G):
-                y = int(self.tokens[b, i])
+            i, z, sib = 0, None, -1
+            while i < G and z is None and sib < 0:
+                P, Q = self.p[b, i], self.q[b, i]
                 if self.mode == MODE_GREEDY:
-                    ok = x32.argmax_lowest(self.p[b, i]) == y
+                    t = x32.argmax_lowest(P)
+                    hit = [c for c in range(d) if int(self.cands[b, i, c]) == t]
+                    if hit and hit[0] == 0:
+                        i += 1
+                    elif hit:
+                        sib = hit[0]
+                    else:
+                        z = t
+                    continue
+                for c in range(d):
+                    x = int(self.cands[b, i, c])
+                    if x32.accept(P[x], Q[x], u_accept[b, i, c]):
+                        if c > 0:
+                            sib = c
+                        break
+                    # rejected: the replacement comes from the residual unless another candidate can be tried
+                    more = c + 1 < d and int(self.cands[b, i, c + 1]) >= 0
+                    P2, Q2, ok = x32.tree_after_rejection(P, Q, x) if more else (None, None, False)
+                    if not ok:
+                        mass = x32.residual_masses(P, Q)
+                        if int(mass.sum(dtype=np.uint64)) == 0:
+                            mass = x32.masses(P)
+                        z = x32.draw(mass, u_resid[b])
+                        break
+                    P, Q = P2, Q2
                 else:
-                    ok = x32.accept(self.p[b, i, y], self.q[b, i, y], u_accept[b, i])
-                if not ok:
-                    break
-                a += 1
-            if self.mode == MODE_GREEDY:
-                z = x32.argmax_lowest(self.p[b, a])
-            elif a < G:
-                mass = x32.residual_masses(self.p[b, a], self.q[b, a])
-                if int(mass.sum(dtype=np.uint64)) == 0:
-                    mass = x32.masses(self.p[b, a])
-                z = x32.draw(mass, u_resid[b])
+                    raise AssertionError("unreachable: the last candidate either is accepted or ends the depth")
+                if z is None and sib < 0:
+                    i += 1                                            # the primary was accepted
+            self.acc_prim[b] = i
+            if sib >= 0:
+                # an accepted sibling is a leaf: the next token comes from the target's distribution after it
+                row = G + 1 + i * (d - 1) + (sib - 1)
+                self.p[b, row] = x32.softmax_exact(tl[b, row])
+                self.sib_tok[b] = self.cands[b, i, sib]
+                z = x32.argmax_lowest(self.p[b, row]) if self.mode == MODE_GREEDY else x32.draw(x32.masses(self.p[b, row]), u_resid[b])
+                self.n_accept[b] = i + 1
             else:
-                z = x32.draw(x32.masses(self.p[b, G]), u_resid[b])
-            self.n_accept[b], self.next_token[b] = a, z
+                if z is None:                                         # every primary accepted: bonus token from p_gamma
+                    z = x32.argmax_lowest(self.p[b, G]) if self.mode == MODE_GREEDY else x32.draw(x32.masses(self.p[b, G]), u_resid[b])
+                self.n_accept[b] = i
+            self.next_token[b] = z
         return self.n_accept, self.next_token
 
     # ---- Sec. 4.1 deviation; App. B policies; Algorithm 1 steps 2-3 --------------
@@ -181,10 +225,11 @@ class TabedOracle:
         G = self.gamma
         self.u_policy = u_policy
         for b in range(self.B):
-            a = int(self.n_accept[b])
+            a = int(self.acc_prim[b])                # accepted tokens of the primary chain (the drafter consumed those)
+            sib = int(self.sib_tok[b])
             for i in range(min(a, G - 1) + 1):
-                # the verified token of position i: the accepted draft, or the replacement at the rejected position
-                label = int(self.tokens[b, i]) if i < a else int(self.next_token[b])
+                # the verified token of position i: the accepted draft, or what was emitted at the first other position
+                label = int(self.tokens[b, i]) if i < a else (sib if sib >= 0 else int(self.next_token[b]))
                 dev = self._deviation(self.p[b, i], self.qk[b, i], label)
                 self.running[b] += dev
                 self.count[b] += 1
@@ -201,7 +246,10 @@ class TabedOracle:
                     c = self.caches[b * self.m + k]
                     c.length = c.length - (n_pend + G - 1) + keep
             z = int(self.next_token[b])
-            self.pending[b] = [z] if a < G else [int(self.tokens[b, G - 1]), z]
+            if a == G:
+                self.pending[b] = [int(self.tokens[b, G - 1]), z]
+            else:
+                self.pending[b] = [sib, z] if sib >= 0 else [z]
         return self.w.copy(), np.argmax(self.w, axis=1).astype(np.int32)
 
     def _policy(self, b: int) -> np.ndarray:

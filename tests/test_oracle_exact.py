@@ -333,3 +333,110 @@ def test_grid_weights_and_static():
     assert tuple(X.grid_weight(0)) == (1.0, 0.0) and tuple(X.grid_weight(10)) == (0.0, 1.0)
     for m in (1, 2, 3, 4):
         np.testing.assert_allclose(X.policy_static(m), 1.0 / m, rtol=1e-7)
+
+
+# ---------------------------------------------------------------- token tree of width d
+@pytest.mark.parametrize("V,d", [(2, 2), (3, 2), (3, 3), (5, 2), (5, 3)])
+def test_tree_depth_emitted_law_equals_target_bruteforce(V, d):
+    """Sec. 5 "Verification: Integrating Token Tree" must keep Sec. 3's guarantee: with d candidates per depth, drawn
+    without replacement and tried by recursive rejection, the emitted token still follows the target law.  Every
+    ordered candidate tuple and every accept / reject / replacement branch is enumerated."""
+    rng = np.random.default_rng(40 + 10 * V + d)
+    for trial in range(12):
+        p = rng.dirichlet(np.ones(V) * 0.7)
+        q = rng.dirichlet(np.ones(V) * 0.7)
+        if trial == 0:
+            q = p.copy()
+        if trial == 1:
+            p[0] = 0.0; p /= p.sum()
+        if trial == 2:
+            q[-1] = 0.0; q /= q.sum()                       # the drafter never proposes a token the target wants
+        outs = D.tree_depth_outcomes(p, q, d)
+        assert abs(sum(pr for pr, _, _ in outs) - 1.0) < 1e-12
+        np.testing.assert_allclose(D.tree_depth_emitted_law(p, q, d), p, atol=1e-12)
+        # more candidates can only raise the chance that a drafted token is accepted
+        acc = [sum(pr for pr, _, lvl in D.tree_depth_outcomes(p, q, w) if lvl >= 0) for w in range(1, d + 1)]
+        assert all(acc[i + 1] >= acc[i] - 1e-12 for i in range(len(acc) - 1))
+        assert abs(acc[0] - np.minimum(p, q).sum()) < 1e-12        # width 1 is plain speculative sampling
+
+
+def test_tree_two_depth_block_law_bruteforce():
+    """Two depths, width 2 and 3, table-defined conditionals: the first emitted token follows p0 and, whenever a
+    drafted token was accepted at depth 0 (primary or sibling), the second emitted token follows p1(. | first)."""
+    rng = np.random.default_rng(77)
+    V = 3
+    for d in (2, 3):
+        p0, q0 = rng.dirichlet(np.ones(V)), rng.dirichlet(np.ones(V))
+        p1 = rng.dirichlet(np.ones(V), size=V); q1 = rng.dirichlet(np.ones(V), size=V)
+        first = np.zeros(V); joint = np.zeros((V, V)); accepted = np.zeros(V)
+        for prob, tok, lvl in D.tree_depth_outcomes(p0, q0, d):
+            first[tok] += prob
+            if lvl < 0:
+                continue                                    # replacement: the round ends with one token
+            accepted[tok] += prob
+            # primary: depth 1 is another tree depth on (p1, q1)[tok]; sibling: a leaf, the next token comes from p1[tok]
+            second = D.tree_depth_emitted_law(p1[tok], q1[tok], d) if lvl == 0 else p1[tok]
+            joint[tok] += prob * second
+        np.testing.assert_allclose(first, p0, atol=1e-12)
+        np.testing.assert_allclose(joint, accepted[:, None] * p1, atol=1e-12)
+
+
+def test_draw_candidates_without_replacement():
+    rng = np.random.default_rng(78)
+    q = X.softmax_exact((rng.standard_normal(6) * 1.2).astype(F))
+    N = 2048
+    ks = np.arange(N) * ((1 << 23) // N) + 5
+    # distinct tokens; the second candidate follows q restricted to the others
+    pair = np.zeros((6, 6))
+    for k0 in ks[::32]:
+        for k1 in ks[::32]:
+            c = X.draw_candidates(q, np.array([lattice(k0), lattice(k1)], F))
+            assert c[0] != c[1] and c[0] == X.draw(X.masses(q), lattice(k0))
+            pair[c[0], c[1]] += 1
+    pair /= pair.sum()
+    qd = q.astype(np.float64)
+    ref = qd[:, None] * qd[None, :] / (1.0 - qd[:, None])
+    np.fill_diagonal(ref, 0.0)
+    assert np.max(np.abs(pair - ref)) < 0.03
+    # greedy: the d most likely tokens in order, lowest id on ties; more candidates than tokens -> -1
+    assert list(X.draw_candidates(np.array([0.2, 0.5, 0.2, 0.1], F), np.zeros(3, F), greedy=True)) == [1, 0, 2]
+    assert list(X.draw_candidates(np.array([0.5, 0.5], F), np.zeros(3, F), greedy=True)) == [0, 1, -1]
+    # all mass on one token: there is no second candidate
+    assert list(X.draw_candidates(np.array([0.0, 1.0, 0.0], F), np.array([lattice(3), lattice(9)], F))) == [1, -1]
+
+
+@pytest.mark.parametrize("V", [3, 5])
+def test_exact_tree_depth_preserves_target_law_by_lattice_enumeration(V):
+    """Width 2 in the kernel's arithmetic, composed from 1-D lattice sweeps: P(x0), P(x1 | x0), the two acceptance
+    probabilities and the replacement law after two rejections."""
+    rng = np.random.default_rng(300 + V)
+    N = 2048
+    ks = (np.arange(N) * ((1 << 23) // N) + 11)
+    for trial in range(2):
+        p = X.softmax_exact((rng.standard_normal(V) * 1.3).astype(F))
+        q = X.softmax_exact((rng.standard_normal(V) * 1.3).astype(F))
+        mq = X.masses(q)
+        px0 = np.bincount([X.draw(mq, lattice(k)) for k in ks], minlength=V) / N
+        law = np.zeros(V)
+        for x0 in range(V):
+            if px0[x0] == 0:
+                continue
+            a0 = np.mean([X.accept(p[x0], q[x0], lattice(k)) for k in ks])
+            law[x0] += px0[x0] * a0
+            p2, q2, ok = X.tree_after_rejection(p, q, x0)
+            np.testing.assert_allclose(p2, D.tree_after_rejection(p, q, x0)[0], atol=1e-6)
+            np.testing.assert_allclose(q2, D.tree_after_rejection(p, q, x0)[1], atol=1e-6)
+            assert ok and q2[x0] == 0
+            m1 = mq.copy(); m1[x0] = 0
+            px1 = np.bincount([X.draw(m1, lattice(k)) for k in ks], minlength=V) / N
+            for x1 in range(V):
+                if px1[x1] == 0:
+                    continue
+                a1 = np.mean([X.accept(p2[x1], q2[x1], lattice(k)) for k in ks])
+                law[x1] += px0[x0] * (1 - a0) * px1[x1] * a1
+                mr = X.residual_masses(p2, q2)
+                if int(mr.sum()) == 0:
+                    mr = X.masses(p2)
+                pz = np.bincount([X.draw(mr, lattice(k)) for k in ks], minlength=V) / N
+                law += px0[x0] * (1 - a0) * px1[x1] * (1 - a1) * pz
+        assert np.max(np.abs(law - p.astype(np.float64))) < 8.0 * V / N

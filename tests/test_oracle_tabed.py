@@ -438,3 +438,76 @@ def test_adaboost_weights_follow_the_printed_formula():
         w, am = o.update_weights()
         win = np.array(errs[-4:])
         np.testing.assert_allclose(w[0], D.policy_adaboost(win.sum(axis=0), len(win), V, 1.0), atol=2e-6)
+
+
+# ---------------------------------------------------------------- token tree of width d in the round machine
+def test_tree_round_sibling_acceptance_and_bookkeeping():
+    """Forced cases on a width-2 tree: (a) the primary of depth 0 is impossible under the target and its sibling is
+    certain -> the sibling is accepted, the block ends there, the next token comes from the target's distribution
+    after the sibling (its leaf row), two tokens are pending and the caches keep only what the drafter consumed;
+    (b) both candidates impossible -> replacement from the residual; (c) every primary certain -> all accepted."""
+    rng = np.random.default_rng(41)
+    G, V, m, d = 3, 30, 2, 2
+    cfg = W.DrafterCfg(1, 32, 2, 2, 64, V, "fp32")
+    wl = W.Workload(name="tree_t", config_id=95, drafter=cfg, n_inputs=m, n_requests=1, gamma=G, window_h=0, rounds=1,
+                    policy=W.POLICY_SOFTMAX_INV_ERR, prefixes=((("tokens", 5),), (("tokens", 3),)), kv_capacity=64)
+    for case in ("sibling", "none", "all"):
+        o = TabedOracle(n_inputs=m, n_requests=1, gamma=G, window_h=0, policy=W.POLICY_SOFTMAX_INV_ERR, vocab=V,
+                        drafter=OracleDrafter(cfg, W.make_weights(wl)), kv_capacity=64, tree_width=d)
+        for k, segs in enumerate(W.make_prefixes(wl, 0)):
+            o.prefill(k, segs)
+        o.set_pending([4])
+        len0 = o.kv_lengths().copy()
+        toks, q = o.draft_round(lat(rng, (1, G, d)))
+        assert np.all(o.cands[0, :, 0] == toks[0]) and np.all(o.cands[0, :, 0] != o.cands[0, :, 1])
+        tl = np.zeros((1, o.n_target_rows(), V), F)
+        assert o.n_target_rows() == G + 1 + G
+        hot = lambda t: 60.0 * np.eye(V, dtype=F)[t] - 30.0
+        leaf_tok = 11
+        if case == "sibling":
+            tl[0, 0] = hot(o.cands[0, 0, 1])                  # the target wants the sibling of depth 0
+            tl[0, G + 1] = hot(leaf_tok)                      # ... and after it, token 11
+        elif case == "none":
+            other = [t for t in range(V) if t not in o.cands[0, 0]][0]
+            tl[0, 0] = hot(other)
+        else:
+            for i in range(G):
+                tl[0, i] = hot(toks[0, i])
+            tl[0, G] = hot(leaf_tok)
+        a, z = o.verify(tl, lat(rng, (1, G, d)), lat(rng, (1,)))
+        w, am = o.update_weights()
+        if case == "sibling":
+            assert a[0] == 1 and o.acc_prim[0] == 0 and o.sib_tok[0] == o.cands[0, 0, 1] and z[0] == leaf_tok
+            assert o.pending[0] == [int(o.cands[0, 0, 1]), leaf_tok] and o.count[0] == 1
+            assert np.array_equal(o.kv_lengths(), len0 + 1)                    # the pending token only
+        elif case == "none":
+            assert a[0] == 0 and o.sib_tok[0] == -1 and z[0] == other and o.pending[0] == [other] and o.count[0] == 1
+            assert np.array_equal(o.kv_lengths(), len0 + 1)
+        else:
+            assert a[0] == G and o.acc_prim[0] == G and z[0] == leaf_tok and o.count[0] == G
+            assert o.pending[0] == [int(toks[0, G - 1]), leaf_tok] and np.array_equal(o.kv_lengths(), len0 + 1 + G - 1)
+
+
+def test_tree_round_accepts_at_least_as_much_as_the_chain():
+    """Same uniforms for the primary chain: a width-3 tree never accepts fewer tokens in a round than the chain does
+    on the same drafts (the siblings only add chances), and its primary chain is the chain's draft."""
+    rng = np.random.default_rng(42)
+    G, V, m = 4, 80, 2
+    tot = [0, 0]
+    for trial in range(30):
+        lg = rand_logits(rng, G, 1, m, V, 1.5)
+        ud3, ua3, ur = lat(rng, (1, G, 3)), lat(rng, (1, G, 3)), lat(rng, (1,))
+        o1 = mk(m=m, B=1, gamma=G, h=0, V=V)
+        o3 = TabedOracle(n_inputs=m, n_requests=1, gamma=G, window_h=0, policy=W.POLICY_SOFTMAX_INV_ERR, vocab=V, tree_width=3)
+        t1, _ = o1.draft_round_logits(lg, ud3[:, :, 0])
+        t3, _ = o3.draft_round_logits(lg, ud3)
+        assert np.array_equal(t1, t3) and np.array_equal(o1.q, o3.q)
+        tl = (rng.standard_normal((1, o3.n_target_rows(), V)) * 1.5).astype(F)
+        tl[0, :G] += lg[:, 0, 0, :]
+        a1, _ = o1.verify(tl[:, :G + 1], ua3[:, :, 0], ur)
+        a3, _ = o3.verify(tl, ua3, ur)
+        assert a3[0] >= a1[0] and o3.acc_prim[0] >= min(a1[0], o3.acc_prim[0])
+        if o3.sib_tok[0] < 0:
+            assert o3.acc_prim[0] == a3[0]
+        tot[0] += int(a1[0]); tot[1] += int(a3[0])
+    assert tot[1] > tot[0]
