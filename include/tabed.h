@@ -80,11 +80,27 @@ extern "C" {
 #define TABED_MODE_GREEDY 1     /* argmax decoding, lowest id on ties             */
 
 #define TABED_MAX_INPUTS 8
+#define TABED_MAX_TREE_WIDTH 4
+
+/* Token tree of width d (Sec. 5, "Verification: Integrating Token Tree"; config.tree_width = d > 1).  The paper names the
+ * method and the widths 2 and 3; the construction taken here: at every depth of the block the drafter proposes d
+ * distinct candidates, drawn from the ensembled q WITHOUT replacement (greedy mode: its d most likely tokens); the
+ * first one (the primary) is the token the chain continues with, the others are leaves.  The target scores the chain
+ * and every leaf in one pass (G + 1 + G (d - 1) rows).  At the first depth whose primary is rejected the siblings are
+ * tried in order by recursive rejection: after a rejection p' = norm(max(0, p' - q')), q' = q' restricted to the
+ * untried tokens, renormalised; candidate x is accepted iff p'(x) >= q'(x) or u q'(x) < p'(x); if all are rejected the
+ * replacement is drawn from the last residual.  An accepted sibling ends the block; the next token then comes from the
+ * target's distribution at its leaf.  The emitted tokens follow the target's law as in Sec. 3.  Shapes with d > 1:
+ * u_draft, out_tokens, u_accept are [B][G][d] (candidate-minor; column 0 = the primary chain); target_logits is
+ * [B][G + 1 + G (d - 1)][V]: rows 0..G the chain's positions, row G + 1 + i (d - 1) + (c - 1) the leaf after sibling c of
+ * depth i.  n_accept counts an accepted sibling too.  d = 1 is exactly the plain round.  With d > 1 drafting runs on
+ * the tensor-core or per-operation path. */
 
 /* tabed_debug_view selectors (device buffers owned by the handle) */
 #define TABED_VIEW_QK          0   /* float  [B][G][m][V]  per-drafter distributions of the round     */
 #define TABED_VIEW_Q           1   /* float  [B][G][V]     ensembled distributions of the round        */
-#define TABED_VIEW_P           2   /* float  [B][G+1][V]   target distributions (after tabed_verify)   */
+#define TABED_VIEW_P           2   /* float  [B][G+1][V]   target distributions (after tabed_verify); with a token tree
+                                                           [B][G+1+G(d-1)][V], of the leaves only the one that was used */
 #define TABED_VIEW_LOGITS      3   /* float  [G][B][m][V]  drafter logits of the round's own forward   */
 #define TABED_VIEW_KV_LEN      4   /* int32  [R]           committed cache length of every row         */
 #define TABED_VIEW_WEIGHTS     5   /* float  [B][m]        current ensemble weights w*                 */
@@ -93,6 +109,8 @@ extern "C" {
 #define TABED_VIEW_PENDING     7   /* int32  [B][3]        {count, token0, token1}                     */
 #define TABED_VIEW_GRID_J      8   /* int32  [B]           j* of the grid policy (-1 before any update)*/
 #define TABED_VIEW_ERROR_FLAG  9   /* int32  [1]           non-zero if a device-side check failed      */
+#define TABED_VIEW_ACC_PRIMARY 11  /* int32  [B]           accepted tokens of the primary chain (after tabed_verify)   */
+#define TABED_VIEW_SIBLING     12  /* int32  [B]           token of the accepted sibling of a token tree, or -1        */
 #define TABED_VIEW_TRACE      10   /* uint64 [G][5L+8][8]  phase timeline of the persistent drafting kernel
                                                            (tabed_debug_trace): one record per grid barrier */
 
@@ -130,6 +148,7 @@ typedef struct {
   int32_t kv_capacity;        /* tokens per row */
   int32_t device;             /* CUDA device ordinal */
   void*   stream;             /* cudaStream_t, caller-owned; NULL = legacy default stream */
+  int32_t tree_width;         /* d: candidates per depth of the token tree, 1..TABED_MAX_TREE_WIDTH; 0 or 1 = a plain chain */
 } tabed_config;
 
 /* Device pointers to the drafter M_q, element type per config.dtype (float or bf16), every matrix

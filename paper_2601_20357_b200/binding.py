@@ -22,7 +22,7 @@ POLICY_STATIC, POLICY_GRID_MT, POLICY_SOFTMAX_INV_ERR, POLICY_RANDOM, POLICY_GRI
 DIST_KL, DIST_TVD = 0, 1
 MODE_SAMPLE, MODE_GREEDY = 0, 1
 (VIEW_QK, VIEW_Q, VIEW_P, VIEW_LOGITS, VIEW_KV_LEN, VIEW_WEIGHTS, VIEW_WINDOW_SUM, VIEW_PENDING,
- VIEW_GRID_J, VIEW_ERROR_FLAG, VIEW_TRACE) = range(11)
+ VIEW_GRID_J, VIEW_ERROR_FLAG, VIEW_TRACE, VIEW_ACC_PRIMARY, VIEW_SIBLING) = range(13)
 PATH_AUTO, PATH_PER_OP, PATH_PERSISTENT, PATH_TENSOR_CORE = 0, 1, 2, 3
 MAX_DEV = 11
 (PROF_QKV, PROF_ATTENTION, PROF_OPROJ, PROF_GATEUP, PROF_DOWN, PROF_LM_HEAD, PROF_ENSEMBLE, PROF_VERIFY,
@@ -51,7 +51,8 @@ class TabedConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "d_ffn", "vocab", "dtype")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
                [(n, C.c_int32) for n in ("n_inputs", "n_requests", "gamma", "window_h", "policy", "distance", "sample_mode")] + \
-               [("tau", C.c_float), ("kv_capacity", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p)]
+               [("tau", C.c_float), ("kv_capacity", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p),
+                ("tree_width", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -154,11 +155,13 @@ class Tabed:
     def __init__(self, *, n_inputs: int, n_requests: int, gamma: int, window_h: int, policy: int, vocab: int,
                  distance: int = DIST_KL, sample_mode: int = MODE_SAMPLE, tau: float = 1.0,
                  drafter=None, weights: Optional[Dict[str, object]] = None, kv_capacity: int = 0,
-                 device: int = 0, stream: Optional[torch.cuda.Stream] = None):
+                 device: int = 0, stream: Optional[torch.cuda.Stream] = None, tree_width: int = 1):
         self._h = C.c_void_p()
+        self.D = max(1, tree_width)                     # candidates per depth of the token tree
         self.device = torch.device("cuda", device)
         self.m, self.B, self.G, self.V = n_inputs, n_requests, gamma, vocab
         self.R = n_inputs * n_requests
+        self.Rt = gamma + 1 + gamma * (self.D - 1)      # rows of target logits per request
         self.policy = policy
         cfg = TabedConfig()
         cfg.n_inputs, cfg.n_requests, cfg.gamma, cfg.window_h = n_inputs, n_requests, gamma, window_h
@@ -166,6 +169,7 @@ class Tabed:
         cfg.vocab, cfg.device = vocab, device
         cfg.stream = stream.cuda_stream if stream is not None else None
         cfg.kv_capacity = kv_capacity
+        cfg.tree_width = tree_width
         self.drafter = drafter
         self._keep = []
         wptr = None
@@ -239,22 +243,22 @@ class Tabed:
 
     def draft_round(self, u_draft, out_tokens, out_q=None) -> None:
         d = self.device
-        _check(lib().tabed_draft_round(self._h, _ptr(u_draft, torch.float32, self.B * self.G, "u_draft", d),
-                                       _ptr(out_tokens, torch.int32, self.B * self.G, "out_tokens", d),
+        _check(lib().tabed_draft_round(self._h, _ptr(u_draft, torch.float32, self.B * self.G * self.D, "u_draft", d),
+                                       _ptr(out_tokens, torch.int32, self.B * self.G * self.D, "out_tokens", d),
                                        _ptr(out_q, torch.float32, self.B * self.G * self.V, "out_q", d)), "tabed_draft_round")
 
     def draft_round_logits(self, drafter_logits, u_draft, out_tokens, out_q=None) -> None:
         d = self.device
         _check(lib().tabed_draft_round_logits(
             self._h, _ptr(drafter_logits, torch.float32, self.G * self.R * self.V, "drafter_logits", d),
-            _ptr(u_draft, torch.float32, self.B * self.G, "u_draft", d),
-            _ptr(out_tokens, torch.int32, self.B * self.G, "out_tokens", d),
+            _ptr(u_draft, torch.float32, self.B * self.G * self.D, "u_draft", d),
+            _ptr(out_tokens, torch.int32, self.B * self.G * self.D, "out_tokens", d),
             _ptr(out_q, torch.float32, self.B * self.G * self.V, "out_q", d)), "tabed_draft_round_logits")
 
     def verify(self, target_logits, u_accept, u_resid, out_n_accept, out_next_token) -> None:
         d = self.device
-        _check(lib().tabed_verify(self._h, _ptr(target_logits, torch.float32, self.B * (self.G + 1) * self.V, "target_logits", d),
-                                  _ptr(u_accept, torch.float32, self.B * self.G, "u_accept", d),
+        _check(lib().tabed_verify(self._h, _ptr(target_logits, torch.float32, self.B * self.Rt * self.V, "target_logits", d),
+                                  _ptr(u_accept, torch.float32, self.B * self.G * self.D, "u_accept", d),
                                   _ptr(u_resid, torch.float32, self.B, "u_resid", d),
                                   _ptr(out_n_accept, torch.int32, self.B, "out_n_accept", d),
                                   _ptr(out_next_token, torch.int32, self.B, "out_next_token", d)), "tabed_verify")
@@ -273,10 +277,10 @@ class Tabed:
                    out_w=None, out_w_argmax=None) -> None:
         cpu = torch.device("cpu")
         _check(lib().tabed_round_host(
-            self._h, _ptr(u_draft, torch.float32, self.B * self.G, "u_draft", cpu),
-            _ptr(u_accept, torch.float32, self.B * self.G, "u_accept", cpu), _ptr(u_resid, torch.float32, self.B, "u_resid", cpu),
-            _ptr(target_logits, torch.float32, self.B * (self.G + 1) * self.V, "target_logits", cpu),
-            _ptr(out_tokens, torch.int32, self.B * self.G, "out_tokens", cpu),
+            self._h, _ptr(u_draft, torch.float32, self.B * self.G * self.D, "u_draft", cpu),
+            _ptr(u_accept, torch.float32, self.B * self.G * self.D, "u_accept", cpu), _ptr(u_resid, torch.float32, self.B, "u_resid", cpu),
+            _ptr(target_logits, torch.float32, self.B * self.Rt * self.V, "target_logits", cpu),
+            _ptr(out_tokens, torch.int32, self.B * self.G * self.D, "out_tokens", cpu),
             _ptr(out_n_accept, torch.int32, self.B, "out_n_accept", cpu),
             _ptr(out_next_token, torch.int32, self.B, "out_next_token", cpu),
             _ptr(out_w, torch.float32, self.R, "out_w", cpu), _ptr(out_w_argmax, torch.int32, self.B, "out_w_argmax", cpu)),
@@ -289,7 +293,8 @@ class Tabed:
         _check(lib().tabed_debug_view(self._h, what, C.byref(ptr), C.byref(nbytes)), "tabed_debug_view")
         B, G, m, V, R = self.B, self.G, self.m, self.V, self.R
         shape, ts = {
-            VIEW_QK: ((B, G, m, V), "<f4"), VIEW_Q: ((B, G, V), "<f4"), VIEW_P: ((B, G + 1, V), "<f4"),
+            VIEW_QK: ((B, G, m, V), "<f4"), VIEW_Q: ((B, G, V), "<f4"), VIEW_P: ((B, self.Rt, V), "<f4"),
+            VIEW_ACC_PRIMARY: ((B,), "<i4"), VIEW_SIBLING: ((B,), "<i4"),
             VIEW_LOGITS: ((G, B, m, V), "<f4"), VIEW_KV_LEN: ((R,), "<i4"), VIEW_WEIGHTS: ((B, m), "<f4"),
             VIEW_WINDOW_SUM: ((B, MAX_DEV), "<i8"), VIEW_PENDING: ((B, 3), "<i4"), VIEW_GRID_J: ((B,), "<i4"),
             VIEW_ERROR_FLAG: ((1,), "<i4"),

@@ -321,7 +321,9 @@ struct PolicyArgs {
   int B, G, m, n_dev, h, policy, tvd, V;
   float tau;                 // temperature of the softmax policy; the constant C of the AdaBoost policy
   const float* u_policy;     // [B][m] uniforms of the random policy
-  const int* n_accept; const int* next_token; const int* tokens;   // [B], [B], [B][G]
+  const int* n_accept;       // [B] accepted tokens of the primary chain
+  const int* sib_tok;        // [B] token of the accepted sibling (token tree) or -1
+  const int* next_token; const int* tokens;   // [B], [B][G]
   long long* dev;            // [B][G][kMaxDev] deviation sums of the round's verified positions
   long long* ring;           // [B][h][kMaxDev]
   int* ring_head; int* ring_count; long long* pushed;              // [B]

@@ -31,6 +31,7 @@ constexpr int kReqWarps = kReqThreads / 32;
 constexpr int kReqMaxCluster = 16;          // CTAs per cluster (16 needs the non-portable opt-in, 8 is portable)
 constexpr int kReqMaxRows = 17;             // rows of one request handled together: gamma + 1 <= 17, m <= 8
 constexpr int kReqStep = kReqThreads * 4;   // vocabulary elements one pass of the CTA covers
+constexpr int kReqMaxWidth = 4;             // candidates per depth of a token tree
 
 struct ReqCtx {
   unsigned CS, rank;
@@ -82,8 +83,11 @@ struct ReqShared {
   float all_max[kReqMaxCluster][kReqMaxRows];
   unsigned long long all_sum[kReqMaxCluster][kReqMaxRows];
   ReqBest all_best[kReqMaxCluster][kReqMaxRows];
-  unsigned long long all_mass[2][kReqMaxCluster];
+  unsigned long long all_mass[4][kReqMaxCluster];
   unsigned long long scan[kReqWarps];
+  unsigned long long scan2[kReqWarps];
+  unsigned long long bc_mass[kReqMaxWidth];        // token and mass of candidate c, told to every CTA by the one that drew it
+  int bc_tok[kReqMaxWidth];
   int ok[kReqMaxRows];
   int result;
 };
@@ -184,6 +188,25 @@ __device__ __forceinline__ void req_gather_mass(cg::cluster_group& cluster, cons
   cluster.sync();
 }
 
+// Two block sums at once (buffers `which` and `which + 1`), one cluster barrier.
+__device__ __forceinline__ void req_gather_mass2(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, unsigned long long m0,
+                                                 unsigned long long m1, int which) {
+  m0 = warp_sum_u64(m0); m1 = warp_sum_u64(m1);
+  if (c.lane == 0) { S.scan[c.warp] = m0; S.scan2[c.warp] = m1; }
+  __syncthreads();
+  if (c.tid == 0) {
+    unsigned long long t0 = 0, t1 = 0;
+#pragma unroll
+    for (int w = 0; w < kReqWarps; ++w) { t0 += S.scan[w]; t1 += S.scan2[w]; }
+    for (unsigned r = 0; r < c.CS; ++r) {
+      unsigned long long* dst = cluster.map_shared_rank(&S.all_mass[0][0], r);
+      dst[which * kReqMaxCluster + c.rank] = t0;
+      dst[(which + 1) * kReqMaxCluster + c.rank] = t1;
+    }
+  }
+  cluster.sync();
+}
+
 // For the draw every thread owns a CONTIGUOUS range of the slice (so that a prefix over the threads is a prefix
 // over the vocabulary): [t_lo, t_hi), a multiple of 4 elements long.
 __device__ __forceinline__ void req_thread_range(const ReqCtx& c, int slice, int* t_lo, int* t_hi) {
@@ -277,6 +300,8 @@ __device__ __forceinline__ int req_best_of(const ReqCtx& c, const ReqShared& S, 
 // ------------------------------------------------------------------------------------------------
 struct EnsembleArgs {
   int V, m, greedy, slice;
+  int D;                                        // candidates per step (1: a plain chain); candidate c uses u[.. + c]
+  int* cand; int cand_stride;                   // optional: all candidates, cand[b * cand_stride + c] (-1: none left)
   const float* logits;
   const float* w;                               // [B][m]
   const float* u; int u_stride;                 // u[b * u_stride]
@@ -337,33 +362,104 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
       for (int j = 0; j < 4; ++j) if (v + j < c.v_hi && acc[j] > best.val) { best.val = acc[j]; best.idx = v + j; }
     }
   }
-  int y = 0, status = 0;
-  bool mine = false;
+  // the step's candidates: candidate 0 continues the chain; further ones (token tree) are drawn without replacement
+  const int D = A.D;
+  int chosen[kReqMaxWidth] = {-1, -1, -1, -1};
+  auto emit = [&](int cnd, int y) {
+    if (cnd == 0) A.out0[b * A.out0_stride] = y;
+    if (A.out1) A.out1[b * A.out1_stride + cnd] = y;
+    if (A.cand) A.cand[b * A.cand_stride + cnd] = y;
+  };
   if (A.greedy) {
-    req_gather_best(cluster, c, S, best, 0, true);
-    cluster.sync();
-    y = req_best_of(c, S, 0);
-    mine = c.rank == 0;
-  } else {
-    // masses of q over each thread's contiguous range (the slice was just written by this CTA: L1/L2 hold it)
-    __syncthreads();
-    int t_lo, t_hi;
-    req_thread_range(c, A.slice, &t_lo, &t_hi);
-#pragma unroll 4
-    for (int v = t_lo; v < t_hi; v += 4) {
-      float x[4];
-      req_ld4_rw(q_row, v, t_hi, vec_q, 0.0f, x);
+#pragma unroll 1
+    for (int cnd = 0; cnd < D; ++cnd) {
+      if (cnd > 0) {
+        // most likely token among those not chosen yet (the slice was written by this CTA: L1/L2 hold it)
+        best = ReqBest{-1.0f, 0x7fffffff};
+        __syncthreads();
+#pragma unroll 2
+        for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+          float x[4];
+          req_ld4_rw(q_row, v, c.v_hi, vec_q, -1.0f, x);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(x[j]);
+          for (int j = 0; j < 4; ++j) {
+            const int t = v + j;
+            if (t < c.v_hi && t != chosen[0] && t != chosen[1] && t != chosen[2] && x[j] > best.val) { best.val = x[j]; best.idx = t; }
+          }
+        }
+      }
+      // (the merge of the warps' bests uses one row of the exchange buffers per candidate)
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        ReqBest other;
+        other.val = __shfl_xor_sync(0xffffffffu, best.val, o);
+        other.idx = __shfl_xor_sync(0xffffffffu, best.idx, o);
+        best_merge(best, other);
+      }
+      if (c.lane == 0) S.red_b[c.warp][cnd] = best;
+      __syncthreads();
+      if (c.tid == 0) {
+        ReqBest t = S.red_b[0][cnd];
+#pragma unroll
+        for (int w = 1; w < kReqWarps; ++w) best_merge(t, S.red_b[w][cnd]);
+        for (unsigned r = 0; r < c.CS; ++r) cluster.map_shared_rank(&S.all_best[0][0], r)[c.rank * kReqMaxRows + cnd] = t;
+      }
+      cluster.sync();
+      ReqBest t = S.all_best[0][cnd];
+      for (unsigned r = 1; r < c.CS; ++r) best_merge(t, S.all_best[r][cnd]);
+      const int y = t.val < 0.0f ? -1 : t.idx;              // fewer tokens than candidates
+      chosen[cnd] = y;
+      if (c.rank == 0 && c.tid == 0) emit(cnd, y);
     }
-    req_gather_mass(cluster, c, S, mass, 0);
-    mine = req_draw(c, S, 0, A.u[b * A.u_stride], mass, t_lo, t_hi, [&](int v) { return mass_of(q_row[v]); }, &y, &status);
-    if (status == 1 && c.rank == 0) { mine = true; y = 0; }
+    return;
   }
-  if (mine && c.tid == 0) {
-    if (status && A.err) atomicOr(A.err, status);
-    A.out0[b * A.out0_stride] = y;
-    if (A.out1) A.out1[b * A.out1_stride] = y;
+  // masses of q over each thread's contiguous range (the slice was just written by this CTA: L1/L2 hold it)
+  __syncthreads();
+  int t_lo, t_hi;
+  req_thread_range(c, A.slice, &t_lo, &t_hi);
+#pragma unroll 4
+  for (int v = t_lo; v < t_hi; v += 4) {
+    float x[4];
+    req_ld4_rw(q_row, v, t_hi, vec_q, 0.0f, x);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(x[j]);
+  }
+  req_gather_mass(cluster, c, S, mass, 0);
+  auto mass_left = [&](int v) { return (v == chosen[0] || v == chosen[1] || v == chosen[2]) ? 0ull : mass_of(q_row[v]); };
+#pragma unroll 1
+  for (int cnd = 0; cnd < D; ++cnd) {
+    int y = 0, status = 0;
+    const bool mine = req_draw(c, S, 0, A.u[b * A.u_stride + cnd], mass, t_lo, t_hi, mass_left, &y, &status);
+    if (status == 1) {
+      // nothing (left) to draw from: an error for the chain's own token, "no candidate" for a sibling
+      if (c.rank == 0 && c.tid == 0) {
+        if (cnd == 0) { if (A.err) atomicOr(A.err, 1); emit(0, 0); }
+        for (int k = cnd > 0 ? cnd : 1; k < D; ++k) emit(k, -1);
+      }
+      break;
+    }
+    if (mine && c.tid == 0) {
+      if (status && A.err) atomicOr(A.err, status);
+      emit(cnd, y);
+    }
+    if (cnd + 1 == D) break;
+    // tell every CTA which token went and how much mass leaves with it
+    if (mine && c.tid == 0) {
+      const unsigned long long my = (status == 0) ? mass_of(q_row[y]) : 0ull;
+      for (unsigned r = 0; r < c.CS; ++r) {
+        cluster.map_shared_rank(&S.bc_tok[0], r)[cnd] = (status == 0) ? y : -1;
+        cluster.map_shared_rank(&S.bc_mass[0], r)[cnd] = my;
+      }
+    }
+    cluster.sync();
+    const int yt = S.bc_tok[cnd];
+    chosen[cnd] = yt;
+    if (yt >= 0) {
+      const unsigned long long my = S.bc_mass[cnd];
+      if (c.tid == 0) S.all_mass[0][yt / A.slice] -= my;
+      if (yt >= t_lo && yt < t_hi) mass -= my;
+      __syncthreads();
+    }
   }
 }
 
@@ -387,12 +483,16 @@ __device__ __forceinline__ bool req_last_of_request(cg::cluster_group& cluster, 
 // ------------------------------------------------------------------------------------------------
 struct VerifyArgs {
   int V, G, greedy, slice;
-  const float* logits;                          // target [B][G+1][V]
+  int D;                                        // candidates per depth (token tree; 1: a plain chain)
+  const float* logits;                          // target [B][Rt][V], Rt = G + 1 + G (D - 1): the chain's positions, then the
+                                                // leaf after sibling c of depth i at row G + 1 + i (D - 1) + (c - 1)
   const float* q; long long q_req_stride;       // ensembled [B][..][V], position pitch V
-  const int* tokens;                            // [B][G]
-  const float* u_accept;                        // [B][G]
+  const int* tokens;                            // [B][G] the primary chain
+  const int* cand;                              // [B][G][D] all candidates (column 0 = tokens)
+  const float* u_accept;                        // [B][G][D]
   const float* u_resid;                         // [B]
-  float* p;                                     // [B][G+1][V]
+  float* p;                                     // [B][Rt][V]
+  int *acc_prim, *sib_tok;                      // [B] accepted tokens of the primary chain; the accepted sibling's token or -1
   int* row_flag;                                // [B][G+1] scratch: accept flag of position i (greedy: argmax of p_i)
   int* ticket;                                  // [B] scratch, zero between launches
   int *n_accept, *out_n_accept, *next_token, *out_next_token;
@@ -405,11 +505,11 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
   __shared__ ReqShared S;
   __shared__ int s_last;
   const ReqCtx c = req_ctx(cluster, A.V, A.slice);
-  const int G = A.G, V = A.V, rows = G + 1;
+  const int G = A.G, V = A.V, rows = G + 1, D = A.D, Rt = G + 1 + G * (D - 1);
   const int unit = blockIdx.x / c.CS, b = unit / rows, i = unit - b * rows;
   pdl_wait();
-  const float* lg = A.logits + ((long long)b * rows + i) * V;
-  float* p_b = A.p + (long long)b * rows * V;
+  const float* lg = A.logits + ((long long)b * Rt + i) * V;
+  float* p_b = A.p + (long long)b * Rt * V;
   const float* q_b = A.q + (long long)b * A.q_req_stride;
   const bool vec = req_vec_ok(A.logits, V), vec_p = (V & 3) == 0;
   req_row_maxima(cluster, c, S, lg, V, 1, vec);
@@ -439,66 +539,149 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
       const int y = A.tokens[b * G + i];
       const float py = __fdiv_rn(xexp(__fsub_rn(__ldg(lg + y), mx)), sn);          // the value stored in p_i[y]
       const float qy = __ldg(q_b + (long long)i * V + y);
-      flag = (py >= qy) || (__fmul_rn(A.u_accept[b * G + i], qy) < py);
+      flag = (py >= qy) || (__fmul_rn(A.u_accept[(b * G + i) * D], qy) < py);
     } else flag = 1;
     A.row_flag[b * rows + i] = flag;
   }
   if (!req_last_of_request(cluster, c, &s_last, A.ticket + b, rows)) return;
 
-  // ---- the request's last cluster: acceptance prefix, replacement / bonus token -----------------------
+  // ---- the request's last cluster: acceptance prefix, siblings of the first rejected depth, next token --------
   int a = 0;
   for (; a < G; ++a) {
     const int f = __ldcg(A.row_flag + b * rows + a);
     if (A.greedy ? (f != A.tokens[b * G + a]) : (f == 0)) break;
   }
-  if (c.rank == 0 && c.tid == 0) {
-    A.n_accept[b] = a;
-    if (A.out_n_accept) A.out_n_accept[b] = a;
-  }
-  int z = 0, status = 0;
-  bool mine = false;
+  const float u = A.u_resid[b];
+  int t_lo, t_hi;
+  req_thread_range(c, A.slice, &t_lo, &t_hi);
+  int n_acc = a, sib = -1, z = 0, status = 0;
+  bool mine = false, have_z = false;
+  // Next token from the target's distribution of one row, computed here (a leaf of the tree): softmax, then draw / argmax.
+  auto from_row = [&](int row) {
+    const float* lr = A.logits + ((long long)b * Rt + row) * V;
+    float* pr = p_b + (long long)row * V;
+    req_row_maxima(cluster, c, S, lr, V, 1, vec);
+    req_row_sums(cluster, c, S, lr, V, 1, vec);
+    const float mx2 = req_max_of(c, S, 0), sn2 = req_norm_of(c, S, 0);
+    unsigned long long mass = 0;
+    ReqBest best{-1.0f, 0x7fffffff};
+#pragma unroll 2
+    for (int v = t_lo; v < t_hi; v += 4) {
+      float x[4];
+      req_ld4(lr, v, t_hi, vec, -INFINITY, x);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        x[j] = __fdiv_rn(xexp(__fsub_rn(x[j], mx2)), sn2);
+        if (v + j < t_hi) { mass += mass_of(x[j]); if (x[j] > best.val) { best.val = x[j]; best.idx = v + j; } }
+      }
+      req_st4(pr, v, t_hi, vec_p, x);
+    }
+    if (A.greedy) {
+      req_gather_best(cluster, c, S, best, 0, true);
+      cluster.sync();
+      z = req_best_of(c, S, 0);
+      mine = c.rank == 0;
+    } else {
+      req_gather_mass(cluster, c, S, mass, 0);
+      mine = req_draw(c, S, 0, u, mass, t_lo, t_hi,
+                      [&](int v) { return mass_of(__fdiv_rn(xexp(__fsub_rn(__ldg(lr + v), mx2)), sn2)); }, &z, &status);
+      if (status == 1 && c.rank == 0) { mine = true; z = 0; }
+    }
+  };
   if (A.greedy) {
-    z = __ldcg(A.row_flag + b * rows + a);
-    mine = c.rank == 0;
-  } else {
-    // replacement token from norm(max(0, p_a - q_a)) (from p_a if that has no mass); bonus token from p_G.
-    // p_a was written by another cluster of this launch: read through L2.
-    const float* p_a = p_b + (long long)a * V;
-    const float* q_a = (a < G) ? q_b + (long long)a * V : nullptr;
-    auto p_at = [&](int v) { return __ldcg(p_a + v); };
-    int t_lo, t_hi;
-    req_thread_range(c, A.slice, &t_lo, &t_hi);
-    auto ld_p4 = [&](int v, float (&x)[4]) {
-      if (vec_p && v + 4 <= t_hi) { const float4 t = __ldcg(reinterpret_cast<const float4*>(p_a + v)); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
-      else { for (int j = 0; j < 4; ++j) x[j] = (v + j < t_hi) ? __ldcg(p_a + v + j) : 0.0f; }
+    if (a < G) {
+      const int t = __ldcg(A.row_flag + b * rows + a);            // the target's token at the first depth that differs
+      for (int cnd = 1; cnd < D; ++cnd) if (sib < 0 && A.cand[(b * G + a) * D + cnd] == t) sib = cnd;
+      if (sib < 0) { z = t; mine = c.rank == 0; have_z = true; }
+    } else {
+      z = __ldcg(A.row_flag + b * rows + G); mine = c.rank == 0; have_z = true;
+    }
+  } else if (a < G) {
+    // Recursive rejection over the depth's candidates.  Level l distributions are functions of (p_a, q_a) and of the
+    // scalars of the levels before: r = max(0, p - q); p' = r / Rn; q' = q / Qn with the tried tokens at 0.
+    const float* p_a = p_b + (long long)a * V;                   // written by another cluster of this launch: read through L2
+    const float* q_a = q_b + (long long)a * V;
+    float Rn[kReqMaxWidth], Qn[kReqMaxWidth];
+    int xs[kReqMaxWidth];
+#pragma unroll
+    for (int k = 0; k < kReqMaxWidth; ++k) { xs[k] = k < D ? A.cand[(b * G + a) * D + k] : -1; Rn[k] = 1.0f; Qn[k] = 1.0f; }
+    auto elem = [&](int v, int level, float& pl, float& ql) {
+      pl = __ldcg(p_a + v); ql = __ldg(q_a + v);
+#pragma unroll
+      for (int l = 1; l < kReqMaxWidth; ++l) {
+        if (l > level) break;
+        const float r = resid_val(pl, ql);
+        pl = __fdiv_rn(r, Rn[l]);
+        ql = (v == xs[l - 1]) ? 0.0f : __fdiv_rn(ql, Qn[l]);
+      }
     };
-    const bool vec_qa = q_a && req_vec_ok(A.q, A.q_req_stride) && (V & 3) == 0;
+    int level = 0;
+#pragma unroll 1
+    while (true) {
+      // this level's residual masses (per thread range) and the mass of q_level
+      unsigned long long mr = 0, mq = 0;
+#pragma unroll 4
+      for (int v = t_lo; v < t_hi; ++v) {
+        float pl, ql;
+        elem(v, level, pl, ql);
+        mr += mass_of(resid_val(pl, ql));
+        mq += mass_of(ql);
+      }
+      const int buf = 2 * (level & 1);
+      req_gather_mass2(cluster, c, S, mr, mq, buf);
+      unsigned long long MR = 0, MQ = 0;
+      for (unsigned r = 0; r < c.CS; ++r) { MR += S.all_mass[buf][r]; MQ += S.all_mass[buf + 1][r]; }
+      float px, qx;
+      elem(xs[level], level, px, qx);
+      const unsigned long long MQrest = MQ - mass_of(qx);
+      const bool more = level + 1 < D && xs[level + 1] >= 0 && MR != 0ull && MQrest != 0ull;
+      if (!more) {
+        // the replacement: from this level's residual, or from p_level itself if that has no mass
+        if (MR != 0ull) {
+          mine = req_draw(c, S, buf, u, mr, t_lo, t_hi,
+                          [&](int v) { float pl, ql; elem(v, level, pl, ql); return mass_of(resid_val(pl, ql)); }, &z, &status);
+        } else {
+          unsigned long long mp = 0;
+#pragma unroll 1
+          for (int v = t_lo; v < t_hi; ++v) { float pl, ql; elem(v, level, pl, ql); mp += mass_of(pl); }
+          req_gather_mass(cluster, c, S, mp, buf ^ 2);
+          mine = req_draw(c, S, buf ^ 2, u, mp, t_lo, t_hi, [&](int v) { float pl, ql; elem(v, level, pl, ql); return mass_of(pl); }, &z, &status);
+        }
+        if (status == 1 && c.rank == 0) { mine = true; z = 0; }
+        have_z = true;
+        break;
+      }
+      Rn[level + 1] = norm_of(MR);
+      Qn[level + 1] = norm_of(MQrest);
+      ++level;
+      elem(xs[level], level, px, qx);
+      if ((px >= qx) || (__fmul_rn(A.u_accept[(b * G + a) * D + level], qx) < px)) { sib = level; break; }
+    }
+  }
+  if (sib >= 0) {
+    n_acc = a + 1;
+    from_row(G + 1 + a * (D - 1) + (sib - 1));                   // the leaf after the accepted sibling
+  } else if (!have_z) {
+    // every primary accepted: bonus token from p_G
+    const float* p_g = p_b + (long long)G * V;
     unsigned long long mass = 0;
 #pragma unroll 4
     for (int v = t_lo; v < t_hi; v += 4) {
-      float pa[4], qa[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-      ld_p4(v, pa);
-      if (q_a) req_ld4(q_a, v, t_hi, vec_qa, 0.0f, qa);
+      float x[4];
+      if (vec_p && v + 4 <= t_hi) { const float4 t = __ldcg(reinterpret_cast<const float4*>(p_g + v)); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
+      else { for (int j = 0; j < 4; ++j) x[j] = (v + j < t_hi) ? __ldcg(p_g + v + j) : 0.0f; }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(q_a ? resid_val(pa[j], qa[j]) : pa[j]);
+      for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(x[j]);
     }
     req_gather_mass(cluster, c, S, mass, 0);
-    const float u = A.u_resid[b];
-    mine = req_draw(c, S, 0, u, mass, t_lo, t_hi, [&](int v) { return mass_of(q_a ? resid_val(p_at(v), __ldg(q_a + v)) : p_at(v)); }, &z, &status);
-    if (status == 1 && q_a) {
-      // residual without mass (p_a == q_a bitwise): draw from p_a itself.  Every CTA sees the same zero total.
-      mass = 0;
-#pragma unroll 4
-      for (int v = t_lo; v < t_hi; v += 4) {
-        float pa[4];
-        ld_p4(v, pa);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) if (v + j < t_hi) mass += mass_of(pa[j]);
-      }
-      req_gather_mass(cluster, c, S, mass, 1);
-      mine = req_draw(c, S, 1, u, mass, t_lo, t_hi, [&](int v) { return mass_of(p_at(v)); }, &z, &status);
-    }
+    mine = req_draw(c, S, 0, u, mass, t_lo, t_hi, [&](int v) { return mass_of(__ldcg(p_g + v)); }, &z, &status);
     if (status == 1 && c.rank == 0) { mine = true; z = 0; }
+  }
+  if (c.rank == 0 && c.tid == 0) {
+    A.n_accept[b] = n_acc;
+    if (A.out_n_accept) A.out_n_accept[b] = n_acc;
+    A.acc_prim[b] = a;
+    A.sib_tok[b] = sib >= 0 ? A.cand[(b * G + a) * D + sib] : -1;
   }
   if (mine && c.tid == 0) {
     if (status && A.err) atomicOr(A.err, status);
@@ -514,9 +697,10 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
 // ------------------------------------------------------------------------------------------------
 struct UpdateArgs {
   int V, slice, grid_policy;
+  int Rt;                         // rows of p per request (G + 1, more with a token tree)
   int hard;                       // 0: soft labels (distance sums); 1: hard labels - whether each grid candidate's most likely
                                   // token is the verified token (matches); 2: whether each drafter's is NOT (errors)
-  const float* p;                 // [B][G+1][V]
+  const float* p;                 // [B][Rt][V]
   const float* qk;                // [B][G][m][V]
   int* ticket;                    // [B] scratch, zero between launches
   PolicyArgs P;                   // P.dev: [B][G][kMaxDev] scratch (every verified entry is rewritten each round)
@@ -604,12 +788,13 @@ __global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs 
       ReqBest t = U.all_b[0][c.tid];
       for (unsigned r = 1; r < c.CS; ++r) best_merge(t, U.all_b[r][c.tid]);
       // the verified token of position i: the accepted draft, or the replacement at the rejected position
-      const int label = (i < a) ? P.tokens[b * G + i] : P.next_token[b];
+      const int sib = P.sib_tok[b];
+      const int label = (i < a) ? P.tokens[b * G + i] : (sib >= 0 ? sib : P.next_token[b]);
       const int hit = t.idx == label;
       P.dev[((long long)b * G + i) * kMaxDev + c.tid] = (A.hard == 1) ? hit : 1 - hit;
     }
   } else {
-    const float* p_i = A.p + ((long long)b * (G + 1) + i) * V;
+    const float* p_i = A.p + ((long long)b * A.Rt + i) * V;
     const float* qbase = A.qk + ((long long)b * G + i) * m * V;
     long long acc[kMaxDev];
 #pragma unroll
@@ -791,9 +976,12 @@ __device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int la
     const int keep = cnt + (a < A.G ? a : A.G - 1);
     for (int k = 0; k < A.m; ++k) A.kv_len[b * A.m + k] += keep;
   }
-  const int z = A.next_token[b];
-  if (a < A.G) { pend[0] = 1; pend[1] = z; pend[2] = 0; }
-  else { pend[0] = 2; pend[1] = A.tokens[b * A.G + A.G - 1]; pend[2] = z; }
+  // ... and what the target emitted beyond them is pending: the replacement; or an accepted sibling (token tree) or the
+  // last accepted draft of a fully accepted block, followed by the next token
+  const int z = A.next_token[b], sib = A.sib_tok[b];
+  if (a == A.G) { pend[0] = 2; pend[1] = A.tokens[b * A.G + A.G - 1]; pend[2] = z; }
+  else if (sib >= 0) { pend[0] = 2; pend[1] = sib; pend[2] = z; }
+  else { pend[0] = 1; pend[1] = z; pend[2] = 0; }
 }
 
 }  // namespace tabed

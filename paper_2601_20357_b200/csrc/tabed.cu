@@ -46,6 +46,8 @@ struct tabed_handle {
   bool has_drafter = false;
   cudaStream_t stream = nullptr;
   int R = 0, B = 0, m = 0, G = 0, V = 0, d = 0, F = 0, H = 0, Hkv = 0, hd = 0, L = 0, cap = 0;
+  int D = 1, Rt = 0;                // token tree: candidates per depth; target rows per request G + 1 + G (D - 1)
+  int *cand = nullptr, *acc_prim = nullptr, *sib_tok = nullptr;   // [B][G][D] candidates; [B] accepted primaries; [B] sibling token
   int n_dev = 0, n_chunks = 0, ns = 1, max_splits = 0, qkv_w = 0;
   size_t esz = 4;
   // drafter (caller-owned device memory)
@@ -73,6 +75,7 @@ struct tabed_handle {
   // host-side state
   int phase = PH_IDLE;
   bool round_has_forward = false;
+  bool cand_is_tokens = false;      // the round's candidates are its tokens (drafted by the persistent kernel: chains only)
   const float* logits_override = nullptr;   // tabed_debug_override_logits
   const float* u_policy = nullptr;          // tabed_set_policy_uniforms (random weight policy)
   std::vector<int> len_ub;          // upper bound of every row's committed length
@@ -371,7 +374,7 @@ void run_step(tabed_handle* h, StepArgs sa, int n_slots, int max_pos, float* log
 // Algorithm 1 steps 6-7 for all requests on logits [B][m][V]: one launch, one cluster per request.
 void run_ensemble(tabed_handle* h, const float* logits, const float* w, const float* u, int u_stride,
                   int* y0, int y0_stride, int* y1, int y1_stride, float* qk_out, long long qk_stride,
-                  float* q_out, long long q_stride) {
+                  float* q_out, long long q_stride, int n_cand = 1, int* cand = nullptr, int cand_stride = 0) {
   ProfScope ps(h, TABED_PROF_ENSEMBLE);
   EnsembleArgs a{};
   const int cs = pick_cluster(h, h->B, &a.slice);
@@ -379,6 +382,7 @@ void run_ensemble(tabed_handle* h, const float* logits, const float* w, const fl
   a.logits = logits; a.w = w; a.u = u; a.u_stride = u_stride;
   a.qk_out = qk_out; a.qk_req_stride = qk_stride; a.q_out = q_out; a.q_req_stride = q_stride;
   a.out0 = y0; a.out0_stride = y0_stride; a.out1 = y1; a.out1_stride = y1_stride; a.err = h->err;
+  a.D = n_cand; a.cand = cand; a.cand_stride = cand_stride;
   launch_request_clusters(h, k_ensemble_req, h->B, cs, a);
 }
 
@@ -398,7 +402,7 @@ PhaseGeom pick_geom(int n_tiles, int K, int kcap) {
 int setup_persistent(tabed_handle* h) {
   const tabed_config& c = h->cfg;
   h->persist_ok = false;
-  if (c.dtype != TABED_DTYPE_BF16) return TABED_OK;
+  if (c.dtype != TABED_DTYPE_BF16 || h->D > 1) return TABED_OK;      // (the in-kernel draw proposes one candidate per step)
   const int grp = h->H / h->Hkv;
   if (2 * h->R > kPSlots || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
       grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || (h->cap + 127) / 128 > kAttnSplitMax)
@@ -737,7 +741,8 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   const tabed_config& c = *cfg;
   if (c.vocab < 2 || c.n_inputs < 1 || c.n_inputs > TABED_MAX_INPUTS || c.n_requests < 1 || c.gamma < 1 ||
       c.gamma > 16 || c.window_h < 0 || c.window_h > 64 || c.policy < 0 || c.policy > TABED_POLICY_ADABOOST || c.distance < 0 ||
-      c.distance > 1 || c.sample_mode < 0 || c.sample_mode > 1 || !(c.tau > 0.0f) || c.device < 0)
+      c.distance > 1 || c.sample_mode < 0 || c.sample_mode > 1 || !(c.tau > 0.0f) || c.device < 0 || c.tree_width < 0 ||
+      c.tree_width > TABED_MAX_TREE_WIDTH)
     return TABED_ERR_INVALID_ARG;
   if ((c.policy == TABED_POLICY_GRID_MT || c.policy == TABED_POLICY_GRID_HARD) && c.n_inputs != 2) return TABED_ERR_INVALID_ARG;
   if ((long long)c.n_requests * c.n_inputs > 4096) return TABED_ERR_UNSUPPORTED;
@@ -774,6 +779,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   if (!h) return TABED_ERR_CUDA;
   h->cfg = c; h->stream = reinterpret_cast<cudaStream_t>(c.stream);
   h->B = c.n_requests; h->m = c.n_inputs; h->R = h->B * h->m; h->G = c.gamma; h->V = c.vocab;
+  h->D = std::max(1, c.tree_width); h->Rt = h->G + 1 + h->G * (h->D - 1);
   h->n_dev = (c.policy == TABED_POLICY_GRID_MT || c.policy == TABED_POLICY_GRID_HARD) ? kGridCand : h->m;
   h->n_chunks = (h->V + kChunk - 1) / kChunk;
   h->ns = pick_ns(h->R);
@@ -807,11 +813,13 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   A(&h->dev, B * G * kMaxDev); A(&h->ring, B * std::max(1, c.window_h) * kMaxDev); A(&h->running, B * kMaxDev);
   A(&h->req_ticket, 2 * B); A(&h->row_flag, B * (G + 1));
   A(&h->pushed, B); A(&h->ring_head, B); A(&h->ring_count, B); A(&h->grid_j, B);
-  A(&h->qk, B * G * m * V); A(&h->q, B * G * V); A(&h->p, B * (G + 1) * V); A(&h->scratch_q, B * V);
+  const size_t Dw = h->D, Rt = h->Rt;
+  A(&h->qk, B * G * m * V); A(&h->q, B * G * V); A(&h->p, B * Rt * V); A(&h->scratch_q, B * V);
   A(&h->tokens, B * G); A(&h->n_accept, B); A(&h->next_token, B); A(&h->w_argmax, B);
+  A(&h->cand, B * G * Dw); A(&h->acc_prim, B); A(&h->sib_tok, B);
   A(&h->chunk_mass, B * h->n_chunks); A(&h->chunk_best, B * h->n_chunks);
   A(&h->err, 1);
-  A(&h->st_u_draft, B * G); A(&h->st_u_accept, B * G); A(&h->st_u_resid, B); A(&h->st_target, B * (G + 1) * V); A(&h->st_tokens, B * G);
+  A(&h->st_u_draft, B * G * Dw); A(&h->st_u_accept, B * G * Dw); A(&h->st_u_resid, B); A(&h->st_target, B * Rt * V); A(&h->st_tokens, B * G * Dw);
   if (h->has_drafter) {
     h->L = c.n_layers; h->d = c.d_model; h->F = c.d_ffn; h->H = c.n_heads; h->Hkv = c.n_kv_heads;
     h->hd = c.d_model / c.n_heads; h->cap = c.kv_capacity; h->esz = c.dtype == TABED_DTYPE_FP32 ? 4 : 2;
@@ -1042,6 +1050,7 @@ static int draft_common(tabed_handle* h, const float* ext_logits, const float* u
       return TABED_ERR_CUDA;
     h->phase = PH_DRAFTED;
     h->round_has_forward = true;
+    h->cand_is_tokens = true;
     return check_cuda();
   }
   for (int i = 0; i < h->G; ++i) {
@@ -1056,13 +1065,15 @@ static int draft_common(tabed_handle* h, const float* ext_logits, const float* u
     } else {
       lg = ext_logits + i * RV;
     }
-    run_ensemble(h, lg, h->w, u_draft + i, h->G, h->tokens + i, h->G, out_tokens + i, h->G,
-                 h->qk + (long long)i * h->m * h->V, GV * h->m, h->q + (long long)i * h->V, GV);
+    run_ensemble(h, lg, h->w, u_draft + i * h->D, h->G * h->D, h->tokens + i, h->G, out_tokens + i * h->D, h->G * h->D,
+                 h->qk + (long long)i * h->m * h->V, GV * h->m, h->q + (long long)i * h->V, GV,
+                 h->D, h->cand + i * h->D, h->G * h->D);
   }
   if (out_q && cudaMemcpyAsync(out_q, h->q, sizeof(float) * h->B * GV, cudaMemcpyDeviceToDevice, h->stream) != cudaSuccess)
     return TABED_ERR_CUDA;
   h->phase = PH_DRAFTED;
   h->round_has_forward = fwd;
+  h->cand_is_tokens = false;
   return check_cuda();
 }
 
@@ -1085,6 +1096,7 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   VerifyArgs a{};
   const int cs = pick_cluster(h, h->B * (h->G + 1), &a.slice);
   a.row_flag = h->row_flag; a.ticket = h->req_ticket;
+  a.D = h->D; a.cand = h->cand_is_tokens ? h->tokens : h->cand; a.acc_prim = h->acc_prim; a.sib_tok = h->sib_tok;
   a.V = h->V; a.G = h->G; a.greedy = h->cfg.sample_mode == TABED_MODE_GREEDY;
   a.logits = target_logits; a.q = h->q; a.q_req_stride = (long long)h->G * h->V; a.tokens = h->tokens;
   a.u_accept = u_accept; a.u_resid = u_resid; a.p = h->p;
@@ -1106,7 +1118,7 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
     ProfScope ps(h, TABED_PROF_UPDATE);
     UpdateArgs u{};
     const int cs = pick_cluster(h, h->B * h->G, &u.slice);
-    u.ticket = h->req_ticket + h->B;
+    u.ticket = h->req_ticket + h->B; u.Rt = h->Rt;
     u.V = h->V;
     u.grid_policy = (h->cfg.policy == TABED_POLICY_GRID_MT || h->cfg.policy == TABED_POLICY_GRID_HARD) ? 1 : 0;
     u.hard = h->cfg.policy == TABED_POLICY_GRID_HARD ? 1 : (h->cfg.policy == TABED_POLICY_ADABOOST ? 2 : 0);
@@ -1114,7 +1126,7 @@ int tabed_update_weights(tabed_handle* h, float* out_w, int32_t* out_w_argmax) {
     PolicyArgs& a = u.P;
     a.B = h->B; a.G = h->G; a.m = h->m; a.n_dev = h->n_dev; a.h = h->cfg.window_h; a.policy = h->cfg.policy; a.tvd = tvd;
     a.V = h->V; a.u_policy = h->u_policy;
-    a.tau = h->cfg.tau; a.n_accept = h->n_accept; a.next_token = h->next_token; a.tokens = h->tokens;
+    a.tau = h->cfg.tau; a.n_accept = h->acc_prim; a.sib_tok = h->sib_tok; a.next_token = h->next_token; a.tokens = h->tokens;
     a.dev = h->dev; a.ring = h->ring; a.ring_head = h->ring_head; a.ring_count = h->ring_count; a.pushed = h->pushed;
     a.running = h->running; a.w = h->w; a.grid_j = h->grid_j;
     a.kv_len = (h->has_drafter && h->round_has_forward) ? h->kv_len : nullptr;
@@ -1136,12 +1148,12 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
     return TABED_ERR_NULL_PTR;
   if (h->phase != PH_IDLE || !h->has_drafter) return TABED_ERR_BAD_STATE;
   DeviceGuard guard(h->cfg.device);
-  const size_t BG = (size_t)h->B * h->G;
+  const size_t BG = (size_t)h->B * h->G * h->D;
   cudaStream_t st = h->stream;
   if (cudaMemcpyAsync(h->st_u_draft, u_draft, BG * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(h->st_u_accept, u_accept, BG * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(h->st_u_resid, u_resid, (size_t)h->B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(h->st_target, target_logits, (size_t)h->B * (h->G + 1) * h->V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      cudaMemcpyAsync(h->st_target, target_logits, (size_t)h->B * h->Rt * h->V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return TABED_ERR_CUDA;
   const std::vector<int> len_before = h->len_ub, cnt_before = h->pend_cnt;
   const bool known_before = h->pend_known;
@@ -1152,11 +1164,15 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
   if (rc != TABED_OK) return rc;
   rc = tabed_update_weights(h, nullptr, h->w_argmax);
   if (rc != TABED_OK) return rc;
-  if (cudaMemcpyAsync(out_tokens, h->tokens, BG * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+  if (cudaMemcpyAsync(out_tokens, h->st_tokens, BG * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaMemcpyAsync(out_n_accept, h->n_accept, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaMemcpyAsync(out_next_token, h->next_token, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       (out_w && cudaMemcpyAsync(out_w, h->w, (size_t)h->B * h->m * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) ||
       (out_w_argmax && cudaMemcpyAsync(out_w_argmax, h->w_argmax, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess))
+    return TABED_ERR_CUDA;
+  std::vector<int> h_prim(h->B), h_sib(h->B);
+  if (cudaMemcpyAsync(h_prim.data(), h->acc_prim, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(h_sib.data(), h->sib_tok, (size_t)h->B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return TABED_ERR_CUDA;
   // the device-side error word comes back with the results (this call synchronises anyway)
   int bits = 0;
@@ -1166,9 +1182,9 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
   if (known_before) {
     // exact lengths: a row keeps its pending token(s) and the accepted drafts that were fed
     for (int b = 0; b < h->B; ++b) {
-      const int a = out_n_accept[b], keep = cnt_before[b] + std::min(a, h->G - 1);
+      const int a = h_prim[b], keep = cnt_before[b] + std::min(a, h->G - 1);       // accepted tokens of the primary chain
       for (int k = 0; k < h->m; ++k) h->len_ub[b * h->m + k] = std::min(len_before[b * h->m + k] + keep, h->cap);
-      h->pend_cnt[b] = (a >= h->G) ? 2 : 1;
+      h->pend_cnt[b] = (a >= h->G || h_sib[b] >= 0) ? 2 : 1;
     }
     h->pend_known = true;
   }
@@ -1295,7 +1311,9 @@ int tabed_debug_view(tabed_handle* h, int32_t what, void** dev_ptr, size_t* byte
   switch (what) {
     case TABED_VIEW_QK: *dev_ptr = h->qk; *bytes = B * G * m * V * 4; break;
     case TABED_VIEW_Q: *dev_ptr = h->q; *bytes = B * G * V * 4; break;
-    case TABED_VIEW_P: *dev_ptr = h->p; *bytes = B * (G + 1) * V * 4; break;
+    case TABED_VIEW_P: *dev_ptr = h->p; *bytes = B * (size_t)h->Rt * V * 4; break;
+    case TABED_VIEW_ACC_PRIMARY: *dev_ptr = h->acc_prim; *bytes = B * 4; break;
+    case TABED_VIEW_SIBLING: *dev_ptr = h->sib_tok; *bytes = B * 4; break;
     case TABED_VIEW_LOGITS: if (!h->has_drafter) return TABED_ERR_BAD_STATE; *dev_ptr = h->logits_own; *bytes = G * R * V * 4; break;
     case TABED_VIEW_KV_LEN: if (!h->has_drafter) return TABED_ERR_BAD_STATE; *dev_ptr = h->kv_len; *bytes = R * 4; break;
     case TABED_VIEW_WEIGHTS: *dev_ptr = h->w; *bytes = B * m * 4; break;

@@ -89,6 +89,12 @@ class Workload:
     distance: int = DIST_KL
     sample_mode: int = MODE_SAMPLE
     tau: float = 1.0
+    tree_width: int = 1            # candidates per depth of the token tree (Sec. 5); 1 = a plain chain
+
+    @property
+    def n_target_rows(self) -> int:
+        """Rows of target logits per request: the chain's gamma + 1 positions, then one leaf per sibling candidate."""
+        return self.gamma + 1 + self.gamma * (self.tree_width - 1)
 
     @property
     def n_rows(self) -> int:
@@ -307,12 +313,14 @@ def lattice_uniforms(g: np.random.Generator, shape) -> np.ndarray:
 
 
 def round_uniforms(wl: Workload, rnd: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
-    """(u_draft [B][gamma], u_accept [B][gamma], u_resid [B]) of one round."""
+    """(u_draft [B][gamma], u_accept [B][gamma], u_resid [B]) of one round; with a token tree of width d the first two
+    are [B][gamma][d] (one uniform per candidate)."""
     g = substream(wl.config_id, "uniforms", rnd)
-    u = lattice_uniforms(g, (wl.n_requests, 2 * wl.gamma + 1))
-    G = wl.gamma
-    return (np.ascontiguousarray(u[:, :G]), np.ascontiguousarray(u[:, G:2 * G]),
-            np.ascontiguousarray(u[:, 2 * G]))
+    G, d = wl.gamma, wl.tree_width
+    u = lattice_uniforms(g, (wl.n_requests, 2 * G * d + 1))
+    shape = (wl.n_requests, G) if d == 1 else (wl.n_requests, G, d)
+    return (np.ascontiguousarray(u[:, :G * d]).reshape(shape), np.ascontiguousarray(u[:, G * d:2 * G * d]).reshape(shape),
+            np.ascontiguousarray(u[:, 2 * G * d]))
 
 
 def policy_uniforms(wl: Workload, rnd: int) -> np.ndarray:
@@ -345,6 +353,14 @@ def target_logits(wl: Workload, rnd: int, drafter_logits: np.ndarray) -> np.ndar
     out[:, G] = mix[:, G - 1]
     g = substream(wl.config_id, "target_noise", rnd)
     out += np.float32(wl.sigma(rnd)) * g.standard_normal(out.shape, dtype=np.float32)
+    if wl.tree_width > 1:
+        # leaves of the token tree: the target's distribution after sibling c of depth i stands in as the mix of the
+        # next step (the last step's for the deepest leaves) plus fresh noise
+        d = wl.tree_width
+        leaves = np.repeat(mix[:, np.minimum(np.arange(G) + 1, G - 1)], d - 1, axis=1)      # [B][G (d-1)][V]
+        g2 = substream(wl.config_id, "target_noise_leaves", rnd)
+        leaves = leaves + np.float32(wl.sigma(rnd)) * g2.standard_normal(leaves.shape, dtype=np.float32)
+        out = np.concatenate([out, leaves.astype(np.float32)], axis=1)
     return out
 
 

@@ -51,14 +51,14 @@ def t(a: np.ndarray, dtype=None) -> torch.Tensor:
 def make_oracle(wl: W.Workload, drafter: Optional[OracleDrafter]) -> TabedOracle:
     return TabedOracle(n_inputs=wl.n_inputs, n_requests=wl.n_requests, gamma=wl.gamma, window_h=wl.window_h,
                        policy=wl.policy, vocab=wl.drafter.vocab, distance=wl.distance, sample_mode=wl.sample_mode,
-                       tau=wl.tau, drafter=drafter, kv_capacity=wl.kv_capacity)
+                       tau=wl.tau, drafter=drafter, kv_capacity=wl.kv_capacity, tree_width=wl.tree_width)
 
 
 def make_gpu(wl: W.Workload, weights_dev=None) -> TB.Tabed:
     return TB.Tabed(n_inputs=wl.n_inputs, n_requests=wl.n_requests, gamma=wl.gamma, window_h=wl.window_h,
                     policy=wl.policy, vocab=wl.drafter.vocab, distance=wl.distance, sample_mode=wl.sample_mode,
                     tau=wl.tau, drafter=wl.drafter if weights_dev is not None else None, weights=weights_dev,
-                    kv_capacity=wl.kv_capacity)
+                    kv_capacity=wl.kv_capacity, tree_width=wl.tree_width)
 
 
 @dataclasses.dataclass
@@ -119,8 +119,10 @@ def assert_decisions_equal(p: Pair, toks_g, a_g, z_g, w_g, am_g, bit_exact_float
     """Compare one finished round of the CUDA handle with the checker's round."""
     o, g = p.orc, p.gpu
     torch.cuda.synchronize()
-    assert np.array_equal(toks_g.cpu().numpy(), o.tokens), "drafted tokens"
+    assert np.array_equal(toks_g.cpu().numpy().reshape(o.cands.shape), o.cands), "drafted tokens (all candidates)"
     assert np.array_equal(a_g.cpu().numpy(), o.n_accept), "accept counts"
+    assert np.array_equal(g.debug_view(TB.VIEW_ACC_PRIMARY).cpu().numpy(), o.acc_prim), "accepted tokens of the primary chain"
+    assert np.array_equal(g.debug_view(TB.VIEW_SIBLING).cpu().numpy(), o.sib_tok), "accepted sibling"
     assert np.array_equal(z_g.cpu().numpy(), o.next_token), "replacement / bonus token"
     assert np.array_equal(am_g.cpu().numpy(), np.argmax(o.w, axis=1)), "weight argmax"
     wg = w_g.cpu().numpy()
@@ -140,6 +142,18 @@ def assert_decisions_equal(p: Pair, toks_g, a_g, z_g, w_g, am_g, bit_exact_float
     check_error_flag(g)
 
 
+def assert_p_equal(p: Pair):
+    """Target distributions, bitwise: the chain's positions and, with a token tree, the one leaf that was used."""
+    o, g = p.orc, p.gpu
+    G, d = o.gamma, o.d
+    gp = g.debug_view(TB.VIEW_P).cpu().numpy()
+    assert np.array_equal(gp[:, :G + 1], o.p[:, :G + 1]), "target p (bitwise)"
+    for b in range(o.B):
+        if o.sib_tok[b] >= 0:
+            row = G + 1 + int(o.acc_prim[b]) * (d - 1) + (list(o.cands[b, o.acc_prim[b]]).index(int(o.sib_tok[b])) - 1)
+            assert np.array_equal(gp[b, row], o.p[b, row]), "target p at the accepted leaf (bitwise)"
+
+
 def logits_round(p: Pair, rnd: int, logits: np.ndarray, target: Optional[np.ndarray] = None):
     """One round on supplied drafter logits through tabed_draft_round_logits; everything bit-exact."""
     wl, o, g = p.wl, p.orc, p.gpu
@@ -151,7 +165,7 @@ def logits_round(p: Pair, rnd: int, logits: np.ndarray, target: Optional[np.ndar
     o_w, o_am = o.update_weights(up)
     if up is not None:
         g.set_policy_uniforms(t(up))
-    toks = torch.empty((wl.n_requests, wl.gamma), dtype=torch.int32, device=DEV)
+    toks = torch.empty((wl.n_requests, wl.gamma, wl.tree_width), dtype=torch.int32, device=DEV)
     out_q = torch.empty((wl.n_requests, wl.gamma, wl.drafter.vocab), dtype=torch.float32, device=DEV)
     a = torch.empty(wl.n_requests, dtype=torch.int32, device=DEV)
     z = torch.empty_like(a)
@@ -162,7 +176,7 @@ def logits_round(p: Pair, rnd: int, logits: np.ndarray, target: Optional[np.ndar
     torch.cuda.synchronize()
     assert np.array_equal(out_q.cpu().numpy(), o.q), "ensembled q (bitwise)"
     assert np.array_equal(g.debug_view(TB.VIEW_QK).cpu().numpy(), o.qk), "per-drafter q^(k) (bitwise)"
-    assert np.array_equal(g.debug_view(TB.VIEW_P).cpu().numpy(), o.p), "target p (bitwise)"
+    assert_p_equal(p)
     g.update_weights(w, am)
     assert_decisions_equal(p, toks, a, z, w, am, bit_exact_floats=True)
 
@@ -185,7 +199,7 @@ def lockstep_round(p: Pair, rnd: int, override: bool = True):
     o.update_weights(up)
     if up is not None:
         g.set_policy_uniforms(t(up))
-    toks = torch.empty((B, G), dtype=torch.int32, device=DEV)
+    toks = torch.empty((B, G, wl.tree_width), dtype=torch.int32, device=DEV)
     a = torch.empty(B, dtype=torch.int32, device=DEV)
     z = torch.empty_like(a)
     am = torch.empty_like(a)
@@ -206,12 +220,12 @@ def lockstep_round(p: Pair, rnd: int, override: bool = True):
     qk_own = torch.empty((B, m, V), dtype=torch.float32, device=DEV)
     y_tmp = torch.empty(B, dtype=torch.int32, device=DEV)
     for i in range(G):
-        g.ensemble_step(own[i].contiguous(), None, t(ud[:, i].copy()), y_tmp, None, qk_own)
+        g.ensemble_step(own[i].contiguous(), None, t(ud.reshape(B, G, -1)[:, i, 0].copy()), y_tmp, None, qk_own)
         err = np.max(np.abs(qk_own.cpu().numpy().astype(np.float64) - o.qk[:, i].astype(np.float64)))
         assert err <= PROB_TOL, f"probabilities step {i}: {err}"
     if override:
         assert np.array_equal(g.debug_view(TB.VIEW_QK).cpu().numpy(), o.qk)
-        assert np.array_equal(g.debug_view(TB.VIEW_P).cpu().numpy(), o.p)
+        assert_p_equal(p)
     g.update_weights(w, am)
     assert_decisions_equal(p, toks, a, z, w, am, bit_exact_floats=override)
     if override:

@@ -39,6 +39,14 @@ DECISION_CASES = {
     "llava_small_random": (W.LLAVA_SMALL, dict(policy=W.POLICY_RANDOM), 3),
     "llava_small_adaboost_all": (W.LLAVA_SMALL, dict(policy=W.POLICY_ADABOOST, window_h=0, tau=0.5), 4),
     "batched_serving_adaboost": (W.BATCHED_SERVING, dict(policy=W.POLICY_ADABOOST), 3),
+    "tiny_tree2": (W.TINY, dict(tree_width=2), 8),
+    "tiny_tree3_softmax": (W.TINY, dict(tree_width=3, policy=W.POLICY_SOFTMAX_INV_ERR), 8),
+    "tiny_tree3_greedy": (W.TINY, dict(tree_width=3, sample_mode=W.MODE_GREEDY), 6),
+    "tiny_tree2_grid_hard": (W.TINY, dict(tree_width=2, policy=W.POLICY_GRID_HARD), 6),
+    "llava_small_tree2": (W.LLAVA_SMALL, dict(tree_width=2), 5),
+    "llava_small_tree3": (W.LLAVA_SMALL, dict(tree_width=3), 5),
+    "batched_serving_tree2": (W.BATCHED_SERVING, dict(tree_width=2), 3),
+    "large_vocab_tree3_greedy": (W.LARGE_VOCAB, dict(tree_width=3, sample_mode=W.MODE_GREEDY), 2),
     "llava_small": (W.LLAVA_SMALL, {}, 4),
     "large_vocab": (W.LARGE_VOCAB, {}, 3),
     "long_context": (W.LONG_CONTEXT, {}, 3),
@@ -66,6 +74,44 @@ def test_decision_chain_ragged_vocabularies(V, m, B, G):
     pair = H.Pair(wl, H.make_gpu(wl), H.make_oracle(wl, None))
     for rnd in range(4):
         H.logits_round(pair, rnd, W.logits_like_drafter(wl, rnd, scale=1.5))
+    pair.gpu.destroy()
+
+
+@pytest.mark.parametrize("V,m,B,G,d", [(2, 2, 2, 3, 3), (97, 3, 2, 2, 2), (4099, 2, 3, 3, 3), (2049, 1, 1, 4, 4)])
+def test_token_tree_ragged_vocabularies(V, m, B, G, d):
+    """Token tree of width d on vocabularies that are not multiples of the vector width or of a CTA slice, including
+    V = 2 with three candidates (the third does not exist) and the widest tree."""
+    cfg = W.DrafterCfg(1, 64, 2, 2, 64, V, "fp32")
+    for mode in (W.MODE_SAMPLE, W.MODE_GREEDY):
+        wl = W.Workload(name=f"tree_ragged{V}", config_id=700 + V % 89 + mode, drafter=cfg, n_inputs=m, n_requests=B, gamma=G,
+                        window_h=3, rounds=5, policy=W.POLICY_GRID_MT if m == 2 else W.POLICY_SOFTMAX_INV_ERR,
+                        alpha=tuple([1.0 / m] * m), sigma_schedule=((0, 0.7),), tree_width=d, sample_mode=mode)
+        pair = H.Pair(wl, H.make_gpu(wl), H.make_oracle(wl, None))
+        sib = 0
+        for rnd in range(5):
+            H.logits_round(pair, rnd, W.logits_like_drafter(wl, rnd, scale=1.5))
+            sib += int((pair.orc.sib_tok >= 0).sum())
+        if V > 2 and mode == W.MODE_SAMPLE:
+            assert sib > 0                                   # some round ended on an accepted sibling
+        pair.gpu.destroy()
+
+
+def test_token_tree_lockstep_with_the_drafters_forward():
+    """Width-2 tree with the library's own forward pass: the fp32 drafter (per-operation kernels) and a bf16 drafter
+    with 18 rows (tensor-core path); the chain the drafter continues is the primary candidates, the caches keep only
+    what it consumed, an accepted sibling leaves two tokens pending."""
+    pair = H.build_pair(W.TINY.replace(tree_width=2, policy=W.POLICY_SOFTMAX_INV_ERR))
+    for rnd in range(8):
+        H.lockstep_round(pair, rnd, override=True)
+    pair.gpu.destroy()
+    wl = small_bf16_workload(B=6).replace(tree_width=3)
+    pair = H.build_pair(wl)
+    assert pair.gpu.current_path() == TB.PATH_TENSOR_CORE
+    sib = 0
+    for rnd in range(4):
+        H.lockstep_round(pair, rnd, override=True)
+        sib += int((pair.orc.sib_tok >= 0).sum())
+    assert sib > 0
     pair.gpu.destroy()
 
 
