@@ -124,7 +124,8 @@ def oracle_setup(wl):
     weights = W.make_weights(wl)
     orc = TabedOracle(n_inputs=wl.n_inputs, n_requests=wl.n_requests, gamma=wl.gamma, window_h=wl.window_h,
                       policy=wl.policy, vocab=wl.drafter.vocab, distance=wl.distance, sample_mode=wl.sample_mode,
-                      tau=wl.tau, drafter=OracleDrafter(wl.drafter, weights), kv_capacity=wl.kv_capacity)
+                      tau=wl.tau, drafter=OracleDrafter(wl.drafter, weights), kv_capacity=wl.kv_capacity,
+                      tree_width=wl.tree_width)
     if wl.synthetic_kv_len is not None:
         lens = W.synthetic_kv_lengths(wl)
         for row in range(wl.n_rows):
@@ -185,7 +186,8 @@ def time_oracle(wl, rounds, warmup=0, budget_s=None):
 def config_of(wl):
     """The `config` object both arms print (identical keys and values for one workload)."""
     return {"workload": wl.name, "n_inputs": wl.n_inputs, "n_requests": wl.n_requests, "rows": wl.n_rows, "gamma": wl.gamma,
-            "window_h": wl.window_h, "vocab": wl.drafter.vocab, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model}
+            "window_h": wl.window_h, "vocab": wl.drafter.vocab, "layers": wl.drafter.n_layers, "d_model": wl.drafter.d_model,
+            "tree_width": wl.tree_width}
 
 
 def run_reference(args, wl):
@@ -272,7 +274,8 @@ def gpu_setup(wl, device, prefill_path=None, prefill_times=None):
     weights = TB.weights_to_device(wl.drafter, W.make_weights(wl), device)
     g = TB.Tabed(n_inputs=wl.n_inputs, n_requests=wl.n_requests, gamma=wl.gamma, window_h=wl.window_h,
                  policy=wl.policy, vocab=wl.drafter.vocab, distance=wl.distance, sample_mode=wl.sample_mode,
-                 tau=wl.tau, drafter=wl.drafter, weights=weights, kv_capacity=wl.kv_capacity, device=device.index)
+                 tau=wl.tau, drafter=wl.drafter, weights=weights, kv_capacity=wl.kv_capacity, device=device.index,
+                 tree_width=wl.tree_width)
     tdt = torch.float32 if wl.drafter.dtype == "fp32" else torch.bfloat16
     dev = lambda a, dt=None: (torch.from_numpy(np.ascontiguousarray(a)).to(device) if dt is None
                               else torch.from_numpy(np.ascontiguousarray(a)).to(device).to(dt))
@@ -356,7 +359,7 @@ def measure(wl, device, K, Wm, *, rank=0, dist=None, path="auto", breakdown=Fals
 
     # uniforms for every round, resident on the device
     u = [tuple(torch.from_numpy(x).to(device) for x in W.round_uniforms(wl, r)) for r in range(total)]
-    toks = torch.empty((B, G), dtype=torch.int32, device=device)
+    toks = torch.empty((B, G, wl.tree_width), dtype=torch.int32, device=device)
     a = torch.empty(B, dtype=torch.int32, device=device)
     z = torch.empty_like(a)
     am = torch.empty_like(a)
@@ -365,9 +368,12 @@ def measure(wl, device, K, Wm, *, rank=0, dist=None, path="auto", breakdown=Fals
     def synth_target(rnd):
         lg = g.debug_view(TB.VIEW_LOGITS)                               # [G][B][m][V]
         mix = torch.einsum("gbnv,bn->bgv", lg, alpha)
-        tl = torch.empty((B, G + 1, V), dtype=torch.float32, device=device)
+        tl = torch.empty((B, wl.n_target_rows, V), dtype=torch.float32, device=device)
         tl[:, :G] = mix
         tl[:, G] = mix[:, G - 1]
+        if wl.tree_width > 1:               # leaves of the token tree: the mix of the next step (the last step's for the deepest)
+            nxt = torch.clamp(torch.arange(G, device=device) + 1, max=G - 1)
+            tl[:, G + 1:] = mix[:, nxt].repeat_interleave(wl.tree_width - 1, dim=1)
         tl += wl.sigma(rnd) * torch.randn(tl.shape, generator=gen, device=device)
         return tl
 
@@ -490,7 +496,7 @@ def measure(wl, device, K, Wm, *, rank=0, dist=None, path="auto", breakdown=Fals
         torch.cuda.synchronize(device)
         pin = lambda x: x.cpu().pin_memory()
         hu = [(pin(u[Wm + i][0]), pin(u[Wm + i][1]), pin(u[Wm + i][2]), pin(targets[Wm + i])) for i in range(ne)]
-        h_toks = torch.empty((B, G), dtype=torch.int32).pin_memory()
+        h_toks = torch.empty((B, G, wl.tree_width), dtype=torch.int32).pin_memory()
         h_a = torch.empty(B, dtype=torch.int32).pin_memory()
         h_z = torch.empty(B, dtype=torch.int32).pin_memory()
         h_am = torch.empty(B, dtype=torch.int32).pin_memory()
@@ -627,6 +633,7 @@ def main():
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--trace", default=None, help="write the persistent kernel's phase timeline of one round to this file")
     ap.add_argument("--trace-cta", type=int, default=0, help="the CTA whose phase timeline --trace records")
+    ap.add_argument("--tree-width", type=int, default=1, help="candidates per depth of the token tree (Sec. 5); 1 = a plain chain")
     ap.add_argument("--requests", type=int, default=0, help="override the workload's number of concurrent requests (profiling aid)")
     ap.add_argument("--prefill", action="store_true",
                     help="time the feeding of the workload's prompts instead of rounds: chunks of positions through the "
@@ -637,6 +644,8 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     wl = W.WORKLOADS[args.config]
+    if args.tree_width > 1:
+        wl = wl.replace(tree_width=args.tree_width)
     if args.requests > 0:
         wl = wl.replace(n_requests=args.requests, name=f"{wl.name}[B={args.requests}]")
     if args.impl == "reference":

@@ -112,7 +112,7 @@ extern "C" {
 #define TABED_VIEW_ACC_PRIMARY 11  /* int32  [B]           accepted tokens of the primary chain (after tabed_verify)   */
 #define TABED_VIEW_SIBLING     12  /* int32  [B]           token of the accepted sibling of a token tree, or -1        */
 #define TABED_VIEW_TRACE      10   /* uint64 [G][5L+8][8]  phase timeline of the persistent drafting kernel
-                                                           (tabed_debug_trace): one record per grid barrier */
+                                                           (tabed_debug_trace): one record per phase */
 
 /* How tabed_draft_round runs Algorithm 1 (tabed_select_path).  Results obey the same contract on
  * every path: identical integer decisions for identical logits; logits agree within the forward
@@ -267,9 +267,9 @@ int tabed_last_device_error(tabed_handle* h);
  * by itself.  Errors: BAD_STATE (mid-round), CUDA. */
 int tabed_sync_lengths(tabed_handle* h);
 
-/* Test aid for the failure path of the device-side waits: launches ONE CTA that takes the persistent
- * kernel's grid barrier with an arrival count nobody else completes, so that its bounded wait (about
- * 2^21 polls, a fraction of a second) runs out, records the failure and returns by itself - the GPU keeps
+/* Test aid for the failure path of the device-side waits: launches ONE CTA that waits, with the persistent
+ * kernel's own bounded poll, for a flagged word that nobody writes, so that the wait (about 2^21 polls, a
+ * fraction of a second) runs out, records the failure and returns by itself - the GPU keeps
  * answering.  Returns what tabed_last_device_error then reports (TABED_ERR_TIMEOUT).
  * Errors: UNSUPPORTED (handle without the persistent kernel), CUDA. */
 int tabed_debug_barrier_timeout(tabed_handle* h);
@@ -283,13 +283,12 @@ int tabed_current_path(const tabed_handle* h);
 
 /* Switch the phase timeline of the persistent kernel off (on = 0) or on (on = 1 + the index of the CTA
  * that records; CTA 0 if the grid is smaller): when on, that CTA stores one record of
- * 8 words per grid barrier into TABED_VIEW_TRACE (first index = drafting step): [0] the GPU's
- * nanosecond timer after the barrier; [1..6] SM clock cycles that that CTA spent since the previous
- * barrier resolving and staging activations, waiting for weight tiles, in the tensor-core products,
- * issuing weight copies, in epilogues (or, for the phases without weights, in all of the phase), and
- * in the barrier itself; [7] unused.  Barrier order within a step: per layer QKV, attention, O,
- * gate/up, down; then LM head, [2 more when tabed_debug_override_logits is set],
- * exp-sum, mix.
+ * 8 words per phase into TABED_VIEW_TRACE (first index = drafting step): [0] the GPU's
+ * nanosecond timer at the end of the phase; [1..5] SM clock cycles that that CTA spent in the phase
+ * waiting for and staging activations, waiting for weight tiles, in the tensor-core products,
+ * issuing weight copies and in epilogues, and in the rest (for the phases without weights: all of the
+ * phase); [6..7] unused.  Phase order within a step: per layer QKV, attention, O, gate/up, down; then
+ * LM head, [1 more when tabed_debug_override_logits is set], exp-sum, mix.
  * Errors: UNSUPPORTED (no persistent path). */
 int tabed_debug_trace(tabed_handle* h, int32_t on);
 

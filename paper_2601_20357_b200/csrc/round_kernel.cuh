@@ -28,7 +28,7 @@
 //   * loops are deliberately not unrolled except the few hot ones: every phase runs its code once,
 //     so unrolling buys nothing and only inflates the instruction footprint.
 //
-// Waits are bounded: a grid barrier or a copy that does not complete within the spin limit sets an
+// Waits are bounded: a flagged word or a copy that does not arrive within the spin limit sets an
 // error bit, the CTA drains its copies in flight and returns.
 #pragma once
 #include <cuda_bf16.h>
@@ -80,28 +80,25 @@ struct RoundArgs {
   const int* kv_len;                    // [R] committed lengths (constant during the round)
   const int* pending;                   // [B][3]
   __nv_bfloat16 *kc, *vc;               // [R][L][Hkv][cap][hd]
-  // activations exchanged through L2
-  float *xa, *x1;                       // [8][d] residual entering a layer / after its attention block
-  float* ssq;                           // [d/16][8] sums of squares of the last residual, per 16-row tile
-  float *qkv, *mid, *attn_out;          // [8][qkv_w], [8][F] (holds bf16 values here), [8][H*hd]
-  float *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2]
+  // activations exchanged through L2 as {value, epoch} pairs (one 8-byte store, polled by the consumer)
+  uint2 *xa, *x1;                       // [8][d] residual entering a layer / after its attention block
+  uint2* qkv;                           // [8][qkv_w]
+  uint2* mid;                           // [8][F/2] two bf16 values of the gated product per pair
+  uint2 *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2] (max, sum)
   int max_splits;
-  int* tickets;                         // [8][Hkv] partial attention results of a (slot, KV head) pair in the current layer
+  unsigned epoch0;                      // the launch's first epoch; phase p of step s stamps epoch0 + s * (5 L + 8) + p + 1
   // ensemble
   float* logits_own;                    // [G][R][V]
   const float* logits_override;         // or null
   const float* w;                       // [B][m]
   const float* u;                       // [B][G]
   float *qk, *q;                        // [B][G][m][V], [B][G][V]
-  uint32_t* rowmax;                     // [G][R]
-  unsigned long long* rowsum;           // [G][R]
-  unsigned long long* chunk_mass;       // [B][n_chunks]
-  ChunkBest* chunk_best;                // [B][n_chunks]
+  uint2 *rowmax, *rowmax2;              // [CTAs][8] every CTA's maxima of the logit rows (LM head; the logits of a replay)
+  uint2* rowsum;                        // [CTAs][8][2] every CTA's integer exp sums, low and high word
+  uint2* chunk_mass;                    // [B][n_chunks][2] mass of a chunk of q, low and high word (greedy: best value, its index)
   int n_chunks;
   int *tokens, *out_tokens;             // [B][G]
-  // synchronisation / diagnostics
-  unsigned* bar;                        // [2] grid barrier counters, used alternately by launches
-  int bar_sel;
+  // diagnostics
   int* err;
   unsigned long long* trace;            // optional [G][trace_stride][kTraceRec] phase timeline
   int trace_stride, trace_cta;          // the CTA that records
@@ -147,6 +144,21 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+// Flagged words: an aligned 8-byte {value, epoch} pair is written by ONE store and read by one load, so a
+// reader sees either the old pair or the new one; a 16-byte load returns two such pairs.
+__device__ __forceinline__ void ll_store(uint2* p, uint32_t value, uint32_t epoch) {
+  asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(value), "r"(epoch) : "memory");
+}
+__device__ __forceinline__ uint2 ll_load1(const uint2* p) {
+  uint2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 ll_load2(const uint2* p) {           // p 16-byte aligned: pairs p[0], p[1]
+  uint4 v;
+  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ unsigned long long global_timer() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -187,7 +199,10 @@ struct PShared {
   PSlot slot[kPSlots];
   int lm_src[kPSlots];
   int att[8];                           // attention geometry of the step: T, g_lo, g_hi, then this CTA's first chunk (s, gk, split, nsplit, g0)
+  int pair_base[kPSlots], pair_ns[kPSlots];   // per slot: chunks before its first pair, chunks per pair (0: inactive)
   int tok[kPSlots];
+  float rowmax_f[kPSlots];
+  unsigned long long row_part[kPSlots];
   int dead, flag, result, chunk;
   unsigned long long thr;
 };
@@ -252,42 +267,85 @@ __device__ __forceinline__ bool wait_full(PShared& S, int slot, unsigned parity,
   return true;
 }
 
-// Grid-wide barrier on a counter that only grows during a launch.  (One flag per CTA polled by all
-// CTAs in parallel was measured 3-4x slower: 148 x 148 concurrent polls saturate the L2 slice.)
-// Returns false if the wait ran out.
-// The barrier in two halves, for work that may overlap the wait (loads that do not depend on the
-// other CTAs are requested between the halves: a fence would wait for them).
-__device__ __forceinline__ void grid_barrier_arrive(unsigned* bar) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(bar, 1u);
+// Bounded polls of flagged words.  On a timeout the error bit is set and S.dead raised; the caller leaves
+// after its next block-wide barrier.
+__device__ __noinline__ void ll_timeout(PShared& S, int* err) {
+  atomicOr(err, PERR_BARRIER);
+  S.dead = 1;
+}
+__device__ __forceinline__ uint32_t ll_wait1(const uint2* p, uint32_t epoch, PShared& S, int* err) {
+  uint2 v = ll_load1(p);
+  unsigned spins = 0;
+  while (v.y != epoch) {
+    if (++spins > kSpinLimit) { ll_timeout(S, err); break; }
+    if (spins > 256) __nanosleep(spins > 4096 ? 64 : 20);
+    v = ll_load1(p);
+  }
+  return v.x;
+}
+// A long wait must not flood L2 with polls (75 000 threads would): after two rounds in which some lane of the warp
+// still misses a word, ONE lane keeps polling one missing word, with growing pauses, while the others idle; then the
+// whole warp looks again.  All 32 lanes call these helpers together (lanes without work pass n = 0 / null).
+__device__ __forceinline__ void ll_backoff_wait1(const uint2* p, uint32_t epoch, unsigned& spins, PShared& S, int* err) {
+  unsigned ns = 40;
+  while (ll_load1(p).y != epoch) {
+    if (++spins > kSpinLimit) { ll_timeout(S, err); break; }
+    __nanosleep(ns);
+    if (ns < 400) ns += 40;
   }
 }
-__device__ __noinline__ bool grid_barrier_wait(PShared& S, unsigned* bar, unsigned target, int* err) {
-  if (threadIdx.x == 0) {
-    unsigned spins = 0;
-    while ((int)(ld_acquire_u32(bar) - target) < 0) {
-      if (++spins > kSpinLimit) { atomicOr(err, PERR_BARRIER); S.dead = 1; break; }
-      if (spins > 4096) __nanosleep(64);
-    }
+// Several 16-byte loads in flight (the word pairs at addr(j), j < n); every round re-requests ALL the ones that do
+// not carry the epoch yet, together, so that a wait costs one more trip to L2 however many words were missing.
+template <int N, typename AddrFn>
+__device__ __forceinline__ void ll_poll(AddrFn addr, int n, uint32_t epoch, uint4 (&v)[N], PShared& S, int* err) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int j = 0; j < N; ++j) {
+    const uint2* pj = j < n ? addr(j) : nullptr;              // (a null address: nothing to wait for)
+    v[j] = pj ? ll_load2(pj) : make_uint4(0u, epoch, 0u, epoch);
   }
-  __syncthreads();
-  return S.dead == 0;
+  unsigned spins = 0, rounds = 0;
+  while (true) {
+    const uint2* pmiss = nullptr;                             // one word this lane still misses
+#pragma unroll
+    for (int j = 0; j < N; ++j)
+      if (j < n && !pmiss && (v[j].y != epoch || v[j].w != epoch)) pmiss = addr(j) + (v[j].y != epoch ? 0 : 1);
+    const unsigned who = __ballot_sync(0xffffffffu, pmiss != nullptr);
+    if (!who) break;
+    if (++spins > kSpinLimit) { ll_timeout(S, err); break; }
+    if (++rounds > 2) {
+      if (lane == __ffs(who) - 1) ll_backoff_wait1(pmiss, epoch, spins, S, err);
+      __syncwarp();
+      if (S.dead) break;
+    }
+#pragma unroll
+    for (int j = 0; j < N; ++j) if (j < n && (v[j].y != epoch || v[j].w != epoch)) v[j] = ll_load2(addr(j));
+  }
 }
-__device__ __noinline__ bool grid_barrier(PShared& S, unsigned* bar, unsigned target, int* err) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(bar, 1u);
-    unsigned spins = 0;
-    while ((int)(ld_acquire_u32(bar) - target) < 0) {
-      if (++spins > kSpinLimit) { atomicOr(err, PERR_BARRIER); S.dead = 1; break; }
-      if (spins > 4096) __nanosleep(64);
+__device__ __forceinline__ uint4 ll_wait2(const uint2* p, uint32_t epoch, PShared& S, int* err) {       // p null: lane without a word
+  uint4 v[1] = {make_uint4(0u, epoch, 0u, epoch)};
+  ll_poll<1>([&](int) { return p; }, p ? 1 : 0, epoch, v, S, err);
+  return v[0];
+}
+// two single words in flight (either may be null)
+__device__ __forceinline__ void ll_wait1x2(const uint2* p0, const uint2* p1, uint32_t epoch, uint32_t& x0, uint32_t& x1, PShared& S, int* err) {
+  const int lane = threadIdx.x & 31;
+  uint2 a = p0 ? ll_load1(p0) : make_uint2(0u, epoch), b = p1 ? ll_load1(p1) : make_uint2(0u, epoch);
+  unsigned spins = 0, rounds = 0;
+  while (true) {
+    const bool ra = a.y != epoch, rb = b.y != epoch;
+    const unsigned who = __ballot_sync(0xffffffffu, ra || rb);
+    if (!who) break;
+    if (++spins > kSpinLimit) { ll_timeout(S, err); break; }
+    if (++rounds > 2) {
+      if (lane == __ffs(who) - 1) ll_backoff_wait1(ra ? p0 : p1, epoch, spins, S, err);
+      __syncwarp();
+      if (S.dead) break;
     }
+    if (ra) a = ll_load1(p0);
+    if (rb) b = ll_load1(p1);
   }
-  __syncthreads();
-  return S.dead == 0;
+  x0 = a.x; x1 = b.x;
 }
 
 __device__ __forceinline__ unsigned long long block_sum_u64_p(unsigned long long v, PShared& S) {
@@ -336,9 +394,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(U);               // [areas][act_slots][apitch]
   float* cpart = reinterpret_cast<float*>(U + A.act_bytes);               // [2][kPW][128]
   float* s_o = reinterpret_cast<float*>(U);                               // attention: [kPW][grp*hd]
-  const int kvd = A.Hkv * A.hd, HD = A.H * A.hd, grp = A.H / A.Hkv, half = A.hd >> 1;
+  const int kvd = A.Hkv * A.hd, grp = A.H / A.Hkv, half = A.hd >> 1;
   const int R = A.R, B = A.B, m = A.m, G = A.G, V = A.V, d = A.d;
-  const int d4 = d >> 2, n_phase = 4 * A.L + 1;
+  const int n_phase = 4 * A.L + 1;
 
   // ---- set-up -----------------------------------------------------------------------------------
   if (tid == 0) {
@@ -351,13 +409,6 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll 1
   for (int i = tid; i < A.L * (int)(sizeof(LayerW) / sizeof(void*)); i += kPT)
     reinterpret_cast<const void**>(S.layers)[i] = reinterpret_cast<const void* const*>(A.layers)[i];
-  if (cta == 0) {
-#pragma unroll 1
-    for (int i = tid; i < G * R; i += kPT) { A.rowmax[i] = 0u; A.rowsum[i] = 0ull; }
-#pragma unroll 1
-    for (int i = tid; i < kPSlots * A.Hkv; i += kPT) A.tickets[i] = 0;
-    if (tid == 0) A.bar[A.bar_sel ^ 1] = 0u;          // the next launch's counter
-  }
   // unit list of one decoder step: tiles of phase p are dealt round-robin over the CTAs, starting
   // where phase p-1 stopped, so that every CTA streams about the same number of bytes
 #pragma unroll 1
@@ -404,9 +455,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll 1
     for (unsigned k = 0; k < (unsigned)A.n_ring && k < total_units; ++k) issue_unit(A, S, ring, k, per_step);
   }
-  unsigned* bar = A.bar + A.bar_sel;
-  unsigned bar_target = 0;
   bool alive = true;
+  const unsigned EPS = 5u * (unsigned)A.L + 8u;          // epochs per decoder step
   unsigned cons_done = 0;                                // units consumed so far (for the drain)
 
   // phase timeline (CTA 0, thread 0): per grid barrier one record of kTraceRec words:
@@ -424,28 +474,17 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       t_mark = t_now;                                 \
     }                                                 \
   } while (0)
-#define GRID_SYNC_TAIL()                                                   \
-  do {                                                                     \
-    TSEC(5);                                                               \
-    if (TRACE && tr_on && trace_n < A.trace_stride) {                      \
-      unsigned long long* rec = A.trace + ((size_t)step * A.trace_stride + trace_n++) * kTraceRec; \
-      rec[0] = global_timer();                                             \
-      for (int k = 0; k < 6; ++k) { rec[1 + k] = (unsigned long long)t_sec[k]; t_sec[k] = 0; }     \
-    }                                                                      \
-    if (!alive) goto drain;                                                \
-  } while (0)
-#define GRID_SYNC()                                                        \
+  // End of a phase: nothing is waited for here (the next phase polls the words it needs); the timeline gets
+  // its record, and a CTA that has seen a wait run out leaves.
+#define PHASE_END()                                                        \
   do {                                                                     \
     TSEC(4);                                                               \
-    bar_target += (unsigned)NC;                                            \
-    alive = grid_barrier(S, bar, bar_target, A.err);                       \
-    TSEC(5);                                                               \
     if (TRACE && tr_on && trace_n < A.trace_stride) {                      \
       unsigned long long* rec = A.trace + ((size_t)step * A.trace_stride + trace_n++) * kTraceRec; \
       rec[0] = global_timer();                                             \
       for (int k = 0; k < 6; ++k) { rec[1 + k] = (unsigned long long)t_sec[k]; t_sec[k] = 0; }     \
     }                                                                      \
-    if (!alive) goto drain;                                                \
+    if (__syncthreads_or(S.dead)) { alive = false; goto drain; }           \
   } while (0)
   if (tr_on) t_mark = clock64();
 
@@ -491,8 +530,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       const int sl = A.split_len;
       int T = 0;
 #pragma unroll 1
-      for (int s = 0; s < ns; ++s)
-        if (S.slot[s].active) T += A.Hkv * ((S.slot[s].pos + sl) / sl);
+      for (int s = 0; s < kPSlots; ++s) {
+        const int nsp = (s < ns && S.slot[s].active) ? (S.slot[s].pos + sl) / sl : 0;
+        S.pair_base[s] = T; S.pair_ns[s] = nsp;
+        T += A.Hkv * nsp;
+      }
       // (T <= 8 slots x 64 heads x 256 chunks, so c * T stays far below 2^31)
       const int lo = cta * T / NC, hi = (cta + 1) * T / NC;
       int s = 0, rem = lo, acc = 0, nsplit = 0;
@@ -521,119 +563,121 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       const bool norm_kind = kind == KIND_QKV || kind == KIND_GU || kind == KIND_LM;
       const unsigned ka = (unsigned)step * per_step + S.pstart[phase], kb = (unsigned)step * per_step + S.pstart[phase + 1];
 
-      if (kind == KIND_QKV && layer == 0) {
-        // the residual entering layer 0 is the embedding itself: publish this CTA's slice of it
-        const int lo = (int)((long long)cta * d / NC), hi = (int)((long long)(cta + 1) * d / NC), wsl = hi - lo;
-        if (tid < ns * wsl) {
-          const int s = tid / wsl, e = lo + (tid - s * wsl);
-          if (S.slot[s].active) A.xa[(size_t)s * d + e] = __bfloat162float(A.embed[(size_t)S.slot[s].tok * d + e]);
-        }
-      }
+      // epochs of the words this phase reads and writes
+      const unsigned ep_base = A.epoch0 + (unsigned)step * EPS;
+      const unsigned ep_prev_dn = ep_base + 5u * (unsigned)layer;                    // down projection of the layer before
+      const unsigned ep_qkv = ep_base + 5u * (unsigned)layer + 1u, ep_att = ep_qkv + 1u, ep_o = ep_qkv + 2u, ep_gu = ep_qkv + 3u,
+                     ep_dn = ep_qkv + 4u, ep_lm = ep_base + 5u * (unsigned)A.L + 1u;
       if (norm_kind && ka < kb) {
         // ---- stage RMSNorm(x) * gain as bf16, whole rows (these phases have kchunk == d) -----------
+        // Warp w serves input row w % n_in; a row's warps walk its 16-byte pieces (two flagged words = two
+        // elements) with every load in flight at once.  The sum of squares is taken per warp and the warps of a
+        // row are added in warp order: the same bits in every CTA and in every run.
         const bool from_embed = kind == KIND_QKV && layer == 0;
-        const float* xbuf = (kind == KIND_GU) ? A.x1 : A.xa;
+        const uint2* xbuf = (kind == KIND_GU) ? A.x1 : A.xa;
+        const unsigned ep_in = (kind == KIND_GU) ? ep_o : (kind == KIND_LM ? ep_base + 5u * (unsigned)A.L : ep_prev_dn);
         const __nv_bfloat16* gain = (kind == KIND_QKV) ? lw.n1 : (kind == KIND_GU ? lw.n2 : A.final_norm);
-        const int total = n_in * d4;
-#pragma unroll 1
-        for (int it0 = 0; it0 < total; it0 += 2 * kPT) {
-          float4 xv[2];
-          uint2 gv[2];
-          int ss[2];
+        const int s = warp % n_in, wi = warp / n_in, nw = (kPW - s + n_in - 1) / n_in;
+        const int src = (kind == KIND_LM) ? S.lm_src[s] : s;
+        const bool on = kind == KIND_LM || S.slot[s].active;
+        const int d2 = d >> 1;                                   // 16-byte pieces of a row
+        constexpr int kMaxPieces = 8;
+        float2 xv[kMaxPieces];
+        {
+          int n = 0;
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const int item = it0 + j * kPT + tid;
-            xv[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            gv[j] = make_uint2(0u, 0u);
-            ss[j] = -1;
-            if (item < total) {
-              const int s = item / d4, e4 = item - s * d4;
-              const int src = (kind == KIND_LM) ? S.lm_src[s] : s;
-              ss[j] = s * 65536 + e4;
-              gv[j] = __ldg(reinterpret_cast<const uint2*>(gain) + e4);
-              if (kind == KIND_LM || S.slot[s].active) {
-                if (from_embed) xv[j] = bf16x4_to_float4(__ldg(reinterpret_cast<const uint2*>(A.embed + (size_t)S.slot[s].tok * d) + e4));
-                else xv[j] = __ldcg(reinterpret_cast<const float4*>(xbuf + (size_t)src * d) + e4);
+          for (int k = 0; k < kMaxPieces; ++k) {
+            if (wi * 32 + lane + k * nw * 32 < d2) n = k + 1;
+            xv[k] = make_float2(0.0f, 0.0f);
+          }
+          const uint2* p0 = xbuf + (size_t)src * d + 2 * (wi * 32 + lane);
+          if (on) {
+            if (from_embed) {
+              const uint32_t* er = reinterpret_cast<const uint32_t*>(A.embed + (size_t)S.slot[s].tok * d);
+#pragma unroll
+              for (int k = 0; k < kMaxPieces; ++k) {
+                const int e2 = wi * 32 + lane + k * nw * 32;
+                if (e2 < d2) { const uint32_t w2 = __ldg(er + e2); xv[k] = make_float2(__uint_as_float(w2 << 16), __uint_as_float(w2 & 0xFFFF0000u)); }
+              }
+            } else {
+              // (four loads in flight at a time: rows of up to 4 x 64 x warps elements need one trip)
+              const int n_warp = __shfl_sync(0xffffffffu, n, 0);      // lane 0 has the most pieces
+#pragma unroll
+              for (int k0 = 0; k0 < kMaxPieces; k0 += 4) {
+                if (k0 >= n_warp) break;
+                uint4 raw[4];
+                const uint2* pk = p0 + (size_t)k0 * nw * 64;
+                ll_poll<4>([&](int j) { return pk + (size_t)j * nw * 64; }, n - k0, ep_in, raw, S, A.err);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) if (k0 + k < n) xv[k0 + k] = make_float2(__uint_as_float(raw[k].x), __uint_as_float(raw[k].z));
               }
             }
           }
-          if (it0 == 0) {
-            // statistics: warp w owns slot w
-            if (warp < kPSlots) {
-              float sq = 0.0f;
-              if (from_embed) {
-                if (warp < ns && S.slot[warp].active) {
-                  const uint2* er = reinterpret_cast<const uint2*>(A.embed + (size_t)S.slot[warp].tok * d);
-#pragma unroll 1
-                  for (int e4 = lane; e4 < d4; e4 += 32) {
-                    const float4 v = bf16x4_to_float4(__ldg(er + e4));
-                    sq = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, sq))));
-                  }
-                }
-              } else {
-#pragma unroll 1
-                for (int t = lane; t < (d >> 4); t += 32) sq += __ldcg(A.ssq + (size_t)t * kPSlots + warp);
-              }
-              sq = warp_sum_f32(sq);
-              if (lane == 0) S.scale[warp] = 1.0f / sqrtf(sq / (float)d + A.eps);
-            }
-            __syncthreads();
-          }
+        }
+        float sq = 0.0f;
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            if (ss[j] < 0) continue;
-            const int s = ss[j] >> 16, e4 = ss[j] & 65535;
-            const float sc = S.scale[(kind == KIND_LM) ? S.lm_src[s] : s];
-            const float4 gf = bf16x4_to_float4(gv[j]);
-            uint2 pk;
-            pk.x = pack_bf16(xv[j].x * sc * gf.x, xv[j].y * sc * gf.y);
-            pk.y = pack_bf16(xv[j].z * sc * gf.z, xv[j].w * sc * gf.w);
-            *reinterpret_cast<uint2*>(act + s * apitch + e4 * 4) = pk;
+        for (int k = 0; k < kMaxPieces; ++k) sq = fmaf(xv[k].x, xv[k].x, fmaf(xv[k].y, xv[k].y, sq));
+        sq = warp_sum_f32(sq);
+        if (lane == 0) S.red[warp][0] = sq;
+        __syncthreads();
+        float tot = 0.0f;
+#pragma unroll 1
+        for (int w2 = s; w2 < kPW; w2 += n_in) tot += S.red[w2][0];
+        const float sc = 1.0f / sqrtf(tot / (float)d + A.eps);
+#pragma unroll
+        for (int k = 0; k < kMaxPieces; ++k) {
+          const int e2 = wi * 32 + lane + k * nw * 32;
+          if (e2 < d2) {
+            const uint32_t g2 = __ldg(reinterpret_cast<const uint32_t*>(gain) + e2);
+            *reinterpret_cast<uint32_t*>(act + s * apitch + 2 * e2) =
+                pack_bf16(xv[k].x * sc * __uint_as_float(g2 << 16), xv[k].y * sc * __uint_as_float(g2 & 0xFFFF0000u));
           }
         }
         __syncthreads();
       } else if (kind == KIND_O && ka < kb) {
         // ---- stage the attention output, whole rows: put every pair's partial results together -----
-        // The first four partial results of a pair are requested together with their count (entries past the
-        // count are ignored), so the common case costs one round trip to L2.
+        // How many partial results a (slot, KV head) pair has follows from the step's chunk geometry (the same
+        // arithmetic as in the CTAs that produce them).
         const int nvec = g.kchunk >> 2;
-        const int spec = A.max_splits < 4 ? A.max_splits : 4;
+        const int T = S.att[0];
 #pragma unroll 1
-        for (int idx = tid; idx < n_in * nvec; idx += kPT) {
-          const int s = idx / nvec, j = (idx - s * nvec) << 2;
+        for (int idx0 = 0; idx0 < n_in * nvec; idx0 += kPT) {
+          const int idx = idx0 + tid;
+          const bool item = idx < n_in * nvec;
+          const int s = item ? idx / nvec : 0, j = item ? (idx - s * nvec) << 2 : 0;
           const int head = j / A.hd, dd = j - head * A.hd;
           const size_t base = ((size_t)s * A.H + head) * A.max_splits;
-          float2 ml[4];
-          float4 x[4];
-          const int n_seg = S.slot[s].active ? __ldcg(A.tickets + s * A.Hkv + head / grp) : 0;
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            ml[q] = q < spec ? __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + q) * 2)) : make_float2(-INFINITY, 0.0f);
-            x[q] = q < spec ? __ldcg(reinterpret_cast<const float4*>(A.part_o + (base + q) * A.hd + dd)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+          int n_seg = 0;
+          if (item && S.slot[s].active) {
+            const int nsp = S.pair_ns[s], g0 = S.pair_base[s] + (head / grp) * nsp;
+            n_seg = (T >= NC) ? ((g0 + nsp) * NC - 1) / T - ((g0 + 1) * NC - 1) / T + 1 : nsp;
           }
           float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
           float M = -INFINITY, den = 0.0f;
+          const int n_seg_warp = __reduce_max_sync(0xffffffffu, n_seg);
 #pragma unroll 1
-          for (int j0 = 0; j0 < n_seg; j0 += 4) {        // running maximum over the partial results in their fixed order
-            if (j0 > 0) {
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const bool ok = j0 + q < n_seg;
-                ml[q] = ok ? __ldcg(reinterpret_cast<const float2*>(A.part_ml + (base + j0 + q) * 2)) : make_float2(-INFINITY, 0.0f);
-                x[q] = ok ? __ldcg(reinterpret_cast<const float4*>(A.part_o + (base + j0 + q) * A.hd + dd)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-              }
-            }
+          for (int j0 = 0; j0 < n_seg_warp; j0 += 2) {   // running maximum over the partial results in their fixed order
+            uint4 raw[6];                                 // per partial result: (max, sum), output dims dd..dd+1, dd+2..dd+3
+            const int nq = max(0, min(2, n_seg - j0));
+            const uint2* pml = A.part_ml + (base + j0) * 2;
+            const uint2* po = A.part_o + (base + j0) * A.hd + dd;
+            const int hd_ = A.hd;
+            ll_poll<6>([&](int j) { const int q = j / 3, t = j - 3 * q; return t == 0 ? pml + 2 * q : po + (size_t)q * hd_ + 2 * (t - 1); },
+                       3 * nq, ep_att, raw, S, A.err);
+            uint4 rml[2] = {raw[0], raw[3]}, ro0[2] = {raw[1], raw[4]}, ro1[2] = {raw[2], raw[5]};
             float Mn = M;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) if (j0 + q < n_seg) Mn = fmaxf(Mn, ml[q].x);
+            for (int q = 0; q < 2; ++q) if (q < nq) Mn = fmaxf(Mn, __uint_as_float(rml[q].x));
             const float fo = (M > -INFINITY) ? expf(M - Mn) : 0.0f;
             v.x *= fo; v.y *= fo; v.z *= fo; v.w *= fo; den *= fo;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              if (j0 + q < n_seg && ml[q].x > -INFINITY) {
-                const float f = expf(ml[q].x - Mn);
-                v.x = fmaf(f, x[q].x, v.x); v.y = fmaf(f, x[q].y, v.y); v.z = fmaf(f, x[q].z, v.z); v.w = fmaf(f, x[q].w, v.w);
-                den = fmaf(f, ml[q].y, den);
+            for (int q = 0; q < 2; ++q) {
+              const float mq = __uint_as_float(rml[q].x);
+              if (q < nq && mq > -INFINITY) {
+                const float f = expf(mq - Mn);
+                v.x = fmaf(f, __uint_as_float(ro0[q].x), v.x); v.y = fmaf(f, __uint_as_float(ro0[q].z), v.y);
+                v.z = fmaf(f, __uint_as_float(ro1[q].x), v.z); v.w = fmaf(f, __uint_as_float(ro1[q].z), v.w);
+                den = fmaf(f, __uint_as_float(rml[q].z), den);
               }
             }
             M = Mn;
@@ -641,7 +685,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           if (n_seg > 0) { const float r = 1.0f / den; v.x *= r; v.y *= r; v.z *= r; v.w *= r; }
           uint2 pk;
           pk.x = pack_bf16(v.x, v.y); pk.y = pack_bf16(v.z, v.w);
-          *reinterpret_cast<uint2*>(act + s * apitch + j) = pk;
+          if (item) *reinterpret_cast<uint2*>(act + s * apitch + j) = pk;
         }
         __syncthreads();
       }
@@ -660,18 +704,32 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         if (kind == KIND_DN) {
           // stage this round's chunks of the gated product (left as bf16 by the gate/up epilogue): area of
           // group w <- columns of its sub-unit, 16 bytes at a time
-          const int nvec = g.kchunk >> 3;
-          const __nv_bfloat16* midb = reinterpret_cast<const __nv_bfloat16*>(A.mid);
+          // (a flagged word carries two bf16 values; a 16-byte load brings four of them; four loads in flight)
+          const int nvec = g.kchunk >> 2;
+          const int total = kWG * n_in * nvec;
 #pragma unroll 1
-          for (int idx = tid; idx < kWG * n_in * nvec; idx += kPT) {
-            const int w2 = idx / (n_in * nvec), r2 = idx - w2 * (n_in * nvec);
-            const int s = r2 / nvec, j = (r2 - s * nvec) << 3;
-            const unsigned kq = k0 + (unsigned)w2;
-            if (kq < kb) {
-              const int sq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10) % g.nsub;
-              const uint4 v = __ldcg(reinterpret_cast<const uint4*>(midb + (size_t)s * A.F + (size_t)sq * g.kchunk + j));
-              *reinterpret_cast<uint4*>(act + w2 * area_elems + s * apitch + j) = v;
+          for (int it0 = 0; it0 < total; it0 += 8 * kPT) {
+            const uint2* ptr[8];
+            uint4 raw[8];
+            int dst[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const int idx = it0 + q * kPT + tid;
+              ptr[q] = nullptr; dst[q] = -1;
+              if (idx < total) {
+                const int w2 = idx / (n_in * nvec), r2 = idx - w2 * (n_in * nvec);
+                const int s = r2 / nvec, j = (r2 - s * nvec) << 2;
+                const unsigned kq = k0 + (unsigned)w2;
+                if (kq < kb && S.slot[s].active) {
+                  const int sq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10) % g.nsub;
+                  ptr[q] = A.mid + (((size_t)s * A.F + (size_t)sq * g.kchunk + j) >> 1);
+                  dst[q] = w2 * area_elems + s * apitch + j;
+                }
+              }
             }
+            ll_poll<8>([&](int j) { return ptr[j]; }, 8, ep_gu, raw, S, A.err);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) if (dst[q] >= 0) *reinterpret_cast<uint2*>(act + dst[q]) = make_uint2(raw[q].x, raw[q].z);
           }
           __syncthreads();
           TSEC(0);
@@ -683,6 +741,21 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         }
         if (__syncthreads_or(!landed)) { alive = false; goto drain; }
         TSEC(1);
+        // the residual word this thread's epilogue adds to is requested now (it arrived phases ago) and is there when
+        // the products are done
+        const uint2* base_p = nullptr;
+        uint2 base_w = make_uint2(0u, 0u);
+        if ((kind == KIND_O && layer > 0) || kind == KIND_DN) {
+          const int q = tid >> 7, e = tid & 127, r = e & 15, n = e >> 4;
+          const unsigned kq = k0 + (unsigned)q;
+          if (kq < kb) {
+            const int uq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10), sq = uq % g.nsub;
+            if ((q % nsub_eff) == 0 && (sq + nsub_eff == g.nsub) && n < n_in && S.slot[n].active) {
+              base_p = (kind == KIND_O ? A.xa : A.x1) + (size_t)n * d + (uq / g.nsub) * 16 + r;
+              base_w = ll_load1(base_p);
+            }
+          }
+        }
         if (has) {
           if (sub < kWG) { c[0] = 0.0f; c[1] = 0.0f; c[2] = 0.0f; c[3] = 0.0f; }     // first round of a tile
           const unsigned char* tile_s = ring + (size_t)(k % (unsigned)A.n_ring) * A.slot_bytes;
@@ -708,10 +781,6 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         }
         __syncthreads();                        // slots fully read, partial tiles complete
         TSEC(2);
-        if (has && wl == 0 && lane == 0) {      // refill the slot this group has just released
-          const unsigned kn = k + (unsigned)A.n_ring;
-          if (kn < total_units) issue_unit(A, S, ring, kn, per_step);
-        }
         cons_done = (kb < k0 + kWG) ? kb : k0 + kWG;
         // epilogue: thread (group q, row r, slot n); the first group of a tile's set sums the set's warps
         {
@@ -724,9 +793,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           const int tile = uq / g.nsub;
           const bool slot_on = n < n_in && (kind == KIND_LM || S.slot[n].active);
           const int o = tile * 16 + r;
+          // the residual this tile adds to: its words arrived phases ago (layer 0: the embedding itself)
           float base = 0.0f;
-          if (lead && slot_on && (kind == KIND_O || kind == KIND_DN))
-            base = __ldcg((kind == KIND_O ? A.xa : A.x1) + (size_t)n * d + o);
+          if (lead && slot_on && (kind == KIND_O || kind == KIND_DN)) {
+            const unsigned ep_b = kind == KIND_O ? ep_prev_dn : ep_o;
+            if (kind == KIND_O && layer == 0) base = __bfloat162float(A.embed[(size_t)S.slot[n].tok * d + o]);
+            else base = __uint_as_float(base_w.y == ep_b ? base_w.x : ll_wait1(base_p, ep_b, S, A.err));
+          }
           float v = 0.0f;
           if (lead) {
             const int w_hi = (q + nsub_eff) * kGW;
@@ -735,37 +808,44 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           if (kind == KIND_GU) {
             const float up = __shfl_down_sync(0xffffffffu, v, 8);
-            if (lead && r < 8 && slot_on)            // bf16: the down projection rounds its input to bf16 anyway
-              reinterpret_cast<__nv_bfloat16*>(A.mid)[(size_t)n * A.F + tile * 8 + r] = __float2bfloat16_rn(v / (1.0f + expf(-v)) * up);
+            // bf16: the down projection rounds its input to bf16 anyway; two neighbours share a flagged word
+            const float gated = v / (1.0f + expf(-v)) * up;
+            const float right = __shfl_down_sync(0xffffffffu, gated, 1);
+            if (lead && r < 8 && (r & 1) == 0 && slot_on)
+              ll_store(A.mid + (((size_t)n * A.F + tile * 8 + r) >> 1), pack_bf16(gated, right), ep_gu);
           } else if (kind == KIND_LM) {
             if (lead && slot_on && o < V) {
               A.logits_own[((size_t)step * R + n) * V + o] = v;
               lm_max = fmaxf(lm_max, v);
             }
           } else if (kind == KIND_QKV) {
-            if (lead && slot_on) A.qkv[(size_t)n * A.qkv_w + o] = v;
+            if (lead && slot_on) ll_store(A.qkv + (size_t)n * A.qkv_w + o, __float_as_uint(v), ep_qkv);
           } else {
-            // residual add + this tile's share of the next RMSNorm's sum of squares
-            const float xn = base + v;
-            float sq2 = (lead && slot_on) ? xn * xn : 0.0f;
-#pragma unroll
-            for (int o2 = 8; o2 > 0; o2 >>= 1) sq2 += __shfl_xor_sync(0xffffffffu, sq2, o2);
-            if (lead && slot_on) {
-              (kind == KIND_O ? A.x1 : A.xa)[(size_t)n * d + o] = xn;
-              if (r == 0) A.ssq[(size_t)tile * kPSlots + n] = sq2;
-            }
+            // residual add
+            if (lead && slot_on)
+              ll_store((kind == KIND_O ? A.x1 : A.xa) + (size_t)n * d + o, __float_as_uint(base + v), kind == KIND_O ? ep_o : ep_dn);
           }
+        }
+        // refill the slot this group has just released: after the results are on their way (the copy's issue is not
+        // free), by the group's last warp, whose lanes serve the highest slot numbers and are mostly idle above
+        if (has && wl == kGW - 1 && lane == 0) {
+          const unsigned kn = k + (unsigned)A.n_ring;
+          if (kn < total_units) issue_unit(A, S, ring, kn, per_step);
         }
         TSEC(3);
       }
       if (kind == KIND_LM) {
-        // running maxima of the logits: 16 lanes of a slot, then the CTA, then one atomic per row
+        // running maxima of the logits: 16 lanes of a slot, then the CTA; every CTA publishes its maxima (0: it
+        // stored no logit of the row) behind a fence, so whoever has them all may also read the logits
 #pragma unroll
         for (int o2 = 8; o2 > 0; o2 >>= 1) lm_max = fmaxf(lm_max, __shfl_xor_sync(0xffffffffu, lm_max, o2));
         const int n = (tid & 127) >> 4;
         if ((tid & 15) == 0 && n < R && lm_max > -INFINITY) atomicMax(&S.lmmax[n], ord_encode(lm_max));
         __syncthreads();
-        if (tid < R && S.lmmax[tid] != 0u) atomicMax(A.rowmax + step * R + tid, S.lmmax[tid]);
+        if (tid < R) {
+          __threadfence();
+          ll_store(A.rowmax + (size_t)cta * kPSlots + tid, S.lmmax[tid], ep_lm);
+        }
       }
       // ---- attention over the rows' caches (after the QKV phase) -----------------------------------
       // The caches of all (slot, KV head) pairs are cut into chunks of split_len positions; the chunks, in
@@ -833,17 +913,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       uint4 kreg[4], vreg[4];
       Walk cur{0, 0, 0, 0, 0}, nxt{0, 0, 0, 0, 0};
       int T = 0, g_lo = 0, g_hi = 0;
+      PHASE_END();                                  // (its block-wide barrier also orders the geometry written at step start)
       if (kind == KIND_QKV) {
-        TSEC(4);
-        bar_target += (unsigned)NC;
-        grid_barrier_arrive(bar);                 // (its block-wide barrier also orders the geometry written at step start)
         T = S.att[0]; g_lo = S.att[1]; g_hi = S.att[2];
         cur.s = S.att[3]; cur.gk = S.att[4]; cur.split = S.att[5]; cur.nsplit = S.att[6]; cur.g0 = S.att[7];
+        // the cached positions do not depend on this step's projections: their loads are in flight while the q, k, v
+        // words are waited for
         if (g_lo < g_hi) issue_loads(cur, kreg, vreg, true, true);
-        alive = grid_barrier_wait(S, bar, bar_target, A.err);
-        GRID_SYNC_TAIL();
-      } else {
-        GRID_SYNC();
       }
 
       if (kind == KIND_QKV) {
@@ -867,11 +943,15 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             // that every element is fetched by a different thread in one round trip.
             const int n_q = grp * half, n_k = n_fresh * half, n_v = n_fresh * A.hd;
 #pragma unroll 1
-            for (int idx = tid; idx < n_q + n_k + n_v; idx += kPT) {
-              int sj, col, pj, i;
-              float* dst;
+            for (int idx0 = 0; idx0 < n_q + n_k + n_v; idx0 += kPT) {
+              const int idx = idx0 + tid;
+              const bool item = idx < n_q + n_k + n_v;
+              int sj = s, col = 0, pj = pos, i = 0;
+              float* dst = &S.q[0][0];
               bool pair = true;
-              if (idx < n_q) {
+              if (!item) {
+                pair = false;
+              } else if (idx < n_q) {
                 const int t = idx / half; i = idx - t * half;
                 sj = s; pj = pos; col = (gk * grp + t) * A.hd + i; dst = &S.q[t][i];
               } else if (idx < n_q + n_k) {
@@ -881,11 +961,14 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
                 const int j = (idx - n_q - n_k) / A.hd; i = (idx - n_q - n_k) - j * A.hd;
                 sj = s - j * R; pj = pos; col = d + kvd + gk * A.hd + i; dst = &S.vf[j][i]; pair = false;
               }
-              const float* pr = A.qkv + (size_t)sj * A.qkv_w + col;
+              const uint2* pr = A.qkv + (size_t)sj * A.qkv_w + col;
               float cs = 1.0f, sn = 0.0f, x2 = 0.0f;
-              if (pair) { cs = A.rope_cos[(size_t)pj * half + i]; sn = A.rope_sin[(size_t)pj * half + i]; x2 = __ldcg(pr + half); }
-              const float x1 = __ldcg(pr);
-              dst[0] = round_bf16(x1 * cs - x2 * sn);
+              if (pair) { cs = A.rope_cos[(size_t)pj * half + i]; sn = A.rope_sin[(size_t)pj * half + i]; }
+              uint32_t w1, w2;
+              ll_wait1x2(item ? pr : nullptr, pair ? pr + half : nullptr, ep_qkv, w1, w2, S, A.err);          // both in flight
+              const float x1 = __uint_as_float(w1);
+              if (pair) x2 = __uint_as_float(w2);
+              if (item) dst[0] = round_bf16(x1 * cs - x2 * sn);
               if (pair) dst[half] = round_bf16(x2 * cs + x1 * sn);
             }
             __syncthreads();
@@ -894,6 +977,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               const size_t off = ((((size_t)S.slot[s].row * A.L + layer) * A.Hkv + gk) * A.cap) * A.hd;
               A.kc[off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.kf[0][tid]);
               A.vc[off + (size_t)pos * A.hd + tid] = __float2bfloat16_rn(S.vf[0][tid]);
+              __threadfence();        // read from the cache one step later, by CTAs that have seen this CTA's partial results
             }
           }
           if (mma_path) {
@@ -1061,9 +1145,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             // Its place among the pair's partial results: with at least as many chunks as CTAs every CTA owns
             // chunks, so the segments of a pair sit on consecutive CTAs; with fewer, a segment is one chunk.
             const int c_first = ((cur.g0 + 1) * NC - 1) / T;
-            const int ord = (T >= NC) ? cta - c_first : split;
-            if (ord == 0 && tid == 0)                  // how many partial results the pair has (read by the O-projection phase)
-              A.tickets[s * A.Hkv + gk] = (T >= NC) ? ((cur.g0 + nsplit) * NC - 1) / T - c_first + 1 : nsplit;
+            const int ord = (T >= NC) ? cta - c_first : split;       // (the O-projection phase works out the count itself)
 #pragma unroll 1
             for (int idx = tid; idx < grp * A.hd; idx += kPT) {
               const int t = idx / A.hd, dd = idx - t * A.hd;
@@ -1085,8 +1167,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
               }
               const int head = gk * grp + t;
               const size_t pi = ((size_t)s * A.H + head) * A.max_splits + ord;
-              A.part_o[pi * A.hd + dd] = v;
-              if (dd == 0) { A.part_ml[pi * 2] = M; A.part_ml[pi * 2 + 1] = l; }
+              ll_store(A.part_o + pi * A.hd + dd, __float_as_uint(v), ep_att);
+              if (dd == 0) { ll_store(A.part_ml + pi * 2, __float_as_uint(M), ep_att); ll_store(A.part_ml + pi * 2 + 1, __float_as_uint(l), ep_att); }
             }
             TSEC(2);
             __syncthreads();
@@ -1094,20 +1176,24 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           cur = nxt;
         }
-        GRID_SYNC();
+        PHASE_END();
       }
     }  // phases
 
     // ---- ensemble: exact softmax of the m rows, weighted average, draw (Algorithm 1 steps 6-7) -----
+    // Three exchanges, each a table of flagged words that every CTA polls whole: every CTA's maxima of the rows
+    // (published by the LM head), every CTA's integer exp sums, the mass of every chunk of q.
     {
       const float* lg = A.logits_override ? A.logits_override + (size_t)step * R * V : A.logits_own + (size_t)step * R * V;
-      uint32_t* rowmax = A.rowmax + step * R;
-      unsigned long long* rowsum = A.rowsum + step * R;
       const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(lg) & 15) == 0);
       const int n_chunks = A.n_chunks;
+      const unsigned ep_base = A.epoch0 + (unsigned)step * EPS;
+      const unsigned ep_lm = ep_base + 5u * (unsigned)A.L + 1u, ep_max2 = ep_lm + 1u, ep_sum = ep_lm + 2u, ep_mix = ep_lm + 3u;
+      const uint2* max_tab = A.rowmax;
+      unsigned ep_max = ep_lm;
       if (A.logits_override) {                        // the maxima gathered by the LM head belong to other logits
-        if (cta == 0 && tid < R) rowmax[tid] = 0u;
-        GRID_SYNC();
+        if (tid < kPSlots) S.lmmax[tid] = 0u;
+        __syncthreads();
 #pragma unroll 1
         for (int item = cta; item < R * n_chunks; item += NC) {
           const int row = item / n_chunks, ch = item - row * n_chunks;
@@ -1115,24 +1201,58 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           load4_cg(lg + (size_t)row * V, ch * kChunk + tid * kPPer, V, vec, -INFINITY, a);
           float mx = fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
           mx = warp_max_f32(mx);
-          if (lane == 0 && mx > -INFINITY) atomicMax(rowmax + row, ord_encode(mx));
+          if (lane == 0 && mx > -INFINITY) atomicMax(&S.lmmax[row], ord_encode(mx));
         }
-        GRID_SYNC();
+        __syncthreads();
+        if (tid < R) ll_store(A.rowmax2 + (size_t)cta * kPSlots + tid, S.lmmax[tid], ep_max2);
+        max_tab = A.rowmax2; ep_max = ep_max2;
+        PHASE_END();
       }
+      // every CTA's maxima -> the rows' maxima (a maximum does not care about order)
+      if (tid < kPSlots) { S.lmmax[tid] = 0u; S.row_part[tid] = 0ull; }
+      __syncthreads();
+#pragma unroll 1
+      for (int i0 = 0; i0 < NC * R; i0 += kPT) {
+        const int i = i0 + tid, c2 = i / R, row = i - c2 * R;
+        uint32_t e, unused;
+        ll_wait1x2(i < NC * R ? max_tab + (size_t)c2 * kPSlots + row : nullptr, nullptr, ep_max, e, unused, S, A.err);
+        if (i < NC * R && e) atomicMax(&S.lmmax[row], e);
+      }
+      __threadfence();                                // the logits behind the flagged words
+      __syncthreads();
+      if (tid < R) S.rowmax_f[tid] = ord_decode(S.lmmax[tid]);
+      __syncthreads();
 #pragma unroll 1
       for (int item = cta; item < R * n_chunks; item += NC) {
         const int row = item / n_chunks, ch = item - row * n_chunks;
         const int v0 = ch * kChunk + tid * kPPer;
         float a[kPPer];
         load4_cg(lg + (size_t)row * V, v0, V, vec, -INFINITY, a);
-        const float mx = ord_decode(__ldcg(rowmax + row));
+        const float mx = S.rowmax_f[row];
         unsigned long long sm = 0;
 #pragma unroll
         for (int j = 0; j < kPPer; ++j) if (v0 + j < V) sm += mass_of(xexp(__fsub_rn(a[j], mx)));
         sm = block_sum_u64_p(sm, S);
-        if (tid == 0 && sm) atomicAdd(rowsum + row, sm);
+        if (tid == 0) S.row_part[row] += sm;
       }
-      GRID_SYNC();
+      __syncthreads();
+      if (tid < R) {
+        const unsigned long long t = S.row_part[tid];
+        uint2* dst = A.rowsum + ((size_t)cta * kPSlots + tid) * 2;
+        ll_store(dst, (uint32_t)t, ep_sum); ll_store(dst + 1, (uint32_t)(t >> 32), ep_sum);
+      }
+      PHASE_END();
+      // every CTA's sums -> the rows' normalisers (integer sums: order-free)
+      if (tid < kPSlots) S.row_part[tid] = 0ull;
+      __syncthreads();
+#pragma unroll 1
+      for (int i0 = 0; i0 < NC * R; i0 += kPT) {
+        const int i = i0 + tid, c2 = i / R, row = i - c2 * R;
+        const uint4 w4 = ll_wait2(i < NC * R ? A.rowsum + ((size_t)c2 * kPSlots + row) * 2 : nullptr, ep_sum, S, A.err);
+        const unsigned long long t = (unsigned long long)w4.x | ((unsigned long long)w4.z << 32);
+        if (i < NC * R && t) atomicAdd(&S.row_part[row], t);
+      }
+      __syncthreads();
 #pragma unroll 1
       for (int item = cta; item < B * n_chunks; item += NC) {
         const int b = item / n_chunks, ch = item - b * n_chunks;
@@ -1142,8 +1262,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         __syncthreads();
         if (tid < m) {
           const int row = b * m + tid;
-          S.mix_mx[tid] = ord_decode(__ldcg(rowmax + row));
-          S.mix_sn[tid] = norm_of(__ldcg(rowsum + row));
+          S.mix_mx[tid] = S.rowmax_f[row];
+          S.mix_sn[tid] = norm_of(S.row_part[row]);
           S.mix_w[tid] = A.w[row];
         }
         float nxt[kPPer];
@@ -1165,12 +1285,16 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           store4(qk_b + (size_t)k * V, v0, V, (V & 3) == 0, a);
         }
         store4(A.q + ((size_t)b * G + step) * V, v0, V, (V & 3) == 0, acc);
+        uint2* cm_dst = A.chunk_mass + ((size_t)b * n_chunks + ch) * 2;
         if (!A.greedy) {
           unsigned long long sm = 0;
 #pragma unroll
           for (int j = 0; j < kPPer; ++j) if (v0 + j < V) sm += mass_of(acc[j]);
-          sm = block_sum_u64_p(sm, S);
-          if (tid == 0) A.chunk_mass[(size_t)b * n_chunks + ch] = sm;
+          sm = block_sum_u64_p(sm, S);                  // (its barriers: every thread's part of q is stored)
+          if (tid == 0) {
+            __threadfence();                            // q before the word that announces it
+            ll_store(cm_dst, (uint32_t)sm, ep_mix); ll_store(cm_dst + 1, (uint32_t)(sm >> 32), ep_mix);
+          }
         } else {
           float bv = -1.0f; int bi = 0x7fffffff;
 #pragma unroll
@@ -1188,22 +1312,24 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll 1
             for (int i = 1; i < kPW; ++i)
               if (S.bestv[i] > bv || (S.bestv[i] == bv && S.besti[i] < bi)) { bv = S.bestv[i]; bi = S.besti[i]; }
-            A.chunk_best[(size_t)b * n_chunks + ch] = ChunkBest{bv, bi};
+            __threadfence();
+            ll_store(cm_dst, __float_as_uint(bv), ep_mix); ll_store(cm_dst + 1, (uint32_t)bi, ep_mix);
           }
         }
       }
-      GRID_SYNC();
+      PHASE_END();
       // every CTA locates the drawn token itself (the next step's embedding gather needs it)
 #pragma unroll 1
       for (int b = 0; b < B; ++b) {
         if (A.greedy) {
           float bv = -1.0f; int bi = 0x7fffffff;
 #pragma unroll 1
-          for (int c2 = tid; c2 < n_chunks; c2 += kPT) {
-            ChunkBest cb;
-            *reinterpret_cast<unsigned long long*>(&cb) =
-                __ldcg(reinterpret_cast<const unsigned long long*>(A.chunk_best + (size_t)b * n_chunks + c2));
-            if (cb.val > bv || (cb.val == bv && cb.idx < bi)) { bv = cb.val; bi = cb.idx; }
+          for (int c0 = 0; c0 < n_chunks; c0 += kPT) {
+            const int c2 = c0 + tid;
+            const uint4 w4 = ll_wait2(c2 < n_chunks ? A.chunk_mass + ((size_t)b * n_chunks + c2) * 2 : nullptr, ep_mix, S, A.err);
+            const float cv = __uint_as_float(w4.x);
+            const int ci = (int)w4.z;
+            if (c2 < n_chunks && (cv > bv || (cv == bv && ci < bi))) { bv = cv; bi = ci; }
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
@@ -1223,15 +1349,20 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           __syncthreads();
           continue;
         }
-        const unsigned long long* cm = A.chunk_mass + (size_t)b * n_chunks;
+        const uint2* cm = A.chunk_mass + (size_t)b * n_chunks * 2;
         // chunk masses in parallel into shared memory, then one thread walks them
         unsigned long long T = 0;
 #pragma unroll 1
         for (int c0 = 0; c0 < n_chunks; c0 += kPT) {
-          const unsigned long long mine = (c0 + tid < n_chunks) ? __ldcg(cm + c0 + tid) : 0ull;
+          unsigned long long mine = 0ull;
+          {
+            const uint4 w4 = ll_wait2(c0 + tid < n_chunks ? cm + (size_t)(c0 + tid) * 2 : nullptr, ep_mix, S, A.err);
+            if (c0 + tid < n_chunks) mine = (unsigned long long)w4.x | ((unsigned long long)w4.z << 32);
+          }
           if (n_chunks <= kPT && tid < n_chunks) S.cm[tid] = mine;       // one trip to L2 serves the sum and the walk
           T += block_sum_u64_p(mine, S);
         }
+        __threadfence();                              // q behind the words that announce it
         __syncthreads();
         if (tid == 0) {
           S.result = 0x7fffffff;
@@ -1242,7 +1373,10 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
             unsigned long long pre = 0;
 #pragma unroll 1
             for (; c2 < n_chunks - 1; ++c2) {
-              const unsigned long long nx = pre + (n_chunks <= kPT ? S.cm[c2] : __ldcg(cm + c2));
+              unsigned long long mc;
+              if (n_chunks <= kPT) mc = S.cm[c2];
+              else { const uint4 w4 = ll_load2(cm + (size_t)c2 * 2); mc = (unsigned long long)w4.x | ((unsigned long long)w4.z << 32); }   // (seen valid above)
+              const unsigned long long nx = pre + mc;
               if (nx > thr) break;
               pre = nx;
             }
@@ -1295,7 +1429,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       __syncthreads();
     }
   }  // steps
-#undef GRID_SYNC
+#undef PHASE_END
 #undef TSEC
   return;
 

@@ -89,13 +89,16 @@ struct tabed_handle {
   int n_cta = 0; size_t persist_smem = 0;
   unsigned launches_persist = 0;
   LayerW* layer_tab = nullptr;
-  float *xa = nullptr, *x1 = nullptr;
-  int* tickets = nullptr; unsigned* bar = nullptr; float* ssq = nullptr;
+  // its exchange buffers of flagged words {value, epoch} and the epoch the next launch starts from
+  uint2 *ll_xa = nullptr, *ll_x1 = nullptr, *ll_qkv = nullptr, *ll_mid = nullptr, *ll_po = nullptr, *ll_pml = nullptr;
+  uint2 *ll_rowmax = nullptr, *ll_rowmax2 = nullptr, *ll_rowsum = nullptr, *ll_cmass = nullptr;
+  std::vector<std::pair<void*, size_t>> ll_all;       // every exchange buffer (cleared when the epoch counter wraps)
+  unsigned ll_epoch = 0;
+  uint2* ll_probe = nullptr;        // a word nobody ever writes (tabed_debug_barrier_timeout)
   // tensor-core streaming attention of the per-operation paths (bf16 caches, head size 64)
   int* attn_tickets = nullptr; int n_sm = 0;
   bool atc_ok = false; CUtensorMap tm_k, tm_v;
   unsigned char* packed = nullptr;
-  uint32_t* rowmax_g = nullptr; unsigned long long* rowsum_g = nullptr;
   unsigned long long* trace = nullptr; int trace_stride = 0; bool trace_on = false; int trace_cta = 0;
   // tensor-core projections for many rows (bf16 drafter, more than 8 slots per step)
   bool tc_ok = false;                        // tcgen05 projections are set up (prefill in chunks; drafting when tc_auto)
@@ -429,6 +432,11 @@ int setup_persistent(tabed_handle* h) {
     per_step += (long)((A.geom[k].n_tiles + n_cta - 1) / n_cta) * A.geom[k].nsub * (k == KIND_LM ? 1 : h->L);
   }
   if (per_step > kMaxUnits) return TABED_OK;
+  {
+    // the staging of a whole input row: its warps keep at most 8 pieces of 16 bytes per lane in flight
+    const int act_slots = std::min(kPSlots, 2 * h->R), warps_per_row = kPW / act_slots;
+    if ((h->d / 2 + warps_per_row * 32 - 1) / (warps_per_row * 32) > 8) return TABED_OK;
+  }
   A.slot_bytes = 16 * (kmax * 2 + 16);
   A.act_slots = std::min(kPSlots, 2 * h->R);
   const int dn_areas = std::min(A.geom[KIND_DN].nsub, kWG);
@@ -452,8 +460,16 @@ int setup_persistent(tabed_handle* h) {
   int rc = TABED_OK;
   auto A2 = [&](auto** ptr, size_t count) { if (rc == TABED_OK) rc = dev_alloc(h, ptr, count); };
   const size_t d = h->d;
-  A2(&h->layer_tab, (size_t)h->L); A2(&h->xa, kPSlots * d); A2(&h->x1, kPSlots * d);
-  A2(&h->tickets, (size_t)kPSlots * h->Hkv); A2(&h->bar, 2); A2(&h->ssq, (size_t)(h->d / 16) * kPSlots);
+  A2(&h->layer_tab, (size_t)h->L);
+  auto LL = [&](uint2** ptr, size_t count) {
+    if (rc == TABED_OK) rc = dev_alloc(h, ptr, count);           // zeroed: no launch ever stamps epoch 0
+    if (rc == TABED_OK) h->ll_all.push_back({*ptr, std::max<size_t>(count, 1) * sizeof(uint2)});
+  };
+  LL(&h->ll_xa, kPSlots * d); LL(&h->ll_x1, kPSlots * d); LL(&h->ll_qkv, (size_t)kPSlots * h->qkv_w);
+  LL(&h->ll_mid, (size_t)kPSlots * h->F / 2);
+  LL(&h->ll_po, (size_t)kPSlots * h->H * h->max_splits * h->hd); LL(&h->ll_pml, (size_t)kPSlots * h->H * h->max_splits * 2);
+  LL(&h->ll_rowmax, (size_t)n_cta * kPSlots); LL(&h->ll_rowmax2, (size_t)n_cta * kPSlots); LL(&h->ll_rowsum, (size_t)n_cta * kPSlots * 2);
+  LL(&h->ll_cmass, (size_t)h->B * h->n_chunks * 2); LL(&h->ll_probe, 2);
   // private copy of the weights, unit by unit (one contiguous block per bulk copy)
   size_t unit_bytes[5], kind_bytes[5];
   for (int k = 0; k < 5; ++k) {
@@ -472,7 +488,6 @@ int setup_persistent(tabed_handle* h) {
     h->allocs.push_back(ptr);
     h->packed = reinterpret_cast<unsigned char*>(ptr);
   }
-  A2(&h->rowmax_g, (size_t)h->G * h->R); A2(&h->rowsum_g, (size_t)h->G * h->R);
   h->trace_stride = 5 * h->L + 8;
   A2(&h->trace, (size_t)h->G * h->trace_stride * kTraceRec);
   if (rc != TABED_OK) return rc;
@@ -505,11 +520,11 @@ int setup_persistent(tabed_handle* h) {
   A.eps = c.rms_eps; A.attn_scale = 1.0f / sqrtf((float)h->hd);
   A.R = h->R; A.B = h->B; A.m = h->m; A.G = h->G; A.greedy = c.sample_mode == TABED_MODE_GREEDY;
   A.kv_len = h->kv_len; A.pending = h->pending; A.kc = (bf*)h->kc; A.vc = (bf*)h->vc;
-  A.xa = h->xa; A.x1 = h->x1; A.qkv = h->qkv; A.mid = h->mid; A.attn_out = h->attn_out;
-  A.part_o = h->part_o; A.part_ml = h->part_ml; A.max_splits = h->max_splits; A.tickets = h->tickets;
+  A.xa = h->ll_xa; A.x1 = h->ll_x1; A.qkv = h->ll_qkv; A.mid = h->ll_mid;
+  A.part_o = h->ll_po; A.part_ml = h->ll_pml; A.max_splits = h->max_splits;
   A.logits_own = h->logits_own; A.w = h->w; A.qk = h->qk; A.q = h->q;
-  A.rowmax = h->rowmax_g; A.rowsum = h->rowsum_g; A.chunk_mass = h->chunk_mass; A.chunk_best = h->chunk_best;
-  A.n_chunks = h->n_chunks; A.tokens = h->tokens; A.bar = h->bar; A.ssq = h->ssq; A.err = h->err; A.packed = h->packed;
+  A.rowmax = h->ll_rowmax; A.rowmax2 = h->ll_rowmax2; A.rowsum = h->ll_rowsum; A.chunk_mass = h->ll_cmass;
+  A.n_chunks = h->n_chunks; A.tokens = h->tokens; A.err = h->err; A.packed = h->packed;
   A.trace_stride = h->trace_stride;
   h->persist_ok = true;
   return TABED_OK;
@@ -520,7 +535,14 @@ int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_
   A.u = u_draft; A.out_tokens = out_tokens; A.logits_override = h->logits_override;
   (void)max_pos;
   A.split_len = (h->hd <= 64) ? 256 : 128;          // positions per attention item: 4 register passes of the CTA
-  A.bar_sel = (int)(h->launches_persist & 1u);
+  // epochs: this launch stamps epoch0 + 1 ... epoch0 + G (5 L + 8); when the counter nears its end the buffers are cleared
+  const unsigned span = (unsigned)h->G * (5u * (unsigned)h->L + 8u);
+  if (h->ll_epoch > 0xFFFFFFFFu - 2u * span) {
+    for (auto& b : h->ll_all) if (cudaMemsetAsync(b.first, 0, b.second, h->stream) != cudaSuccess) return TABED_ERR_CUDA;
+    h->ll_epoch = 0;
+  }
+  A.epoch0 = h->ll_epoch;
+  h->ll_epoch += span;
   A.trace = h->trace_on ? h->trace : nullptr; A.trace_cta = h->trace_cta;
   void* args[] = {&A};
   const void* kern = h->trace_on ? (const void*)k_draft_round<true> : (const void*)k_draft_round<false>;
@@ -1192,14 +1214,14 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
 }
 
 namespace {
-// One CTA takes the grid barrier against a target that needs a second arrival: the bounded wait runs out,
-// the error bit is set and the kernel returns.
-__global__ void __launch_bounds__(kPT) k_barrier_probe(unsigned* bar, int* err) {
+// One CTA polls a flagged word for an epoch that nobody writes: the bounded wait runs out, the error bit is set
+// and the kernel returns.
+__global__ void __launch_bounds__(kPT) k_wait_probe(const uint2* word, int* err) {
   __shared__ PShared S;
   if (threadIdx.x == 0) S.dead = 0;
   __syncthreads();
-  const unsigned base = *bar;
-  grid_barrier(S, bar, base + 2u, err);
+  if (threadIdx.x == 0) ll_wait1(word, 0xFFFFFFFFu, S, err);
+  __syncthreads();
 }
 }  // namespace
 
@@ -1208,11 +1230,8 @@ int tabed_debug_barrier_timeout(tabed_handle* h) {
   if (!h->persist_ok) return TABED_ERR_UNSUPPORTED;
   if (h->phase != PH_IDLE) return TABED_ERR_BAD_STATE;
   DeviceGuard guard(h->cfg.device);
-  // (the counter of the launch after next: this launch's own counter is reset by the next persistent launch)
-  unsigned* bar = h->bar + (h->launches_persist & 1u);
-  k_barrier_probe<<<1, kPT, 0, h->stream>>>(bar, h->err);
+  k_wait_probe<<<1, kPT, 0, h->stream>>>(h->ll_probe, h->err);
   h->launches++;
-  if (cudaMemsetAsync(bar, 0, sizeof(unsigned), h->stream) != cudaSuccess) { cudaGetLastError(); return TABED_ERR_CUDA; }
   return tabed_last_device_error(h);
 }
 

@@ -133,7 +133,7 @@ def test_phase_trace_is_monotonic():
     pair.gpu.debug_trace(True)
     H.lockstep_round(pair, 0, override=True)
     tr = pair.gpu.debug_view(TB.VIEW_TRACE).cpu().numpy().astype(np.int64)
-    n_bar = 5 * wl.drafter.n_layers + 5                # two more barriers per step while logits are overridden
+    n_bar = 5 * wl.drafter.n_layers + 4                # one more record per step while logits are overridden
     flat = tr[:, :n_bar, 0].reshape(-1)
     assert np.all(flat > 0) and np.all(np.diff(flat) > 0)
     assert (flat[-1] - flat[0]) < 50_000_000          # one round stays far below 50 ms
