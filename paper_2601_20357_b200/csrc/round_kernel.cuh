@@ -51,6 +51,7 @@ constexpr int kPPer = kChunk / kPT;      // vocabulary elements per thread and c
 constexpr int kPMaxD = 2048;             // d_model bound
 constexpr int kTraceRec = 8;             // words per record of the phase timeline
 constexpr int kPMaxL = 64;               // layers (their pointer table lives in shared memory)
+constexpr int kPMaxHeads = 64;           // query heads
 constexpr int kMaxUnits = 1024;          // units of one CTA in one decoder step (config 3 needs 168)
 constexpr int kMaxPhase = 4 * kPMaxL + 1;
 
@@ -200,6 +201,7 @@ struct PShared {
   int lm_src[kPSlots];
   int att[8];                           // attention geometry of the step: T, g_lo, g_hi, then this CTA's first chunk (s, gk, split, nsplit, g0)
   int pair_base[kPSlots], pair_ns[kPSlots];   // per slot: chunks before its first pair, chunks per pair (0: inactive)
+  unsigned char nseg[kPSlots][kPMaxHeads];    // per (slot, head): partial attention results of the step
   int tok[kPSlots];
   float rowmax_f[kPSlots];
   unsigned long long row_part[kPSlots];
@@ -207,12 +209,17 @@ struct PShared {
   unsigned long long thr;
 };
 
-__device__ __forceinline__ uint32_t unit_pack(int kind, int layer, int u) { return (uint32_t)kind | ((uint32_t)layer << 3) | ((uint32_t)u << 10); }
+// a unit of the list: kind (3 bits), layer (7), sub-unit of its tile (6), tile (16) - no division where it is used
+__device__ __forceinline__ uint32_t unit_pack(int kind, int layer, int tile, int sub) {
+  return (uint32_t)kind | ((uint32_t)layer << 3) | ((uint32_t)sub << 10) | ((uint32_t)tile << 16);
+}
+__device__ __forceinline__ int unit_sub(uint32_t e) { return (int)((e >> 10) & 63u); }
+__device__ __forceinline__ int unit_tile(uint32_t e) { return (int)(e >> 16); }
 
 // Issue the bulk copy of unit number k (counted over the whole round) into its ring slot (one thread).
 __device__ __forceinline__ void issue_unit(const RoundArgs& A, PShared& S, unsigned char* ring, unsigned k, unsigned per_step) {
   const uint32_t e = S.ulist[k % per_step];
-  const int kind = e & 7, layer = (e >> 3) & 127, u = e >> 10;
+  const int kind = e & 7, layer = (e >> 3) & 127, u = unit_tile(e) * A.geom[kind].nsub + unit_sub(e);
   const unsigned bytes = 16u * ((unsigned)A.geom[kind].kchunk * 2u + 16u);
   const unsigned char* src = A.packed + A.pack_off[kind] + (size_t)u * bytes +
                              (kind == KIND_LM ? 0ull : (unsigned long long)layer * A.pack_layer_stride);
@@ -446,7 +453,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #pragma unroll 1
     for (int t = first; t < A.geom[kind].n_tiles; t += NC)
 #pragma unroll 1
-      for (int sb = 0; sb < nsub; ++sb) S.ulist[n++] = unit_pack(kind, p >> 2, t * nsub + sb);
+      for (int sb = 0; sb < nsub; ++sb) S.ulist[n++] = unit_pack(kind, p >> 2, t, sb);
   }
   __syncthreads();
   const unsigned per_step = S.pstart[n_phase];
@@ -550,6 +557,20 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       S.att[0] = T; S.att[1] = lo; S.att[2] = hi; S.att[3] = s; S.att[4] = gk; S.att[5] = nsplit ? rem - gk * nsplit : 0;
       S.att[6] = nsplit; S.att[7] = acc + gk * nsplit;
     }
+    if (warp == kPW - 1) {
+      // partial results every (slot, head) pair will have (first read by the O-projection staging): the last warp's lanes
+      // share the pairs
+      __syncwarp();
+      const int T = S.att[0];
+#pragma unroll 1
+      for (int pr2 = lane; pr2 < kPSlots * A.Hkv; pr2 += 32) {
+        const int s3 = pr2 / A.Hkv, gk3 = pr2 - s3 * A.Hkv;
+        const int nsp = S.pair_ns[s3], g0 = S.pair_base[s3] + gk3 * nsp;
+        const int cnt = nsp == 0 ? 0 : ((T >= NC) ? ((g0 + nsp) * NC - 1) / T - ((g0 + 1) * NC - 1) / T + 1 : nsp);
+#pragma unroll 1
+        for (int t3 = 0; t3 < grp; ++t3) S.nseg[s3][gk3 * grp + t3] = (unsigned char)cnt;
+      }
+    }
 
 #pragma unroll 1
     for (int phase = 0; phase < n_phase; ++phase) {
@@ -583,6 +604,12 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         const int d2 = d >> 1;                                   // 16-byte pieces of a row
         constexpr int kMaxPieces = 8;
         float2 xv[kMaxPieces];
+        uint32_t gw[kMaxPieces];                                 // the gains do not wait for anybody
+#pragma unroll
+        for (int k = 0; k < kMaxPieces; ++k) {
+          const int e2 = wi * 32 + lane + k * nw * 32;
+          gw[k] = e2 < d2 ? __ldg(reinterpret_cast<const uint32_t*>(gain) + e2) : 0u;
+        }
         {
           int n = 0;
 #pragma unroll
@@ -628,7 +655,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         for (int k = 0; k < kMaxPieces; ++k) {
           const int e2 = wi * 32 + lane + k * nw * 32;
           if (e2 < d2) {
-            const uint32_t g2 = __ldg(reinterpret_cast<const uint32_t*>(gain) + e2);
+            const uint32_t g2 = gw[k];
             *reinterpret_cast<uint32_t*>(act + s * apitch + 2 * e2) =
                 pack_bf16(xv[k].x * sc * __uint_as_float(g2 << 16), xv[k].y * sc * __uint_as_float(g2 & 0xFFFF0000u));
           }
@@ -638,20 +665,18 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         // ---- stage the attention output, whole rows: put every pair's partial results together -----
         // How many partial results a (slot, KV head) pair has follows from the step's chunk geometry (the same
         // arithmetic as in the CTAs that produce them).
+        // Warp w serves input row w % n_in; the row's warps walk its groups of 4 output dims.
         const int nvec = g.kchunk >> 2;
-        const int T = S.att[0];
+        const int s = warp % n_in, wi = warp / n_in, nw = (kPW - s + n_in - 1) / n_in;
+        const int hd_shift = 31 - __clz(A.hd);                 // head size is a power of two
 #pragma unroll 1
-        for (int idx0 = 0; idx0 < n_in * nvec; idx0 += kPT) {
-          const int idx = idx0 + tid;
-          const bool item = idx < n_in * nvec;
-          const int s = item ? idx / nvec : 0, j = item ? (idx - s * nvec) << 2 : 0;
-          const int head = j / A.hd, dd = j - head * A.hd;
+        for (int jv0 = wi * 32; jv0 < nvec; jv0 += nw * 32) {
+          const int jv = jv0 + lane;
+          const bool item = jv < nvec;
+          const int j = item ? jv << 2 : 0;
+          const int head = j >> hd_shift, dd = j - (head << hd_shift);
           const size_t base = ((size_t)s * A.H + head) * A.max_splits;
-          int n_seg = 0;
-          if (item && S.slot[s].active) {
-            const int nsp = S.pair_ns[s], g0 = S.pair_base[s] + (head / grp) * nsp;
-            n_seg = (T >= NC) ? ((g0 + nsp) * NC - 1) / T - ((g0 + 1) * NC - 1) / T + 1 : nsp;
-          }
+          const int n_seg = (item && S.slot[s].active) ? S.nseg[s][head] : 0;
           float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
           float M = -INFINITY, den = 0.0f;
           const int n_seg_warp = __reduce_max_sync(0xffffffffu, n_seg);
@@ -699,37 +724,38 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       for (unsigned k0 = ka; k0 < kb; k0 += kWG) {
         const unsigned k = k0 + (unsigned)wgrp;
         const bool has = k < kb;
-        int u = 0, sub = 0;
-        if (has) { u = (int)(S.ulist[k - (unsigned)step * per_step] >> 10); sub = u % g.nsub; }
+        int sub = 0;
+        if (has) sub = unit_sub(S.ulist[k - (unsigned)step * per_step]);
         if (kind == KIND_DN) {
           // stage this round's chunks of the gated product (left as bf16 by the gate/up epilogue): area of
           // group w <- columns of its sub-unit, 16 bytes at a time
-          // (a flagged word carries two bf16 values; a 16-byte load brings four of them; four loads in flight)
-          const int nvec = g.kchunk >> 2;
-          const int total = kWG * n_in * nvec;
+          // (a flagged word carries two bf16 values; a 16-byte load brings four of them).  Warp w serves the area of
+          // group w / kGW; its kGW warps walk the chunk's 16-byte pieces of every input row, all loads in flight.
+          const int nvec = g.kchunk >> 2;                       // 16-byte pieces of a chunk
+          const int w2 = warp / kGW, part = warp - w2 * kGW;
+          const unsigned kq = k0 + (unsigned)w2;
+          const int sq = kq < kb ? unit_sub(S.ulist[kq - (unsigned)step * per_step]) : 0;
+          int jj = part * 32 + lane, s2 = 0;                    // this lane's next (piece, row)
 #pragma unroll 1
-          for (int it0 = 0; it0 < total; it0 += 8 * kPT) {
+          while (__shfl_sync(0xffffffffu, jj, 0) < nvec) {      // (lane 0 has the most pieces: a warp-uniform trip count)
             const uint2* ptr[8];
             uint4 raw[8];
             int dst[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              const int idx = it0 + q * kPT + tid;
-              ptr[q] = nullptr; dst[q] = -1;
-              if (idx < total) {
-                const int w2 = idx / (n_in * nvec), r2 = idx - w2 * (n_in * nvec);
-                const int s = r2 / nvec, j = (r2 - s * nvec) << 2;
-                const unsigned kq = k0 + (unsigned)w2;
-                if (kq < kb && S.slot[s].active) {
-                  const int sq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10) % g.nsub;
-                  ptr[q] = A.mid + (((size_t)s * A.F + (size_t)sq * g.kchunk + j) >> 1);
-                  dst[q] = w2 * area_elems + s * apitch + j;
+            for (int t = 0; t < 8; ++t) {
+              ptr[t] = nullptr; dst[t] = -1;
+              if (jj < nvec) {
+                if (kq < kb && S.slot[s2].active) {
+                  const int j = jj << 2;
+                  ptr[t] = A.mid + (((size_t)s2 * A.F + (size_t)sq * g.kchunk + j) >> 1);
+                  dst[t] = w2 * area_elems + s2 * apitch + j;
                 }
+                if (++s2 == n_in) { s2 = 0; jj += kGW * 32; }
               }
             }
             ll_poll<8>([&](int j) { return ptr[j]; }, 8, ep_gu, raw, S, A.err);
 #pragma unroll
-            for (int q = 0; q < 8; ++q) if (dst[q] >= 0) *reinterpret_cast<uint2*>(act + dst[q]) = make_uint2(raw[q].x, raw[q].z);
+            for (int t = 0; t < 8; ++t) if (dst[t] >= 0) *reinterpret_cast<uint2*>(act + dst[t]) = make_uint2(raw[t].x, raw[t].z);
           }
           __syncthreads();
           TSEC(0);
@@ -749,9 +775,9 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           const int q = tid >> 7, e = tid & 127, r = e & 15, n = e >> 4;
           const unsigned kq = k0 + (unsigned)q;
           if (kq < kb) {
-            const int uq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10), sq = uq % g.nsub;
-            if ((q % nsub_eff) == 0 && (sq + nsub_eff == g.nsub) && n < n_in && S.slot[n].active) {
-              base_p = (kind == KIND_O ? A.xa : A.x1) + (size_t)n * d + (uq / g.nsub) * 16 + r;
+            const uint32_t eq = S.ulist[kq - (unsigned)step * per_step];
+            if ((q & (nsub_eff - 1)) == 0 && (unit_sub(eq) + nsub_eff == g.nsub) && n < n_in && S.slot[n].active) {
+              base_p = (kind == KIND_O ? A.xa : A.x1) + (size_t)n * d + unit_tile(eq) * 16 + r;
               base_w = ll_load1(base_p);
             }
           }
@@ -786,11 +812,10 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         {
           const int q = tid >> 7, e = tid & 127, r = e & 15, n = e >> 4;
           const unsigned kq = k0 + (unsigned)q;
-          int uq = 0, sq = 0;
+          int sq = 0, tile = 0;
           const bool on = kq < kb;
-          if (on) { uq = (int)(S.ulist[kq - (unsigned)step * per_step] >> 10); sq = uq % g.nsub; }
-          const bool lead = on && (q % nsub_eff) == 0 && (sq + nsub_eff == g.nsub);   // tile complete in this round
-          const int tile = uq / g.nsub;
+          if (on) { const uint32_t eq = S.ulist[kq - (unsigned)step * per_step]; sq = unit_sub(eq); tile = unit_tile(eq); }
+          const bool lead = on && (q & (nsub_eff - 1)) == 0 && (sq + nsub_eff == g.nsub);   // tile complete in this round (nsub_eff is 1, 2 or 4)
           const bool slot_on = n < n_in && (kind == KIND_LM || S.slot[n].active);
           const int o = tile * 16 + r;
           // the residual this tile adds to: its words arrived phases ago (layer 0: the embedding itself)

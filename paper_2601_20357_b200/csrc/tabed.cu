@@ -408,7 +408,7 @@ int setup_persistent(tabed_handle* h) {
   if (c.dtype != TABED_DTYPE_BF16 || h->D > 1) return TABED_OK;      // (the in-kernel draw proposes one candidate per step)
   const int grp = h->H / h->Hkv;
   if (2 * h->R > kPSlots || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
-      grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || (h->cap + 127) / 128 > kAttnSplitMax)
+      grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || h->H > kPMaxHeads || (h->cap + 127) / 128 > kAttnSplitMax)
     return TABED_OK;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess) return TABED_ERR_CUDA;
