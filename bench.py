@@ -536,9 +536,11 @@ def write_trace(path, cta, wl, tr, mhz):
     names_b = [f"L{l}.{nm}" for l in range(L) for nm in ("qkv", "attn", "o", "gateup", "down")] + ["lm_head", "expsum", "mix"]
     with open(path, "w") as f:
         f.write("# made by: python " + " ".join(a if a != path else "<this file>" for a in sys.argv) + "\n")
-        f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA {cta}): us from the previous grid barrier to this one,\n"
-                f"# then that CTA's share of it in us (cycles / {mhz:.0f} MHz): stage, wait-tiles, mma, issue+epilogue, other, barrier\n"
-                f"# (attention phases: load+stage q/k/v, scores+softmax, PV+write, split merge, -, barrier)\n")
+        f.write(f"# phase timeline of k_draft_round, workload {wl.name} (CTA {cta}): us from the end of the previous phase to the end of this one,\n"
+                f"# then that CTA's share of it in us (cycles / {mhz:.0f} MHz): waiting for + staging activations, waiting for weight tiles, products,\n"
+                f"# epilogue + refill, rest, (unused)\n"
+                f"# (attention phases: waiting for + staging q/k/v, scores+softmax, PV+write, split merge, rest, -;\n"
+                f"#  a phase in which the CTA owns no tile shows only the time it took to walk through it)\n")
         prev = None
         for st in range(G):
             for j in range(nb_step):

@@ -122,9 +122,10 @@ extern "C" {
 #define TABED_PATH_AUTO        0   /* persistent kernel if the drafter qualifies, else tensor-core
                                       projections if it qualifies, else per-operation                    */
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
-#define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, 2*B*m <= 8
-                                      slots, d_model <= 2048 and a multiple of 16, d_ffn a multiple of 16,
-                                      (H/Hkv)*head_dim <= 512, <= 64 layers, kv_capacity <= 32768        */
+#define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, tree_width 1,
+                                      2*B*m <= 8 slots, d_model <= 2048 (<= 1024 with more than 4 slots) and
+                                      a multiple of 16, d_ffn a multiple of 16, H <= 64, (H/Hkv)*head_dim <= 512, <= 64 layers,
+                                      kv_capacity <= 32768                                                */
 #define TABED_PATH_TENSOR_CORE 3   /* one kernel per operation with the projections as tcgen05 contractions
                                       over all rows: any bf16 drafter with d_model, d_ffn, H*head_dim
                                       multiples of 8 (the automatic choice when the persistent kernel

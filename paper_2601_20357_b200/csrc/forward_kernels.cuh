@@ -303,8 +303,11 @@ __global__ void __launch_bounds__(kGemvThreads) k_gemv(GemvArgs A) {
 // cache at the slot's position.  Pairs (i, i + hd/2), angle pos * theta^(-2i/hd) from a table.
 // Cache layout [R][L][Hkv][cap][hd].   grid (slots), block 128.
 // ------------------------------------------------------------------------------------------------
-template <typename T>
 // part != nullptr: the QKV projection is still ks split-K slabs [ks][slab], summed here in slab order.
+// One thread handles one rotation pair (or two v elements) at a time and requests all the slabs' values of it
+// before it adds any, so that a slot costs one or two trips to L2, not one per slab.
+constexpr int kRopeMaxSlabs = 8;
+template <typename T>
 __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restrict__ slots, int H, int Hkv, int hd,
                               const float* __restrict__ rope_cos, const float* __restrict__ rope_sin,
                               T* __restrict__ kc, T* __restrict__ vc, int layer, int L, int cap,
@@ -317,17 +320,23 @@ __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restric
   const int half = hd >> 1;
   float* row = qkv + (long long)s * (H + 2 * Hkv) * hd;
   const float* prow = part ? part + (long long)s * (H + 2 * Hkv) * hd : nullptr;
-  auto value = [&](int col) {
-    if (!prow) return row[col];
-    float v = 0.0f;
-    int k = 0;
-    for (; k + 4 <= ks; k += 4) {                  // four slabs in flight, summed in slab order
-      const float a0 = prow[(size_t)k * slab + col], a1 = prow[(size_t)(k + 1) * slab + col];
-      const float a2 = prow[(size_t)(k + 2) * slab + col], a3 = prow[(size_t)(k + 3) * slab + col];
-      v += a0; v += a1; v += a2; v += a3;
+  // values of two columns, the slabs added in slab order
+  auto value2 = [&](int col_a, int col_b, float& va, float& vb) {
+    if (!prow) { va = row[col_a]; vb = row[col_b]; return; }
+    if (ks <= kRopeMaxSlabs) {
+      float a[kRopeMaxSlabs], b2[kRopeMaxSlabs];
+#pragma unroll
+      for (int k = 0; k < kRopeMaxSlabs; ++k) {
+        a[k] = k < ks ? prow[(size_t)k * slab + col_a] : 0.0f;
+        b2[k] = k < ks ? prow[(size_t)k * slab + col_b] : 0.0f;
+      }
+      va = 0.0f; vb = 0.0f;
+#pragma unroll
+      for (int k = 0; k < kRopeMaxSlabs; ++k) if (k < ks) { va += a[k]; vb += b2[k]; }
+    } else {
+      va = 0.0f; vb = 0.0f;
+      for (int k = 0; k < ks; ++k) { va += prow[(size_t)k * slab + col_a]; vb += prow[(size_t)k * slab + col_b]; }
     }
-    for (; k < ks; ++k) v += prow[(size_t)k * slab + col];
-    return v;
   };
   const float* c = rope_cos + (long long)sd.pos * half;
   const float* sn = rope_sin + (long long)sd.pos * half;
@@ -335,9 +344,11 @@ __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restric
   for (int idx = threadIdx.x; idx < (H + Hkv) * half; idx += blockDim.x) {
     const int head = idx / half, i = idx - head * half;
     float* p = row + head * hd;
-    const float x1 = value(head * hd + i), x2 = value(head * hd + i + half);
-    const float r1 = x1 * c[i] - x2 * sn[i];
-    const float r2 = x2 * c[i] + x1 * sn[i];
+    const float ci = c[i], si = sn[i];
+    float x1, x2;
+    value2(head * hd + i, head * hd + i + half, x1, x2);
+    const float r1 = x1 * ci - x2 * si;
+    const float r2 = x2 * ci + x1 * si;
     if (head < H) {
       p[i] = Elem<T>::round(r1); p[i + half] = Elem<T>::round(r2);
     } else {
@@ -346,10 +357,12 @@ __global__ void k_rope_append(float* __restrict__ qkv, const SlotDesc* __restric
       Elem<T>::store(dst + i, r1); Elem<T>::store(dst + i + half, r2);
     }
   }
-  for (int idx = threadIdx.x; idx < Hkv * hd; idx += blockDim.x) {
-    const int g = idx / hd, i = idx - g * hd;
+  for (int idx = threadIdx.x; idx < Hkv * half; idx += blockDim.x) {
+    const int g = idx / half, i = idx - g * half;
     T* dst = vc + ((((long long)sd.row * L + layer) * Hkv + g) * cap + sd.pos) * hd;
-    Elem<T>::store(dst + i, value((H + Hkv) * hd + idx));
+    float v1, v2;
+    value2((H + Hkv) * hd + g * hd + i, (H + Hkv) * hd + g * hd + i + half, v1, v2);
+    Elem<T>::store(dst + i, v1); Elem<T>::store(dst + i + half, v2);
   }
 }
 

@@ -309,34 +309,49 @@ __global__ void __launch_bounds__(256) k_prep_row(const PrepRowArgs P) {
   __shared__ float red[8];
   __shared__ float s_scale;
   float* xr = P.x + (size_t)s * P.d;
-  float ss = 0.0f;
-  // pass 1: resolve, write back, sum of squares.  Thread owns groups of 8 consecutive elements.
-  for (int k = tid * 8; k < P.d; k += 256 * 8) {
-    float f[8];
+  // resolve 8 consecutive elements: the residual plus the slabs, all requested before any is added (slab order kept)
+  auto resolve = [&](int k, float (&f)[8]) {
     const float4 a = *reinterpret_cast<const float4*>(xr + k), b = *reinterpret_cast<const float4*>(xr + k + 4);
     f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
-    for (int q0 = 0; q0 < P.ks; q0 += 4) {          // four slabs in flight, added in slab order
-      float4 c[4], e[4];
+    for (int q0 = 0; q0 < P.ks; q0 += 8) {
+      float4 c[8], e[8];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < 8; ++j) {
         const bool ok = q0 + j < P.ks;
         const float* pp = P.partial + (size_t)(ok ? q0 + j : 0) * P.slab + (size_t)s * P.d + k;
         c[j] = ok ? *reinterpret_cast<const float4*>(pp) : make_float4(0.f, 0.f, 0.f, 0.f);
         e[j] = ok ? *reinterpret_cast<const float4*>(pp + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < 8; ++j) {
         if (q0 + j < P.ks) {
           f[0] += c[j].x; f[1] += c[j].y; f[2] += c[j].z; f[3] += c[j].w; f[4] += e[j].x; f[5] += e[j].y; f[6] += e[j].z; f[7] += e[j].w;
         }
       }
     }
+  };
+  auto emit = [&](int k, const float (&f)[8], float sc) {
+    float g[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) g[j] = P.gain ? f[j] * sc * __bfloat162float(P.gain[k + j]) : f[j];
+    uint4 v;
+    v.x = pack_bf16(g[0], g[1]); v.y = pack_bf16(g[2], g[3]); v.z = pack_bf16(g[4], g[5]); v.w = pack_bf16(g[6], g[7]);
+    const int kc = k / kTcKC, k8 = (k % kTcKC) >> 3;
+    *reinterpret_cast<uint4*>(P.dst + (size_t)kc * tc_block_bytes(P.n_pad) + ((size_t)k8 * (P.n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
+  };
+  const bool one_pass = P.d <= 256 * 8;              // every thread owns at most one group of 8: it stays in registers
+  float keep[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float ss = 0.0f;
+  // pass 1: resolve, write back, sum of squares.  Thread owns groups of 8 consecutive elements.
+  for (int k = tid * 8; k < P.d; k += 256 * 8) {
+    float f[8];
+    resolve(k, f);
     if (P.write_back && P.ks > 0) {
       *reinterpret_cast<float4*>(xr + k) = make_float4(f[0], f[1], f[2], f[3]);
       *reinterpret_cast<float4*>(xr + k + 4) = make_float4(f[4], f[5], f[6], f[7]);
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) ss = fmaf(f[j], f[j], ss);
+    for (int j = 0; j < 8; ++j) { ss = fmaf(f[j], f[j], ss); keep[j] = f[j]; }
   }
   ss = warp_sum_f32(ss);
   if ((tid & 31) == 0) red[tid >> 5] = ss;
@@ -348,26 +363,20 @@ __global__ void __launch_bounds__(256) k_prep_row(const PrepRowArgs P) {
   }
   __syncthreads();
   const float sc = s_scale;
-  // pass 2: (re-read; the values are in L1/L2) scale, round, store 16-byte pieces of the canonical layout
-  for (int k = tid * 8; k < P.d; k += 256 * 8) {
-    float f[8];
-    const float4 a = *reinterpret_cast<const float4*>(xr + k), b = *reinterpret_cast<const float4*>(xr + k + 4);
-    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
-    if (!(P.write_back && P.ks > 0)) {
-      for (int q = 0; q < P.ks; ++q) {
-        const float* pp = P.partial + (size_t)q * P.slab + (size_t)s * P.d + k;
-        const float4 c = *reinterpret_cast<const float4*>(pp), e = *reinterpret_cast<const float4*>(pp + 4);
-        f[0] += c.x; f[1] += c.y; f[2] += c.z; f[3] += c.w; f[4] += e.x; f[5] += e.y; f[6] += e.z; f[7] += e.w;
+  // pass 2: scale, round, store 16-byte pieces of the canonical layout (long rows: resolved again, the values are in L1/L2)
+  if (one_pass) {
+    if (tid * 8 < P.d) emit(tid * 8, keep, sc);
+  } else {
+    for (int k = tid * 8; k < P.d; k += 256 * 8) {
+      float f[8];
+      if (P.write_back && P.ks > 0) {
+        const float4 a = *reinterpret_cast<const float4*>(xr + k), b = *reinterpret_cast<const float4*>(xr + k + 4);
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+      } else {
+        resolve(k, f);
       }
+      emit(k, f, sc);
     }
-    if (P.gain) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) f[j] = f[j] * sc * __bfloat162float(P.gain[k + j]);
-    }
-    uint4 v;
-    v.x = pack_bf16(f[0], f[1]); v.y = pack_bf16(f[2], f[3]); v.z = pack_bf16(f[4], f[5]); v.w = pack_bf16(f[6], f[7]);
-    const int kc = k / kTcKC, k8 = (k % kTcKC) >> 3;
-    *reinterpret_cast<uint4*>(P.dst + (size_t)kc * tc_block_bytes(P.n_pad) + ((size_t)k8 * (P.n_pad / 8) + (r >> 3)) * 128 + (r & 7) * 16) = v;
   }
 }
 
@@ -385,12 +394,22 @@ __global__ void k_swiglu_prep(const float* __restrict__ partial, int ks, size_t 
   uint4 v = make_uint4(0u, 0u, 0u, 0u);
   if (f0 < F) {
     float g[8] = {0, 0, 0, 0, 0, 0, 0, 0}, u[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int q = 0; q < ks; ++q) {
-      const float* pg = partial + (size_t)q * slab + (size_t)s * (2 * F) + f0;
-      const float4 a = *reinterpret_cast<const float4*>(pg), b = *reinterpret_cast<const float4*>(pg + 4);
-      const float4 c = *reinterpret_cast<const float4*>(pg + F), e = *reinterpret_cast<const float4*>(pg + F + 4);
-      g[0] += a.x; g[1] += a.y; g[2] += a.z; g[3] += a.w; g[4] += b.x; g[5] += b.y; g[6] += b.z; g[7] += b.w;
-      u[0] += c.x; u[1] += c.y; u[2] += c.z; u[3] += c.w; u[4] += e.x; u[5] += e.y; u[6] += e.z; u[7] += e.w;
+    for (int q0 = 0; q0 < ks; q0 += 4) {              // four slabs requested together, added in slab order
+      float4 a[4], b[4], c[4], e[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool ok = q0 + j < ks;
+        const float* pg = partial + (size_t)(ok ? q0 + j : 0) * slab + (size_t)s * (2 * F) + f0;
+        const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+        a[j] = ok ? *reinterpret_cast<const float4*>(pg) : z; b[j] = ok ? *reinterpret_cast<const float4*>(pg + 4) : z;
+        c[j] = ok ? *reinterpret_cast<const float4*>(pg + F) : z; e[j] = ok ? *reinterpret_cast<const float4*>(pg + F + 4) : z;
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (q0 + j >= ks) continue;
+        g[0] += a[j].x; g[1] += a[j].y; g[2] += a[j].z; g[3] += a[j].w; g[4] += b[j].x; g[5] += b[j].y; g[6] += b[j].z; g[7] += b[j].w;
+        u[0] += c[j].x; u[1] += c[j].y; u[2] += c[j].z; u[3] += c[j].w; u[4] += e[j].x; u[5] += e[j].y; u[6] += e[j].z; u[7] += e[j].w;
+      }
     }
     float m[8];
 #pragma unroll

@@ -8,23 +8,32 @@
 //   * the weights never stop streaming: every CTA owns a fixed share of the weight tiles of every
 //     phase (its unit list is built once, in shared memory), and a ring of shared-memory slots is
 //     kept full by bulk asynchronous copies (cp.async.bulk + mbarrier) several phases ahead of the
-//     arithmetic, so HBM stays busy across the grid barriers;
+//     arithmetic, so HBM stays busy across the phase boundaries;
 //   * the weights are read from a private copy laid out for this kernel at set-up: every unit (16
 //     output rows x kchunk input columns, rows padded to a bank-conflict-free shared-memory pitch)
 //     is one contiguous block, hence ONE bulk copy;
-//   * a phase is: grid barrier -> stage the (tiny) activations from L2 -> tensor-core products of
-//     the weight tiles already sitting in shared memory -> results back to L2.  The chain of phases
-//     is the critical path, so it is kept short: 5 barriers per layer (QKV, attention, O, gate/up,
-//     down).  A 16-row tile always takes its whole input dimension on ONE CTA (long rows as
-//     sub-units whose products accumulate in registers), so no projection leaves split-K partial
-//     sums behind and the residual adds and RMSNorm statistics ride in the epilogues;
+//   * there is NO grid barrier.  Every activation that crosses CTAs travels as an 8-byte word
+//     {value, epoch} written with one 64-bit store; the epoch names the launch, the step and the
+//     phase that produced it, so a consumer polls the data itself and starts as soon as ITS inputs
+//     have arrived (one L2 round trip per phase instead of an arrive/spin pair, and no CTA waits
+//     for producers it does not read).  A phase is: stage the (tiny) activations by polling their
+//     words -> tensor-core products of the weight tiles already sitting in shared memory -> flagged
+//     results back to L2.  5 phases per layer (QKV, attention, O, gate/up, down).  A 16-row tile
+//     always takes its whole input dimension on ONE CTA (long rows as sub-units whose products
+//     accumulate in registers), so no projection leaves split-K partial sums behind; residual adds
+//     ride in the epilogues and every consumer computes the RMSNorm sum of squares itself from the
+//     words it stages (warp per input row, fixed order: deterministic);
+//   * a poll re-requests all words still missing together; after two empty rounds one lane per
+//     warp keeps polling with a back-off while the others idle, so that long waits do not flood L2
+//     - all 32 lanes of a warp therefore enter the staging helpers together;
 //   * four warp groups work on four units at a time (mma.sync m16n8k16, bf16 x bf16 -> fp32:
 //     16 weight rows x up to 8 slots).  The contraction is HBM-bound (<= 8 flop per weight byte);
 //     the tensor pipe only keeps the ALUs off the critical path;
-//   * attention: a CTA walks a contiguous range of cache chunks; its first chunk's K, V are requested
-//     between the two halves of the grid barrier; head size 64 runs on mma fragments loaded straight
-//     from global memory; the partial results of a cache are put together by the next phase's staging;
-//   * all cross-CTA data is read with ld.global.cg (L2) because L1 is not coherent across SMs;
+//   * attention: a CTA walks a contiguous range of cache chunks; head size 64 runs on mma
+//     fragments loaded straight from global memory; the partial results of a cache are put
+//     together by the next phase's staging (a per-step table says how many partials each
+//     (slot, head) has);
+//   * all cross-CTA data is read with relaxed gpu-scope loads (L2): L1 is not coherent across SMs;
 //   * loops are deliberately not unrolled except the few hot ones: every phase runs its code once,
 //     so unrolling buys nothing and only inflates the instruction footprint.
 //

@@ -69,6 +69,8 @@ struct tabed_handle {
   unsigned long long* chunk_mass = nullptr; ChunkBest* chunk_best = nullptr;
   int* err = nullptr;
   int cs_max = 8;                   // largest cluster the per-request kernels may use on this device (8 portable, 16 opt-in)
+  int cs_active[5] = {0, 0, 0, 0, 0};   // clusters of 1, 2, 4, 8, 16 CTAs that the device keeps resident at once
+  int cta_budget = 3;               // CTAs per SM a launch of the per-request kernels may have in total (3, 6, 12 measured: 3 best)
   // staging for the host-buffer entry point
   float *st_u_draft = nullptr, *st_u_accept = nullptr, *st_u_resid = nullptr, *st_target = nullptr;
   int* st_tokens = nullptr;
@@ -170,13 +172,15 @@ void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_clusters
   h->launches++;
 }
 
-// CTAs per cluster: as many as keep about two CTAs per SM busy over all clusters, no finer than ~1024
+// CTAs per cluster: as many as the budget of CTAs per SM over all clusters allows, no finer than ~1024
 // vocabulary elements per CTA; slice = vocabulary elements per CTA (a multiple of 4, so that slices start on
 // 16-byte boundaries).
 int pick_cluster(const tabed_handle* h, int n_clusters, int* slice) {
   const int by_v = (h->V + 1023) / 1024, n_sm = h->n_sm > 0 ? h->n_sm : 148;
   int cs = 1;
-  while (cs * 2 <= h->cs_max && (long long)n_clusters * cs * 2 <= 3ll * n_sm && cs < by_v) cs *= 2;
+  // (measured on 32 requests: many small CTAs in several waves beat one wave of large ones - the passes are bound by
+  // dependent latencies and arithmetic, and more resident warps hide both)
+  while (cs * 2 <= h->cs_max && (long long)n_clusters * cs * 2 <= (long long)h->cta_budget * n_sm && cs < by_v) cs *= 2;
   *slice = ((h->V + cs - 1) / cs + 3) & ~3;
   return cs;
 }
@@ -826,6 +830,19 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
       for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_update_req})
         ok = ok && cudaOccupancyMaxActiveClusters(&n16, fn, &lc) == cudaSuccess && n16 >= 1;
       if (ok) h->cs_max = kReqMaxCluster;
+      // how many clusters of each size fit at once (the most demanding of the three kernels): a launch is sized for one wave
+      for (int i = 0; i < 5; ++i) {
+        const int cs = 1 << i;
+        if (cs > h->cs_max) break;
+        lc.gridDim = dim3(cs); at[0].val.clusterDim.x = cs;
+        int best = 1 << 30;
+        for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_update_req}) {
+          int n = 0;
+          if (cudaOccupancyMaxActiveClusters(&n, fn, &lc) != cudaSuccess) n = 0;
+          best = std::min(best, n);
+        }
+        h->cs_active[i] = best;
+      }
     }
     cudaGetLastError();
   }
