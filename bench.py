@@ -39,8 +39,8 @@ NCU_TRAFFIC = {("llava_small", "draft_round"): {"bytes": 690.05e6, "algorithmic_
                                                 "source": "profiles/k_draft_round_llava_small_ncu_full.md"},
                ("long_context", "draft_round"): {"bytes": 3028.2e6, "algorithmic_bytes_of_that_launch": 3006.2e6,
                                                  "source": "profiles/k_draft_round_llava_small_ncu_full.md (second part)"},
-               # captured on 16 of the 32 requests (capture-size rule) and scaled by the rows: 367.3 MB x 2
-               ("batched_serving", "attention"): {"bytes": 734.7e6, "algorithmic_bytes_of_that_launch": 707.5e6,
+               # captured on 16 of the 32 requests (capture-size rule) and scaled by the rows: 366.3 MB x 2
+               ("batched_serving", "attention"): {"bytes": 732.6e6, "algorithmic_bytes_of_that_launch": 707.5e6,
                                                   "source": "profiles/k_attn_tc_bf16_batched_serving_ncu_full.md "
                                                             "(16 requests captured, scaled x2 to the 32 of the workload)"}}
 

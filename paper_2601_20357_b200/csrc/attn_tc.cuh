@@ -7,11 +7,12 @@
 //   * a chunk of K and of V is one TMA tile each (cp.async.bulk.tensor, 128 rows x 64 dims, 128-byte
 //     swizzle), landing in a ring of shared-memory stages several chunks ahead of the arithmetic and
 //     signalling an mbarrier: the bytes in flight live in shared memory, not in registers;
-//   * the arithmetic runs on the tensor cores (mma.sync m16n8k16): rows of the A operand are the
-//     query heads that share the KV head (at most 8 of 16 rows are used: the contraction is far
-//     from the tensor roofline, the point is to keep the issue slots free).  q and the softmax
-//     weights are split into a bf16 head and a bf16 remainder (two products each), K and V are bf16
-//     already, so products are exact to ~2^-17 relative and the sums are fp32;
+//   * the arithmetic runs on the tensor cores (mma.sync m16n8k16) with the cache tile as the A operand
+//     (16 positions, resp. 16 dims, as its rows) and the query heads that share the KV head as the 8
+//     columns of B, so a tile costs half the mma it would with the (at most 8) heads as the 16 rows;
+//     the contraction is far from the tensor roofline, the point is to keep the issue slots free.
+//     q and the softmax weights are split into a bf16 head and a bf16 remainder (two products each),
+//     K and V are bf16 already, so products are exact to ~2^-17 relative and the sums are fp32;
 //   * a warp owns 16 positions of every chunk and carries its own running (max, sum, output) in
 //     registers across the chunks of a segment (the part of one cache that this CTA owns).  The
 //     warps run free of one another: each waits for a stage's "full" mbarrier on its own and
@@ -77,6 +78,13 @@ __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, u
   const float h0 = round_bf16(x0), h1 = round_bf16(x1);
   hi = pack_bf16(h0, h1);
   lo = pack_bf16(x0 - h0, x1 - h1);
+}
+
+// transposes an 8 x 8 matrix of 16-bit elements held one row per quad (lane (g, t): row g, columns 2t, 2t+1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -194,10 +202,16 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (g_lo + i + 1 < g_hi) advance(ahead);
     }
   }
-  // per-warp running state of the current segment (row g of the accumulators = head g of the group)
-  uint32_t qh[4][2], ql[4][2];                  // A fragments of q (rows 8..15 are zero)
-  float o[8][4];
-  float m_run = -INFINITY, l_run = 0.0f;        // maximum in base-2 units
+  // per-warp running state of the current segment.  The products are taken with the POSITIONS (scores) and the DIMS
+  // (output) as the 16 rows of the A operand and the group's query heads as the 8 columns of B: a cache tile is then
+  // covered by half as many mma as with the heads as rows (of which at most 8 of 16 would be used).
+  //   scores^T [16 positions x 8 heads] = K [16 x 64] q^T [64 x 8]          (4 k-steps, q as bf16 head + remainder)
+  //   out^T    [64 dims x 8 heads]     += V^T [64 x 16] P^T [16 x 8]        (4 m-tiles, P as bf16 head + remainder)
+  // Lane (g, t) holds columns (heads) 2t, 2t+1 of rows g, g+8; the softmax weights change from accumulator layout
+  // (positions as rows) to B-operand layout (positions as the summed index) with movmatrix.
+  uint32_t qh[4][2], ql[4][2];                  // B fragments of q^T per k-step (column g = head g; zero beyond the group)
+  float o[4][4];                                // out^T: m-tile j = dims 16j .. 16j+15
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};      // heads 2t, 2t+1; maxima in base-2 units
   int seg_first_split = 0, st = 0, seg_buf = 0;
   unsigned phase = 0;
   const float scale2 = A.scale * 1.4426950408889634f;
@@ -220,9 +234,9 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     }
     if (seg_start) {
       seg_first_split = split;
-      m_run = -INFINITY; l_run = 0.0f;
+      m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.0f;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
+      for (int j = 0; j < 4; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
       const float* qrow = sq + ((size_t)st * grp + g) * HD;
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
@@ -237,64 +251,56 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     }
     if (warp * 16 < cnt) {
       const uint32_t kst = smem_u32(stage0 + (size_t)st * 2 * kAtcTile), vst = kst + kAtcTile;
-      // scores of 16 positions: two n-tiles of 8, k = 64 dims in 4 steps; the products with the head and
-      // with the remainder of q accumulate separately (shorter dependent chains)
-      float sc[2][4], sr[2][4];
+      // scores of the warp's 16 positions for all heads of the group; four accumulators (q's head / remainder,
+      // even / odd k-step) keep the dependent chains two mma long
+      float sc[4][4];
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.0f;
-        sr[j][0] = sr[j][1] = sr[j][2] = sr[j][3] = 0.0f;
+      for (int j = 0; j < 4; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.0f;
+      const uint32_t krow = kst + (uint32_t)(warp * 16 + (ti & 1) * 8 + r8) * 128u;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        uint32_t ka[4];
+        ldsm_x4(ka, krow + (uint32_t)(((2 * kk + (ti >> 1)) ^ r8) << 4));
+        mma_bf16(sc[kk & 1], ka, qh[kk]);
+        mma_bf16(sc[2 + (kk & 1)], ka, ql[kk]);
       }
+      // softmax over the 16 positions, base 2: entries 0, 1 belong to position g, entries 2, 3 to position g + 8
+      float sv[4];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t a0h[4] = {qh[2 * half][0], 0u, qh[2 * half][1], 0u}, a0l[4] = {ql[2 * half][0], 0u, ql[2 * half][1], 0u};
-        const uint32_t a1h[4] = {qh[2 * half + 1][0], 0u, qh[2 * half + 1][1], 0u}, a1l[4] = {ql[2 * half + 1][0], 0u, ql[2 * half + 1][1], 0u};
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          uint32_t kb[4];
-          ldsm_x4(kb, kst + (uint32_t)(warp * 16 + j * 8 + r8) * 128u + (uint32_t)(((half * 4 + ti) ^ r8) << 4));
-          const uint32_t b0[2] = {kb[0], kb[1]}, b1[2] = {kb[2], kb[3]};
-          mma_bf16(sc[j], a0h, b0); mma_bf16(sr[j], a0l, b0);
-          mma_bf16(sc[j], a1h, b1); mma_bf16(sr[j], a1l, b1);
-        }
+      for (int e = 0; e < 4; ++e) {
+        sv[e] = ((sc[0][e] + sc[1][e]) + (sc[2][e] + sc[3][e])) * scale2;
+        if (cnt < SPLIT && warp * 16 + (e >> 1) * 8 + g >= cnt) sv[e] = -INFINITY;
       }
-      // softmax over the warp's 16 positions (row g lives in the 4 lanes of a quad), base 2
-      float mx = -INFINITY;
+      float mx0 = fmaxf(sv[0], sv[2]), mx1 = fmaxf(sv[1], sv[3]);
 #pragma unroll
-      for (int j = 0; j < 2; ++j)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          sc[j][e] = (sc[j][e] + sr[j][e]) * scale2;
-          if (cnt < SPLIT && warp * 16 + j * 8 + 2 * t4 + e >= cnt) sc[j][e] = -INFINITY;
-          mx = fmaxf(mx, sc[j][e]);
-        }
-      mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
-      if (__any_sync(FULL, mx > m_run)) {          // the running maximum moves: rescale what has been gathered
-        const float m_new = fmaxf(m_run, mx);
-        const float f_old = ex2_approx(m_run - m_new);
-        l_run *= f_old;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { o[j][0] *= f_old; o[j][1] *= f_old; }
-        m_run = m_new;
+      for (int ofs = 4; ofs < 32; ofs <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(FULL, mx0, ofs));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(FULL, mx1, ofs));
       }
-      float pw[2][2];
+      if (__any_sync(FULL, mx0 > m_run[0] || mx1 > m_run[1])) {      // a running maximum moves: rescale what has been gathered
+        const float n0 = fmaxf(m_run[0], mx0), n1 = fmaxf(m_run[1], mx1);
+        const float f0 = ex2_approx(m_run[0] - n0), f1 = ex2_approx(m_run[1] - n1);
+        l_run[0] *= f0; l_run[1] *= f1;
 #pragma unroll
-      for (int j = 0; j < 2; ++j)
+        for (int j = 0; j < 4; ++j) { o[j][0] *= f0; o[j][2] *= f0; o[j][1] *= f1; o[j][3] *= f1; }
+        m_run[0] = n0; m_run[1] = n1;
+      }
+      float pw[4];
 #pragma unroll
-        for (int e = 0; e < 2; ++e) { pw[j][e] = ex2_approx(sc[j][e] - m_run); l_run += pw[j][e]; }
-      uint32_t ph[4] = {0u, 0u, 0u, 0u}, pl[4] = {0u, 0u, 0u, 0u};
-      split_bf16x2(pw[0][0], pw[0][1], ph[0], pl[0]);
-      split_bf16x2(pw[1][0], pw[1][1], ph[2], pl[2]);
-      // output += P V: k = the 16 positions, n = 64 dims in 8 tiles (V tiles transposed on load)
-      const uint32_t vrow = vst + (uint32_t)(warp * 16 + (ti & 1) * 8 + r8) * 128u;
+      for (int e = 0; e < 4; ++e) { pw[e] = ex2_approx(sv[e] - m_run[e & 1]); l_run[e & 1] += pw[e]; }
+      uint32_t ph[2], pl[2], h01, l01, h23, l23;
+      split_bf16x2(pw[0], pw[1], h01, l01);
+      split_bf16x2(pw[2], pw[3], h23, l23);
+      ph[0] = movmatrix_trans(h01); ph[1] = movmatrix_trans(h23);
+      pl[0] = movmatrix_trans(l01); pl[1] = movmatrix_trans(l23);
+      // out^T += V^T P^T: the V tile transposed on load (rows = dims), the 16 positions are the summed index
+      const uint32_t vrow = vst + (uint32_t)(warp * 16 + (ti >> 1) * 8 + r8) * 128u;
 #pragma unroll
-      for (int jn = 0; jn < 8; jn += 2) {
-        uint32_t vb[4];
-        ldsm_x4_trans(vb, vrow + (uint32_t)(((jn + (ti >> 1)) ^ r8) << 4));
-        const uint32_t b0[2] = {vb[0], vb[1]}, b1[2] = {vb[2], vb[3]};
-        mma_bf16(o[jn], ph, b0); mma_bf16(o[jn + 1], ph, b1);
-        mma_bf16(o[jn], pl, b0); mma_bf16(o[jn + 1], pl, b1);
+      for (int j = 0; j < 4; ++j) {
+        uint32_t va[4];
+        ldsm_x4_trans(va, vrow + (uint32_t)(((2 * j + (ti & 1)) ^ r8) << 4));
+        mma_bf16(o[j], va, ph);
+        mma_bf16(o[j], va, pl);
       }
     }
     // (the mma above have consumed every ldmatrix result)
@@ -317,16 +323,24 @@ k_attn_tc_bf16(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (++st == n_stages) { st = 0; phase ^= 1u; }
     if (seg_end) {
       // this warp's state -> shared memory; the last warp to get here combines the eight states
-      float l_tot = l_run + __shfl_xor_sync(FULL, l_run, 1);
-      l_tot += __shfl_xor_sync(FULL, l_tot, 2);
+      float l_tot[2] = {l_run[0], l_run[1]};
+#pragma unroll
+      for (int ofs = 4; ofs < 32; ofs <<= 1) {
+        l_tot[0] += __shfl_xor_sync(FULL, l_tot[0], ofs);
+        l_tot[1] += __shfl_xor_sync(FULL, l_tot[1], ofs);
+      }
       float* so_b = so + (size_t)seg_buf * NW * grp * HD;
       float* sm_b = sm + seg_buf * NW * grp;
       float* sl_b = sl + seg_buf * NW * grp;
-      if (g < grp) {
-        float* dst = so_b + ((size_t)warp * grp + g) * HD + 2 * t4;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) *reinterpret_cast<float2*>(dst + 8 * j) = make_float2(o[j][0], o[j][1]);
-        if (t4 == 0) { sm_b[warp * grp + g] = m_run; sl_b[warp * grp + g] = l_tot; }
+      for (int e = 0; e < 2; ++e) {
+        const int head = 2 * t4 + e;
+        if (head < grp) {
+          float* dst = so_b + ((size_t)warp * grp + head) * HD + g;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { dst[16 * j] = o[j][e]; dst[16 * j + 8] = o[j][2 + e]; }
+          if (g == 0) { sm_b[warp * grp + head] = m_run[e]; sl_b[warp * grp + head] = l_tot[e]; }
+        }
       }
       __syncwarp();
       int last = 0;
