@@ -144,6 +144,12 @@ __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
 __device__ __forceinline__ void ldsm_x2(uint32_t (&r)[2], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
 }
+// transposes an 8 x 8 matrix of 16-bit elements held one row per quad (lane (g, t): row g, columns 2t, 2t+1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -914,10 +920,11 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         w.g0 = acc + w.gk * nsplit;
       };
       // Head size 64 with chunks of 256 positions runs on the tensor cores: a warp owns 16 positions of the chunk and
-      // loads K and V straight into mma fragments.  The order of the summed index of a product is free, so the
-      // 64 dims of q.k are dealt to the k-steps such that lane (g, t) needs the 16-byte pieces t and t + 4 of row g
-      // of a K n-tile; in P.V the output column (n-tile j, column g) stands for dim 8 g + j, so the lane needs
-      // piece g of the four positions 2t, 2t+1, 8+2t, 9+2t (pairs of positions are interleaved with byte permutes).
+      // loads K and V straight into mma A fragments (positions, resp. dims, as rows; the heads of the group are the 8
+      // columns of B).  The order of the summed index of a product is free, so the 64 dims of q.k are dealt to the
+      // k-steps such that lane (g, t) needs the 16-byte pieces t and t + 4 of rows g and g + 8; in V^T P^T row g of
+      // m-tile j stands for dim 8g + 2j (row g + 8 for 8g + 2j + 1), so the lane needs piece g of the four positions
+      // 2t, 2t+1, 8+2t, 9+2t (pairs of positions are interleaved with byte permutes).
       const bool mma_path = (A.hd == 64) && (split_len == kPW * 16);
       const int gq = lane >> 2, t4 = lane & 3;
       auto issue_loads = [&](const Walk& w, uint4 (&kr)[4], uint4 (&vr)[4], bool want_k, bool want_v) {
@@ -1016,6 +1023,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           }
           if (mma_path) {
             // ---- per warp: scores, softmax, P V of its 16 positions for all heads of the group at once ----
+            // The cache tile is the A operand (16 positions, resp. 16 dims, as rows), the group's heads are the 8
+            // columns of B: scores^T = K q^T (4 mma), out^T = V^T P^T (8 mma with P as bf16 head + remainder).
             const int lim = min(cnt, fresh_lo - p_lo);
             uint32_t qa[4][2];
             {
@@ -1028,78 +1037,88 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
                 qa[kk][1] = gq < grp ? pack_bf16(y.x, y.y) : 0u;
               }
             }
-            float sc2[2][4];
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-              sc2[j][0] = sc2[j][1] = sc2[j][2] = sc2[j][3] = 0.0f;
-              const uint32_t kw[8] = {kreg[2 * j].x, kreg[2 * j].y, kreg[2 * j].z, kreg[2 * j].w,
-                                      kreg[2 * j + 1].x, kreg[2 * j + 1].y, kreg[2 * j + 1].z, kreg[2 * j + 1].w};
-#pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                const uint32_t af[4] = {qa[kk][0], 0u, qa[kk][1], 0u}, bfr[2] = {kw[2 * kk], kw[2 * kk + 1]};
-                mma_bf16(sc2[j], af, bfr);
-              }
+            // entries 0, 1: position g, heads 2t, 2t+1; entries 2, 3: position g + 8
+            float sc[2][4];
+            sc[0][0] = sc[0][1] = sc[0][2] = sc[0][3] = 0.0f;
+            sc[1][0] = sc[1][1] = sc[1][2] = sc[1][3] = 0.0f;
+            {
+              const uint32_t a0[4] = {kreg[0].x, kreg[2].x, kreg[0].y, kreg[2].y}, a1[4] = {kreg[0].z, kreg[2].z, kreg[0].w, kreg[2].w};
+              const uint32_t a2[4] = {kreg[1].x, kreg[3].x, kreg[1].y, kreg[3].y}, a3[4] = {kreg[1].z, kreg[3].z, kreg[1].w, kreg[3].w};
+              mma_bf16(sc[0], a0, qa[0]); mma_bf16(sc[1], a1, qa[1]);
+              mma_bf16(sc[0], a2, qa[2]); mma_bf16(sc[1], a3, qa[3]);
             }
             if (have_next) issue_loads(nxt, kreg, vreg, true, false);   // K registers are free
-            float mx = -INFINITY;
+            float sv[4], mxe[2];
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
+            for (int e = 0; e < 4; ++e)
+              sv[e] = (warp * 16 + (e >> 1) * 8 + gq < lim) ? (sc[0][e] + sc[1][e]) * A.attn_scale : -INFINITY;
+            mxe[0] = fmaxf(sv[0], sv[2]); mxe[1] = fmaxf(sv[1], sv[3]);
 #pragma unroll
-              for (int e = 0; e < 2; ++e) {
-                sc2[j][e] = (warp * 16 + j * 8 + 2 * t4 + e < lim) ? sc2[j][e] * A.attn_scale : -INFINITY;
-                mx = fmaxf(mx, sc2[j][e]);
-              }
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            float pw[2][2], sum = 0.0f;
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-#pragma unroll
-              for (int e = 0; e < 2; ++e) { pw[j][e] = (sc2[j][e] > -INFINITY) ? __expf(sc2[j][e] - mx) : 0.0f; sum += pw[j][e]; }
-            // the weights as a bf16 head and a bf16 remainder: two products, fp32 sums
-            uint32_t ph[4] = {0u, 0u, 0u, 0u}, pl[4] = {0u, 0u, 0u, 0u};
-            {
-              const float h00 = round_bf16(pw[0][0]), h01 = round_bf16(pw[0][1]), h10 = round_bf16(pw[1][0]), h11 = round_bf16(pw[1][1]);
-              ph[0] = pack_bf16(h00, h01); pl[0] = pack_bf16(pw[0][0] - h00, pw[0][1] - h01);
-              ph[2] = pack_bf16(h10, h11); pl[2] = pack_bf16(pw[1][0] - h10, pw[1][1] - h11);
+            for (int o = 4; o < 32; o <<= 1) {
+              mxe[0] = fmaxf(mxe[0], __shfl_xor_sync(0xffffffffu, mxe[0], o));
+              mxe[1] = fmaxf(mxe[1], __shfl_xor_sync(0xffffffffu, mxe[1], o));
             }
-            float oc[8][4];
+            float pw[4], sume[2];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) pw[e] = (sv[e] > -INFINITY) ? __expf(sv[e] - mxe[e & 1]) : 0.0f;
+            sume[0] = pw[0] + pw[2]; sume[1] = pw[1] + pw[3];
+            // the weights as a bf16 head and a bf16 remainder (two products, fp32 sums), moved from accumulator layout
+            // (positions as rows) to B-operand layout (positions as the summed index)
+            uint32_t ph[2], pl[2];
+            {
+              const float h0 = round_bf16(pw[0]), h1 = round_bf16(pw[1]), h2 = round_bf16(pw[2]), h3 = round_bf16(pw[3]);
+              ph[0] = movmatrix_trans(pack_bf16(h0, h1)); ph[1] = movmatrix_trans(pack_bf16(h2, h3));
+              pl[0] = movmatrix_trans(pack_bf16(pw[0] - h0, pw[1] - h1)); pl[1] = movmatrix_trans(pack_bf16(pw[2] - h2, pw[3] - h3));
+            }
+            // out^T: m-tile j, row g = dim 8g + 2j, row g + 8 = dim 8g + 2j + 1 (the lane holds piece g of its four positions)
+            float oc[4][4];
             {
               const uint32_t va[4] = {vreg[0].x, vreg[0].y, vreg[0].z, vreg[0].w}, vb[4] = {vreg[1].x, vreg[1].y, vreg[1].z, vreg[1].w};
               const uint32_t vc2[4] = {vreg[2].x, vreg[2].y, vreg[2].z, vreg[2].w}, vd[4] = {vreg[3].x, vreg[3].y, vreg[3].z, vreg[3].w};
 #pragma unroll
-              for (int jn = 0; jn < 8; ++jn) {
-                oc[jn][0] = oc[jn][1] = oc[jn][2] = oc[jn][3] = 0.0f;
-                const unsigned sel = (jn & 1) ? 0x7632u : 0x5410u;
-                const uint32_t bfr[2] = {__byte_perm(va[jn >> 1], vb[jn >> 1], sel), __byte_perm(vc2[jn >> 1], vd[jn >> 1], sel)};
-                mma_bf16(oc[jn], ph, bfr);
-                mma_bf16(oc[jn], pl, bfr);
+              for (int j = 0; j < 4; ++j) {
+                oc[j][0] = oc[j][1] = oc[j][2] = oc[j][3] = 0.0f;
+                const uint32_t af[4] = {__byte_perm(va[j], vb[j], 0x5410u), __byte_perm(va[j], vb[j], 0x7632u),
+                                        __byte_perm(vc2[j], vd[j], 0x5410u), __byte_perm(vc2[j], vd[j], 0x7632u)};
+                mma_bf16(oc[j], af, ph);
+                mma_bf16(oc[j], af, pl);
               }
             }
             if (have_next) issue_loads(nxt, kreg, vreg, false, true);   // ... and the V registers
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            if (gq < grp) {
-              // accumulate into the warp's running state of this segment: lane t of the quad holds dims 16t .. 16t+15
-              float* so_w = s_o + ((size_t)warp * grp + gq) * 64 + 16 * t4;
-              float m_old = -INFINITY, l_old = 0.0f;
-              if (!seg_start) { m_old = S.red[warp][gq]; l_old = S.red2[warp][gq]; }
-              const float M = fmaxf(m_old, mx);
-              const float f_old = (m_old > -INFINITY) ? __expf(m_old - M) : 0.0f;
-              const float f_new = (mx > -INFINITY) ? __expf(mx - M) : 0.0f;
 #pragma unroll
-              for (int hf = 0; hf < 2; ++hf)
+            for (int o = 4; o < 32; o <<= 1) {
+              sume[0] += __shfl_xor_sync(0xffffffffu, sume[0], o);
+              sume[1] += __shfl_xor_sync(0xffffffffu, sume[1], o);
+            }
+            // accumulate into the warp's running state of this segment: the lane holds dims 8g .. 8g+7 of heads 2t, 2t+1
+            float m_new[2] = {0.0f, 0.0f}, l_new[2] = {0.0f, 0.0f};
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int head = 2 * t4 + e;
+              if (head < grp) {
+                float* so_w = s_o + ((size_t)warp * grp + head) * 64 + 8 * gq;
+                float m_old = -INFINITY, l_old = 0.0f;
+                if (!seg_start) { m_old = S.red[warp][head]; l_old = S.red2[warp][head]; }
+                const float M = fmaxf(m_old, mxe[e]);
+                const float f_old = (m_old > -INFINITY) ? __expf(m_old - M) : 0.0f;
+                const float f_new = (mxe[e] > -INFINITY) ? __expf(mxe[e] - M) : 0.0f;
 #pragma unroll
                 for (int q4 = 0; q4 < 2; ++q4) {
                   float4 c4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                  float4* pp = reinterpret_cast<float4*>(so_w + 8 * hf + 4 * q4);
+                  float4* pp = reinterpret_cast<float4*>(so_w + 4 * q4);
                   if (!seg_start) { c4 = *pp; c4.x *= f_old; c4.y *= f_old; c4.z *= f_old; c4.w *= f_old; }
-                  c4.x = fmaf(oc[4 * q4 + 0][hf], f_new, c4.x); c4.y = fmaf(oc[4 * q4 + 1][hf], f_new, c4.y);
-                  c4.z = fmaf(oc[4 * q4 + 2][hf], f_new, c4.z); c4.w = fmaf(oc[4 * q4 + 3][hf], f_new, c4.w);
+                  c4.x = fmaf(oc[2 * q4][e], f_new, c4.x); c4.y = fmaf(oc[2 * q4][2 + e], f_new, c4.y);
+                  c4.z = fmaf(oc[2 * q4 + 1][e], f_new, c4.z); c4.w = fmaf(oc[2 * q4 + 1][2 + e], f_new, c4.w);
                   *pp = c4;
                 }
-              __syncwarp(__activemask());
-              if (t4 == 0) { S.red[warp][gq] = M; S.red2[warp][gq] = l_old * f_old + sum * f_new; }
+                m_new[e] = M; l_new[e] = l_old * f_old + sume[e] * f_new;
+              }
+            }
+            __syncwarp();                                  // every lane has read the old maxima and sums
+            if (gq == 0) {
+#pragma unroll
+              for (int e = 0; e < 2; ++e)
+                if (2 * t4 + e < grp) { S.red[warp][2 * t4 + e] = m_new[e]; S.red2[warp][2 * t4 + e] = l_new[e]; }
             }
             __syncwarp();
           } else
