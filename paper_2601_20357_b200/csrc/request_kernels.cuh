@@ -90,6 +90,7 @@ struct ReqShared {
   int bc_tok[kReqMaxWidth];
   int ok[kReqMaxRows];
   int result;
+  float par[3][kMaxInputs];                        // per-row scalars of a pass (maximum, normaliser, weight)
 };
 
 // Row maxima of `rows` rows (row i at base + i * pitch) over this CTA's slice, gathered over the cluster:
@@ -99,7 +100,7 @@ __device__ __forceinline__ void req_row_maxima(cg::cluster_group& cluster, const
 #pragma unroll 1
   for (int i0 = 0; i0 < rows; i0 += 4) {
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 4
+#pragma unroll 1
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float x[4][4];
 #pragma unroll
@@ -139,7 +140,7 @@ __device__ __forceinline__ void req_row_sums(cg::cluster_group& cluster, const R
     float mx[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) mx[j] = (i0 + j < rows) ? req_max_of(c, S, i0 + j) : 0.0f;
-#pragma unroll 4
+#pragma unroll 1
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float x[2][4];
 #pragma unroll
@@ -323,13 +324,14 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
   const bool vec = req_vec_ok(A.logits, V);
   req_row_maxima(cluster, c, S, lg, V, m, vec);
   req_row_sums(cluster, c, S, lg, V, m, vec);
-  float mx[kMaxInputs], sn[kMaxInputs], wk[kMaxInputs];
-#pragma unroll
-  for (int k = 0; k < kMaxInputs; ++k) {
-    mx[k] = k < m ? req_max_of(c, S, k) : 0.0f;
-    sn[k] = k < m ? req_norm_of(c, S, k) : 1.0f;
-    wk[k] = k < m ? A.w[b * m + k] : 0.0f;
+  // (the loop over the inputs below is a real loop - the kernel's code runs once per CTA, so its size is what
+  // the instruction fetch pays for - hence the rows' scalars sit in shared memory, not in registers)
+  if (c.tid < m) {
+    S.par[0][c.tid] = req_max_of(c, S, c.tid);
+    S.par[1][c.tid] = req_norm_of(c, S, c.tid);
+    S.par[2][c.tid] = A.w[b * m + c.tid];
   }
+  __syncthreads();
   float* q_row = A.q_out + (long long)b * A.q_req_stride;
   float* qk_b = A.qk_out ? A.qk_out + (long long)b * A.qk_req_stride : nullptr;
   const bool vec_q = req_vec_ok(A.q_out, A.q_req_stride) && (V & 3) == 0;
@@ -341,17 +343,17 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
     float acc[4];
     float nxt[4];
     req_ld4(lg, v, c.v_hi, vec, -INFINITY, nxt);
-#pragma unroll
-    for (int k = 0; k < kMaxInputs; ++k) {
-      if (k >= m) break;
+#pragma unroll 1
+    for (int k = 0; k < m; ++k) {
       float a[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) a[j] = nxt[j];
       if (k + 1 < m) req_ld4(lg + (long long)(k + 1) * V, v, c.v_hi, vec, -INFINITY, nxt);
+      const float mxk = S.par[0][k], snk = S.par[1][k], wkk = S.par[2][k];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx[k])), sn[k]);
-        const float t = __fmul_rn(wk[k], a[j]);
+        a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mxk)), snk);
+        const float t = __fmul_rn(wkk, a[j]);
         acc[j] = (k == 0) ? t : __fadd_rn(acc[j], t);
       }
       if (qk_b) req_st4(qk_b + (long long)k * V, v, c.v_hi, vec_qk, a);
@@ -377,7 +379,7 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
         // most likely token among those not chosen yet (the slice was written by this CTA: L1/L2 hold it)
         best = ReqBest{-1.0f, 0x7fffffff};
         __syncthreads();
-#pragma unroll 2
+#pragma unroll 1
         for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
           float x[4];
           req_ld4_rw(q_row, v, c.v_hi, vec_q, -1.0f, x);
@@ -417,7 +419,7 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
   __syncthreads();
   int t_lo, t_hi;
   req_thread_range(c, A.slice, &t_lo, &t_hi);
-#pragma unroll 4
+#pragma unroll 1
   for (int v = t_lo; v < t_hi; v += 4) {
     float x[4];
     req_ld4_rw(q_row, v, t_hi, vec_q, 0.0f, x);
@@ -497,7 +499,12 @@ struct VerifyArgs {
   int* ticket;                                  // [B] scratch, zero between launches
   int *n_accept, *out_n_accept, *next_token, *out_next_token;
   int* err;
+  int tail_inline;                              // 1: the request's last cluster runs the tail; 0: k_verify_tail does (a launch of
+                                                // its own with one LARGE cluster per request - with many requests the clusters
+                                                // of this kernel are small and the tail would crawl through a row on 1-2 CTAs)
 };
+
+__device__ __forceinline__ void verify_tail(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, const VerifyArgs& A, int b);
 
 __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs A) {
   pdl_trigger();
@@ -518,7 +525,7 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
   {
     // p_i = e / S; in greedy mode also its argmax
     ReqBest best{-1.0f, 0x7fffffff};
-#pragma unroll 4
+#pragma unroll 1
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float a[4];
       req_ld4(lg, v, c.v_hi, vec, -INFINITY, a);
@@ -543,9 +550,27 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
     } else flag = 1;
     A.row_flag[b * rows + i] = flag;
   }
+  if (!A.tail_inline) return;
   if (!req_last_of_request(cluster, c, &s_last, A.ticket + b, rows)) return;
+  verify_tail(cluster, c, S, A, b);
+}
 
-  // ---- the request's last cluster: acceptance prefix, siblings of the first rejected depth, next token --------
+// The tail alone: one cluster per request, after k_verify_req (tail_inline = 0) has stored p and the row flags.
+__global__ void __launch_bounds__(kReqThreads, 2) k_verify_tail(const VerifyArgs A) {
+  pdl_trigger();
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ ReqShared S;
+  const ReqCtx c = req_ctx(cluster, A.V, A.slice);
+  pdl_wait();
+  verify_tail(cluster, c, S, A, (int)(blockIdx.x / c.CS));
+}
+
+// ---- per request: acceptance prefix, siblings of the first rejected depth, next token (Sec. 3 item 3; Sec. 5 token tree) ----
+__device__ __forceinline__ void verify_tail(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, const VerifyArgs& A, int b) {
+  const int G = A.G, V = A.V, rows = G + 1, D = A.D, Rt = G + 1 + G * (D - 1);
+  float* p_b = A.p + (long long)b * Rt * V;
+  const float* q_b = A.q + (long long)b * A.q_req_stride;
+  const bool vec = req_vec_ok(A.logits, V), vec_p = (V & 3) == 0;
   int a = 0;
   for (; a < G; ++a) {
     const int f = __ldcg(A.row_flag + b * rows + a);
@@ -565,7 +590,7 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
     const float mx2 = req_max_of(c, S, 0), sn2 = req_norm_of(c, S, 0);
     unsigned long long mass = 0;
     ReqBest best{-1.0f, 0x7fffffff};
-#pragma unroll 2
+#pragma unroll 1
     for (int v = t_lo; v < t_hi; v += 4) {
       float x[4];
       req_ld4(lr, v, t_hi, vec, -INFINITY, x);
@@ -620,7 +645,7 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
     while (true) {
       // this level's residual masses (per thread range) and the mass of q_level
       unsigned long long mr = 0, mq = 0;
-#pragma unroll 4
+#pragma unroll 1
       for (int v = t_lo; v < t_hi; ++v) {
         float pl, ql;
         elem(v, level, pl, ql);
@@ -665,7 +690,7 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
     // every primary accepted: bonus token from p_G
     const float* p_g = p_b + (long long)G * V;
     unsigned long long mass = 0;
-#pragma unroll 4
+#pragma unroll 1
     for (int v = t_lo; v < t_hi; v += 4) {
       float x[4];
       if (vec_p && v + 4 <= t_hi) { const float4 t = __ldcg(reinterpret_cast<const float4*>(p_g + v)); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
@@ -715,7 +740,7 @@ struct UpdShared {
 
 __device__ __forceinline__ void policy_commit(const PolicyArgs& A, int b, int lane, int last);
 
-__global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs A) {
+__global__ void __launch_bounds__(kReqThreads, 2) k_update_req(const UpdateArgs A) {
   pdl_trigger();
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ UpdShared U;
@@ -729,57 +754,54 @@ __global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs 
   const int last = min(a, G - 1);
   if (i > last) return;                             // (the whole cluster: position not verified)
   const bool vec = (V & 3) == 0;
+  // The loops over the deviation index (drafter or grid candidate) are real loops with the accumulators in local
+  // memory: the kernel's code runs once per CTA, so its size is what the instruction fetch pays for.
+  const float* qbase = A.qk + ((long long)b * G + i) * m * V;
   if (A.hard) {
     // most likely token (lowest id on ties) of every grid candidate's ensemble, or of every drafter
-    const float* qbase = A.qk + ((long long)b * G + i) * m * V;
     ReqBest best[kMaxDev];
-#pragma unroll
-    for (int kd = 0; kd < kMaxDev; ++kd) best[kd] = ReqBest{-1.0f, 0x7fffffff};
+#pragma unroll 1
+    for (int kd = 0; kd < n_dev; ++kd) best[kd] = ReqBest{-1.0f, 0x7fffffff};
 #pragma unroll 1
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
+      float q0[4], q1[4];
       if (A.grid_policy) {
-        float q0[4], q1[4];
         req_ld4(qbase, v, c.v_hi, vec, 0.0f, q0);
         req_ld4(qbase + V, v, c.v_hi, vec, 0.0f, q1);
-#pragma unroll
-        for (int jc = 0; jc < kGridCand; ++jc) {
-          const float c1 = __fdiv_rn((float)jc, 10.0f);
+      }
+#pragma unroll 1
+      for (int kd = 0; kd < n_dev; ++kd) {
+        float x[4];
+        if (A.grid_policy) {
+          const float c1 = __fdiv_rn((float)kd, 10.0f);
           const float c0 = __fsub_rn(1.0f, c1);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float mix = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
-            if (v + j < c.v_hi && mix > best[jc].val) { best[jc].val = mix; best[jc].idx = v + j; }
-          }
+          for (int j = 0; j < 4; ++j) x[j] = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
+        } else {
+          req_ld4(qbase + (long long)kd * V, v, c.v_hi, vec, 0.0f, x);
         }
-      } else {
+        ReqBest t = best[kd];
 #pragma unroll
-        for (int k = 0; k < kMaxInputs; ++k) {
-          if (k >= m) break;
-          float qv[4];
-          req_ld4(qbase + (long long)k * V, v, c.v_hi, vec, 0.0f, qv);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) if (v + j < c.v_hi && qv[j] > best[k].val) { best[k].val = qv[j]; best[k].idx = v + j; }
-        }
+        for (int j = 0; j < 4; ++j) if (v + j < c.v_hi && x[j] > t.val) { t.val = x[j]; t.idx = v + j; }
+        best[kd] = t;
       }
     }
+#pragma unroll 1
+    for (int kd = 0; kd < n_dev; ++kd) {
+      ReqBest mine = best[kd];
 #pragma unroll
-    for (int kd = 0; kd < kMaxDev; ++kd) {
-      if (kd < n_dev) {
-        ReqBest mine = best[kd];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          ReqBest other;
-          other.val = __shfl_xor_sync(0xffffffffu, mine.val, o);
-          other.idx = __shfl_xor_sync(0xffffffffu, mine.idx, o);
-          best_merge(mine, other);
-        }
-        if (c.lane == 0) U.red_b[c.warp][kd] = mine;
+      for (int o = 16; o > 0; o >>= 1) {
+        ReqBest other;
+        other.val = __shfl_xor_sync(0xffffffffu, mine.val, o);
+        other.idx = __shfl_xor_sync(0xffffffffu, mine.idx, o);
+        best_merge(mine, other);
       }
+      if (c.lane == 0) U.red_b[c.warp][kd] = mine;
     }
     __syncthreads();
     if (c.tid < n_dev) {
       ReqBest t = U.red_b[0][c.tid];
-#pragma unroll
+#pragma unroll 1
       for (int w = 1; w < kReqWarps; ++w) best_merge(t, U.red_b[w][c.tid]);
       cluster.map_shared_rank(&U.all_b[0][0], 0)[c.rank * kMaxDev + c.tid] = t;
     }
@@ -795,74 +817,57 @@ __global__ void __launch_bounds__(kReqThreads, 1) k_update_req(const UpdateArgs 
     }
   } else {
     const float* p_i = A.p + ((long long)b * A.Rt + i) * V;
-    const float* qbase = A.qk + ((long long)b * G + i) * m * V;
     long long acc[kMaxDev];
-#pragma unroll
-    for (int kd = 0; kd < kMaxDev; ++kd) acc[kd] = 0;
+#pragma unroll 1
+    for (int kd = 0; kd < n_dev; ++kd) acc[kd] = 0;
 #pragma unroll 1
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
-      float pv[4], lp[4];
+      float pv[4], lp[4], q0[4], q1[4], nxt[4];
       req_ld4(p_i, v, c.v_hi, vec, 0.0f, pv);
-      if (!A.grid_policy) {
-        float qv[kMaxInputs][4];
-#pragma unroll
-        for (int k = 0; k < kMaxInputs; ++k)
-          if (k < m) req_ld4(qbase + (long long)k * V, v, c.v_hi, vec, 0.0f, qv[k]);
-        if (!tvd) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
-        }
-#pragma unroll
-        for (int k = 0; k < kMaxInputs; ++k) {
-          if (k >= m) break;
-          long long s = 0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (v + j >= c.v_hi) continue;
-            float t;
-            if (tvd) t = fabsf(__fsub_rn(pv[j], qv[k][j]));
-            else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(qv[k][j], kFltMin)))) : 0.0f;
-            s += __float2ll_rz(__fmul_rn(t, kMassScale));
-          }
-          acc[k] += s;
-        }
-      } else {
-        float q0[4], q1[4];
+      if (A.grid_policy) {
         req_ld4(qbase, v, c.v_hi, vec, 0.0f, q0);
         req_ld4(qbase + V, v, c.v_hi, vec, 0.0f, q1);
-        if (!tvd) {
+      } else {
+        req_ld4(qbase, v, c.v_hi, vec, 0.0f, nxt);
+      }
+      if (!tvd) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
-        }
-#pragma unroll
-        for (int jc = 0; jc < kGridCand; ++jc) {
-          const float c1 = __fdiv_rn((float)jc, 10.0f);
+        for (int j = 0; j < 4; ++j) lp[j] = xlog(fmaxf(pv[j], kFltMin));
+      }
+#pragma unroll 1
+      for (int kd = 0; kd < n_dev; ++kd) {
+        float x[4];
+        if (A.grid_policy) {
+          const float c1 = __fdiv_rn((float)kd, 10.0f);
           const float c0 = __fsub_rn(1.0f, c1);
-          long long s = 0;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (v + j >= c.v_hi) continue;
-            const float mix = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
-            float t;
-            if (tvd) t = fabsf(__fsub_rn(pv[j], mix));
-            else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(mix, kFltMin)))) : 0.0f;
-            s += __float2ll_rz(__fmul_rn(t, kMassScale));
-          }
-          acc[jc] += s;
+          for (int j = 0; j < 4; ++j) x[j] = __fadd_rn(__fmul_rn(c0, q0[j]), __fmul_rn(c1, q1[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) x[j] = nxt[j];
+          if (kd + 1 < n_dev) req_ld4(qbase + (long long)(kd + 1) * V, v, c.v_hi, vec, 0.0f, nxt);      // the next row while this one is worked on
         }
+        long long sum = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (v + j >= c.v_hi) continue;
+          float t;
+          if (tvd) t = fabsf(__fsub_rn(pv[j], x[j]));
+          else t = (pv[j] > 0.0f) ? __fmul_rn(pv[j], __fsub_rn(lp[j], xlog(fmaxf(x[j], kFltMin)))) : 0.0f;
+          sum += __float2ll_rz(__fmul_rn(t, kMassScale));
+        }
+        acc[kd] += sum;
       }
     }
-#pragma unroll
-    for (int kd = 0; kd < kMaxDev; ++kd) {
-      if (kd < n_dev) {
-        const long long t = warp_sum_i64(acc[kd]);
-        if (c.lane == 0) U.red[c.warp][kd] = t;
-      }
+#pragma unroll 1
+    for (int kd = 0; kd < n_dev; ++kd) {
+      const long long t = warp_sum_i64(acc[kd]);
+      if (c.lane == 0) U.red[c.warp][kd] = t;
     }
     __syncthreads();
     if (c.tid < n_dev) {
       long long t = 0;
-#pragma unroll
+#pragma unroll 1
       for (int w = 0; w < kReqWarps; ++w) t += U.red[w][c.tid];
       cluster.map_shared_rank(&U.all_dev[0][0], 0)[c.rank * kMaxDev + c.tid] = t;
     }

@@ -818,6 +818,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
     h->cs_max = 8;
     if (cudaFuncSetAttribute(k_ensemble_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
         cudaFuncSetAttribute(k_verify_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+        cudaFuncSetAttribute(k_verify_tail, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
         cudaFuncSetAttribute(k_update_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
       cudaLaunchConfig_t lc = {};
       lc.gridDim = dim3(kReqMaxCluster); lc.blockDim = dim3(kReqThreads);
@@ -827,7 +828,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
       lc.attrs = at; lc.numAttrs = 1;
       int n16 = 0;
       bool ok = true;
-      for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_update_req})
+      for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_verify_tail, (const void*)k_update_req})
         ok = ok && cudaOccupancyMaxActiveClusters(&n16, fn, &lc) == cudaSuccess && n16 >= 1;
       if (ok) h->cs_max = kReqMaxCluster;
       // how many clusters of each size fit at once (the most demanding of the three kernels): a launch is sized for one wave
@@ -836,7 +837,7 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
         if (cs > h->cs_max) break;
         lc.gridDim = dim3(cs); at[0].val.clusterDim.x = cs;
         int best = 1 << 30;
-        for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_update_req}) {
+        for (const void* fn : {(const void*)k_ensemble_req, (const void*)k_verify_req, (const void*)k_verify_tail, (const void*)k_update_req}) {
           int n = 0;
           if (cudaOccupancyMaxActiveClusters(&n, fn, &lc) != cudaSuccess) n = 0;
           best = std::min(best, n);
@@ -1142,7 +1143,16 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   a.n_accept = h->n_accept; a.out_n_accept = out_n_accept == h->n_accept ? nullptr : out_n_accept;
   a.next_token = h->next_token; a.out_next_token = out_next_token == h->next_token ? nullptr : out_next_token;
   a.err = h->err;
+  // With many requests the per-row clusters are small; the tail (one row-wide pass after the other) then runs as a
+  // launch of its own with one cluster per request, as large as the budget allows.
+  int slice_tail = 0;
+  const int cs_tail = pick_cluster(h, h->B, &slice_tail);
+  a.tail_inline = cs_tail >= 4 * cs ? 0 : 1;
   launch_request_clusters(h, k_verify_req, h->B * (h->G + 1), cs, a);
+  if (!a.tail_inline) {
+    a.slice = slice_tail;
+    launch_request_clusters(h, k_verify_tail, h->B, cs_tail, a);
+  }
   h->phase = PH_VERIFIED;
   return check_cuda();
 }
