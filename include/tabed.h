@@ -250,6 +250,9 @@ int tabed_set_policy_uniforms(tabed_handle* h, const float* u_policy);
 /* Host-buffer round: tabed_draft_round -> tabed_verify -> tabed_update_weights with HOST pointers
  * (pageable or pinned) for every argument, same shapes as above.  Copies the inputs to the
  * device, runs the round, copies the results back and synchronises the stream before returning.
+ * The target's logits (the bulk of the input) are copied on a stream of the library's own while the
+ * drafting runs on config.stream; that copy starts after all earlier work on config.stream and the
+ * verification waits for it, so the caller sees the ordering of a single stream.
  * out_w and out_w_argmax may be NULL. */
 int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accept,
                      const float* u_resid, const float* target_logits, int32_t* out_tokens,

@@ -116,6 +116,11 @@ struct tabed_handle {
   // per-kernel-class timing (tabed_profile_begin / tabed_profile_end)
   int prof_class = -1;
   std::vector<cudaEvent_t> prof_events;     // start/stop pairs
+  // tabed_round_host: the target's logits (by far the largest input) travel on a stream of the library's own while
+  // the drafting runs on the caller's; the two events order that copy after the caller's earlier work and before
+  // the verification
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_round_begin = nullptr, ev_target_ready = nullptr;
   size_t prof_used = 0;
 };
 
@@ -860,6 +865,10 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
   A(&h->chunk_mass, B * h->n_chunks); A(&h->chunk_best, B * h->n_chunks);
   A(&h->err, 1);
   A(&h->st_u_draft, B * G * Dw); A(&h->st_u_accept, B * G * Dw); A(&h->st_u_resid, B); A(&h->st_target, B * Rt * V); A(&h->st_tokens, B * G * Dw);
+  if (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) != cudaSuccess) h->copy_stream = nullptr;
+  if (cudaEventCreateWithFlags(&h->ev_round_begin, cudaEventDisableTiming) != cudaSuccess) h->ev_round_begin = nullptr;
+  if (cudaEventCreateWithFlags(&h->ev_target_ready, cudaEventDisableTiming) != cudaSuccess) h->ev_target_ready = nullptr;
+  cudaGetLastError();                               // (without them tabed_round_host copies on the caller's stream)
   if (h->has_drafter) {
     h->L = c.n_layers; h->d = c.d_model; h->F = c.d_ffn; h->H = c.n_heads; h->Hkv = c.n_kv_heads;
     h->hd = c.d_model / c.n_heads; h->cap = c.kv_capacity; h->esz = c.dtype == TABED_DTYPE_FP32 ? 4 : 2;
@@ -958,6 +967,9 @@ void tabed_destroy(tabed_handle* h) {
   cudaStreamSynchronize(h->stream);
   for (void* ptr : h->allocs) cudaFree(ptr);
   for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+  if (h->copy_stream) { cudaStreamSynchronize(h->copy_stream); cudaStreamDestroy(h->copy_stream); }
+  if (h->ev_round_begin) cudaEventDestroy(h->ev_round_begin);
+  if (h->ev_target_ready) cudaEventDestroy(h->ev_target_ready);
   cudaGetLastError();
   delete h;
 }
@@ -1201,16 +1213,27 @@ int tabed_round_host(tabed_handle* h, const float* u_draft, const float* u_accep
   DeviceGuard guard(h->cfg.device);
   const size_t BG = (size_t)h->B * h->G * h->D;
   cudaStream_t st = h->stream;
+  const size_t target_bytes = (size_t)h->B * h->Rt * h->V * 4;
   if (cudaMemcpyAsync(h->st_u_draft, u_draft, BG * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(h->st_u_accept, u_accept, BG * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(h->st_u_resid, u_resid, (size_t)h->B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(h->st_target, target_logits, (size_t)h->B * h->Rt * h->V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      cudaMemcpyAsync(h->st_u_resid, u_resid, (size_t)h->B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return TABED_ERR_CUDA;
+  const bool side = h->copy_stream && h->ev_round_begin && h->ev_target_ready;
+  if (side) {
+    // after everything the caller's stream holds so far (the staging buffer's last reader among it), beside the drafting
+    if (cudaEventRecord(h->ev_round_begin, st) != cudaSuccess || cudaStreamWaitEvent(h->copy_stream, h->ev_round_begin, 0) != cudaSuccess ||
+        cudaMemcpyAsync(h->st_target, target_logits, target_bytes, cudaMemcpyHostToDevice, h->copy_stream) != cudaSuccess ||
+        cudaEventRecord(h->ev_target_ready, h->copy_stream) != cudaSuccess)
+      return TABED_ERR_CUDA;
+  } else if (cudaMemcpyAsync(h->st_target, target_logits, target_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    return TABED_ERR_CUDA;
+  }
   const std::vector<int> len_before = h->len_ub, cnt_before = h->pend_cnt;
   const bool known_before = h->pend_known;
   // outputs land in library buffers first (tokens / n_accept / next_token / w / w_argmax)
   int rc = tabed_draft_round(h, h->st_u_draft, h->st_tokens, nullptr);
-  if (rc != TABED_OK) return rc;
+  if (rc != TABED_OK) { if (side) cudaStreamSynchronize(h->copy_stream); return rc; }
+  if (side && cudaStreamWaitEvent(st, h->ev_target_ready, 0) != cudaSuccess) return TABED_ERR_CUDA;
   rc = tabed_verify(h, h->st_target, h->st_u_accept, h->st_u_resid, h->n_accept, h->next_token);
   if (rc != TABED_OK) return rc;
   rc = tabed_update_weights(h, nullptr, h->w_argmax);
