@@ -29,6 +29,7 @@ namespace tabed {
 constexpr int kTcM = 128;          // weight rows per tile (MMA M)
 constexpr int kTcKC = 128;         // input columns per pipeline stage
 constexpr int kTcStages = 3;        // pipeline stages (2 when more than 128 slots share the shared memory)
+constexpr int kTcMaxStages = 8;
 constexpr int kTcThreads = 128;
 constexpr int kPrefillChunk = 256;        // positions of one row prefilled as slots of one weight pass
 constexpr int kTcMaxN = 256;       // slots per launch (MMA N is their count rounded up to 16)
@@ -50,6 +51,9 @@ struct TcGemmArgs {
   int k_chunks;                    // chunks of 128 columns over the whole input dimension
   int ks;                          // k-splits; unit (m_tile, split) covers chunks [split*cps, min((split+1)*cps, k_chunks))
   int cps;                         // chunks per split
+  int kc;                          // input columns per pipeline stage: 128 (a whole block) or 64 (half a block: a block's
+                                   // 16-byte column groups are its outer index, so half of it is contiguous too)
+  int n_stages;                    // pipeline stages, <= kTcMaxStages
   int* err;
 };
 
@@ -72,19 +76,21 @@ __device__ __forceinline__ bool tc_wait(uint64_t* bar, unsigned parity, int* err
 // grid (m_tiles * ks), block 128, dynamic shared memory kTcStages * (A block + B block) + 1 KB
 __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   extern __shared__ __align__(1024) unsigned char tc_smem[];
-  __shared__ uint64_t s_full[kTcStages], s_empty[kTcStages], s_done;
+  __shared__ uint64_t s_full[kTcMaxStages], s_empty[kTcMaxStages], s_done;
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   pdl_trigger();
   const int m_tile = blockIdx.x / G.ks, split = blockIdx.x - m_tile * G.ks;
-  const int c_lo = split * G.cps, c_hi = min(c_lo + G.cps, G.k_chunks), n_ch = c_hi - c_lo;
-  const size_t a_bytes = tc_block_bytes(kTcM), b_bytes = tc_block_bytes(G.n_pad);
-  const int n_stages = tc_stages(G.n_pad);
+  // the CTA's range of the input dimension in units of one stage (kc columns); a_bytes, b_bytes = one stage of each operand
+  const int per_chunk = kTcKC / G.kc;
+  const int c_lo = split * G.cps, c_hi = min(c_lo + G.cps, G.k_chunks), n_ch = (c_hi - c_lo) * per_chunk;
+  const size_t a_bytes = tc_block_bytes(kTcM) / per_chunk, b_bytes = tc_block_bytes(G.n_pad) / per_chunk;
+  const int n_stages = G.n_stages;
   const uint32_t tmem_cols = G.n_pad <= 32 ? 32u : (G.n_pad <= 64 ? 64u : (G.n_pad <= 128 ? 128u : 256u));
 
   if (tid == 0) {
-    for (int s = 0; s < kTcStages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
+    for (int s = 0; s < n_stages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
     mbar_init(&s_done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_bad = 0;
@@ -98,8 +104,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = s_tmem;
-  const unsigned char* a_src = G.a_packed + ((size_t)m_tile * G.k_chunks + c_lo) * a_bytes;
-  const unsigned char* b_src = G.b_packed + (size_t)c_lo * b_bytes;
+  const unsigned char* a_src = G.a_packed + ((size_t)m_tile * G.k_chunks + c_lo) * tc_block_bytes(kTcM);
+  const unsigned char* b_src = G.b_packed + (size_t)c_lo * tc_block_bytes(G.n_pad);
   const int pre = n_ch < n_stages ? n_ch : n_stages;
   // The weights do not depend on the kernels before this one: their first stages are requested before
   // the wait on those kernels (transaction bytes announced without an arrival, so a stage's barrier
@@ -151,7 +157,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
       const uint32_t b_s = a_s + (uint32_t)a_bytes;
       const uint32_t a_lbo = (kTcM / 8) * 128, b_lbo = (uint32_t)(G.n_pad / 8) * 128;
 #pragma unroll 1
-      for (int j = 0; j < kTcKC / 16; ++j) {
+      for (int j = 0; j < G.kc / 16; ++j) {
         const uint64_t da = tc_smem_desc(a_s + (uint32_t)j * 2u * a_lbo, a_lbo, 128u);
         const uint64_t db = tc_smem_desc(b_s + (uint32_t)j * 2u * b_lbo, b_lbo, 128u);
         const uint32_t acc = (c > 0 || j > 0) ? 1u : 0u;
