@@ -15,7 +15,7 @@
 //   needs no tensor map: the weights are re-laid once at set-up (k_pack_tc), the activations by the kernel
 //   that normalises and rounds them (k_prep_act).
 // * One thread issues the copies and the MMAs; tcgen05.commit releases a stage / signals the epilogue;
-//   four warps read the accumulator with tcgen05.ld (warp w owns TMEM lanes 32w..32w+31) and store
+//   eight warps read the accumulator with tcgen05.ld (warps w and w + 4 own TMEM lanes 32w..32w+31, half of the columns each) and store
 //   coalesced rows.  Every wait is bounded; on a timeout the CTA sets an error bit, drains and frees TMEM.
 #pragma once
 #include <cuda_bf16.h>
@@ -30,7 +30,7 @@ constexpr int kTcM = 128;          // weight rows per tile (MMA M)
 constexpr int kTcKC = 128;         // input columns per pipeline stage
 constexpr int kTcStages = 3;        // pipeline stages (2 when more than 128 slots share the shared memory)
 constexpr int kTcMaxStages = 8;
-constexpr int kTcThreads = 128;
+constexpr int kTcThreads = 256;      // eight warps: warps w and w + 4 read the same 32 accumulator lanes, half of the columns each
 constexpr int kPrefillChunk = 256;        // positions of one row prefilled as slots of one weight pass
 constexpr int kTcMaxN = 256;       // slots per launch (MMA N is their count rounded up to 16)
 __host__ __device__ inline int tc_stages(int n_pad) { return n_pad > 128 ? 2 : kTcStages; }
@@ -201,11 +201,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
   }
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   if (done_ok) {
-    const int row = m_tile * kTcM + warp * 32 + lane;
+    const int lq = warp & 3;                                        // the warp's quarter of the 128 accumulator lanes
+    const int row = m_tile * kTcM + lq * 32 + lane;
     float* out = G.partial + (size_t)split * G.slab + row;
+    // the warp's columns: the first or the second half of the groups of 16
+    const int n16 = G.n_pad >> 4, c_begin = (warp >> 2) ? ((n16 + 1) >> 1) << 4 : 0, c_end = (warp >> 2) ? G.n_pad : ((n16 + 1) >> 1) << 4;
     // two loads of 16 columns in flight: the next one is requested before the current one is stored
     auto ld16 = [&](uint32_t (&v)[16], int c0) {
-      const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+      const uint32_t taddr = tmem + ((uint32_t)(lq * 32) << 16) + (uint32_t)c0;
       asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
@@ -218,24 +221,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_gemm_tc(const TcGemmArgs G) {
           if (c0 + j < G.n_slots) out[(size_t)(c0 + j) * G.rows_total] = __uint_as_float(v[j]);
       }
     };
-    if (n_ch > 0) {
+    if (n_ch > 0 && c_begin < c_end) {
       uint32_t va[16], vb[16];
-      ld16(va, 0);
+      ld16(va, c_begin);
 #pragma unroll 1
-      for (int c0 = 0; c0 < G.n_pad; c0 += 32) {
+      for (int c0 = c_begin; c0 < c_end; c0 += 32) {
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        const bool more = c0 + 16 < G.n_pad;
+        const bool more = c0 + 16 < c_end;
         if (more) ld16(vb, c0 + 16);
         st16(va, c0);
         if (more) {
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          if (c0 + 32 < G.n_pad) ld16(va, c0 + 32);
+          if (c0 + 32 < c_end) ld16(va, c0 + 32);
           st16(vb, c0 + 16);
         }
       }
-    } else {
+    } else if (n_ch == 0) {
       if (row < G.rows_valid)
-        for (int c = 0; c < G.n_slots; ++c) out[(size_t)c * G.rows_total] = 0.0f;
+        for (int c = c_begin; c < min(c_end, G.n_slots); ++c) out[(size_t)c * G.rows_total] = 0.0f;
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
