@@ -123,13 +123,15 @@ extern "C" {
                                       projections if it qualifies, else per-operation                    */
 #define TABED_PATH_PER_OP      1   /* one kernel per operation (any drafter, any number of rows)        */
 #define TABED_PATH_PERSISTENT  2   /* the whole round in one cooperative kernel: bf16 drafter, tree_width 1,
-                                      2*B*m <= 8 slots, d_model <= 2048 (<= 1024 with more than 4 slots) and
+                                      B*m <= 8 rows (with more than 4 rows at least two layers: the first of
+                                      two pending tokens then gets a weight pass of its own), d_model <= 2048
+                                      (<= 1024 with more than 4 slots: 3 - 4 or 5 - 8 rows) and
                                       a multiple of 16, d_ffn a multiple of 16, H <= 64, (H/Hkv)*head_dim <= 512, <= 64 layers,
                                       kv_capacity <= 32768                                                */
 #define TABED_PATH_TENSOR_CORE 3   /* one kernel per operation with the projections as tcgen05 contractions
                                       over all rows: any bf16 drafter with d_model, d_ffn, H*head_dim
                                       multiples of 8 (the automatic choice when the persistent kernel
-                                      does not take the shape, i.e. more than 4 rows)                     */
+                                      does not take the shape, i.e. more than 8 rows)                     */
 
 typedef struct tabed_handle tabed_handle;   /* opaque, library-owned */
 

@@ -37,6 +37,10 @@
 //   * loops are deliberately not unrolled except the few hot ones: every phase runs its code once,
 //     so unrolling buys nothing and only inflates the instruction footprint.
 //
+// Rows: up to 4 rows feed both pending tokens of a fully accepted block in the first step's weight pass
+// (2 R <= 8 slots); with 5 - 8 rows the first of the two gets a pass of its own before step 0 (all layers,
+// no LM head, only the rows that have two pending tokens are active), so a pass never has more than 8 slots.
+//
 // Waits are bounded: a flagged word or a copy that does not arrive within the spin limit sets an
 // error bit, the CTA drains its copies in flight and returns.
 #pragma once
@@ -96,7 +100,9 @@ struct RoundArgs {
   uint2* mid;                           // [8][F/2] two bf16 values of the gated product per pair
   uint2 *part_o, *part_ml;              // attention partials [8][H][max_splits][hd], [..][2] (max, sum)
   int max_splits;
-  unsigned epoch0;                      // the launch's first epoch; phase p of step s stamps epoch0 + s * (5 L + 8) + p + 1
+  unsigned epoch0;                      // the launch's first epoch; phase p of pass i stamps epoch0 + i * (5 L + 8) + p + 1
+  int prepass;                          // more than kPSlots / 2 rows: a fully accepted block's first pending token is fed in a
+                                        // pass of its own (all layers, no LM head) before step 0, instead of as R more slots
   // ensemble
   float* logits_own;                    // [G][R][V]
   const float* logits_override;         // or null
@@ -232,8 +238,9 @@ __device__ __forceinline__ int unit_sub(uint32_t e) { return (int)((e >> 10) & 6
 __device__ __forceinline__ int unit_tile(uint32_t e) { return (int)(e >> 16); }
 
 // Issue the bulk copy of unit number k (counted over the whole round) into its ring slot (one thread).
-__device__ __forceinline__ void issue_unit(const RoundArgs& A, PShared& S, unsigned char* ring, unsigned k, unsigned per_step) {
-  const uint32_t e = S.ulist[k % per_step];
+// The stream of units is [the list without its LM-head units, if the round has the extra pass] then the whole list per step.
+__device__ __forceinline__ void issue_unit(const RoundArgs& A, PShared& S, unsigned char* ring, unsigned k, unsigned per_step, unsigned pre_units) {
+  const uint32_t e = S.ulist[k < pre_units ? k : (k - pre_units) % per_step];
   const int kind = e & 7, layer = (e >> 3) & 127, u = unit_tile(e) * A.geom[kind].nsub + unit_sub(e);
   const unsigned bytes = 16u * ((unsigned)A.geom[kind].kchunk * 2u + 16u);
   const unsigned char* src = A.packed + A.pack_off[kind] + (size_t)u * bytes +
@@ -472,10 +479,17 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   }
   __syncthreads();
   const unsigned per_step = S.pstart[n_phase];
-  const unsigned total_units = per_step * (unsigned)G;
+  // the extra pass: only in a round in which some request has two pending tokens (the same answer in every CTA)
+  int pre = 0;
+  if (A.prepass) {
+#pragma unroll 1
+    for (int b = 0; b < B; ++b) if (A.pending[b * 3] == 2) pre = 1;
+  }
+  const unsigned pre_units = pre ? S.pstart[n_phase - 1] : 0u;     // its units: every phase but the LM head
+  const unsigned total_units = pre_units + per_step * (unsigned)G;
   if (tid == 0) {
 #pragma unroll 1
-    for (unsigned k = 0; k < (unsigned)A.n_ring && k < total_units; ++k) issue_unit(A, S, ring, k, per_step);
+    for (unsigned k = 0; k < (unsigned)A.n_ring && k < total_units; ++k) issue_unit(A, S, ring, k, per_step, pre_units);
   }
   bool alive = true;
   const unsigned EPS = 5u * (unsigned)A.L + 8u;          // epochs per decoder step
@@ -501,8 +515,8 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
 #define PHASE_END()                                                        \
   do {                                                                     \
     TSEC(4);                                                               \
-    if (TRACE && tr_on && trace_n < A.trace_stride) {                      \
-      unsigned long long* rec = A.trace + ((size_t)step * A.trace_stride + trace_n++) * kTraceRec; \
+    if (TRACE && tr_on && step >= 0 && trace_n < A.trace_stride) {         \
+      unsigned long long* rec = A.trace + ((size_t)(step < 0 ? 0 : step) * A.trace_stride + trace_n++) * kTraceRec; \
       rec[0] = global_timer();                                             \
       for (int k = 0; k < 6; ++k) { rec[1 + k] = (unsigned long long)t_sec[k]; t_sec[k] = 0; }     \
     }                                                                      \
@@ -511,11 +525,13 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
   if (tr_on) t_mark = clock64();
 
 #pragma unroll 1
-  for (int step = 0; step < G; ++step) {
+  for (int it = 0; it < G + pre; ++it) {
+    const int step = it - pre;                          // -1: the extra pass
+    const unsigned ubase = step < 0 ? 0u : pre_units + (unsigned)step * per_step;    // first unit of this pass in the stream
     int trace_n = 0;
     // ---- slot table of the step ------------------------------------------------------------------
     int ns = R;
-    if (step == 0) {
+    if (step == 0 && !A.prepass) {
 #pragma unroll 1
       for (int b = 0; b < B; ++b) if (A.pending[b * 3] == 2) ns = 2 * R;
     }
@@ -525,7 +541,15 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         const int row = tid % R, b = row / m, second = tid >= R;
         const int* pend = A.pending + b * 3;
         sl.row = row;
-        if (step == 0) {
+        if (step < 0) {                                 // the first of two pending tokens, for the rows that have two
+          sl.pos = A.kv_len[row];
+          sl.tok = pend[1];
+          sl.active = pend[0] == 2;
+        } else if (step == 0 && A.prepass) {            // the last pending token
+          sl.pos = A.kv_len[row] + pend[0] - 1;
+          sl.tok = pend[pend[0]];
+          sl.active = 1;
+        } else if (step == 0) {
           sl.pos = A.kv_len[row] + second;
           sl.tok = pend[1 + second];
           sl.active = second ? (pend[0] == 2) : 1;
@@ -540,7 +564,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       S.lmmax[tid] = 0u;
       if (tid < R) {
         const int b = tid / m;
-        S.lm_src[tid] = (step == 0 && A.pending[b * 3] == 2) ? R + tid : tid;
+        S.lm_src[tid] = (step == 0 && !A.prepass && A.pending[b * 3] == 2) ? R + tid : tid;
       }
     }
     __syncthreads();
@@ -588,7 +612,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
     }
 
 #pragma unroll 1
-    for (int phase = 0; phase < n_phase; ++phase) {
+    for (int phase = 0; phase < (step < 0 ? n_phase - 1 : n_phase); ++phase) {
       const int kind = (phase == n_phase - 1) ? KIND_LM : (phase & 3);
       const int layer = phase >> 2;
       const LayerW& lw = S.layers[kind == KIND_LM ? 0 : layer];
@@ -597,10 +621,10 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       const int area_elems = A.act_slots * apitch;           // one staging area: [act_slots][apitch]
       const int n_in = (kind == KIND_LM) ? R : ns;           // activation rows of the phase
       const bool norm_kind = kind == KIND_QKV || kind == KIND_GU || kind == KIND_LM;
-      const unsigned ka = (unsigned)step * per_step + S.pstart[phase], kb = (unsigned)step * per_step + S.pstart[phase + 1];
+      const unsigned ka = ubase + S.pstart[phase], kb = ubase + S.pstart[phase + 1];
 
       // epochs of the words this phase reads and writes
-      const unsigned ep_base = A.epoch0 + (unsigned)step * EPS;
+      const unsigned ep_base = A.epoch0 + (unsigned)it * EPS;
       const unsigned ep_prev_dn = ep_base + 5u * (unsigned)layer;                    // down projection of the layer before
       const unsigned ep_qkv = ep_base + 5u * (unsigned)layer + 1u, ep_att = ep_qkv + 1u, ep_o = ep_qkv + 2u, ep_gu = ep_qkv + 3u,
                      ep_dn = ep_qkv + 4u, ep_lm = ep_base + 5u * (unsigned)A.L + 1u;
@@ -740,7 +764,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         const unsigned k = k0 + (unsigned)wgrp;
         const bool has = k < kb;
         int sub = 0;
-        if (has) sub = unit_sub(S.ulist[k - (unsigned)step * per_step]);
+        if (has) sub = unit_sub(S.ulist[k - ubase]);
         if (kind == KIND_DN) {
           // stage this round's chunks of the gated product (left as bf16 by the gate/up epilogue): area of
           // group w <- columns of its sub-unit, 16 bytes at a time
@@ -749,7 +773,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           const int nvec = g.kchunk >> 2;                       // 16-byte pieces of a chunk
           const int w2 = warp / kGW, part = warp - w2 * kGW;
           const unsigned kq = k0 + (unsigned)w2;
-          const int sq = kq < kb ? unit_sub(S.ulist[kq - (unsigned)step * per_step]) : 0;
+          const int sq = kq < kb ? unit_sub(S.ulist[kq - ubase]) : 0;
           int jj = part * 32 + lane, s2 = 0;                    // this lane's next (piece, row)
 #pragma unroll 1
           while (__shfl_sync(0xffffffffu, jj, 0) < nvec) {      // (lane 0 has the most pieces: a warp-uniform trip count)
@@ -790,7 +814,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           const int q = tid >> 7, e = tid & 127, r = e & 15, n = e >> 4;
           const unsigned kq = k0 + (unsigned)q;
           if (kq < kb) {
-            const uint32_t eq = S.ulist[kq - (unsigned)step * per_step];
+            const uint32_t eq = S.ulist[kq - ubase];
             if ((q & (nsub_eff - 1)) == 0 && (unit_sub(eq) + nsub_eff == g.nsub) && n < n_in && S.slot[n].active) {
               base_p = (kind == KIND_O ? A.xa : A.x1) + (size_t)n * d + unit_tile(eq) * 16 + r;
               base_w = ll_load1(base_p);
@@ -829,7 +853,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
           const unsigned kq = k0 + (unsigned)q;
           int sq = 0, tile = 0;
           const bool on = kq < kb;
-          if (on) { const uint32_t eq = S.ulist[kq - (unsigned)step * per_step]; sq = unit_sub(eq); tile = unit_tile(eq); }
+          if (on) { const uint32_t eq = S.ulist[kq - ubase]; sq = unit_sub(eq); tile = unit_tile(eq); }
           const bool lead = on && (q & (nsub_eff - 1)) == 0 && (sq + nsub_eff == g.nsub);   // tile complete in this round (nsub_eff is 1, 2 or 4)
           const bool slot_on = n < n_in && (kind == KIND_LM || S.slot[n].active);
           const int o = tile * 16 + r;
@@ -870,7 +894,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
         // free), by the group's last warp, whose lanes serve the highest slot numbers and are mostly idle above
         if (has && wl == kGW - 1 && lane == 0) {
           const unsigned kn = k + (unsigned)A.n_ring;
-          if (kn < total_units) issue_unit(A, S, ring, kn, per_step);
+          if (kn < total_units) issue_unit(A, S, ring, kn, per_step, pre_units);
         }
         TSEC(3);
       }
@@ -1233,6 +1257,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       }
     }  // phases
 
+    if (step < 0) continue;                             // the extra pass ends with its last layer
     // ---- ensemble: exact softmax of the m rows, weighted average, draw (Algorithm 1 steps 6-7) -----
     // Three exchanges, each a table of flagged words that every CTA polls whole: every CTA's maxima of the rows
     // (published by the LM head), every CTA's integer exp sums, the mass of every chunk of q.
@@ -1240,7 +1265,7 @@ __global__ void __launch_bounds__(kPT, 1) k_draft_round(const RoundArgs A) {
       const float* lg = A.logits_override ? A.logits_override + (size_t)step * R * V : A.logits_own + (size_t)step * R * V;
       const bool vec = ((V & 3) == 0) && ((reinterpret_cast<uintptr_t>(lg) & 15) == 0);
       const int n_chunks = A.n_chunks;
-      const unsigned ep_base = A.epoch0 + (unsigned)step * EPS;
+      const unsigned ep_base = A.epoch0 + (unsigned)it * EPS;
       const unsigned ep_lm = ep_base + 5u * (unsigned)A.L + 1u, ep_max2 = ep_lm + 1u, ep_sum = ep_lm + 2u, ep_mix = ep_lm + 3u;
       const uint2* max_tab = A.rowmax;
       unsigned ep_max = ep_lm;

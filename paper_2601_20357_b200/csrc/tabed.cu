@@ -416,7 +416,11 @@ int setup_persistent(tabed_handle* h) {
   h->persist_ok = false;
   if (c.dtype != TABED_DTYPE_BF16 || h->D > 1) return TABED_OK;      // (the in-kernel draw proposes one candidate per step)
   const int grp = h->H / h->Hkv;
-  if (2 * h->R > kPSlots || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
+  // up to kPSlots / 2 rows both pending tokens of a fully accepted block share the first step's weight pass (2 R slots);
+  // with more rows (up to kPSlots) the first of them gets a pass of its own, which needs two layers for its cache
+  // writes to be ordered before the first step's reads
+  const bool prepass = 2 * h->R > kPSlots;
+  if (h->R > kPSlots || (prepass && h->L < 2) || h->B > kPSlots || h->d % 16 || h->d > kPMaxD || h->F % 16 || (h->Hkv * h->hd) % 16 ||
       grp > kMaxGroup || grp * h->hd > 512 || h->L > kPMaxL || h->H > kPMaxHeads || (h->cap + 127) / 128 > kAttnSplitMax)
     return TABED_OK;
   cudaDeviceProp prop;
@@ -443,11 +447,12 @@ int setup_persistent(tabed_handle* h) {
   if (per_step > kMaxUnits) return TABED_OK;
   {
     // the staging of a whole input row: its warps keep at most 8 pieces of 16 bytes per lane in flight
-    const int act_slots = std::min(kPSlots, 2 * h->R), warps_per_row = kPW / act_slots;
+    const int act_slots = prepass ? h->R : 2 * h->R, warps_per_row = kPW / act_slots;
     if ((h->d / 2 + warps_per_row * 32 - 1) / (warps_per_row * 32) > 8) return TABED_OK;
   }
   A.slot_bytes = 16 * (kmax * 2 + 16);
-  A.act_slots = std::min(kPSlots, 2 * h->R);
+  A.act_slots = prepass ? h->R : 2 * h->R;
+  A.prepass = prepass ? 1 : 0;
   const int dn_areas = std::min(A.geom[KIND_DN].nsub, kWG);
   const size_t act_raw = std::max((size_t)A.act_slots * (h->d + 8) * 2, (size_t)dn_areas * A.act_slots * (A.geom[KIND_DN].kchunk + 8) * 2);
   A.act_bytes = (int)((act_raw + 127) / 128 * 128);
@@ -544,8 +549,8 @@ int launch_persistent_round(tabed_handle* h, const float* u_draft, int32_t* out_
   A.u = u_draft; A.out_tokens = out_tokens; A.logits_override = h->logits_override;
   (void)max_pos;
   A.split_len = (h->hd <= 64) ? 256 : 128;          // positions per attention item: 4 register passes of the CTA
-  // epochs: this launch stamps epoch0 + 1 ... epoch0 + G (5 L + 8); when the counter nears its end the buffers are cleared
-  const unsigned span = (unsigned)h->G * (5u * (unsigned)h->L + 8u);
+  // epochs: this launch stamps epoch0 + 1 ... epoch0 + (G [+ 1]) (5 L + 8); when the counter nears its end the buffers are cleared
+  const unsigned span = (unsigned)(h->G + (A.prepass ? 1 : 0)) * (5u * (unsigned)h->L + 8u);
   if (h->ll_epoch > 0xFFFFFFFFu - 2u * span) {
     for (auto& b : h->ll_all) if (cudaMemsetAsync(b.first, 0, b.second, h->stream) != cudaSuccess) return TABED_ERR_CUDA;
     h->ll_epoch = 0;

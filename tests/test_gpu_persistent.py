@@ -81,6 +81,28 @@ def test_lockstep_mixed_pending_counts_across_requests():
     pair.gpu.destroy()
 
 
+def test_lockstep_six_rows_extra_pass_every_round():
+    """R = 6 rows (more than half of the kernel's 8 slots): both pending tokens of a fully accepted block no longer fit
+    into one weight pass, the first is fed in a pass of its own (all layers, no LM head) before step 0.  m = 1 with a
+    noise-free target makes q = p, so every block is fully accepted and every round after the first takes that pass."""
+    wl = wl_small(m=1, B=6, sigma=0.0, prefixes=((("tokens", 21),),), alpha=(1.0,), cid=81, policy=W.POLICY_STATIC)
+    pair = run_lockstep(wl, 4)
+    assert int(pair.orc.n_accept.min()) == wl.gamma
+    pair.gpu.destroy()
+
+
+@pytest.mark.parametrize("B,m", [(2, 3), (4, 2), (1, 5), (1, 8)])
+def test_lockstep_five_to_eight_rows_mixed_pending(B, m):
+    """5 - 8 rows on the persistent kernel; sigma small so that some requests' blocks are fully accepted and others'
+    not: in the extra pass only the rows with two pending tokens are active, the others wait for step 0."""
+    prefixes = ((("tokens", 140),), (("embeds", 12), ("tokens", 3)), (("tokens", 40),), (("tokens", 7),),
+                (("embeds", 20),), (("tokens", 64),), (("tokens", 3),), (("tokens", 90),))[:m]
+    alpha = tuple([0.9] + [0.1 / (m - 1)] * (m - 1))
+    wl = wl_small(m=m, B=B, sigma=0.05, prefixes=prefixes, alpha=alpha, cid=82 + B * 10 + m, gamma=3)
+    pair = run_lockstep(wl, 6)
+    pair.gpu.destroy()
+
+
 @pytest.mark.parametrize("heads,kv_heads,d", [(8, 2, 256), (2, 1, 256), (4, 4, 512)])
 def test_lockstep_head_sizes(heads, kv_heads, d):
     """head_dim 32 (8 heads, 4 per KV head), 128 (2 heads sharing one KV head), 128 without grouping."""
