@@ -95,8 +95,10 @@ struct ReqShared {
 
 // Row maxima of `rows` rows (row i at base + i * pitch) over this CTA's slice, gathered over the cluster:
 // afterwards S.all_max[r][i] holds CTA r's maximum of row i in every CTA.  Four rows' loads are in flight together.
+// ebuf (optional, shared memory, row pitch epitch floats): the CTA's slice of every row is kept there, so that the later
+// passes of the exact softmax neither go back to global memory nor take an exponential twice.
 __device__ __forceinline__ void req_row_maxima(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, const float* __restrict__ base,
-                                               long long pitch, int rows, bool vec) {
+                                               long long pitch, int rows, bool vec, float* ebuf = nullptr, int epitch = 0) {
 #pragma unroll 1
   for (int i0 = 0; i0 < rows; i0 += 4) {
     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -108,7 +110,10 @@ __device__ __forceinline__ void req_row_maxima(cg::cluster_group& cluster, const
         if (i0 + j < rows) req_ld4(base + (long long)(i0 + j) * pitch, v, c.v_hi, vec, -INFINITY, x[j]);
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        if (i0 + j < rows) mx[j] = fmaxf(fmaxf(mx[j], fmaxf(x[j][0], x[j][1])), fmaxf(x[j][2], x[j][3]));
+        if (i0 + j < rows) {
+          mx[j] = fmaxf(fmaxf(mx[j], fmaxf(x[j][0], x[j][1])), fmaxf(x[j][2], x[j][3]));
+          if (ebuf) *reinterpret_cast<float4*>(ebuf + (size_t)(i0 + j) * epitch + (v - c.v_lo)) = make_float4(x[j][0], x[j][1], x[j][2], x[j][3]);
+        }
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -132,8 +137,9 @@ __device__ __forceinline__ float req_max_of(const ReqCtx& c, const ReqShared& S,
 }
 
 // Integer sums of the exp masses of the rows (softmax normalisers), gathered over the cluster.
+// With ebuf: reads the logits left there by req_row_maxima and leaves the exponentials in their place.
 __device__ __forceinline__ void req_row_sums(cg::cluster_group& cluster, const ReqCtx& c, ReqShared& S, const float* __restrict__ base,
-                                             long long pitch, int rows, bool vec) {
+                                             long long pitch, int rows, bool vec, float* ebuf = nullptr, int epitch = 0) {
 #pragma unroll 1
   for (int i0 = 0; i0 < rows; i0 += 2) {
     unsigned long long sm[2] = {0ull, 0ull};
@@ -145,12 +151,23 @@ __device__ __forceinline__ void req_row_sums(cg::cluster_group& cluster, const R
       float x[2][4];
 #pragma unroll
       for (int j = 0; j < 2; ++j)
-        if (i0 + j < rows) req_ld4(base + (long long)(i0 + j) * pitch, v, c.v_hi, vec, -INFINITY, x[j]);
+        if (i0 + j < rows) {
+          if (ebuf) {
+            const float4 t = *reinterpret_cast<const float4*>(ebuf + (size_t)(i0 + j) * epitch + (v - c.v_lo));
+            x[j][0] = t.x; x[j][1] = t.y; x[j][2] = t.z; x[j][3] = t.w;
+          } else {
+            req_ld4(base + (long long)(i0 + j) * pitch, v, c.v_hi, vec, -INFINITY, x[j]);
+          }
+        }
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         if (i0 + j >= rows) continue;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) if (v + e < c.v_hi) sm[j] += mass_of(xexp(__fsub_rn(x[j][e], mx[j])));
+        for (int e = 0; e < 4; ++e) {
+          x[j][e] = (v + e < c.v_hi) ? xexp(__fsub_rn(x[j][e], mx[j])) : 0.0f;
+          if (v + e < c.v_hi) sm[j] += mass_of(x[j][e]);
+        }
+        if (ebuf) *reinterpret_cast<float4*>(ebuf + (size_t)(i0 + j) * epitch + (v - c.v_lo)) = make_float4(x[j][0], x[j][1], x[j][2], x[j][3]);
       }
     }
 #pragma unroll
@@ -311,7 +328,10 @@ struct EnsembleArgs {
   int* out0; int out0_stride;                   // y[b * out0_stride]
   int* out1; int out1_stride;                   // optional second copy
   int* err;
+  int ebuf_pitch;                               // > 0: the launch has m * ebuf_pitch floats of dynamic shared memory for the slices
 };
+
+extern __shared__ float4 req_dyn_smem[];
 
 __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleArgs A) {
   pdl_trigger();
@@ -319,11 +339,13 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
   __shared__ ReqShared S;
   const ReqCtx c = req_ctx(cluster, A.V, A.slice);
   const int b = blockIdx.x / c.CS, m = A.m, V = A.V;
+  float* ebuf = A.ebuf_pitch > 0 ? reinterpret_cast<float*>(req_dyn_smem) : nullptr;
+  const int epitch = A.ebuf_pitch;
   pdl_wait();
   const float* lg = A.logits + (long long)b * m * V;
   const bool vec = req_vec_ok(A.logits, V);
-  req_row_maxima(cluster, c, S, lg, V, m, vec);
-  req_row_sums(cluster, c, S, lg, V, m, vec);
+  req_row_maxima(cluster, c, S, lg, V, m, vec, ebuf, epitch);
+  req_row_sums(cluster, c, S, lg, V, m, vec, ebuf, epitch);
   // (the loop over the inputs below is a real loop - the kernel's code runs once per CTA, so its size is what
   // the instruction fetch pays for - hence the rows' scalars sit in shared memory, not in registers)
   if (c.tid < m) {
@@ -341,18 +363,23 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_ensemble_req(const EnsembleA
 #pragma unroll 1
   for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
     float acc[4];
-    float nxt[4];
-    req_ld4(lg, v, c.v_hi, vec, -INFINITY, nxt);
+    float nxt[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (!ebuf) req_ld4(lg, v, c.v_hi, vec, -INFINITY, nxt);
 #pragma unroll 1
     for (int k = 0; k < m; ++k) {
       float a[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) a[j] = nxt[j];
-      if (k + 1 < m) req_ld4(lg + (long long)(k + 1) * V, v, c.v_hi, vec, -INFINITY, nxt);
       const float mxk = S.par[0][k], snk = S.par[1][k], wkk = S.par[2][k];
+      if (ebuf) {
+        const float4 t = *reinterpret_cast<const float4*>(ebuf + (size_t)k * epitch + (v - c.v_lo));     // the exponentials
+        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) a[j] = xexp(__fsub_rn(nxt[j], mxk));
+        if (k + 1 < m) req_ld4(lg + (long long)(k + 1) * V, v, c.v_hi, vec, -INFINITY, nxt);
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mxk)), snk);
+        a[j] = __fdiv_rn(a[j], snk);
         const float t = __fmul_rn(wkk, a[j]);
         acc[j] = (k == 0) ? t : __fadd_rn(acc[j], t);
       }
@@ -499,6 +526,7 @@ struct VerifyArgs {
   int* ticket;                                  // [B] scratch, zero between launches
   int *n_accept, *out_n_accept, *next_token, *out_next_token;
   int* err;
+  int ebuf_pitch;                               // > 0: the launch has ebuf_pitch floats of dynamic shared memory for the row's slice
   int tail_inline;                              // 1: the request's last cluster runs the tail; 0: k_verify_tail does (a launch of
                                                 // its own with one LARGE cluster per request - with many requests the clusters
                                                 // of this kernel are small and the tail would crawl through a row on 1-2 CTAs)
@@ -519,8 +547,9 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
   float* p_b = A.p + (long long)b * Rt * V;
   const float* q_b = A.q + (long long)b * A.q_req_stride;
   const bool vec = req_vec_ok(A.logits, V), vec_p = (V & 3) == 0;
-  req_row_maxima(cluster, c, S, lg, V, 1, vec);
-  req_row_sums(cluster, c, S, lg, V, 1, vec);
+  float* ebuf = A.ebuf_pitch > 0 ? reinterpret_cast<float*>(req_dyn_smem) : nullptr;
+  req_row_maxima(cluster, c, S, lg, V, 1, vec, ebuf, A.ebuf_pitch);
+  req_row_sums(cluster, c, S, lg, V, 1, vec, ebuf, A.ebuf_pitch);
   const float mx = req_max_of(c, S, 0), sn = req_norm_of(c, S, 0);
   {
     // p_i = e / S; in greedy mode also its argmax
@@ -528,10 +557,17 @@ __global__ void __launch_bounds__(kReqThreads, 2) k_verify_req(const VerifyArgs 
 #pragma unroll 1
     for (int v = c.v_lo + c.tid * 4; v < c.v_hi; v += kReqStep) {
       float a[4];
-      req_ld4(lg, v, c.v_hi, vec, -INFINITY, a);
+      if (ebuf) {
+        const float4 t = *reinterpret_cast<const float4*>(ebuf + (v - c.v_lo));                       // the exponentials
+        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
+      } else {
+        req_ld4(lg, v, c.v_hi, vec, -INFINITY, a);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) a[j] = xexp(__fsub_rn(a[j], mx));
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        a[j] = __fdiv_rn(xexp(__fsub_rn(a[j], mx)), sn);
+        a[j] = __fdiv_rn(a[j], sn);
         if (A.greedy && v + j < c.v_hi && a[j] > best.val) { best.val = a[j]; best.idx = v + j; }
       }
       req_st4(p_b + (long long)i * V, v, c.v_hi, vec_p, a);

@@ -70,6 +70,7 @@ struct tabed_handle {
   int* err = nullptr;
   int cs_max = 8;                   // largest cluster the per-request kernels may use on this device (8 portable, 16 opt-in)
   int cs_active[5] = {0, 0, 0, 0, 0};   // clusters of 1, 2, 4, 8, 16 CTAs that the device keeps resident at once
+  bool req_dyn_ok = false;          // the cluster kernels may take up to kReqDynSmemMax of dynamic shared memory
   int cta_budget = 3;               // CTAs per SM a launch of the per-request kernels may have in total (3, 6, 12 measured: 3 best)
   // staging for the host-buffer entry point
   float *st_u_draft = nullptr, *st_u_accept = nullptr, *st_u_resid = nullptr, *st_target = nullptr;
@@ -163,10 +164,12 @@ void launch_pdl(tabed_handle* h, void (*kern)(KArgs...), dim3 grid, dim3 block, 
 #define TABED_LAUNCH_PDL(h, kern, grid, block, smem, ...) launch_pdl((h), (kern), dim3(grid), dim3(block), (smem), __VA_ARGS__)
 
 // `n_clusters` clusters of `cs` CTAs, as a programmatic dependent of the kernel before it in the stream.
+constexpr size_t kReqDynSmemMax = 64u * 1024u;      // slices kept in shared memory by the softmax passes (two CTAs per SM still fit)
+
 template <typename ArgT>
-void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_clusters, int cs, const ArgT& args) {
+void launch_request_clusters(tabed_handle* h, void (*kern)(ArgT), int n_clusters, int cs, const ArgT& args, size_t dyn_smem = 0) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(n_clusters * cs)); cfg.blockDim = dim3(kReqThreads); cfg.dynamicSmemBytes = 0; cfg.stream = h->stream;
+  cfg.gridDim = dim3((unsigned)(n_clusters * cs)); cfg.blockDim = dim3(kReqThreads); cfg.dynamicSmemBytes = dyn_smem; cfg.stream = h->stream;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -395,7 +398,10 @@ void run_ensemble(tabed_handle* h, const float* logits, const float* w, const fl
   a.qk_out = qk_out; a.qk_req_stride = qk_stride; a.q_out = q_out; a.q_req_stride = q_stride;
   a.out0 = y0; a.out0_stride = y0_stride; a.out1 = y1; a.out1_stride = y1_stride; a.err = h->err;
   a.D = n_cand; a.cand = cand; a.cand_stride = cand_stride;
-  launch_request_clusters(h, k_ensemble_req, h->B, cs, a);
+  // the CTA's slices of the m rows stay in shared memory between the softmax passes when they fit
+  size_t dyn = (size_t)h->m * a.slice * sizeof(float);
+  if (dyn <= kReqDynSmemMax && h->req_dyn_ok) a.ebuf_pitch = a.slice; else dyn = 0;
+  launch_request_clusters(h, k_ensemble_req, h->B, cs, a, dyn);
 }
 
 // ---- persistent drafting-round kernel: geometry and set-up -----------------------------------------
@@ -831,6 +837,8 @@ int tabed_init(const tabed_config* cfg, const tabed_weights* wts, tabed_handle**
     if (cudaGetDeviceProperties(&pr, c.device) == cudaSuccess) h->n_sm = pr.multiProcessorCount;
     // the per-request cluster kernels: clusters of 16 CTAs where the device can place one (non-portable size)
     h->cs_max = 8;
+    h->req_dyn_ok = cudaFuncSetAttribute(k_ensemble_req, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kReqDynSmemMax) == cudaSuccess &&
+                    cudaFuncSetAttribute(k_verify_req, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kReqDynSmemMax) == cudaSuccess;
     if (cudaFuncSetAttribute(k_ensemble_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
         cudaFuncSetAttribute(k_verify_req, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
         cudaFuncSetAttribute(k_verify_tail, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
@@ -1170,9 +1178,11 @@ int tabed_verify(tabed_handle* h, const float* target_logits, const float* u_acc
   int slice_tail = 0;
   const int cs_tail = pick_cluster(h, h->B, &slice_tail);
   a.tail_inline = cs_tail >= 4 * cs ? 0 : 1;
-  launch_request_clusters(h, k_verify_req, h->B * (h->G + 1), cs, a);
+  size_t dyn = (size_t)a.slice * sizeof(float);
+  if (dyn <= kReqDynSmemMax && h->req_dyn_ok) a.ebuf_pitch = a.slice; else dyn = 0;
+  launch_request_clusters(h, k_verify_req, h->B * (h->G + 1), cs, a, dyn);
   if (!a.tail_inline) {
-    a.slice = slice_tail;
+    a.slice = slice_tail; a.ebuf_pitch = 0;
     launch_request_clusters(h, k_verify_tail, h->B, cs_tail, a);
   }
   h->phase = PH_VERIFIED;
