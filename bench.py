@@ -37,6 +37,8 @@ PAPER_CONTEXT = ("paper (A100 80GB, fp16): expected walltime speedup 1.74x over 
 # captures summarised under profiles/ ; keyed by (workload, kernel class).  Entries are removed when the kernel changes.
 NCU_TRAFFIC = {("llava_small", "draft_round"): {"bytes": 690.13e6, "algorithmic_bytes_of_that_launch": 698.0e6,
                                                 "source": "profiles/k_draft_round_llava_small_ncu_full.md"},
+               ("large_vocab", "draft_round"): {"bytes": 3303.0e6, "algorithmic_bytes_of_that_launch": 3290.5e6,
+                                                "source": "profiles/k_draft_round_llava_small_ncu_full.md (third part)"},
                ("long_context", "draft_round"): {"bytes": 3016.1e6, "algorithmic_bytes_of_that_launch": 3006.5e6,
                                                  "source": "profiles/k_draft_round_llava_small_ncu_full.md (second part)"},
                # captured on 16 of the 32 requests (capture-size rule) and scaled by the rows: 366.3 MB x 2
