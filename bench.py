@@ -601,7 +601,9 @@ def run_ours(args, wl):
     line = {
         "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32 accumulate over bf16 weights/KV" if wl.drafter.dtype == "bf16" else "f32",
+        "dtype": "bf16" if wl.drafter.dtype == "bf16" else "f32",
+        "dtype_note": ("bf16 weights, KV caches and matmul inputs with fp32 accumulation; decisions (softmax, mix, draw, accept, "
+                       "deviations) in exactly rounded fp32 and integer arithmetic"),
         "data": "synthetic",
         "config": config_of(wl),
         "details": {"l2": "256 MB written between rounds (stands for the target model's pass); rounds timed one by one "
